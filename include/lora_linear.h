@@ -1,0 +1,142 @@
+/*
+ * lora_linear.h - C ABI of the B200 (sm_100a) LoRA projection layer, forward and backward.
+ *
+ * The layer is the low-rank-adapter form of a decoder projection with a frozen weight
+ * (Section 3.2.2, LoRA fine-tuning; adapter rank r and alpha as in Section 4.5, scale = alpha / r):
+ *
+ *     forward    Y  = X W^T + scale (X A^T) B^T
+ *     backward   dX = dY W + scale (dY B) A
+ *                dB = scale dY^T (X A^T)
+ *                dA = scale (dY B)^T X
+ *
+ * Layouts: every tensor is dense row-major, last index contiguous.
+ *     X [T, d_in]  W [d_out, d_in]  A [r, d_in]  B [d_out, r]  Y, dY [T, d_out]  dX [T, d_in]   bf16
+ *     dA [r, d_in]  dB [d_out, r]                                                                   fp32
+ * T is the number of packed trajectory tokens of the batch; packing boundaries do not reach a
+ * projection layer, so no sequence offsets are passed.
+ *
+ * Conventions
+ *   - Every function returns an int: LORA_OK (0) or a negative lora_status_t.  Nothing throws,
+ *     nothing calls exit().
+ *   - Tensor pointers are DEVICE pointers owned by the caller (unless a parameter is named h_*),
+ *     16-byte aligned.  Inputs are read-only; outputs are overwritten, never accumulated into.
+ *     No output may alias an input or another output.
+ *   - d_in and d_out must be multiples of 8; r a multiple of 8 with 8 <= r <= 64; T >= 0.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work and return; they do not
+ *     synchronise.  A plan must not be used from two host threads, or on two streams, at once.
+ *   - The library never allocates device memory except one 256-byte status word block per plan;
+ *     backward scratch is caller-provided (lora_plan_set_workspace).
+ *   - There is no CPU fallback: without a CUDA device of compute capability 10.x the calls fail
+ *     with LORA_ERR_NO_DEVICE.
+ */
+#ifndef LORA_LINEAR_H_
+#define LORA_LINEAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum lora_status {
+  LORA_OK = 0,
+  LORA_ERR_INVALID_ARG = -1,       /* null pointer, negative size, bad buffer length            */
+  LORA_ERR_UNSUPPORTED_SHAPE = -2, /* d_in/d_out not multiples of 8, r outside {8,16,...,64}     */
+  LORA_ERR_MISALIGNED = -3,        /* a tensor pointer is not 16-byte aligned                    */
+  LORA_ERR_WORKSPACE = -4,         /* backward called without (enough) workspace                 */
+  LORA_ERR_CUDA = -5,              /* a CUDA runtime / driver call failed (launch, descriptor)   */
+  LORA_ERR_DEVICE_TIMEOUT = -6,    /* a bounded device-side wait ran out (lora_last_device_status)*/
+  LORA_ERR_NO_DEVICE = -7          /* no usable sm_100 device                                    */
+} lora_status_t;
+
+typedef struct lora_plan lora_plan_t; /* opaque, host memory owned by the library */
+
+typedef struct lora_shape {
+  int64_t T;     /* tokens (rows of X, Y, dY, dX) */
+  int64_t d_in;  /* input features                */
+  int64_t d_out; /* output features               */
+  int64_t r;     /* adapter rank                  */
+} lora_shape_t;
+
+/* What the per-shape selector chose (Section 3.2.2 "dynamic profiling" analogue at kernel level). */
+typedef struct lora_kernel_config {
+  int32_t block_m;         /* token rows per GEMM tile (128)                                   */
+  int32_t fwd_block_n;     /* output columns per tile of the forward GEMM (64, 128 or 192)     */
+  int32_t dx_block_n;      /* output columns per tile of the dX GEMM                           */
+  int32_t block_k;         /* contraction elements per pipeline stage (64)                     */
+  int32_t stages;          /* depth of the TMA -> MMA shared-memory ring                       */
+  int32_t group_m;         /* tile rasterisation: m-tiles per band (L2 reuse)                  */
+  int32_t split_k;         /* split-K factor of the dense GEMMs (1 = none)                     */
+  int32_t r_pad;           /* rank padded to the MMA granularity (multiple of 16)              */
+  int32_t fwd_ctas;        /* persistent CTAs of the forward GEMM                              */
+  int32_t dx_ctas;         /* persistent CTAs of the dX GEMM                                   */
+  int32_t tail_delay;      /* k-blocks of the next tile issued before a tile's rank-r MMA      */
+  int32_t grad_feat_chunk; /* features per CTA of the adapter-gradient kernels                 */
+  int32_t grad_stages;     /* ring depth of the adapter-gradient kernels                       */
+  int32_t da_feat_chunks;  /* dA kernel grid: feature chunks x token chunks                    */
+  int32_t da_token_chunks;
+  int32_t db_feat_chunks;  /* dB kernel grid                                                   */
+  int32_t db_token_chunks;
+  int32_t reserved[3];
+} lora_kernel_config_t;
+
+/* Host-only: run the tile / split selector for a shape on a device with `num_sms` SMs.
+ * Needs no GPU.  Returns LORA_ERR_UNSUPPORTED_SHAPE for shapes the kernels do not cover. */
+int lora_select_config(const lora_shape_t* shape, int num_sms, lora_kernel_config_t* out);
+
+/* Host-only: bytes of backward scratch lora_linear_bwd needs for a shape (forward needs none). */
+int lora_workspace_bytes(const lora_shape_t* shape, int num_sms, size_t* bwd_bytes);
+
+/* Create / destroy a plan for one shape on CUDA device `device` (runs the selector, allocates the
+ * 256-byte device status block).  The plan is host memory owned by the library. */
+int lora_plan_create(const lora_shape_t* shape, int device, lora_plan_t** out);
+int lora_plan_destroy(lora_plan_t* plan);
+
+/* Scratch sizes of a plan; either pointer may be NULL.  fwd_bytes is always 0. */
+int lora_plan_workspace_bytes(const lora_plan_t* plan, size_t* fwd_bytes, size_t* bwd_bytes);
+
+/* Register caller-owned device scratch (256-byte aligned, at least bwd_bytes).  The memory stays
+ * owned by the caller and must outlive every backward call that uses the plan. */
+int lora_plan_set_workspace(lora_plan_t* plan, void* dev_ptr, size_t bytes);
+
+/* Copy the selector's choice / a one-line description into caller memory. */
+int lora_plan_get_config(const lora_plan_t* plan, lora_kernel_config_t* out);
+int lora_plan_describe(const lora_plan_t* plan, char* buf, size_t n);
+
+/* Forward:  Y = X W^T + scale (X A^T) B^T.
+ * One fused kernel: TMA-staged bf16 tiles, tcgen05 MMA into TMEM; X A^T rides the main loop as
+ * extra accumulator columns and the rank-r product is one more MMA group before the epilogue. */
+int lora_linear_fwd(lora_plan_t* plan, const void* X, const void* W, const void* A, const void* B,
+                    float scale, void* Y, void* stream);
+
+/* Backward:  dX = dY W + scale (dY B) A,  dA = scale (dY B)^T X,  dB = scale dY^T (X A^T).
+ * Does not depend on a preceding forward call (X A^T is recomputed).  Needs the workspace.
+ * dA and dB are fp32 and are overwritten. */
+int lora_linear_bwd(lora_plan_t* plan, const void* dY, const void* X, const void* W, const void* A,
+                    const void* B, float scale, void* dX, void* dA, void* dB, void* stream);
+
+/* One training step of the layer with HOST input/output buffers: copies h_X, h_A, h_B, h_dY to the
+ * device staging area, runs forward and backward, copies Y, dX, dA, dB back, all on `stream`
+ * (asynchronous when the host buffers are pinned).  W is the frozen weight and stays resident on
+ * the device.  `staging` is caller-owned device memory of at least lora_step_host_staging_bytes. */
+int lora_step_host_staging_bytes(const lora_shape_t* shape, size_t* bytes);
+int lora_linear_step_host(lora_plan_t* plan, const void* h_X, const void* W, const void* h_A,
+                          const void* h_B, const void* h_dY, float scale, void* h_Y, void* h_dX,
+                          void* h_dA, void* h_dB, void* staging, size_t staging_bytes, void* stream);
+
+/* Synchronise `stream`, then report whether any kernel of this plan gave up on a bounded wait.
+ * *code is LORA_OK or LORA_ERR_DEVICE_TIMEOUT; msg (may be NULL) receives a short description.
+ * The status word is cleared. */
+int lora_last_device_status(lora_plan_t* plan, void* stream, int* code, char* msg, size_t n);
+
+/* Static string for a status code. */
+const char* lora_strerror(int code);
+
+/* Number of kernels the library has launched in this process (all plans). */
+int64_t lora_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LORA_LINEAR_H_ */

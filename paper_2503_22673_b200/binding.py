@@ -1,0 +1,255 @@
+"""ctypes binding of liblora_linear.so: argument marshalling only.
+
+Every step of the layer runs in the CUDA kernels behind the C ABI (include/lora_linear.h); torch is
+used for device memory and streams.  There is no fallback: if the library cannot be built or loaded,
+or no sm_100 device is present, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+from . import build as _build
+
+LORA_OK = 0
+LORA_ERR_INVALID_ARG = -1
+LORA_ERR_UNSUPPORTED_SHAPE = -2
+LORA_ERR_MISALIGNED = -3
+LORA_ERR_WORKSPACE = -4
+LORA_ERR_CUDA = -5
+LORA_ERR_DEVICE_TIMEOUT = -6
+LORA_ERR_NO_DEVICE = -7
+
+EXPORTS = [
+    "lora_select_config", "lora_workspace_bytes", "lora_plan_create", "lora_plan_destroy",
+    "lora_plan_workspace_bytes", "lora_plan_set_workspace", "lora_plan_get_config", "lora_plan_describe",
+    "lora_linear_fwd", "lora_linear_bwd", "lora_step_host_staging_bytes", "lora_linear_step_host",
+    "lora_last_device_status", "lora_strerror", "lora_launch_count",
+]
+
+
+class LoraShape(ctypes.Structure):
+    _fields_ = [("T", ctypes.c_int64), ("d_in", ctypes.c_int64), ("d_out", ctypes.c_int64), ("r", ctypes.c_int64)]
+
+
+class LoraKernelConfig(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "block_m", "fwd_block_n", "dx_block_n", "block_k", "stages", "group_m", "split_k", "r_pad", "fwd_ctas",
+        "dx_ctas", "tail_delay", "grad_feat_chunk", "grad_stages", "da_feat_chunks", "da_token_chunks",
+        "db_feat_chunks", "db_token_chunks")] + [("reserved", ctypes.c_int32 * 3)]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_ if n != "reserved"}
+
+
+class LoraError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+_lib = None
+
+
+def load(rebuild: bool = False) -> ctypes.CDLL:
+    """Load (building first if sources are newer) the CUDA library.  Raises if that is impossible."""
+    global _lib
+    if _lib is not None and not rebuild:
+        return _lib
+    path = _build.build(force=rebuild)
+    lib = ctypes.CDLL(path)
+    vp, i64 = ctypes.c_void_p, ctypes.c_int64
+    sz_p = ctypes.POINTER(ctypes.c_size_t)
+    lib.lora_select_config.argtypes = [ctypes.POINTER(LoraShape), ctypes.c_int, ctypes.POINTER(LoraKernelConfig)]
+    lib.lora_workspace_bytes.argtypes = [ctypes.POINTER(LoraShape), ctypes.c_int, sz_p]
+    lib.lora_plan_create.argtypes = [ctypes.POINTER(LoraShape), ctypes.c_int, ctypes.POINTER(vp)]
+    lib.lora_plan_destroy.argtypes = [vp]
+    lib.lora_plan_workspace_bytes.argtypes = [vp, sz_p, sz_p]
+    lib.lora_plan_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
+    lib.lora_plan_get_config.argtypes = [vp, ctypes.POINTER(LoraKernelConfig)]
+    lib.lora_plan_describe.argtypes = [vp, ctypes.c_char_p, ctypes.c_size_t]
+    lib.lora_linear_fwd.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp]
+    lib.lora_linear_bwd.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
+    lib.lora_step_host_staging_bytes.argtypes = [ctypes.POINTER(LoraShape), sz_p]
+    lib.lora_linear_step_host.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp,
+                                          ctypes.c_size_t, vp]
+    lib.lora_last_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int), ctypes.c_char_p, ctypes.c_size_t]
+    lib.lora_strerror.argtypes = [ctypes.c_int]
+    lib.lora_strerror.restype = ctypes.c_char_p
+    lib.lora_launch_count.argtypes = []
+    lib.lora_launch_count.restype = i64
+    for name in EXPORTS:
+        if name not in ("lora_strerror", "lora_launch_count"):
+            getattr(lib, name).restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load().lora_strerror(int(code)).decode()
+
+
+def launch_count() -> int:
+    return int(load().lora_launch_count())
+
+
+def _check(code: int, where: str) -> None:
+    if code != LORA_OK:
+        raise LoraError(code, where)
+
+
+def select_config(T: int, d_in: int, d_out: int, r: int, num_sms: int = 148) -> dict:
+    """Run the host-side tile selector (needs no GPU)."""
+    cfg = LoraKernelConfig()
+    shape = LoraShape(T, d_in, d_out, r)
+    _check(load().lora_select_config(ctypes.byref(shape), num_sms, ctypes.byref(cfg)), "lora_select_config")
+    return cfg.as_dict()
+
+
+def workspace_bytes(T: int, d_in: int, d_out: int, r: int, num_sms: int = 148) -> int:
+    out = ctypes.c_size_t(0)
+    shape = LoraShape(T, d_in, d_out, r)
+    _check(load().lora_workspace_bytes(ctypes.byref(shape), num_sms, ctypes.byref(out)), "lora_workspace_bytes")
+    return int(out.value)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> ctypes.c_void_p:
+    return ctypes.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> ctypes.c_void_p:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _want(t: torch.Tensor, name: str, shape: Tuple[int, ...], dtype: torch.dtype, device: torch.device) -> None:
+    if tuple(t.shape) != tuple(shape) or t.dtype != dtype or not t.is_contiguous() or t.device != device:
+        raise ValueError(f"{name}: want contiguous {dtype} {tuple(shape)} on {device}, got {t.dtype} "
+                         f"{tuple(t.shape)} contiguous={t.is_contiguous()} on {t.device}")
+
+
+class LoraLinearPlan:
+    """A plan for one (T, d_in, d_out, r) shape on one device; owns its backward workspace tensor."""
+
+    def __init__(self, T: int, d_in: int, d_out: int, r: int, device: int = 0):
+        if not torch.cuda.is_available():
+            raise LoraError(LORA_ERR_NO_DEVICE, "LoraLinearPlan")
+        self._lib = load()
+        self.T, self.d_in, self.d_out, self.r = int(T), int(d_in), int(d_out), int(r)
+        self.device = torch.device("cuda", device)
+        self._shape = LoraShape(self.T, self.d_in, self.d_out, self.r)
+        self._h = ctypes.c_void_p(0)
+        _check(self._lib.lora_plan_create(ctypes.byref(self._shape), device, ctypes.byref(self._h)), "lora_plan_create")
+        bwd = ctypes.c_size_t(0)
+        _check(self._lib.lora_plan_workspace_bytes(self._h, None, ctypes.byref(bwd)), "lora_plan_workspace_bytes")
+        self.workspace_bytes = int(bwd.value)
+        self._ws = None
+
+    # -- lifetime ------------------------------------------------------------------------------
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h.value:
+            self._lib.lora_plan_destroy(self._h)
+            self._h = ctypes.c_void_p(0)
+            self._ws = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- introspection -------------------------------------------------------------------------
+    def config(self) -> dict:
+        cfg = LoraKernelConfig()
+        _check(self._lib.lora_plan_get_config(self._h, ctypes.byref(cfg)), "lora_plan_get_config")
+        return cfg.as_dict()
+
+    def describe(self) -> str:
+        buf = ctypes.create_string_buffer(1024)
+        _check(self._lib.lora_plan_describe(self._h, buf, 1024), "lora_plan_describe")
+        return buf.value.decode()
+
+    def device_status(self, stream: Optional[torch.cuda.Stream] = None) -> Tuple[int, str]:
+        code = ctypes.c_int(0)
+        buf = ctypes.create_string_buffer(256)
+        _check(self._lib.lora_last_device_status(self._h, _stream_ptr(stream), ctypes.byref(code), buf, 256),
+               "lora_last_device_status")
+        return int(code.value), buf.value.decode()
+
+    # -- workspace -----------------------------------------------------------------------------
+    def ensure_workspace(self) -> None:
+        if self._ws is None:
+            self._ws = torch.empty(max(self.workspace_bytes, 256), dtype=torch.uint8, device=self.device)
+            _check(self._lib.lora_plan_set_workspace(self._h, _ptr(self._ws), self._ws.numel()),
+                   "lora_plan_set_workspace")
+
+    def set_workspace(self, ws: Optional[torch.Tensor]) -> None:
+        self._ws = ws
+        n = 0 if ws is None else ws.numel() * ws.element_size()
+        _check(self._lib.lora_plan_set_workspace(self._h, _ptr(ws), n), "lora_plan_set_workspace")
+
+    # -- the two calls -------------------------------------------------------------------------
+    def fwd(self, X, W, A, B, scale: float, Y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """Y = X W^T + scale (X A^T) B^T."""
+        bf = torch.bfloat16
+        _want(X, "X", (self.T, self.d_in), bf, self.device)
+        _want(W, "W", (self.d_out, self.d_in), bf, self.device)
+        _want(A, "A", (self.r, self.d_in), bf, self.device)
+        _want(B, "B", (self.d_out, self.r), bf, self.device)
+        if Y is None:
+            Y = torch.empty((self.T, self.d_out), dtype=bf, device=self.device)
+        _want(Y, "Y", (self.T, self.d_out), bf, self.device)
+        _check(self._lib.lora_linear_fwd(self._h, _ptr(X), _ptr(W), _ptr(A), _ptr(B), float(scale), _ptr(Y),
+                                         _stream_ptr(stream)), "lora_linear_fwd")
+        return Y
+
+    def bwd(self, dY, X, W, A, B, scale: float, dX=None, dA=None, dB=None, stream=None):
+        """(dX, dA, dB) = (dY W + scale (dY B) A,  scale (dY B)^T X,  scale dY^T (X A^T))."""
+        bf = torch.bfloat16
+        _want(dY, "dY", (self.T, self.d_out), bf, self.device)
+        _want(X, "X", (self.T, self.d_in), bf, self.device)
+        _want(W, "W", (self.d_out, self.d_in), bf, self.device)
+        _want(A, "A", (self.r, self.d_in), bf, self.device)
+        _want(B, "B", (self.d_out, self.r), bf, self.device)
+        if dX is None:
+            dX = torch.empty((self.T, self.d_in), dtype=bf, device=self.device)
+        if dA is None:
+            dA = torch.empty((self.r, self.d_in), dtype=torch.float32, device=self.device)
+        if dB is None:
+            dB = torch.empty((self.d_out, self.r), dtype=torch.float32, device=self.device)
+        _want(dX, "dX", (self.T, self.d_in), bf, self.device)
+        _want(dA, "dA", (self.r, self.d_in), torch.float32, self.device)
+        _want(dB, "dB", (self.d_out, self.r), torch.float32, self.device)
+        self.ensure_workspace()
+        _check(self._lib.lora_linear_bwd(self._h, _ptr(dY), _ptr(X), _ptr(W), _ptr(A), _ptr(B), float(scale),
+                                         _ptr(dX), _ptr(dA), _ptr(dB), _stream_ptr(stream)), "lora_linear_bwd")
+        return dX, dA, dB
+
+    # -- host-buffer step (end-to-end measurement and host callers) ------------------------------
+    def step_host_staging_bytes(self) -> int:
+        out = ctypes.c_size_t(0)
+        _check(self._lib.lora_step_host_staging_bytes(ctypes.byref(self._shape), ctypes.byref(out)),
+               "lora_step_host_staging_bytes")
+        return int(out.value)
+
+    def step_host(self, hX, W, hA, hB, hdY, scale: float, hY, hdX, hdA, hdB, staging: torch.Tensor, stream=None):
+        """fwd + bwd with host tensors for everything except the frozen W (device)."""
+        self.ensure_workspace()
+        for t in (hX, hA, hB, hdY, hY, hdX, hdA, hdB):
+            if t.device.type != "cpu" or not t.is_contiguous():
+                raise ValueError("step_host wants contiguous CPU tensors")
+        _check(self._lib.lora_linear_step_host(
+            self._h, _ptr(hX), _ptr(W), _ptr(hA), _ptr(hB), _ptr(hdY), float(scale), _ptr(hY), _ptr(hdX), _ptr(hdA),
+            _ptr(hdB), _ptr(staging), staging.numel() * staging.element_size(), _stream_ptr(stream)),
+            "lora_linear_step_host")
+
+
+def lora_linear_fwd(plan: LoraLinearPlan, X, W, A, B, scale, Y=None, stream=None):
+    return plan.fwd(X, W, A, B, scale, Y, stream)
+
+
+def lora_linear_bwd(plan: LoraLinearPlan, dY, X, W, A, B, scale, dX=None, dA=None, dB=None, stream=None):
+    return plan.bwd(dY, X, W, A, B, scale, dX, dA, dB, stream)

@@ -1,0 +1,292 @@
+// Adapter gradients of the LoRA layer (Section 3.2.2, LoRA): tall-skinny contractions over the tokens.
+//
+//   dA = s (dY B)^T X      streams X  [T, d_in]  once, second factor Qt = s (dY B)^T  [r_pad, T] (bf16)
+//   dB = s dY^T (X A^T)    streams dY [T, d_out] once, second factor Pt = s (X A^T)^T [r_pad, T] (bf16)
+//
+// Both are out[c, j] = sum_t S[t, c] * Rt[j, t]: the streamed matrix S is the MN-major A operand of a
+// tcgen05 MMA (M = 128 features, N = r_pad, K = tokens) read from the very 128-byte-swizzled tiles TMA
+// delivers, so the token reduction runs on the tensor cores while the kernel stays bound by the HBM
+// stream.  The dA kernel additionally recomputes X A^T for the slab it holds (same tiles, this time as the
+// K-major operand with M = 128 tokens), because the backward pass is not given the forward's X A^T.
+//
+// Grid: (feature chunks, token chunks).  A CTA keeps feat_chunk x r_pad fp32 sums in TMEM over all of its
+// token slabs.  Cross-CTA sums (over token chunks for the gradient, over feature chunks for X A^T) are
+// written as partials; the last CTA to arrive (a counter, no spinning) adds them in a fixed order, so the
+// result is bitwise reproducible.
+#include "kernels.h"
+#include "sm100_ptx.cuh"
+
+namespace lora {
+
+namespace {
+
+constexpr int kGradBarriers = 2 * kGradMaxStages + 10;
+
+__global__ void __launch_bounds__(kGradThreads, 1)
+lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix [T, C], box 64(c) x 128(t)
+                 const __grid_constant__ CUtensorMap tm_r,   // second factor [r_pad, T], box 64(t) x r_pad
+                 const __grid_constant__ CUtensorMap tm_a,   // A [r, C], box 64(c) x r_pad (with_p only)
+                 const GradParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int NB = p.feat_chunk >> 7;                 // 128-feature accumulator blocks
+  const int rt_box = p.r_pad * 128;                 // bytes of one 64-token box of the second factor
+  const uint32_t ring = smem_u32(smem);
+  const uint32_t rt_base = ring + p.stages * kGradStageBytes;           // 2 buffers x 2 boxes
+  const uint32_t a_base = rt_base + 4 * rt_box;                          // feat_chunk/64 boxes of r_pad x 64
+  const int a_bytes = p.with_p ? (p.feat_chunk >> 6) * rt_box : 0;
+  uint8_t* tail = smem + p.stages * kGradStageBytes + 4 * rt_box + a_bytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tail);
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kGradMaxStages + s); };
+  auto rt_full = [&](int b) { return bar0 + 8u * (2 * kGradMaxStages + b); };
+  auto rt_empty = [&](int b) { return bar0 + 8u * (2 * kGradMaxStages + 2 + b); };
+  auto p_full = [&](int b) { return bar0 + 8u * (2 * kGradMaxStages + 4 + b); };
+  auto p_empty = [&](int b) { return bar0 + 8u * (2 * kGradMaxStages + 6 + b); };
+  const uint32_t a_full = bar0 + 8u * (2 * kGradMaxStages + 8);
+  const uint32_t out_full = bar0 + 8u * (2 * kGradMaxStages + 9);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kGradBarriers);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* last_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int fc = blockIdx.x, tc = blockIdx.y;
+  const int c0 = fc * p.feat_chunk;
+  const int s_begin = static_cast<int>(static_cast<long long>(tc) * p.n_slabs / p.n_token_chunks);
+  const int s_end = static_cast<int>(static_cast<long long>(tc + 1) * p.n_slabs / p.n_token_chunks);
+  const int S = p.stages;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(rt_full(b), 1);
+      mbar_init(rt_empty(b), 1);
+      mbar_init(p_full(b), 1);
+      mbar_init(p_empty(b), 128);
+    }
+    mbar_init(a_full, 1);
+    mbar_init(out_full, 1);
+    *abort_flag = 0;
+    *last_flag = 0;
+    fence_barrier_init();
+    tma_prefetch_desc(&tm_s);
+    tma_prefetch_desc(&tm_r);
+    if (p.with_p) tma_prefetch_desc(&tm_a);
+    if (blockIdx.x == 0 && blockIdx.y == 0 && p.zero_words != nullptr)
+      for (int i = 0; i < p.n_zero_words; ++i) p.zero_words[i] = 0u;
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_slot), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_p = tmem_base + NB * p.r_pad;     // two r_pad-column buffers for X A^T
+
+  if (warp == 0) {
+    // ================================ TMA producer ================================
+    if (lane == 0) {
+      bool ok = true;
+      if (p.with_p) {
+        mbar_arrive_expect_tx(a_full, a_bytes);
+        for (int b = 0; b < (p.feat_chunk >> 6); ++b) tma_load_2d(a_base + b * rt_box, &tm_a, a_full, c0 + 64 * b, 0);
+      }
+      int it = 0;
+      for (int s = s_begin; s < s_end && ok; ++s) {
+        const int ls = s - s_begin, rb = ls & 1, t0 = s * kGradSlab;
+        ok = mbar_wait(rt_empty(rb), ((ls >> 1) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY);
+        if (!ok) break;
+        mbar_arrive_expect_tx(rt_full(rb), 2 * rt_box);
+        tma_load_2d(rt_base + (2 * rb) * rt_box, &tm_r, rt_full(rb), t0, 0);
+        tma_load_2d(rt_base + (2 * rb + 1) * rt_box, &tm_r, rt_full(rb), t0 + 64, 0);
+        for (int nb = 0; nb < NB && ok; ++nb) {
+          const int slot = it % S;
+          ok = mbar_wait(empty_bar(slot), ((it / S) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY);
+          ++it;
+          if (!ok) break;
+          const uint32_t dst = ring + slot * kGradStageBytes;
+          mbar_arrive_expect_tx(full_bar(slot), kGradStageBytes);
+          tma_load_2d(dst, &tm_s, full_bar(slot), c0 + nb * 128, t0);
+          tma_load_2d(dst + 16384, &tm_s, full_bar(slot), c0 + nb * 128 + 64, t0);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ================================ MMA issuer ================================
+    if (lane == 0) {
+      const uint32_t idesc_out = mma_idesc_bf16(128, p.r_pad, true, false);   // A operand = S tile, MN-major
+      const uint32_t idesc_p = mma_idesc_bf16(128, p.r_pad, false, false);    // A operand = S tile, K-major
+      bool ok = true;
+      if (p.with_p) ok = mbar_wait(a_full, 0, abort_flag, p.status, DEV_TIMEOUT_FULL);
+      int it = 0;
+      for (int s = s_begin; s < s_end && ok; ++s) {
+        const int ls = s - s_begin, rb = ls & 1, use = ls >> 1;
+        ok = mbar_wait(rt_full(rb), use & 1, abort_flag, p.status, DEV_TIMEOUT_FULL);
+        if (ok && p.with_p) ok = mbar_wait(p_empty(rb), (use & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_ACC_EMPTY);
+        if (!ok) break;
+        for (int nb = 0; nb < NB && ok; ++nb) {
+          const int slot = it % S;
+          ok = mbar_wait(full_bar(slot), (it / S) & 1, abort_flag, p.status, DEV_TIMEOUT_FULL);
+          ++it;
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t tile = ring + slot * kGradStageBytes;
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {   // 128 tokens = 8 x K16
+            const uint64_t ad = smem_desc_sw128(tile + ks * 2048, 16384, 1024);
+            const uint64_t bd = smem_desc_sw128(rt_base + (2 * rb + (ks >> 2)) * rt_box + (ks & 3) * 32, 16, 1024);
+            mma_bf16_ss(tmem_base + nb * p.r_pad, ad, bd, idesc_out, (ls | ks) != 0 ? 1u : 0u);
+          }
+          if (p.with_p) {
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) { // 128 features = 2 boxes x 4 x K16
+              const int bx = kk >> 2, ks = kk & 3;
+              const uint64_t ad = smem_desc_sw128(tile + bx * 16384 + ks * 32, 16, 1024);
+              const uint64_t bd = smem_desc_sw128(a_base + (nb * 2 + bx) * rt_box + ks * 32, 16, 1024);
+              mma_bf16_ss(tmem_p + rb * p.r_pad, ad, bd, idesc_p, (nb | kk) != 0 ? 1u : 0u);
+            }
+          }
+          mma_commit(empty_bar(slot));
+        }
+        if (!ok) break;
+        mma_commit(rt_empty(rb));
+        if (p.with_p) mma_commit(p_full(rb));
+      }
+      if (ok) mma_commit(out_full);
+    }
+  } else {
+    // ================================ epilogue (128 threads) ================================
+    const int e = threadIdx.x - 64;
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
+    bool alive = true;
+    if (p.with_p) {
+      // ---- X A^T of each slab: partial over this CTA's features -> global; last CTA finishes it ----
+      for (int s = s_begin; s < s_end; ++s) {
+        const int ls = s - s_begin, pb = ls & 1, use = ls >> 1;
+        const int t = s * kGradSlab + row;
+        bool ok = mbar_wait(p_full(pb), use & 1, abort_flag, p.status, DEV_TIMEOUT_SIDE);
+        if (named_bar_or(1, 128, !ok)) { alive = false; break; }
+        tc_fence_after();
+        for (int c16 = 0; c16 < p.r_pad / 16; ++c16) {
+          uint32_t v[16];
+          tmem_ld16(tmem_p + lane_addr + pb * p.r_pad + c16 * 16, v);
+          tmem_ld_wait();
+          if (t < p.T) {
+#pragma unroll
+            for (int q = 0; q < 16; ++q)
+              p.p_part[(static_cast<size_t>(fc) * p.r_pad + c16 * 16 + q) * p.ld_t + t] = __uint_as_float(v[q]);
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(p_empty(pb));
+        __threadfence();
+        named_bar_sync(2, 128);
+        if (e == 0) {
+          const unsigned old = atomicAdd(&p.slab_counters[s], 1u);
+          *last_flag = (old == static_cast<unsigned>(p.n_feat_chunks - 1)) ? 1 : 0;
+        }
+        named_bar_sync(2, 128);
+        const bool last = *last_flag != 0;
+        named_bar_sync(2, 128);          // everyone has read the flag before it is rewritten
+        if (last && t < p.T) {
+          __threadfence();
+          unsigned short* pt = reinterpret_cast<unsigned short*>(p.pt_out);
+          for (int j = 0; j < p.r_pad; ++j) {
+            float acc = 0.f;
+            for (int f = 0; f < p.n_feat_chunks; ++f)
+              acc += __ldcg(&p.p_part[(static_cast<size_t>(f) * p.r_pad + j) * p.ld_t + t]);
+            pt[static_cast<size_t>(j) * p.ld_t + t] =
+                static_cast<unsigned short>(pack_bf16x2(acc * p.scale, 0.f) & 0xFFFFu);
+          }
+        }
+      }
+    }
+    if (alive) {
+      bool ok = mbar_wait(out_full, 0, abort_flag, p.status, DEV_TIMEOUT_ACC);
+      if (!named_bar_or(1, 128, !ok)) {
+        tc_fence_after();
+        // ---- this CTA's sums over its token chunk -> partial buffer ----
+        for (int nb = 0; nb < NB; ++nb) {
+          const int c = c0 + nb * 128 + row;
+          for (int c16 = 0; c16 < p.r_pad / 16; ++c16) {
+            uint32_t v[16];
+            tmem_ld16(tmem_base + lane_addr + nb * p.r_pad + c16 * 16, v);
+            tmem_ld_wait();
+            if (c < p.C) {
+#pragma unroll
+              for (int q = 0; q < 16; ++q)
+                p.out_part[(static_cast<size_t>(tc) * p.r_pad + c16 * 16 + q) * p.c_pad + c] = __uint_as_float(v[q]);
+            }
+          }
+        }
+        __threadfence();
+        named_bar_sync(2, 128);
+        if (e == 0) {
+          const unsigned old = atomicAdd(&p.feat_counters[fc], 1u);
+          *last_flag = (old == static_cast<unsigned>(p.n_token_chunks - 1)) ? 1 : 0;
+        }
+        named_bar_sync(2, 128);
+        if (*last_flag != 0) {
+          __threadfence();
+          // ---- fixed-order sum over the token chunks -> final gradient ----
+          for (int nb = 0; nb < NB; ++nb) {
+            const int c = c0 + nb * 128 + row;
+            if (c >= p.C) continue;
+            for (int j = 0; j < p.r; ++j) {
+              float acc = 0.f;
+              for (int k = 0; k < p.n_token_chunks; ++k)
+                acc += __ldcg(&p.out_part[(static_cast<size_t>(k) * p.r_pad + j) * p.c_pad + c]);
+              if (p.out_is_da) p.out[static_cast<size_t>(j) * p.C + c] = acc;
+              else p.out[static_cast<size_t>(c) * p.r + j] = acc;
+            }
+          }
+        }
+      }
+    }
+  }
+
+  // ================================ teardown ================================
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag && threadIdx.x == 0) {
+    const long long t0 = clock64();          // bounded grace period for copies still in flight
+    while (clock64() - t0 < 2000000LL) {
+    }
+  }
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+}  // namespace
+
+size_t grad_smem_bytes(const GradParams& p) {
+  const size_t a_bytes = p.with_p ? static_cast<size_t>(p.feat_chunk >> 6) * p.r_pad * 128 : 0;
+  return static_cast<size_t>(p.stages) * kGradStageBytes + 4 * static_cast<size_t>(p.r_pad) * 128 + a_bytes +
+         kGradBarriers * 8 + 16 + 1024;
+}
+
+cudaError_t grad_configure() {
+  return cudaFuncSetAttribute(lora_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+}
+
+cudaError_t launch_grad(const CUtensorMap& tmS, const CUtensorMap& tmR, const CUtensorMap& tmA, const GradParams& p,
+                        cudaStream_t stream) {
+  dim3 grid(p.n_feat_chunks, p.n_token_chunks);
+  lora_grad_kernel<<<grid, kGradThreads, grad_smem_bytes(p), stream>>>(tmS, tmR, tmA, p);
+  return cudaGetLastError();
+}
+
+}  // namespace lora

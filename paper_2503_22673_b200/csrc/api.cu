@@ -1,0 +1,594 @@
+// C ABI of the LoRA projection layer: argument checks, the per-shape selector, plans, tensor maps and
+// kernel launches.  See include/lora_linear.h for the contract of every entry point.
+#include "../../include/lora_linear.h"
+
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "kernels.h"
+
+namespace {
+
+using namespace lora;
+
+std::atomic<long long> g_launches{0};
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int ceil_div(long long a, long long b) { return static_cast<int>((a + b - 1) / b); }
+
+// ------------------------------------------------------------------------------------------------
+// selector
+// ------------------------------------------------------------------------------------------------
+// Cost model of one GEMM tile per 16-wide k-step, in SM cycles: the tensor pipe needs N_total / 2 cycles
+// (128 x N_total x 16 MACs at 4096 MAC/cycle), the operand fetch from shared memory (128 + N_total) rows
+// x 32 B at 128 B/cycle.  The tile width with the lowest (waves x per-tile cost) wins; wide tiles win on
+// large grids, narrow tiles when the grid cannot fill the SMs.
+int pick_block_n(long long T, long long N, int r_pad, int num_sms) {
+  const int cands[3] = {192, 128, 64};
+  int best = 192;
+  double best_cost = 1e300;
+  for (int bn : cands) {
+    const long long tiles = static_cast<long long>(ceil_div(T, kBlockM)) * ceil_div(N, bn);
+    const long long waves = (tiles + num_sms - 1) / num_sms;
+    const double ntot = bn + r_pad;
+    const double per_tile = (ntot / 2.0 > (128.0 + ntot) / 4.0) ? ntot / 2.0 : (128.0 + ntot) / 4.0;
+    // fixed per-tile cost (rank-r MMA, accumulator hand-over), in the same unit, for a K of ~4096
+    const double cost = static_cast<double>(waves) * (per_tile + 4.0);
+    if (cost < best_cost - 1e-9) {
+      best_cost = cost;
+      best = bn;
+    }
+  }
+  return best;
+}
+
+struct GradGrid {
+  int feat_chunk, n_feat, n_tok, stages;
+};
+
+GradGrid pick_grad_grid(long long T, long long C, int r_pad, bool with_p, int num_sms) {
+  GradGrid g;
+  int fc = (r_pad <= 32) ? 512 : 256;
+  const int c128 = ceil_div(C, 128) * 128;
+  if (fc > c128) fc = c128;
+  g.feat_chunk = fc;
+  g.n_feat = ceil_div(C, fc);
+  const int n_slabs = ceil_div(T, kGradSlab);
+  int n_tok = (num_sms + g.n_feat / 2) / g.n_feat;
+  if (n_tok < 1) n_tok = 1;
+  if (n_tok > n_slabs) n_tok = n_slabs;
+  if (n_tok < 1) n_tok = 1;
+  g.n_tok = n_tok;
+  const size_t fixed = 4 * static_cast<size_t>(r_pad) * 128 + (with_p ? static_cast<size_t>(fc / 64) * r_pad * 128 : 0) + 4096;
+  int stages = static_cast<int>((232448 - fixed) / kGradStageBytes);
+  if (stages > kGradMaxStages) stages = kGradMaxStages;
+  if (stages < 2) stages = 2;
+  g.stages = stages;
+  return g;
+}
+
+int check_shape(const lora_shape_t* s) {
+  if (s == nullptr) return LORA_ERR_INVALID_ARG;
+  if (s->T < 0 || s->d_in <= 0 || s->d_out <= 0 || s->r <= 0) return LORA_ERR_INVALID_ARG;
+  if (s->T > (1ll << 30) || s->d_in > (1ll << 24) || s->d_out > (1ll << 24)) return LORA_ERR_UNSUPPORTED_SHAPE;
+  if (s->d_in % 8 != 0 || s->d_out % 8 != 0) return LORA_ERR_UNSUPPORTED_SHAPE;
+  if (s->r % 8 != 0 || s->r < 8 || s->r > 64) return LORA_ERR_UNSUPPORTED_SHAPE;
+  return LORA_OK;
+}
+
+int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
+  const int rc = check_shape(s);
+  if (rc != LORA_OK) return rc;
+  if (num_sms <= 0 || c == nullptr) return LORA_ERR_INVALID_ARG;
+  std::memset(c, 0, sizeof(*c));
+  const long long T = s->T > 0 ? s->T : 1;
+  c->block_m = kBlockM;
+  c->block_k = kBlockK;
+  c->r_pad = static_cast<int>((s->r + 15) / 16 * 16);
+  c->fwd_block_n = pick_block_n(T, s->d_out, c->r_pad, num_sms);
+  c->dx_block_n = pick_block_n(T, s->d_in, c->r_pad, num_sms);
+  c->stages = 4;
+  c->group_m = 8;
+  c->split_k = 1;
+  c->tail_delay = 8;
+  const long long fwd_tiles = static_cast<long long>(ceil_div(T, kBlockM)) * ceil_div(s->d_out, c->fwd_block_n);
+  const long long dx_tiles = static_cast<long long>(ceil_div(T, kBlockM)) * ceil_div(s->d_in, c->dx_block_n);
+  c->fwd_ctas = static_cast<int>(fwd_tiles < num_sms ? fwd_tiles : num_sms);
+  c->dx_ctas = static_cast<int>(dx_tiles < num_sms ? dx_tiles : num_sms);
+  const GradGrid ga = pick_grad_grid(T, s->d_in, c->r_pad, true, num_sms);
+  const GradGrid gb = pick_grad_grid(T, s->d_out, c->r_pad, false, num_sms);
+  c->grad_feat_chunk = ga.feat_chunk;
+  c->grad_stages = ga.stages < gb.stages ? ga.stages : gb.stages;
+  c->da_feat_chunks = ga.n_feat;
+  c->da_token_chunks = ga.n_tok;
+  c->db_feat_chunks = gb.n_feat;
+  c->db_token_chunks = gb.n_tok;
+  c->reserved[0] = gb.feat_chunk;   // feature chunk of the dB kernel (differs from dA's only for small d_out)
+  return LORA_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// backward workspace layout
+// ------------------------------------------------------------------------------------------------
+struct WsLayout {
+  size_t qt, pt, p_part, da_part, db_part, counters, total;
+  int ld_t, c_pad_a, c_pad_b, n_slabs, n_counters;
+};
+
+WsLayout ws_layout(const lora_shape_t& s, const lora_kernel_config_t& c) {
+  WsLayout w;
+  const long long T = s.T > 0 ? s.T : 1;
+  w.ld_t = static_cast<int>(align_up(static_cast<size_t>(T), 64));
+  w.c_pad_a = static_cast<int>(align_up(static_cast<size_t>(s.d_in), 32));
+  w.c_pad_b = static_cast<int>(align_up(static_cast<size_t>(s.d_out), 32));
+  w.n_slabs = ceil_div(T, kGradSlab);
+  w.n_counters = w.n_slabs + c.da_feat_chunks + c.db_feat_chunks;
+  size_t off = 0;
+  w.qt = off;       off += align_up(static_cast<size_t>(c.r_pad) * w.ld_t * 2, kAlign);
+  w.pt = off;       off += align_up(static_cast<size_t>(c.r_pad) * w.ld_t * 2, kAlign);
+  w.p_part = off;   off += align_up(static_cast<size_t>(c.da_feat_chunks) * c.r_pad * w.ld_t * 4, kAlign);
+  w.da_part = off;  off += align_up(static_cast<size_t>(c.da_token_chunks) * c.r_pad * w.c_pad_a * 4, kAlign);
+  w.db_part = off;  off += align_up(static_cast<size_t>(c.db_token_chunks) * c.r_pad * w.c_pad_b * 4, kAlign);
+  w.counters = off; off += align_up(static_cast<size_t>(w.n_counters) * 4, kAlign);
+  w.total = off;
+  return w;
+}
+
+// ------------------------------------------------------------------------------------------------
+// tensor maps
+// ------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = []() -> EncodeTiledFn {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess) return nullptr;
+    if (q != cudaDriverEntryPointSuccess) return nullptr;
+    return reinterpret_cast<EncodeTiledFn>(f);
+  }();
+  return fn;
+}
+
+// 2-D row-major tensor of `elem_bytes`-wide elements, 128-byte swizzle, zero fill outside the tensor.
+bool make_tmap(CUtensorMap* m, const void* ptr, CUtensorMapDataType dt, int elem_bytes, uint64_t inner, uint64_t outer,
+               uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_outer) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  const cuuint64_t dims[2] = {inner, outer};
+  const cuuint64_t strides[1] = {pitch_bytes};
+  const cuuint32_t box[2] = {box_inner, box_outer};
+  const cuuint32_t estr[2] = {1, 1};
+  (void)elem_bytes;
+  const CUresult r = fn(m, dt, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+bool make_bf16_tmap(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t outer, uint64_t pitch_elems,
+                    uint32_t box_inner, uint32_t box_outer) {
+  return make_tmap(m, ptr, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, inner, outer, pitch_elems * 2, box_inner, box_outer);
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------
+// plan
+// ------------------------------------------------------------------------------------------------
+struct lora_plan {
+  lora_shape_t shape;
+  lora_kernel_config_t cfg;
+  WsLayout ws;
+  int device;
+  int num_sms;
+  unsigned* d_status;   // 64 words of device memory
+  void* workspace;
+  size_t workspace_bytes;
+};
+
+namespace {
+
+struct DeviceGuard {
+  int prev = -1;
+  bool switched = false;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = (cudaSetDevice(dev) == cudaSuccess);
+  }
+  ~DeviceGuard() {
+    if (switched) cudaSetDevice(prev);
+  }
+};
+
+int launch_fwd(lora_plan* pl, const void* X, const void* W, const void* A, const void* B, float scale, void* Y,
+               cudaStream_t st) {
+  const lora_shape_t& s = pl->shape;
+  const lora_kernel_config_t& c = pl->cfg;
+  CUtensorMap tmX, tmW, tmA, tmB, tmY;
+  bool ok = make_bf16_tmap(&tmX, X, s.d_in, s.T, s.d_in, 64, kBlockM);
+  ok = ok && make_bf16_tmap(&tmW, W, s.d_in, s.d_out, s.d_in, 64, c.fwd_block_n);
+  ok = ok && make_bf16_tmap(&tmA, A, s.d_in, s.r, s.d_in, 64, c.r_pad);
+  ok = ok && make_bf16_tmap(&tmB, B, s.r, s.d_out, s.r, 64, c.fwd_block_n);
+  ok = ok && make_bf16_tmap(&tmY, Y, s.d_out, s.T, s.d_out, 64, kBlockM);
+  if (!ok) return LORA_ERR_CUDA;
+  GemmParams p{};
+  p.M = static_cast<int>(s.T);
+  p.N = static_cast<int>(s.d_out);
+  p.K = static_cast<int>(s.d_in);
+  p.r_pad = c.r_pad;
+  p.block_n = c.fwd_block_n;
+  p.tiles_m = ceil_div(s.T, kBlockM);
+  p.tiles_n = ceil_div(s.d_out, c.fwd_block_n);
+  p.num_tiles = p.tiles_m * p.tiles_n;
+  p.kblocks = ceil_div(s.d_in, kBlockK);
+  p.group_m = c.group_m;
+  p.stages = c.stages;
+  p.tail_delay = c.tail_delay;
+  p.scale = scale;
+  p.rt_out = nullptr;
+  p.ld_rt = 0;
+  p.status = pl->d_status;
+  p.zero_words = nullptr;
+  p.n_zero_words = 0;
+  if (launch_gemm_fwd(tmX, tmW, tmA, tmB, tmY, p, c.fwd_ctas, st) != cudaSuccess) return LORA_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return LORA_OK;
+}
+
+int launch_bwd(lora_plan* pl, const void* dY, const void* X, const void* W, const void* A, const void* B, float scale,
+               void* dX, void* dA, void* dB, cudaStream_t st) {
+  const lora_shape_t& s = pl->shape;
+  const lora_kernel_config_t& c = pl->cfg;
+  const WsLayout& w = pl->ws;
+  uint8_t* ws = static_cast<uint8_t*>(pl->workspace);
+  __nv_bfloat16* qt = reinterpret_cast<__nv_bfloat16*>(ws + w.qt);
+  __nv_bfloat16* pt = reinterpret_cast<__nv_bfloat16*>(ws + w.pt);
+  unsigned* counters = reinterpret_cast<unsigned*>(ws + w.counters);
+
+  // ---- dX = dY W + s (dY B) A ; also leaves Qt = s (dY B)^T in the workspace ----
+  {
+    CUtensorMap tmdY, tmW, tmB, tmA, tmdX;
+    bool ok = make_bf16_tmap(&tmdY, dY, s.d_out, s.T, s.d_out, 64, kBlockM);
+    ok = ok && make_bf16_tmap(&tmW, W, s.d_in, s.d_out, s.d_in, 64, 64);
+    ok = ok && make_bf16_tmap(&tmB, B, s.r, s.d_out, s.r, 64, 64);
+    ok = ok && make_bf16_tmap(&tmA, A, s.d_in, s.r, s.d_in, 64, c.r_pad);
+    ok = ok && make_bf16_tmap(&tmdX, dX, s.d_in, s.T, s.d_in, 64, kBlockM);
+    if (!ok) return LORA_ERR_CUDA;
+    GemmParams p{};
+    p.M = static_cast<int>(s.T);
+    p.N = static_cast<int>(s.d_in);
+    p.K = static_cast<int>(s.d_out);
+    p.r_pad = c.r_pad;
+    p.block_n = c.dx_block_n;
+    p.tiles_m = ceil_div(s.T, kBlockM);
+    p.tiles_n = ceil_div(s.d_in, c.dx_block_n);
+    p.num_tiles = p.tiles_m * p.tiles_n;
+    p.kblocks = ceil_div(s.d_out, kBlockK);
+    p.group_m = c.group_m;
+    p.stages = c.stages;
+    p.tail_delay = c.tail_delay;
+    p.scale = scale;
+    p.rt_out = qt;
+    p.ld_rt = w.ld_t;
+    p.status = pl->d_status;
+    p.zero_words = counters;
+    p.n_zero_words = w.n_counters;
+    if (launch_gemm_dx(tmdY, tmW, tmB, tmA, tmdX, p, c.dx_ctas, st) != cudaSuccess) return LORA_ERR_CUDA;
+    g_launches.fetch_add(1);
+  }
+  // ---- dA = Qt-contraction over X; recomputes X A^T and leaves Pt = s (X A^T)^T ----
+  {
+    CUtensorMap tmS, tmR, tmA;
+    bool ok = make_bf16_tmap(&tmS, X, s.d_in, s.T, s.d_in, 64, kGradSlab);
+    ok = ok && make_bf16_tmap(&tmR, qt, s.T, c.r_pad, w.ld_t, 64, c.r_pad);
+    ok = ok && make_bf16_tmap(&tmA, A, s.d_in, s.r, s.d_in, 64, c.r_pad);
+    if (!ok) return LORA_ERR_CUDA;
+    GradParams g{};
+    g.T = static_cast<int>(s.T);
+    g.C = static_cast<int>(s.d_in);
+    g.r = static_cast<int>(s.r);
+    g.r_pad = c.r_pad;
+    g.feat_chunk = c.grad_feat_chunk;
+    g.n_feat_chunks = c.da_feat_chunks;
+    g.n_token_chunks = c.da_token_chunks;
+    g.n_slabs = w.n_slabs;
+    g.stages = c.grad_stages;
+    g.with_p = 1;
+    g.out_is_da = 1;
+    g.scale = scale;
+    g.out = static_cast<float*>(dA);
+    g.out_part = reinterpret_cast<float*>(ws + w.da_part);
+    g.c_pad = w.c_pad_a;
+    g.p_part = reinterpret_cast<float*>(ws + w.p_part);
+    g.pt_out = pt;
+    g.ld_t = w.ld_t;
+    g.slab_counters = counters;
+    g.feat_counters = counters + w.n_slabs;
+    g.status = pl->d_status;
+    g.zero_words = nullptr;
+    g.n_zero_words = 0;
+    if (launch_grad(tmS, tmR, tmA, g, st) != cudaSuccess) return LORA_ERR_CUDA;
+    g_launches.fetch_add(1);
+  }
+  // ---- dB = Pt-contraction over dY ----
+  {
+    CUtensorMap tmS, tmR;
+    bool ok = make_bf16_tmap(&tmS, dY, s.d_out, s.T, s.d_out, 64, kGradSlab);
+    ok = ok && make_bf16_tmap(&tmR, pt, s.T, c.r_pad, w.ld_t, 64, c.r_pad);
+    if (!ok) return LORA_ERR_CUDA;
+    GradParams g{};
+    g.T = static_cast<int>(s.T);
+    g.C = static_cast<int>(s.d_out);
+    g.r = static_cast<int>(s.r);
+    g.r_pad = c.r_pad;
+    g.feat_chunk = c.reserved[0];
+    g.n_feat_chunks = c.db_feat_chunks;
+    g.n_token_chunks = c.db_token_chunks;
+    g.n_slabs = w.n_slabs;
+    g.stages = c.grad_stages;
+    g.with_p = 0;
+    g.out_is_da = 0;
+    g.scale = scale;
+    g.out = static_cast<float*>(dB);
+    g.out_part = reinterpret_cast<float*>(ws + w.db_part);
+    g.c_pad = w.c_pad_b;
+    g.p_part = nullptr;
+    g.pt_out = nullptr;
+    g.ld_t = w.ld_t;
+    g.slab_counters = nullptr;
+    g.feat_counters = counters + w.n_slabs + c.da_feat_chunks;
+    g.status = pl->d_status;
+    g.zero_words = nullptr;
+    g.n_zero_words = 0;
+    if (launch_grad(tmS, tmR, tmR, g, st) != cudaSuccess) return LORA_ERR_CUDA;
+    g_launches.fetch_add(1);
+  }
+  return LORA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int lora_select_config(const lora_shape_t* shape, int num_sms, lora_kernel_config_t* out) {
+  return select_config(shape, num_sms, out);
+}
+
+int lora_workspace_bytes(const lora_shape_t* shape, int num_sms, size_t* bwd_bytes) {
+  if (bwd_bytes == nullptr) return LORA_ERR_INVALID_ARG;
+  lora_kernel_config_t c;
+  const int rc = select_config(shape, num_sms, &c);
+  if (rc != LORA_OK) return rc;
+  *bwd_bytes = ws_layout(*shape, c).total;
+  return LORA_OK;
+}
+
+int lora_plan_create(const lora_shape_t* shape, int device, lora_plan_t** out) {
+  if (out == nullptr) return LORA_ERR_INVALID_ARG;
+  *out = nullptr;
+  int rc = check_shape(shape);
+  if (rc != LORA_OK) return rc;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || count <= 0) {
+    cudaGetLastError();
+    return LORA_ERR_NO_DEVICE;
+  }
+  if (device < 0 || device >= count) return LORA_ERR_INVALID_ARG;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return LORA_ERR_CUDA;
+  if (prop.major != 10) return LORA_ERR_NO_DEVICE;
+  DeviceGuard guard(device);
+  lora_plan* pl = new (std::nothrow) lora_plan();
+  if (pl == nullptr) return LORA_ERR_INVALID_ARG;
+  pl->shape = *shape;
+  pl->device = device;
+  pl->num_sms = prop.multiProcessorCount;
+  rc = select_config(shape, pl->num_sms, &pl->cfg);
+  if (rc != LORA_OK) {
+    delete pl;
+    return rc;
+  }
+  pl->ws = ws_layout(*shape, pl->cfg);
+  pl->workspace = nullptr;
+  pl->workspace_bytes = 0;
+  pl->d_status = nullptr;
+  if (gemm_configure() != cudaSuccess || grad_configure() != cudaSuccess || encode_fn() == nullptr ||
+      cudaMalloc(&pl->d_status, 256) != cudaSuccess || cudaMemset(pl->d_status, 0, 256) != cudaSuccess) {
+    cudaGetLastError();
+    if (pl->d_status) cudaFree(pl->d_status);
+    delete pl;
+    return LORA_ERR_CUDA;
+  }
+  *out = pl;
+  return LORA_OK;
+}
+
+int lora_plan_destroy(lora_plan_t* plan) {
+  if (plan == nullptr) return LORA_ERR_INVALID_ARG;
+  DeviceGuard guard(plan->device);
+  if (plan->d_status) cudaFree(plan->d_status);
+  delete plan;
+  return LORA_OK;
+}
+
+int lora_plan_workspace_bytes(const lora_plan_t* plan, size_t* fwd_bytes, size_t* bwd_bytes) {
+  if (plan == nullptr) return LORA_ERR_INVALID_ARG;
+  if (fwd_bytes) *fwd_bytes = 0;
+  if (bwd_bytes) *bwd_bytes = plan->ws.total;
+  return LORA_OK;
+}
+
+int lora_plan_set_workspace(lora_plan_t* plan, void* dev_ptr, size_t bytes) {
+  if (plan == nullptr) return LORA_ERR_INVALID_ARG;
+  if (dev_ptr == nullptr) {
+    plan->workspace = nullptr;
+    plan->workspace_bytes = 0;
+    return bytes == 0 ? LORA_OK : LORA_ERR_INVALID_ARG;
+  }
+  if ((reinterpret_cast<uintptr_t>(dev_ptr) & (kAlign - 1)) != 0) return LORA_ERR_MISALIGNED;
+  if (bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
+  plan->workspace = dev_ptr;
+  plan->workspace_bytes = bytes;
+  return LORA_OK;
+}
+
+int lora_plan_get_config(const lora_plan_t* plan, lora_kernel_config_t* out) {
+  if (plan == nullptr || out == nullptr) return LORA_ERR_INVALID_ARG;
+  *out = plan->cfg;
+  return LORA_OK;
+}
+
+int lora_plan_describe(const lora_plan_t* plan, char* buf, size_t n) {
+  if (plan == nullptr || buf == nullptr || n == 0) return LORA_ERR_INVALID_ARG;
+  const lora_kernel_config_t& c = plan->cfg;
+  std::snprintf(buf, n,
+                "T=%lld d_in=%lld d_out=%lld r=%lld | sms=%d tile fwd 128x%dx64 dx 128x%dx64 stages=%d group_m=%d "
+                "split_k=%d r_pad=%d ctas fwd=%d dx=%d tail_delay=%d | grad chunk=%d stages=%d dA grid=%dx%d dB grid=%dx%d "
+                "| bwd workspace=%zu B",
+                (long long)plan->shape.T, (long long)plan->shape.d_in, (long long)plan->shape.d_out,
+                (long long)plan->shape.r, plan->num_sms, c.fwd_block_n, c.dx_block_n, c.stages, c.group_m, c.split_k,
+                c.r_pad, c.fwd_ctas, c.dx_ctas, c.tail_delay, c.grad_feat_chunk, c.grad_stages, c.da_feat_chunks,
+                c.da_token_chunks, c.db_feat_chunks, c.db_token_chunks, plan->ws.total);
+  return LORA_OK;
+}
+
+int lora_linear_fwd(lora_plan_t* plan, const void* X, const void* W, const void* A, const void* B, float scale,
+                    void* Y, void* stream) {
+  if (plan == nullptr) return LORA_ERR_INVALID_ARG;
+  if (plan->shape.T == 0) return LORA_OK;
+  if (!X || !W || !A || !B || !Y) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(W) || !aligned16(A) || !aligned16(B) || !aligned16(Y)) return LORA_ERR_MISALIGNED;
+  DeviceGuard guard(plan->device);
+  return launch_fwd(plan, X, W, A, B, scale, Y, static_cast<cudaStream_t>(stream));
+}
+
+int lora_linear_bwd(lora_plan_t* plan, const void* dY, const void* X, const void* W, const void* A, const void* B,
+                    float scale, void* dX, void* dA, void* dB, void* stream) {
+  if (plan == nullptr) return LORA_ERR_INVALID_ARG;
+  if (!dA || !dB) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(dA) || !aligned16(dB)) return LORA_ERR_MISALIGNED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  DeviceGuard guard(plan->device);
+  if (plan->shape.T == 0) {   // empty batch: the sums over tokens are empty
+    if (cudaMemsetAsync(dA, 0, sizeof(float) * plan->shape.r * plan->shape.d_in, st) != cudaSuccess ||
+        cudaMemsetAsync(dB, 0, sizeof(float) * plan->shape.d_out * plan->shape.r, st) != cudaSuccess)
+      return LORA_ERR_CUDA;
+    return LORA_OK;
+  }
+  if (!dY || !X || !W || !A || !B || !dX) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(dY) || !aligned16(X) || !aligned16(W) || !aligned16(A) || !aligned16(B) || !aligned16(dX))
+    return LORA_ERR_MISALIGNED;
+  if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
+  return launch_bwd(plan, dY, X, W, A, B, scale, dX, dA, dB, st);
+}
+
+int lora_step_host_staging_bytes(const lora_shape_t* shape, size_t* bytes) {
+  if (bytes == nullptr) return LORA_ERR_INVALID_ARG;
+  const int rc = check_shape(shape);
+  if (rc != LORA_OK) return rc;
+  const size_t T = shape->T, di = shape->d_in, dout = shape->d_out, r = shape->r;
+  size_t off = 0;
+  off += align_up(T * di * 2, kAlign) * 2;      // X, dX
+  off += align_up(T * dout * 2, kAlign) * 2;      // dY, Y
+  off += align_up(r * di * 2, kAlign);          // A
+  off += align_up(dout * r * 2, kAlign);          // B
+  off += align_up(r * di * 4, kAlign);          // dA
+  off += align_up(dout * r * 4, kAlign);          // dB
+  *bytes = off;
+  return LORA_OK;
+}
+
+int lora_linear_step_host(lora_plan_t* plan, const void* h_X, const void* W, const void* h_A, const void* h_B,
+                          const void* h_dY, float scale, void* h_Y, void* h_dX, void* h_dA, void* h_dB, void* staging,
+                          size_t staging_bytes, void* stream) {
+  if (plan == nullptr) return LORA_ERR_INVALID_ARG;
+  if (!h_X || !W || !h_A || !h_B || !h_dY || !h_Y || !h_dX || !h_dA || !h_dB || !staging) return LORA_ERR_INVALID_ARG;
+  size_t need = 0;
+  lora_step_host_staging_bytes(&plan->shape, &need);
+  if (staging_bytes < need) return LORA_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(staging) & (kAlign - 1)) != 0) return LORA_ERR_MISALIGNED;
+  const size_t T = plan->shape.T, di = plan->shape.d_in, dout = plan->shape.d_out, r = plan->shape.r;
+  uint8_t* base = static_cast<uint8_t*>(staging);
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    uint8_t* p = base + off;
+    off += align_up(bytes, kAlign);
+    return p;
+  };
+  uint8_t* dXin = take(T * di * 2);
+  uint8_t* ddX = take(T * di * 2);
+  uint8_t* ddY = take(T * dout * 2);
+  uint8_t* dYout = take(T * dout * 2);
+  uint8_t* dAin = take(r * di * 2);
+  uint8_t* dBin = take(dout * r * 2);
+  uint8_t* ddA = take(r * di * 4);
+  uint8_t* ddB = take(dout * r * 4);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  DeviceGuard guard(plan->device);
+  bool ok = true;
+  if (T > 0) {
+    ok = ok && cudaMemcpyAsync(dXin, h_X, T * di * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(ddY, h_dY, T * dout * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  }
+  ok = ok && cudaMemcpyAsync(dAin, h_A, r * di * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(dBin, h_B, dout * r * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (!ok) return LORA_ERR_CUDA;
+  int rc = lora_linear_fwd(plan, dXin, W, dAin, dBin, scale, dYout, stream);
+  if (rc != LORA_OK) return rc;
+  rc = lora_linear_bwd(plan, ddY, dXin, W, dAin, dBin, scale, ddX, ddA, ddB, stream);
+  if (rc != LORA_OK) return rc;
+  if (T > 0) {
+    ok = ok && cudaMemcpyAsync(h_Y, dYout, T * dout * 2, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(h_dX, ddX, T * di * 2, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  }
+  ok = ok && cudaMemcpyAsync(h_dA, ddA, r * di * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(h_dB, ddB, dout * r * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  return ok ? LORA_OK : LORA_ERR_CUDA;
+}
+
+int lora_last_device_status(lora_plan_t* plan, void* stream, int* code, char* msg, size_t n) {
+  if (plan == nullptr || code == nullptr) return LORA_ERR_INVALID_ARG;
+  DeviceGuard guard(plan->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaStreamSynchronize(st) != cudaSuccess) return LORA_ERR_CUDA;
+  unsigned word = 0;
+  if (cudaMemcpy(&word, plan->d_status, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return LORA_ERR_CUDA;
+  if (word == 0) {
+    *code = LORA_OK;
+    if (msg && n) std::snprintf(msg, n, "ok");
+    return LORA_OK;
+  }
+  *code = LORA_ERR_DEVICE_TIMEOUT;
+  static const char* what[] = {"",          "MMA waited for a TMA stage",        "TMA producer waited for a free stage",
+                               "epilogue waited for the rank-r accumulator",     "MMA waited for the bf16 rank-r operand",
+                               "epilogue waited for the accumulator",            "MMA waited for a drained accumulator",
+                               "other wait"};
+  if (msg && n) std::snprintf(msg, n, "device wait ran out: %s (CTA %u)", what[word & 7u], word >> 8);
+  if (cudaMemset(plan->d_status, 0, 256) != cudaSuccess) return LORA_ERR_CUDA;
+  return LORA_OK;
+}
+
+const char* lora_strerror(int code) {
+  switch (code) {
+    case LORA_OK: return "ok";
+    case LORA_ERR_INVALID_ARG: return "invalid argument";
+    case LORA_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case LORA_ERR_MISALIGNED: return "pointer not sufficiently aligned";
+    case LORA_ERR_WORKSPACE: return "workspace missing or too small";
+    case LORA_ERR_CUDA: return "CUDA call failed";
+    case LORA_ERR_DEVICE_TIMEOUT: return "a device-side wait ran out";
+    case LORA_ERR_NO_DEVICE: return "no sm_100 CUDA device";
+    default: return "unknown status";
+  }
+}
+
+int64_t lora_launch_count(void) { return g_launches.load(); }
+
+}  // extern "C"

@@ -1,0 +1,83 @@
+// Internal launcher interface between the C ABI (api.cu) and the kernels.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace lora {
+
+// ---- dense GEMM + fused rank-r adapter (forward Y, backward dX) -------------------------------
+constexpr int kBlockM = 128;          // token rows per tile (one TMEM lane per row)
+constexpr int kBlockK = 64;           // contraction elements per stage (one 128-byte swizzle row)
+constexpr int kStageABytes = kBlockM * 128;
+constexpr int kStageBBytes = 256 * 128;
+constexpr int kStageBytes = kStageABytes + kStageBBytes;
+constexpr int kStagingBytes = 128 * 128;   // one 128 x 64 bf16 output chunk / the bf16 rank-r operand
+constexpr int kGemmThreads = 192;          // warp 0 TMA, warp 1 MMA + TMEM, warps 2..5 epilogue
+constexpr int kMaxStages = 8;
+constexpr int kGemmBarriers = 2 * kMaxStages + 8;
+
+struct GemmParams {
+  int M, N, K;            // output rows (tokens), output columns, contraction length
+  int r_pad;              // rank rounded up to a multiple of 16
+  int block_n;            // output columns per tile: 64, 128 or 192
+  int tiles_m, tiles_n, num_tiles, kblocks;
+  int group_m;            // m-tiles per rasterisation band
+  int stages;             // ring depth
+  int tail_delay;         // main-loop k-blocks of the next tile issued before the previous tile's rank-r MMA
+  float scale;
+  __nv_bfloat16* rt_out;  // backward only: scale * (dY B)^T as bf16 [r_pad][ld_rt]; nullptr otherwise
+  int ld_rt;
+  unsigned* status;       // device status word
+  unsigned* zero_words;   // words this kernel clears for the kernels that follow it (may be null)
+  int n_zero_words;
+};
+
+size_t gemm_smem_bytes(int stages);
+
+// Y / dX = act * Wop + scale * (act * sideop) * tailop, see gemm_lora.cu
+cudaError_t launch_gemm_fwd(const CUtensorMap& tmX, const CUtensorMap& tmW, const CUtensorMap& tmA,
+                            const CUtensorMap& tmB, const CUtensorMap& tmY, const GemmParams& p, int ctas,
+                            cudaStream_t stream);
+cudaError_t launch_gemm_dx(const CUtensorMap& tmdY, const CUtensorMap& tmW, const CUtensorMap& tmB,
+                           const CUtensorMap& tmA, const CUtensorMap& tmdX, const GemmParams& p, int ctas,
+                           cudaStream_t stream);
+cudaError_t gemm_configure();   // opt in to the large dynamic shared memory (once per device)
+
+// ---- adapter gradients: tall-skinny contraction over tokens -----------------------------------
+constexpr int kGradThreads = 192;
+constexpr int kGradSlab = 128;             // tokens per slab
+constexpr int kGradStageBytes = 2 * kBlockM * 128;   // 128 tokens x 128 features, bf16
+constexpr int kGradMaxStages = 6;
+
+struct GradParams {
+  int T, C;               // tokens, features of the streamed matrix (d_in for dA, d_out for dB)
+  int r, r_pad;
+  int feat_chunk;         // features per CTA (multiple of 128)
+  int n_feat_chunks, n_token_chunks, n_slabs;
+  int stages;
+  int with_p;             // 1: also accumulate X A^T for the slab (dA kernel)
+  int out_is_da;          // 1: out[j * C + c] (dA), 0: out[c * r + j] (dB)
+  float scale;
+  float* out;             // final fp32 gradient
+  float* out_part;        // [n_token_chunks][r_pad][C_pad]  partial sums (fixed-order reduction)
+  int c_pad;              // row pitch of out_part
+  float* p_part;          // [n_feat_chunks][r_pad][ld_t] partial X A^T (with_p)
+  __nv_bfloat16* pt_out;  // [r_pad][ld_t]: scale * (X A^T)^T as bf16 (with_p)
+  int ld_t;
+  unsigned* feat_counters;  // [n_feat_chunks] arrivals per feature chunk
+  unsigned* slab_counters;  // [n_slabs] arrivals per token slab (with_p)
+  unsigned* status;
+  unsigned* zero_words;
+  int n_zero_words;
+};
+
+size_t grad_smem_bytes(const GradParams& p);
+cudaError_t grad_configure();
+// tmS: streamed matrix [T, C] box [64 features, 128 tokens]; tmR: [r_pad, T] box [64 tokens, r_pad];
+// tmA: A [r, C] box [64 features, r_pad] (only read when with_p)
+cudaError_t launch_grad(const CUtensorMap& tmS, const CUtensorMap& tmR, const CUtensorMap& tmA,
+                        const GradParams& p, cudaStream_t stream);
+
+}  // namespace lora

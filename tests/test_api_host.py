@@ -1,0 +1,111 @@
+"""Host-side checks that need no GPU: the library loads, exports what include/lora_linear.h
+declares, and the selector / workspace / argument checks behave."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2503_22673_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "lora_linear.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(lora_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = binding.load()
+    names = _declared_symbols()
+    assert "lora_linear_fwd" in names and "lora_linear_bwd" in names
+    for n in names:
+        assert hasattr(lib, n), n
+    assert sorted(binding.EXPORTS) == names
+
+
+def test_strerror_and_launch_count():
+    assert binding.strerror(0) == "ok"
+    assert "shape" in binding.strerror(binding.LORA_ERR_UNSUPPORTED_SHAPE)
+    assert binding.strerror(-12345) == "unknown status"
+    assert binding.launch_count() >= 0
+
+
+@pytest.mark.parametrize("shape", [(8192, 4096, 4096, 16), (16384, 4096, 14336, 16), (16384, 14336, 4096, 64),
+                                   (256, 512, 512, 8), (32768, 4096, 1024, 16), (1, 8, 8, 8), (300, 520, 200, 24)])
+def test_selector_invariants(shape):
+    T, d_in, d_out, r = shape
+    c = binding.select_config(T, d_in, d_out, r, 148)
+    assert c["block_m"] == 128 and c["block_k"] == 64
+    assert c["r_pad"] % 16 == 0 and r <= c["r_pad"] < r + 16
+    for bn in (c["fwd_block_n"], c["dx_block_n"]):
+        assert bn in (64, 128, 192) and bn + c["r_pad"] <= 256          # one MMA covers tile + adapter columns
+    m_tiles = -(-T // 128)
+    assert 1 <= c["fwd_ctas"] <= min(148, m_tiles * -(-d_out // c["fwd_block_n"]))
+    assert 1 <= c["dx_ctas"] <= min(148, m_tiles * -(-d_in // c["dx_block_n"]))
+    assert c["stages"] * (128 * 128 + 256 * 128) + 2 * 16384 + 1024 + 256 <= 232448      # fits 227 KiB
+    assert c["split_k"] == 1
+    n_slabs = -(-T // 128)
+    assert 1 <= c["da_token_chunks"] <= n_slabs and 1 <= c["db_token_chunks"] <= n_slabs
+    fc = c["grad_feat_chunk"]
+    assert fc % 128 == 0 and (fc // 128) * c["r_pad"] + 2 * c["r_pad"] <= 512             # TMEM columns
+    assert c["da_feat_chunks"] == -(-d_in // fc)
+    assert 2 <= c["grad_stages"] <= 6
+
+
+def test_selector_prefers_narrow_tiles_on_small_grids():
+    small = binding.select_config(256, 512, 512, 8, 148)
+    big = binding.select_config(16384, 4096, 14336, 16, 148)
+    assert small["fwd_block_n"] == 64 and small["fwd_ctas"] == 16
+    assert big["fwd_block_n"] >= 128 and big["fwd_ctas"] == 148
+
+
+@pytest.mark.parametrize("bad,code", [((128, 4100, 64, 16), binding.LORA_ERR_UNSUPPORTED_SHAPE),
+                                      ((128, 64, 60, 16), binding.LORA_ERR_UNSUPPORTED_SHAPE),
+                                      ((128, 64, 64, 12), binding.LORA_ERR_UNSUPPORTED_SHAPE),
+                                      ((128, 64, 64, 72), binding.LORA_ERR_UNSUPPORTED_SHAPE),
+                                      ((-1, 64, 64, 16), binding.LORA_ERR_INVALID_ARG),
+                                      ((128, 0, 64, 16), binding.LORA_ERR_INVALID_ARG)])
+def test_selector_rejects_bad_shapes(bad, code):
+    with pytest.raises(binding.LoraError) as ei:
+        binding.select_config(*bad)
+    assert ei.value.code == code
+    with pytest.raises(binding.LoraError):
+        binding.workspace_bytes(*bad)
+
+
+def test_workspace_is_small_next_to_the_streams():
+    # scratch for Qt, Pt and the fixed-order partial sums; forward needs none
+    T, d_in, d_out, r = 8192, 4096, 4096, 16
+    ws = binding.workspace_bytes(T, d_in, d_out, r)
+    assert 0 < ws < (T * d_in * 2) // 2
+    assert binding.workspace_bytes(0, d_in, d_out, r) > 0
+
+
+def test_null_arguments_are_rejected_without_a_gpu():
+    lib = binding.load()
+    assert lib.lora_plan_create(None, 0, None) == binding.LORA_ERR_INVALID_ARG
+    assert lib.lora_plan_destroy(None) == binding.LORA_ERR_INVALID_ARG
+    assert lib.lora_linear_fwd(None, None, None, None, None, 1.0, None, None) == binding.LORA_ERR_INVALID_ARG
+    assert lib.lora_linear_bwd(None, None, None, None, None, None, 1.0, None, None, None, None) == \
+        binding.LORA_ERR_INVALID_ARG
+    assert lib.lora_select_config(None, 148, None) == binding.LORA_ERR_INVALID_ARG
+    out = ctypes.c_size_t(0)
+    s = binding.LoraShape(128, 64, 64, 16)
+    assert lib.lora_step_host_staging_bytes(ctypes.byref(s), ctypes.byref(out)) == 0
+    assert out.value >= 2 * 128 * 64 * 2 * 2
+
+
+def test_plan_creation_fails_loudly_without_a_device():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    lib = binding.load()
+    h = ctypes.c_void_p(0)
+    s = binding.LoraShape(128, 64, 64, 16)
+    assert lib.lora_plan_create(ctypes.byref(s), 0, ctypes.byref(h)) == binding.LORA_ERR_NO_DEVICE
+    assert not h.value
+    with pytest.raises(binding.LoraError):
+        binding.LoraLinearPlan(128, 64, 64, 16)
