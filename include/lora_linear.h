@@ -116,6 +116,18 @@ int lora_linear_fwd(lora_plan_t* plan, const void* X, const void* W, const void*
 int lora_linear_bwd(lora_plan_t* plan, const void* dY, const void* X, const void* W, const void* A,
                     const void* B, float scale, void* dX, void* dA, void* dB, void* stream);
 
+/* The three stages of lora_linear_bwd as separate calls, for callers that schedule them themselves.
+ * They communicate through the plan's workspace and must run in this order on one stream (or with
+ * equivalent event dependencies):
+ *   lora_linear_bwd_dx   dX = dY W + scale (dY B) A ; leaves scale (dY B)^T in the workspace
+ *   lora_linear_bwd_da   dA = scale (dY B)^T X, streams X once ; leaves scale (X A^T)^T in the workspace
+ *   lora_linear_bwd_db   dB = scale dY^T (X A^T), streams dY once
+ * `scale` must be the same in all three. */
+int lora_linear_bwd_dx(lora_plan_t* plan, const void* dY, const void* W, const void* A, const void* B,
+                       float scale, void* dX, void* stream);
+int lora_linear_bwd_da(lora_plan_t* plan, const void* X, const void* A, float scale, void* dA, void* stream);
+int lora_linear_bwd_db(lora_plan_t* plan, const void* dY, float scale, void* dB, void* stream);
+
 /* One training step of the layer with HOST input/output buffers: copies h_X, h_A, h_B, h_dY to the
  * device staging area, runs forward and backward, copies Y, dX, dA, dB back, all on `stream`
  * (asynchronous when the host buffers are pinned).  W is the frozen weight and stays resident on

@@ -26,7 +26,8 @@ LORA_ERR_NO_DEVICE = -7
 EXPORTS = [
     "lora_select_config", "lora_workspace_bytes", "lora_plan_create", "lora_plan_destroy",
     "lora_plan_workspace_bytes", "lora_plan_set_workspace", "lora_plan_get_config", "lora_plan_describe",
-    "lora_linear_fwd", "lora_linear_bwd", "lora_step_host_staging_bytes", "lora_linear_step_host",
+    "lora_linear_fwd", "lora_linear_bwd", "lora_linear_bwd_dx", "lora_linear_bwd_da", "lora_linear_bwd_db",
+    "lora_step_host_staging_bytes", "lora_linear_step_host",
     "lora_last_device_status", "lora_strerror", "lora_launch_count",
 ]
 
@@ -73,6 +74,9 @@ def load(rebuild: bool = False) -> ctypes.CDLL:
     lib.lora_plan_describe.argtypes = [vp, ctypes.c_char_p, ctypes.c_size_t]
     lib.lora_linear_fwd.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp]
     lib.lora_linear_bwd.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
+    lib.lora_linear_bwd_dx.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp]
+    lib.lora_linear_bwd_da.argtypes = [vp, vp, vp, ctypes.c_float, vp, vp]
+    lib.lora_linear_bwd_db.argtypes = [vp, vp, ctypes.c_float, vp, vp]
     lib.lora_step_host_staging_bytes.argtypes = [ctypes.POINTER(LoraShape), sz_p]
     lib.lora_linear_step_host.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp,
                                           ctypes.c_size_t, vp]
@@ -226,6 +230,26 @@ class LoraLinearPlan:
         self.ensure_workspace()
         _check(self._lib.lora_linear_bwd(self._h, _ptr(dY), _ptr(X), _ptr(W), _ptr(A), _ptr(B), float(scale),
                                          _ptr(dX), _ptr(dA), _ptr(dB), _stream_ptr(stream)), "lora_linear_bwd")
+        return dX, dA, dB
+
+    def bwd_stages(self, dY, X, W, A, B, scale: float, dX, dA, dB, stream=None, events=None):
+        """The same three kernels as ``bwd``, issued through the stage entry points; ``events`` (four
+        torch.cuda.Event, optional) are recorded before, between and after them on the stream."""
+        self.ensure_workspace()
+        sp = _stream_ptr(stream)
+        st = stream if stream is not None else torch.cuda.current_stream()
+        if events is not None:
+            events[0].record(st)
+        _check(self._lib.lora_linear_bwd_dx(self._h, _ptr(dY), _ptr(W), _ptr(A), _ptr(B), float(scale), _ptr(dX), sp),
+               "lora_linear_bwd_dx")
+        if events is not None:
+            events[1].record(st)
+        _check(self._lib.lora_linear_bwd_da(self._h, _ptr(X), _ptr(A), float(scale), _ptr(dA), sp), "lora_linear_bwd_da")
+        if events is not None:
+            events[2].record(st)
+        _check(self._lib.lora_linear_bwd_db(self._h, _ptr(dY), float(scale), _ptr(dB), sp), "lora_linear_bwd_db")
+        if events is not None:
+            events[3].record(st)
         return dX, dA, dB
 
     # -- host-buffer step (end-to-end measurement and host callers) ------------------------------

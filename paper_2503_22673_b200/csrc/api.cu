@@ -242,17 +242,30 @@ int launch_fwd(lora_plan* pl, const void* X, const void* W, const void* A, const
   return LORA_OK;
 }
 
-int launch_bwd(lora_plan* pl, const void* dY, const void* X, const void* W, const void* A, const void* B, float scale,
-               void* dX, void* dA, void* dB, cudaStream_t st) {
+struct WsPtrs {
+  uint8_t* base;
+  __nv_bfloat16 *qt, *pt;
+  unsigned* counters;
+};
+
+WsPtrs ws_ptrs(lora_plan* pl) {
+  WsPtrs q;
+  q.base = static_cast<uint8_t*>(pl->workspace);
+  q.qt = reinterpret_cast<__nv_bfloat16*>(q.base + pl->ws.qt);
+  q.pt = reinterpret_cast<__nv_bfloat16*>(q.base + pl->ws.pt);
+  q.counters = reinterpret_cast<unsigned*>(q.base + pl->ws.counters);
+  return q;
+}
+
+// ---- dX = dY W + s (dY B) A ; also leaves Qt = s (dY B)^T in the workspace and clears the counters ----
+int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const void* B, float scale, void* dX,
+              cudaStream_t st) {
   const lora_shape_t& s = pl->shape;
   const lora_kernel_config_t& c = pl->cfg;
   const WsLayout& w = pl->ws;
-  uint8_t* ws = static_cast<uint8_t*>(pl->workspace);
-  __nv_bfloat16* qt = reinterpret_cast<__nv_bfloat16*>(ws + w.qt);
-  __nv_bfloat16* pt = reinterpret_cast<__nv_bfloat16*>(ws + w.pt);
-  unsigned* counters = reinterpret_cast<unsigned*>(ws + w.counters);
-
-  // ---- dX = dY W + s (dY B) A ; also leaves Qt = s (dY B)^T in the workspace ----
+  const WsPtrs q = ws_ptrs(pl);
+  __nv_bfloat16* qt = q.qt;
+  unsigned* counters = q.counters;
   {
     CUtensorMap tmdY, tmW, tmB, tmA, tmdX;
     bool ok = make_bf16_tmap(&tmdY, dY, s.d_out, s.T, s.d_out, 64, kBlockM);
@@ -283,7 +296,18 @@ int launch_bwd(lora_plan* pl, const void* dY, const void* X, const void* W, cons
     if (launch_gemm_dx(tmdY, tmW, tmB, tmA, tmdX, p, c.dx_ctas, st) != cudaSuccess) return LORA_ERR_CUDA;
     g_launches.fetch_add(1);
   }
-  // ---- dA = Qt-contraction over X; recomputes X A^T and leaves Pt = s (X A^T)^T ----
+  return LORA_OK;
+}
+
+// ---- dA = Qt-contraction over X; recomputes X A^T and leaves Pt = s (X A^T)^T ----
+int launch_da(lora_plan* pl, const void* X, const void* A, float scale, void* dA, cudaStream_t st) {
+  const lora_shape_t& s = pl->shape;
+  const lora_kernel_config_t& c = pl->cfg;
+  const WsLayout& w = pl->ws;
+  const WsPtrs q = ws_ptrs(pl);
+  uint8_t* ws = q.base;
+  __nv_bfloat16 *qt = q.qt, *pt = q.pt;
+  unsigned* counters = q.counters;
   {
     CUtensorMap tmS, tmR, tmA;
     bool ok = make_bf16_tmap(&tmS, X, s.d_in, s.T, s.d_in, 64, kGradSlab);
@@ -317,7 +341,18 @@ int launch_bwd(lora_plan* pl, const void* dY, const void* X, const void* W, cons
     if (launch_grad(tmS, tmR, tmA, g, st) != cudaSuccess) return LORA_ERR_CUDA;
     g_launches.fetch_add(1);
   }
-  // ---- dB = Pt-contraction over dY ----
+  return LORA_OK;
+}
+
+// ---- dB = Pt-contraction over dY ----
+int launch_db(lora_plan* pl, const void* dY, float scale, void* dB, cudaStream_t st) {
+  const lora_shape_t& s = pl->shape;
+  const lora_kernel_config_t& c = pl->cfg;
+  const WsLayout& w = pl->ws;
+  const WsPtrs q = ws_ptrs(pl);
+  uint8_t* ws = q.base;
+  __nv_bfloat16* pt = q.pt;
+  unsigned* counters = q.counters;
   {
     CUtensorMap tmS, tmR;
     bool ok = make_bf16_tmap(&tmS, dY, s.d_out, s.T, s.d_out, 64, kGradSlab);
@@ -486,7 +521,47 @@ int lora_linear_bwd(lora_plan_t* plan, const void* dY, const void* X, const void
   if (!aligned16(dY) || !aligned16(X) || !aligned16(W) || !aligned16(A) || !aligned16(B) || !aligned16(dX))
     return LORA_ERR_MISALIGNED;
   if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
-  return launch_bwd(plan, dY, X, W, A, B, scale, dX, dA, dB, st);
+  int rc = launch_dx(plan, dY, W, A, B, scale, dX, st);
+  if (rc == LORA_OK) rc = launch_da(plan, X, A, scale, dA, st);
+  if (rc == LORA_OK) rc = launch_db(plan, dY, scale, dB, st);
+  return rc;
+}
+
+int lora_linear_bwd_dx(lora_plan_t* plan, const void* dY, const void* W, const void* A, const void* B, float scale,
+                       void* dX, void* stream) {
+  if (plan == nullptr) return LORA_ERR_INVALID_ARG;
+  if (plan->shape.T == 0) return LORA_OK;
+  if (!dY || !W || !A || !B || !dX) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(dY) || !aligned16(W) || !aligned16(A) || !aligned16(B) || !aligned16(dX)) return LORA_ERR_MISALIGNED;
+  if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
+  DeviceGuard guard(plan->device);
+  return launch_dx(plan, dY, W, A, B, scale, dX, static_cast<cudaStream_t>(stream));
+}
+
+int lora_linear_bwd_da(lora_plan_t* plan, const void* X, const void* A, float scale, void* dA, void* stream) {
+  if (plan == nullptr || !dA) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(dA)) return LORA_ERR_MISALIGNED;
+  DeviceGuard guard(plan->device);
+  if (plan->shape.T == 0)
+    return cudaMemsetAsync(dA, 0, sizeof(float) * plan->shape.r * plan->shape.d_in, static_cast<cudaStream_t>(stream)) ==
+                   cudaSuccess ? LORA_OK : LORA_ERR_CUDA;
+  if (!X || !A) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(A)) return LORA_ERR_MISALIGNED;
+  if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
+  return launch_da(plan, X, A, scale, dA, static_cast<cudaStream_t>(stream));
+}
+
+int lora_linear_bwd_db(lora_plan_t* plan, const void* dY, float scale, void* dB, void* stream) {
+  if (plan == nullptr || !dB) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(dB)) return LORA_ERR_MISALIGNED;
+  DeviceGuard guard(plan->device);
+  if (plan->shape.T == 0)
+    return cudaMemsetAsync(dB, 0, sizeof(float) * plan->shape.d_out * plan->shape.r, static_cast<cudaStream_t>(stream)) ==
+                   cudaSuccess ? LORA_OK : LORA_ERR_CUDA;
+  if (!dY) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(dY)) return LORA_ERR_MISALIGNED;
+  if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
+  return launch_db(plan, dY, scale, dB, static_cast<cudaStream_t>(stream));
 }
 
 int lora_step_host_staging_bytes(const lora_shape_t* shape, size_t* bytes) {
