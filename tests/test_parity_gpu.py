@@ -1,0 +1,255 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs.
+
+Tolerances (stated for the layer's outputs): max|gpu - ref| / max|ref| <= 2e-2 for the bf16 outputs Y and dX,
+<= 5e-3 for the fp32 adapter gradients dA and dB.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import lora_oracle as oracle
+from paper_2503_22673_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 2e-2
+TOL_F32 = 5e-3
+
+
+def dev(bits: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).cuda()
+
+
+def host64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def guarded(shape, dtype, guard_elems=2048):
+    """An output tensor carved out of a larger NaN-poisoned buffer, to catch stray writes."""
+    n = int(np.prod(shape))
+    buf = torch.full((n + 2 * guard_elems,), float("nan"), dtype=dtype, device="cuda")
+    return buf, buf[guard_elems:guard_elems + n].view(*shape)
+
+
+def guards_intact(buf, n, guard_elems=2048):
+    return bool(torch.isnan(buf[:guard_elems]).all() and torch.isnan(buf[guard_elems + n:]).all())
+
+
+def run_layer(p, t):
+    d = {k: dev(v) for k, v in t.items()}
+    plan = binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r)
+    bufs = {}
+    out = {}
+    for name, shape, dt in (("Y", (p.T, p.d_out), torch.bfloat16), ("dX", (p.T, p.d_in), torch.bfloat16),
+                            ("dA", (p.r, p.d_in), torch.float32), ("dB", (p.d_out, p.r), torch.float32)):
+        bufs[name], out[name] = guarded(shape, dt)
+    plan.fwd(d["X"], d["W"], d["A"], d["B"], p.scale, out["Y"])
+    plan.bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], p.scale, out["dX"], out["dA"], out["dB"])
+    code, msg = plan.device_status()
+    assert code == 0, msg
+    for name in out:
+        assert guards_intact(bufs[name], out[name].numel()), f"{name}: write outside the tensor"
+        assert not torch.isnan(out[name].float()).any(), f"{name}: element left unwritten"
+    plan.close()
+    return out
+
+
+def check_full(p, t):
+    out = run_layer(p, t)
+    f = {k: inputs.bf16_to_f64(v) for k, v in t.items()}
+    Y = oracle.forward(f["X"], f["W"], f["A"], f["B"], p.scale)
+    dX, dA, dB = oracle.backward(f["dY"], f["X"], f["W"], f["A"], f["B"], p.scale)
+    errs = {"Y": oracle.rel_err(host64(out["Y"]), Y), "dX": oracle.rel_err(host64(out["dX"]), dX),
+            "dA": oracle.rel_err(host64(out["dA"]), dA), "dB": oracle.rel_err(host64(out["dB"]), dB)}
+    assert errs["Y"] <= TOL_BF16 and errs["dX"] <= TOL_BF16, errs
+    assert errs["dA"] <= TOL_F32 and errs["dB"] <= TOL_F32, errs
+    return out, errs
+
+
+# ---------------------------------------------------------------------------------------------
+# small and ragged shapes, element by element
+# ---------------------------------------------------------------------------------------------
+SMALL = [
+    # T, d_in, d_out, r, scale      (tile rows 128/256; tile columns up to 240; k-blocks of 64; token slabs of 128)
+    (1, 8, 8, 8, 2.0),
+    (7, 72, 200, 8, 1.7),
+    (127, 520, 72, 16, 2.0),
+    (129, 200, 520, 24, 0.5),
+    (255, 1032, 264, 32, 1.7),
+    (257, 264, 1032, 48, 2.0),
+    (300, 520, 200, 64, 0.5),
+    (640, 768, 1160, 16, 2.0),        # several tiles per row and column, ragged last column tile
+    (1000, 2048, 512, 64, 0.5),       # r = 64 with a long contraction
+    (2100, 512, 3080, 32, 2.0),       # more tiles than CTAs on a 148-SM part: persistent loop + ragged tail
+    (4500, 1024, 4096, 16, 2.0),      # many tiles per persistent CTA
+]
+
+
+@pytest.mark.parametrize("T,d_in,d_out,r,scale", SMALL)
+def test_small_shapes_elementwise(T, d_in, d_out, r, scale):
+    p, t = inputs.draw_custom(T, d_in, d_out, r, scale, seed=3)
+    check_full(p, t)
+
+
+def test_tiny_workload_config0():
+    (p, t), = list(inputs.draw_workload(0, seed=0))
+    check_full(p, t)
+
+
+def test_paper_benchmark_adapter_setting_r32_alpha64():
+    # Section 4.5: q/k/v/o adapted with lora_r = 32, alpha = 64 (scale 2); reduced token count
+    for d_out in (4096, 1024):
+        p, t = inputs.draw_custom(512, 4096, d_out, 32, 2.0, seed=5)
+        check_full(p, t)
+
+
+# ---------------------------------------------------------------------------------------------
+# exact cases
+# ---------------------------------------------------------------------------------------------
+def _pad_example():
+    """The hand-derived rank-1 example (tests/golden/rank1_example.txt) zero-padded to the smallest
+    shape the kernels take (multiples of 8).  Every value is a small integer: results must be exact."""
+    from tests.test_oracle import GOLDEN, _read_golden
+    g = _read_golden(GOLDEN)
+    T, d_in, d_out, r = 2, 8, 8, 8
+
+    def pad(a, shape):
+        out = np.zeros(shape)
+        out[:a.shape[0], :a.shape[1]] = a
+        return out
+    t = {"X": pad(g["X"], (T, d_in)), "W": pad(g["W"], (d_out, d_in)), "A": pad(g["A"], (r, d_in)),
+         "B": pad(g["B"], (d_out, r)), "dY": pad(g["dY"], (T, d_out))}
+    want = {"Y": pad(g["Y"], (T, d_out)), "dX": pad(g["dX"], (T, d_in)), "dA": pad(g["dA"], (r, d_in)),
+            "dB": pad(g["dB"], (d_out, r))}
+    return float(g["s"][0, 0]), t, want
+
+
+def test_hand_derived_example_is_exact_on_gpu():
+    s, t, want = _pad_example()
+    p = inputs.Projection("rank1", 2, 8, 8, 8, s)
+    bits = {k: inputs.f32_to_bf16_bits(v.astype(np.float32)) for k, v in t.items()}
+    out = run_layer(p, bits)
+    for k in want:
+        assert np.array_equal(host64(out[k]), want[k]), k
+
+
+def test_closed_forms_zero_factors():
+    p, t = inputs.draw_custom(300, 264, 200, 16, 2.0, seed=7)
+    f = {k: inputs.bf16_to_f64(v) for k, v in t.items()}
+    # B = 0: Y = X W^T, dX = dY W, dA = 0 exactly
+    tb = dict(t, B=np.zeros_like(t["B"]))
+    out = run_layer(p, tb)
+    assert torch.count_nonzero(out["dA"]) == 0
+    assert oracle.rel_err(host64(out["Y"]), f["X"] @ f["W"].T) <= TOL_BF16
+    assert oracle.rel_err(host64(out["dX"]), f["dY"] @ f["W"]) <= TOL_BF16
+    _, _, dB = oracle.backward(f["dY"], f["X"], f["W"], f["A"], 0 * f["B"], p.scale)
+    assert oracle.rel_err(host64(out["dB"]), dB) <= TOL_F32
+    # the adapter path adds exactly +0: Y is bitwise what it is with A = 0 as well
+    ta = dict(t, A=np.zeros_like(t["A"]))
+    out_a = run_layer(p, ta)
+    assert torch.equal(out["Y"].view(torch.int16), out_a["Y"].view(torch.int16))
+    assert torch.count_nonzero(out_a["dB"]) == 0
+    # W = 0: only the rank-r path is left, at full scale
+    tw = dict(t, W=np.zeros_like(t["W"]))
+    out_w = run_layer(p, tw)
+    assert oracle.rel_err(host64(out_w["Y"]), p.scale * (f["X"] @ f["A"].T) @ f["B"].T) <= TOL_BF16
+    assert oracle.rel_err(host64(out_w["dX"]), p.scale * (f["dY"] @ f["B"]) @ f["A"]) <= TOL_BF16
+
+
+def test_linearity_in_scale():
+    p, t = inputs.draw_custom(256, 264, 136, 16, 1.0, seed=9)
+    outs = {}
+    for s in (0.0, 1.0, 1.7):
+        outs[s] = {k: host64(v) for k, v in run_layer(inputs.Projection("lin", 256, 264, 136, 16, s), t).items()}
+    assert np.count_nonzero(outs[0.0]["dA"]) == 0 and np.count_nonzero(outs[0.0]["dB"]) == 0
+    for k in ("dA", "dB"):
+        assert oracle.rel_err(outs[1.7][k], 1.7 * outs[1.0][k]) <= TOL_F32
+    for k in ("Y", "dX"):
+        lhs = outs[1.7][k] - outs[0.0][k]
+        rhs = 1.7 * (outs[1.0][k] - outs[0.0][k])
+        assert np.max(np.abs(lhs - rhs)) <= 2 * TOL_BF16 * np.max(np.abs(outs[1.7][k]))
+
+
+def test_bitwise_reproducible():
+    p, t = inputs.draw_custom(1500, 1032, 776, 16, 2.0, seed=11)
+    a = run_layer(p, t)
+    b = run_layer(p, t)
+    for k in a:
+        it = torch.int32 if a[k].dtype == torch.float32 else torch.int16
+        assert torch.equal(a[k].view(it), b[k].view(it)), k
+
+
+def test_stage_entry_points_match_the_single_call():
+    p, t = inputs.draw_custom(700, 520, 392, 16, 2.0, seed=13)
+    d = {k: dev(v) for k, v in t.items()}
+    plan = binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r)
+    dX1, dA1, dB1 = plan.bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], p.scale)
+    dX2, dA2, dB2 = torch.empty_like(dX1), torch.empty_like(dA1), torch.empty_like(dB1)
+    plan.bwd_stages(d["dY"], d["X"], d["W"], d["A"], d["B"], p.scale, dX2, dA2, dB2)
+    torch.cuda.synchronize()
+    assert torch.equal(dX1.view(torch.int16), dX2.view(torch.int16))
+    assert torch.equal(dA1, dA2) and torch.equal(dB1, dB2)
+    plan.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# argument handling on a device
+# ---------------------------------------------------------------------------------------------
+def test_empty_batch_and_argument_errors():
+    plan = binding.LoraLinearPlan(0, 64, 72, 16)
+    bf = torch.bfloat16
+    X = torch.empty(0, 64, dtype=bf, device="cuda")
+    W = torch.zeros(72, 64, dtype=bf, device="cuda")
+    A = torch.zeros(16, 64, dtype=bf, device="cuda")
+    B = torch.zeros(72, 16, dtype=bf, device="cuda")
+    dY = torch.empty(0, 72, dtype=bf, device="cuda")
+    assert plan.fwd(X, W, A, B, 2.0).shape == (0, 72)
+    dX, dA, dB = plan.bwd(dY, X, W, A, B, 2.0,
+                          dA=torch.full((16, 64), 3.0, device="cuda"), dB=torch.full((72, 16), 3.0, device="cuda"))
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(dA) == 0 and torch.count_nonzero(dB) == 0
+    plan.close()
+
+    plan = binding.LoraLinearPlan(128, 64, 72, 16)
+    X = torch.zeros(128, 64, dtype=bf, device="cuda")
+    dY = torch.zeros(128, 72, dtype=bf, device="cuda")
+    lib = binding.load()
+    Y = torch.zeros(128 * 72 + 8, dtype=bf, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    # misaligned output pointer
+    rc = lib.lora_linear_fwd(plan._h, X.data_ptr(), W.data_ptr(), A.data_ptr(), B.data_ptr(), 2.0, Y.data_ptr() + 2, stream)
+    assert rc == binding.LORA_ERR_MISALIGNED
+    rc = lib.lora_linear_fwd(plan._h, X.data_ptr(), None, A.data_ptr(), B.data_ptr(), 2.0, Y.data_ptr(), stream)
+    assert rc == binding.LORA_ERR_INVALID_ARG
+    # backward without a workspace
+    dXb = torch.zeros(128, 64, dtype=bf, device="cuda")
+    dAb = torch.zeros(16, 64, device="cuda")
+    dBb = torch.zeros(72, 16, device="cuda")
+    rc = lib.lora_linear_bwd(plan._h, dY.data_ptr(), X.data_ptr(), W.data_ptr(), A.data_ptr(), B.data_ptr(), 2.0,
+                             dXb.data_ptr(), dAb.data_ptr(), dBb.data_ptr(), stream)
+    assert rc == binding.LORA_ERR_WORKSPACE
+    small = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.LoraError) as ei:
+        plan.set_workspace(small)
+    assert ei.value.code == binding.LORA_ERR_WORKSPACE
+    assert "T=128" in plan.describe()
+    assert plan.device_status()[0] == 0
+    plan.close()
+
+
+def test_host_buffer_step_matches_device_calls():
+    p, t = inputs.draw_custom(384, 264, 200, 16, 2.0, seed=17)
+    d = {k: dev(v) for k, v in t.items()}
+    plan = binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r)
+    Y = plan.fwd(d["X"], d["W"], d["A"], d["B"], p.scale)
+    dX, dA, dB = plan.bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], p.scale)
+    h = {k: d[k].cpu().pin_memory() for k in ("X", "A", "B", "dY")}
+    hY, hdX = torch.empty_like(Y, device="cpu").pin_memory(), torch.empty_like(dX, device="cpu").pin_memory()
+    hdA, hdB = torch.empty_like(dA, device="cpu").pin_memory(), torch.empty_like(dB, device="cpu").pin_memory()
+    staging = torch.empty(plan.step_host_staging_bytes(), dtype=torch.uint8, device="cuda")
+    plan.step_host(h["X"], d["W"], h["A"], h["B"], h["dY"], p.scale, hY, hdX, hdA, hdB, staging)
+    torch.cuda.synchronize()
+    assert torch.equal(hY.view(torch.int16), Y.cpu().view(torch.int16))
+    assert torch.equal(hdX.view(torch.int16), dX.cpu().view(torch.int16))
+    assert torch.equal(hdA, dA.cpu()) and torch.equal(hdB, dB.cpu())
+    plan.close()
