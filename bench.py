@@ -1,0 +1,383 @@
+#!/usr/bin/env python
+"""Throughput of the LoRA projection layer (forward + backward) on B200.
+
+A step is one pass of the whole hot path - forward GEMM with the fused adapter, dX GEMM with the fused
+adapter, dA kernel, dB kernel - over one batch of seeded synthetic input.  The default workload is the
+Llama-3-8B q_proj shape (T = 8192 packed tokens, 4096 -> 4096, r = 16, s = 2).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload {0..4}] [--impl reference]
+
+Prints ONE JSON line.  With N > 1 (torchrun, one rank per GPU) every rank runs an independent replica
+on its own batch: the layer has no collective, so the job's value is the sum over ranks divided by the
+slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+L2_BYTES = 126 * 1024 * 1024
+METRIC = "lora_linear_fwd_bwd_tflops"
+UNIT = "TFLOP/s"
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel from an
+# ncu capture summarised under profiles/; only valid for the kernel source it was taken on.
+NCU_TRAFFIC = {"gemm_sha": None, "bytes_per_launch": None}
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            m = json.load(f)
+        return {"hbm_gbs": float(m["hbm_gbs"]), "bf16_tflops": float(m["bf16_tflops"]),
+                "bf16_tflops_sustained": float(m.get("bf16_tflops_sustained", m["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def gemm_source_sha() -> str:
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2503_22673_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        if name.startswith("gemm") or name in ("sm100_ptx.cuh", "kernels.h"):
+            with open(os.path.join(csrc, name), "rb") as f:
+                h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def workload_name(idx: int) -> str:
+    return {0: "config0 tiny T=256 512->512 r8 s2", 1: "config1 q_proj T=8192 4096->4096 r16 s2",
+            2: "config2 gate/up_proj T=16384 4096->14336 r16 s2", 3: "config3 down_proj T=16384 14336->4096 r64 s0.5",
+            4: "config4 seven Llama-3-8B projections T=32768 r16 s2"}[idx]
+
+
+# ----------------------------------------------------------------------------------------------------
+# CPU oracle timing (reported baseline; also the --impl reference arm)
+# ----------------------------------------------------------------------------------------------------
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 0) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+
+
+def oracle_step_time(proj, f64, rows: int) -> float:
+    """One oracle forward + backward on the first `rows` token rows (all of W, A, B)."""
+    from oracle import lora_oracle as oracle
+    X, dY = f64["X"][:rows], f64["dY"][:rows]
+    t0 = time.perf_counter()
+    oracle.forward(X, f64["W"], f64["A"], f64["B"], proj.scale)
+    oracle.backward(dY, X, f64["W"], f64["A"], f64["B"], proj.scale)
+    return time.perf_counter() - t0
+
+
+def sample_flops(proj, rows: int) -> float:
+    return 4.0 * rows * proj.d_in * proj.d_out + 6.0 * rows * proj.r * (proj.d_in + proj.d_out)
+
+
+def oracle_inputs(workload_idx: int, max_rows: int):
+    from paper_2503_22673_b200 import inputs
+    proto = inputs.workload(workload_idx)[0]
+    rows = min(proto.T, max_rows)
+    proj, t = next(iter(inputs.draw_workload(workload_idx, seed=0, T=rows)))
+    f64 = {k: inputs.bf16_to_f64(v) for k, v in t.items()}
+    return proto, proj, f64, rows
+
+
+def pick_rows(proj, f64, avail: int, budget_s: float) -> int:
+    cal = min(avail, 128)
+    t_cal = oracle_step_time(proj, f64, cal)              # calibration (also warms the BLAS pool)
+    t_cal = min(t_cal, oracle_step_time(proj, f64, cal))
+    rows = int(budget_s / max(t_cal / cal, 1e-9))
+    rows = min(avail, max(cal, rows - rows % 128))
+    return rows
+
+
+def cpu_baseline(workload_idx: int, budget_s: float = 12.0):
+    proto, proj, f64, avail = oracle_inputs(workload_idx, 4096)
+    rows = pick_rows(proj, f64, avail, budget_s)
+    t = oracle_step_time(proj, f64, rows)
+    return {"value": sample_flops(proto, rows) / t / 1e12, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+            "sample": f"{proto.name}: {rows} of {proto.T} token rows, full W/A/B, fp64 numpy, one fwd+bwd in {t:.2f} s",
+            "tokens_per_s": rows / t}
+
+
+def run_reference(args):
+    rank, _, _ = dist_env()
+    if rank != 0:
+        return
+    proto, proj, f64, avail = oracle_inputs(args.workload, 4096)
+    total_steps = max(args.steps + args.warmup, 1)
+    rows = pick_rows(proj, f64, avail, min(3.0, 100.0 / total_steps))
+    for _ in range(args.warmup):
+        oracle_step_time(proj, f64, rows)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step_time(proj, f64, rows)
+    dt = time.perf_counter() - t0
+    value = sample_flops(proto, rows) * args.steps / dt / 1e12
+    sample = f"{proto.name}: {rows} of {proto.T} token rows per step, full W/A/B, fp64 numpy"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / max(args.steps, 1) * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(args.workload), "T": proto.T, "d_in": proto.d_in, "d_out": proto.d_out,
+                   "r": proto.r, "scale": proto.scale, "sampled_rows_per_step": rows},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "tokens_per_s": rows * args.steps / dt, "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------------------
+# CUDA path
+# ----------------------------------------------------------------------------------------------------
+def to_dev(bits: np.ndarray, device) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).to(device)
+
+
+def run_ours(args):
+    from paper_2503_22673_b200 import binding, inputs
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device - the layer has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    pk = peaks()
+
+    # ---- inputs: n_sets independent seeded batches, rotated so that no step finds its operands in L2 ----
+    protos = inputs.workload(args.workload)
+    bytes_per_set = sum(2 * (p.T * p.d_in * 2 + p.T * p.d_out * 2) + 2 * p.d_out * p.d_in for p in protos)
+    n_sets = max(2, min(6, -(-4 * L2_BYTES // bytes_per_set)))
+    if args.workload == 4:
+        n_sets = 2
+    sets = []
+    for s_i in range(n_sets):
+        cur = []
+        for proj, t in inputs.draw_workload(args.workload, seed=1000 * rank + s_i):
+            d = {k: to_dev(v, device) for k, v in t.items()}
+            d["Y"] = torch.empty((proj.T, proj.d_out), dtype=torch.bfloat16, device=device)
+            d["dX"] = torch.empty((proj.T, proj.d_in), dtype=torch.bfloat16, device=device)
+            d["dA"] = torch.empty((proj.r, proj.d_in), dtype=torch.float32, device=device)
+            d["dB"] = torch.empty((proj.d_out, proj.r), dtype=torch.float32, device=device)
+            cur.append((proj, d))
+        sets.append(cur)
+    plans = [binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r, device=local_rank) for p in protos]
+    for pl in plans:
+        pl.ensure_workspace()
+    flops_step = float(sum(p.flops for p in protos))
+    tokens_step = protos[0].T
+
+    def step(k, events=None):
+        cur = sets[k % n_sets]
+        for j, (proj, d) in enumerate(cur):
+            ev = events[j] if events is not None else None
+            if ev is not None:
+                ev[0].record()
+            plans[j].fwd(d["X"], d["W"], d["A"], d["B"], proj.scale, d["Y"])
+            plans[j].bwd_stages(d["dY"], d["X"], d["W"], d["A"], d["B"], proj.scale, d["dX"], d["dA"], d["dB"],
+                                events=ev[1:] if ev is not None else None)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+
+    n_warm = max(args.warmup, 3)
+    for k in range(n_warm):
+        step(k)
+    torch.cuda.synchronize()
+    for pl in plans:
+        code, msg = pl.device_status()
+        if code != 0:
+            raise SystemExit(f"bench.py: device status after warm-up: {msg}")
+
+    # ---- timed region: K steps, device-timed, per-kernel events inside ----
+    events = [[[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in protos] for _ in range(args.steps)]
+    ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    launches0 = binding.launch_count()
+    barrier()
+    torch.cuda.synchronize()
+    ev_a.record()
+    for k in range(args.steps):
+        step(n_warm + k, events[k])
+    ev_b.record()
+    torch.cuda.synchronize()
+    barrier()
+    launches = binding.launch_count() - launches0
+    clocks = sampler.stop() if sampler is not None else None
+    ms_total = ev_a.elapsed_time(ev_b)
+    if world > 1:
+        import torch.distributed as dist
+        tmax = torch.tensor([ms_total], device=device)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms_total = float(tmax.item())
+    ms_step = ms_total / args.steps
+
+    # per-kernel mean durations (ms) and rooflines
+    kern = {}
+    for j, p in enumerate(protos):
+        dur = [statistics.mean(events[k][j][i].elapsed_time(events[k][j][i + 1]) for k in range(args.steps)) for i in range(4)]
+        gemm_flops = 2.0 * p.T * p.d_in * p.d_out + 2.0 * p.T * p.r * (p.d_in + p.d_out)
+        da_bytes = 2.0 * p.T * p.d_in + 2.0 * p.T * p.r * 2 + 4.0 * p.r * p.d_in      # X once, Qt in, Pt out, dA out
+        db_bytes = 2.0 * p.T * p.d_out + 2.0 * p.T * p.r + 4.0 * p.r * p.d_out        # dY once, Pt in, dB out
+        kern[p.name] = {
+            "fwd_gemm": {"ms": dur[0], "tflops": gemm_flops / dur[0] / 1e9,
+                         "frac_of_bf16_peak": gemm_flops / dur[0] / 1e9 / pk["bf16_tflops"]},
+            "dx_gemm": {"ms": dur[1], "tflops": gemm_flops / dur[1] / 1e9,
+                        "frac_of_bf16_peak": gemm_flops / dur[1] / 1e9 / pk["bf16_tflops"]},
+            "dA": {"ms": dur[2], "gbs": da_bytes / dur[2] / 1e6, "frac_of_hbm_peak": da_bytes / dur[2] / 1e6 / pk["hbm_gbs"]},
+            "dB": {"ms": dur[3], "gbs": db_bytes / dur[3] / 1e6, "frac_of_hbm_peak": db_bytes / dur[3] / 1e6 / pk["hbm_gbs"]},
+        }
+    dom_p = max(protos, key=lambda p: max(kern[p.name]["fwd_gemm"]["ms"], kern[p.name]["dx_gemm"]["ms"]))
+    dom_k = "dx_gemm" if kern[dom_p.name]["dx_gemm"]["ms"] >= kern[dom_p.name]["fwd_gemm"]["ms"] else "fwd_gemm"
+    dom = kern[dom_p.name][dom_k]
+    roofline = {"bound": "tensor", "kernel": f"lora GEMM, {'dX' if dom_k == 'dx_gemm' else 'forward'} ({dom_p.name})",
+                "achieved": dom["tflops"], "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": dom["tflops"] / pk["bf16_tflops"], "peak_kind": f"bf16 burst, of {pk['source']}",
+                "ms_per_launch": dom["ms"],
+                "traffic": NCU_TRAFFIC["bytes_per_launch"] if NCU_TRAFFIC["gemm_sha"] == gemm_source_sha() else None}
+
+    # ---- end to end: host buffers through the C ABI, copies inside the timed region ----
+    h_sets, staging = [], []
+    for j, (p, d0) in enumerate(sets[0]):
+        h = {k: d0[k].cpu().pin_memory() for k in ("X", "A", "B", "dY")}
+        ho = {k: torch.empty_like(d0[k], device="cpu").pin_memory() for k in ("Y", "dX", "dA", "dB")}
+        h_sets.append((h, ho))
+        staging.append(torch.empty(plans[j].step_host_staging_bytes(), dtype=torch.uint8, device=device))
+
+    def step_host():
+        for j, (p, d0) in enumerate(sets[0]):
+            h, ho = h_sets[j]
+            plans[j].step_host(h["X"], d0["W"], h["A"], h["B"], h["dY"], p.scale, ho["Y"], ho["dX"], ho["dA"], ho["dB"],
+                               staging[j])
+
+    n_e2e = max(3, min(args.steps, 10 if args.workload != 4 else 3))
+    for _ in range(2):
+        step_host()
+    torch.cuda.synchronize()
+    e_a, e_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e_a.record()
+    for _ in range(n_e2e):
+        step_host()
+    e_b.record()
+    torch.cuda.synchronize()
+    barrier()
+    ms_e2e = e_a.elapsed_time(e_b) / n_e2e
+    if world > 1:
+        import torch.distributed as dist
+        tm = torch.tensor([ms_e2e], device=device)
+        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+        ms_e2e = float(tm.item())
+    h2d = sum(t.numel() * t.element_size() for h, _ in h_sets for t in h.values())
+    d2h = sum(t.numel() * t.element_size() for _, ho in h_sets for t in ho.values())
+    e2e = {"value": world * flops_step / ms_e2e / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+           "ms_per_step": ms_e2e, "steps": n_e2e,
+           "note": "host X, A, B, dY in; Y, dX, dA, dB out (pinned); frozen W resident on the device"}
+
+    if rank != 0:
+        return
+    cpu = cpu_baseline(args.workload) if world == 1 and not args.no_cpu_baseline else None
+    value = world * flops_step / ms_step / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": n_warm,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": workload_name(args.workload), "projections": [p.name for p in protos], "T": protos[0].T,
+                   "r": protos[0].r, "scale": protos[0].scale, "input_sets_rotated": n_sets,
+                   "l2": f"{n_sets} independent input/output sets ({bytes_per_set * n_sets / 2**20:.0f} MiB) rotated per step; "
+                         "each step's operands exceed the 126 MB L2",
+                   "replicas": "independent replica per GPU, no collective"},
+        "tokens_per_s": world * tokens_step / ms_step * 1e3,
+        "frac_of_bf16_peak": value / world / pk["bf16_tflops"], "peak_source": pk["source"],
+        "kernels": kern, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+        "plan": plans[0].describe(),
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", type=int, default=1)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
