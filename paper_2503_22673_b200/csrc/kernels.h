@@ -32,9 +32,27 @@ struct GemmParams {
   unsigned* status;       // device status word
   unsigned* zero_words;   // words this kernel clears for the kernels that follow it (may be null)
   int n_zero_words;
+  __nv_bfloat16* out;     // CTA-pair kernel only: output base and row pitch (elements) for the ragged last chunk
+  int ld_out;
 };
 
 size_t gemm_smem_bytes(int stages);
+
+// ---- CTA-pair (cta_group::2) variant: 256-row tiles, block_n a multiple of 16 with block_n + r_pad <= 256 ----
+constexpr int kPairBlockM = 256;
+constexpr int kPairStageBytesFwd = 32768;   // 128 x 64 activations + 128 x 64 weight/adapter rows per CTA
+constexpr int kPairStageBytesBwd = 36864;   // + up to 4 KiB of unswizzled B columns for the side product
+size_t gemm_pair_smem_bytes(bool bwd, int stages);
+cudaError_t gemm_pair_configure();
+// forward: tmW0 = W box 64 x half rows (leader CTA), tmW1 = W box 64 x (block_n - half) rows (peer CTA),
+// half = (block_n + r_pad) / 2; tmA box 64 x r_pad; tmB box 64 x block_n/2 rows
+cudaError_t launch_gemm_pair_fwd(const CUtensorMap& tmX, const CUtensorMap& tmW0, const CUtensorMap& tmW1,
+                                 const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
+                                 const GemmParams& p, int ctas, cudaStream_t stream);
+// backward: tmW box 64(n) x 64(k); tmB unswizzled box 8(r) x 64(k); tmA box 64(n) x r_pad
+cudaError_t launch_gemm_pair_dx(const CUtensorMap& tmdY, const CUtensorMap& tmW, const CUtensorMap& tmB,
+                                const CUtensorMap& tmA, const CUtensorMap& tmdX, const GemmParams& p, int ctas,
+                                cudaStream_t stream);
 
 // Y / dX = act * Wop + scale * (act * sideop) * tailop, see gemm_lora.cu
 cudaError_t launch_gemm_fwd(const CUtensorMap& tmX, const CUtensorMap& tmW, const CUtensorMap& tmA,
