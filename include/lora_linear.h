@@ -137,6 +137,30 @@ int lora_linear_step_host(lora_plan_t* plan, const void* h_X, const void* W, con
                           const void* h_B, const void* h_dY, float scale, void* h_Y, void* h_dX,
                           void* h_dA, void* h_dB, void* staging, size_t staging_bytes, void* stream);
 
+/* Token contraction without any allocation (the paper has no counterpart; this is a library convenience).
+ *
+ *     out[c, j] = sum_t S[t, c] * Rt[j, t]          S [T, C] bf16, Rt [r, ld_rt] bf16 (ld_rt >= T), out [C, r] fp32
+ *
+ * This is the kernel behind dB = scale dY^T (X A^T) with S = dY and Rt = the caller's bf16 copy of
+ * scale (X A^T)^T, usable on its own.  It is meant for callers that must not allocate device memory when
+ * they call in: code running under a memory pool that forbids cudaMalloc after start-up, real-time or
+ * inference loops where an allocation would stall the device, and hosts that hand this library a fixed
+ * memory budget.  No plan is needed (creating one allocates a status block).  Nothing in this call
+ * allocates or frees: the partial sums, arrival counters and status word live in one static device array
+ * of lora_grad_contract_noalloc_max_scratch() bytes (8 MiB) that every GPU loading the library holds until
+ * the process exits.
+ *   - Shapes whose partial sums do not fit (roughly SMs/ceil(C/512) x r_pad x C x 4 bytes > 8 MiB) are
+ *     rejected with LORA_ERR_WORKSPACE; C % 8 == 0, r in {8,...,64}, ld_rt % 8 == 0, T >= 1.
+ *   - The first call on a device looks up the array's device address and raises the kernel's shared-memory
+ *     limit; make that first call before any stream capture.  The current device is used.
+ *   - All calls share the one array and it keeps the last call's contents; the call clears the counters
+ *     it needs on `stream` first.  Two calls whose kernels overlap on the GPU (different streams, or
+ *     different host threads) race on it: serialise them.
+ *   - A bounded device wait that ran out is not reported by this call (there is no plan to ask). */
+int lora_grad_contract_noalloc(const void* S, const void* Rt, int64_t T, int64_t C, int64_t r, int64_t ld_rt,
+                               void* out, void* stream);
+int64_t lora_grad_contract_noalloc_max_scratch(void);
+
 /* Synchronise `stream`, then report whether any kernel of this plan gave up on a bounded wait.
  * *code is LORA_OK or LORA_ERR_DEVICE_TIMEOUT; msg (may be NULL) receives a short description.
  * The status word is cleared. */

@@ -29,6 +29,7 @@ EXPORTS = [
     "lora_linear_fwd", "lora_linear_bwd", "lora_linear_bwd_dx", "lora_linear_bwd_da", "lora_linear_bwd_db",
     "lora_step_host_staging_bytes", "lora_linear_step_host",
     "lora_last_device_status", "lora_strerror", "lora_launch_count",
+    "lora_grad_contract_noalloc", "lora_grad_contract_noalloc_max_scratch",
 ]
 
 
@@ -85,8 +86,11 @@ def load(rebuild: bool = False) -> ctypes.CDLL:
     lib.lora_strerror.restype = ctypes.c_char_p
     lib.lora_launch_count.argtypes = []
     lib.lora_launch_count.restype = i64
+    lib.lora_grad_contract_noalloc.argtypes = [vp, vp, i64, i64, i64, i64, vp, vp]
+    lib.lora_grad_contract_noalloc_max_scratch.argtypes = []
+    lib.lora_grad_contract_noalloc_max_scratch.restype = i64
     for name in EXPORTS:
-        if name not in ("lora_strerror", "lora_launch_count"):
+        if name not in ("lora_strerror", "lora_launch_count", "lora_grad_contract_noalloc_max_scratch"):
             getattr(lib, name).restype = ctypes.c_int
     _lib = lib
     return lib
@@ -277,3 +281,22 @@ def lora_linear_fwd(plan: LoraLinearPlan, X, W, A, B, scale, Y=None, stream=None
 
 def lora_linear_bwd(plan: LoraLinearPlan, dY, X, W, A, B, scale, dX=None, dA=None, dB=None, stream=None):
     return plan.bwd(dY, X, W, A, B, scale, dX, dA, dB, stream)
+
+
+def grad_contract_noalloc(S: torch.Tensor, Rt: torch.Tensor, out: torch.Tensor, stream=None) -> torch.Tensor:
+    """out[c, j] = sum_t S[t, c] * Rt[j, t] through the entry point that allocates nothing.
+
+    For callers that may not allocate device memory at call time (fixed memory pools, latency-critical
+    loops): the kernel's scratch is a static device array inside the library, so the caller passes only
+    the inputs S [T, C] bf16, Rt [r, ld] bf16 (ld >= T) and the output out [C, r] fp32.  Calls share that
+    array, so do not let two of them overlap on the GPU.
+    """
+    T, C = S.shape
+    r, ld = Rt.shape
+    if S.dtype != torch.bfloat16 or Rt.dtype != torch.bfloat16 or out.dtype != torch.float32:
+        raise ValueError("grad_contract_noalloc: S, Rt bf16 and out fp32 expected")
+    if not (S.is_contiguous() and Rt.is_contiguous() and out.is_contiguous()) or tuple(out.shape) != (C, r):
+        raise ValueError("grad_contract_noalloc: contiguous S [T,C], Rt [r,ld], out [C,r] expected")
+    _check(load().lora_grad_contract_noalloc(_ptr(S), _ptr(Rt), T, C, r, ld, _ptr(out), _stream_ptr(stream)),
+           "lora_grad_contract_noalloc")
+    return out

@@ -16,6 +16,10 @@
 #include "kernels.h"
 #include "sm100_ptx.cuh"
 
+#include <mutex>
+
+#include "../../include/lora_linear.h"
+
 namespace lora {
 
 namespace {
@@ -289,4 +293,137 @@ cudaError_t launch_grad(const CUtensorMap& tmS, const CUtensorMap& tmR, const CU
   return cudaGetLastError();
 }
 
+// ================================================================================================
+// No-allocation variant of the dB-style contraction: scratch lives in a static device array
+// ================================================================================================
+namespace {
+
+// Scratch held by every GPU that loads this library, until the process exits: one status block, the
+// arrival counters and the per-token-chunk partial sums of the contraction kernel.
+constexpr size_t kNoAllocScratchBytes = 8u << 20;
+constexpr size_t kNoAllocHeaderBytes = 4096;     // [0,256) status words, [256,4096) arrival counters
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+struct NoAllocDevice {
+  bool ready = false;
+  unsigned char* scratch = nullptr;   // device address of g_noalloc_scratch on this device
+  int num_sms = 0;
+};
+constexpr int kNoAllocMaxDevices = 64;
+NoAllocDevice g_noalloc_dev[kNoAllocMaxDevices];
+std::mutex g_noalloc_mutex;
+
+typedef CUresult (*NoAllocEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+bool noalloc_tmap(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t outer, uint64_t pitch_elems,
+                  uint32_t box_inner, uint32_t box_outer) {
+  static NoAllocEncodeFn fn = []() -> NoAllocEncodeFn {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess) return nullptr;
+    return q == cudaDriverEntryPointSuccess ? reinterpret_cast<NoAllocEncodeFn>(f) : nullptr;
+  }();
+  if (fn == nullptr) return false;
+  const cuuint64_t dims[2] = {inner, outer};
+  const cuuint64_t strides[1] = {pitch_elems * 2};
+  const cuuint32_t box[2] = {box_inner, box_outer};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
 }  // namespace lora
+
+extern "C" int lora_grad_contract_noalloc(const void* S, const void* Rt, int64_t T, int64_t C, int64_t r,
+                                          int64_t ld_rt, void* out, void* stream) {
+  using namespace lora;
+  if (!S || !Rt || !out) return LORA_ERR_INVALID_ARG;
+  if (T <= 0 || C <= 0 || r <= 0 || ld_rt < T) return LORA_ERR_INVALID_ARG;
+  if (C % 8 != 0 || r % 8 != 0 || r > 64 || ld_rt % 8 != 0 || T > (1ll << 30) || C > (1ll << 24))
+    return LORA_ERR_UNSUPPORTED_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(S) | reinterpret_cast<uintptr_t>(Rt) | reinterpret_cast<uintptr_t>(out)) & 15u)
+    return LORA_ERR_MISALIGNED;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNoAllocMaxDevices) return LORA_ERR_NO_DEVICE;
+  NoAllocDevice nd;
+  {
+    // one-time set-up per device (the device is current): resolve the device address of the static array.
+    // In host code `g_noalloc_scratch` is only a handle; handing it to a kernel would be a wrong pointer.
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    NoAllocDevice& slot = g_noalloc_dev[dev];
+    if (!slot.ready) {
+      int major = 0, sms = 0;
+      if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess || major != 10)
+        return LORA_ERR_NO_DEVICE;
+      if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        return LORA_ERR_CUDA;
+      void* ptr = nullptr;
+      if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) {
+        cudaGetLastError();
+        return LORA_ERR_CUDA;
+      }
+      if (grad_configure() != cudaSuccess) {
+        cudaGetLastError();
+        return LORA_ERR_CUDA;
+      }
+      slot.scratch = static_cast<unsigned char*>(ptr);
+      slot.num_sms = sms;
+      slot.ready = true;
+    }
+    nd = slot;
+  }
+  // grid: the same rule the planned path uses (feature chunks x token chunks, at most one CTA per SM)
+  GradParams g{};
+  g.T = static_cast<int>(T);
+  g.C = static_cast<int>(C);
+  g.r = static_cast<int>(r);
+  g.r_pad = static_cast<int>((r + 15) / 16 * 16);
+  int fc = g.r_pad <= 32 ? 512 : 256;
+  const int c128 = static_cast<int>((C + 127) / 128 * 128);
+  if (fc > c128) fc = c128;
+  g.feat_chunk = fc;
+  g.n_feat_chunks = static_cast<int>((C + fc - 1) / fc);
+  g.n_slabs = static_cast<int>((T + kGradSlab - 1) / kGradSlab);
+  int n_tok = nd.num_sms / g.n_feat_chunks;
+  if (n_tok < 1) n_tok = 1;
+  if (n_tok > g.n_slabs) n_tok = g.n_slabs;
+  g.n_token_chunks = n_tok;
+  const size_t fixed = 4 * static_cast<size_t>(g.r_pad) * 128 + 4096;
+  int stages = static_cast<int>((232448 - fixed) / kGradStageBytes);
+  g.stages = stages > kGradMaxStages ? kGradMaxStages : stages;
+  g.c_pad = static_cast<int>((C + 31) / 32 * 32);
+  const size_t part_bytes = static_cast<size_t>(n_tok) * g.r_pad * g.c_pad * sizeof(float);
+  if (static_cast<size_t>(g.n_feat_chunks) * 4 > kNoAllocHeaderBytes - 256 ||
+      kNoAllocHeaderBytes + part_bytes > kNoAllocScratchBytes)
+    return LORA_ERR_WORKSPACE;      // the problem needs more scratch than the static array holds
+  g.with_p = 0;
+  g.out_is_da = 0;
+  g.scale = 1.0f;
+  g.out = static_cast<float*>(out);
+  g.out_part = reinterpret_cast<float*>(nd.scratch + kNoAllocHeaderBytes);
+  g.p_part = nullptr;
+  g.pt_out = nullptr;
+  g.ld_t = static_cast<int>(ld_rt);
+  g.slab_counters = nullptr;
+  g.feat_counters = reinterpret_cast<unsigned*>(nd.scratch + 256);
+  g.status = reinterpret_cast<unsigned*>(nd.scratch);
+  g.zero_words = nullptr;
+  g.n_zero_words = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the array keeps the previous call's contents: the arrival counters (and status) must start at zero
+  if (cudaMemsetAsync(nd.scratch, 0, kNoAllocHeaderBytes, st) != cudaSuccess) return LORA_ERR_CUDA;
+  CUtensorMap tmS, tmR;
+  if (!noalloc_tmap(&tmS, S, static_cast<uint64_t>(C), static_cast<uint64_t>(T), static_cast<uint64_t>(C), 64, kGradSlab) ||
+      !noalloc_tmap(&tmR, Rt, static_cast<uint64_t>(T), static_cast<uint64_t>(r), static_cast<uint64_t>(ld_rt), 64, g.r_pad))
+    return LORA_ERR_CUDA;
+  if (launch_grad(tmS, tmR, tmR, g, st) != cudaSuccess) return LORA_ERR_CUDA;
+  return LORA_OK;
+}
+
+extern "C" int64_t lora_grad_contract_noalloc_max_scratch(void) {
+  return static_cast<int64_t>(lora::kNoAllocScratchBytes);
+}
