@@ -61,11 +61,11 @@ typedef struct lora_shape {
 
 /* What the per-shape selector chose (Section 3.2.2 "dynamic profiling" analogue at kernel level). */
 typedef struct lora_kernel_config {
-  int32_t block_m;         /* token rows per GEMM tile (128)                                   */
-  int32_t fwd_block_n;     /* output columns per tile of the forward GEMM (64, 128 or 192)     */
+  int32_t block_m;         /* token rows per GEMM tile: 128 (one CTA) or 256 (CTA pair)        */
+  int32_t fwd_block_n;     /* output columns per tile of the forward GEMM (multiple of 16)     */
   int32_t dx_block_n;      /* output columns per tile of the dX GEMM                           */
   int32_t block_k;         /* contraction elements per pipeline stage (64)                     */
-  int32_t stages;          /* depth of the TMA -> MMA shared-memory ring                       */
+  int32_t stages;          /* depth of the TMA -> MMA shared-memory ring, forward GEMM         */
   int32_t group_m;         /* tile rasterisation: m-tiles per band (L2 reuse)                  */
   int32_t split_k;         /* split-K factor of the dense GEMMs (1 = none)                     */
   int32_t r_pad;           /* rank padded to the MMA granularity (multiple of 16)              */
@@ -78,7 +78,9 @@ typedef struct lora_kernel_config {
   int32_t da_token_chunks;
   int32_t db_feat_chunks;  /* dB kernel grid                                                   */
   int32_t db_token_chunks;
-  int32_t reserved[3];
+  int32_t db_feat_chunk;   /* features per CTA of the dB kernel (grad_feat_chunk is dA's)      */
+  int32_t cta_group;       /* 1: one CTA per tile; 2: two CTAs (one TPC) share a 256-row tile  */
+  int32_t dx_stages;       /* ring depth of the dX GEMM                                        */
 } lora_kernel_config_t;
 
 /* Host-only: run the tile / split selector for a shape on a device with `num_sms` SMs.

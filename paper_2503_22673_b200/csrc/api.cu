@@ -4,6 +4,7 @@
 
 #include <atomic>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -37,6 +38,29 @@ int pick_block_n(long long T, long long N, int r_pad, int num_sms) {
     const double per_tile = (ntot / 2.0 > (128.0 + ntot) / 4.0) ? ntot / 2.0 : (128.0 + ntot) / 4.0;
     // fixed per-tile cost (rank-r MMA, accumulator hand-over), in the same unit, for a K of ~4096
     const double cost = static_cast<double>(waves) * (per_tile + 4.0);
+    if (cost < best_cost - 1e-9) {
+      best_cost = cost;
+      best = bn;
+    }
+  }
+  return best;
+}
+
+// CTA-pair tiles (256 rows): block_n is any multiple of 16 with block_n + r_pad <= 256.  Cost per tile is its
+// MMA width (block_n + r_pad columns, the adapter columns ride along) plus a fixed hand-over cost; the
+// width with the fewest (waves x cost) wins, ties go to the wider tile.
+int pick_pair_block_n(long long T, long long N, int r_pad, int num_pairs) {
+  if (const char* f = std::getenv("LORA_FORCE_BLOCK_N")) {
+    const int v = std::atoi(f);
+    if (v >= 64 && v % 16 == 0 && v + r_pad <= 256) return v;
+  }
+  int best = 256 - r_pad;
+  double best_cost = 1e300;
+  const int lo = r_pad + 32 > 144 ? r_pad + 32 : 144;
+  for (int bn = 256 - r_pad; bn >= lo; bn -= 16) {
+    const long long tiles = static_cast<long long>(ceil_div(T, kPairBlockM)) * ceil_div(N, bn);
+    const long long waves = (tiles + num_pairs - 1) / num_pairs;
+    const double cost = static_cast<double>(waves) * (bn + r_pad + 8.0);
     if (cost < best_cost - 1e-9) {
       best_cost = cost;
       best = bn;
@@ -91,13 +115,32 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
   c->fwd_block_n = pick_block_n(T, s->d_out, c->r_pad, num_sms);
   c->dx_block_n = pick_block_n(T, s->d_in, c->r_pad, num_sms);
   c->stages = 4;
+  c->dx_stages = 4;
   c->group_m = 8;
   c->split_k = 1;
   c->tail_delay = 8;
-  const long long fwd_tiles = static_cast<long long>(ceil_div(T, kBlockM)) * ceil_div(s->d_out, c->fwd_block_n);
-  const long long dx_tiles = static_cast<long long>(ceil_div(T, kBlockM)) * ceil_div(s->d_in, c->dx_block_n);
-  c->fwd_ctas = static_cast<int>(fwd_tiles < num_sms ? fwd_tiles : num_sms);
-  c->dx_ctas = static_cast<int>(dx_tiles < num_sms ? dx_tiles : num_sms);
+  c->cta_group = (T > kBlockM && num_sms >= 2) ? 2 : 1;
+  if (const char* f = std::getenv("LORA_FORCE_CTA_GROUP")) {
+    const int v = std::atoi(f);
+    if (v == 1 || (v == 2 && num_sms >= 2)) c->cta_group = v;
+  }
+  if (c->cta_group == 2) {
+    const int pairs = num_sms / 2;
+    c->block_m = kPairBlockM;
+    c->fwd_block_n = pick_pair_block_n(T, s->d_out, c->r_pad, pairs);
+    c->dx_block_n = pick_pair_block_n(T, s->d_in, c->r_pad, pairs);
+    c->stages = 6;
+    c->dx_stages = 5;
+    const long long fwd_t = static_cast<long long>(ceil_div(T, kPairBlockM)) * ceil_div(s->d_out, c->fwd_block_n);
+    const long long dx_t = static_cast<long long>(ceil_div(T, kPairBlockM)) * ceil_div(s->d_in, c->dx_block_n);
+    c->fwd_ctas = 2 * static_cast<int>(fwd_t < pairs ? fwd_t : pairs);
+    c->dx_ctas = 2 * static_cast<int>(dx_t < pairs ? dx_t : pairs);
+  } else {
+    const long long fwd_tiles = static_cast<long long>(ceil_div(T, kBlockM)) * ceil_div(s->d_out, c->fwd_block_n);
+    const long long dx_tiles = static_cast<long long>(ceil_div(T, kBlockM)) * ceil_div(s->d_in, c->dx_block_n);
+    c->fwd_ctas = static_cast<int>(fwd_tiles < num_sms ? fwd_tiles : num_sms);
+    c->dx_ctas = static_cast<int>(dx_tiles < num_sms ? dx_tiles : num_sms);
+  }
   const GradGrid ga = pick_grad_grid(T, s->d_in, c->r_pad, true, num_sms);
   const GradGrid gb = pick_grad_grid(T, s->d_out, c->r_pad, false, num_sms);
   c->grad_feat_chunk = ga.feat_chunk;
@@ -106,7 +149,7 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
   c->da_token_chunks = ga.n_tok;
   c->db_feat_chunks = gb.n_feat;
   c->db_token_chunks = gb.n_tok;
-  c->reserved[0] = gb.feat_chunk;   // feature chunk of the dB kernel (differs from dA's only for small d_out)
+  c->db_feat_chunk = gb.feat_chunk;   // feature chunk of the dB kernel (differs from dA's only for small d_out)
   return LORA_OK;
 }
 
@@ -157,7 +200,7 @@ EncodeTiledFn encode_fn() {
 
 // 2-D row-major tensor of `elem_bytes`-wide elements, 128-byte swizzle, zero fill outside the tensor.
 bool make_tmap(CUtensorMap* m, const void* ptr, CUtensorMapDataType dt, int elem_bytes, uint64_t inner, uint64_t outer,
-               uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_outer) {
+               uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_outer, bool swizzle128 = true) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
   const cuuint64_t dims[2] = {inner, outer};
@@ -166,14 +209,16 @@ bool make_tmap(CUtensorMap* m, const void* ptr, CUtensorMapDataType dt, int elem
   const cuuint32_t estr[2] = {1, 1};
   (void)elem_bytes;
   const CUresult r = fn(m, dt, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
 
 bool make_bf16_tmap(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t outer, uint64_t pitch_elems,
-                    uint32_t box_inner, uint32_t box_outer) {
-  return make_tmap(m, ptr, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, inner, outer, pitch_elems * 2, box_inner, box_outer);
+                    uint32_t box_inner, uint32_t box_outer, bool swizzle128 = true) {
+  return make_tmap(m, ptr, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, inner, outer, pitch_elems * 2, box_inner, box_outer,
+                   swizzle128);
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -211,20 +256,25 @@ int launch_fwd(lora_plan* pl, const void* X, const void* W, const void* A, const
                cudaStream_t st) {
   const lora_shape_t& s = pl->shape;
   const lora_kernel_config_t& c = pl->cfg;
-  CUtensorMap tmX, tmW, tmA, tmB, tmY;
+  const bool pair = c.cta_group == 2;
+  const int half = (c.fwd_block_n + c.r_pad) / 2;
+  CUtensorMap tmX, tmW, tmW1, tmA, tmB, tmY;
   bool ok = make_bf16_tmap(&tmX, X, s.d_in, s.T, s.d_in, 64, kBlockM);
-  ok = ok && make_bf16_tmap(&tmW, W, s.d_in, s.d_out, s.d_in, 64, c.fwd_block_n);
+  ok = ok && make_bf16_tmap(&tmW, W, s.d_in, s.d_out, s.d_in, 64, pair ? half : c.fwd_block_n);
+  if (pair) ok = ok && make_bf16_tmap(&tmW1, W, s.d_in, s.d_out, s.d_in, 64, c.fwd_block_n - half);
   ok = ok && make_bf16_tmap(&tmA, A, s.d_in, s.r, s.d_in, 64, c.r_pad);
-  ok = ok && make_bf16_tmap(&tmB, B, s.r, s.d_out, s.r, 64, c.fwd_block_n);
+  ok = ok && make_bf16_tmap(&tmB, B, s.r, s.d_out, s.r, 64, pair ? c.fwd_block_n / 2 : c.fwd_block_n);
   ok = ok && make_bf16_tmap(&tmY, Y, s.d_out, s.T, s.d_out, 64, kBlockM);
   if (!ok) return LORA_ERR_CUDA;
   GemmParams p{};
+  p.out = static_cast<__nv_bfloat16*>(Y);
+  p.ld_out = static_cast<int>(s.d_out);
   p.M = static_cast<int>(s.T);
   p.N = static_cast<int>(s.d_out);
   p.K = static_cast<int>(s.d_in);
   p.r_pad = c.r_pad;
   p.block_n = c.fwd_block_n;
-  p.tiles_m = ceil_div(s.T, kBlockM);
+  p.tiles_m = ceil_div(s.T, c.block_m);
   p.tiles_n = ceil_div(s.d_out, c.fwd_block_n);
   p.num_tiles = p.tiles_m * p.tiles_n;
   p.kblocks = ceil_div(s.d_in, kBlockK);
@@ -237,7 +287,9 @@ int launch_fwd(lora_plan* pl, const void* X, const void* W, const void* A, const
   p.status = pl->d_status;
   p.zero_words = nullptr;
   p.n_zero_words = 0;
-  if (launch_gemm_fwd(tmX, tmW, tmA, tmB, tmY, p, c.fwd_ctas, st) != cudaSuccess) return LORA_ERR_CUDA;
+  const cudaError_t le = pair ? launch_gemm_pair_fwd(tmX, tmW, tmW1, tmA, tmB, tmY, p, c.fwd_ctas, st)
+                              : launch_gemm_fwd(tmX, tmW, tmA, tmB, tmY, p, c.fwd_ctas, st);
+  if (le != cudaSuccess) return LORA_ERR_CUDA;
   g_launches.fetch_add(1);
   return LORA_OK;
 }
@@ -270,22 +322,26 @@ int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const
     CUtensorMap tmdY, tmW, tmB, tmA, tmdX;
     bool ok = make_bf16_tmap(&tmdY, dY, s.d_out, s.T, s.d_out, 64, kBlockM);
     ok = ok && make_bf16_tmap(&tmW, W, s.d_in, s.d_out, s.d_in, 64, 64);
-    ok = ok && make_bf16_tmap(&tmB, B, s.r, s.d_out, s.r, 64, 64);
+    const bool pair = c.cta_group == 2;
+    if (pair) ok = ok && make_bf16_tmap(&tmB, B, s.r, s.d_out, s.r, 8, 64, false);   // unswizzled 8-column boxes
+    else ok = ok && make_bf16_tmap(&tmB, B, s.r, s.d_out, s.r, 64, 64);
     ok = ok && make_bf16_tmap(&tmA, A, s.d_in, s.r, s.d_in, 64, c.r_pad);
     ok = ok && make_bf16_tmap(&tmdX, dX, s.d_in, s.T, s.d_in, 64, kBlockM);
     if (!ok) return LORA_ERR_CUDA;
     GemmParams p{};
+    p.out = static_cast<__nv_bfloat16*>(dX);
+    p.ld_out = static_cast<int>(s.d_in);
     p.M = static_cast<int>(s.T);
     p.N = static_cast<int>(s.d_in);
     p.K = static_cast<int>(s.d_out);
     p.r_pad = c.r_pad;
     p.block_n = c.dx_block_n;
-    p.tiles_m = ceil_div(s.T, kBlockM);
+    p.tiles_m = ceil_div(s.T, c.block_m);
     p.tiles_n = ceil_div(s.d_in, c.dx_block_n);
     p.num_tiles = p.tiles_m * p.tiles_n;
     p.kblocks = ceil_div(s.d_out, kBlockK);
     p.group_m = c.group_m;
-    p.stages = c.stages;
+    p.stages = c.dx_stages;
     p.tail_delay = c.tail_delay;
     p.scale = scale;
     p.rt_out = qt;
@@ -293,7 +349,9 @@ int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const
     p.status = pl->d_status;
     p.zero_words = counters;
     p.n_zero_words = w.n_counters;
-    if (launch_gemm_dx(tmdY, tmW, tmB, tmA, tmdX, p, c.dx_ctas, st) != cudaSuccess) return LORA_ERR_CUDA;
+    const cudaError_t le = pair ? launch_gemm_pair_dx(tmdY, tmW, tmB, tmA, tmdX, p, c.dx_ctas, st)
+                                : launch_gemm_dx(tmdY, tmW, tmB, tmA, tmdX, p, c.dx_ctas, st);
+    if (le != cudaSuccess) return LORA_ERR_CUDA;
     g_launches.fetch_add(1);
   }
   return LORA_OK;
@@ -363,7 +421,7 @@ int launch_db(lora_plan* pl, const void* dY, float scale, void* dB, cudaStream_t
     g.C = static_cast<int>(s.d_out);
     g.r = static_cast<int>(s.r);
     g.r_pad = c.r_pad;
-    g.feat_chunk = c.reserved[0];
+    g.feat_chunk = c.db_feat_chunk;
     g.n_feat_chunks = c.db_feat_chunks;
     g.n_token_chunks = c.db_token_chunks;
     g.n_slabs = w.n_slabs;
@@ -434,7 +492,7 @@ int lora_plan_create(const lora_shape_t* shape, int device, lora_plan_t** out) {
   pl->workspace = nullptr;
   pl->workspace_bytes = 0;
   pl->d_status = nullptr;
-  if (gemm_configure() != cudaSuccess || grad_configure() != cudaSuccess || encode_fn() == nullptr ||
+  if (gemm_configure() != cudaSuccess || gemm_pair_configure() != cudaSuccess || grad_configure() != cudaSuccess || encode_fn() == nullptr ||
       cudaMalloc(&pl->d_status, 256) != cudaSuccess || cudaMemset(pl->d_status, 0, 256) != cudaSuccess) {
     cudaGetLastError();
     if (pl->d_status) cudaFree(pl->d_status);
@@ -484,11 +542,12 @@ int lora_plan_describe(const lora_plan_t* plan, char* buf, size_t n) {
   if (plan == nullptr || buf == nullptr || n == 0) return LORA_ERR_INVALID_ARG;
   const lora_kernel_config_t& c = plan->cfg;
   std::snprintf(buf, n,
-                "T=%lld d_in=%lld d_out=%lld r=%lld | sms=%d tile fwd 128x%dx64 dx 128x%dx64 stages=%d group_m=%d "
+                "T=%lld d_in=%lld d_out=%lld r=%lld | sms=%d cta_group=%d tile fwd %dx%dx64 dx %dx%dx64 stages=%d/%d group_m=%d "
                 "split_k=%d r_pad=%d ctas fwd=%d dx=%d tail_delay=%d | grad chunk=%d stages=%d dA grid=%dx%d dB grid=%dx%d "
                 "| bwd workspace=%zu B",
                 (long long)plan->shape.T, (long long)plan->shape.d_in, (long long)plan->shape.d_out,
-                (long long)plan->shape.r, plan->num_sms, c.fwd_block_n, c.dx_block_n, c.stages, c.group_m, c.split_k,
+                (long long)plan->shape.r, plan->num_sms, c.cta_group, c.block_m, c.fwd_block_n, c.block_m, c.dx_block_n,
+                c.stages, c.dx_stages, c.group_m, c.split_k,
                 c.r_pad, c.fwd_ctas, c.dx_ctas, c.tail_delay, c.grad_feat_chunk, c.grad_stages, c.da_feat_chunks,
                 c.da_token_chunks, c.db_feat_chunks, c.db_token_chunks, plan->ws.total);
   return LORA_OK;

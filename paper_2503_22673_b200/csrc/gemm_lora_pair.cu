@@ -1,0 +1,400 @@
+// CTA-pair variant of the dense projection GEMM with the rank-r LoRA adapter fused in (Section 3.2.2, LoRA):
+//
+//   forward   Y  = X  W^T + s (X  A^T) B^T      act = X,  contraction over d_in
+//   backward  dX = dY W   + s (dY B  ) A        act = dY, contraction over d_out
+//
+// Two CTAs on the two SMs of a TPC (cluster of 2) own one 256 x block_n output tile.  Each CTA stages its own
+// 128 activation rows and HALF of the weight tile; one tcgen05.mma.cta_group::2 (M = 256) issued by the leader
+// CTA reads both shared memories, so every weight byte is fetched from L2 once per 256 rows instead of once per
+// 128.  That halves the L2 -> shared-memory traffic per FLOP, which is what bounds the single-CTA kernel.
+// No TMA multicast is used anywhere: each CTA issues plain loads for its own half.
+//
+// Roles per CTA: warp 0 TMA producer (both CTAs), warp 1 MMA issuer (leader only) + TMEM allocation,
+// warps 2..5 epilogue (both CTAs, 128 rows each).  Barriers:
+//   full[s]      leader's; the leader arms it with the byte count of BOTH CTAs, both CTAs' loads credit it
+//   empty[s]     per CTA; tcgen05.commit multicast to both CTAs when the MMAs that read the stage are done
+//   side_full[b] per CTA; commit multicast: P (or Q) columns of accumulator b are complete
+//   ps_ready[b]  leader's; 256 arrivals: both epilogues have written their bf16 s*P rows to shared memory
+//   acc_full[b]  per CTA; commit multicast: accumulator b incl. the rank-r product is complete
+//   acc_empty[b] leader's; 256 arrivals: both epilogues have drained accumulator b
+// Forward: the weight/adapter rows of a tile are K-major and contiguous, so ONE MMA of width block_n + r_pad
+// gives the dense accumulator and P side by side (leader holds rows [0, half), peer the rest incl. A).
+// Backward: W, B, A are MN-major operands in their natural layout; Q = dY B is a second, narrow MMA per k-step
+// whose B operand (r_pad/2 columns per CTA) uses the unswizzled 8 x 16-byte core-matrix layout.
+#include "kernels.h"
+#include "sm100_ptx.cuh"
+
+namespace lora {
+
+namespace {
+
+struct PairTile {
+  int m_idx, n_idx;
+};
+
+__device__ __forceinline__ PairTile pair_tile(int id, const GemmParams& p) {
+  const int per_band = p.group_m * p.tiles_n;
+  const int band = id / per_band;
+  const int rem = id - band * per_band;
+  const int rows = min(p.group_m, p.tiles_m - band * p.group_m);
+  PairTile c;
+  c.m_idx = band * p.group_m + rem % rows;
+  c.n_idx = rem / rows;
+  return c;
+}
+
+template <bool kBwd>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M, K], box 64(k) x 128
+                      const __grid_constant__ CUtensorMap tm_w0,    // fwd: W box 64(k) x half ; bwd: W box 64(n) x 64(k)
+                      const __grid_constant__ CUtensorMap tm_w1,    // fwd: W box 64(k) x (block_n - half) ; bwd unused
+                      const __grid_constant__ CUtensorMap tm_side,  // fwd: A box 64(k) x r_pad ; bwd: B unswizzled box 8(r) x 64(k)
+                      const __grid_constant__ CUtensorMap tm_tail,  // fwd: B box 64(r) x block_n/2 ; bwd: A box 64(n) x r_pad
+                      const __grid_constant__ CUtensorMap tm_out,   // Y / dX [M, N], box 64 x 128
+                      const GemmParams p) {
+  constexpr int kStage = kBwd ? kPairStageBytesBwd : kPairStageBytesFwd;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t ring = smem_u32(smem);
+  const uint32_t staging = ring + p.stages * kStage;
+  uint8_t* staging_ptr = smem + p.stages * kStage;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(staging_ptr + 2 * kStagingBytes);
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
+  auto side_full = [&](int b) { return bar0 + 8u * (2 * kMaxStages + b); };
+  auto ps_ready = [&](int b) { return bar0 + 8u * (2 * kMaxStages + 2 + b); };
+  auto acc_full = [&](int b) { return bar0 + 8u * (2 * kMaxStages + 4 + b); };
+  auto acc_empty = [&](int b) { return bar0 + 8u * (2 * kMaxStages + 6 + b); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kGemmBarriers);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_cta_rank();
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(side_full(b), 1);
+      mbar_init(ps_ready(b), 256);
+      mbar_init(acc_full(b), 1);
+      mbar_init(acc_empty(b), 256);
+    }
+    *abort_flag = 0;
+    fence_barrier_init();
+    tma_prefetch_desc(&tm_act);
+    tma_prefetch_desc(&tm_w0);
+    tma_prefetch_desc(&tm_w1);
+    tma_prefetch_desc(&tm_side);
+    tma_prefetch_desc(&tm_tail);
+    tma_prefetch_desc(&tm_out);
+    if (blockIdx.x == 0 && p.zero_words != nullptr)
+      for (int i = 0; i < p.n_zero_words; ++i) p.zero_words[i] = 0u;
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(tmem_slot), 512);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();           // the peer's barriers exist before anything is signalled across the pair
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int G = gridDim.x >> 1;                 // CTA pairs
+  const int pair = blockIdx.x >> 1;
+  const int n_my = (p.num_tiles > pair) ? (p.num_tiles - 1 - pair) / G + 1 : 0;
+  const int KB = p.kblocks;
+  const int D = min(KB, p.tail_delay);
+  const int S = p.stages;
+  const int BN = p.block_n;
+  const int half = (BN + p.r_pad) >> 1;         // forward: weight/adapter rows held by each CTA
+  const int side_boxes = p.r_pad >> 4;          // backward: 8-column unswizzled boxes of B per CTA
+
+  if (warp == 0) {
+    // ================================ TMA producer (both CTAs) ================================
+    if (lane == 0) {
+      int it = 0;
+      bool ok = true;
+      auto acquire = [&]() -> int {
+        const int slot = it % S;
+        ok = mbar_wait(empty_bar(slot), ((it / S) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY);
+        ++it;
+        return slot;
+      };
+      auto load_main = [&](int i, int kb) {
+        const PairTile tc = pair_tile(pair + i * G, p);
+        const int m0 = tc.m_idx * kPairBlockM + static_cast<int>(rank) * 128, n0 = tc.n_idx * BN, k0 = kb * kBlockK;
+        const int slot = acquire();
+        if (!ok) return;
+        const uint32_t a_dst = ring + slot * kStage, b_dst = a_dst + 16384;
+        const uint32_t fb = map_to_cta(full_bar(slot), 0);
+        if (!kBwd) {
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(slot), 2 * 16384 + (BN + p.r_pad) * 128);
+          tma_load_2d_pair(a_dst, &tm_act, fb, k0, m0);
+          if (rank == 0) {
+            tma_load_2d_pair(b_dst, &tm_w0, fb, k0, n0);
+          } else {
+            tma_load_2d_pair(b_dst, &tm_w1, fb, k0, n0 + half);
+            tma_load_2d_pair(b_dst + (BN - half) * 128, &tm_side, fb, k0, 0);
+          }
+        } else {
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(slot), 2 * (16384 + 16384 + side_boxes * 1024));
+          tma_load_2d_pair(a_dst, &tm_act, fb, k0, m0);
+          const int nb = n0 + static_cast<int>(rank) * (BN >> 1);
+          tma_load_2d_pair(b_dst, &tm_w0, fb, nb, k0);
+          tma_load_2d_pair(b_dst + 8192, &tm_w0, fb, nb + 64, k0);
+          for (int b = 0; b < side_boxes; ++b)
+            tma_load_2d_pair(b_dst + 16384 + b * 1024, &tm_side, fb, static_cast<int>(rank) * (p.r_pad >> 1) + 8 * b, k0);
+        }
+      };
+      auto load_tail = [&](int i) {
+        const PairTile tc = pair_tile(pair + i * G, p);
+        const int nb = tc.n_idx * BN + static_cast<int>(rank) * (BN >> 1);
+        const int slot = acquire();
+        if (!ok) return;
+        const uint32_t b_dst = ring + slot * kStage + 16384;
+        const uint32_t fb = map_to_cta(full_bar(slot), 0);
+        if (!kBwd) {
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(slot), BN * 128);
+          tma_load_2d_pair(b_dst, &tm_tail, fb, 0, nb);
+        } else {
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(slot), 2 * 2 * p.r_pad * 128);
+          tma_load_2d_pair(b_dst, &tm_tail, fb, nb, 0);
+          tma_load_2d_pair(b_dst + 8192, &tm_tail, fb, nb + 64, 0);
+        }
+      };
+      for (int i = 0; i < n_my && ok; ++i) {
+        for (int kb = 0; kb < KB && ok; ++kb) {
+          if (i > 0 && kb == D) load_tail(i - 1);
+          if (ok) load_main(i, kb);
+        }
+        if (ok && i > 0 && D == KB) load_tail(i - 1);
+      }
+      if (ok && n_my > 0) load_tail(n_my - 1);
+    }
+  } else if (warp == 1) {
+    // ================================ MMA issuer (leader CTA only) ================================
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc_main = kBwd ? mma_idesc_bf16(256, BN, false, true) : mma_idesc_bf16(256, BN + p.r_pad, false, false);
+      const uint32_t idesc_side = mma_idesc_bf16(256, p.r_pad, false, true);
+      const uint32_t idesc_tail = mma_idesc_bf16(256, BN, false, kBwd);
+      int it = 0;
+      bool ok = true;
+      auto mma_main = [&](int i, int kb) {
+        const int buf = i & 1, use = i >> 1;
+        if (kb == 0) {
+          ok = mbar_wait_cluster(acc_empty(buf), (use & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_ACC_EMPTY);
+          if (!ok) return;
+        }
+        const int slot = it % S;
+        ok = mbar_wait_cluster(full_bar(slot), (it / S) & 1, abort_flag, p.status, DEV_TIMEOUT_FULL);
+        ++it;
+        if (!ok) return;
+        tc_fence_after();
+        const uint32_t a_addr = ring + slot * kStage, b_addr = a_addr + 16384, s_addr = b_addr + 16384;
+        const uint32_t acc = tmem_base + buf * 256;
+#pragma unroll
+        for (int ks = 0; ks < kBlockK / 16; ++ks) {
+          const uint32_t accum = (kb | ks) != 0 ? 1u : 0u;
+          const uint64_t ad = smem_desc_sw128(a_addr + ks * 32, 16, 1024);
+          if (!kBwd) {
+            mma_bf16_ss_pair(acc, ad, smem_desc_sw128(b_addr + ks * 32, 16, 1024), idesc_main, accum);
+          } else {
+            mma_bf16_ss_pair(acc, ad, smem_desc_sw128(b_addr + ks * 2048, 8192, 1024), idesc_main, accum);
+            mma_bf16_ss_pair(acc + BN, ad, smem_desc_noswizzle(s_addr + ks * 256, 128, 1024), idesc_side, accum);
+          }
+        }
+        mma_commit_pair(empty_bar(slot));
+        if (kb == KB - 1) mma_commit_pair(side_full(buf));
+      };
+      auto mma_tail = [&](int i) {
+        const int buf = i & 1, use = i >> 1;
+        ok = mbar_wait_cluster(ps_ready(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_PS);
+        if (!ok) return;
+        const int slot = it % S;
+        ok = mbar_wait_cluster(full_bar(slot), (it / S) & 1, abort_flag, p.status, DEV_TIMEOUT_FULL);
+        ++it;
+        if (!ok) return;
+        tc_fence_after();
+        const uint32_t b_addr = ring + slot * kStage + 16384;
+        for (int ks = 0; ks < p.r_pad / 16; ++ks) {
+          const uint64_t ad = smem_desc_sw128(staging + ks * 32, 16, 1024);
+          const uint64_t bd = kBwd ? smem_desc_sw128(b_addr + ks * 2048, 8192, 1024)
+                                   : smem_desc_sw128(b_addr + ks * 32, 16, 1024);
+          mma_bf16_ss_pair(tmem_base + buf * 256, ad, bd, idesc_tail, 1u);
+        }
+        mma_commit_pair(empty_bar(slot));
+        mma_commit_pair(acc_full(buf));
+      };
+      for (int i = 0; i < n_my && ok; ++i) {
+        for (int kb = 0; kb < KB && ok; ++kb) {
+          if (i > 0 && kb == D) mma_tail(i - 1);
+          if (ok) mma_main(i, kb);
+        }
+        if (ok && i > 0 && D == KB) mma_tail(i - 1);
+      }
+      if (ok && n_my > 0) mma_tail(n_my - 1);
+    }
+  } else {
+    // ================================ epilogue (128 threads per CTA) ================================
+    const int e = threadIdx.x - 64;
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+    const int full_chunks = BN >> 6;
+    const int rem_cols = BN & 63;                  // 0, 16, 32 or 48 columns stored with plain stores
+    for (int i = 0; i < n_my; ++i) {
+      const PairTile tc = pair_tile(pair + i * G, p);
+      const int m0 = tc.m_idx * kPairBlockM + static_cast<int>(rank) * 128, n0 = tc.n_idx * BN;
+      const int buf = i & 1, use = i >> 1;
+      if (e == 0) tma_store_wait_read<0>();
+      bool ok = mbar_wait(side_full(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_SIDE);
+      if (named_bar_or(1, 128, !ok)) break;
+      tc_fence_after();
+      for (int c16 = 0; c16 < p.r_pad / 16; ++c16) {
+        uint32_t v[16];
+        tmem_ld16(lane_addr + buf * 256 + BN + c16 * 16, v);
+        tmem_ld_wait();
+        uint32_t w[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          w[q] = pack_bf16x2(__uint_as_float(v[2 * q]) * p.scale, __uint_as_float(v[2 * q + 1]) * p.scale);
+        *reinterpret_cast<uint4*>(staging_ptr + sw128_offset(row, 2 * c16)) = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4*>(staging_ptr + sw128_offset(row, 2 * c16 + 1)) = make_uint4(w[4], w[5], w[6], w[7]);
+        if (kBwd && p.rt_out != nullptr && tc.n_idx == 0 && m0 + row < p.M) {
+          unsigned short* rt = reinterpret_cast<unsigned short*>(p.rt_out);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            rt[static_cast<size_t>(c16 * 16 + 2 * q) * p.ld_rt + m0 + row] = static_cast<unsigned short>(w[q] & 0xFFFFu);
+            rt[static_cast<size_t>(c16 * 16 + 2 * q + 1) * p.ld_rt + m0 + row] = static_cast<unsigned short>(w[q] >> 16);
+          }
+        }
+      }
+      fence_proxy_async_smem();
+      tc_fence_before();
+      mbar_arrive_cluster(map_to_cta(ps_ready(buf), 0));
+      ok = mbar_wait(acc_full(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_ACC);
+      if (named_bar_or(1, 128, !ok)) break;
+      tc_fence_after();
+      for (int c = 0; c < full_chunks; ++c) {
+        uint32_t v0[32], v1[32];
+        tmem_ld32(lane_addr + buf * 256 + c * 64, v0);
+        tmem_ld32(lane_addr + buf * 256 + c * 64 + 32, v1);
+        tmem_ld_wait();
+        if (c == full_chunks - 1 && rem_cols == 0) {
+          tc_fence_before();
+          mbar_arrive_cluster(map_to_cta(acc_empty(buf), 0));
+        }
+        if (n0 + c * 64 >= p.N) continue;
+        if (e == 0) tma_store_wait_read<1>();
+        named_bar_sync(2, 128);
+        uint8_t* dst = staging_ptr + (c & 1) * kStagingBytes;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          uint4 w;
+          w.x = pack_bf16x2(__uint_as_float(v0[8 * q + 0]), __uint_as_float(v0[8 * q + 1]));
+          w.y = pack_bf16x2(__uint_as_float(v0[8 * q + 2]), __uint_as_float(v0[8 * q + 3]));
+          w.z = pack_bf16x2(__uint_as_float(v0[8 * q + 4]), __uint_as_float(v0[8 * q + 5]));
+          w.w = pack_bf16x2(__uint_as_float(v0[8 * q + 6]), __uint_as_float(v0[8 * q + 7]));
+          *reinterpret_cast<uint4*>(dst + sw128_offset(row, q)) = w;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          uint4 w;
+          w.x = pack_bf16x2(__uint_as_float(v1[8 * q + 0]), __uint_as_float(v1[8 * q + 1]));
+          w.y = pack_bf16x2(__uint_as_float(v1[8 * q + 2]), __uint_as_float(v1[8 * q + 3]));
+          w.z = pack_bf16x2(__uint_as_float(v1[8 * q + 4]), __uint_as_float(v1[8 * q + 5]));
+          w.w = pack_bf16x2(__uint_as_float(v1[8 * q + 6]), __uint_as_float(v1[8 * q + 7]));
+          *reinterpret_cast<uint4*>(dst + sw128_offset(row, 4 + q)) = w;
+        }
+        fence_proxy_async_smem();
+        named_bar_sync(2, 128);
+        if (e == 0) {
+          tma_store_2d(&tm_out, staging + (c & 1) * kStagingBytes, n0 + c * 64, m0);
+          tma_store_commit();
+        }
+      }
+      if (rem_cols != 0) {
+        // ragged last chunk (block_n is not a multiple of 64): 16 columns at a time, plain 16-byte stores
+        const int cbase = full_chunks * 64;
+        for (int c16 = 0; c16 < rem_cols / 16; ++c16) {
+          uint32_t v[16];
+          tmem_ld16(lane_addr + buf * 256 + cbase + c16 * 16, v);
+          tmem_ld_wait();
+          if (c16 == rem_cols / 16 - 1) {
+            tc_fence_before();
+            mbar_arrive_cluster(map_to_cta(acc_empty(buf), 0));
+          }
+          const int col = n0 + cbase + c16 * 16;
+          if (m0 + row < p.M) {
+            uint4 w0, w1;
+            w0.x = pack_bf16x2(__uint_as_float(v[0]), __uint_as_float(v[1]));
+            w0.y = pack_bf16x2(__uint_as_float(v[2]), __uint_as_float(v[3]));
+            w0.z = pack_bf16x2(__uint_as_float(v[4]), __uint_as_float(v[5]));
+            w0.w = pack_bf16x2(__uint_as_float(v[6]), __uint_as_float(v[7]));
+            w1.x = pack_bf16x2(__uint_as_float(v[8]), __uint_as_float(v[9]));
+            w1.y = pack_bf16x2(__uint_as_float(v[10]), __uint_as_float(v[11]));
+            w1.z = pack_bf16x2(__uint_as_float(v[12]), __uint_as_float(v[13]));
+            w1.w = pack_bf16x2(__uint_as_float(v[14]), __uint_as_float(v[15]));
+            __nv_bfloat16* orow = p.out + static_cast<size_t>(m0 + row) * p.ld_out;
+            if (col < p.N) *reinterpret_cast<uint4*>(orow + col) = w0;
+            if (col + 8 < p.N) *reinterpret_cast<uint4*>(orow + col + 8) = w1;
+          }
+        }
+      }
+    }
+    if (e == 0) tma_store_wait_all<0>();
+  }
+
+  // ================================ teardown ================================
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag && threadIdx.x == 0) {
+    const long long t0 = clock64();          // bounded grace period for copies still in flight
+    while (clock64() - t0 < 2000000LL) {
+    }
+  }
+  __syncthreads();
+  cluster_sync_all();                        // neither CTA leaves while the other may still touch its memory
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, 512);
+  }
+}
+
+}  // namespace
+
+size_t gemm_pair_smem_bytes(bool bwd, int stages) {
+  return static_cast<size_t>(stages) * (bwd ? kPairStageBytesBwd : kPairStageBytesFwd) + 2 * kStagingBytes +
+         kGemmBarriers * 8 + 16 + 1024;
+}
+
+cudaError_t gemm_pair_configure() {
+  cudaError_t e = cudaFuncSetAttribute(lora_gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(lora_gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+}
+
+cudaError_t launch_gemm_pair_fwd(const CUtensorMap& tmX, const CUtensorMap& tmW0, const CUtensorMap& tmW1,
+                                 const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
+                                 const GemmParams& p, int ctas, cudaStream_t stream) {
+  lora_gemm_pair_kernel<false><<<ctas, kGemmThreads, gemm_pair_smem_bytes(false, p.stages), stream>>>(
+      tmX, tmW0, tmW1, tmA, tmB, tmY, p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_pair_dx(const CUtensorMap& tmdY, const CUtensorMap& tmW, const CUtensorMap& tmB,
+                                const CUtensorMap& tmA, const CUtensorMap& tmdX, const GemmParams& p, int ctas,
+                                cudaStream_t stream) {
+  lora_gemm_pair_kernel<true><<<ctas, kGemmThreads, gemm_pair_smem_bytes(true, p.stages), stream>>>(
+      tmdY, tmW, tmW, tmB, tmA, tmdX, p);
+  return cudaGetLastError();
+}
+
+}  // namespace lora
