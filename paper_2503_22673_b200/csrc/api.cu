@@ -141,6 +141,18 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
     c->fwd_ctas = static_cast<int>(fwd_tiles < num_sms ? fwd_tiles : num_sms);
     c->dx_ctas = static_cast<int>(dx_tiles < num_sms ? dx_tiles : num_sms);
   }
+  if (const char* f = std::getenv("LORA_FORCE_STAGES")) {   // tuning knob: shallower rings
+    const int v = std::atoi(f);
+    if (v >= 2 && v <= c->stages) c->stages = v;
+    if (v >= 2 && v <= c->dx_stages) c->dx_stages = v;
+  }
+  if (const char* f = std::getenv("LORA_FORCE_CTAS")) {   // tuning knob: cap the persistent GEMM grids
+    const int v = std::atoi(f) / c->cta_group * c->cta_group;
+    if (v >= c->cta_group) {
+      if (v < c->fwd_ctas) c->fwd_ctas = v;
+      if (v < c->dx_ctas) c->dx_ctas = v;
+    }
+  }
   const GradGrid ga = pick_grad_grid(T, s->d_in, c->r_pad, true, num_sms);
   const GradGrid gb = pick_grad_grid(T, s->d_out, c->r_pad, false, num_sms);
   c->grad_feat_chunk = ga.feat_chunk;

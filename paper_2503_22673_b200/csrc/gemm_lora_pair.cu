@@ -9,9 +9,13 @@
 // 128.  That halves the L2 -> shared-memory traffic per FLOP, which is what bounds the single-CTA kernel.
 // No TMA multicast is used anywhere: each CTA issues plain loads for its own half.
 //
-// Roles per CTA: warp 0 TMA producer (both CTAs), warp 1 MMA issuer (leader only) + TMEM allocation,
-// warps 2..5 epilogue (both CTAs, 128 rows each).  Barriers:
-//   full[s]      leader's; the leader arms it with the byte count of BOTH CTAs, both CTAs' loads credit it
+// Roles per CTA: warps 0..3 TMA producers (both CTAs), warp 4 MMA issuer (leader only) + TMEM allocation,
+// warps 5..8 epilogue (both CTAs, 128 rows each).  One warp's TMA copies sustain only ~30 B/clk (measured),
+// far below what the tensor pipe consumes, while copies from different warps proceed in parallel: so the
+// activation tile and the weight tile are issued by different warps, and even / odd ring items by different
+// warp pairs.  Barriers:
+//   full[s]      leader's, 2 arrivals (its activation and its weight producer), each arming the byte count of
+//                that operand for BOTH CTAs; both CTAs' loads credit it
 //   empty[s]     per CTA; tcgen05.commit multicast to both CTAs when the MMAs that read the stage are done
 //   side_full[b] per CTA; commit multicast: P (or Q) columns of accumulator b are complete
 //   ps_ready[b]  leader's; 256 arrivals: both epilogues have written their bf16 s*P rows to shared memory
@@ -44,7 +48,7 @@ __device__ __forceinline__ PairTile pair_tile(int id, const GemmParams& p) {
 }
 
 template <bool kBwd>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M, K], box 64(k) x 128
                       const __grid_constant__ CUtensorMap tm_w0,    // fwd: W box 64(k) x half ; bwd: W box 64(n) x 64(k)
                       const __grid_constant__ CUtensorMap tm_w1,    // fwd: W box 64(k) x (block_n - half) ; bwd unused
@@ -75,7 +79,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
-      mbar_init(full_bar(s), 1);
+      mbar_init(full_bar(s), 2);
       mbar_init(empty_bar(s), 1);
     }
     for (int b = 0; b < 2; ++b) {
@@ -95,7 +99,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
     if (blockIdx.x == 0 && p.zero_words != nullptr)
       for (int i = 0; i < p.n_zero_words; ++i) p.zero_words[i] = 0u;
   }
-  if (warp == 1) {
+  if (warp == 4) {
     tmem_alloc_pair(smem_u32(tmem_slot), 512);
     tmem_relinquish_pair();
   }
@@ -115,58 +119,76 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
   const int half = (BN + p.r_pad) >> 1;         // forward: weight/adapter rows held by each CTA
   const int side_boxes = p.r_pad >> 4;          // backward: 8-column unswizzled boxes of B per CTA
 
-  if (warp == 0) {
-    // ================================ TMA producer (both CTAs) ================================
-    if (lane == 0) {
+  if (warp < 4) {
+    // ================================ TMA producers (both CTAs) ================================
+    // warp = 2 * parity + operand: operand 0 = activation tile, 1 = weight (+ adapter) tile; the warp handles the
+    // ring items whose index has its parity.  Every lane runs the loop (uniform control flow), one elected lane
+    // issues the copies.
+    {
+      const int op = warp & 1, par = warp >> 1;
       int it = 0;
       bool ok = true;
+      // returns the slot, or -1 if the item belongs to the other warp pair
       auto acquire = [&]() -> int {
+        const int my = ((it & 1) == par);
         const int slot = it % S;
-        ok = mbar_wait(empty_bar(slot), ((it / S) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY);
+        if (my) {
+          ok = mbar_wait(empty_bar(slot), ((it / S) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY);
+          ok = __all_sync(0xffffffffu, ok);
+        }
         ++it;
-        return slot;
+        return my ? slot : -1;
       };
       auto load_main = [&](int i, int kb) {
+        const int slot = acquire();
+        if (slot < 0 || !ok) return;
         const PairTile tc = pair_tile(pair + i * G, p);
         const int m0 = tc.m_idx * kPairBlockM + static_cast<int>(rank) * 128, n0 = tc.n_idx * BN, k0 = kb * kBlockK;
-        const int slot = acquire();
-        if (!ok) return;
         const uint32_t a_dst = ring + slot * kStage, b_dst = a_dst + 16384;
         const uint32_t fb = map_to_cta(full_bar(slot), 0);
-        if (!kBwd) {
-          if (rank == 0) mbar_arrive_expect_tx(full_bar(slot), 2 * 16384 + (BN + p.r_pad) * 128);
-          tma_load_2d_pair(a_dst, &tm_act, fb, k0, m0);
-          if (rank == 0) {
-            tma_load_2d_pair(b_dst, &tm_w0, fb, k0, n0);
+        if (elect_one()) {
+          if (op == 0) {
+            if (rank == 0) mbar_arrive_expect_tx(full_bar(slot), 2 * 16384);
+            tma_load_2d_pair(a_dst, &tm_act, fb, k0, m0);
+          } else if (!kBwd) {
+            if (rank == 0) {
+              mbar_arrive_expect_tx(full_bar(slot), (BN + p.r_pad) * 128);
+              tma_load_2d_pair(b_dst, &tm_w0, fb, k0, n0);
+            } else {
+              tma_load_2d_pair(b_dst, &tm_w1, fb, k0, n0 + half);
+              tma_load_2d_pair(b_dst + (BN - half) * 128, &tm_side, fb, k0, 0);
+            }
           } else {
-            tma_load_2d_pair(b_dst, &tm_w1, fb, k0, n0 + half);
-            tma_load_2d_pair(b_dst + (BN - half) * 128, &tm_side, fb, k0, 0);
+            if (rank == 0) mbar_arrive_expect_tx(full_bar(slot), 2 * (16384 + side_boxes * 1024));
+            const int nb = n0 + static_cast<int>(rank) * (BN >> 1);
+            tma_load_2d_pair(b_dst, &tm_w0, fb, nb, k0);
+            tma_load_2d_pair(b_dst + 8192, &tm_w0, fb, nb + 64, k0);
+            for (int b = 0; b < side_boxes; ++b)
+              tma_load_2d_pair(b_dst + 16384 + b * 1024, &tm_side, fb, static_cast<int>(rank) * (p.r_pad >> 1) + 8 * b, k0);
           }
-        } else {
-          if (rank == 0) mbar_arrive_expect_tx(full_bar(slot), 2 * (16384 + 16384 + side_boxes * 1024));
-          tma_load_2d_pair(a_dst, &tm_act, fb, k0, m0);
-          const int nb = n0 + static_cast<int>(rank) * (BN >> 1);
-          tma_load_2d_pair(b_dst, &tm_w0, fb, nb, k0);
-          tma_load_2d_pair(b_dst + 8192, &tm_w0, fb, nb + 64, k0);
-          for (int b = 0; b < side_boxes; ++b)
-            tma_load_2d_pair(b_dst + 16384 + b * 1024, &tm_side, fb, static_cast<int>(rank) * (p.r_pad >> 1) + 8 * b, k0);
         }
+        __syncwarp();
       };
       auto load_tail = [&](int i) {
+        const int slot = acquire();
+        if (slot < 0 || !ok) return;
         const PairTile tc = pair_tile(pair + i * G, p);
         const int nb = tc.n_idx * BN + static_cast<int>(rank) * (BN >> 1);
-        const int slot = acquire();
-        if (!ok) return;
         const uint32_t b_dst = ring + slot * kStage + 16384;
         const uint32_t fb = map_to_cta(full_bar(slot), 0);
-        if (!kBwd) {
-          if (rank == 0) mbar_arrive_expect_tx(full_bar(slot), BN * 128);
-          tma_load_2d_pair(b_dst, &tm_tail, fb, 0, nb);
-        } else {
-          if (rank == 0) mbar_arrive_expect_tx(full_bar(slot), 2 * 2 * p.r_pad * 128);
-          tma_load_2d_pair(b_dst, &tm_tail, fb, nb, 0);
-          tma_load_2d_pair(b_dst + 8192, &tm_tail, fb, nb + 64, 0);
+        if (elect_one()) {
+          if (op == 0) {
+            if (rank == 0) mbar_arrive(full_bar(slot));          // no activation tile in a rank-r item
+          } else if (!kBwd) {
+            if (rank == 0) mbar_arrive_expect_tx(full_bar(slot), BN * 128);
+            tma_load_2d_pair(b_dst, &tm_tail, fb, 0, nb);
+          } else {
+            if (rank == 0) mbar_arrive_expect_tx(full_bar(slot), 2 * 2 * p.r_pad * 128);
+            tma_load_2d_pair(b_dst, &tm_tail, fb, nb, 0);
+            tma_load_2d_pair(b_dst + 8192, &tm_tail, fb, nb + 64, 0);
+          }
         }
+        __syncwarp();
       };
       for (int i = 0; i < n_my && ok; ++i) {
         for (int kb = 0; kb < KB && ok; ++kb) {
@@ -177,9 +199,10 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       }
       if (ok && n_my > 0) load_tail(n_my - 1);
     }
-  } else if (warp == 1) {
+  } else if (warp == 4) {
     // ================================ MMA issuer (leader CTA only) ================================
-    if (lane == 0 && rank == 0) {
+    // Whole warp of the leader CTA runs the loop; one elected lane issues every MMA and commit.
+    if (rank == 0) {
       const uint32_t idesc_main = kBwd ? mma_idesc_bf16(256, BN, false, true) : mma_idesc_bf16(256, BN + p.r_pad, false, false);
       const uint32_t idesc_side = mma_idesc_bf16(256, p.r_pad, false, true);
       const uint32_t idesc_tail = mma_idesc_bf16(256, BN, false, kBwd);
@@ -189,47 +212,57 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
         const int buf = i & 1, use = i >> 1;
         if (kb == 0) {
           ok = mbar_wait_cluster(acc_empty(buf), (use & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_ACC_EMPTY);
+          ok = __all_sync(0xffffffffu, ok);
           if (!ok) return;
         }
         const int slot = it % S;
         ok = mbar_wait_cluster(full_bar(slot), (it / S) & 1, abort_flag, p.status, DEV_TIMEOUT_FULL);
+        ok = __all_sync(0xffffffffu, ok);
         ++it;
         if (!ok) return;
         tc_fence_after();
         const uint32_t a_addr = ring + slot * kStage, b_addr = a_addr + 16384, s_addr = b_addr + 16384;
         const uint32_t acc = tmem_base + buf * 256;
+        if (elect_one()) {
 #pragma unroll
-        for (int ks = 0; ks < kBlockK / 16; ++ks) {
-          const uint32_t accum = (kb | ks) != 0 ? 1u : 0u;
-          const uint64_t ad = smem_desc_sw128(a_addr + ks * 32, 16, 1024);
-          if (!kBwd) {
-            mma_bf16_ss_pair(acc, ad, smem_desc_sw128(b_addr + ks * 32, 16, 1024), idesc_main, accum);
-          } else {
-            mma_bf16_ss_pair(acc, ad, smem_desc_sw128(b_addr + ks * 2048, 8192, 1024), idesc_main, accum);
-            mma_bf16_ss_pair(acc + BN, ad, smem_desc_noswizzle(s_addr + ks * 256, 128, 1024), idesc_side, accum);
+          for (int ks = 0; ks < kBlockK / 16; ++ks) {
+            const uint32_t accum = (kb | ks) != 0 ? 1u : 0u;
+            const uint64_t ad = smem_desc_sw128(a_addr + ks * 32, 16, 1024);
+            if (!kBwd) {
+              mma_bf16_ss_pair(acc, ad, smem_desc_sw128(b_addr + ks * 32, 16, 1024), idesc_main, accum);
+            } else {
+              mma_bf16_ss_pair(acc, ad, smem_desc_sw128(b_addr + ks * 2048, 8192, 1024), idesc_main, accum);
+              mma_bf16_ss_pair(acc + BN, ad, smem_desc_noswizzle(s_addr + ks * 256, 128, 1024), idesc_side, accum);
+            }
           }
+          mma_commit_pair(empty_bar(slot));
+          if (kb == KB - 1) mma_commit_pair(side_full(buf));
         }
-        mma_commit_pair(empty_bar(slot));
-        if (kb == KB - 1) mma_commit_pair(side_full(buf));
+        __syncwarp();
       };
       auto mma_tail = [&](int i) {
         const int buf = i & 1, use = i >> 1;
         ok = mbar_wait_cluster(ps_ready(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_PS);
+        ok = __all_sync(0xffffffffu, ok);
         if (!ok) return;
         const int slot = it % S;
         ok = mbar_wait_cluster(full_bar(slot), (it / S) & 1, abort_flag, p.status, DEV_TIMEOUT_FULL);
+        ok = __all_sync(0xffffffffu, ok);
         ++it;
         if (!ok) return;
         tc_fence_after();
         const uint32_t b_addr = ring + slot * kStage + 16384;
-        for (int ks = 0; ks < p.r_pad / 16; ++ks) {
-          const uint64_t ad = smem_desc_sw128(staging + ks * 32, 16, 1024);
-          const uint64_t bd = kBwd ? smem_desc_sw128(b_addr + ks * 2048, 8192, 1024)
-                                   : smem_desc_sw128(b_addr + ks * 32, 16, 1024);
-          mma_bf16_ss_pair(tmem_base + buf * 256, ad, bd, idesc_tail, 1u);
+        if (elect_one()) {
+          for (int ks = 0; ks < p.r_pad / 16; ++ks) {
+            const uint64_t ad = smem_desc_sw128(staging + ks * 32, 16, 1024);
+            const uint64_t bd = kBwd ? smem_desc_sw128(b_addr + ks * 2048, 8192, 1024)
+                                     : smem_desc_sw128(b_addr + ks * 32, 16, 1024);
+            mma_bf16_ss_pair(tmem_base + buf * 256, ad, bd, idesc_tail, 1u);
+          }
+          mma_commit_pair(empty_bar(slot));
+          mma_commit_pair(acc_full(buf));
         }
-        mma_commit_pair(empty_bar(slot));
-        mma_commit_pair(acc_full(buf));
+        __syncwarp();
       };
       for (int i = 0; i < n_my && ok; ++i) {
         for (int kb = 0; kb < KB && ok; ++kb) {
@@ -242,7 +275,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
     }
   } else {
     // ================================ epilogue (128 threads per CTA) ================================
-    const int e = threadIdx.x - 64;
+    const int e = threadIdx.x - 160;
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
     const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
@@ -361,7 +394,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
   }
   __syncthreads();
   cluster_sync_all();                        // neither CTA leaves while the other may still touch its memory
-  if (warp == 1) {
+  if (warp == 4) {
     __syncwarp();
     tc_fence_after();
     tmem_dealloc_pair(tmem_base, 512);
@@ -384,7 +417,7 @@ cudaError_t gemm_pair_configure() {
 cudaError_t launch_gemm_pair_fwd(const CUtensorMap& tmX, const CUtensorMap& tmW0, const CUtensorMap& tmW1,
                                  const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
                                  const GemmParams& p, int ctas, cudaStream_t stream) {
-  lora_gemm_pair_kernel<false><<<ctas, kGemmThreads, gemm_pair_smem_bytes(false, p.stages), stream>>>(
+  lora_gemm_pair_kernel<false><<<ctas, kPairThreads, gemm_pair_smem_bytes(false, p.stages), stream>>>(
       tmX, tmW0, tmW1, tmA, tmB, tmY, p);
   return cudaGetLastError();
 }
@@ -392,7 +425,7 @@ cudaError_t launch_gemm_pair_fwd(const CUtensorMap& tmX, const CUtensorMap& tmW0
 cudaError_t launch_gemm_pair_dx(const CUtensorMap& tmdY, const CUtensorMap& tmW, const CUtensorMap& tmB,
                                 const CUtensorMap& tmA, const CUtensorMap& tmdX, const GemmParams& p, int ctas,
                                 cudaStream_t stream) {
-  lora_gemm_pair_kernel<true><<<ctas, kGemmThreads, gemm_pair_smem_bytes(true, p.stages), stream>>>(
+  lora_gemm_pair_kernel<true><<<ctas, kPairThreads, gemm_pair_smem_bytes(true, p.stages), stream>>>(
       tmdY, tmW, tmW, tmB, tmA, tmdX, p);
   return cudaGetLastError();
 }

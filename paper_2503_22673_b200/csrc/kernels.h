@@ -40,6 +40,7 @@ size_t gemm_smem_bytes(int stages);
 
 // ---- CTA-pair (cta_group::2) variant: 256-row tiles, block_n a multiple of 16 with block_n + r_pad <= 256 ----
 constexpr int kPairBlockM = 256;
+constexpr int kPairThreads = 288;           // warps 0..3 TMA producers, warp 4 MMA + TMEM, warps 5..8 epilogue
 constexpr int kPairStageBytesFwd = 32768;   // 128 x 64 activations + 128 x 64 weight/adapter rows per CTA
 constexpr int kPairStageBytesBwd = 36864;   // + up to 4 KiB of unswizzled B columns for the side product
 size_t gemm_pair_smem_bytes(bool bwd, int stages);
