@@ -81,6 +81,7 @@ typedef struct lora_kernel_config {
   int32_t db_feat_chunk;   /* features per CTA of the dB kernel (grad_feat_chunk is dA's)      */
   int32_t cta_group;       /* 1: one CTA per tile; 2: two CTAs (one TPC) share a 256-row tile  */
   int32_t dx_stages;       /* ring depth of the dX GEMM                                        */
+  int32_t prefetch_dist;   /* k-blocks by which L2 prefetches run ahead of the ring (pair GEMM)*/
 } lora_kernel_config_t;
 
 /* Host-only: run the tile / split selector for a shape on a device with `num_sms` SMs.

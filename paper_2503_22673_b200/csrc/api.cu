@@ -60,7 +60,7 @@ int pick_pair_block_n(long long T, long long N, int r_pad, int num_pairs) {
   for (int bn = 256 - r_pad; bn >= lo; bn -= 16) {
     const long long tiles = static_cast<long long>(ceil_div(T, kPairBlockM)) * ceil_div(N, bn);
     const long long waves = (tiles + num_pairs - 1) / num_pairs;
-    const double cost = static_cast<double>(waves) * (bn + r_pad + 8.0);
+    const double cost = static_cast<double>(waves) * (bn + r_pad + 48.0);   // +48: accumulator hand-over, rank-r MMA, ramp
     if (cost < best_cost - 1e-9) {
       best_cost = cost;
       best = bn;
@@ -119,6 +119,7 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
   c->group_m = 8;
   c->split_k = 1;
   c->tail_delay = 8;
+  c->prefetch_dist = 0;    // L2 prefetch ahead of the ring was measured slower (it competes with the producers' copies)
   c->cta_group = (T > kBlockM && num_sms >= 2) ? 2 : 1;
   if (const char* f = std::getenv("LORA_FORCE_CTA_GROUP")) {
     const int v = std::atoi(f);
@@ -293,6 +294,7 @@ int launch_fwd(lora_plan* pl, const void* X, const void* W, const void* A, const
   p.group_m = c.group_m;
   p.stages = c.stages;
   p.tail_delay = c.tail_delay;
+  p.prefetch_dist = c.prefetch_dist;
   p.scale = scale;
   p.rt_out = nullptr;
   p.ld_rt = 0;
@@ -355,6 +357,7 @@ int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const
     p.group_m = c.group_m;
     p.stages = c.dx_stages;
     p.tail_delay = c.tail_delay;
+    p.prefetch_dist = c.prefetch_dist;
     p.scale = scale;
     p.rt_out = qt;
     p.ld_rt = w.ld_t;

@@ -122,156 +122,140 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
   if (warp < 4) {
     // ================================ TMA producers (both CTAs) ================================
     // warp = 2 * parity + operand: operand 0 = activation tile, 1 = weight (+ adapter) tile; the warp handles the
-    // ring items whose index has its parity.  Every lane runs the loop (uniform control flow), one elected lane
-    // issues the copies.
-    {
-      const int op = warp & 1, par = warp >> 1;
-      int it = 0;
-      bool ok = true;
-      // returns the slot, or -1 if the item belongs to the other warp pair
-      auto acquire = [&]() -> int {
-        const int my = ((it & 1) == par);
-        const int slot = it % S;
-        if (my) {
-          ok = mbar_wait(empty_bar(slot), ((it / S) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY);
-          ok = __all_sync(0xffffffffu, ok);
-        }
-        ++it;
-        return my ? slot : -1;
-      };
-      auto load_main = [&](int i, int kb) {
-        const int slot = acquire();
-        if (slot < 0 || !ok) return;
-        const PairTile tc = pair_tile(pair + i * G, p);
-        const int m0 = tc.m_idx * kPairBlockM + static_cast<int>(rank) * 128, n0 = tc.n_idx * BN, k0 = kb * kBlockK;
-        const uint32_t a_dst = ring + slot * kStage, b_dst = a_dst + 16384;
-        const uint32_t fb = map_to_cta(full_bar(slot), 0);
-        if (elect_one()) {
-          if (op == 0) {
-            if (rank == 0) mbar_arrive_expect_tx(full_bar(slot), 2 * 16384);
-            tma_load_2d_pair(a_dst, &tm_act, fb, k0, m0);
-          } else if (!kBwd) {
-            if (rank == 0) {
-              mbar_arrive_expect_tx(full_bar(slot), (BN + p.r_pad) * 128);
-              tma_load_2d_pair(b_dst, &tm_w0, fb, k0, n0);
-            } else {
-              tma_load_2d_pair(b_dst, &tm_w1, fb, k0, n0 + half);
-              tma_load_2d_pair(b_dst + (BN - half) * 128, &tm_side, fb, k0, 0);
-            }
+    // ring items whose index has its parity.  Ring position, phase and tile coordinates are carried as counters
+    // (no division in the loop); one lane polls, one elected lane issues.
+    const int op = warp & 1, par = warp >> 1;
+    int slot = 0, phase = 0, odd = 0;
+    bool ok = true;
+    // claims the next ring item; returns its slot or -1 when the item belongs to the other warp pair
+    auto acquire = [&]() -> int {
+      const int mine = (odd == par), cur = slot;
+      if (mine) ok = warp_wait(empty_bar(cur), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY, false, 20);
+      if (++slot == S) { slot = 0; phase ^= 1; }
+      odd ^= 1;
+      return mine ? cur : -1;
+    };
+    auto load_main = [&](int m0, int n0, int k0) {
+      const int cur = acquire();
+      if (cur < 0 || !ok) return;
+      const uint32_t a_dst = ring + cur * kStage, b_dst = a_dst + 16384;
+      const uint32_t fb = map_to_cta(full_bar(cur), 0);
+      if (elect_one()) {
+        if (op == 0) {
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), 2 * 16384);
+          tma_load_2d_pair(a_dst, &tm_act, fb, k0, m0);
+        } else if (!kBwd) {
+          if (rank == 0) {
+            mbar_arrive_expect_tx(full_bar(cur), (BN + p.r_pad) * 128);
+            tma_load_2d_pair(b_dst, &tm_w0, fb, k0, n0);
           } else {
-            if (rank == 0) mbar_arrive_expect_tx(full_bar(slot), 2 * (16384 + side_boxes * 1024));
-            const int nb = n0 + static_cast<int>(rank) * (BN >> 1);
-            tma_load_2d_pair(b_dst, &tm_w0, fb, nb, k0);
-            tma_load_2d_pair(b_dst + 8192, &tm_w0, fb, nb + 64, k0);
-            for (int b = 0; b < side_boxes; ++b)
-              tma_load_2d_pair(b_dst + 16384 + b * 1024, &tm_side, fb, static_cast<int>(rank) * (p.r_pad >> 1) + 8 * b, k0);
+            tma_load_2d_pair(b_dst, &tm_w1, fb, k0, n0 + half);
+            tma_load_2d_pair(b_dst + (BN - half) * 128, &tm_side, fb, k0, 0);
           }
+        } else {
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), 2 * (16384 + side_boxes * 1024));
+          const int nb = n0 + static_cast<int>(rank) * (BN >> 1);
+          tma_load_2d_pair(b_dst, &tm_w0, fb, nb, k0);
+          tma_load_2d_pair(b_dst + 8192, &tm_w0, fb, nb + 64, k0);
+          for (int b = 0; b < side_boxes; ++b)
+            tma_load_2d_pair(b_dst + 16384 + b * 1024, &tm_side, fb, static_cast<int>(rank) * (p.r_pad >> 1) + 8 * b, k0);
         }
-        __syncwarp();
-      };
-      auto load_tail = [&](int i) {
-        const int slot = acquire();
-        if (slot < 0 || !ok) return;
-        const PairTile tc = pair_tile(pair + i * G, p);
-        const int nb = tc.n_idx * BN + static_cast<int>(rank) * (BN >> 1);
-        const uint32_t b_dst = ring + slot * kStage + 16384;
-        const uint32_t fb = map_to_cta(full_bar(slot), 0);
-        if (elect_one()) {
-          if (op == 0) {
-            if (rank == 0) mbar_arrive(full_bar(slot));          // no activation tile in a rank-r item
-          } else if (!kBwd) {
-            if (rank == 0) mbar_arrive_expect_tx(full_bar(slot), BN * 128);
-            tma_load_2d_pair(b_dst, &tm_tail, fb, 0, nb);
-          } else {
-            if (rank == 0) mbar_arrive_expect_tx(full_bar(slot), 2 * 2 * p.r_pad * 128);
-            tma_load_2d_pair(b_dst, &tm_tail, fb, nb, 0);
-            tma_load_2d_pair(b_dst + 8192, &tm_tail, fb, nb + 64, 0);
-          }
-        }
-        __syncwarp();
-      };
-      for (int i = 0; i < n_my && ok; ++i) {
-        for (int kb = 0; kb < KB && ok; ++kb) {
-          if (i > 0 && kb == D) load_tail(i - 1);
-          if (ok) load_main(i, kb);
-        }
-        if (ok && i > 0 && D == KB) load_tail(i - 1);
       }
-      if (ok && n_my > 0) load_tail(n_my - 1);
+      __syncwarp();
+    };
+    auto load_tail = [&](int n0) {
+      const int cur = acquire();
+      if (cur < 0 || !ok) return;
+      const int nb = n0 + static_cast<int>(rank) * (BN >> 1);
+      const uint32_t b_dst = ring + cur * kStage + 16384;
+      const uint32_t fb = map_to_cta(full_bar(cur), 0);
+      if (elect_one()) {
+        if (op == 0) {
+          if (rank == 0) mbar_arrive(full_bar(cur));          // no activation tile in a rank-r item
+        } else if (!kBwd) {
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), BN * 128);
+          tma_load_2d_pair(b_dst, &tm_tail, fb, 0, nb);
+        } else {
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), 2 * 2 * p.r_pad * 128);
+          tma_load_2d_pair(b_dst, &tm_tail, fb, nb, 0);
+          tma_load_2d_pair(b_dst + 8192, &tm_tail, fb, nb + 64, 0);
+        }
+      }
+      __syncwarp();
+    };
+    int prev_n0 = 0;
+    for (int i = 0; i < n_my && ok; ++i) {
+      const PairTile tc = pair_tile(pair + i * G, p);
+      const int m0 = tc.m_idx * kPairBlockM + static_cast<int>(rank) * 128, n0 = tc.n_idx * BN;
+      for (int kb = 0; kb < KB && ok; ++kb) {
+        if (i > 0 && kb == D) load_tail(prev_n0);
+        if (ok) load_main(m0, n0, kb * kBlockK);
+      }
+      if (ok && i > 0 && D == KB) load_tail(prev_n0);
+      prev_n0 = n0;
     }
+    if (ok && n_my > 0) load_tail(prev_n0);
   } else if (warp == 4) {
     // ================================ MMA issuer (leader CTA only) ================================
-    // Whole warp of the leader CTA runs the loop; one elected lane issues every MMA and commit.
+    // Whole warp of the leader CTA runs the loop; one lane polls, one elected lane issues every MMA and commit.
+    // Descriptors are advanced by adding byte offsets (>> 4) to precomputed bases.
     if (rank == 0) {
       const uint32_t idesc_main = kBwd ? mma_idesc_bf16(256, BN, false, true) : mma_idesc_bf16(256, BN + p.r_pad, false, false);
       const uint32_t idesc_side = mma_idesc_bf16(256, p.r_pad, false, true);
       const uint32_t idesc_tail = mma_idesc_bf16(256, BN, false, kBwd);
-      int it = 0;
+      const uint64_t ad0 = smem_desc_sw128(ring, 16, 1024);
+      const uint64_t bd0 = kBwd ? smem_desc_sw128(ring + 16384, 8192, 1024) : smem_desc_sw128(ring + 16384, 16, 1024);
+      const uint64_t sd0 = smem_desc_noswizzle(ring + 32768, 128, 1024);
+      const uint64_t pd0 = smem_desc_sw128(staging, 16, 1024);
+      constexpr uint32_t kBStep = kBwd ? (2048 >> 4) : (32 >> 4);     // descriptor step per 16-wide k-step
+      int slot = 0, phase = 0;
       bool ok = true;
-      auto mma_main = [&](int i, int kb) {
-        const int buf = i & 1, use = i >> 1;
-        if (kb == 0) {
-          ok = mbar_wait_cluster(acc_empty(buf), (use & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_ACC_EMPTY);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) return;
-        }
-        const int slot = it % S;
-        ok = mbar_wait_cluster(full_bar(slot), (it / S) & 1, abort_flag, p.status, DEV_TIMEOUT_FULL);
-        ok = __all_sync(0xffffffffu, ok);
-        ++it;
+      auto next = [&]() { if (++slot == S) { slot = 0; phase ^= 1; } };
+      auto mma_main = [&](int buf, bool first_kb, bool last_kb) {
+        ok = warp_wait(full_bar(slot), phase, abort_flag, p.status, DEV_TIMEOUT_FULL, true, 0);
         if (!ok) return;
         tc_fence_after();
-        const uint32_t a_addr = ring + slot * kStage, b_addr = a_addr + 16384, s_addr = b_addr + 16384;
-        const uint32_t acc = tmem_base + buf * 256;
         if (elect_one()) {
+          const uint32_t so = static_cast<uint32_t>(slot * kStage) >> 4;
+          const uint32_t acc = tmem_base + buf * 256;
 #pragma unroll
           for (int ks = 0; ks < kBlockK / 16; ++ks) {
-            const uint32_t accum = (kb | ks) != 0 ? 1u : 0u;
-            const uint64_t ad = smem_desc_sw128(a_addr + ks * 32, 16, 1024);
-            if (!kBwd) {
-              mma_bf16_ss_pair(acc, ad, smem_desc_sw128(b_addr + ks * 32, 16, 1024), idesc_main, accum);
-            } else {
-              mma_bf16_ss_pair(acc, ad, smem_desc_sw128(b_addr + ks * 2048, 8192, 1024), idesc_main, accum);
-              mma_bf16_ss_pair(acc + BN, ad, smem_desc_noswizzle(s_addr + ks * 256, 128, 1024), idesc_side, accum);
-            }
+            const uint32_t accum = (!first_kb || ks != 0) ? 1u : 0u;
+            const uint64_t ad = ad0 + so + ks * 2;
+            mma_bf16_ss_pair(acc, ad, bd0 + so + ks * kBStep, idesc_main, accum);
+            if (kBwd) mma_bf16_ss_pair(acc + BN, ad, sd0 + so + ks * 16, idesc_side, accum);
           }
           mma_commit_pair(empty_bar(slot));
-          if (kb == KB - 1) mma_commit_pair(side_full(buf));
+          if (last_kb) mma_commit_pair(side_full(buf));
         }
         __syncwarp();
+        next();
       };
-      auto mma_tail = [&](int i) {
-        const int buf = i & 1, use = i >> 1;
-        ok = mbar_wait_cluster(ps_ready(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_PS);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) return;
-        const int slot = it % S;
-        ok = mbar_wait_cluster(full_bar(slot), (it / S) & 1, abort_flag, p.status, DEV_TIMEOUT_FULL);
-        ok = __all_sync(0xffffffffu, ok);
-        ++it;
+      auto mma_tail = [&](int buf, int use) {
+        ok = warp_wait(ps_ready(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_PS, true, 0);
+        if (ok) ok = warp_wait(full_bar(slot), phase, abort_flag, p.status, DEV_TIMEOUT_FULL, true, 0);
         if (!ok) return;
         tc_fence_after();
-        const uint32_t b_addr = ring + slot * kStage + 16384;
         if (elect_one()) {
-          for (int ks = 0; ks < p.r_pad / 16; ++ks) {
-            const uint64_t ad = smem_desc_sw128(staging + ks * 32, 16, 1024);
-            const uint64_t bd = kBwd ? smem_desc_sw128(b_addr + ks * 2048, 8192, 1024)
-                                     : smem_desc_sw128(b_addr + ks * 32, 16, 1024);
-            mma_bf16_ss_pair(tmem_base + buf * 256, ad, bd, idesc_tail, 1u);
-          }
+          const uint32_t so = static_cast<uint32_t>(slot * kStage) >> 4;
+          for (int ks = 0; ks < p.r_pad / 16; ++ks)
+            mma_bf16_ss_pair(tmem_base + buf * 256, pd0 + ks * 2, bd0 + so + ks * kBStep, idesc_tail, 1u);
           mma_commit_pair(empty_bar(slot));
           mma_commit_pair(acc_full(buf));
         }
         __syncwarp();
+        next();
       };
       for (int i = 0; i < n_my && ok; ++i) {
+        const int buf = i & 1, use = i >> 1;
+        ok = warp_wait(acc_empty(buf), (use & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_ACC_EMPTY, true, 0);
         for (int kb = 0; kb < KB && ok; ++kb) {
-          if (i > 0 && kb == D) mma_tail(i - 1);
-          if (ok) mma_main(i, kb);
+          if (i > 0 && kb == D) mma_tail(buf ^ 1, (i - 1) >> 1);
+          if (ok) mma_main(buf, kb == 0, kb == KB - 1);
         }
-        if (ok && i > 0 && D == KB) mma_tail(i - 1);
+        if (ok && i > 0 && D == KB) mma_tail(buf ^ 1, (i - 1) >> 1);
       }
-      if (ok && n_my > 0) mma_tail(n_my - 1);
+      if (ok && n_my > 0) mma_tail((n_my - 1) & 1, (n_my - 1) >> 1);
     }
   } else {
     // ================================ epilogue (128 threads per CTA) ================================
@@ -286,7 +270,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       const int m0 = tc.m_idx * kPairBlockM + static_cast<int>(rank) * 128, n0 = tc.n_idx * BN;
       const int buf = i & 1, use = i >> 1;
       if (e == 0) tma_store_wait_read<0>();
-      bool ok = mbar_wait(side_full(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_SIDE);
+      bool ok = warp_wait(side_full(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_SIDE, false, 64);
       if (named_bar_or(1, 128, !ok)) break;
       tc_fence_after();
       for (int c16 = 0; c16 < p.r_pad / 16; ++c16) {
@@ -311,7 +295,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       fence_proxy_async_smem();
       tc_fence_before();
       mbar_arrive_cluster(map_to_cta(ps_ready(buf), 0));
-      ok = mbar_wait(acc_full(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_ACC);
+      ok = warp_wait(acc_full(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_ACC, false, 32);
       if (named_bar_or(1, 128, !ok)) break;
       tc_fence_after();
       for (int c = 0; c < full_chunks; ++c) {

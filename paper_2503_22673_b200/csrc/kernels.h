@@ -25,6 +25,7 @@ struct GemmParams {
   int tiles_m, tiles_n, num_tiles, kblocks;
   int group_m;            // m-tiles per rasterisation band
   int stages;             // ring depth
+  int prefetch_dist;      // CTA-pair kernel: k-blocks by which L2 prefetches run ahead of the ring (0 = off)
   int tail_delay;         // main-loop k-blocks of the next tile issued before the previous tile's rank-r MMA
   float scale;
   __nv_bfloat16* rt_out;  // backward only: scale * (dY B)^T as bf16 [r_pad][ld_rt]; nullptr otherwise

@@ -83,6 +83,41 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+// One lane polls, the rest of the warp sleeps in the shuffle: waiting warps must not eat the issue slots of
+// the warp that feeds the tensor pipe.  `backoff_ns` > 0 adds a nanosleep between polls (long waits).
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status,
+                                          unsigned code, bool cluster_scope, unsigned backoff_ns) {
+  int ok = 1;
+  if ((threadIdx.x & 31) == 0) {
+    auto probe = [&]() {
+      uint32_t r;
+      if (cluster_scope) {
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(r) : "r"(bar), "r"(parity) : "memory");
+      } else {
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(r) : "r"(bar), "r"(parity) : "memory");
+      }
+      return r != 0;
+    };
+    if (!probe()) {
+      const long long t0 = clock64();
+      for (;;) {
+        if (probe()) break;
+        if (backoff_ns) __nanosleep(backoff_ns);
+        if (*abort_flag) { ok = 0; break; }
+        if (clock64() - t0 > kWaitLimitCycles) {
+          *abort_flag = 1;
+          atomicCAS(status, 0u, code | (static_cast<unsigned>(blockIdx.x) << 8));
+          ok = 0;
+          break;
+        }
+      }
+    }
+  }
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
 // ----------------------------------------------------------------------------------------
 // named barriers among a subset of warps
 // ----------------------------------------------------------------------------------------
@@ -127,6 +162,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const CUtensorMap
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
       ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(x), "r"(y)
       : "memory");
+}
+// bring a tile into L2 only (no shared-memory destination, no completion tracking)
+__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* m, int x, int y) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(reinterpret_cast<uint64_t>(m)),
+               "r"(x), "r"(y)
+               : "memory");
 }
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, uint32_t src_smem, int x, int y) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
