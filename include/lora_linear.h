@@ -81,7 +81,8 @@ typedef struct lora_kernel_config {
   int32_t db_feat_chunk;   /* features per CTA of the dB kernel (grad_feat_chunk is dA's)      */
   int32_t cta_group;       /* 1: one CTA per tile; 2: two CTAs (one TPC) share a 256-row tile  */
   int32_t dx_stages;       /* ring depth of the dX GEMM                                        */
-  int32_t prefetch_dist;   /* k-blocks by which L2 prefetches run ahead of the ring (pair GEMM)*/
+  int32_t prefetch_dist;   /* k-blocks by which L2 prefetches run ahead of the ring (0: unused)*/
+  int32_t db_stages;       /* ring depth of the dB kernel (grad_stages is dA's)                */
 } lora_kernel_config_t;
 
 /* Host-only: run the tile / split selector for a shape on a device with `num_sms` SMs.
@@ -149,15 +150,15 @@ int lora_linear_step_host(lora_plan_t* plan, const void* h_X, const void* W, con
  * they call in: code running under a memory pool that forbids cudaMalloc after start-up, real-time or
  * inference loops where an allocation would stall the device, and hosts that hand this library a fixed
  * memory budget.  No plan is needed (creating one allocates a status block).  Nothing in this call
- * allocates or frees: the partial sums, arrival counters and status word live in one static device array
+ * allocates or frees: the partial sums and status word live in one static device array
  * of lora_grad_contract_noalloc_max_scratch() bytes (8 MiB) that every GPU loading the library holds until
  * the process exits.
  *   - Shapes whose partial sums do not fit (roughly SMs/ceil(C/512) x r_pad x C x 4 bytes > 8 MiB) are
  *     rejected with LORA_ERR_WORKSPACE; C % 8 == 0, r in {8,...,64}, ld_rt % 8 == 0, T >= 1.
  *   - The first call on a device looks up the array's device address and raises the kernel's shared-memory
  *     limit; make that first call before any stream capture.  The current device is used.
- *   - All calls share the one array and it keeps the last call's contents; the call clears the counters
- *     it needs on `stream` first.  Two calls whose kernels overlap on the GPU (different streams, or
+ *   - All calls share the one array and it keeps the last call's contents; the call clears the status
+ *     words on `stream` first and rewrites every partial sum before reading it.  Two calls whose kernels overlap on the GPU (different streams, or
  *     different host threads) race on it: serialise them.
  *   - A bounded device wait that ran out is not reported by this call (there is no plan to ask). */
 int lora_grad_contract_noalloc(const void* S, const void* Rt, int64_t T, int64_t C, int64_t r, int64_t ld_rt,

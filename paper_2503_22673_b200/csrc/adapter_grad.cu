@@ -9,10 +9,13 @@
 // stream.  The dA kernel additionally recomputes X A^T for the slab it holds (same tiles, this time as the
 // K-major operand with M = 128 tokens), because the backward pass is not given the forward's X A^T.
 //
-// Grid: (feature chunks, token chunks).  A CTA keeps feat_chunk x r_pad fp32 sums in TMEM over all of its
-// token slabs.  Cross-CTA sums (over token chunks for the gradient, over feature chunks for X A^T) are
-// written as partials; the last CTA to arrive (a counter, no spinning) adds them in a fixed order, so the
-// result is bitwise reproducible.
+// Grid: (feature chunks, token chunks), at most one CTA per SM.  A CTA keeps feat_chunk x r_pad fp32 sums in
+// TMEM over all of its token slabs.  Cross-CTA sums (over token chunks for the gradient, over feature chunks
+// for X A^T) are written as fp32 partials and added in a fixed order by lora_grad_finalize_kernel, so the
+// result is bitwise reproducible and no CTA ever waits for another.
+//
+// Warps: 0, 1 TMA producers of the streamed tiles (even / odd ring items: one warp's copies sustain only
+// ~30 B/clk), 2 MMA issuer + TMEM, 3 loader of the second factor, 4..7 epilogue.
 #include "kernels.h"
 #include "sm100_ptx.cuh"
 
@@ -34,12 +37,11 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int NB = p.feat_chunk >> 7;                 // 128-feature accumulator blocks
-  const int rt_box = p.r_pad * 128;                 // bytes of one 64-token box of the second factor
+  const int rt_box = p.r_pad * 128;                 // bytes of one 64-wide box with r_pad rows
+  const int stage_bytes = kGradStageBytes + (p.with_p ? 2 * rt_box : 0);   // X tile (+ the matching A columns)
   const uint32_t ring = smem_u32(smem);
-  const uint32_t rt_base = ring + p.stages * kGradStageBytes;           // 2 buffers x 2 boxes
-  const uint32_t a_base = rt_base + 4 * rt_box;                          // feat_chunk/64 boxes of r_pad x 64
-  const int a_bytes = p.with_p ? (p.feat_chunk >> 6) * rt_box : 0;
-  uint8_t* tail = smem + p.stages * kGradStageBytes + 4 * rt_box + a_bytes;
+  const uint32_t rt_base = ring + p.stages * stage_bytes;               // 2 buffers x 2 boxes of the second factor
+  uint8_t* tail = smem + p.stages * stage_bytes + 4 * rt_box;
   uint64_t* bars = reinterpret_cast<uint64_t*>(tail);
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
@@ -48,11 +50,9 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
   auto rt_empty = [&](int b) { return bar0 + 8u * (2 * kGradMaxStages + 2 + b); };
   auto p_full = [&](int b) { return bar0 + 8u * (2 * kGradMaxStages + 4 + b); };
   auto p_empty = [&](int b) { return bar0 + 8u * (2 * kGradMaxStages + 6 + b); };
-  const uint32_t a_full = bar0 + 8u * (2 * kGradMaxStages + 8);
-  const uint32_t out_full = bar0 + 8u * (2 * kGradMaxStages + 9);
+  const uint32_t out_full = bar0 + 8u * (2 * kGradMaxStages + 8);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kGradBarriers);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  volatile int* last_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -73,18 +73,14 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
       mbar_init(p_full(b), 1);
       mbar_init(p_empty(b), 128);
     }
-    mbar_init(a_full, 1);
     mbar_init(out_full, 1);
     *abort_flag = 0;
-    *last_flag = 0;
     fence_barrier_init();
     tma_prefetch_desc(&tm_s);
     tma_prefetch_desc(&tm_r);
     if (p.with_p) tma_prefetch_desc(&tm_a);
-    if (blockIdx.x == 0 && blockIdx.y == 0 && p.zero_words != nullptr)
-      for (int i = 0; i < p.n_zero_words; ++i) p.zero_words[i] = 0u;
   }
-  if (warp == 1) {
+  if (warp == 2) {
     tmem_alloc(smem_u32(tmem_slot), 512);
     tmem_relinquish();
   }
@@ -94,90 +90,103 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_p = tmem_base + NB * p.r_pad;     // two r_pad-column buffers for X A^T
 
-  if (warp == 0) {
-    // ================================ TMA producer ================================
-    if (lane == 0) {
-      bool ok = true;
-      if (p.with_p) {
-        mbar_arrive_expect_tx(a_full, a_bytes);
-        for (int b = 0; b < (p.feat_chunk >> 6); ++b) tma_load_2d(a_base + b * rt_box, &tm_a, a_full, c0 + 64 * b, 0);
+  if (warp < 2) {
+    // ================================ TMA producers: streamed tiles, even / odd ring items ================================
+    int slot = 0, phase = 0, odd = 0;
+    bool ok = true;
+    for (int s = s_begin; s < s_end && ok; ++s) {
+      const int t0 = s * kGradSlab;
+      for (int nb = 0; nb < NB && ok; ++nb) {
+        if (odd == warp) {
+          ok = warp_wait(empty_bar(slot), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY, false, 20);
+          if (ok && elect_one()) {
+            const uint32_t dst = ring + slot * stage_bytes, fb = full_bar(slot);
+            const int cc = c0 + nb * 128;
+            mbar_arrive_expect_tx(fb, stage_bytes);
+            tma_load_2d(dst, &tm_s, fb, cc, t0);
+            tma_load_2d(dst + 16384, &tm_s, fb, cc + 64, t0);
+            if (p.with_p) {
+              tma_load_2d(dst + 32768, &tm_a, fb, cc, 0);
+              tma_load_2d(dst + 32768 + rt_box, &tm_a, fb, cc + 64, 0);
+            }
+          }
+          __syncwarp();
+        }
+        if (++slot == S) { slot = 0; phase ^= 1; }
+        odd ^= 1;
       }
-      int it = 0;
-      for (int s = s_begin; s < s_end && ok; ++s) {
-        const int ls = s - s_begin, rb = ls & 1, t0 = s * kGradSlab;
-        ok = mbar_wait(rt_empty(rb), ((ls >> 1) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY);
-        if (!ok) break;
+    }
+  } else if (warp == 3) {
+    // ================================ loader of the second factor (one 128-token slab at a time) ================================
+    bool ok = true;
+    int rb = 0, rphase = 0;
+    for (int s = s_begin; s < s_end && ok; ++s) {
+      ok = warp_wait(rt_empty(rb), rphase ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY, false, 20);
+      if (ok && elect_one()) {
+        const int t0 = s * kGradSlab;
         mbar_arrive_expect_tx(rt_full(rb), 2 * rt_box);
         tma_load_2d(rt_base + (2 * rb) * rt_box, &tm_r, rt_full(rb), t0, 0);
         tma_load_2d(rt_base + (2 * rb + 1) * rt_box, &tm_r, rt_full(rb), t0 + 64, 0);
-        for (int nb = 0; nb < NB && ok; ++nb) {
-          const int slot = it % S;
-          ok = mbar_wait(empty_bar(slot), ((it / S) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY);
-          ++it;
-          if (!ok) break;
-          const uint32_t dst = ring + slot * kGradStageBytes;
-          mbar_arrive_expect_tx(full_bar(slot), kGradStageBytes);
-          tma_load_2d(dst, &tm_s, full_bar(slot), c0 + nb * 128, t0);
-          tma_load_2d(dst + 16384, &tm_s, full_bar(slot), c0 + nb * 128 + 64, t0);
-        }
       }
+      __syncwarp();
+      if (++rb == 2) { rb = 0; rphase ^= 1; }
     }
-  } else if (warp == 1) {
+  } else if (warp == 2) {
     // ================================ MMA issuer ================================
-    if (lane == 0) {
-      const uint32_t idesc_out = mma_idesc_bf16(128, p.r_pad, true, false);   // A operand = S tile, MN-major
-      const uint32_t idesc_p = mma_idesc_bf16(128, p.r_pad, false, false);    // A operand = S tile, K-major
-      bool ok = true;
-      if (p.with_p) ok = mbar_wait(a_full, 0, abort_flag, p.status, DEV_TIMEOUT_FULL);
-      int it = 0;
-      for (int s = s_begin; s < s_end && ok; ++s) {
-        const int ls = s - s_begin, rb = ls & 1, use = ls >> 1;
-        ok = mbar_wait(rt_full(rb), use & 1, abort_flag, p.status, DEV_TIMEOUT_FULL);
-        if (ok && p.with_p) ok = mbar_wait(p_empty(rb), (use & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_ACC_EMPTY);
+    const uint32_t idesc_out = mma_idesc_bf16(128, p.r_pad, true, false);   // A operand = S tile, MN-major
+    const uint32_t idesc_p = mma_idesc_bf16(128, p.r_pad, false, false);    // A operand = S tile, K-major
+    const uint64_t a_mn0 = smem_desc_sw128(ring, 16384, 1024);              // S tile as [features x tokens]
+    const uint64_t a_k0 = smem_desc_sw128(ring, 16, 1024);                  // S tile as [tokens x features]
+    const uint64_t w_k0 = smem_desc_sw128(ring + 32768, 16, 1024);          // A columns of the stage
+    const uint64_t r_k0 = smem_desc_sw128(rt_base, 16, 1024);               // second factor
+    bool ok = true;
+    int slot = 0, phase = 0, rb = 0, rphase = 0;
+    for (int s = s_begin; s < s_end && ok; ++s) {
+      ok = warp_wait(rt_full(rb), rphase, abort_flag, p.status, DEV_TIMEOUT_FULL, false, 0);
+      if (ok && p.with_p) ok = warp_wait(p_empty(rb), rphase ^ 1, abort_flag, p.status, DEV_TIMEOUT_ACC_EMPTY, false, 0);
+      for (int nb = 0; nb < NB && ok; ++nb) {
+        ok = warp_wait(full_bar(slot), phase, abort_flag, p.status, DEV_TIMEOUT_FULL, false, 0);
         if (!ok) break;
-        for (int nb = 0; nb < NB && ok; ++nb) {
-          const int slot = it % S;
-          ok = mbar_wait(full_bar(slot), (it / S) & 1, abort_flag, p.status, DEV_TIMEOUT_FULL);
-          ++it;
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t tile = ring + slot * kGradStageBytes;
+        tc_fence_after();
+        if (elect_one()) {
+          const uint32_t so = static_cast<uint32_t>(slot * stage_bytes) >> 4;
+          const uint32_t ro = static_cast<uint32_t>(2 * rb * rt_box) >> 4;
+          const uint32_t rbox = static_cast<uint32_t>(rt_box) >> 4;
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {   // 128 tokens = 8 x K16
-            const uint64_t ad = smem_desc_sw128(tile + ks * 2048, 16384, 1024);
-            const uint64_t bd = smem_desc_sw128(rt_base + (2 * rb + (ks >> 2)) * rt_box + (ks & 3) * 32, 16, 1024);
-            mma_bf16_ss(tmem_base + nb * p.r_pad, ad, bd, idesc_out, (ls | ks) != 0 ? 1u : 0u);
-          }
+          for (int ks = 0; ks < 8; ++ks)     // 128 tokens = 8 x K16; second factor: box ks/4, 32 B per k-step
+            mma_bf16_ss(tmem_base + nb * p.r_pad, a_mn0 + so + ks * 128, r_k0 + ro + (ks >> 2) * rbox + (ks & 3) * 2,
+                        idesc_out, (s != s_begin || ks != 0) ? 1u : 0u);
           if (p.with_p) {
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) { // 128 features = 2 boxes x 4 x K16
-              const int bx = kk >> 2, ks = kk & 3;
-              const uint64_t ad = smem_desc_sw128(tile + bx * 16384 + ks * 32, 16, 1024);
-              const uint64_t bd = smem_desc_sw128(a_base + (nb * 2 + bx) * rt_box + ks * 32, 16, 1024);
-              mma_bf16_ss(tmem_p + rb * p.r_pad, ad, bd, idesc_p, (nb | kk) != 0 ? 1u : 0u);
-            }
+            for (int kk = 0; kk < 8; ++kk)   // 128 features = 2 boxes x 4 x K16
+              mma_bf16_ss(tmem_p + rb * p.r_pad, a_k0 + so + (kk >> 2) * 1024 + (kk & 3) * 2,
+                          w_k0 + so + (kk >> 2) * rbox + (kk & 3) * 2, idesc_p, (nb != 0 || kk != 0) ? 1u : 0u);
           }
           mma_commit(empty_bar(slot));
+          if (nb == NB - 1) {
+            mma_commit(rt_empty(rb));
+            if (p.with_p) mma_commit(p_full(rb));
+          }
         }
-        if (!ok) break;
-        mma_commit(rt_empty(rb));
-        if (p.with_p) mma_commit(p_full(rb));
+        __syncwarp();
+        if (++slot == S) { slot = 0; phase ^= 1; }
       }
-      if (ok) mma_commit(out_full);
+      if (++rb == 2) { rb = 0; rphase ^= 1; }
     }
+    if (ok && elect_one()) mma_commit(out_full);
+    __syncwarp();
   } else {
-    // ================================ epilogue (128 threads) ================================
-    const int e = threadIdx.x - 64;
+    // ================================ epilogue (warps 4..7, 128 threads) ================================
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
     const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
     bool alive = true;
     if (p.with_p) {
-      // ---- X A^T of each slab: partial over this CTA's features -> global; last CTA finishes it ----
+      // ---- X A^T of each slab, partial over this CTA's features -> p_part[fc][j][t] ----
+      int pb = 0, pphase = 0;
       for (int s = s_begin; s < s_end; ++s) {
-        const int ls = s - s_begin, pb = ls & 1, use = ls >> 1;
         const int t = s * kGradSlab + row;
-        bool ok = mbar_wait(p_full(pb), use & 1, abort_flag, p.status, DEV_TIMEOUT_SIDE);
+        bool ok = warp_wait(p_full(pb), pphase, abort_flag, p.status, DEV_TIMEOUT_SIDE, false, 32);
         if (named_bar_or(1, 128, !ok)) { alive = false; break; }
         tc_fence_after();
         for (int c16 = 0; c16 < p.r_pad / 16; ++c16) {
@@ -192,33 +201,14 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
         }
         tc_fence_before();
         mbar_arrive(p_empty(pb));
-        __threadfence();
-        named_bar_sync(2, 128);
-        if (e == 0) {
-          const unsigned old = atomicAdd(&p.slab_counters[s], 1u);
-          *last_flag = (old == static_cast<unsigned>(p.n_feat_chunks - 1)) ? 1 : 0;
-        }
-        named_bar_sync(2, 128);
-        const bool last = *last_flag != 0;
-        named_bar_sync(2, 128);          // everyone has read the flag before it is rewritten
-        if (last && t < p.T) {
-          __threadfence();
-          unsigned short* pt = reinterpret_cast<unsigned short*>(p.pt_out);
-          for (int j = 0; j < p.r_pad; ++j) {
-            float acc = 0.f;
-            for (int f = 0; f < p.n_feat_chunks; ++f)
-              acc += __ldcg(&p.p_part[(static_cast<size_t>(f) * p.r_pad + j) * p.ld_t + t]);
-            pt[static_cast<size_t>(j) * p.ld_t + t] =
-                static_cast<unsigned short>(pack_bf16x2(acc * p.scale, 0.f) & 0xFFFFu);
-          }
-        }
+        if (++pb == 2) { pb = 0; pphase ^= 1; }
       }
     }
     if (alive) {
-      bool ok = mbar_wait(out_full, 0, abort_flag, p.status, DEV_TIMEOUT_ACC);
+      bool ok = warp_wait(out_full, 0, abort_flag, p.status, DEV_TIMEOUT_ACC, false, 32);
       if (!named_bar_or(1, 128, !ok)) {
         tc_fence_after();
-        // ---- this CTA's sums over its token chunk -> partial buffer ----
+        // ---- this CTA's sums over its token chunk -> out_part[tc][j][c] ----
         for (int nb = 0; nb < NB; ++nb) {
           const int c = c0 + nb * 128 + row;
           for (int c16 = 0; c16 < p.r_pad / 16; ++c16) {
@@ -229,28 +219,6 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
 #pragma unroll
               for (int q = 0; q < 16; ++q)
                 p.out_part[(static_cast<size_t>(tc) * p.r_pad + c16 * 16 + q) * p.c_pad + c] = __uint_as_float(v[q]);
-            }
-          }
-        }
-        __threadfence();
-        named_bar_sync(2, 128);
-        if (e == 0) {
-          const unsigned old = atomicAdd(&p.feat_counters[fc], 1u);
-          *last_flag = (old == static_cast<unsigned>(p.n_token_chunks - 1)) ? 1 : 0;
-        }
-        named_bar_sync(2, 128);
-        if (*last_flag != 0) {
-          __threadfence();
-          // ---- fixed-order sum over the token chunks -> final gradient ----
-          for (int nb = 0; nb < NB; ++nb) {
-            const int c = c0 + nb * 128 + row;
-            if (c >= p.C) continue;
-            for (int j = 0; j < p.r; ++j) {
-              float acc = 0.f;
-              for (int k = 0; k < p.n_token_chunks; ++k)
-                acc += __ldcg(&p.out_part[(static_cast<size_t>(k) * p.r_pad + j) * p.c_pad + c]);
-              if (p.out_is_da) p.out[static_cast<size_t>(j) * p.C + c] = acc;
-              else p.out[static_cast<size_t>(c) * p.r + j] = acc;
             }
           }
         }
@@ -267,19 +235,42 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
     }
   }
   __syncthreads();
-  if (warp == 1) {
+  if (warp == 2) {
     __syncwarp();
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
   }
 }
 
+// Fixed-order sums of the partials:  out = sum over token chunks of out_part ;  Pt = bf16(scale * sum over feature
+// chunks of p_part).  One thread per output element, consecutive threads on consecutive addresses.
+__global__ void __launch_bounds__(256) lora_grad_finalize_kernel(const GradParams p) {
+  const long long n_out = static_cast<long long>(p.r) * p.C;
+  const long long n_pt = p.with_p ? static_cast<long long>(p.r_pad) * p.T : 0;
+  const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx < n_out) {
+    const int j = static_cast<int>(idx / p.C), c = static_cast<int>(idx - static_cast<long long>(j) * p.C);
+    float acc = 0.f;
+    for (int k = 0; k < p.n_token_chunks; ++k)
+      acc += __ldcg(&p.out_part[(static_cast<size_t>(k) * p.r_pad + j) * p.c_pad + c]);
+    if (p.out_is_da) p.out[static_cast<size_t>(j) * p.C + c] = acc;
+    else p.out[static_cast<size_t>(c) * p.r + j] = acc;
+  } else if (idx < n_out + n_pt) {
+    const long long i2 = idx - n_out;
+    const int j = static_cast<int>(i2 / p.T), t = static_cast<int>(i2 - static_cast<long long>(j) * p.T);
+    float acc = 0.f;
+    for (int f = 0; f < p.n_feat_chunks; ++f)
+      acc += __ldcg(&p.p_part[(static_cast<size_t>(f) * p.r_pad + j) * p.ld_t + t]);
+    reinterpret_cast<unsigned short*>(p.pt_out)[static_cast<size_t>(j) * p.ld_t + t] =
+        static_cast<unsigned short>(pack_bf16x2(acc * p.scale, 0.f) & 0xFFFFu);
+  }
+}
+
 }  // namespace
 
 size_t grad_smem_bytes(const GradParams& p) {
-  const size_t a_bytes = p.with_p ? static_cast<size_t>(p.feat_chunk >> 6) * p.r_pad * 128 : 0;
-  return static_cast<size_t>(p.stages) * kGradStageBytes + 4 * static_cast<size_t>(p.r_pad) * 128 + a_bytes +
-         kGradBarriers * 8 + 16 + 1024;
+  const size_t stage = kGradStageBytes + (p.with_p ? 2 * static_cast<size_t>(p.r_pad) * 128 : 0);
+  return static_cast<size_t>(p.stages) * stage + 4 * static_cast<size_t>(p.r_pad) * 128 + kGradBarriers * 8 + 16 + 1024;
 }
 
 cudaError_t grad_configure() {
@@ -290,6 +281,10 @@ cudaError_t launch_grad(const CUtensorMap& tmS, const CUtensorMap& tmR, const CU
                         cudaStream_t stream) {
   dim3 grid(p.n_feat_chunks, p.n_token_chunks);
   lora_grad_kernel<<<grid, kGradThreads, grad_smem_bytes(p), stream>>>(tmS, tmR, tmA, p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  const long long n = static_cast<long long>(p.r) * p.C + (p.with_p ? static_cast<long long>(p.r_pad) * p.T : 0);
+  lora_grad_finalize_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(p);
   return cudaGetLastError();
 }
 
@@ -298,10 +293,10 @@ cudaError_t launch_grad(const CUtensorMap& tmS, const CUtensorMap& tmR, const CU
 // ================================================================================================
 namespace {
 
-// Scratch held by every GPU that loads this library, until the process exits: one status block, the
-// arrival counters and the per-token-chunk partial sums of the contraction kernel.
+// Scratch held by every GPU that loads this library, until the process exits: one status block and the
+// per-token-chunk partial sums of the contraction kernel.
 constexpr size_t kNoAllocScratchBytes = 8u << 20;
-constexpr size_t kNoAllocHeaderBytes = 4096;     // [0,256) status words, [256,4096) arrival counters
+constexpr size_t kNoAllocHeaderBytes = 4096;     // [0,256) status words, rest reserved
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
 
 struct NoAllocDevice {
@@ -382,7 +377,7 @@ extern "C" int lora_grad_contract_noalloc(const void* S, const void* Rt, int64_t
   g.C = static_cast<int>(C);
   g.r = static_cast<int>(r);
   g.r_pad = static_cast<int>((r + 15) / 16 * 16);
-  int fc = g.r_pad <= 32 ? 512 : 256;
+  int fc = g.r_pad <= 32 ? 512 : 768;
   const int c128 = static_cast<int>((C + 127) / 128 * 128);
   if (fc > c128) fc = c128;
   g.feat_chunk = fc;
@@ -397,8 +392,7 @@ extern "C" int lora_grad_contract_noalloc(const void* S, const void* Rt, int64_t
   g.stages = stages > kGradMaxStages ? kGradMaxStages : stages;
   g.c_pad = static_cast<int>((C + 31) / 32 * 32);
   const size_t part_bytes = static_cast<size_t>(n_tok) * g.r_pad * g.c_pad * sizeof(float);
-  if (static_cast<size_t>(g.n_feat_chunks) * 4 > kNoAllocHeaderBytes - 256 ||
-      kNoAllocHeaderBytes + part_bytes > kNoAllocScratchBytes)
+  if (kNoAllocHeaderBytes + part_bytes > kNoAllocScratchBytes)
     return LORA_ERR_WORKSPACE;      // the problem needs more scratch than the static array holds
   g.with_p = 0;
   g.out_is_da = 0;
@@ -408,13 +402,10 @@ extern "C" int lora_grad_contract_noalloc(const void* S, const void* Rt, int64_t
   g.p_part = nullptr;
   g.pt_out = nullptr;
   g.ld_t = static_cast<int>(ld_rt);
-  g.slab_counters = nullptr;
-  g.feat_counters = reinterpret_cast<unsigned*>(nd.scratch + 256);
   g.status = reinterpret_cast<unsigned*>(nd.scratch);
-  g.zero_words = nullptr;
-  g.n_zero_words = 0;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // the array keeps the previous call's contents: the arrival counters (and status) must start at zero
+  // the array keeps the previous call's contents: the status words must start at zero (the partial sums are
+  // fully rewritten before they are read)
   if (cudaMemsetAsync(nd.scratch, 0, kNoAllocHeaderBytes, st) != cudaSuccess) return LORA_ERR_CUDA;
   CUtensorMap tmS, tmR;
   if (!noalloc_tmap(&tmS, S, static_cast<uint64_t>(C), static_cast<uint64_t>(T), static_cast<uint64_t>(C), 64, kGradSlab) ||

@@ -75,19 +75,20 @@ struct GradGrid {
 
 GradGrid pick_grad_grid(long long T, long long C, int r_pad, bool with_p, int num_sms) {
   GradGrid g;
-  int fc = (r_pad <= 32) ? 512 : 256;
+  // TMEM: (feat_chunk / 128) accumulator blocks of r_pad columns + two r_pad-column buffers for X A^T <= 512
+  int fc = (r_pad <= 32) ? 512 : 768;
   const int c128 = ceil_div(C, 128) * 128;
   if (fc > c128) fc = c128;
   g.feat_chunk = fc;
   g.n_feat = ceil_div(C, fc);
   const int n_slabs = ceil_div(T, kGradSlab);
-  int n_tok = (num_sms + g.n_feat / 2) / g.n_feat;
-  if (n_tok < 1) n_tok = 1;
+  int n_tok = num_sms / g.n_feat;             // at most one CTA per SM: a second wave would double the time
   if (n_tok > n_slabs) n_tok = n_slabs;
   if (n_tok < 1) n_tok = 1;
   g.n_tok = n_tok;
-  const size_t fixed = 4 * static_cast<size_t>(r_pad) * 128 + (with_p ? static_cast<size_t>(fc / 64) * r_pad * 128 : 0) + 4096;
-  int stages = static_cast<int>((232448 - fixed) / kGradStageBytes);
+  const size_t stage = kGradStageBytes + (with_p ? 2 * static_cast<size_t>(r_pad) * 128 : 0);
+  const size_t fixed = 4 * static_cast<size_t>(r_pad) * 128 + 2048;
+  int stages = static_cast<int>((232448 - fixed) / stage);
   if (stages > kGradMaxStages) stages = kGradMaxStages;
   if (stages < 2) stages = 2;
   g.stages = stages;
@@ -157,7 +158,8 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
   const GradGrid ga = pick_grad_grid(T, s->d_in, c->r_pad, true, num_sms);
   const GradGrid gb = pick_grad_grid(T, s->d_out, c->r_pad, false, num_sms);
   c->grad_feat_chunk = ga.feat_chunk;
-  c->grad_stages = ga.stages < gb.stages ? ga.stages : gb.stages;
+  c->grad_stages = ga.stages;
+  c->db_stages = gb.stages;
   c->da_feat_chunks = ga.n_feat;
   c->da_token_chunks = ga.n_tok;
   c->db_feat_chunks = gb.n_feat;
@@ -170,8 +172,8 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
 // backward workspace layout
 // ------------------------------------------------------------------------------------------------
 struct WsLayout {
-  size_t qt, pt, p_part, da_part, db_part, counters, total;
-  int ld_t, c_pad_a, c_pad_b, n_slabs, n_counters;
+  size_t qt, pt, p_part, da_part, db_part, total;
+  int ld_t, c_pad_a, c_pad_b, n_slabs;
 };
 
 WsLayout ws_layout(const lora_shape_t& s, const lora_kernel_config_t& c) {
@@ -181,14 +183,12 @@ WsLayout ws_layout(const lora_shape_t& s, const lora_kernel_config_t& c) {
   w.c_pad_a = static_cast<int>(align_up(static_cast<size_t>(s.d_in), 32));
   w.c_pad_b = static_cast<int>(align_up(static_cast<size_t>(s.d_out), 32));
   w.n_slabs = ceil_div(T, kGradSlab);
-  w.n_counters = w.n_slabs + c.da_feat_chunks + c.db_feat_chunks;
   size_t off = 0;
   w.qt = off;       off += align_up(static_cast<size_t>(c.r_pad) * w.ld_t * 2, kAlign);
   w.pt = off;       off += align_up(static_cast<size_t>(c.r_pad) * w.ld_t * 2, kAlign);
   w.p_part = off;   off += align_up(static_cast<size_t>(c.da_feat_chunks) * c.r_pad * w.ld_t * 4, kAlign);
   w.da_part = off;  off += align_up(static_cast<size_t>(c.da_token_chunks) * c.r_pad * w.c_pad_a * 4, kAlign);
   w.db_part = off;  off += align_up(static_cast<size_t>(c.db_token_chunks) * c.r_pad * w.c_pad_b * 4, kAlign);
-  w.counters = off; off += align_up(static_cast<size_t>(w.n_counters) * 4, kAlign);
   w.total = off;
   return w;
 }
@@ -299,8 +299,6 @@ int launch_fwd(lora_plan* pl, const void* X, const void* W, const void* A, const
   p.rt_out = nullptr;
   p.ld_rt = 0;
   p.status = pl->d_status;
-  p.zero_words = nullptr;
-  p.n_zero_words = 0;
   const cudaError_t le = pair ? launch_gemm_pair_fwd(tmX, tmW, tmW1, tmA, tmB, tmY, p, c.fwd_ctas, st)
                               : launch_gemm_fwd(tmX, tmW, tmA, tmB, tmY, p, c.fwd_ctas, st);
   if (le != cudaSuccess) return LORA_ERR_CUDA;
@@ -311,7 +309,6 @@ int launch_fwd(lora_plan* pl, const void* X, const void* W, const void* A, const
 struct WsPtrs {
   uint8_t* base;
   __nv_bfloat16 *qt, *pt;
-  unsigned* counters;
 };
 
 WsPtrs ws_ptrs(lora_plan* pl) {
@@ -319,11 +316,10 @@ WsPtrs ws_ptrs(lora_plan* pl) {
   q.base = static_cast<uint8_t*>(pl->workspace);
   q.qt = reinterpret_cast<__nv_bfloat16*>(q.base + pl->ws.qt);
   q.pt = reinterpret_cast<__nv_bfloat16*>(q.base + pl->ws.pt);
-  q.counters = reinterpret_cast<unsigned*>(q.base + pl->ws.counters);
   return q;
 }
 
-// ---- dX = dY W + s (dY B) A ; also leaves Qt = s (dY B)^T in the workspace and clears the counters ----
+// ---- dX = dY W + s (dY B) A ; also leaves Qt = s (dY B)^T in the workspace ----
 int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const void* B, float scale, void* dX,
               cudaStream_t st) {
   const lora_shape_t& s = pl->shape;
@@ -331,7 +327,6 @@ int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const
   const WsLayout& w = pl->ws;
   const WsPtrs q = ws_ptrs(pl);
   __nv_bfloat16* qt = q.qt;
-  unsigned* counters = q.counters;
   {
     CUtensorMap tmdY, tmW, tmB, tmA, tmdX;
     bool ok = make_bf16_tmap(&tmdY, dY, s.d_out, s.T, s.d_out, 64, kBlockM);
@@ -362,8 +357,6 @@ int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const
     p.rt_out = qt;
     p.ld_rt = w.ld_t;
     p.status = pl->d_status;
-    p.zero_words = counters;
-    p.n_zero_words = w.n_counters;
     const cudaError_t le = pair ? launch_gemm_pair_dx(tmdY, tmW, tmB, tmA, tmdX, p, c.dx_ctas, st)
                                 : launch_gemm_dx(tmdY, tmW, tmB, tmA, tmdX, p, c.dx_ctas, st);
     if (le != cudaSuccess) return LORA_ERR_CUDA;
@@ -380,7 +373,6 @@ int launch_da(lora_plan* pl, const void* X, const void* A, float scale, void* dA
   const WsPtrs q = ws_ptrs(pl);
   uint8_t* ws = q.base;
   __nv_bfloat16 *qt = q.qt, *pt = q.pt;
-  unsigned* counters = q.counters;
   {
     CUtensorMap tmS, tmR, tmA;
     bool ok = make_bf16_tmap(&tmS, X, s.d_in, s.T, s.d_in, 64, kGradSlab);
@@ -406,13 +398,9 @@ int launch_da(lora_plan* pl, const void* X, const void* A, float scale, void* dA
     g.p_part = reinterpret_cast<float*>(ws + w.p_part);
     g.pt_out = pt;
     g.ld_t = w.ld_t;
-    g.slab_counters = counters;
-    g.feat_counters = counters + w.n_slabs;
     g.status = pl->d_status;
-    g.zero_words = nullptr;
-    g.n_zero_words = 0;
     if (launch_grad(tmS, tmR, tmA, g, st) != cudaSuccess) return LORA_ERR_CUDA;
-    g_launches.fetch_add(1);
+    g_launches.fetch_add(2);
   }
   return LORA_OK;
 }
@@ -425,7 +413,6 @@ int launch_db(lora_plan* pl, const void* dY, float scale, void* dB, cudaStream_t
   const WsPtrs q = ws_ptrs(pl);
   uint8_t* ws = q.base;
   __nv_bfloat16* pt = q.pt;
-  unsigned* counters = q.counters;
   {
     CUtensorMap tmS, tmR;
     bool ok = make_bf16_tmap(&tmS, dY, s.d_out, s.T, s.d_out, 64, kGradSlab);
@@ -440,7 +427,7 @@ int launch_db(lora_plan* pl, const void* dY, float scale, void* dB, cudaStream_t
     g.n_feat_chunks = c.db_feat_chunks;
     g.n_token_chunks = c.db_token_chunks;
     g.n_slabs = w.n_slabs;
-    g.stages = c.grad_stages;
+    g.stages = c.db_stages;
     g.with_p = 0;
     g.out_is_da = 0;
     g.scale = scale;
@@ -450,13 +437,9 @@ int launch_db(lora_plan* pl, const void* dY, float scale, void* dB, cudaStream_t
     g.p_part = nullptr;
     g.pt_out = nullptr;
     g.ld_t = w.ld_t;
-    g.slab_counters = nullptr;
-    g.feat_counters = counters + w.n_slabs + c.da_feat_chunks;
     g.status = pl->d_status;
-    g.zero_words = nullptr;
-    g.n_zero_words = 0;
     if (launch_grad(tmS, tmR, tmR, g, st) != cudaSuccess) return LORA_ERR_CUDA;
-    g_launches.fetch_add(1);
+    g_launches.fetch_add(2);
   }
   return LORA_OK;
 }
@@ -558,12 +541,13 @@ int lora_plan_describe(const lora_plan_t* plan, char* buf, size_t n) {
   const lora_kernel_config_t& c = plan->cfg;
   std::snprintf(buf, n,
                 "T=%lld d_in=%lld d_out=%lld r=%lld | sms=%d cta_group=%d tile fwd %dx%dx64 dx %dx%dx64 stages=%d/%d group_m=%d "
-                "split_k=%d r_pad=%d ctas fwd=%d dx=%d tail_delay=%d | grad chunk=%d stages=%d dA grid=%dx%d dB grid=%dx%d "
+                "split_k=%d r_pad=%d ctas fwd=%d dx=%d tail_delay=%d | grad chunk=%d/%d stages=%d/%d dA grid=%dx%d dB grid=%dx%d "
                 "| bwd workspace=%zu B",
                 (long long)plan->shape.T, (long long)plan->shape.d_in, (long long)plan->shape.d_out,
                 (long long)plan->shape.r, plan->num_sms, c.cta_group, c.block_m, c.fwd_block_n, c.block_m, c.dx_block_n,
                 c.stages, c.dx_stages, c.group_m, c.split_k,
-                c.r_pad, c.fwd_ctas, c.dx_ctas, c.tail_delay, c.grad_feat_chunk, c.grad_stages, c.da_feat_chunks,
+                c.r_pad, c.fwd_ctas, c.dx_ctas, c.tail_delay, c.grad_feat_chunk, c.db_feat_chunk, c.grad_stages, c.db_stages,
+                c.da_feat_chunks,
                 c.da_token_chunks, c.db_feat_chunks, c.db_token_chunks, plan->ws.total);
   return LORA_OK;
 }

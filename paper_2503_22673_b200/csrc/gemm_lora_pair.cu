@@ -96,8 +96,6 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
     tma_prefetch_desc(&tm_side);
     tma_prefetch_desc(&tm_tail);
     tma_prefetch_desc(&tm_out);
-    if (blockIdx.x == 0 && p.zero_words != nullptr)
-      for (int i = 0; i < p.n_zero_words; ++i) p.zero_words[i] = 0u;
   }
   if (warp == 4) {
     tmem_alloc_pair(smem_u32(tmem_slot), 512);

@@ -31,8 +31,6 @@ struct GemmParams {
   __nv_bfloat16* rt_out;  // backward only: scale * (dY B)^T as bf16 [r_pad][ld_rt]; nullptr otherwise
   int ld_rt;
   unsigned* status;       // device status word
-  unsigned* zero_words;   // words this kernel clears for the kernels that follow it (may be null)
-  int n_zero_words;
   __nv_bfloat16* out;     // CTA-pair kernel only: output base and row pitch (elements) for the ragged last chunk
   int ld_out;
 };
@@ -66,7 +64,7 @@ cudaError_t launch_gemm_dx(const CUtensorMap& tmdY, const CUtensorMap& tmW, cons
 cudaError_t gemm_configure();   // opt in to the large dynamic shared memory (once per device)
 
 // ---- adapter gradients: tall-skinny contraction over tokens -----------------------------------
-constexpr int kGradThreads = 192;
+constexpr int kGradThreads = 256;          // warps 0,1 TMA producers, 2 MMA + TMEM, 3 second-factor loader, 4..7 epilogue
 constexpr int kGradSlab = 128;             // tokens per slab
 constexpr int kGradStageBytes = 2 * kBlockM * 128;   // 128 tokens x 128 features, bf16
 constexpr int kGradMaxStages = 6;
@@ -86,17 +84,14 @@ struct GradParams {
   float* p_part;          // [n_feat_chunks][r_pad][ld_t] partial X A^T (with_p)
   __nv_bfloat16* pt_out;  // [r_pad][ld_t]: scale * (X A^T)^T as bf16 (with_p)
   int ld_t;
-  unsigned* feat_counters;  // [n_feat_chunks] arrivals per feature chunk
-  unsigned* slab_counters;  // [n_slabs] arrivals per token slab (with_p)
   unsigned* status;
-  unsigned* zero_words;
-  int n_zero_words;
 };
 
 size_t grad_smem_bytes(const GradParams& p);
 cudaError_t grad_configure();
 // tmS: streamed matrix [T, C] box [64 features, 128 tokens]; tmR: [r_pad, T] box [64 tokens, r_pad];
-// tmA: A [r, C] box [64 features, r_pad] (only read when with_p)
+// tmA: A [r, C] box [64 features, r_pad] (only read when with_p).  Launches the streaming kernel and the
+// fixed-order finalize kernel (2 launches).
 cudaError_t launch_grad(const CUtensorMap& tmS, const CUtensorMap& tmR, const CUtensorMap& tmA,
                         const GradParams& p, cudaStream_t stream);
 

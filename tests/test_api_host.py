@@ -38,28 +38,47 @@ def test_strerror_and_launch_count():
 def test_selector_invariants(shape):
     T, d_in, d_out, r = shape
     c = binding.select_config(T, d_in, d_out, r, 148)
-    assert c["block_m"] == 128 and c["block_k"] == 64
+    assert c["block_k"] == 64
     assert c["r_pad"] % 16 == 0 and r <= c["r_pad"] < r + 16
-    for bn in (c["fwd_block_n"], c["dx_block_n"]):
-        assert bn in (64, 128, 192) and bn + c["r_pad"] <= 256          # one MMA covers tile + adapter columns
-    m_tiles = -(-T // 128)
-    assert 1 <= c["fwd_ctas"] <= min(148, m_tiles * -(-d_out // c["fwd_block_n"]))
-    assert 1 <= c["dx_ctas"] <= min(148, m_tiles * -(-d_in // c["dx_block_n"]))
-    assert c["stages"] * (128 * 128 + 256 * 128) + 2 * 16384 + 1024 + 256 <= 232448      # fits 227 KiB
+    assert c["cta_group"] == (2 if T > 128 else 1)
+    if c["cta_group"] == 2:
+        assert c["block_m"] == 256
+        for bn in (c["fwd_block_n"], c["dx_block_n"]):
+            assert bn % 16 == 0 and bn + c["r_pad"] <= 256        # tile + adapter columns fit one MMA / one TMEM buffer
+        units = 74                                                  # CTA pairs
+        per = 2
+        assert c["stages"] * 32768 + 2 * 16384 + 2048 <= 232448     # forward ring + staging fit 227 KiB
+        assert c["dx_stages"] * 36864 + 2 * 16384 + 2048 <= 232448
+    else:
+        assert c["block_m"] == 128
+        for bn in (c["fwd_block_n"], c["dx_block_n"]):
+            assert bn in (64, 128, 192) and bn + c["r_pad"] <= 256
+        units, per = 148, 1
+        assert c["stages"] * (128 * 128 + 256 * 128) + 2 * 16384 + 2048 <= 232448
+    m_tiles = -(-T // c["block_m"])
+    assert per <= c["fwd_ctas"] <= per * min(units, m_tiles * -(-d_out // c["fwd_block_n"]))
+    assert per <= c["dx_ctas"] <= per * min(units, m_tiles * -(-d_in // c["dx_block_n"]))
+    assert c["fwd_ctas"] % per == 0 and c["dx_ctas"] % per == 0
     assert c["split_k"] == 1
     n_slabs = -(-T // 128)
     assert 1 <= c["da_token_chunks"] <= n_slabs and 1 <= c["db_token_chunks"] <= n_slabs
-    fc = c["grad_feat_chunk"]
-    assert fc % 128 == 0 and (fc // 128) * c["r_pad"] + 2 * c["r_pad"] <= 512             # TMEM columns
-    assert c["da_feat_chunks"] == -(-d_in // fc)
-    assert 2 <= c["grad_stages"] <= 6
+    for fc, nf, nt, st, with_p in ((c["grad_feat_chunk"], c["da_feat_chunks"], c["da_token_chunks"], c["grad_stages"], 1),
+                                   (c["db_feat_chunk"], c["db_feat_chunks"], c["db_token_chunks"], c["db_stages"], 0)):
+        assert fc % 128 == 0 and (fc // 128) * c["r_pad"] + 2 * c["r_pad"] <= 512        # TMEM columns
+        assert nf * nt <= max(148, nf)                                                   # one wave of CTAs
+        assert 2 <= st <= 6
+        assert st * (32768 + with_p * 2 * c["r_pad"] * 128) + 4 * c["r_pad"] * 128 + 2048 <= 232448
+    assert c["da_feat_chunks"] == -(-d_in // c["grad_feat_chunk"])
+    assert c["db_feat_chunks"] == -(-d_out // c["db_feat_chunk"])
 
 
-def test_selector_prefers_narrow_tiles_on_small_grids():
-    small = binding.select_config(256, 512, 512, 8, 148)
+def test_selector_picks_by_grid_size():
+    small = binding.select_config(128, 512, 512, 8, 148)          # one 128-row tile: single-CTA kernel, narrow tiles
     big = binding.select_config(16384, 4096, 14336, 16, 148)
-    assert small["fwd_block_n"] == 64 and small["fwd_ctas"] == 16
-    assert big["fwd_block_n"] >= 128 and big["fwd_ctas"] == 148
+    assert small["cta_group"] == 1 and small["fwd_block_n"] == 64 and small["fwd_ctas"] == 8
+    assert big["cta_group"] == 2 and big["fwd_block_n"] == 240 and big["fwd_ctas"] == 148
+    kv = binding.select_config(32768, 4096, 1024, 16, 148)        # 1024 columns: 5 x 208 wastes less than 5 x 240
+    assert kv["fwd_block_n"] == 208
 
 
 @pytest.mark.parametrize("bad,code", [((128, 4100, 64, 16), binding.LORA_ERR_UNSUPPORTED_SHAPE),
