@@ -35,7 +35,7 @@ UNIT = "TFLOP/s"
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel from an
 # ncu capture summarised under profiles/; only valid for the kernel source it was taken on.
-NCU_TRAFFIC = {"gemm_sha": None, "bytes_per_launch": None}
+NCU_TRAFFIC = {"gemm_sha": "b693718445d8025a", "bytes_per_launch": {"fwd_gemm": 226.9e6, "dx_gemm": 225.0e6}}
 
 
 def peaks():
@@ -303,7 +303,8 @@ def run_ours(args):
                 "achieved": dom["tflops"], "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
                 "frac": dom["tflops"] / pk["bf16_tflops"], "peak_kind": f"bf16 burst, of {pk['source']}",
                 "ms_per_launch": dom["ms"],
-                "traffic": NCU_TRAFFIC["bytes_per_launch"] if NCU_TRAFFIC["gemm_sha"] == gemm_source_sha() else None}
+                "traffic": (NCU_TRAFFIC["bytes_per_launch"][dom_k] if NCU_TRAFFIC["gemm_sha"] == gemm_source_sha()
+                            and args.workload == 1 else None)}
 
     # ---- end to end: host buffers through the C ABI, copies inside the timed region ----
     h_sets, staging = [], []
