@@ -99,6 +99,21 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(value: float, device, world: int) -> float:
+    """Slowest rank's figure (all ranks must call it); identity for a single process."""
+    if world == 1:
+        return float(value)
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(world: int, flops_per_rank_step: float, ms_step: float) -> float:
+    """Whole-job TFLOP/s: every rank does one step's FLOPs in the slowest rank's time (replicas, weak scaling)."""
+    return world * flops_per_rank_step / ms_step / 1e9
+
+
 def dist_env():
     return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
 
@@ -273,12 +288,7 @@ def run_ours(args):
     barrier()
     launches = binding.launch_count() - launches0
     clocks = sampler.stop() if sampler is not None else None
-    ms_total = ev_a.elapsed_time(ev_b)
-    if world > 1:
-        import torch.distributed as dist
-        tmax = torch.tensor([ms_total], device=device)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms_total = float(tmax.item())
+    ms_total = max_over_ranks(ev_a.elapsed_time(ev_b), device, world)
     ms_step = ms_total / args.steps
 
     # per-kernel mean durations (ms) and rooflines
@@ -332,22 +342,17 @@ def run_ours(args):
     e_b.record()
     torch.cuda.synchronize()
     barrier()
-    ms_e2e = e_a.elapsed_time(e_b) / n_e2e
-    if world > 1:
-        import torch.distributed as dist
-        tm = torch.tensor([ms_e2e], device=device)
-        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-        ms_e2e = float(tm.item())
+    ms_e2e = max_over_ranks(e_a.elapsed_time(e_b) / n_e2e, device, world)
     h2d = sum(t.numel() * t.element_size() for h, _ in h_sets for t in h.values())
     d2h = sum(t.numel() * t.element_size() for _, ho in h_sets for t in ho.values())
-    e2e = {"value": world * flops_step / ms_e2e / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+    e2e = {"value": job_value(world, flops_step, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
            "ms_per_step": ms_e2e, "steps": n_e2e,
            "note": "host X, A, B, dY in; Y, dX, dA, dB out (pinned); frozen W resident on the device"}
 
     if rank != 0:
         return
     cpu = cpu_baseline(args.workload) if world == 1 and not args.no_cpu_baseline else None
-    value = world * flops_step / ms_step / 1e9
+    value = job_value(world, flops_step, ms_step)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": n_warm,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

@@ -1,0 +1,98 @@
+"""GPU parity at the full benchmark sizes, in the launch configuration bench.py times (default plan).
+
+The oracle cannot produce a full 16384 x 14336 output in seconds, so Y and dX are compared on sampled token rows
+(rows are independent: oracle.forward_rows / backward_dx_rows compute them one by one; every column tile is
+covered because whole rows are compared, and the sample holds the first and last row of the matrix, rows on both
+sides of tile borders and random ones).  dA and dB are compared in full.  Two adjoint identities that hold at
+any size are checked on the GPU outputs as a whole:  <dY, Y> = <dX, X>  and  <dA, A> = <dB, B>.
+
+Tolerances: max|gpu - ref| / max|ref| <= 2e-2 (Y, dX, bf16), <= 5e-3 (dA, dB, fp32).
+"""
+import gc
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import lora_oracle as oracle
+from paper_2503_22673_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 2e-2
+TOL_F32 = 5e-3
+
+
+def dev(bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).cuda()
+
+
+def host64(t):
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def sample_rows(T, n_random=40, seed=0):
+    fixed = [0, 1, 127, 128, 129, 255, 256, 257, 511, 512, T // 2 - 1, T // 2, T - 257, T - 256, T - 129, T - 128, T - 2, T - 1]
+    rng = np.random.default_rng(seed)
+    rows = sorted({r for r in fixed if 0 <= r < T} | set(rng.integers(0, T, n_random).tolist()))
+    return np.asarray(rows, dtype=np.int64)
+
+
+def dot64(a, b):
+    return float((a.double() * b.double()).sum().item())
+
+
+def check_projection(p, t, x_dev=None):
+    d = {k: dev(v) for k, v in t.items() if k != "X"}
+    d["X"] = x_dev if x_dev is not None else dev(t["X"])
+    plan = binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r)
+    Y = plan.fwd(d["X"], d["W"], d["A"], d["B"], p.scale)
+    dX, dA, dB = plan.bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], p.scale)
+    code, msg = plan.device_status()
+    assert code == 0, msg
+    rows = sample_rows(p.T)
+    W, A, B = (inputs.bf16_to_f64(t[k]) for k in ("W", "A", "B"))
+    rows_t = torch.from_numpy(rows).cuda()
+    # ---- sampled rows of Y and dX ----
+    Yr = oracle.forward_rows(np.arange(len(rows)), inputs.bf16_to_f64(t["X"][rows]), W, A, B, p.scale)
+    dXr = oracle.backward_dx_rows(np.arange(len(rows)), inputs.bf16_to_f64(t["dY"][rows]), W, A, B, p.scale)
+    eY = oracle.rel_err(host64(Y[rows_t]), Yr)
+    eX = oracle.rel_err(host64(dX[rows_t]), dXr)
+    del W
+    # ---- adapter gradients in full ----
+    Xf = inputs.bf16_to_f64(t["X"])
+    dYf = inputs.bf16_to_f64(t["dY"])
+    dAr, dBr = oracle.backward_adapter_grads(dYf, Xf, A, B, p.scale)
+    del Xf, dYf
+    eA = oracle.rel_err(host64(dA), dAr)
+    eB = oracle.rel_err(host64(dB), dBr)
+    # ---- identities on the complete GPU outputs ----
+    lhs, rhs = dot64(d["dY"], Y), dot64(dX, d["X"])
+    a, b = dot64(dA, d["A"]), dot64(dB, d["B"])
+    scale_yx = (d["dY"].double().norm() * Y.double().norm()).item()
+    plan.close()
+    errs = {"Y": eY, "dX": eX, "dA": eA, "dB": eB, "adjoint_yx": abs(lhs - rhs) / scale_yx,
+            "adjoint_ab": abs(a - b) / max(abs(a), abs(b), 1e-30)}
+    assert eY <= TOL_BF16 and eX <= TOL_BF16, (p.name, errs)
+    assert eA <= TOL_F32 and eB <= TOL_F32, (p.name, errs)
+    assert errs["adjoint_yx"] <= 1e-3, (p.name, errs)      # bf16 rounding of Y and dX averages out over T x d entries
+    assert errs["adjoint_ab"] <= 2e-2, (p.name, errs)      # both sides carry the bf16 rounding of s*P and s*Q
+    del d, Y, dX, dA, dB
+    gc.collect()
+    torch.cuda.empty_cache()
+    return errs
+
+
+@pytest.mark.parametrize("idx", [1, 2, 3])
+def test_single_projection_workloads_full_size(idx):
+    (p, t), = list(inputs.draw_workload(idx, seed=0))
+    check_projection(p, t)
+
+
+def test_seven_projection_layer_full_size():
+    x_dev = {}
+    for p, t in inputs.draw_workload(4, seed=0):
+        if p.x_group not in x_dev:
+            x_dev.clear()
+            x_dev[p.x_group] = dev(t["X"])
+        check_projection(p, t, x_dev[p.x_group])
