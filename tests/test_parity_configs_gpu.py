@@ -70,13 +70,16 @@ def check_projection(p, t, x_dev=None):
     lhs, rhs = dot64(d["dY"], Y), dot64(dX, d["X"])
     a, b = dot64(dA, d["A"]), dot64(dB, d["B"])
     scale_yx = (d["dY"].double().norm() * Y.double().norm()).item()
+    scale_ab = (dA.double().norm() * d["A"].double().norm() + dB.double().norm() * d["B"].double().norm()).item()
     plan.close()
     errs = {"Y": eY, "dX": eX, "dA": eA, "dB": eB, "adjoint_yx": abs(lhs - rhs) / scale_yx,
-            "adjoint_ab": abs(a - b) / max(abs(a), abs(b), 1e-30)}
+            "adjoint_ab": abs(a - b) / scale_ab}
     assert eY <= TOL_BF16 and eX <= TOL_BF16, (p.name, errs)
     assert eA <= TOL_F32 and eB <= TOL_F32, (p.name, errs)
     assert errs["adjoint_yx"] <= 1e-3, (p.name, errs)      # bf16 rounding of Y and dX averages out over T x d entries
-    assert errs["adjoint_ab"] <= 2e-2, (p.name, errs)      # both sides carry the bf16 rounding of s*P and s*Q
+    # both sides carry the bf16 rounding of s*P and s*Q; the inner products cancel heavily, so the difference is
+    # measured against the norms (Cauchy-Schwarz scale), not against the value itself
+    assert errs["adjoint_ab"] <= 5e-3, (p.name, errs)
     del d, Y, dX, dA, dB
     gc.collect()
     torch.cuda.empty_cache()
