@@ -83,6 +83,10 @@ typedef struct lora_kernel_config {
   int32_t dx_stages;       /* ring depth of the dX GEMM                                        */
   int32_t prefetch_dist;   /* k-blocks by which L2 prefetches run ahead of the ring (0: unused)*/
   int32_t db_stages;       /* ring depth of the dB kernel (grad_stages is dA's)                */
+  int32_t q_feat_chunk;    /* Q = dY B pre-pass (CTA-pair backward): features per CTA, grid, ring depth */
+  int32_t q_feat_chunks;
+  int32_t q_token_chunks;
+  int32_t q_stages;
 } lora_kernel_config_t;
 
 /* Host-only: run the tile / split selector for a shape on a device with `num_sms` SMs.

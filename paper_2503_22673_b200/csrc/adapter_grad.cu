@@ -14,6 +14,9 @@
 // for X A^T) are written as fp32 partials and added in a fixed order by lora_grad_finalize_kernel, so the
 // result is bitwise reproducible and no CTA ever waits for another.
 //
+// The side product has two operand forms: A [r, C] (K-major rows, for X A^T) or B [C, r] (MN-major, its natural
+// layout, for dY B); with do_out = 0 the kernel computes only the side product (the Q = dY B pre-pass of backward).
+//
 // Warps: 0, 1 TMA producers of the streamed tiles (even / odd ring items: one warp's copies sustain only
 // ~30 B/clk), 2 MMA issuer + TMEM, 3 loader of the second factor, 4..7 epilogue.
 #include "kernels.h"
@@ -32,13 +35,15 @@ constexpr int kGradBarriers = 2 * kGradMaxStages + 10;
 __global__ void __launch_bounds__(kGradThreads, 1)
 lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix [T, C], box 64(c) x 128(t)
                  const __grid_constant__ CUtensorMap tm_r,   // second factor [r_pad, T], box 64(t) x r_pad
-                 const __grid_constant__ CUtensorMap tm_a,   // A [r, C], box 64(c) x r_pad (with_p only)
+                 const __grid_constant__ CUtensorMap tm_a,   // side operand (with_p): A [r, C] box 64(c) x r_pad, or
+                                                             // B [C, r] box 64(r, zero-filled) x 64(c) when side_mn
                  const GradParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int NB = p.feat_chunk >> 7;                 // 128-feature accumulator blocks
   const int rt_box = p.r_pad * 128;                 // bytes of one 64-wide box with r_pad rows
-  const int stage_bytes = kGradStageBytes + (p.with_p ? 2 * rt_box : 0);   // X tile (+ the matching A columns)
+  const int side_box = p.side_mn ? 8192 : rt_box;   // bytes of the side operand for 64 features
+  const int stage_bytes = kGradStageBytes + (p.with_p ? 2 * side_box : 0);   // S tile (+ the matching side operand)
   const uint32_t ring = smem_u32(smem);
   const uint32_t rt_base = ring + p.stages * stage_bytes;               // 2 buffers x 2 boxes of the second factor
   uint8_t* tail = smem + p.stages * stage_bytes + 4 * rt_box;
@@ -88,7 +93,7 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_p = tmem_base + NB * p.r_pad;     // two r_pad-column buffers for X A^T
+  const uint32_t tmem_p = tmem_base + (p.do_out ? NB * p.r_pad : 0);     // two r_pad-column buffers for the side product
 
   if (warp < 2) {
     // ================================ TMA producers: streamed tiles, even / odd ring items ================================
@@ -105,9 +110,12 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
             mbar_arrive_expect_tx(fb, stage_bytes);
             tma_load_2d(dst, &tm_s, fb, cc, t0);
             tma_load_2d(dst + 16384, &tm_s, fb, cc + 64, t0);
-            if (p.with_p) {
+            if (p.with_p && !p.side_mn) {
               tma_load_2d(dst + 32768, &tm_a, fb, cc, 0);
-              tma_load_2d(dst + 32768 + rt_box, &tm_a, fb, cc + 64, 0);
+              tma_load_2d(dst + 32768 + side_box, &tm_a, fb, cc + 64, 0);
+            } else if (p.with_p) {
+              tma_load_2d(dst + 32768, &tm_a, fb, 0, cc);
+              tma_load_2d(dst + 32768 + side_box, &tm_a, fb, 0, cc + 64);
             }
           }
           __syncwarp();
@@ -120,7 +128,7 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
     // ================================ loader of the second factor (one 128-token slab at a time) ================================
     bool ok = true;
     int rb = 0, rphase = 0;
-    for (int s = s_begin; s < s_end && ok; ++s) {
+    for (int s = s_begin; s < s_end && ok && p.do_out; ++s) {
       ok = warp_wait(rt_empty(rb), rphase ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY, false, 20);
       if (ok && elect_one()) {
         const int t0 = s * kGradSlab;
@@ -134,15 +142,17 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
   } else if (warp == 2) {
     // ================================ MMA issuer ================================
     const uint32_t idesc_out = mma_idesc_bf16(128, p.r_pad, true, false);   // A operand = S tile, MN-major
-    const uint32_t idesc_p = mma_idesc_bf16(128, p.r_pad, false, false);    // A operand = S tile, K-major
+    const uint32_t idesc_p = mma_idesc_bf16(128, p.r_pad, false, p.side_mn != 0);   // A operand = S tile, K-major
     const uint64_t a_mn0 = smem_desc_sw128(ring, 16384, 1024);              // S tile as [features x tokens]
     const uint64_t a_k0 = smem_desc_sw128(ring, 16, 1024);                  // S tile as [tokens x features]
-    const uint64_t w_k0 = smem_desc_sw128(ring + 32768, 16, 1024);          // A columns of the stage
+    const uint64_t w_k0 = smem_desc_sw128(ring + 32768, 16, 1024);          // side operand of the stage
+    const uint32_t sbox = static_cast<uint32_t>(side_box) >> 4;
+    const uint32_t sstep = p.side_mn ? 128u : 2u;                           // descriptor step per 16 features
     const uint64_t r_k0 = smem_desc_sw128(rt_base, 16, 1024);               // second factor
     bool ok = true;
     int slot = 0, phase = 0, rb = 0, rphase = 0;
     for (int s = s_begin; s < s_end && ok; ++s) {
-      ok = warp_wait(rt_full(rb), rphase, abort_flag, p.status, DEV_TIMEOUT_FULL, false, 0);
+      if (p.do_out) ok = warp_wait(rt_full(rb), rphase, abort_flag, p.status, DEV_TIMEOUT_FULL, false, 0);
       if (ok && p.with_p) ok = warp_wait(p_empty(rb), rphase ^ 1, abort_flag, p.status, DEV_TIMEOUT_ACC_EMPTY, false, 0);
       for (int nb = 0; nb < NB && ok; ++nb) {
         ok = warp_wait(full_bar(slot), phase, abort_flag, p.status, DEV_TIMEOUT_FULL, false, 0);
@@ -152,19 +162,21 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
           const uint32_t so = static_cast<uint32_t>(slot * stage_bytes) >> 4;
           const uint32_t ro = static_cast<uint32_t>(2 * rb * rt_box) >> 4;
           const uint32_t rbox = static_cast<uint32_t>(rt_box) >> 4;
+          if (p.do_out) {
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks)     // 128 tokens = 8 x K16; second factor: box ks/4, 32 B per k-step
-            mma_bf16_ss(tmem_base + nb * p.r_pad, a_mn0 + so + ks * 128, r_k0 + ro + (ks >> 2) * rbox + (ks & 3) * 2,
-                        idesc_out, (s != s_begin || ks != 0) ? 1u : 0u);
+            for (int ks = 0; ks < 8; ++ks)   // 128 tokens = 8 x K16; second factor: box ks/4, 32 B per k-step
+              mma_bf16_ss(tmem_base + nb * p.r_pad, a_mn0 + so + ks * 128, r_k0 + ro + (ks >> 2) * rbox + (ks & 3) * 2,
+                          idesc_out, (s != s_begin || ks != 0) ? 1u : 0u);
+          }
           if (p.with_p) {
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk)   // 128 features = 2 boxes x 4 x K16
               mma_bf16_ss(tmem_p + rb * p.r_pad, a_k0 + so + (kk >> 2) * 1024 + (kk & 3) * 2,
-                          w_k0 + so + (kk >> 2) * rbox + (kk & 3) * 2, idesc_p, (nb != 0 || kk != 0) ? 1u : 0u);
+                          w_k0 + so + (kk >> 2) * sbox + (kk & 3) * sstep, idesc_p, (nb != 0 || kk != 0) ? 1u : 0u);
           }
           mma_commit(empty_bar(slot));
           if (nb == NB - 1) {
-            mma_commit(rt_empty(rb));
+            if (p.do_out) mma_commit(rt_empty(rb));
             if (p.with_p) mma_commit(p_full(rb));
           }
         }
@@ -173,7 +185,7 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
       }
       if (++rb == 2) { rb = 0; rphase ^= 1; }
     }
-    if (ok && elect_one()) mma_commit(out_full);
+    if (ok && p.do_out && elect_one()) mma_commit(out_full);
     __syncwarp();
   } else {
     // ================================ epilogue (warps 4..7, 128 threads) ================================
@@ -204,7 +216,7 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
         if (++pb == 2) { pb = 0; pphase ^= 1; }
       }
     }
-    if (alive) {
+    if (alive && p.do_out) {
       bool ok = warp_wait(out_full, 0, abort_flag, p.status, DEV_TIMEOUT_ACC, false, 32);
       if (!named_bar_or(1, 128, !ok)) {
         tc_fence_after();
@@ -242,25 +254,39 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
   }
 }
 
+// Sum of `n` floats spaced `stride` apart, added in index order; loads are issued eight at a time so that their
+// latencies overlap (the additions stay sequential, so the result does not depend on the batching).
+__device__ __forceinline__ float ordered_sum(const float* p, int n, size_t stride) {
+  float acc = 0.f;
+  int k = 0;
+  for (; k + 8 <= n; k += 8) {
+    float v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __ldcg(p + static_cast<size_t>(k + i) * stride);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc += v[i];
+  }
+  for (; k < n; ++k) acc += __ldcg(p + static_cast<size_t>(k) * stride);
+  return acc;
+}
+
 // Fixed-order sums of the partials:  out = sum over token chunks of out_part ;  Pt = bf16(scale * sum over feature
 // chunks of p_part).  One thread per output element, consecutive threads on consecutive addresses.
 __global__ void __launch_bounds__(256) lora_grad_finalize_kernel(const GradParams p) {
-  const long long n_out = static_cast<long long>(p.r) * p.C;
+  const long long n_out = p.do_out ? static_cast<long long>(p.r) * p.C : 0;
   const long long n_pt = p.with_p ? static_cast<long long>(p.r_pad) * p.T : 0;
   const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (idx < n_out) {
     const int j = static_cast<int>(idx / p.C), c = static_cast<int>(idx - static_cast<long long>(j) * p.C);
-    float acc = 0.f;
-    for (int k = 0; k < p.n_token_chunks; ++k)
-      acc += __ldcg(&p.out_part[(static_cast<size_t>(k) * p.r_pad + j) * p.c_pad + c]);
+    const float acc = ordered_sum(p.out_part + static_cast<size_t>(j) * p.c_pad + c, p.n_token_chunks,
+                                  static_cast<size_t>(p.r_pad) * p.c_pad);
     if (p.out_is_da) p.out[static_cast<size_t>(j) * p.C + c] = acc;
     else p.out[static_cast<size_t>(c) * p.r + j] = acc;
   } else if (idx < n_out + n_pt) {
     const long long i2 = idx - n_out;
     const int j = static_cast<int>(i2 / p.T), t = static_cast<int>(i2 - static_cast<long long>(j) * p.T);
-    float acc = 0.f;
-    for (int f = 0; f < p.n_feat_chunks; ++f)
-      acc += __ldcg(&p.p_part[(static_cast<size_t>(f) * p.r_pad + j) * p.ld_t + t]);
+    const float acc = ordered_sum(p.p_part + static_cast<size_t>(j) * p.ld_t + t, p.n_feat_chunks,
+                                  static_cast<size_t>(p.r_pad) * p.ld_t);
     reinterpret_cast<unsigned short*>(p.pt_out)[static_cast<size_t>(j) * p.ld_t + t] =
         static_cast<unsigned short>(pack_bf16x2(acc * p.scale, 0.f) & 0xFFFFu);
   }
@@ -269,7 +295,7 @@ __global__ void __launch_bounds__(256) lora_grad_finalize_kernel(const GradParam
 }  // namespace
 
 size_t grad_smem_bytes(const GradParams& p) {
-  const size_t stage = kGradStageBytes + (p.with_p ? 2 * static_cast<size_t>(p.r_pad) * 128 : 0);
+  const size_t stage = kGradStageBytes + (p.with_p ? 2 * (p.side_mn ? size_t(8192) : static_cast<size_t>(p.r_pad) * 128) : 0);
   return static_cast<size_t>(p.stages) * stage + 4 * static_cast<size_t>(p.r_pad) * 128 + kGradBarriers * 8 + 16 + 1024;
 }
 
@@ -283,7 +309,7 @@ cudaError_t launch_grad(const CUtensorMap& tmS, const CUtensorMap& tmR, const CU
   lora_grad_kernel<<<grid, kGradThreads, grad_smem_bytes(p), stream>>>(tmS, tmR, tmA, p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  const long long n = static_cast<long long>(p.r) * p.C + (p.with_p ? static_cast<long long>(p.r_pad) * p.T : 0);
+  const long long n = (p.do_out ? static_cast<long long>(p.r) * p.C : 0) + (p.with_p ? static_cast<long long>(p.r_pad) * p.T : 0);
   lora_grad_finalize_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(p);
   return cudaGetLastError();
 }
@@ -395,6 +421,8 @@ extern "C" int lora_grad_contract_noalloc(const void* S, const void* Rt, int64_t
   if (kNoAllocHeaderBytes + part_bytes > kNoAllocScratchBytes)
     return LORA_ERR_WORKSPACE;      // the problem needs more scratch than the static array holds
   g.with_p = 0;
+  g.side_mn = 0;
+  g.do_out = 1;
   g.out_is_da = 0;
   g.scale = 1.0f;
   g.out = static_cast<float*>(out);

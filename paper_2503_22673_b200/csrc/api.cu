@@ -130,9 +130,9 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
     const int pairs = num_sms / 2;
     c->block_m = kPairBlockM;
     c->fwd_block_n = pick_pair_block_n(T, s->d_out, c->r_pad, pairs);
-    c->dx_block_n = pick_pair_block_n(T, s->d_in, c->r_pad, pairs);
+    c->dx_block_n = pick_pair_block_n(T, s->d_in, 0, pairs);      // no adapter columns in the K-extended dX GEMM
     c->stages = 6;
-    c->dx_stages = 5;
+    c->dx_stages = 6;
     const long long fwd_t = static_cast<long long>(ceil_div(T, kPairBlockM)) * ceil_div(s->d_out, c->fwd_block_n);
     const long long dx_t = static_cast<long long>(ceil_div(T, kPairBlockM)) * ceil_div(s->d_in, c->dx_block_n);
     c->fwd_ctas = 2 * static_cast<int>(fwd_t < pairs ? fwd_t : pairs);
@@ -164,7 +164,20 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
   c->da_token_chunks = ga.n_tok;
   c->db_feat_chunks = gb.n_feat;
   c->db_token_chunks = gb.n_tok;
-  c->db_feat_chunk = gb.feat_chunk;   // feature chunk of the dB kernel (differs from dA's only for small d_out)
+  c->db_feat_chunk = gb.feat_chunk;
+  {  // Q = dY B pre-pass of the CTA-pair backward: side product only, so the feature chunk is not bound by TMEM
+    const int n_slabs = ceil_div(T, kGradSlab);
+    int nf = ceil_div(num_sms, n_slabs);
+    int fc = ceil_div(ceil_div(s->d_out, nf), 128) * 128;
+    nf = ceil_div(s->d_out, fc);
+    int nt = num_sms / nf;
+    if (nt > n_slabs) nt = n_slabs;
+    if (nt < 1) nt = 1;
+    c->q_feat_chunk = fc;
+    c->q_feat_chunks = nf;
+    c->q_token_chunks = nt;
+    c->q_stages = 4;
+  }   // feature chunk of the dB kernel (differs from dA's only for small d_out)
   return LORA_OK;
 }
 
@@ -172,7 +185,7 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
 // backward workspace layout
 // ------------------------------------------------------------------------------------------------
 struct WsLayout {
-  size_t qt, pt, p_part, da_part, db_part, total;
+  size_t qt, pt, q_part, p_part, da_part, db_part, total;
   int ld_t, c_pad_a, c_pad_b, n_slabs;
 };
 
@@ -186,6 +199,7 @@ WsLayout ws_layout(const lora_shape_t& s, const lora_kernel_config_t& c) {
   size_t off = 0;
   w.qt = off;       off += align_up(static_cast<size_t>(c.r_pad) * w.ld_t * 2, kAlign);
   w.pt = off;       off += align_up(static_cast<size_t>(c.r_pad) * w.ld_t * 2, kAlign);
+  w.q_part = off;   off += align_up(static_cast<size_t>(c.q_feat_chunks) * c.r_pad * w.ld_t * 4, kAlign);
   w.p_part = off;   off += align_up(static_cast<size_t>(c.da_feat_chunks) * c.r_pad * w.ld_t * 4, kAlign);
   w.da_part = off;  off += align_up(static_cast<size_t>(c.da_token_chunks) * c.r_pad * w.c_pad_a * 4, kAlign);
   w.db_part = off;  off += align_up(static_cast<size_t>(c.db_token_chunks) * c.r_pad * w.c_pad_b * 4, kAlign);
@@ -327,12 +341,39 @@ int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const
   const WsLayout& w = pl->ws;
   const WsPtrs q = ws_ptrs(pl);
   __nv_bfloat16* qt = q.qt;
+  if (c.cta_group == 2) {
+    // ---- pre-pass: Qt = s (dY B)^T, dY streamed once by the skinny kernel (side product only) ----
+    CUtensorMap tmS, tmSide;
+    bool ok = make_bf16_tmap(&tmS, dY, s.d_out, s.T, s.d_out, 64, kGradSlab);
+    ok = ok && make_bf16_tmap(&tmSide, B, s.r, s.d_out, s.r, 64, 64);
+    if (!ok) return LORA_ERR_CUDA;
+    GradParams g{};
+    g.T = static_cast<int>(s.T);
+    g.C = static_cast<int>(s.d_out);
+    g.r = static_cast<int>(s.r);
+    g.r_pad = c.r_pad;
+    g.feat_chunk = c.q_feat_chunk;
+    g.n_feat_chunks = c.q_feat_chunks;
+    g.n_token_chunks = c.q_token_chunks;
+    g.n_slabs = w.n_slabs;
+    g.stages = c.q_stages;
+    g.with_p = 1;
+    g.side_mn = 1;
+    g.do_out = 0;
+    g.scale = scale;
+    g.p_part = reinterpret_cast<float*>(q.base + w.q_part);
+    g.pt_out = qt;
+    g.ld_t = w.ld_t;
+    g.status = pl->d_status;
+    if (launch_grad(tmS, tmS, tmSide, g, st) != cudaSuccess) return LORA_ERR_CUDA;
+    g_launches.fetch_add(2);
+  }
   {
     CUtensorMap tmdY, tmW, tmB, tmA, tmdX;
     bool ok = make_bf16_tmap(&tmdY, dY, s.d_out, s.T, s.d_out, 64, kBlockM);
     ok = ok && make_bf16_tmap(&tmW, W, s.d_in, s.d_out, s.d_in, 64, 64);
     const bool pair = c.cta_group == 2;
-    if (pair) ok = ok && make_bf16_tmap(&tmB, B, s.r, s.d_out, s.r, 8, 64, false);   // unswizzled 8-column boxes
+    if (pair) ok = ok && make_bf16_tmap(&tmB, qt, s.T, c.r_pad, w.ld_t, 64, c.r_pad);   // Qt from the pre-pass below
     else ok = ok && make_bf16_tmap(&tmB, B, s.r, s.d_out, s.r, 64, 64);
     ok = ok && make_bf16_tmap(&tmA, A, s.d_in, s.r, s.d_in, 64, c.r_pad);
     ok = ok && make_bf16_tmap(&tmdX, dX, s.d_in, s.T, s.d_in, 64, kBlockM);
@@ -354,7 +395,7 @@ int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const
     p.tail_delay = c.tail_delay;
     p.prefetch_dist = c.prefetch_dist;
     p.scale = scale;
-    p.rt_out = qt;
+    p.rt_out = pair ? nullptr : qt;     // the single-CTA kernel computes Q itself and hands it on
     p.ld_rt = w.ld_t;
     p.status = pl->d_status;
     const cudaError_t le = pair ? launch_gemm_pair_dx(tmdY, tmW, tmB, tmA, tmdX, p, c.dx_ctas, st)
@@ -390,6 +431,8 @@ int launch_da(lora_plan* pl, const void* X, const void* A, float scale, void* dA
     g.n_slabs = w.n_slabs;
     g.stages = c.grad_stages;
     g.with_p = 1;
+    g.side_mn = 0;
+    g.do_out = 1;
     g.out_is_da = 1;
     g.scale = scale;
     g.out = static_cast<float*>(dA);
@@ -429,6 +472,8 @@ int launch_db(lora_plan* pl, const void* dY, float scale, void* dB, cudaStream_t
     g.n_slabs = w.n_slabs;
     g.stages = c.db_stages;
     g.with_p = 0;
+    g.side_mn = 0;
+    g.do_out = 1;
     g.out_is_da = 0;
     g.scale = scale;
     g.out = static_cast<float*>(dB);

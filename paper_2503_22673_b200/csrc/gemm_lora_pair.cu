@@ -23,8 +23,10 @@
 //   acc_empty[b] leader's; 256 arrivals: both epilogues have drained accumulator b
 // Forward: the weight/adapter rows of a tile are K-major and contiguous, so ONE MMA of width block_n + r_pad
 // gives the dense accumulator and P side by side (leader holds rows [0, half), peer the rest incl. A).
-// Backward: W, B, A are MN-major operands in their natural layout; Q = dY B is a second, narrow MMA per k-step
-// whose B operand (r_pad/2 columns per CTA) uses the unswizzled 8 x 16-byte core-matrix layout.
+// Backward: W and A are MN-major operands in their natural layout (no transposed weight copy).  s (dY B)^T is
+// computed beforehand by the skinny streaming kernel (narrow side MMAs in the main loop cost ~40 cycles each
+// whatever their width), so the tile is a plain K-extended GEMM: after the d_out/64 main k-blocks one more
+// k-block of depth r_pad multiplies the Qt tile (MN-major A operand, straight from TMA) with the rows of A.
 #include "kernels.h"
 #include "sm100_ptx.cuh"
 
@@ -52,7 +54,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M, K], box 64(k) x 128
                       const __grid_constant__ CUtensorMap tm_w0,    // fwd: W box 64(k) x half ; bwd: W box 64(n) x 64(k)
                       const __grid_constant__ CUtensorMap tm_w1,    // fwd: W box 64(k) x (block_n - half) ; bwd unused
-                      const __grid_constant__ CUtensorMap tm_side,  // fwd: A box 64(k) x r_pad ; bwd: B unswizzled box 8(r) x 64(k)
+                      const __grid_constant__ CUtensorMap tm_side,  // fwd: A box 64(k) x r_pad ; bwd: Qt [r_pad, T] box 64(t) x r_pad
                       const __grid_constant__ CUtensorMap tm_tail,  // fwd: B box 64(r) x block_n/2 ; bwd: A box 64(n) x r_pad
                       const __grid_constant__ CUtensorMap tm_out,   // Y / dX [M, N], box 64 x 128
                       const GemmParams p) {
@@ -115,7 +117,6 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
   const int S = p.stages;
   const int BN = p.block_n;
   const int half = (BN + p.r_pad) >> 1;         // forward: weight/adapter rows held by each CTA
-  const int side_boxes = p.r_pad >> 4;          // backward: 8-column unswizzled boxes of B per CTA
 
   if (warp < 4) {
     // ================================ TMA producers (both CTAs) ================================
@@ -151,25 +152,30 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
             tma_load_2d_pair(b_dst + (BN - half) * 128, &tm_side, fb, k0, 0);
           }
         } else {
-          if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), 2 * (16384 + side_boxes * 1024));
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), 2 * 16384);
           const int nb = n0 + static_cast<int>(rank) * (BN >> 1);
           tma_load_2d_pair(b_dst, &tm_w0, fb, nb, k0);
           tma_load_2d_pair(b_dst + 8192, &tm_w0, fb, nb + 64, k0);
-          for (int b = 0; b < side_boxes; ++b)
-            tma_load_2d_pair(b_dst + 16384 + b * 1024, &tm_side, fb, static_cast<int>(rank) * (p.r_pad >> 1) + 8 * b, k0);
         }
       }
       __syncwarp();
     };
-    auto load_tail = [&](int n0) {
+    auto load_tail = [&](int m0, int n0) {
       const int cur = acquire();
       if (cur < 0 || !ok) return;
       const int nb = n0 + static_cast<int>(rank) * (BN >> 1);
-      const uint32_t b_dst = ring + cur * kStage + 16384;
+      const uint32_t a_dst = ring + cur * kStage, b_dst = a_dst + 16384;
       const uint32_t fb = map_to_cta(full_bar(cur), 0);
       if (elect_one()) {
         if (op == 0) {
-          if (rank == 0) mbar_arrive(full_bar(cur));          // no activation tile in a rank-r item
+          if (!kBwd) {
+            if (rank == 0) mbar_arrive(full_bar(cur));        // forward: the rank-r operand comes from the epilogue
+          } else {
+            // backward: s (dY B)^T for this CTA's 128 tokens, two 64-token groups of r_pad rows (MN-major A operand)
+            if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), 2 * 2 * p.r_pad * 128);
+            tma_load_2d_pair(a_dst, &tm_side, fb, m0, 0);
+            tma_load_2d_pair(a_dst + p.r_pad * 128, &tm_side, fb, m0 + 64, 0);
+          }
         } else if (!kBwd) {
           if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), BN * 128);
           tma_load_2d_pair(b_dst, &tm_tail, fb, 0, nb);
@@ -181,30 +187,34 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       }
       __syncwarp();
     };
+    // Item order.  Forward: the rank-r item of tile i-1 comes D k-blocks into tile i (its operand is made by the
+    // epilogue meanwhile).  Backward: the rank-r item is simply the last k-block of its own tile.
     int prev_n0 = 0;
     for (int i = 0; i < n_my && ok; ++i) {
       const PairTile tc = pair_tile(pair + i * G, p);
       const int m0 = tc.m_idx * kPairBlockM + static_cast<int>(rank) * 128, n0 = tc.n_idx * BN;
       for (int kb = 0; kb < KB && ok; ++kb) {
-        if (i > 0 && kb == D) load_tail(prev_n0);
+        if (!kBwd && i > 0 && kb == D) load_tail(0, prev_n0);
         if (ok) load_main(m0, n0, kb * kBlockK);
       }
-      if (ok && i > 0 && D == KB) load_tail(prev_n0);
+      if (!kBwd && ok && i > 0 && D == KB) load_tail(0, prev_n0);
+      if (kBwd && ok) load_tail(m0, n0);
       prev_n0 = n0;
     }
-    if (ok && n_my > 0) load_tail(prev_n0);
+    if (!kBwd && ok && n_my > 0) load_tail(0, prev_n0);
   } else if (warp == 4) {
     // ================================ MMA issuer (leader CTA only) ================================
     // Whole warp of the leader CTA runs the loop; one lane polls, one elected lane issues every MMA and commit.
     // Descriptors are advanced by adding byte offsets (>> 4) to precomputed bases.
     if (rank == 0) {
       const uint32_t idesc_main = kBwd ? mma_idesc_bf16(256, BN, false, true) : mma_idesc_bf16(256, BN + p.r_pad, false, false);
-      const uint32_t idesc_side = mma_idesc_bf16(256, p.r_pad, false, true);
-      const uint32_t idesc_tail = mma_idesc_bf16(256, BN, false, kBwd);
+      const uint32_t idesc_tail = mma_idesc_bf16(256, BN, kBwd, kBwd);   // backward: Qt and A are both MN-major
       const uint64_t ad0 = smem_desc_sw128(ring, 16, 1024);
       const uint64_t bd0 = kBwd ? smem_desc_sw128(ring + 16384, 8192, 1024) : smem_desc_sw128(ring + 16384, 16, 1024);
-      const uint64_t sd0 = smem_desc_noswizzle(ring + 32768, 128, 1024);
-      const uint64_t pd0 = smem_desc_sw128(staging, 16, 1024);
+      // rank-r A operand: forward = bf16 s*P rows written by the epilogue (K-major, in the staging buffer);
+      // backward = Qt tile delivered by TMA into the stage's activation part (MN-major, two 64-token groups)
+      const uint64_t pd0 = kBwd ? smem_desc_sw128(ring, p.r_pad * 128, 1024) : smem_desc_sw128(staging, 16, 1024);
+      constexpr uint32_t kPStep = kBwd ? (2048 >> 4) : (32 >> 4);
       constexpr uint32_t kBStep = kBwd ? (2048 >> 4) : (32 >> 4);     // descriptor step per 16-wide k-step
       int slot = 0, phase = 0;
       bool ok = true;
@@ -221,23 +231,22 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
             const uint32_t accum = (!first_kb || ks != 0) ? 1u : 0u;
             const uint64_t ad = ad0 + so + ks * 2;
             mma_bf16_ss_pair(acc, ad, bd0 + so + ks * kBStep, idesc_main, accum);
-            if (kBwd) mma_bf16_ss_pair(acc + BN, ad, sd0 + so + ks * 16, idesc_side, accum);
           }
           mma_commit_pair(empty_bar(slot));
-          if (last_kb) mma_commit_pair(side_full(buf));
+          if (!kBwd && last_kb) mma_commit_pair(side_full(buf));
         }
         __syncwarp();
         next();
       };
       auto mma_tail = [&](int buf, int use) {
-        ok = warp_wait(ps_ready(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_PS, true, 0);
+        if (!kBwd) ok = warp_wait(ps_ready(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_PS, true, 0);
         if (ok) ok = warp_wait(full_bar(slot), phase, abort_flag, p.status, DEV_TIMEOUT_FULL, true, 0);
         if (!ok) return;
         tc_fence_after();
         if (elect_one()) {
           const uint32_t so = static_cast<uint32_t>(slot * kStage) >> 4;
           for (int ks = 0; ks < p.r_pad / 16; ++ks)
-            mma_bf16_ss_pair(tmem_base + buf * 256, pd0 + ks * 2, bd0 + so + ks * kBStep, idesc_tail, 1u);
+            mma_bf16_ss_pair(tmem_base + buf * 256, pd0 + (kBwd ? so : 0u) + ks * kPStep, bd0 + so + ks * kBStep, idesc_tail, 1u);
           mma_commit_pair(empty_bar(slot));
           mma_commit_pair(acc_full(buf));
         }
@@ -248,12 +257,13 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
         const int buf = i & 1, use = i >> 1;
         ok = warp_wait(acc_empty(buf), (use & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_ACC_EMPTY, true, 0);
         for (int kb = 0; kb < KB && ok; ++kb) {
-          if (i > 0 && kb == D) mma_tail(buf ^ 1, (i - 1) >> 1);
+          if (!kBwd && i > 0 && kb == D) mma_tail(buf ^ 1, (i - 1) >> 1);
           if (ok) mma_main(buf, kb == 0, kb == KB - 1);
         }
-        if (ok && i > 0 && D == KB) mma_tail(buf ^ 1, (i - 1) >> 1);
+        if (!kBwd && ok && i > 0 && D == KB) mma_tail(buf ^ 1, (i - 1) >> 1);
+        if (kBwd && ok) mma_tail(buf, use);
       }
-      if (ok && n_my > 0) mma_tail((n_my - 1) & 1, (n_my - 1) >> 1);
+      if (!kBwd && ok && n_my > 0) mma_tail((n_my - 1) & 1, (n_my - 1) >> 1);
     }
   } else {
     // ================================ epilogue (128 threads per CTA) ================================
@@ -267,32 +277,37 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       const PairTile tc = pair_tile(pair + i * G, p);
       const int m0 = tc.m_idx * kPairBlockM + static_cast<int>(rank) * 128, n0 = tc.n_idx * BN;
       const int buf = i & 1, use = i >> 1;
-      if (e == 0) tma_store_wait_read<0>();
-      bool ok = warp_wait(side_full(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_SIDE, false, 64);
-      if (named_bar_or(1, 128, !ok)) break;
-      tc_fence_after();
-      for (int c16 = 0; c16 < p.r_pad / 16; ++c16) {
-        uint32_t v[16];
-        tmem_ld16(lane_addr + buf * 256 + BN + c16 * 16, v);
-        tmem_ld_wait();
-        uint32_t w[8];
+      bool ok = true;
+      if (e == 0) tma_store_wait_read<0>();       // the previous tile's stores have left both staging buffers
+      if (!kBwd) {
+        // ---- forward: P = X A^T from TMEM -> scale -> bf16 -> shared memory as the rank-r MMA operand ----
+        ok = warp_wait(side_full(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_SIDE, false, 64);
+        if (named_bar_or(1, 128, !ok)) break;
+        tc_fence_after();
+        for (int c16 = 0; c16 < p.r_pad / 16; ++c16) {
+          uint32_t v[16];
+          tmem_ld16(lane_addr + buf * 256 + BN + c16 * 16, v);
+          tmem_ld_wait();
+          uint32_t w[8];
 #pragma unroll
-        for (int q = 0; q < 8; ++q)
-          w[q] = pack_bf16x2(__uint_as_float(v[2 * q]) * p.scale, __uint_as_float(v[2 * q + 1]) * p.scale);
-        *reinterpret_cast<uint4*>(staging_ptr + sw128_offset(row, 2 * c16)) = make_uint4(w[0], w[1], w[2], w[3]);
-        *reinterpret_cast<uint4*>(staging_ptr + sw128_offset(row, 2 * c16 + 1)) = make_uint4(w[4], w[5], w[6], w[7]);
-        if (kBwd && p.rt_out != nullptr && tc.n_idx == 0 && m0 + row < p.M) {
-          unsigned short* rt = reinterpret_cast<unsigned short*>(p.rt_out);
+          for (int q = 0; q < 8; ++q)
+            w[q] = pack_bf16x2(__uint_as_float(v[2 * q]) * p.scale, __uint_as_float(v[2 * q + 1]) * p.scale);
+          *reinterpret_cast<uint4*>(staging_ptr + sw128_offset(row, 2 * c16)) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(staging_ptr + sw128_offset(row, 2 * c16 + 1)) = make_uint4(w[4], w[5], w[6], w[7]);
+          if (p.rt_out != nullptr && tc.n_idx == 0 && m0 + row < p.M) {
+            // keep s (X A^T)^T for a backward pass that reuses it
+            unsigned short* rt = reinterpret_cast<unsigned short*>(p.rt_out);
 #pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            rt[static_cast<size_t>(c16 * 16 + 2 * q) * p.ld_rt + m0 + row] = static_cast<unsigned short>(w[q] & 0xFFFFu);
-            rt[static_cast<size_t>(c16 * 16 + 2 * q + 1) * p.ld_rt + m0 + row] = static_cast<unsigned short>(w[q] >> 16);
+            for (int q = 0; q < 8; ++q) {
+              rt[static_cast<size_t>(c16 * 16 + 2 * q) * p.ld_rt + m0 + row] = static_cast<unsigned short>(w[q] & 0xFFFFu);
+              rt[static_cast<size_t>(c16 * 16 + 2 * q + 1) * p.ld_rt + m0 + row] = static_cast<unsigned short>(w[q] >> 16);
+            }
           }
         }
+        fence_proxy_async_smem();
+        tc_fence_before();
+        mbar_arrive_cluster(map_to_cta(ps_ready(buf), 0));
       }
-      fence_proxy_async_smem();
-      tc_fence_before();
-      mbar_arrive_cluster(map_to_cta(ps_ready(buf), 0));
       ok = warp_wait(acc_full(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_ACC, false, 32);
       if (named_bar_or(1, 128, !ok)) break;
       tc_fence_after();

@@ -41,7 +41,7 @@ size_t gemm_smem_bytes(int stages);
 constexpr int kPairBlockM = 256;
 constexpr int kPairThreads = 288;           // warps 0..3 TMA producers, warp 4 MMA + TMEM, warps 5..8 epilogue
 constexpr int kPairStageBytesFwd = 32768;   // 128 x 64 activations + 128 x 64 weight/adapter rows per CTA
-constexpr int kPairStageBytesBwd = 36864;   // + up to 4 KiB of unswizzled B columns for the side product
+constexpr int kPairStageBytesBwd = 32768;   // 128 x 64 dY + 64 x 128 W (two 64-column groups) per CTA
 size_t gemm_pair_smem_bytes(bool bwd, int stages);
 cudaError_t gemm_pair_configure();
 // forward: tmW0 = W box 64 x half rows (leader CTA), tmW1 = W box 64 x (block_n - half) rows (peer CTA),
@@ -49,8 +49,8 @@ cudaError_t gemm_pair_configure();
 cudaError_t launch_gemm_pair_fwd(const CUtensorMap& tmX, const CUtensorMap& tmW0, const CUtensorMap& tmW1,
                                  const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
                                  const GemmParams& p, int ctas, cudaStream_t stream);
-// backward: tmW box 64(n) x 64(k); tmB unswizzled box 8(r) x 64(k); tmA box 64(n) x r_pad
-cudaError_t launch_gemm_pair_dx(const CUtensorMap& tmdY, const CUtensorMap& tmW, const CUtensorMap& tmB,
+// backward: tmW box 64(n) x 64(k); tmQt = s (dY B)^T [r_pad, T] box 64(t) x r_pad; tmA box 64(n) x r_pad
+cudaError_t launch_gemm_pair_dx(const CUtensorMap& tmdY, const CUtensorMap& tmW, const CUtensorMap& tmQt,
                                 const CUtensorMap& tmA, const CUtensorMap& tmdX, const GemmParams& p, int ctas,
                                 cudaStream_t stream);
 
@@ -75,7 +75,9 @@ struct GradParams {
   int feat_chunk;         // features per CTA (multiple of 128)
   int n_feat_chunks, n_token_chunks, n_slabs;
   int stages;
-  int with_p;             // 1: also accumulate X A^T for the slab (dA kernel)
+  int with_p;             // 1: also accumulate the side product S * side^T for each slab (X A^T, or dY B)
+  int side_mn;            // side operand: 0 = A [r, C] (K-major rows), 1 = B [C, r] (MN-major, natural layout)
+  int do_out;             // 0: side product only (no second factor, no gradient)
   int out_is_da;          // 1: out[j * C + c] (dA), 0: out[c * r + j] (dB)
   float scale;
   float* out;             // final fp32 gradient

@@ -43,12 +43,15 @@ def test_selector_invariants(shape):
     assert c["cta_group"] == (2 if T > 128 else 1)
     if c["cta_group"] == 2:
         assert c["block_m"] == 256
-        for bn in (c["fwd_block_n"], c["dx_block_n"]):
-            assert bn % 16 == 0 and bn + c["r_pad"] <= 256        # tile + adapter columns fit one MMA / one TMEM buffer
+        assert c["fwd_block_n"] % 16 == 0 and c["fwd_block_n"] + c["r_pad"] <= 256   # tile + adapter columns: one MMA
+        assert c["dx_block_n"] % 16 == 0 and c["dx_block_n"] <= 256                  # K-extended GEMM: no adapter columns
         units = 74                                                  # CTA pairs
         per = 2
         assert c["stages"] * 32768 + 2 * 16384 + 2048 <= 232448     # forward ring + staging fit 227 KiB
-        assert c["dx_stages"] * 36864 + 2 * 16384 + 2048 <= 232448
+        assert c["dx_stages"] * 32768 + 2 * 16384 + 2048 <= 232448
+        assert c["q_feat_chunk"] % 128 == 0 and c["q_feat_chunks"] == -(-d_out // c["q_feat_chunk"])
+        assert 1 <= c["q_feat_chunks"] * c["q_token_chunks"] <= 148 and c["q_token_chunks"] <= -(-T // 128)
+        assert c["q_stages"] * (32768 + 16384) + 4 * c["r_pad"] * 128 + 2048 <= 232448
     else:
         assert c["block_m"] == 128
         for bn in (c["fwd_block_n"], c["dx_block_n"]):
