@@ -38,6 +38,7 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
                  const __grid_constant__ CUtensorMap tm_a,   // side operand (with_p): A [r, C] box 64(c) x r_pad, or
                                                              // B [C, r] box 64(r, zero-filled) x 64(c) when side_mn
                  const GradParams p) {
+  pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int NB = p.feat_chunk >> 7;                 // 128-feature accumulator blocks
@@ -92,6 +93,7 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  pdl_wait();                   // global memory of earlier kernels is visible from here on
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_p = tmem_base + (p.do_out ? NB * p.r_pad : 0);     // two r_pad-column buffers for the side product
 
@@ -273,6 +275,8 @@ __device__ __forceinline__ float ordered_sum(const float* p, int n, size_t strid
 // Fixed-order sums of the partials:  out = sum over token chunks of out_part ;  Pt = bf16(scale * sum over feature
 // chunks of p_part).  One thread per output element, consecutive threads on consecutive addresses.
 __global__ void __launch_bounds__(256) lora_grad_finalize_kernel(const GradParams p) {
+  pdl_launch_dependents();
+  pdl_wait();
   const long long n_out = p.do_out ? static_cast<long long>(p.r) * p.C : 0;
   const long long n_pt = p.with_p ? static_cast<long long>(p.r_pad) * p.T : 0;
   const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -306,12 +310,10 @@ cudaError_t grad_configure() {
 cudaError_t launch_grad(const CUtensorMap& tmS, const CUtensorMap& tmR, const CUtensorMap& tmA, const GradParams& p,
                         cudaStream_t stream) {
   dim3 grid(p.n_feat_chunks, p.n_token_chunks);
-  lora_grad_kernel<<<grid, kGradThreads, grad_smem_bytes(p), stream>>>(tmS, tmR, tmA, p);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e = launch_pdl(lora_grad_kernel, grid, dim3(kGradThreads), grad_smem_bytes(p), stream, tmS, tmR, tmA, p);
   if (e != cudaSuccess) return e;
   const long long n = (p.do_out ? static_cast<long long>(p.r) * p.C : 0) + (p.with_p ? static_cast<long long>(p.r_pad) * p.T : 0);
-  lora_grad_finalize_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(p);
-  return cudaGetLastError();
+  return launch_pdl(lora_grad_finalize_kernel, dim3(static_cast<unsigned>((n + 255) / 256)), dim3(256), 0, stream, p);
 }
 
 // ================================================================================================

@@ -49,6 +49,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY   [M, K
                  const __grid_constant__ CUtensorMap tm_tail,  // fwd B box 64(r) x block_n ; bwd A box 64(n) x r_pad
                  const __grid_constant__ CUtensorMap tm_out,   // Y / dX   [M, N]   box 64 x 128
                  const GemmParams p) {
+  pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t ring = smem_u32(smem);
@@ -93,6 +94,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY   [M, K
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  pdl_wait();                   // global memory of earlier kernels is visible from here on
   const uint32_t tmem_base = *tmem_slot;
 
   const int G = gridDim.x;
@@ -329,15 +331,15 @@ cudaError_t gemm_configure() {
 cudaError_t launch_gemm_fwd(const CUtensorMap& tmX, const CUtensorMap& tmW, const CUtensorMap& tmA,
                             const CUtensorMap& tmB, const CUtensorMap& tmY, const GemmParams& p, int ctas,
                             cudaStream_t stream) {
-  lora_gemm_kernel<false><<<ctas, kGemmThreads, gemm_smem_bytes(p.stages), stream>>>(tmX, tmW, tmA, tmB, tmY, p);
-  return cudaGetLastError();
+  return launch_pdl(lora_gemm_kernel<false>, dim3(ctas), dim3(kGemmThreads), gemm_smem_bytes(p.stages), stream, tmX, tmW, tmA,
+                    tmB, tmY, p);
 }
 
 cudaError_t launch_gemm_dx(const CUtensorMap& tmdY, const CUtensorMap& tmW, const CUtensorMap& tmB,
                            const CUtensorMap& tmA, const CUtensorMap& tmdX, const GemmParams& p, int ctas,
                            cudaStream_t stream) {
-  lora_gemm_kernel<true><<<ctas, kGemmThreads, gemm_smem_bytes(p.stages), stream>>>(tmdY, tmW, tmB, tmA, tmdX, p);
-  return cudaGetLastError();
+  return launch_pdl(lora_gemm_kernel<true>, dim3(ctas), dim3(kGemmThreads), gemm_smem_bytes(p.stages), stream, tmdY, tmW, tmB,
+                    tmA, tmdX, p);
 }
 
 }  // namespace lora

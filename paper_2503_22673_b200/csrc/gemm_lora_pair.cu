@@ -59,6 +59,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
                       const __grid_constant__ CUtensorMap tm_out,   // Y / dX [M, N], box 64 x 128
                       const GemmParams p) {
   constexpr int kStage = kBwd ? kPairStageBytesBwd : kPairStageBytesFwd;
+  pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t ring = smem_u32(smem);
@@ -107,6 +108,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
   __syncthreads();
   cluster_sync_all();           // the peer's barriers exist before anything is signalled across the pair
   tc_fence_after();
+  pdl_wait();                   // everything above overlapped the previous kernel's tail; global memory from here on
   const uint32_t tmem_base = *tmem_slot;
 
   const int G = gridDim.x >> 1;                 // CTA pairs
@@ -414,17 +416,15 @@ cudaError_t gemm_pair_configure() {
 cudaError_t launch_gemm_pair_fwd(const CUtensorMap& tmX, const CUtensorMap& tmW0, const CUtensorMap& tmW1,
                                  const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
                                  const GemmParams& p, int ctas, cudaStream_t stream) {
-  lora_gemm_pair_kernel<false><<<ctas, kPairThreads, gemm_pair_smem_bytes(false, p.stages), stream>>>(
-      tmX, tmW0, tmW1, tmA, tmB, tmY, p);
-  return cudaGetLastError();
+  return launch_pdl(lora_gemm_pair_kernel<false>, dim3(ctas), dim3(kPairThreads), gemm_pair_smem_bytes(false, p.stages), stream,
+                    tmX, tmW0, tmW1, tmA, tmB, tmY, p);
 }
 
 cudaError_t launch_gemm_pair_dx(const CUtensorMap& tmdY, const CUtensorMap& tmW, const CUtensorMap& tmB,
                                 const CUtensorMap& tmA, const CUtensorMap& tmdX, const GemmParams& p, int ctas,
                                 cudaStream_t stream) {
-  lora_gemm_pair_kernel<true><<<ctas, kPairThreads, gemm_pair_smem_bytes(true, p.stages), stream>>>(
-      tmdY, tmW, tmW, tmB, tmA, tmdX, p);
-  return cudaGetLastError();
+  return launch_pdl(lora_gemm_pair_kernel<true>, dim3(ctas), dim3(kPairThreads), gemm_pair_smem_bytes(true, p.stages), stream,
+                    tmdY, tmW, tmW, tmB, tmA, tmdX, p);
 }
 
 }  // namespace lora

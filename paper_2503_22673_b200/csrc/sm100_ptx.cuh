@@ -139,6 +139,13 @@ __device__ __forceinline__ bool named_bar_or(int id, int nthreads, bool pred) {
 }
 
 // ----------------------------------------------------------------------------------------
+// programmatic dependent launch: a kernel launched with the stream-serialization attribute may start while its
+// predecessor drains; it must not touch global memory before pdl_wait() (a no-op for ordinary launches)
+// ----------------------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// ----------------------------------------------------------------------------------------
 // proxy / tcgen05 fences
 // ----------------------------------------------------------------------------------------
 __device__ __forceinline__ void fence_proxy_async_smem() {
