@@ -87,6 +87,7 @@ typedef struct lora_kernel_config {
   int32_t q_feat_chunks;
   int32_t q_token_chunks;
   int32_t q_stages;
+  int32_t fwd_ext;         /* 1: forward runs as X A^T pre-pass + K-extended GEMM (needs the workspace)  */
 } lora_kernel_config_t;
 
 /* Host-only: run the tile / split selector for a shape on a device with `num_sms` SMs.
@@ -101,7 +102,8 @@ int lora_workspace_bytes(const lora_shape_t* shape, int num_sms, size_t* bwd_byt
 int lora_plan_create(const lora_shape_t* shape, int device, lora_plan_t** out);
 int lora_plan_destroy(lora_plan_t* plan);
 
-/* Scratch sizes of a plan; either pointer may be NULL.  fwd_bytes is always 0. */
+/* Scratch sizes of a plan; either pointer may be NULL.  fwd_bytes is 0 unless the selector chose the K-extended
+ * forward (cfg.fwd_ext, large ranks), which uses the same workspace as backward. */
 int lora_plan_workspace_bytes(const lora_plan_t* plan, size_t* fwd_bytes, size_t* bwd_bytes);
 
 /* Register caller-owned device scratch (256-byte aligned, at least bwd_bytes).  The memory stays

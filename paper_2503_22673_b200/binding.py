@@ -41,7 +41,7 @@ class LoraKernelConfig(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "block_m", "fwd_block_n", "dx_block_n", "block_k", "stages", "group_m", "split_k", "r_pad", "fwd_ctas",
         "dx_ctas", "tail_delay", "grad_feat_chunk", "grad_stages", "da_feat_chunks", "da_token_chunks",
-        "db_feat_chunks", "db_token_chunks", "db_feat_chunk", "cta_group", "dx_stages", "prefetch_dist", "db_stages", "q_feat_chunk", "q_feat_chunks", "q_token_chunks", "q_stages")]
+        "db_feat_chunks", "db_token_chunks", "db_feat_chunk", "cta_group", "dx_stages", "prefetch_dist", "db_stages", "q_feat_chunk", "q_feat_chunks", "q_token_chunks", "q_stages", "fwd_ext")]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
@@ -151,9 +151,11 @@ class LoraLinearPlan:
         self._shape = LoraShape(self.T, self.d_in, self.d_out, self.r)
         self._h = ctypes.c_void_p(0)
         _check(self._lib.lora_plan_create(ctypes.byref(self._shape), device, ctypes.byref(self._h)), "lora_plan_create")
-        bwd = ctypes.c_size_t(0)
-        _check(self._lib.lora_plan_workspace_bytes(self._h, None, ctypes.byref(bwd)), "lora_plan_workspace_bytes")
+        bwd, fwd = ctypes.c_size_t(0), ctypes.c_size_t(0)
+        _check(self._lib.lora_plan_workspace_bytes(self._h, ctypes.byref(fwd), ctypes.byref(bwd)),
+               "lora_plan_workspace_bytes")
         self.workspace_bytes = int(bwd.value)
+        self.fwd_workspace_bytes = int(fwd.value)
         self._ws = None
 
     # -- lifetime ------------------------------------------------------------------------------
@@ -210,6 +212,8 @@ class LoraLinearPlan:
         if Y is None:
             Y = torch.empty((self.T, self.d_out), dtype=bf, device=self.device)
         _want(Y, "Y", (self.T, self.d_out), bf, self.device)
+        if self.fwd_workspace_bytes:
+            self.ensure_workspace()
         _check(self._lib.lora_linear_fwd(self._h, _ptr(X), _ptr(W), _ptr(A), _ptr(B), float(scale), _ptr(Y),
                                          _stream_ptr(stream)), "lora_linear_fwd")
         return Y

@@ -131,6 +131,11 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
     c->block_m = kPairBlockM;
     c->fwd_block_n = pick_pair_block_n(T, s->d_out, c->r_pad, pairs);
     c->dx_block_n = pick_pair_block_n(T, s->d_in, 0, pairs);      // no adapter columns in the K-extended dX GEMM
+    // Forward: fused adapter columns cost r_pad / 256 of every MMA; from r_pad = 48 on (>= 19%) a skinny X A^T pre-pass
+    // plus a K-extended GEMM with 256-wide tiles is cheaper (workload 3, r = 64: 1.9 ms fused vs the pre-pass form).
+    c->fwd_ext = c->r_pad >= 48 ? 1 : 0;
+    if (const char* f = std::getenv("LORA_FORCE_FWD_EXT")) c->fwd_ext = std::atoi(f) != 0 ? 1 : 0;
+    if (c->fwd_ext) c->fwd_block_n = pick_pair_block_n(T, s->d_out, 0, pairs);
     c->stages = 6;
     c->dx_stages = 6;
     const long long fwd_t = static_cast<long long>(ceil_div(T, kPairBlockM)) * ceil_div(s->d_out, c->fwd_block_n);
@@ -199,7 +204,12 @@ WsLayout ws_layout(const lora_shape_t& s, const lora_kernel_config_t& c) {
   size_t off = 0;
   w.qt = off;       off += align_up(static_cast<size_t>(c.r_pad) * w.ld_t * 2, kAlign);
   w.pt = off;       off += align_up(static_cast<size_t>(c.r_pad) * w.ld_t * 2, kAlign);
-  w.q_part = off;   off += align_up(static_cast<size_t>(c.q_feat_chunks) * c.r_pad * w.ld_t * 4, kAlign);
+  {
+    int side_chunks = c.q_feat_chunks > c.db_feat_chunks ? c.q_feat_chunks : c.db_feat_chunks;
+    if (side_chunks < 4) side_chunks = 4;   // the X A^T pre-pass of a K-extended forward uses at most 4 feature chunks
+    w.q_part = off;
+    off += align_up(static_cast<size_t>(side_chunks) * c.r_pad * w.ld_t * 4, kAlign);
+  }
   w.p_part = off;   off += align_up(static_cast<size_t>(c.da_feat_chunks) * c.r_pad * w.ld_t * 4, kAlign);
   w.da_part = off;  off += align_up(static_cast<size_t>(c.da_token_chunks) * c.r_pad * w.c_pad_a * 4, kAlign);
   w.db_part = off;  off += align_up(static_cast<size_t>(c.db_token_chunks) * c.r_pad * w.c_pad_b * 4, kAlign);
@@ -264,6 +274,9 @@ struct lora_plan {
   unsigned* d_status;   // 64 words of device memory
   void* workspace;
   size_t workspace_bytes;
+  bool q_ready;          // set while lora_linear_bwd_saved_p runs: Qt was already produced by its dB kernel
+  bool p_saved;          // the workspace holds Pt = s (X A^T)^T of the last forward call
+  float p_saved_scale;
 };
 
 namespace {
@@ -279,17 +292,84 @@ struct DeviceGuard {
   }
 };
 
+struct WsPtrs {
+  uint8_t* base;
+  __nv_bfloat16 *qt, *pt;
+};
+
+WsPtrs ws_ptrs(lora_plan* pl) {
+  WsPtrs q;
+  q.base = static_cast<uint8_t*>(pl->workspace);
+  q.qt = reinterpret_cast<__nv_bfloat16*>(q.base + pl->ws.qt);
+  q.pt = reinterpret_cast<__nv_bfloat16*>(q.base + pl->ws.pt);
+  return q;
+}
+
+// Skinny side-product pass: out_t = s (S side^T)^T as bf16 [r_pad, ld_t], S = X with side = A [r, C] (K-major) or
+// S = dY with side = B [C, r] (MN-major).  Streams S once; partials over feature chunks are summed in fixed order.
+int launch_side_prepass(lora_plan* pl, const void* S, long long C, const void* side, bool side_mn, float scale,
+                        __nv_bfloat16* out_t, cudaStream_t st) {
+  const lora_shape_t& s = pl->shape;
+  const lora_kernel_config_t& c = pl->cfg;
+  const WsLayout& w = pl->ws;
+  CUtensorMap tmS, tmSide;
+  bool ok = make_bf16_tmap(&tmS, S, C, s.T, C, 64, kGradSlab);
+  if (side_mn) ok = ok && make_bf16_tmap(&tmSide, side, s.r, C, s.r, 64, 64);
+  else ok = ok && make_bf16_tmap(&tmSide, side, C, s.r, C, 64, c.r_pad);
+  if (!ok) return LORA_ERR_CUDA;
+  // grid: as few feature chunks as fill the SMs together with the 128-token slabs (no TMEM bound: side product only)
+  const int n_slabs = w.n_slabs;
+  int nf = ceil_div(pl->num_sms, n_slabs);
+  if (nf > 4) nf = 4;
+  const int fc = ceil_div(ceil_div(C, nf), 128) * 128;
+  nf = ceil_div(C, fc);
+  int nt = pl->num_sms / nf;
+  if (nt > n_slabs) nt = n_slabs;
+  if (nt < 1) nt = 1;
+  GradParams g{};
+  g.T = static_cast<int>(s.T);
+  g.C = static_cast<int>(C);
+  g.r = static_cast<int>(s.r);
+  g.r_pad = c.r_pad;
+  g.feat_chunk = fc;
+  g.n_feat_chunks = nf;
+  g.n_token_chunks = nt;
+  g.n_slabs = n_slabs;
+  g.stages = side_mn ? 4 : ((232448 - 4 * c.r_pad * 128 - 2048) / (kGradStageBytes + 2 * c.r_pad * 128) > 6
+                                ? 6 : (232448 - 4 * c.r_pad * 128 - 2048) / (kGradStageBytes + 2 * c.r_pad * 128));
+  g.with_p = 1;
+  g.side_mn = side_mn ? 1 : 0;
+  g.do_out = 0;
+  g.scale = scale;
+  g.p_part = reinterpret_cast<float*>(static_cast<uint8_t*>(pl->workspace) + w.q_part);
+  g.pt_out = out_t;
+  g.ld_t = w.ld_t;
+  g.status = pl->d_status;
+  if (launch_grad(tmS, tmS, tmSide, g, st) != cudaSuccess) return LORA_ERR_CUDA;
+  g_launches.fetch_add(2);
+  return LORA_OK;
+}
+
 int launch_fwd(lora_plan* pl, const void* X, const void* W, const void* A, const void* B, float scale, void* Y,
                cudaStream_t st) {
   const lora_shape_t& s = pl->shape;
   const lora_kernel_config_t& c = pl->cfg;
   const bool pair = c.cta_group == 2;
+  const bool ext = pair && c.fwd_ext != 0;
+  const bool have_ws = pl->workspace != nullptr && pl->workspace_bytes >= pl->ws.total;
+  if (ext && !have_ws) return LORA_ERR_WORKSPACE;
+  __nv_bfloat16* pt = have_ws ? ws_ptrs(pl).pt : nullptr;
+  if (ext) {
+    const int rc = launch_side_prepass(pl, X, s.d_in, A, false, scale, pt, st);   // Pt = s (X A^T)^T
+    if (rc != LORA_OK) return rc;
+  }
   const int half = (c.fwd_block_n + c.r_pad) / 2;
   CUtensorMap tmX, tmW, tmW1, tmA, tmB, tmY;
   bool ok = make_bf16_tmap(&tmX, X, s.d_in, s.T, s.d_in, 64, kBlockM);
-  ok = ok && make_bf16_tmap(&tmW, W, s.d_in, s.d_out, s.d_in, 64, pair ? half : c.fwd_block_n);
-  if (pair) ok = ok && make_bf16_tmap(&tmW1, W, s.d_in, s.d_out, s.d_in, 64, c.fwd_block_n - half);
-  ok = ok && make_bf16_tmap(&tmA, A, s.d_in, s.r, s.d_in, 64, c.r_pad);
+  ok = ok && make_bf16_tmap(&tmW, W, s.d_in, s.d_out, s.d_in, 64, ext ? c.fwd_block_n / 2 : pair ? half : c.fwd_block_n);
+  if (pair && !ext) ok = ok && make_bf16_tmap(&tmW1, W, s.d_in, s.d_out, s.d_in, 64, c.fwd_block_n - half);
+  if (ext) ok = ok && make_bf16_tmap(&tmA, pt, s.T, c.r_pad, pl->ws.ld_t, 64, c.r_pad);
+  else ok = ok && make_bf16_tmap(&tmA, A, s.d_in, s.r, s.d_in, 64, c.r_pad);
   ok = ok && make_bf16_tmap(&tmB, B, s.r, s.d_out, s.r, 64, pair ? c.fwd_block_n / 2 : c.fwd_block_n);
   ok = ok && make_bf16_tmap(&tmY, Y, s.d_out, s.T, s.d_out, 64, kBlockM);
   if (!ok) return LORA_ERR_CUDA;
@@ -310,27 +390,18 @@ int launch_fwd(lora_plan* pl, const void* X, const void* W, const void* A, const
   p.tail_delay = c.tail_delay;
   p.prefetch_dist = c.prefetch_dist;
   p.scale = scale;
-  p.rt_out = nullptr;
-  p.ld_rt = 0;
+  // with a registered workspace the CTA-pair forward leaves Pt = s (X A^T)^T there for lora_linear_bwd_saved_p
+  p.rt_out = (pair && !ext) ? pt : nullptr;
+  p.ld_rt = pl->ws.ld_t;
   p.status = pl->d_status;
-  const cudaError_t le = pair ? launch_gemm_pair_fwd(tmX, tmW, tmW1, tmA, tmB, tmY, p, c.fwd_ctas, st)
-                              : launch_gemm_fwd(tmX, tmW, tmA, tmB, tmY, p, c.fwd_ctas, st);
+  const cudaError_t le = ext    ? launch_gemm_pair_fwd_ext(tmX, tmW, tmA, tmB, tmY, p, c.fwd_ctas, st)
+                         : pair ? launch_gemm_pair_fwd(tmX, tmW, tmW1, tmA, tmB, tmY, p, c.fwd_ctas, st)
+                                : launch_gemm_fwd(tmX, tmW, tmA, tmB, tmY, p, c.fwd_ctas, st);
   if (le != cudaSuccess) return LORA_ERR_CUDA;
   g_launches.fetch_add(1);
+  pl->p_saved = pair && pt != nullptr;
+  pl->p_saved_scale = scale;
   return LORA_OK;
-}
-
-struct WsPtrs {
-  uint8_t* base;
-  __nv_bfloat16 *qt, *pt;
-};
-
-WsPtrs ws_ptrs(lora_plan* pl) {
-  WsPtrs q;
-  q.base = static_cast<uint8_t*>(pl->workspace);
-  q.qt = reinterpret_cast<__nv_bfloat16*>(q.base + pl->ws.qt);
-  q.pt = reinterpret_cast<__nv_bfloat16*>(q.base + pl->ws.pt);
-  return q;
 }
 
 // ---- dX = dY W + s (dY B) A ; also leaves Qt = s (dY B)^T in the workspace ----
@@ -341,32 +412,10 @@ int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const
   const WsLayout& w = pl->ws;
   const WsPtrs q = ws_ptrs(pl);
   __nv_bfloat16* qt = q.qt;
-  if (c.cta_group == 2) {
+  if (c.cta_group == 2 && !pl->q_ready) {
     // ---- pre-pass: Qt = s (dY B)^T, dY streamed once by the skinny kernel (side product only) ----
-    CUtensorMap tmS, tmSide;
-    bool ok = make_bf16_tmap(&tmS, dY, s.d_out, s.T, s.d_out, 64, kGradSlab);
-    ok = ok && make_bf16_tmap(&tmSide, B, s.r, s.d_out, s.r, 64, 64);
-    if (!ok) return LORA_ERR_CUDA;
-    GradParams g{};
-    g.T = static_cast<int>(s.T);
-    g.C = static_cast<int>(s.d_out);
-    g.r = static_cast<int>(s.r);
-    g.r_pad = c.r_pad;
-    g.feat_chunk = c.q_feat_chunk;
-    g.n_feat_chunks = c.q_feat_chunks;
-    g.n_token_chunks = c.q_token_chunks;
-    g.n_slabs = w.n_slabs;
-    g.stages = c.q_stages;
-    g.with_p = 1;
-    g.side_mn = 1;
-    g.do_out = 0;
-    g.scale = scale;
-    g.p_part = reinterpret_cast<float*>(q.base + w.q_part);
-    g.pt_out = qt;
-    g.ld_t = w.ld_t;
-    g.status = pl->d_status;
-    if (launch_grad(tmS, tmS, tmSide, g, st) != cudaSuccess) return LORA_ERR_CUDA;
-    g_launches.fetch_add(2);
+    const int rc = launch_side_prepass(pl, dY, s.d_out, B, true, scale, qt, st);
+    if (rc != LORA_OK) return rc;
   }
   {
     CUtensorMap tmdY, tmW, tmB, tmA, tmdX;
@@ -534,6 +583,9 @@ int lora_plan_create(const lora_shape_t* shape, int device, lora_plan_t** out) {
   pl->ws = ws_layout(*shape, pl->cfg);
   pl->workspace = nullptr;
   pl->workspace_bytes = 0;
+  pl->q_ready = false;
+  pl->p_saved = false;
+  pl->p_saved_scale = 0.f;
   pl->d_status = nullptr;
   if (gemm_configure() != cudaSuccess || gemm_pair_configure() != cudaSuccess || grad_configure() != cudaSuccess || encode_fn() == nullptr ||
       cudaMalloc(&pl->d_status, 256) != cudaSuccess || cudaMemset(pl->d_status, 0, 256) != cudaSuccess) {
@@ -556,7 +608,7 @@ int lora_plan_destroy(lora_plan_t* plan) {
 
 int lora_plan_workspace_bytes(const lora_plan_t* plan, size_t* fwd_bytes, size_t* bwd_bytes) {
   if (plan == nullptr) return LORA_ERR_INVALID_ARG;
-  if (fwd_bytes) *fwd_bytes = 0;
+  if (fwd_bytes) *fwd_bytes = (plan->cfg.cta_group == 2 && plan->cfg.fwd_ext) ? plan->ws.total : 0;
   if (bwd_bytes) *bwd_bytes = plan->ws.total;
   return LORA_OK;
 }

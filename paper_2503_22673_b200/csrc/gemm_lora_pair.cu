@@ -49,7 +49,10 @@ __device__ __forceinline__ PairTile pair_tile(int id, const GemmParams& p) {
   return c;
 }
 
-template <bool kBwd>
+// kBmn: the weight-side operands (W, and A in the rank-r k-block) are MN-major (backward) instead of K-major.
+// kExt: K-extended form - the scaled first adapter product (Pt or Qt, [r_pad, T] bf16) was computed beforehand and
+//       enters as one more k-block; otherwise (forward only) it is fused: extra accumulator columns + epilogue.
+template <bool kBmn, bool kExt>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M, K], box 64(k) x 128
                       const __grid_constant__ CUtensorMap tm_w0,    // fwd: W box 64(k) x half ; bwd: W box 64(n) x 64(k)
@@ -58,7 +61,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
                       const __grid_constant__ CUtensorMap tm_tail,  // fwd: B box 64(r) x block_n/2 ; bwd: A box 64(n) x r_pad
                       const __grid_constant__ CUtensorMap tm_out,   // Y / dX [M, N], box 64 x 128
                       const GemmParams p) {
-  constexpr int kStage = kBwd ? kPairStageBytesBwd : kPairStageBytesFwd;
+  constexpr int kStage = kPairStageBytesFwd;
   pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -145,7 +148,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
         if (op == 0) {
           if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), 2 * 16384);
           tma_load_2d_pair(a_dst, &tm_act, fb, k0, m0);
-        } else if (!kBwd) {
+        } else if (!kExt) {
           if (rank == 0) {
             mbar_arrive_expect_tx(full_bar(cur), (BN + p.r_pad) * 128);
             tma_load_2d_pair(b_dst, &tm_w0, fb, k0, n0);
@@ -153,6 +156,9 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
             tma_load_2d_pair(b_dst, &tm_w1, fb, k0, n0 + half);
             tma_load_2d_pair(b_dst + (BN - half) * 128, &tm_side, fb, k0, 0);
           }
+        } else if (!kBmn) {
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), BN * 128);
+          tma_load_2d_pair(b_dst, &tm_w0, fb, k0, n0 + static_cast<int>(rank) * (BN >> 1));
         } else {
           if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), 2 * 16384);
           const int nb = n0 + static_cast<int>(rank) * (BN >> 1);
@@ -170,15 +176,15 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       const uint32_t fb = map_to_cta(full_bar(cur), 0);
       if (elect_one()) {
         if (op == 0) {
-          if (!kBwd) {
-            if (rank == 0) mbar_arrive(full_bar(cur));        // forward: the rank-r operand comes from the epilogue
+          if (!kExt) {
+            if (rank == 0) mbar_arrive(full_bar(cur));        // fused: the rank-r operand comes from the epilogue
           } else {
-            // backward: s (dY B)^T for this CTA's 128 tokens, two 64-token groups of r_pad rows (MN-major A operand)
+            // K-extended: s (X A^T)^T or s (dY B)^T for this CTA's 128 tokens, two 64-token groups of r_pad rows (MN-major A operand)
             if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), 2 * 2 * p.r_pad * 128);
             tma_load_2d_pair(a_dst, &tm_side, fb, m0, 0);
             tma_load_2d_pair(a_dst + p.r_pad * 128, &tm_side, fb, m0 + 64, 0);
           }
-        } else if (!kBwd) {
+        } else if (!kBmn) {
           if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), BN * 128);
           tma_load_2d_pair(b_dst, &tm_tail, fb, 0, nb);
         } else {
@@ -189,35 +195,35 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       }
       __syncwarp();
     };
-    // Item order.  Forward: the rank-r item of tile i-1 comes D k-blocks into tile i (its operand is made by the
-    // epilogue meanwhile).  Backward: the rank-r item is simply the last k-block of its own tile.
+    // Item order.  Fused: the rank-r item of tile i-1 comes D k-blocks into tile i (its operand is made by the
+    // epilogue meanwhile).  K-extended: the rank-r item is simply the last k-block of its own tile.
     int prev_n0 = 0;
     for (int i = 0; i < n_my && ok; ++i) {
       const PairTile tc = pair_tile(pair + i * G, p);
       const int m0 = tc.m_idx * kPairBlockM + static_cast<int>(rank) * 128, n0 = tc.n_idx * BN;
       for (int kb = 0; kb < KB && ok; ++kb) {
-        if (!kBwd && i > 0 && kb == D) load_tail(0, prev_n0);
+        if (!kExt && i > 0 && kb == D) load_tail(0, prev_n0);
         if (ok) load_main(m0, n0, kb * kBlockK);
       }
-      if (!kBwd && ok && i > 0 && D == KB) load_tail(0, prev_n0);
-      if (kBwd && ok) load_tail(m0, n0);
+      if (!kExt && ok && i > 0 && D == KB) load_tail(0, prev_n0);
+      if (kExt && ok) load_tail(m0, n0);
       prev_n0 = n0;
     }
-    if (!kBwd && ok && n_my > 0) load_tail(0, prev_n0);
+    if (!kExt && ok && n_my > 0) load_tail(0, prev_n0);
   } else if (warp == 4) {
     // ================================ MMA issuer (leader CTA only) ================================
     // Whole warp of the leader CTA runs the loop; one lane polls, one elected lane issues every MMA and commit.
     // Descriptors are advanced by adding byte offsets (>> 4) to precomputed bases.
     if (rank == 0) {
-      const uint32_t idesc_main = kBwd ? mma_idesc_bf16(256, BN, false, true) : mma_idesc_bf16(256, BN + p.r_pad, false, false);
-      const uint32_t idesc_tail = mma_idesc_bf16(256, BN, kBwd, kBwd);   // backward: Qt and A are both MN-major
+      const uint32_t idesc_main = kExt ? mma_idesc_bf16(256, BN, false, kBmn) : mma_idesc_bf16(256, BN + p.r_pad, false, false);
+      const uint32_t idesc_tail = mma_idesc_bf16(256, BN, kExt, kBmn);   // K-extended: Pt / Qt is an MN-major A operand
       const uint64_t ad0 = smem_desc_sw128(ring, 16, 1024);
-      const uint64_t bd0 = kBwd ? smem_desc_sw128(ring + 16384, 8192, 1024) : smem_desc_sw128(ring + 16384, 16, 1024);
+      const uint64_t bd0 = kBmn ? smem_desc_sw128(ring + 16384, 8192, 1024) : smem_desc_sw128(ring + 16384, 16, 1024);
       // rank-r A operand: forward = bf16 s*P rows written by the epilogue (K-major, in the staging buffer);
       // backward = Qt tile delivered by TMA into the stage's activation part (MN-major, two 64-token groups)
-      const uint64_t pd0 = kBwd ? smem_desc_sw128(ring, p.r_pad * 128, 1024) : smem_desc_sw128(staging, 16, 1024);
-      constexpr uint32_t kPStep = kBwd ? (2048 >> 4) : (32 >> 4);
-      constexpr uint32_t kBStep = kBwd ? (2048 >> 4) : (32 >> 4);     // descriptor step per 16-wide k-step
+      const uint64_t pd0 = kExt ? smem_desc_sw128(ring, p.r_pad * 128, 1024) : smem_desc_sw128(staging, 16, 1024);
+      constexpr uint32_t kPStep = kExt ? (2048 >> 4) : (32 >> 4);
+      constexpr uint32_t kBStep = kBmn ? (2048 >> 4) : (32 >> 4);     // descriptor step per 16-wide k-step
       int slot = 0, phase = 0;
       bool ok = true;
       auto next = [&]() { if (++slot == S) { slot = 0; phase ^= 1; } };
@@ -235,20 +241,20 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
             mma_bf16_ss_pair(acc, ad, bd0 + so + ks * kBStep, idesc_main, accum);
           }
           mma_commit_pair(empty_bar(slot));
-          if (!kBwd && last_kb) mma_commit_pair(side_full(buf));
+          if (!kExt && last_kb) mma_commit_pair(side_full(buf));
         }
         __syncwarp();
         next();
       };
       auto mma_tail = [&](int buf, int use) {
-        if (!kBwd) ok = warp_wait(ps_ready(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_PS, true, 0);
+        if (!kExt) ok = warp_wait(ps_ready(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_PS, true, 0);
         if (ok) ok = warp_wait(full_bar(slot), phase, abort_flag, p.status, DEV_TIMEOUT_FULL, true, 0);
         if (!ok) return;
         tc_fence_after();
         if (elect_one()) {
           const uint32_t so = static_cast<uint32_t>(slot * kStage) >> 4;
           for (int ks = 0; ks < p.r_pad / 16; ++ks)
-            mma_bf16_ss_pair(tmem_base + buf * 256, pd0 + (kBwd ? so : 0u) + ks * kPStep, bd0 + so + ks * kBStep, idesc_tail, 1u);
+            mma_bf16_ss_pair(tmem_base + buf * 256, pd0 + (kExt ? so : 0u) + ks * kPStep, bd0 + so + ks * kBStep, idesc_tail, 1u);
           mma_commit_pair(empty_bar(slot));
           mma_commit_pair(acc_full(buf));
         }
@@ -259,13 +265,13 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
         const int buf = i & 1, use = i >> 1;
         ok = warp_wait(acc_empty(buf), (use & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_ACC_EMPTY, true, 0);
         for (int kb = 0; kb < KB && ok; ++kb) {
-          if (!kBwd && i > 0 && kb == D) mma_tail(buf ^ 1, (i - 1) >> 1);
+          if (!kExt && i > 0 && kb == D) mma_tail(buf ^ 1, (i - 1) >> 1);
           if (ok) mma_main(buf, kb == 0, kb == KB - 1);
         }
-        if (!kBwd && ok && i > 0 && D == KB) mma_tail(buf ^ 1, (i - 1) >> 1);
-        if (kBwd && ok) mma_tail(buf, use);
+        if (!kExt && ok && i > 0 && D == KB) mma_tail(buf ^ 1, (i - 1) >> 1);
+        if (kExt && ok) mma_tail(buf, use);
       }
-      if (!kBwd && ok && n_my > 0) mma_tail((n_my - 1) & 1, (n_my - 1) >> 1);
+      if (!kExt && ok && n_my > 0) mma_tail((n_my - 1) & 1, (n_my - 1) >> 1);
     }
   } else {
     // ================================ epilogue (128 threads per CTA) ================================
@@ -281,8 +287,8 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       const int buf = i & 1, use = i >> 1;
       bool ok = true;
       if (e == 0) tma_store_wait_read<0>();       // the previous tile's stores have left both staging buffers
-      if (!kBwd) {
-        // ---- forward: P = X A^T from TMEM -> scale -> bf16 -> shared memory as the rank-r MMA operand ----
+      if (!kExt) {
+        // ---- fused forward: P = X A^T from TMEM -> scale -> bf16 -> shared memory as the rank-r MMA operand ----
         ok = warp_wait(side_full(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_SIDE, false, 64);
         if (named_bar_or(1, 128, !ok)) break;
         tc_fence_after();
@@ -402,29 +408,38 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
 
 }  // namespace
 
-size_t gemm_pair_smem_bytes(bool bwd, int stages) {
-  return static_cast<size_t>(stages) * (bwd ? kPairStageBytesBwd : kPairStageBytesFwd) + 2 * kStagingBytes +
-         kGemmBarriers * 8 + 16 + 1024;
+size_t gemm_pair_smem_bytes(int stages) {
+  return static_cast<size_t>(stages) * kPairStageBytesFwd + 2 * kStagingBytes + kGemmBarriers * 8 + 16 + 1024;
 }
 
 cudaError_t gemm_pair_configure() {
-  cudaError_t e = cudaFuncSetAttribute(lora_gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(lora_gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+  cudaError_t e = cudaFuncSetAttribute(lora_gemm_pair_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(lora_gemm_pair_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(lora_gemm_pair_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+  return e;
 }
 
 cudaError_t launch_gemm_pair_fwd(const CUtensorMap& tmX, const CUtensorMap& tmW0, const CUtensorMap& tmW1,
                                  const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
                                  const GemmParams& p, int ctas, cudaStream_t stream) {
-  return launch_pdl(lora_gemm_pair_kernel<false>, dim3(ctas), dim3(kPairThreads), gemm_pair_smem_bytes(false, p.stages), stream,
+  return launch_pdl(lora_gemm_pair_kernel<false, false>, dim3(ctas), dim3(kPairThreads), gemm_pair_smem_bytes(p.stages), stream,
                     tmX, tmW0, tmW1, tmA, tmB, tmY, p);
 }
 
-cudaError_t launch_gemm_pair_dx(const CUtensorMap& tmdY, const CUtensorMap& tmW, const CUtensorMap& tmB,
+cudaError_t launch_gemm_pair_fwd_ext(const CUtensorMap& tmX, const CUtensorMap& tmW, const CUtensorMap& tmPt,
+                                     const CUtensorMap& tmB, const CUtensorMap& tmY, const GemmParams& p, int ctas,
+                                     cudaStream_t stream) {
+  return launch_pdl(lora_gemm_pair_kernel<false, true>, dim3(ctas), dim3(kPairThreads), gemm_pair_smem_bytes(p.stages), stream,
+                    tmX, tmW, tmW, tmPt, tmB, tmY, p);
+}
+
+cudaError_t launch_gemm_pair_dx(const CUtensorMap& tmdY, const CUtensorMap& tmW, const CUtensorMap& tmQt,
                                 const CUtensorMap& tmA, const CUtensorMap& tmdX, const GemmParams& p, int ctas,
                                 cudaStream_t stream) {
-  return launch_pdl(lora_gemm_pair_kernel<true>, dim3(ctas), dim3(kPairThreads), gemm_pair_smem_bytes(true, p.stages), stream,
-                    tmdY, tmW, tmW, tmB, tmA, tmdX, p);
+  return launch_pdl(lora_gemm_pair_kernel<true, true>, dim3(ctas), dim3(kPairThreads), gemm_pair_smem_bytes(p.stages), stream,
+                    tmdY, tmW, tmW, tmQt, tmA, tmdX, p);
 }
 
 }  // namespace lora

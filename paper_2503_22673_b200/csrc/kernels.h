@@ -61,14 +61,18 @@ size_t gemm_smem_bytes(int stages);
 constexpr int kPairBlockM = 256;
 constexpr int kPairThreads = 288;           // warps 0..3 TMA producers, warp 4 MMA + TMEM, warps 5..8 epilogue
 constexpr int kPairStageBytesFwd = 32768;   // 128 x 64 activations + 128 x 64 weight/adapter rows per CTA
-constexpr int kPairStageBytesBwd = 32768;   // 128 x 64 dY + 64 x 128 W (two 64-column groups) per CTA
-size_t gemm_pair_smem_bytes(bool bwd, int stages);
+size_t gemm_pair_smem_bytes(int stages);
 cudaError_t gemm_pair_configure();
 // forward: tmW0 = W box 64 x half rows (leader CTA), tmW1 = W box 64 x (block_n - half) rows (peer CTA),
 // half = (block_n + r_pad) / 2; tmA box 64 x r_pad; tmB box 64 x block_n/2 rows
 cudaError_t launch_gemm_pair_fwd(const CUtensorMap& tmX, const CUtensorMap& tmW0, const CUtensorMap& tmW1,
                                  const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
                                  const GemmParams& p, int ctas, cudaStream_t stream);
+// K-extended forward (adapter's X A^T computed beforehand): tmW box 64(k) x block_n/2 rows; tmPt = s (X A^T)^T [r_pad, T]
+// box 64(t) x r_pad; tmB box 64(r) x block_n/2 rows
+cudaError_t launch_gemm_pair_fwd_ext(const CUtensorMap& tmX, const CUtensorMap& tmW, const CUtensorMap& tmPt,
+                                     const CUtensorMap& tmB, const CUtensorMap& tmY, const GemmParams& p, int ctas,
+                                     cudaStream_t stream);
 // backward: tmW box 64(n) x 64(k); tmQt = s (dY B)^T [r_pad, T] box 64(t) x r_pad; tmA box 64(n) x r_pad
 cudaError_t launch_gemm_pair_dx(const CUtensorMap& tmdY, const CUtensorMap& tmW, const CUtensorMap& tmQt,
                                 const CUtensorMap& tmA, const CUtensorMap& tmdX, const GemmParams& p, int ctas,
