@@ -126,6 +126,15 @@ int lora_linear_fwd(lora_plan_t* plan, const void* X, const void* W, const void*
 int lora_linear_bwd(lora_plan_t* plan, const void* dY, const void* X, const void* W, const void* A,
                     const void* B, float scale, void* dX, void* dA, void* dB, void* stream);
 
+/* Backward that reuses the forward's X A^T (what an autograd function would stash): valid only directly after a
+ * lora_linear_fwd call on the SAME plan with the same X, A and scale, made while the workspace was registered (the
+ * forward then leaves scale (X A^T)^T, 2 r_pad bytes per token, in the workspace).  Same results as lora_linear_bwd
+ * up to rounding order; one pass over dY and one over X instead of three skinny passes: the dB kernel also produces
+ * scale (dY B)^T, the dX GEMM and the dA kernel consume it.  Returns LORA_ERR_INVALID_ARG when no matching forward
+ * result is held.  For batches of at most 128 tokens it is the same as lora_linear_bwd. */
+int lora_linear_bwd_saved_p(lora_plan_t* plan, const void* dY, const void* X, const void* W, const void* A,
+                            const void* B, float scale, void* dX, void* dA, void* dB, void* stream);
+
 /* The three stages of lora_linear_bwd as separate calls, for callers that schedule them themselves.
  * They communicate through the plan's workspace and must run in this order on one stream (or with
  * equivalent event dependencies):

@@ -26,7 +26,7 @@ LORA_ERR_NO_DEVICE = -7
 EXPORTS = [
     "lora_select_config", "lora_workspace_bytes", "lora_plan_create", "lora_plan_destroy",
     "lora_plan_workspace_bytes", "lora_plan_set_workspace", "lora_plan_get_config", "lora_plan_describe",
-    "lora_linear_fwd", "lora_linear_bwd", "lora_linear_bwd_dx", "lora_linear_bwd_da", "lora_linear_bwd_db",
+    "lora_linear_fwd", "lora_linear_bwd", "lora_linear_bwd_saved_p", "lora_linear_bwd_dx", "lora_linear_bwd_da", "lora_linear_bwd_db",
     "lora_step_host_staging_bytes", "lora_linear_step_host",
     "lora_last_device_status", "lora_strerror", "lora_launch_count",
     "lora_grad_contract_noalloc", "lora_grad_contract_noalloc_max_scratch",
@@ -75,6 +75,7 @@ def load(rebuild: bool = False) -> ctypes.CDLL:
     lib.lora_plan_describe.argtypes = [vp, ctypes.c_char_p, ctypes.c_size_t]
     lib.lora_linear_fwd.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp]
     lib.lora_linear_bwd.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
+    lib.lora_linear_bwd_saved_p.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
     lib.lora_linear_bwd_dx.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp]
     lib.lora_linear_bwd_da.argtypes = [vp, vp, vp, ctypes.c_float, vp, vp]
     lib.lora_linear_bwd_db.argtypes = [vp, vp, ctypes.c_float, vp, vp]
@@ -218,8 +219,11 @@ class LoraLinearPlan:
                                          _stream_ptr(stream)), "lora_linear_fwd")
         return Y
 
-    def bwd(self, dY, X, W, A, B, scale: float, dX=None, dA=None, dB=None, stream=None):
-        """(dX, dA, dB) = (dY W + scale (dY B) A,  scale (dY B)^T X,  scale dY^T (X A^T))."""
+    def bwd(self, dY, X, W, A, B, scale: float, dX=None, dA=None, dB=None, stream=None, saved_p: bool = False):
+        """(dX, dA, dB) = (dY W + scale (dY B) A,  scale (dY B)^T X,  scale dY^T (X A^T)).
+
+        ``saved_p=True`` reuses X A^T from the preceding ``fwd`` on this plan (same X, A, scale; the workspace must
+        have been registered before that forward: call ``ensure_workspace()`` first)."""
         bf = torch.bfloat16
         _want(dY, "dY", (self.T, self.d_out), bf, self.device)
         _want(X, "X", (self.T, self.d_in), bf, self.device)
@@ -236,8 +240,9 @@ class LoraLinearPlan:
         _want(dA, "dA", (self.r, self.d_in), torch.float32, self.device)
         _want(dB, "dB", (self.d_out, self.r), torch.float32, self.device)
         self.ensure_workspace()
-        _check(self._lib.lora_linear_bwd(self._h, _ptr(dY), _ptr(X), _ptr(W), _ptr(A), _ptr(B), float(scale),
-                                         _ptr(dX), _ptr(dA), _ptr(dB), _stream_ptr(stream)), "lora_linear_bwd")
+        fn = self._lib.lora_linear_bwd_saved_p if saved_p else self._lib.lora_linear_bwd
+        _check(fn(self._h, _ptr(dY), _ptr(X), _ptr(W), _ptr(A), _ptr(B), float(scale),
+                  _ptr(dX), _ptr(dA), _ptr(dB), _stream_ptr(stream)), "lora_linear_bwd")
         return dX, dA, dB
 
     def bwd_stages(self, dY, X, W, A, B, scale: float, dX, dA, dB, stream=None, events=None):

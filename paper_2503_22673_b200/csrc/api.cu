@@ -456,7 +456,7 @@ int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const
 }
 
 // ---- dA = Qt-contraction over X; recomputes X A^T and leaves Pt = s (X A^T)^T ----
-int launch_da(lora_plan* pl, const void* X, const void* A, float scale, void* dA, cudaStream_t st) {
+int launch_da(lora_plan* pl, const void* X, const void* A, float scale, void* dA, cudaStream_t st, bool with_p = true) {
   const lora_shape_t& s = pl->shape;
   const lora_kernel_config_t& c = pl->cfg;
   const WsLayout& w = pl->ws;
@@ -478,8 +478,8 @@ int launch_da(lora_plan* pl, const void* X, const void* A, float scale, void* dA
     g.n_feat_chunks = c.da_feat_chunks;
     g.n_token_chunks = c.da_token_chunks;
     g.n_slabs = w.n_slabs;
-    g.stages = c.grad_stages;
-    g.with_p = 1;
+    g.stages = with_p ? c.grad_stages : c.db_stages;
+    g.with_p = with_p ? 1 : 0;
     g.side_mn = 0;
     g.do_out = 1;
     g.out_is_da = 1;
@@ -498,7 +498,7 @@ int launch_da(lora_plan* pl, const void* X, const void* A, float scale, void* dA
 }
 
 // ---- dB = Pt-contraction over dY ----
-int launch_db(lora_plan* pl, const void* dY, float scale, void* dB, cudaStream_t st) {
+int launch_db(lora_plan* pl, const void* dY, float scale, void* dB, cudaStream_t st, const void* B_for_q = nullptr) {
   const lora_shape_t& s = pl->shape;
   const lora_kernel_config_t& c = pl->cfg;
   const WsLayout& w = pl->ws;
@@ -506,9 +506,11 @@ int launch_db(lora_plan* pl, const void* dY, float scale, void* dB, cudaStream_t
   uint8_t* ws = q.base;
   __nv_bfloat16* pt = q.pt;
   {
-    CUtensorMap tmS, tmR;
+    const bool with_q = B_for_q != nullptr;     // also leave Qt = s (dY B)^T (saved-P backward)
+    CUtensorMap tmS, tmR, tmSide;
     bool ok = make_bf16_tmap(&tmS, dY, s.d_out, s.T, s.d_out, 64, kGradSlab);
     ok = ok && make_bf16_tmap(&tmR, pt, s.T, c.r_pad, w.ld_t, 64, c.r_pad);
+    if (with_q) ok = ok && make_bf16_tmap(&tmSide, B_for_q, s.r, s.d_out, s.r, 64, 64);
     if (!ok) return LORA_ERR_CUDA;
     GradParams g{};
     g.T = static_cast<int>(s.T);
@@ -519,20 +521,20 @@ int launch_db(lora_plan* pl, const void* dY, float scale, void* dB, cudaStream_t
     g.n_feat_chunks = c.db_feat_chunks;
     g.n_token_chunks = c.db_token_chunks;
     g.n_slabs = w.n_slabs;
-    g.stages = c.db_stages;
-    g.with_p = 0;
-    g.side_mn = 0;
+    g.stages = with_q ? 4 : c.db_stages;
+    g.with_p = with_q ? 1 : 0;
+    g.side_mn = with_q ? 1 : 0;
     g.do_out = 1;
     g.out_is_da = 0;
     g.scale = scale;
     g.out = static_cast<float*>(dB);
     g.out_part = reinterpret_cast<float*>(ws + w.db_part);
     g.c_pad = w.c_pad_b;
-    g.p_part = nullptr;
-    g.pt_out = nullptr;
+    g.p_part = with_q ? reinterpret_cast<float*>(ws + w.q_part) : nullptr;
+    g.pt_out = with_q ? q.qt : nullptr;
     g.ld_t = w.ld_t;
     g.status = pl->d_status;
-    if (launch_grad(tmS, tmR, tmR, g, st) != cudaSuccess) return LORA_ERR_CUDA;
+    if (launch_grad(tmS, tmR, with_q ? tmSide : tmR, g, st) != cudaSuccess) return LORA_ERR_CUDA;
     g_launches.fetch_add(2);
   }
   return LORA_OK;
@@ -624,6 +626,7 @@ int lora_plan_set_workspace(lora_plan_t* plan, void* dev_ptr, size_t bytes) {
   if (bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
   plan->workspace = dev_ptr;
   plan->workspace_bytes = bytes;
+  plan->p_saved = false;
   return LORA_OK;
 }
 
@@ -679,6 +682,29 @@ int lora_linear_bwd(lora_plan_t* plan, const void* dY, const void* X, const void
   int rc = launch_dx(plan, dY, W, A, B, scale, dX, st);
   if (rc == LORA_OK) rc = launch_da(plan, X, A, scale, dA, st);
   if (rc == LORA_OK) rc = launch_db(plan, dY, scale, dB, st);
+  return rc;
+}
+
+int lora_linear_bwd_saved_p(lora_plan_t* plan, const void* dY, const void* X, const void* W, const void* A, const void* B,
+                            float scale, void* dX, void* dA, void* dB, void* stream) {
+  if (plan == nullptr) return LORA_ERR_INVALID_ARG;
+  if (plan->shape.T == 0 || plan->cfg.cta_group != 2)      // nothing was saved for these: same as the plain call
+    return lora_linear_bwd(plan, dY, X, W, A, B, scale, dX, dA, dB, stream);
+  if (!dY || !X || !W || !A || !B || !dX || !dA || !dB) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(dY) || !aligned16(X) || !aligned16(W) || !aligned16(A) || !aligned16(B) || !aligned16(dX) ||
+      !aligned16(dA) || !aligned16(dB))
+    return LORA_ERR_MISALIGNED;
+  if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
+  if (!plan->p_saved || plan->p_saved_scale != scale) return LORA_ERR_INVALID_ARG;   // no forward result to reuse
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  DeviceGuard guard(plan->device);
+  int rc = launch_db(plan, dY, scale, dB, st, B);          // dB from the saved Pt; leaves Qt
+  if (rc == LORA_OK) {
+    plan->q_ready = true;
+    rc = launch_dx(plan, dY, W, A, B, scale, dX, st);      // K-extended GEMM only
+    plan->q_ready = false;
+  }
+  if (rc == LORA_OK) rc = launch_da(plan, X, A, scale, dA, st, false);
   return rc;
 }
 

@@ -43,7 +43,9 @@ def test_selector_invariants(shape):
     assert c["cta_group"] == (2 if T > 128 else 1)
     if c["cta_group"] == 2:
         assert c["block_m"] == 256
-        assert c["fwd_block_n"] % 16 == 0 and c["fwd_block_n"] + c["r_pad"] <= 256   # tile + adapter columns: one MMA
+        assert c["fwd_ext"] == (1 if c["r_pad"] >= 48 else 0)
+        # fused forward: tile + adapter columns share one MMA; K-extended forward: no adapter columns
+        assert c["fwd_block_n"] % 16 == 0 and c["fwd_block_n"] + (0 if c["fwd_ext"] else c["r_pad"]) <= 256
         assert c["dx_block_n"] % 16 == 0 and c["dx_block_n"] <= 256                  # K-extended GEMM: no adapter columns
         units = 74                                                  # CTA pairs
         per = 2

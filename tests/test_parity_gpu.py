@@ -253,3 +253,29 @@ def test_host_buffer_step_matches_device_calls():
     assert torch.equal(hdX.view(torch.int16), dX.cpu().view(torch.int16))
     assert torch.equal(hdA, dA.cpu()) and torch.equal(hdB, dB.cpu())
     plan.close()
+
+
+def test_backward_with_saved_forward_product_matches_oracle():
+    """lora_linear_bwd_saved_p reuses X A^T of the preceding forward; it must meet the same tolerances."""
+    for (T, d_in, d_out, r, scale) in [(700, 520, 392, 16, 2.0), (1300, 1032, 2056, 64, 0.5), (129, 264, 136, 8, 1.7)]:
+        p, t = inputs.draw_custom(T, d_in, d_out, r, scale, seed=19)
+        d = {k: dev(v) for k, v in t.items()}
+        f = {k: inputs.bf16_to_f64(v) for k, v in t.items()}
+        plan = binding.LoraLinearPlan(T, d_in, d_out, r)
+        lib = binding.load()
+        dX, dA, dB = (torch.full((T, d_in), float("nan"), dtype=torch.bfloat16, device="cuda"),
+                      torch.full((r, d_in), float("nan"), device="cuda"), torch.full((d_out, r), float("nan"), device="cuda"))
+        # without a forward on a registered workspace there is nothing to reuse
+        plan.ensure_workspace()
+        with pytest.raises(binding.LoraError):
+            plan.bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], scale, dX, dA, dB, saved_p=True)
+        Y = plan.fwd(d["X"], d["W"], d["A"], d["B"], scale)
+        with pytest.raises(binding.LoraError):                      # other scale than the forward's
+            plan.bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], scale + 1.0, dX, dA, dB, saved_p=True)
+        plan.bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], scale, dX, dA, dB, saved_p=True)
+        assert plan.device_status()[0] == 0
+        dXr, dAr, dBr = oracle.backward(f["dY"], f["X"], f["W"], f["A"], f["B"], scale)
+        assert oracle.rel_err(host64(Y), oracle.forward(f["X"], f["W"], f["A"], f["B"], scale)) <= TOL_BF16
+        assert oracle.rel_err(host64(dX), dXr) <= TOL_BF16
+        assert oracle.rel_err(host64(dA), dAr) <= TOL_F32 and oracle.rel_err(host64(dB), dBr) <= TOL_F32
+        plan.close()
