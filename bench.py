@@ -316,6 +316,29 @@ def run_ours(args):
                 "traffic": (NCU_TRAFFIC["bytes_per_launch"][dom_k] if NCU_TRAFFIC["gemm_sha"] == gemm_source_sha()
                             and args.workload == 1 else None)}
 
+    # ---- variant: backward that reuses the forward's X A^T (lora_linear_bwd_saved_p), same inputs and rotation ----
+    def step_saved(k):
+        cur = sets[k % n_sets]
+        for j, (proj, d) in enumerate(cur):
+            plans[j].fwd(d["X"], d["W"], d["A"], d["B"], proj.scale, d["Y"])
+            plans[j].bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], proj.scale, d["dX"], d["dA"], d["dB"], saved_p=True)
+
+    n_var = max(3, min(args.steps, 50))
+    for k in range(3):
+        step_saved(k)
+    torch.cuda.synchronize()
+    v_a, v_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    v_a.record()
+    for k in range(n_var):
+        step_saved(3 + k)
+    v_b.record()
+    torch.cuda.synchronize()
+    barrier()
+    ms_var = max_over_ranks(v_a.elapsed_time(v_b) / n_var, device, world)
+    variants = {"bwd_saved_p": {"ms_per_step": ms_var, "value": job_value(world, flops_step, ms_var), "unit": UNIT,
+                                "steps": n_var, "note": "forward + lora_linear_bwd_saved_p (X A^T kept from the forward)"}}
+
     # ---- end to end: host buffers through the C ABI, copies inside the timed region ----
     h_sets, staging = [], []
     for j, (p, d0) in enumerate(sets[0]):
@@ -364,7 +387,7 @@ def run_ours(args):
                    "replicas": "independent replica per GPU, no collective"},
         "tokens_per_s": world * tokens_step / ms_step * 1e3,
         "frac_of_bf16_peak": value / world / pk["bf16_tflops"], "peak_source": pk["source"],
-        "kernels": kern, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+        "kernels": kern, "variants": variants, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
         "plan": plans[0].describe(),
     }
     print(json.dumps(line), flush=True)
