@@ -279,3 +279,32 @@ def test_backward_with_saved_forward_product_matches_oracle():
         assert oracle.rel_err(host64(dX), dXr) <= TOL_BF16
         assert oracle.rel_err(host64(dA), dAr) <= TOL_F32 and oracle.rel_err(host64(dB), dBr) <= TOL_F32
         plan.close()
+
+
+def test_grouped_projections_sharing_x_match_separate_oracles():
+    """q/k/v-style group as one layer (stacked A, block-diagonal B): every projection must match ITS OWN oracle,
+    and dX the sum of the three."""
+    from paper_2503_22673_b200.grouped import GroupedLoraPlan
+    T, d_in, r, scale = 900, 520, 16, 2.0
+    d_outs = [392, 136, 136]
+    projs = [inputs.draw_custom(T, d_in, d, r, scale, seed=30 + g, tag=70 + g) for g, d in enumerate(d_outs)]
+    X_bits = projs[0][1]["X"]
+    f64 = lambda b: inputs.bf16_to_f64(b)
+    gp = GroupedLoraPlan(T, d_in, d_outs, r)
+    W, A, B = gp.pack([dev(t["W"]) for _, t in projs], [dev(t["A"]) for _, t in projs], [dev(t["B"]) for _, t in projs])
+    X = dev(X_bits)
+    dY = torch.cat([dev(t["dY"]) for _, t in projs], dim=1).contiguous()
+    Y = gp.fwd(X, W, A, B, scale)
+    dX, dAs, dBs = gp.bwd(dY, X, W, A, B, scale)
+    assert gp.plan.device_status()[0] == 0
+    dX_ref = 0.0
+    for g, (p, t) in enumerate(projs):
+        Wg, Ag, Bg, dYg = f64(t["W"]), f64(t["A"]), f64(t["B"]), f64(t["dY"])
+        Yr = oracle.forward(f64(X_bits), Wg, Ag, Bg, scale)
+        dXr, dAr, dBr = oracle.backward(dYg, f64(X_bits), Wg, Ag, Bg, scale)
+        dX_ref = dX_ref + dXr
+        assert oracle.rel_err(host64(gp.split_outputs(Y)[g]), Yr) <= TOL_BF16
+        assert oracle.rel_err(host64(dAs[g]), dAr) <= TOL_F32
+        assert oracle.rel_err(host64(dBs[g]), dBr) <= TOL_F32
+    assert oracle.rel_err(host64(dX), dX_ref) <= TOL_BF16
+    gp.close()
