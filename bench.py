@@ -243,10 +243,46 @@ def run_ours(args):
             d["dB"] = torch.empty((proj.d_out, proj.r), dtype=torch.float32, device=device)
             cur.append((proj, d))
         sets.append(cur)
+    if args.grouped and args.workload == 4:
+        # q/k/v and gate/up consume the same X: each group becomes ONE projection (stacked A, block-diagonal B)
+        from paper_2503_22673_b200.grouped import GroupedLoraPlan
+        groups = [[0, 1, 2], [3], [4, 5], [6]]
+        new_protos, new_sets = [], [[] for _ in sets]
+        for idxs in groups:
+            p0 = protos[idxs[0]]
+            if len(idxs) == 1:
+                new_protos.append(p0)
+                for si, cur in enumerate(sets):
+                    new_sets[si].append(cur[idxs[0]])
+                continue
+            d_outs = [protos[i].d_out for i in idxs]
+            gp = inputs.Projection("+".join(protos[i].name for i in idxs), p0.T, p0.d_in, sum(d_outs), p0.r * len(idxs),
+                                   p0.scale)
+            new_protos.append(gp)
+            helper = GroupedLoraPlan(p0.T, p0.d_in, d_outs, p0.r, device=local_rank)
+            for si, cur in enumerate(sets):
+                W, A, B = helper.pack([cur[i][1]["W"] for i in idxs], [cur[i][1]["A"] for i in idxs],
+                                      [cur[i][1]["B"] for i in idxs])
+                d = {"X": cur[idxs[0]][1]["X"], "W": W, "A": A, "B": B,
+                     "dY": torch.cat([cur[i][1]["dY"] for i in idxs], dim=1).contiguous()}
+                d["Y"] = torch.empty((gp.T, gp.d_out), dtype=torch.bfloat16, device=device)
+                d["dX"] = torch.empty((gp.T, gp.d_in), dtype=torch.bfloat16, device=device)
+                d["dA"] = torch.empty((gp.r, gp.d_in), dtype=torch.float32, device=device)
+                d["dB"] = torch.empty((gp.d_out, gp.r), dtype=torch.float32, device=device)
+                new_sets[si].append((gp, d))
+            helper.close()
+        flops_algorithmic = float(sum(p.flops for p in protos))      # the seven projections' own FLOPs
+        protos, sets = new_protos, new_sets
+        del new_sets
+        import gc
+        gc.collect()
+        torch.cuda.empty_cache()
+    else:
+        flops_algorithmic = float(sum(p.flops for p in protos))
     plans = [binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r, device=local_rank) for p in protos]
     for pl in plans:
         pl.ensure_workspace()
-    flops_step = float(sum(p.flops for p in protos))
+    flops_step = flops_algorithmic
     tokens_step = protos[0].T
 
     def step(k, events=None):
@@ -381,7 +417,7 @@ def run_ours(args):
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": workload_name(args.workload), "projections": [p.name for p in protos], "T": protos[0].T,
-                   "r": protos[0].r, "scale": protos[0].scale, "input_sets_rotated": n_sets,
+                   "r": protos[0].r, "scale": protos[0].scale, "input_sets_rotated": n_sets, "grouped": bool(args.grouped and args.workload == 4),
                    "l2": f"{n_sets} independent input/output sets ({bytes_per_set * n_sets / 2**20:.0f} MiB) rotated per step; "
                          "each step's operands exceed the 126 MB L2",
                    "replicas": "independent replica per GPU, no collective"},
@@ -401,6 +437,8 @@ def main():
     ap.add_argument("--workload", type=int, default=1)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--grouped", action="store_true",
+                    help="workload 4 only: run q/k/v and gate/up as one grouped projection each (shared X)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -131,9 +131,11 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
     c->block_m = kPairBlockM;
     c->fwd_block_n = pick_pair_block_n(T, s->d_out, c->r_pad, pairs);
     c->dx_block_n = pick_pair_block_n(T, s->d_in, 0, pairs);      // no adapter columns in the K-extended dX GEMM
-    // Forward: fused adapter columns cost r_pad / 256 of every MMA; from r_pad = 48 on (>= 19%) a skinny X A^T pre-pass
-    // plus a K-extended GEMM with 256-wide tiles is cheaper (workload 3, r = 64: 1.9 ms fused vs the pre-pass form).
-    c->fwd_ext = c->r_pad >= 48 ? 1 : 0;
+    // Forward, fused vs K-extended.  Fused adapter columns cost r_pad / 256 of every MMA (time ~ T d_in d_out r_pad);
+    // the alternative is a skinny X A^T pre-pass (time ~ T d_in, one more read of X) and 256-wide tiles.  Their ratio
+    // is ~1e-5 d_out r_pad at the measured rates (1.2 PFLOP/s GEMM, 3 TB/s pre-pass), so the pre-pass wins for wide
+    // outputs or large ranks: 14336 x 16 and 4096 x 64 take it, 4096 x 16 and 1024 x 16 stay fused.
+    c->fwd_ext = (static_cast<long long>(s->d_out) * c->r_pad >= 100000) ? 1 : 0;
     if (const char* f = std::getenv("LORA_FORCE_FWD_EXT")) c->fwd_ext = std::atoi(f) != 0 ? 1 : 0;
     if (c->fwd_ext) c->fwd_block_n = pick_pair_block_n(T, s->d_out, 0, pairs);
     c->stages = 6;
