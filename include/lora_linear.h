@@ -67,7 +67,7 @@ typedef struct lora_kernel_config {
   int32_t block_k;         /* contraction elements per pipeline stage (64)                     */
   int32_t stages;          /* depth of the TMA -> MMA shared-memory ring, forward GEMM         */
   int32_t group_m;         /* tile rasterisation: m-tiles per band (L2 reuse)                  */
-  int32_t split_k;         /* split-K factor of the dense GEMMs (1 = none)                     */
+  int32_t split_k;         /* k-splits per tile of the forward GEMM (1 = none)                 */
   int32_t r_pad;           /* rank padded to the MMA granularity (multiple of 16)              */
   int32_t fwd_ctas;        /* persistent CTAs of the forward GEMM                              */
   int32_t dx_ctas;         /* persistent CTAs of the dX GEMM                                   */
@@ -87,6 +87,7 @@ typedef struct lora_kernel_config {
   int32_t q_feat_chunks;
   int32_t q_token_chunks;
   int32_t q_stages;
+  int32_t dx_split_k;      /* k-splits per tile of the dX GEMM                                           */
   int32_t fwd_ext;         /* 1: forward runs as X A^T pre-pass + K-extended GEMM (needs the workspace)  */
 } lora_kernel_config_t;
 

@@ -119,6 +119,7 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
   c->dx_stages = 4;
   c->group_m = 8;
   c->split_k = 1;
+  c->dx_split_k = 1;
   c->tail_delay = 8;
   c->prefetch_dist = 0;    // L2 prefetch ahead of the ring was measured slower (it competes with the producers' copies)
   c->cta_group = (T > kBlockM && num_sms >= 2) ? 2 : 1;
@@ -137,13 +138,43 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
     // outputs or large ranks: 14336 x 16 and 4096 x 64 take it, 4096 x 16 and 1024 x 16 stay fused.
     c->fwd_ext = (static_cast<long long>(s->d_out) * c->r_pad >= 100000) ? 1 : 0;
     if (const char* f = std::getenv("LORA_FORCE_FWD_EXT")) c->fwd_ext = std::atoi(f) != 0 ? 1 : 0;
+    // Split along K: when the tiling leaves at least three quarters of the CTA pairs idle and the contraction is long
+    // (>= 64 k-blocks), each tile is cut into k-ranges handled by different pairs (fp32 partial tiles, fixed-order
+    // reduce kernel).  Measured: 257 x 14336 -> 264 forward 86 -> 45 us with 8 splits; on shorter contractions or
+    // fuller grids (256 x 4096 x 4096: 29 tiles) the extra reduce launch costs as much as the split saves.
+    // Only the K-extended kernel form supports it, so such a forward is K-extended too.
+    auto pick_split = [&](long long tiles, int kb) {
+      if (tiles * 4 > pairs || kb < 64) return 1;
+      long long sp = pairs / tiles;
+      if (sp > kb / 16) sp = kb / 16;
+      if (sp > 8) sp = 8;
+      return static_cast<int>(sp < 1 ? 1 : sp);
+    };
+    {
+      const int bn = pick_pair_block_n(T, s->d_out, 0, pairs);
+      const long long tiles = static_cast<long long>(ceil_div(T, kPairBlockM)) * ceil_div(s->d_out, bn);
+      c->split_k = pick_split(tiles, ceil_div(s->d_in, kBlockK));
+      if (c->split_k > 1) c->fwd_ext = 1;
+    }
     if (c->fwd_ext) c->fwd_block_n = pick_pair_block_n(T, s->d_out, 0, pairs);
+    {
+      const long long tiles = static_cast<long long>(ceil_div(T, kPairBlockM)) * ceil_div(s->d_in, c->dx_block_n);
+      c->dx_split_k = pick_split(tiles, ceil_div(s->d_out, kBlockK));
+    }
+    if (const char* f = std::getenv("LORA_FORCE_SPLIT_K")) {
+      const int v = std::atoi(f);
+      if (v >= 1 && v <= 8) {
+        c->split_k = c->dx_split_k = v;
+        if (v > 1 && !c->fwd_ext) { c->fwd_ext = 1; c->fwd_block_n = pick_pair_block_n(T, s->d_out, 0, pairs); }
+      }
+    }
     c->stages = 6;
     c->dx_stages = 6;
     const long long fwd_t = static_cast<long long>(ceil_div(T, kPairBlockM)) * ceil_div(s->d_out, c->fwd_block_n);
     const long long dx_t = static_cast<long long>(ceil_div(T, kPairBlockM)) * ceil_div(s->d_in, c->dx_block_n);
-    c->fwd_ctas = 2 * static_cast<int>(fwd_t < pairs ? fwd_t : pairs);
-    c->dx_ctas = 2 * static_cast<int>(dx_t < pairs ? dx_t : pairs);
+    const long long fwd_items = fwd_t * c->split_k, dx_items = dx_t * c->dx_split_k;
+    c->fwd_ctas = 2 * static_cast<int>(fwd_items < pairs ? fwd_items : pairs);
+    c->dx_ctas = 2 * static_cast<int>(dx_items < pairs ? dx_items : pairs);
   } else {
     const long long fwd_tiles = static_cast<long long>(ceil_div(T, kBlockM)) * ceil_div(s->d_out, c->fwd_block_n);
     const long long dx_tiles = static_cast<long long>(ceil_div(T, kBlockM)) * ceil_div(s->d_in, c->dx_block_n);
@@ -192,7 +223,7 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
 // backward workspace layout
 // ------------------------------------------------------------------------------------------------
 struct WsLayout {
-  size_t qt, pt, q_part, p_part, da_part, db_part, total;
+  size_t qt, pt, q_part, p_part, da_part, db_part, split_part, total;
   int ld_t, c_pad_a, c_pad_b, n_slabs;
 };
 
@@ -215,6 +246,12 @@ WsLayout ws_layout(const lora_shape_t& s, const lora_kernel_config_t& c) {
   w.p_part = off;   off += align_up(static_cast<size_t>(c.da_feat_chunks) * c.r_pad * w.ld_t * 4, kAlign);
   w.da_part = off;  off += align_up(static_cast<size_t>(c.da_token_chunks) * c.r_pad * w.c_pad_a * 4, kAlign);
   w.db_part = off;  off += align_up(static_cast<size_t>(c.db_token_chunks) * c.r_pad * w.c_pad_b * 4, kAlign);
+  {
+    const size_t f = c.split_k > 1 ? static_cast<size_t>(c.split_k) * T * s.d_out * 4 : 0;
+    const size_t b = c.dx_split_k > 1 ? static_cast<size_t>(c.dx_split_k) * T * s.d_in * 4 : 0;
+    w.split_part = off;
+    off += align_up(f > b ? f : b, kAlign);
+  }
   w.total = off;
   return w;
 }
@@ -393,6 +430,10 @@ int launch_fwd(lora_plan* pl, const void* X, const void* W, const void* A, const
   p.prefetch_dist = c.prefetch_dist;
   p.scale = scale;
   // with a registered workspace the CTA-pair forward leaves Pt = s (X A^T)^T there for lora_linear_bwd_saved_p
+  const int kb_total = ceil_div(s.d_in, kBlockK);
+  p.kb_per_split = ext ? ceil_div(kb_total, c.split_k) : kb_total;
+  p.split_k = ext ? ceil_div(kb_total, p.kb_per_split) : 1;
+  p.part = (p.split_k > 1) ? reinterpret_cast<float*>(static_cast<uint8_t*>(pl->workspace) + pl->ws.split_part) : nullptr;
   p.rt_out = (pair && !ext) ? pt : nullptr;
   p.ld_rt = pl->ws.ld_t;
   p.status = pl->d_status;
@@ -401,6 +442,12 @@ int launch_fwd(lora_plan* pl, const void* X, const void* W, const void* A, const
                                 : launch_gemm_fwd(tmX, tmW, tmA, tmB, tmY, p, c.fwd_ctas, st);
   if (le != cudaSuccess) return LORA_ERR_CUDA;
   g_launches.fetch_add(1);
+  if (p.split_k > 1) {
+    if (launch_splitk_reduce(p.part, static_cast<__nv_bfloat16*>(Y), static_cast<long long>(s.T) * s.d_out, p.split_k, st) !=
+        cudaSuccess)
+      return LORA_ERR_CUDA;
+    g_launches.fetch_add(1);
+  }
   pl->p_saved = pair && pt != nullptr;
   pl->p_saved_scale = scale;
   return LORA_OK;
@@ -446,6 +493,10 @@ int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const
     p.tail_delay = c.tail_delay;
     p.prefetch_dist = c.prefetch_dist;
     p.scale = scale;
+    const int kb_total = ceil_div(s.d_out, kBlockK);
+    p.kb_per_split = pair ? ceil_div(kb_total, c.dx_split_k) : kb_total;
+    p.split_k = pair ? ceil_div(kb_total, p.kb_per_split) : 1;
+    p.part = (p.split_k > 1) ? reinterpret_cast<float*>(q.base + w.split_part) : nullptr;
     p.rt_out = pair ? nullptr : qt;     // the single-CTA kernel computes Q itself and hands it on
     p.ld_rt = w.ld_t;
     p.status = pl->d_status;
@@ -453,6 +504,12 @@ int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const
                                 : launch_gemm_dx(tmdY, tmW, tmB, tmA, tmdX, p, c.dx_ctas, st);
     if (le != cudaSuccess) return LORA_ERR_CUDA;
     g_launches.fetch_add(1);
+    if (p.split_k > 1) {
+      if (launch_splitk_reduce(p.part, static_cast<__nv_bfloat16*>(dX), static_cast<long long>(s.T) * s.d_in, p.split_k, st) !=
+          cudaSuccess)
+        return LORA_ERR_CUDA;
+      g_launches.fetch_add(1);
+    }
   }
   return LORA_OK;
 }
@@ -643,11 +700,11 @@ int lora_plan_describe(const lora_plan_t* plan, char* buf, size_t n) {
   const lora_kernel_config_t& c = plan->cfg;
   std::snprintf(buf, n,
                 "T=%lld d_in=%lld d_out=%lld r=%lld | sms=%d cta_group=%d tile fwd %dx%dx64 dx %dx%dx64 stages=%d/%d group_m=%d "
-                "split_k=%d r_pad=%d ctas fwd=%d dx=%d tail_delay=%d | grad chunk=%d/%d stages=%d/%d dA grid=%dx%d dB grid=%dx%d "
+                "split_k=%d/%d r_pad=%d ctas fwd=%d dx=%d tail_delay=%d | grad chunk=%d/%d stages=%d/%d dA grid=%dx%d dB grid=%dx%d "
                 "| bwd workspace=%zu B",
                 (long long)plan->shape.T, (long long)plan->shape.d_in, (long long)plan->shape.d_out,
                 (long long)plan->shape.r, plan->num_sms, c.cta_group, c.block_m, c.fwd_block_n, c.block_m, c.dx_block_n,
-                c.stages, c.dx_stages, c.group_m, c.split_k,
+                c.stages, c.dx_stages, c.group_m, c.split_k, c.dx_split_k,
                 c.r_pad, c.fwd_ctas, c.dx_ctas, c.tail_delay, c.grad_feat_chunk, c.db_feat_chunk, c.grad_stages, c.db_stages,
                 c.da_feat_chunks,
                 c.da_token_chunks, c.db_feat_chunks, c.db_token_chunks, plan->ws.total);

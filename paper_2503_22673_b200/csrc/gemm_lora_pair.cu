@@ -116,7 +116,11 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
 
   const int G = gridDim.x >> 1;                 // CTA pairs
   const int pair = blockIdx.x >> 1;
-  const int n_my = (p.num_tiles > pair) ? (p.num_tiles - 1 - pair) / G + 1 : 0;
+  // work items: (tile, k-split).  split_k > 1 only in the K-extended form: each item covers kb_per_split main k-blocks,
+  // the last split also the rank-r k-block, and the epilogue writes an fp32 partial tile instead of bf16 output
+  const int SK = kExt ? p.split_k : 1;
+  const int n_items = p.num_tiles * SK;
+  const int n_my = (n_items > pair) ? (n_items - 1 - pair) / G + 1 : 0;
   const int KB = p.kblocks;
   const int D = min(KB, p.tail_delay);
   const int S = p.stages;
@@ -199,14 +203,16 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
     // epilogue meanwhile).  K-extended: the rank-r item is simply the last k-block of its own tile.
     int prev_n0 = 0;
     for (int i = 0; i < n_my && ok; ++i) {
-      const PairTile tc = pair_tile(pair + i * G, p);
+      const int item = pair + i * G, sp = item % SK;
+      const PairTile tc = pair_tile(item / SK, p);
       const int m0 = tc.m_idx * kPairBlockM + static_cast<int>(rank) * 128, n0 = tc.n_idx * BN;
-      for (int kb = 0; kb < KB && ok; ++kb) {
+      const int kb0 = sp * p.kb_per_split, kb1 = min(KB, kb0 + p.kb_per_split);
+      for (int kb = kb0; kb < kb1 && ok; ++kb) {
         if (!kExt && i > 0 && kb == D) load_tail(0, prev_n0);
         if (ok) load_main(m0, n0, kb * kBlockK);
       }
       if (!kExt && ok && i > 0 && D == KB) load_tail(0, prev_n0);
-      if (kExt && ok) load_tail(m0, n0);
+      if (kExt && ok && sp == SK - 1) load_tail(m0, n0);
       prev_n0 = n0;
     }
     if (!kExt && ok && n_my > 0) load_tail(0, prev_n0);
@@ -227,7 +233,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       int slot = 0, phase = 0;
       bool ok = true;
       auto next = [&]() { if (++slot == S) { slot = 0; phase ^= 1; } };
-      auto mma_main = [&](int buf, bool first_kb, bool last_kb) {
+      auto mma_main = [&](int buf, bool first_kb, bool last_kb, bool has_tail) {
         ok = warp_wait(full_bar(slot), phase, abort_flag, p.status, DEV_TIMEOUT_FULL, true, 0);
         if (!ok) return;
         tc_fence_after();
@@ -242,6 +248,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
           }
           mma_commit_pair(empty_bar(slot));
           if (!kExt && last_kb) mma_commit_pair(side_full(buf));
+          if (kExt && last_kb && !has_tail) mma_commit_pair(acc_full(buf));
         }
         __syncwarp();
         next();
@@ -263,13 +270,16 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       };
       for (int i = 0; i < n_my && ok; ++i) {
         const int buf = i & 1, use = i >> 1;
+        const int sp = (pair + i * G) % SK;
+        const int kb0 = sp * p.kb_per_split, kb1 = min(KB, kb0 + p.kb_per_split);
+        const bool has_tail = !kExt || sp == SK - 1;
         ok = warp_wait(acc_empty(buf), (use & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_ACC_EMPTY, true, 0);
-        for (int kb = 0; kb < KB && ok; ++kb) {
+        for (int kb = kb0; kb < kb1 && ok; ++kb) {
           if (!kExt && i > 0 && kb == D) mma_tail(buf ^ 1, (i - 1) >> 1);
-          if (ok) mma_main(buf, kb == 0, kb == KB - 1);
+          if (ok) mma_main(buf, kb == kb0, kb == kb1 - 1, has_tail);
         }
         if (!kExt && ok && i > 0 && D == KB) mma_tail(buf ^ 1, (i - 1) >> 1);
-        if (kExt && ok) mma_tail(buf, use);
+        if (kExt && ok && has_tail) mma_tail(buf, use);
       }
       if (!kExt && ok && n_my > 0) mma_tail((n_my - 1) & 1, (n_my - 1) >> 1);
     }
@@ -282,7 +292,8 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
     const int full_chunks = BN >> 6;
     const int rem_cols = BN & 63;                  // 0, 16, 32 or 48 columns stored with plain stores
     for (int i = 0; i < n_my; ++i) {
-      const PairTile tc = pair_tile(pair + i * G, p);
+      const int item = pair + i * G, sp = item % SK;
+      const PairTile tc = pair_tile(item / SK, p);
       const int m0 = tc.m_idx * kPairBlockM + static_cast<int>(rank) * 128, n0 = tc.n_idx * BN;
       const int buf = i & 1, use = i >> 1;
       bool ok = true;
@@ -319,6 +330,27 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       ok = warp_wait(acc_full(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_ACC, false, 32);
       if (named_bar_or(1, 128, !ok)) break;
       tc_fence_after();
+      if (kExt && SK > 1) {
+        // ---- split along K: this item's fp32 partial tile -> part[sp][row][col], 16 columns at a time ----
+        float* prow = p.part + (static_cast<size_t>(sp) * p.M + (m0 + row)) * p.N;
+        for (int c16 = 0; c16 < BN / 16; ++c16) {
+          uint32_t v[16];
+          tmem_ld16(lane_addr + buf * 256 + c16 * 16, v);
+          tmem_ld_wait();
+          if (c16 == BN / 16 - 1) {
+            tc_fence_before();
+            mbar_arrive_cluster(map_to_cta(acc_empty(buf), 0));
+          }
+          const int col = n0 + c16 * 16;
+          if (m0 + row < p.M) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              if (col + 4 * q < p.N)
+                *reinterpret_cast<uint4*>(prow + col + 4 * q) = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+          }
+        }
+        continue;
+      }
       for (int c = 0; c < full_chunks; ++c) {
         uint32_t v0[32], v1[32];
         tmem_ld32(lane_addr + buf * 256 + c * 64, v0);
@@ -406,7 +438,37 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
   }
 }
 
+// out[t, n] = bf16( sum over k-splits of part[sp][t][n] ), splits added in index order; 8 outputs per thread
+__global__ void __launch_bounds__(256) lora_splitk_reduce_kernel(const float* part, __nv_bfloat16* out, long long n_elems,
+                                                                int splits) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const long long i = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) * 8;
+  if (i >= n_elems) return;
+  float acc[8];
+#pragma unroll
+  for (int q = 0; q < 8; ++q) acc[q] = 0.f;
+  for (int s = 0; s < splits; ++s) {
+    const float4 a = __ldcg(reinterpret_cast<const float4*>(part + s * n_elems + i));
+    const float4 b = __ldcg(reinterpret_cast<const float4*>(part + s * n_elems + i + 4));
+    acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
+    acc[4] += b.x; acc[5] += b.y; acc[6] += b.z; acc[7] += b.w;
+  }
+  uint4 w;
+  w.x = pack_bf16x2(acc[0], acc[1]);
+  w.y = pack_bf16x2(acc[2], acc[3]);
+  w.z = pack_bf16x2(acc[4], acc[5]);
+  w.w = pack_bf16x2(acc[6], acc[7]);
+  *reinterpret_cast<uint4*>(out + i) = w;
+}
+
 }  // namespace
+
+cudaError_t launch_splitk_reduce(const float* part, __nv_bfloat16* out, long long n_elems, int splits, cudaStream_t stream) {
+  const long long threads = (n_elems + 7) / 8;
+  return launch_pdl(lora_splitk_reduce_kernel, dim3(static_cast<unsigned>((threads + 255) / 256)), dim3(256), 0, stream, part,
+                    out, n_elems, splits);
+}
 
 size_t gemm_pair_smem_bytes(int stages) {
   return static_cast<size_t>(stages) * kPairStageBytesFwd + 2 * kStagingBytes + kGemmBarriers * 8 + 16 + 1024;

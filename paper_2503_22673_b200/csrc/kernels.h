@@ -51,6 +51,9 @@ struct GemmParams {
   __nv_bfloat16* rt_out;  // backward only: scale * (dY B)^T as bf16 [r_pad][ld_rt]; nullptr otherwise
   int ld_rt;
   unsigned* status;       // device status word
+  int split_k;            // K-extended pair kernel: k-splits per tile (1 = none) and main k-blocks per split
+  int kb_per_split;
+  float* part;            // fp32 partial tiles [split_k][M][N] when split_k > 1
   __nv_bfloat16* out;     // CTA-pair kernel only: output base and row pitch (elements) for the ragged last chunk
   int ld_out;
 };
@@ -63,6 +66,8 @@ constexpr int kPairThreads = 288;           // warps 0..3 TMA producers, warp 4 
 constexpr int kPairStageBytesFwd = 32768;   // 128 x 64 activations + 128 x 64 weight/adapter rows per CTA
 size_t gemm_pair_smem_bytes(int stages);
 cudaError_t gemm_pair_configure();
+// out = bf16(sum of the split_k fp32 partial matrices), fixed order (M x N must be a multiple of 8 elements)
+cudaError_t launch_splitk_reduce(const float* part, __nv_bfloat16* out, long long n_elems, int splits, cudaStream_t stream);
 // forward: tmW0 = W box 64 x half rows (leader CTA), tmW1 = W box 64 x (block_n - half) rows (peer CTA),
 // half = (block_n + r_pad) / 2; tmA box 64 x r_pad; tmB box 64 x block_n/2 rows
 cudaError_t launch_gemm_pair_fwd(const CUtensorMap& tmX, const CUtensorMap& tmW0, const CUtensorMap& tmW1,

@@ -308,3 +308,20 @@ def test_grouped_projections_sharing_x_match_separate_oracles():
         assert oracle.rel_err(host64(dBs[g]), dBr) <= TOL_F32
     assert oracle.rel_err(host64(dX), dX_ref) <= TOL_BF16
     gp.close()
+
+
+def test_split_k_paths_match_oracle(monkeypatch):
+    """Grids that cannot fill the GPU are split along K (fp32 partial tiles + fixed-order reduce).  One shape takes the
+    split by the selector's own rule; the others force it (3 splits) on ragged shapes, forward and dX."""
+    p, t = inputs.draw_custom(257, 14336, 264, 64, 0.5, seed=23)
+    cfg = binding.select_config(p.T, p.d_in, p.d_out, p.r)
+    assert cfg["split_k"] > 1 and cfg["fwd_ext"] == 1
+    check_full(p, t)
+    monkeypatch.setenv("LORA_FORCE_SPLIT_K", "3")
+    for shape in [(700, 520, 392, 16, 2.0), (300, 2048, 1032, 24, 1.7)]:
+        p, t = inputs.draw_custom(*shape, seed=24)
+        a, _ = check_full(p, t)
+        b, _ = check_full(p, t)
+        for k in a:                                   # still bitwise reproducible
+            it = torch.int32 if a[k].dtype == torch.float32 else torch.int16
+            assert torch.equal(a[k].view(it), b[k].view(it)), k
