@@ -21,6 +21,7 @@ Pins (tests/test_oracle.py): a hand-derived rank-1 example stored under tests/go
 pure-Python triple loops on tiny inputs, central finite differences of L = <dY, Y>,
 the merged-weight identity Y = X (W + s B A)^T, the closed forms for B = 0 / A = 0 / W = 0,
 linearity in s, and the adjoint identities <dY,Y> = <dX,X>, <dA,A> = <dB,B>.
+Every function here has at least one such pin; none is "parity unpinned".
 """
 from __future__ import annotations
 
@@ -72,6 +73,18 @@ def backward_adapter_grads(dY, X, A, B, s: float):
     dA = s * ((dY @ B).T @ X)
     dB = s * (dY.T @ (X @ A.T))
     return dA, dB
+
+
+def dense_weight_grad(dY, X) -> np.ndarray:
+    """dW = dY^T X, the gradient of L = <dY, X W^T> with respect to W itself.
+
+    This is the extra contraction full fine-tuning pays for and LoRA avoids (Section 4.5,
+    "Full-model tuning": every weight is updated).  dW[o, i] = sum_t dY[t, o] X[t, i].
+    Pins (tests/test_oracle.py): a hand-derived small example under tests/golden/, Python loops,
+    central differences of L in W, and the two projections dA = s B^T dW, dB = s dW A^T that
+    tie it to the adapter gradients above.
+    """
+    return _f64(dY).T @ _f64(X)
 
 
 def rel_err(got, ref) -> float:

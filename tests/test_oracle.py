@@ -223,6 +223,37 @@ def test_rel_err_measure():
         oracle.rel_err(np.zeros((2, 2)), np.zeros((2, 3)))
 
 
+# ---------------------------------------------------------------- dense weight gradient (full fine-tuning)
+def test_dense_weight_grad_hand_example_is_exact():
+    g = _read_golden(os.path.join(os.path.dirname(__file__), "golden", "dense_dw_example.txt"))
+    dW = oracle.dense_weight_grad(g["dY"], g["X"])
+    assert np.array_equal(dW, g["dW"])
+    assert not np.array_equal(g["X"].T @ g["dY"][:, :2], g["dW"][:2])       # transposed operands are rejected
+
+
+def test_dense_weight_grad_loops_differences_and_projections():
+    X, W, A, B, dY = _tiny(17, T=7, d_in=5, d_out=4, r=2)
+    s, h = 1.3, 1e-3
+    dW = oracle.dense_weight_grad(dY, X)
+    assert dW.shape == W.shape
+    # pure-Python loops
+    ref = [[sum(dY[t][o] * X[t][i] for t in range(7)) for i in range(5)] for o in range(4)]
+    np.testing.assert_allclose(dW, np.array(ref), rtol=1e-12, atol=1e-12)
+    # L = <dY, Y(W)> is linear in W: central differences are exact up to rounding
+    for idx in np.ndindex(W.shape):
+        e = np.zeros_like(W)
+        e[idx] = h
+        fd = (np.sum(dY * oracle.forward(X, W + e, A, B, s)) - np.sum(dY * oracle.forward(X, W - e, A, B, s))) / (2 * h)
+        assert abs(fd - dW[idx]) <= 1e-8 * max(1.0, abs(dW[idx]))
+    # the adapter gradients are projections of dW (chain rule through W + s B A)
+    _, dA, dB = oracle.backward(dY, X, W, A, B, s)
+    np.testing.assert_allclose(s * np.einsum("oj,oi->ji", B, dW), dA, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(s * np.einsum("oi,ji->oj", dW, A), dB, rtol=1e-12, atol=1e-12)
+    # sums over token rows: two halves add up
+    np.testing.assert_allclose(oracle.dense_weight_grad(dY[:3], X[:3]) + oracle.dense_weight_grad(dY[3:], X[3:]), dW,
+                               rtol=1e-12, atol=1e-12)
+
+
 # ---------------------------------------------------------------- the pins bite
 def test_planted_mistakes_are_caught():
     """Plant plausible mistakes in copies of the oracle formulas (on the CPU) and check that
