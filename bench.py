@@ -59,20 +59,29 @@ def gemm_source_sha() -> str:
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+    """Samples SM clocks and throttle reasons with nvidia-smi (every 20 ms, timestamped) while the GPU works."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
         self.proc = None
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50"],
+                ["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
 
-    def stop(self):
+    @staticmethod
+    def _epoch(stamp: str):
+        import datetime
+        try:
+            return datetime.datetime.strptime(stamp.strip(), "%Y/%m/%d %H:%M:%S.%f").timestamp()
+        except ValueError:
+            return None
+
+    def stop(self, t0: float = None, t1: float = None):
+        """Summary of the samples taken between host times t0 and t1 (all samples when none fall inside)."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -81,22 +90,23 @@ class ClockSampler:
         except subprocess.TimeoutExpired:
             self.proc.kill()
             out, _ = self.proc.communicate()
-        sm, mx, reasons = [], [], set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        rows = []
         for line in out.splitlines():
             parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 6:
+            if len(parts) < 7:
                 continue
             try:
-                sm.append(float(parts[0]))
-                mx.append(float(parts[1]))
+                rows.append((self._epoch(parts[0]), float(parts[1]), float(parts[2]),
+                             [n for n, v in zip(names, parts[3:7]) if v.lower().startswith("active")]))
             except ValueError:
                 continue
-            for n, v in zip(names, parts[2:6]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        inside = [r for r in rows if t0 is not None and r[0] is not None and t0 <= r[0] <= t1]
+        window = "timed region" if inside else "whole run (no sample fell inside the timed region)"
+        use = inside if inside else rows
+        sm = [r[1] for r in use]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(r[2] for r in use) if use else None,
+                "samples": len(use), "window": window, "reasons": sorted({n for r in use for n in r[3]})}
 
 
 def max_over_ranks(value: float, device, world: int) -> float:
@@ -309,23 +319,41 @@ def run_ours(args):
         if code != 0:
             raise SystemExit(f"bench.py: device status after warm-up: {msg}")
 
-    # ---- timed region: K steps, device-timed, per-kernel events inside ----
-    events = [[[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in protos] for _ in range(args.steps)]
+    # ---- timed region: K steps back to back, device-timed (events only around the region) ----
     ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler is not None:
+        for k in range(n_warm):          # keep the GPU under the same load while nvidia-smi starts sampling
+            step(k)
     launches0 = binding.launch_count()
     barrier()
     torch.cuda.synchronize()
+    t_host0 = time.time()
     ev_a.record()
     for k in range(args.steps):
-        step(n_warm + k, events[k])
+        step(n_warm + k)
     ev_b.record()
     torch.cuda.synchronize()
+    t_host1 = time.time()
     barrier()
     launches = binding.launch_count() - launches0
-    clocks = sampler.stop() if sampler is not None else None
     ms_total = max_over_ranks(ev_a.elapsed_time(ev_b), device, world)
     ms_step = ms_total / args.steps
+
+    # ---- the same steps once more with events between the kernels: per-kernel durations.  An event record between two
+    #      launches suppresses their programmatic overlap, so this pass is a little slower than the timed region; its
+    #      own per-step time is reported as ms_per_step_instrumented ----
+    events = [[[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in protos] for _ in range(args.steps)]
+    i_a, i_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    i_a.record()
+    for k in range(args.steps):
+        step(n_warm + k, events[k])
+    i_b.record()
+    torch.cuda.synchronize()
+    t_host2 = time.time()
+    ms_step_instr = i_a.elapsed_time(i_b) / args.steps
+    clocks = sampler.stop(t_host0, t_host2) if sampler is not None else None
 
     # per-kernel mean durations (ms) and rooflines
     kern = {}
@@ -381,6 +409,33 @@ def run_ours(args):
     variants = {"bwd_saved_p": {"ms_per_step": ms_var, "value": job_value(world, flops_step, ms_var), "unit": UNIT,
                                 "steps": n_var, "note": "forward + lora_linear_bwd_saved_p (X A^T kept from the forward)"}}
 
+    # ---- extra kernel: the dense weight gradient of full fine-tuning, dW = dY^T X (lora_dense_dw), per projection ----
+    dw_out = [torch.empty((p.d_out, p.d_in), dtype=torch.bfloat16, device=device) for p in protos]
+
+    def step_dw(k):
+        cur = sets[k % n_sets]
+        for j, (proj, d) in enumerate(cur):
+            plans[j].dense_dw(d["dY"], d["X"], dw_out[j])
+
+    for k in range(3):
+        step_dw(k)
+    torch.cuda.synchronize()
+    w_a, w_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    w_a.record()
+    for k in range(n_var):
+        step_dw(3 + k)
+    w_b.record()
+    torch.cuda.synchronize()
+    barrier()
+    ms_dw = max_over_ranks(w_a.elapsed_time(w_b) / n_var, device, world)
+    dw_flops = float(sum(2.0 * p.T * p.d_in * p.d_out for p in protos))
+    variants["full_ft_dense_dw"] = {"ms_per_step": ms_dw, "value": job_value(world, dw_flops, ms_dw), "unit": UNIT,
+                                    "frac_of_bf16_peak": dw_flops / ms_dw / 1e9 / pk["bf16_tflops"], "steps": n_var,
+                                    "note": "lora_dense_dw alone (dW = dY^T X, 2 T d_in d_out FLOPs per projection); not part "
+                                            "of the LoRA step"}
+    del dw_out
+
     # ---- end to end: host buffers through the C ABI, copies inside the timed region ----
     h_sets, staging = [], []
     for j, (p, d0) in enumerate(sets[0]):
@@ -420,8 +475,8 @@ def run_ours(args):
     value = job_value(world, flops_step, ms_step)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": n_warm,
-        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
+        "ms_per_step": ms_step, "ms_per_step_instrumented": ms_step_instr, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": workload_name(args.workload), "projections": [p.name for p in protos], "T": protos[0].T,
                    "r": protos[0].r, "scale": protos[0].scale, "input_sets_rotated": n_sets, "grouped": bool(args.grouped and args.workload == 4),
                    "l2": f"{n_sets} independent input/output sets ({bytes_per_set * n_sets / 2**20:.0f} MiB) rotated per step; "

@@ -89,6 +89,9 @@ typedef struct lora_kernel_config {
   int32_t q_stages;
   int32_t dx_split_k;      /* k-splits per tile of the dX GEMM                                           */
   int32_t fwd_ext;         /* 1: forward runs as X A^T pre-pass + K-extended GEMM (needs the workspace)  */
+  int32_t dw_block_n;      /* dense weight gradient GEMM (lora_dense_dw): d_in columns per tile,         */
+  int32_t dw_split_k;      /*   splits along the tokens, persistent CTAs                                 */
+  int32_t dw_ctas;
 } lora_kernel_config_t;
 
 /* Host-only: run the tile / split selector for a shape on a device with `num_sms` SMs.
@@ -147,6 +150,15 @@ int lora_linear_bwd_dx(lora_plan_t* plan, const void* dY, const void* W, const v
                        float scale, void* dX, void* stream);
 int lora_linear_bwd_da(lora_plan_t* plan, const void* X, const void* A, float scale, void* dA, void* stream);
 int lora_linear_bwd_db(lora_plan_t* plan, const void* dY, float scale, void* dB, void* stream);
+
+/* Dense weight gradient of full fine-tuning (Section 4.5, "Full-model tuning": every weight is updated, so the frozen-W
+ * shortcut of LoRA no longer applies and the layer also owes  dW = dY^T X):
+ *     dW[o, i] = sum_t dY[t, o] X[t, i]        dY [T, d_out] bf16, X [T, d_in] bf16  ->  dW [d_out, d_in] bf16
+ * One tcgen05 GEMM over CTA pairs with both operands read token-major as they are (no transposed copies), fp32
+ * accumulation over all T tokens, one rounding to bf16.  dW is overwritten; T = 0 gives zeros.  The plan's r plays no
+ * role.  Needs the workspace only when the selector split the contraction (cfg.dw_split_k > 1: few output tiles, many
+ * tokens); then the splits are summed in a fixed order.  Independent of the other calls. */
+int lora_dense_dw(lora_plan_t* plan, const void* dY, const void* X, void* dW, void* stream);
 
 /* One training step of the layer with HOST input/output buffers: copies h_X, h_A, h_B, h_dY to the
  * device staging area, runs forward and backward, copies Y, dX, dA, dB back, all on `stream`

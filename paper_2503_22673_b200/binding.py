@@ -27,7 +27,7 @@ EXPORTS = [
     "lora_select_config", "lora_workspace_bytes", "lora_plan_create", "lora_plan_destroy",
     "lora_plan_workspace_bytes", "lora_plan_set_workspace", "lora_plan_get_config", "lora_plan_describe",
     "lora_linear_fwd", "lora_linear_bwd", "lora_linear_bwd_saved_p", "lora_linear_bwd_dx", "lora_linear_bwd_da", "lora_linear_bwd_db",
-    "lora_step_host_staging_bytes", "lora_linear_step_host",
+    "lora_dense_dw", "lora_step_host_staging_bytes", "lora_linear_step_host",
     "lora_last_device_status", "lora_strerror", "lora_launch_count",
     "lora_grad_contract_noalloc", "lora_grad_contract_noalloc_max_scratch",
 ]
@@ -41,7 +41,7 @@ class LoraKernelConfig(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "block_m", "fwd_block_n", "dx_block_n", "block_k", "stages", "group_m", "split_k", "r_pad", "fwd_ctas",
         "dx_ctas", "tail_delay", "grad_feat_chunk", "grad_stages", "da_feat_chunks", "da_token_chunks",
-        "db_feat_chunks", "db_token_chunks", "db_feat_chunk", "cta_group", "dx_stages", "prefetch_dist", "db_stages", "q_feat_chunk", "q_feat_chunks", "q_token_chunks", "q_stages", "dx_split_k", "fwd_ext")]
+        "db_feat_chunks", "db_token_chunks", "db_feat_chunk", "cta_group", "dx_stages", "prefetch_dist", "db_stages", "q_feat_chunk", "q_feat_chunks", "q_token_chunks", "q_stages", "dx_split_k", "fwd_ext", "dw_block_n", "dw_split_k", "dw_ctas")]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
@@ -79,6 +79,7 @@ def load(rebuild: bool = False) -> ctypes.CDLL:
     lib.lora_linear_bwd_dx.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp]
     lib.lora_linear_bwd_da.argtypes = [vp, vp, vp, ctypes.c_float, vp, vp]
     lib.lora_linear_bwd_db.argtypes = [vp, vp, ctypes.c_float, vp, vp]
+    lib.lora_dense_dw.argtypes = [vp, vp, vp, vp, vp]
     lib.lora_step_host_staging_bytes.argtypes = [ctypes.POINTER(LoraShape), sz_p]
     lib.lora_linear_step_host.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp,
                                           ctypes.c_size_t, vp]
@@ -244,6 +245,19 @@ class LoraLinearPlan:
         _check(fn(self._h, _ptr(dY), _ptr(X), _ptr(W), _ptr(A), _ptr(B), float(scale),
                   _ptr(dX), _ptr(dA), _ptr(dB), _stream_ptr(stream)), "lora_linear_bwd")
         return dX, dA, dB
+
+    def dense_dw(self, dY, X, dW: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """dW = dY^T X, the weight gradient of full fine-tuning ([d_out, d_in] bf16)."""
+        bf = torch.bfloat16
+        _want(dY, "dY", (self.T, self.d_out), bf, self.device)
+        _want(X, "X", (self.T, self.d_in), bf, self.device)
+        if dW is None:
+            dW = torch.empty((self.d_out, self.d_in), dtype=bf, device=self.device)
+        _want(dW, "dW", (self.d_out, self.d_in), bf, self.device)
+        if self.config()["dw_split_k"] > 1:
+            self.ensure_workspace()
+        _check(self._lib.lora_dense_dw(self._h, _ptr(dY), _ptr(X), _ptr(dW), _stream_ptr(stream)), "lora_dense_dw")
+        return dW
 
     def bwd_stages(self, dY, X, W, A, B, scale: float, dX, dA, dB, stream=None, events=None):
         """The same three kernels as ``bwd``, issued through the stage entry points; ``events`` (four

@@ -181,6 +181,28 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
     c->fwd_ctas = static_cast<int>(fwd_tiles < num_sms ? fwd_tiles : num_sms);
     c->dx_ctas = static_cast<int>(dx_tiles < num_sms ? dx_tiles : num_sms);
   }
+  if (num_sms >= 2) {
+    // dense weight gradient dW = dY^T X (always on CTA pairs): output rows = d_out, columns = d_in, contraction over
+    // the tokens; same tile-width and split rules as the GEMMs above
+    const int pairs = num_sms / 2;
+    c->dw_block_n = pick_pair_block_n(s->d_out, s->d_in, 0, pairs);
+    const long long tiles = static_cast<long long>(ceil_div(s->d_out, kPairBlockM)) * ceil_div(s->d_in, c->dw_block_n);
+    const int kb = ceil_div(T, kBlockK);
+    long long sp = 1;
+    if (tiles * 4 <= pairs && kb >= 64) {
+      sp = pairs / tiles;
+      if (sp > kb / 16) sp = kb / 16;
+      if (sp > 8) sp = 8;
+      if (sp < 1) sp = 1;
+    }
+    c->dw_split_k = static_cast<int>(sp);
+    const long long items = tiles * sp;
+    c->dw_ctas = 2 * static_cast<int>(items < pairs ? items : pairs);
+  } else {
+    c->dw_block_n = 0;
+    c->dw_split_k = 1;
+    c->dw_ctas = 0;
+  }
   if (const char* f = std::getenv("LORA_FORCE_STAGES")) {   // tuning knob: shallower rings
     const int v = std::atoi(f);
     if (v >= 2 && v <= c->stages) c->stages = v;
@@ -249,8 +271,9 @@ WsLayout ws_layout(const lora_shape_t& s, const lora_kernel_config_t& c) {
   {
     const size_t f = c.split_k > 1 ? static_cast<size_t>(c.split_k) * T * s.d_out * 4 : 0;
     const size_t b = c.dx_split_k > 1 ? static_cast<size_t>(c.dx_split_k) * T * s.d_in * 4 : 0;
+    const size_t g = c.dw_split_k > 1 ? static_cast<size_t>(c.dw_split_k) * s.d_out * s.d_in * 4 : 0;
     w.split_part = off;
-    off += align_up(f > b ? f : b, kAlign);
+    off += align_up(f > b ? (f > g ? f : g) : (b > g ? b : g), kAlign);
   }
   w.total = off;
   return w;
@@ -599,6 +622,46 @@ int launch_db(lora_plan* pl, const void* dY, float scale, void* dB, cudaStream_t
   return LORA_OK;
 }
 
+// ---- dW = dY^T X (full fine-tuning): plain GEMM with both operands MN-major, contraction over the tokens ----
+int launch_dw(lora_plan* pl, const void* dY, const void* X, void* dW, cudaStream_t st) {
+  const lora_shape_t& s = pl->shape;
+  const lora_kernel_config_t& c = pl->cfg;
+  CUtensorMap tmdY, tmX, tmdW;
+  bool ok = make_bf16_tmap(&tmdY, dY, s.d_out, s.T, s.d_out, 64, 64);
+  ok = ok && make_bf16_tmap(&tmX, X, s.d_in, s.T, s.d_in, 64, 64);
+  ok = ok && make_bf16_tmap(&tmdW, dW, s.d_in, s.d_out, s.d_in, 64, kBlockM);
+  if (!ok) return LORA_ERR_CUDA;
+  GemmParams p{};
+  p.out = static_cast<__nv_bfloat16*>(dW);
+  p.ld_out = static_cast<int>(s.d_in);
+  p.M = static_cast<int>(s.d_out);
+  p.N = static_cast<int>(s.d_in);
+  p.K = static_cast<int>(s.T);
+  p.r_pad = 0;
+  p.block_n = c.dw_block_n;
+  p.tiles_m = ceil_div(s.d_out, kPairBlockM);
+  p.tiles_n = ceil_div(s.d_in, c.dw_block_n);
+  p.num_tiles = p.tiles_m * p.tiles_n;
+  p.kblocks = ceil_div(s.T, kBlockK);
+  p.group_m = c.group_m;
+  p.stages = 6;
+  p.tail_delay = c.tail_delay;
+  p.scale = 1.f;
+  p.kb_per_split = ceil_div(p.kblocks, c.dw_split_k);
+  p.split_k = ceil_div(p.kblocks, p.kb_per_split);
+  p.part = (p.split_k > 1) ? reinterpret_cast<float*>(static_cast<uint8_t*>(pl->workspace) + pl->ws.split_part) : nullptr;
+  p.status = pl->d_status;
+  if (launch_gemm_pair_dw(tmdY, tmX, tmdW, p, c.dw_ctas, st) != cudaSuccess) return LORA_ERR_CUDA;
+  g_launches.fetch_add(1);
+  if (p.split_k > 1) {
+    if (launch_splitk_reduce(p.part, static_cast<__nv_bfloat16*>(dW), static_cast<long long>(s.d_out) * s.d_in, p.split_k, st) !=
+        cudaSuccess)
+      return LORA_ERR_CUDA;
+    g_launches.fetch_add(1);
+  }
+  return LORA_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -802,6 +865,22 @@ int lora_linear_bwd_db(lora_plan_t* plan, const void* dY, float scale, void* dB,
   if (!aligned16(dY)) return LORA_ERR_MISALIGNED;
   if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
   return launch_db(plan, dY, scale, dB, static_cast<cudaStream_t>(stream));
+}
+
+int lora_dense_dw(lora_plan_t* plan, const void* dY, const void* X, void* dW, void* stream) {
+  if (plan == nullptr || !dW) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(dW)) return LORA_ERR_MISALIGNED;
+  if (plan->num_sms < 2) return LORA_ERR_NO_DEVICE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  DeviceGuard guard(plan->device);
+  if (plan->shape.T == 0)     // empty batch: the sum over tokens is empty
+    return cudaMemsetAsync(dW, 0, sizeof(__nv_bfloat16) * plan->shape.d_out * plan->shape.d_in, st) == cudaSuccess
+               ? LORA_OK : LORA_ERR_CUDA;
+  if (!dY || !X) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(dY) || !aligned16(X)) return LORA_ERR_MISALIGNED;
+  if (plan->cfg.dw_split_k > 1 && (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total))
+    return LORA_ERR_WORKSPACE;
+  return launch_dw(plan, dY, X, dW, st);
 }
 
 int lora_step_host_staging_bytes(const lora_shape_t* shape, size_t* bytes) {

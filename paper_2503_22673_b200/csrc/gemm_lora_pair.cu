@@ -52,9 +52,12 @@ __device__ __forceinline__ PairTile pair_tile(int id, const GemmParams& p) {
 // kBmn: the weight-side operands (W, and A in the rank-r k-block) are MN-major (backward) instead of K-major.
 // kExt: K-extended form - the scaled first adapter product (Pt or Qt, [r_pad, T] bf16) was computed beforehand and
 //       enters as one more k-block; otherwise (forward only) it is fused: extra accumulator columns + epilogue.
-template <bool kBmn, bool kExt>
+//       With r_pad = 0 the K-extended form has no rank-r k-block at all: a plain GEMM.
+// kAmn: the activation-side operand is MN-major too: its tensor is [K, M] row-major (box 64(m) x 64(k), two per stage).
+//       This is the dense weight gradient dW = dY^T X, where both operands are contracted over their row index.
+template <bool kBmn, bool kExt, bool kAmn = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
-lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M, K], box 64(k) x 128
+lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M, K], box 64(k) x 128 ; kAmn: [K, M], box 64(m) x 64(k)
                       const __grid_constant__ CUtensorMap tm_w0,    // fwd: W box 64(k) x half ; bwd: W box 64(n) x 64(k)
                       const __grid_constant__ CUtensorMap tm_w1,    // fwd: W box 64(k) x (block_n - half) ; bwd unused
                       const __grid_constant__ CUtensorMap tm_side,  // fwd: A box 64(k) x r_pad ; bwd: Qt [r_pad, T] box 64(t) x r_pad
@@ -151,7 +154,12 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       if (elect_one()) {
         if (op == 0) {
           if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), 2 * 16384);
-          tma_load_2d_pair(a_dst, &tm_act, fb, k0, m0);
+          if (!kAmn) {
+            tma_load_2d_pair(a_dst, &tm_act, fb, k0, m0);
+          } else {
+            tma_load_2d_pair(a_dst, &tm_act, fb, m0, k0);
+            tma_load_2d_pair(a_dst + 8192, &tm_act, fb, m0 + 64, k0);
+          }
         } else if (!kExt) {
           if (rank == 0) {
             mbar_arrive_expect_tx(full_bar(cur), (BN + p.r_pad) * 128);
@@ -212,7 +220,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
         if (ok) load_main(m0, n0, kb * kBlockK);
       }
       if (!kExt && ok && i > 0 && D == KB) load_tail(0, prev_n0);
-      if (kExt && ok && sp == SK - 1) load_tail(m0, n0);
+      if (kExt && ok && sp == SK - 1 && p.r_pad > 0) load_tail(m0, n0);
       prev_n0 = n0;
     }
     if (!kExt && ok && n_my > 0) load_tail(0, prev_n0);
@@ -221,9 +229,10 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
     // Whole warp of the leader CTA runs the loop; one lane polls, one elected lane issues every MMA and commit.
     // Descriptors are advanced by adding byte offsets (>> 4) to precomputed bases.
     if (rank == 0) {
-      const uint32_t idesc_main = kExt ? mma_idesc_bf16(256, BN, false, kBmn) : mma_idesc_bf16(256, BN + p.r_pad, false, false);
+      const uint32_t idesc_main = kExt ? mma_idesc_bf16(256, BN, kAmn, kBmn) : mma_idesc_bf16(256, BN + p.r_pad, false, false);
       const uint32_t idesc_tail = mma_idesc_bf16(256, BN, kExt, kBmn);   // K-extended: Pt / Qt is an MN-major A operand
-      const uint64_t ad0 = smem_desc_sw128(ring, 16, 1024);
+      const uint64_t ad0 = kAmn ? smem_desc_sw128(ring, 8192, 1024) : smem_desc_sw128(ring, 16, 1024);
+      constexpr uint32_t kAStep = kAmn ? (2048 >> 4) : (32 >> 4);
       const uint64_t bd0 = kBmn ? smem_desc_sw128(ring + 16384, 8192, 1024) : smem_desc_sw128(ring + 16384, 16, 1024);
       // rank-r A operand: forward = bf16 s*P rows written by the epilogue (K-major, in the staging buffer);
       // backward = Qt tile delivered by TMA into the stage's activation part (MN-major, two 64-token groups)
@@ -243,7 +252,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
 #pragma unroll
           for (int ks = 0; ks < kBlockK / 16; ++ks) {
             const uint32_t accum = (!first_kb || ks != 0) ? 1u : 0u;
-            const uint64_t ad = ad0 + so + ks * 2;
+            const uint64_t ad = ad0 + so + ks * kAStep;
             mma_bf16_ss_pair(acc, ad, bd0 + so + ks * kBStep, idesc_main, accum);
           }
           mma_commit_pair(empty_bar(slot));
@@ -272,7 +281,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
         const int buf = i & 1, use = i >> 1;
         const int sp = (pair + i * G) % SK;
         const int kb0 = sp * p.kb_per_split, kb1 = min(KB, kb0 + p.kb_per_split);
-        const bool has_tail = !kExt || sp == SK - 1;
+        const bool has_tail = !kExt || (sp == SK - 1 && p.r_pad > 0);
         ok = warp_wait(acc_empty(buf), (use & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_ACC_EMPTY, true, 0);
         for (int kb = kb0; kb < kb1 && ok; ++kb) {
           if (!kExt && i > 0 && kb == D) mma_tail(buf ^ 1, (i - 1) >> 1);
@@ -480,6 +489,8 @@ cudaError_t gemm_pair_configure() {
     e = cudaFuncSetAttribute(lora_gemm_pair_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(lora_gemm_pair_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(lora_gemm_pair_kernel<true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
   return e;
 }
 
@@ -502,6 +513,12 @@ cudaError_t launch_gemm_pair_dx(const CUtensorMap& tmdY, const CUtensorMap& tmW,
                                 cudaStream_t stream) {
   return launch_pdl(lora_gemm_pair_kernel<true, true>, dim3(ctas), dim3(kPairThreads), gemm_pair_smem_bytes(p.stages), stream,
                     tmdY, tmW, tmW, tmQt, tmA, tmdX, p);
+}
+
+cudaError_t launch_gemm_pair_dw(const CUtensorMap& tmdYt, const CUtensorMap& tmX, const CUtensorMap& tmdW, const GemmParams& p,
+                                int ctas, cudaStream_t stream) {
+  return launch_pdl(lora_gemm_pair_kernel<true, true, true>, dim3(ctas), dim3(kPairThreads), gemm_pair_smem_bytes(p.stages),
+                    stream, tmdYt, tmX, tmX, tmX, tmX, tmdW, p);
 }
 
 }  // namespace lora

@@ -83,6 +83,11 @@ cudaError_t launch_gemm_pair_dx(const CUtensorMap& tmdY, const CUtensorMap& tmW,
                                 const CUtensorMap& tmA, const CUtensorMap& tmdX, const GemmParams& p, int ctas,
                                 cudaStream_t stream);
 
+// dense weight gradient dW[d_out, d_in] = dY^T X (p.r_pad = 0: no rank-r k-block): tmdYt = dY [T, d_out] box 64(o) x 64(t),
+// tmX = X [T, d_in] box 64(i) x 64(t), tmdW box 64 x 128; p.M = d_out, p.N = d_in, p.K = T
+cudaError_t launch_gemm_pair_dw(const CUtensorMap& tmdYt, const CUtensorMap& tmX, const CUtensorMap& tmdW, const GemmParams& p,
+                                int ctas, cudaStream_t stream);
+
 // Y / dX = act * Wop + scale * (act * sideop) * tailop, see gemm_lora.cu
 cudaError_t launch_gemm_fwd(const CUtensorMap& tmX, const CUtensorMap& tmW, const CUtensorMap& tmA,
                             const CUtensorMap& tmB, const CUtensorMap& tmY, const GemmParams& p, int ctas,
