@@ -160,6 +160,26 @@ int lora_linear_bwd_db(lora_plan_t* plan, const void* dY, float scale, void* dB,
  * tokens); then the splits are summed in a fixed order.  Independent of the other calls. */
 int lora_dense_dw(lora_plan_t* plan, const void* dY, const void* X, void* dW, void* stream);
 
+/* Quantised LoRA (Section 4.5, "Quantised LoRA" / Q+LoRA): the same layer with the frozen W held in 4-bit NormalFloat
+ * (NF4, Dettmers et al. 2023).  The paper names the data type but no storage layout; this library's is:
+ *   - W [d_out, d_in] is cut into blocks of 64 consecutive elements along d_in (d_in % 64 == 0, d_out % 4 == 0);
+ *   - W_absmax [d_in / 64, d_out] float32, block-major: W_absmax[b, o] = max |W[o, 64 b .. 64 b + 63]|;
+ *   - W_codes [d_out, d_in / 2] uint8: each element's code is the index of the NF4 level nearest to w / absmax
+ *     (float32 division; the lower level on an exact tie; an all-zero block gets code 7 = level 0); byte k of a row holds
+ *     element 2k in its low nibble and element 2k + 1 in its high nibble;
+ *   - the value the GEMMs use is  bf16( float32(level[code]) * absmax )  (one float32 product, one rounding).
+ * lora_nf4_quantize builds codes and scales from a bf16 weight on the device (one warp per block).
+ * lora_linear_fwd_nf4 / lora_linear_bwd_nf4 compute exactly what lora_linear_fwd / lora_linear_bwd compute with that
+ * dequantised weight in place of W; dA and dB do not involve W.  The weight is never materialised in bf16: packed codes
+ * and scales are staged by TMA and expanded inside the GEMM kernels, straight into the tensor-core operand tiles.
+ * Both need the workspace and a plan with T > 128 (CTA-pair kernels); otherwise LORA_ERR_UNSUPPORTED_SHAPE /
+ * LORA_ERR_WORKSPACE.  All pointers are device pointers, 16-byte aligned. */
+int lora_nf4_quantize(const void* W, int64_t d_out, int64_t d_in, void* W_codes, void* W_absmax, void* stream);
+int lora_linear_fwd_nf4(lora_plan_t* plan, const void* X, const void* W_codes, const void* W_absmax, const void* A,
+                        const void* B, float scale, void* Y, void* stream);
+int lora_linear_bwd_nf4(lora_plan_t* plan, const void* dY, const void* X, const void* W_codes, const void* W_absmax,
+                        const void* A, const void* B, float scale, void* dX, void* dA, void* dB, void* stream);
+
 /* One training step of the layer with HOST input/output buffers: copies h_X, h_A, h_B, h_dY to the
  * device staging area, runs forward and backward, copies Y, dX, dA, dB back, all on `stream`
  * (asynchronous when the host buffers are pinned).  W is the frozen weight and stays resident on

@@ -27,7 +27,7 @@ EXPORTS = [
     "lora_select_config", "lora_workspace_bytes", "lora_plan_create", "lora_plan_destroy",
     "lora_plan_workspace_bytes", "lora_plan_set_workspace", "lora_plan_get_config", "lora_plan_describe",
     "lora_linear_fwd", "lora_linear_bwd", "lora_linear_bwd_saved_p", "lora_linear_bwd_dx", "lora_linear_bwd_da", "lora_linear_bwd_db",
-    "lora_dense_dw", "lora_step_host_staging_bytes", "lora_linear_step_host",
+    "lora_dense_dw", "lora_nf4_quantize", "lora_linear_fwd_nf4", "lora_linear_bwd_nf4", "lora_step_host_staging_bytes", "lora_linear_step_host",
     "lora_last_device_status", "lora_strerror", "lora_launch_count",
     "lora_grad_contract_noalloc", "lora_grad_contract_noalloc_max_scratch",
 ]
@@ -80,6 +80,9 @@ def load(rebuild: bool = False) -> ctypes.CDLL:
     lib.lora_linear_bwd_da.argtypes = [vp, vp, vp, ctypes.c_float, vp, vp]
     lib.lora_linear_bwd_db.argtypes = [vp, vp, ctypes.c_float, vp, vp]
     lib.lora_dense_dw.argtypes = [vp, vp, vp, vp, vp]
+    lib.lora_nf4_quantize.argtypes = [vp, i64, i64, vp, vp, vp]
+    lib.lora_linear_fwd_nf4.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp]
+    lib.lora_linear_bwd_nf4.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
     lib.lora_step_host_staging_bytes.argtypes = [ctypes.POINTER(LoraShape), sz_p]
     lib.lora_linear_step_host.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp,
                                           ctypes.c_size_t, vp]
@@ -246,6 +249,47 @@ class LoraLinearPlan:
                   _ptr(dX), _ptr(dA), _ptr(dB), _stream_ptr(stream)), "lora_linear_bwd")
         return dX, dA, dB
 
+    # -- NF4 frozen weight (Q+LoRA) ---------------------------------------------------------------
+    def fwd_nf4(self, X, W_codes, W_absmax, A, B, scale: float, Y: Optional[torch.Tensor] = None, stream=None):
+        """Y = X w_hat^T + scale (X A^T) B^T with w_hat = the NF4 weight (codes [d_out, d_in/2] uint8, absmax [d_in/64, d_out] fp32)."""
+        bf = torch.bfloat16
+        _want(X, "X", (self.T, self.d_in), bf, self.device)
+        _want(W_codes, "W_codes", (self.d_out, self.d_in // 2), torch.uint8, self.device)
+        _want(W_absmax, "W_absmax", (self.d_in // 64, self.d_out), torch.float32, self.device)
+        _want(A, "A", (self.r, self.d_in), bf, self.device)
+        _want(B, "B", (self.d_out, self.r), bf, self.device)
+        if Y is None:
+            Y = torch.empty((self.T, self.d_out), dtype=bf, device=self.device)
+        _want(Y, "Y", (self.T, self.d_out), bf, self.device)
+        self.ensure_workspace()
+        _check(self._lib.lora_linear_fwd_nf4(self._h, _ptr(X), _ptr(W_codes), _ptr(W_absmax), _ptr(A), _ptr(B), float(scale),
+                                             _ptr(Y), _stream_ptr(stream)), "lora_linear_fwd_nf4")
+        return Y
+
+    def bwd_nf4(self, dY, X, W_codes, W_absmax, A, B, scale: float, dX=None, dA=None, dB=None, stream=None):
+        """(dX, dA, dB) of the layer with the NF4 weight."""
+        bf = torch.bfloat16
+        _want(dY, "dY", (self.T, self.d_out), bf, self.device)
+        _want(X, "X", (self.T, self.d_in), bf, self.device)
+        _want(W_codes, "W_codes", (self.d_out, self.d_in // 2), torch.uint8, self.device)
+        _want(W_absmax, "W_absmax", (self.d_in // 64, self.d_out), torch.float32, self.device)
+        _want(A, "A", (self.r, self.d_in), bf, self.device)
+        _want(B, "B", (self.d_out, self.r), bf, self.device)
+        if dX is None:
+            dX = torch.empty((self.T, self.d_in), dtype=bf, device=self.device)
+        if dA is None:
+            dA = torch.empty((self.r, self.d_in), dtype=torch.float32, device=self.device)
+        if dB is None:
+            dB = torch.empty((self.d_out, self.r), dtype=torch.float32, device=self.device)
+        _want(dX, "dX", (self.T, self.d_in), bf, self.device)
+        _want(dA, "dA", (self.r, self.d_in), torch.float32, self.device)
+        _want(dB, "dB", (self.d_out, self.r), torch.float32, self.device)
+        self.ensure_workspace()
+        _check(self._lib.lora_linear_bwd_nf4(self._h, _ptr(dY), _ptr(X), _ptr(W_codes), _ptr(W_absmax), _ptr(A), _ptr(B),
+                                             float(scale), _ptr(dX), _ptr(dA), _ptr(dB), _stream_ptr(stream)),
+               "lora_linear_bwd_nf4")
+        return dX, dA, dB
+
     def dense_dw(self, dY, X, dW: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
         """dW = dY^T X, the weight gradient of full fine-tuning ([d_out, d_in] bf16)."""
         bf = torch.bfloat16
@@ -323,3 +367,14 @@ def grad_contract_noalloc(S: torch.Tensor, Rt: torch.Tensor, out: torch.Tensor, 
     _check(load().lora_grad_contract_noalloc(_ptr(S), _ptr(Rt), T, C, r, ld, _ptr(out), _stream_ptr(stream)),
            "lora_grad_contract_noalloc")
     return out
+
+
+def nf4_quantize(W: torch.Tensor, stream=None):
+    """(codes [d_out, d_in/2] uint8, absmax [d_in/64, d_out] fp32) of a bf16 device weight, in this library's NF4 layout."""
+    if W.dtype != torch.bfloat16 or not W.is_contiguous() or W.dim() != 2 or not W.is_cuda:
+        raise ValueError("nf4_quantize: contiguous bf16 CUDA matrix expected")
+    d_out, d_in = W.shape
+    codes = torch.empty((d_out, d_in // 2), dtype=torch.uint8, device=W.device)
+    absmax = torch.empty((d_in // 64, d_out), dtype=torch.float32, device=W.device)
+    _check(load().lora_nf4_quantize(_ptr(W), d_out, d_in, _ptr(codes), _ptr(absmax), _stream_ptr(stream)), "lora_nf4_quantize")
+    return codes, absmax

@@ -9,7 +9,7 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "liblora_linear.so")
-SOURCES = ["api.cu", "gemm_lora.cu", "gemm_lora_pair.cu", "adapter_grad.cu"]
+SOURCES = ["api.cu", "gemm_lora.cu", "gemm_lora_pair.cu", "adapter_grad.cu", "nf4_quant.cu"]
 HEADERS = ["kernels.h", "sm100_ptx.cuh", os.path.join("..", "..", "include", "lora_linear.h")]
 
 

@@ -622,6 +622,108 @@ int launch_db(lora_plan* pl, const void* dY, float scale, void* dB, cudaStream_t
   return LORA_OK;
 }
 
+// ---- NF4 frozen weight (Q+LoRA): both GEMMs run K-extended on CTA pairs with the dequantising kernel variant ----
+bool make_nf4_tmaps(CUtensorMap* tmCodes, CUtensorMap* tmAbsmax, const void* codes, const void* absmax, const lora_shape_t& s,
+                    bool backward) {
+  // codes [d_out, d_in / 2] uint8 (no swizzle): forward box = 32 bytes (one block) x 128 rows, backward 64 bytes x 64 rows;
+  // absmax [d_in / 64, d_out] float: forward box = 128 rows' scales of one block, backward 64 rows' scales of two blocks
+  bool ok = make_tmap(tmCodes, codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, s.d_in / 2, s.d_out, s.d_in / 2, backward ? 64 : 32,
+                      backward ? 64 : 128, false);
+  ok = ok && make_tmap(tmAbsmax, absmax, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, s.d_out, s.d_in / kNf4Block, s.d_out * 4,
+                       backward ? 64 : 128, backward ? 2 : 1, false);
+  return ok;
+}
+
+int launch_fwd_nf4(lora_plan* pl, const void* X, const void* codes, const void* absmax, const void* A, const void* B,
+                   float scale, void* Y, cudaStream_t st) {
+  const lora_shape_t& s = pl->shape;
+  const lora_kernel_config_t& c = pl->cfg;
+  __nv_bfloat16* pt = ws_ptrs(pl).pt;
+  int rc = launch_side_prepass(pl, X, s.d_in, A, false, scale, pt, st);   // Pt = s (X A^T)^T
+  if (rc != LORA_OK) return rc;
+  const int pairs = pl->num_sms / 2;
+  const int bn = pick_pair_block_n(s.T, s.d_out, 0, pairs);
+  CUtensorMap tmX, tmCodes, tmAbsmax, tmPt, tmB, tmY;
+  bool ok = make_bf16_tmap(&tmX, X, s.d_in, s.T, s.d_in, 64, kBlockM);
+  ok = ok && make_nf4_tmaps(&tmCodes, &tmAbsmax, codes, absmax, s, false);
+  ok = ok && make_bf16_tmap(&tmPt, pt, s.T, c.r_pad, pl->ws.ld_t, 64, c.r_pad);
+  ok = ok && make_bf16_tmap(&tmB, B, s.r, s.d_out, s.r, 64, bn / 2);
+  ok = ok && make_bf16_tmap(&tmY, Y, s.d_out, s.T, s.d_out, 64, kBlockM);
+  if (!ok) return LORA_ERR_CUDA;
+  GemmParams p{};
+  p.out = static_cast<__nv_bfloat16*>(Y);
+  p.ld_out = static_cast<int>(s.d_out);
+  p.M = static_cast<int>(s.T);
+  p.N = static_cast<int>(s.d_out);
+  p.K = static_cast<int>(s.d_in);
+  p.r_pad = c.r_pad;
+  p.block_n = bn;
+  p.tiles_m = ceil_div(s.T, kPairBlockM);
+  p.tiles_n = ceil_div(s.d_out, bn);
+  p.num_tiles = p.tiles_m * p.tiles_n;
+  p.kblocks = ceil_div(s.d_in, kBlockK);
+  p.group_m = c.group_m;
+  p.stages = 5;                       // one stage less than the bf16 kernels: the code ring and the level table need the room
+  p.tail_delay = c.tail_delay;
+  p.scale = scale;
+  p.kb_per_split = p.kblocks;
+  p.split_k = 1;
+  p.status = pl->d_status;
+  const int ctas = 2 * (p.num_tiles < pairs ? p.num_tiles : pairs);
+  if (launch_gemm_pair_fwd_nf4(tmX, tmCodes, tmAbsmax, tmPt, tmB, tmY, p, ctas, st) != cudaSuccess) return LORA_ERR_CUDA;
+  g_launches.fetch_add(1);
+  pl->p_saved = false;
+  return LORA_OK;
+}
+
+int launch_dx_nf4(lora_plan* pl, const void* dY, const void* codes, const void* absmax, const void* A, const void* B,
+                  float scale, void* dX, cudaStream_t st) {
+  const lora_shape_t& s = pl->shape;
+  const lora_kernel_config_t& c = pl->cfg;
+  __nv_bfloat16* qt = ws_ptrs(pl).qt;
+  int rc = launch_side_prepass(pl, dY, s.d_out, B, true, scale, qt, st);   // Qt = s (dY B)^T
+  if (rc != LORA_OK) return rc;
+  const int pairs = pl->num_sms / 2;
+  const int bn = 256;                 // each CTA's 128 weight columns are two whole quantisation blocks
+  CUtensorMap tmdY, tmCodes, tmAbsmax, tmQt, tmA, tmdX;
+  bool ok = make_bf16_tmap(&tmdY, dY, s.d_out, s.T, s.d_out, 64, kBlockM);
+  ok = ok && make_nf4_tmaps(&tmCodes, &tmAbsmax, codes, absmax, s, true);
+  ok = ok && make_bf16_tmap(&tmQt, qt, s.T, c.r_pad, pl->ws.ld_t, 64, c.r_pad);
+  ok = ok && make_bf16_tmap(&tmA, A, s.d_in, s.r, s.d_in, 64, c.r_pad);
+  ok = ok && make_bf16_tmap(&tmdX, dX, s.d_in, s.T, s.d_in, 64, kBlockM);
+  if (!ok) return LORA_ERR_CUDA;
+  GemmParams p{};
+  p.out = static_cast<__nv_bfloat16*>(dX);
+  p.ld_out = static_cast<int>(s.d_in);
+  p.M = static_cast<int>(s.T);
+  p.N = static_cast<int>(s.d_in);
+  p.K = static_cast<int>(s.d_out);
+  p.r_pad = c.r_pad;
+  p.block_n = bn;
+  p.tiles_m = ceil_div(s.T, kPairBlockM);
+  p.tiles_n = ceil_div(s.d_in, bn);
+  p.num_tiles = p.tiles_m * p.tiles_n;
+  p.kblocks = ceil_div(s.d_out, kBlockK);
+  p.group_m = c.group_m;
+  p.stages = 5;
+  p.tail_delay = c.tail_delay;
+  p.scale = scale;
+  p.kb_per_split = p.kblocks;
+  p.split_k = 1;
+  p.status = pl->d_status;
+  const int ctas = 2 * (p.num_tiles < pairs ? p.num_tiles : pairs);
+  if (launch_gemm_pair_dx_nf4(tmdY, tmCodes, tmAbsmax, tmQt, tmA, tmdX, p, ctas, st) != cudaSuccess) return LORA_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return LORA_OK;
+}
+
+int check_nf4(const lora_plan* pl) {
+  if (pl->cfg.cta_group != 2) return LORA_ERR_UNSUPPORTED_SHAPE;          // batches of at most 128 tokens: not covered
+  if (pl->shape.d_in % kNf4Block != 0) return LORA_ERR_UNSUPPORTED_SHAPE;
+  if (pl->workspace == nullptr || pl->workspace_bytes < pl->ws.total) return LORA_ERR_WORKSPACE;
+  return LORA_OK;
+}
+
 // ---- dW = dY^T X (full fine-tuning): plain GEMM with both operands MN-major, contraction over the tokens ----
 int launch_dw(lora_plan* pl, const void* dY, const void* X, void* dW, cudaStream_t st) {
   const lora_shape_t& s = pl->shape;
@@ -865,6 +967,56 @@ int lora_linear_bwd_db(lora_plan_t* plan, const void* dY, float scale, void* dB,
   if (!aligned16(dY)) return LORA_ERR_MISALIGNED;
   if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
   return launch_db(plan, dY, scale, dB, static_cast<cudaStream_t>(stream));
+}
+
+int lora_nf4_quantize(const void* W, int64_t d_out, int64_t d_in, void* codes, void* absmax, void* stream) {
+  if (!W || !codes || !absmax) return LORA_ERR_INVALID_ARG;
+  if (d_out <= 0 || d_in <= 0) return LORA_ERR_INVALID_ARG;
+  if (d_in % kNf4Block != 0 || d_out % 4 != 0 || d_out > (1ll << 24) || d_in > (1ll << 24)) return LORA_ERR_UNSUPPORTED_SHAPE;
+  if (!aligned16(W) || !aligned16(codes) || !aligned16(absmax)) return LORA_ERR_MISALIGNED;
+  if (launch_nf4_quantize(static_cast<const __nv_bfloat16*>(W), d_out, d_in, static_cast<uint8_t*>(codes),
+                          static_cast<float*>(absmax), static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return LORA_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return LORA_OK;
+}
+
+int lora_linear_fwd_nf4(lora_plan_t* plan, const void* X, const void* W_codes, const void* W_absmax, const void* A,
+                        const void* B, float scale, void* Y, void* stream) {
+  if (plan == nullptr) return LORA_ERR_INVALID_ARG;
+  if (plan->shape.T == 0) return LORA_OK;
+  if (!X || !W_codes || !W_absmax || !A || !B || !Y) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(W_codes) || !aligned16(W_absmax) || !aligned16(A) || !aligned16(B) || !aligned16(Y))
+    return LORA_ERR_MISALIGNED;
+  const int rc = check_nf4(plan);
+  if (rc != LORA_OK) return rc;
+  DeviceGuard guard(plan->device);
+  return launch_fwd_nf4(plan, X, W_codes, W_absmax, A, B, scale, Y, static_cast<cudaStream_t>(stream));
+}
+
+int lora_linear_bwd_nf4(lora_plan_t* plan, const void* dY, const void* X, const void* W_codes, const void* W_absmax,
+                        const void* A, const void* B, float scale, void* dX, void* dA, void* dB, void* stream) {
+  if (plan == nullptr) return LORA_ERR_INVALID_ARG;
+  if (!dA || !dB) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(dA) || !aligned16(dB)) return LORA_ERR_MISALIGNED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  DeviceGuard guard(plan->device);
+  if (plan->shape.T == 0) {
+    if (cudaMemsetAsync(dA, 0, sizeof(float) * plan->shape.r * plan->shape.d_in, st) != cudaSuccess ||
+        cudaMemsetAsync(dB, 0, sizeof(float) * plan->shape.d_out * plan->shape.r, st) != cudaSuccess)
+      return LORA_ERR_CUDA;
+    return LORA_OK;
+  }
+  if (!dY || !X || !W_codes || !W_absmax || !A || !B || !dX) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(dY) || !aligned16(X) || !aligned16(W_codes) || !aligned16(W_absmax) || !aligned16(A) || !aligned16(B) ||
+      !aligned16(dX))
+    return LORA_ERR_MISALIGNED;
+  int rc = check_nf4(plan);
+  if (rc != LORA_OK) return rc;
+  rc = launch_dx_nf4(plan, dY, W_codes, W_absmax, A, B, scale, dX, st);
+  if (rc == LORA_OK) rc = launch_da(plan, X, A, scale, dA, st);
+  if (rc == LORA_OK) rc = launch_db(plan, dY, scale, dB, st);
+  return rc;
 }
 
 int lora_dense_dw(lora_plan_t* plan, const void* dY, const void* X, void* dW, void* stream) {

@@ -34,6 +34,16 @@ namespace lora {
 
 namespace {
 
+// The 16 NF4 levels (QLoRA, Appendix E: normal quantiles scaled to [-1, 1] with an exact zero), float32.
+__device__ __constant__ float c_nf4_levels[16] = {
+    -1.0f, -0.6961928009986877f, -0.5250730514526367f, -0.39491748809814453f,
+    -0.28444138169288635f, -0.18477343022823334f, -0.09105003625154495f, 0.0f,
+    0.07958029955625534f, 0.16093020141124725f, 0.24611230194568634f, 0.33791524171829224f,
+    0.44070982933044434f, 0.5626170039176941f, 0.7229568362236023f, 1.0f};
+
+constexpr int kPairBarriers = kGemmBarriers + 2 * kNf4CodeSlots;   // + code ring full / empty (NF4 weight only)
+constexpr int kPairBarrierBytes = 512;                             // barriers, TMEM slot, abort flag
+
 struct PairTile {
   int m_idx, n_idx;
 };
@@ -55,8 +65,12 @@ __device__ __forceinline__ PairTile pair_tile(int id, const GemmParams& p) {
 //       With r_pad = 0 the K-extended form has no rank-r k-block at all: a plain GEMM.
 // kAmn: the activation-side operand is MN-major too: its tensor is [K, M] row-major (box 64(m) x 64(k), two per stage).
 //       This is the dense weight gradient dW = dY^T X, where both operands are contracted over their row index.
-template <bool kBmn, bool kExt, bool kAmn = false>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
+// kNf4: the frozen weight is held in 4-bit NormalFloat (Section 4.5, Q+LoRA).  Its packed codes and block scales are
+//       staged by TMA into a small ring; four extra warps turn each 64-element block into bf16(level * absmax) and
+//       write it into the stage's weight tile in exactly the swizzled layout TMA would have produced, so the MMA
+//       side is unchanged.  K-extended form only (tm_w0 = codes, tm_w1 = absmax).
+template <bool kBmn, bool kExt, bool kAmn = false, bool kNf4 = false>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNf4 ? kPairThreadsNf4 : kPairThreads, 1)
 lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M, K], box 64(k) x 128 ; kAmn: [K, M], box 64(m) x 64(k)
                       const __grid_constant__ CUtensorMap tm_w0,    // fwd: W box 64(k) x half ; bwd: W box 64(n) x 64(k)
                       const __grid_constant__ CUtensorMap tm_w1,    // fwd: W box 64(k) x (block_n - half) ; bwd unused
@@ -79,8 +93,13 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
   auto ps_ready = [&](int b) { return bar0 + 8u * (2 * kMaxStages + 2 + b); };
   auto acc_full = [&](int b) { return bar0 + 8u * (2 * kMaxStages + 4 + b); };
   auto acc_empty = [&](int b) { return bar0 + 8u * (2 * kMaxStages + 6 + b); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kGemmBarriers);
+  auto cfull_bar = [&](int c) { return bar0 + 8u * (kGemmBarriers + c); };
+  auto cempty_bar = [&](int c) { return bar0 + 8u * (kGemmBarriers + kNf4CodeSlots + c); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kPairBarriers);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  // NF4 only: ring of packed codes + block scales, and the byte -> (level of low nibble, level of high nibble) table
+  uint8_t* code_ring = staging_ptr + 2 * kStagingBytes + kPairBarrierBytes;
+  float2* nf4_lut = reinterpret_cast<float2*>(code_ring + kNf4CodeSlots * kNf4CodeSlotBytes);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -88,8 +107,14 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
-      mbar_init(full_bar(s), 2);
+      mbar_init(full_bar(s), kNf4 ? 1 + 2 * kNf4DequantThreads : 2);   // NF4: every dequantising thread of the pair arrives
       mbar_init(empty_bar(s), 1);
+    }
+    if (kNf4) {
+      for (int c = 0; c < kNf4CodeSlots; ++c) {
+        mbar_init(cfull_bar(c), 1);
+        mbar_init(cempty_bar(c), kNf4DequantThreads);
+      }
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(side_full(b), 1);
@@ -109,6 +134,10 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
   if (warp == 4) {
     tmem_alloc_pair(smem_u32(tmem_slot), 512);
     tmem_relinquish_pair();
+  }
+  if (kNf4 && threadIdx.x >= kPairThreads) {
+    for (int b = threadIdx.x - kPairThreads; b < 256; b += kNf4DequantThreads)
+      nf4_lut[b] = make_float2(c_nf4_levels[b & 15], c_nf4_levels[b >> 4]);
   }
   tc_fence_before();
   __syncthreads();
@@ -192,9 +221,19 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
             if (rank == 0) mbar_arrive(full_bar(cur));        // fused: the rank-r operand comes from the epilogue
           } else {
             // K-extended: s (X A^T)^T or s (dY B)^T for this CTA's 128 tokens, two 64-token groups of r_pad rows (MN-major A operand)
-            if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), 2 * 2 * p.r_pad * 128);
+            // (NF4: this warp also brings the weight-side operand of the rank-r k-block; the other producer warps
+            // only feed the code ring)
+            const uint32_t side_bytes = 2 * 2 * p.r_pad * 128;
+            const uint32_t tail_bytes = kNf4 ? (kBmn ? 2 * 2 * p.r_pad * 128 : BN * 128) : 0;
+            if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), side_bytes + tail_bytes);
             tma_load_2d_pair(a_dst, &tm_side, fb, m0, 0);
             tma_load_2d_pair(a_dst + p.r_pad * 128, &tm_side, fb, m0 + 64, 0);
+            if (kNf4 && !kBmn) {
+              tma_load_2d_pair(b_dst, &tm_tail, fb, 0, nb);
+            } else if (kNf4) {
+              tma_load_2d_pair(b_dst, &tm_tail, fb, nb, 0);
+              tma_load_2d_pair(b_dst + 8192, &tm_tail, fb, nb + 64, 0);
+            }
           }
         } else if (!kBmn) {
           if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), BN * 128);
@@ -207,10 +246,39 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       }
       __syncwarp();
     };
+    if (kNf4 && op == 1) {
+      // ---- NF4: these two warps feed the code ring (packed codes + block scales of every main k-block) ----
+      int cslot = 0, cphase = 0, codd = 0;
+      for (int i = 0; i < n_my && ok; ++i) {
+        const int item = pair + i * G, sp = item % SK;
+        const PairTile tc = pair_tile(item / SK, p);
+        const int nb = tc.n_idx * BN + static_cast<int>(rank) * (BN >> 1);
+        const int kb0 = sp * p.kb_per_split, kb1 = min(KB, kb0 + p.kb_per_split);
+        for (int kb = kb0; kb < kb1 && ok; ++kb) {
+          if (codd == par) {
+            ok = warp_wait(cempty_bar(cslot), cphase ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY, false, 20);
+            if (ok && elect_one()) {
+              const uint32_t cdst = smem_u32(code_ring) + cslot * kNf4CodeSlotBytes, cb = cfull_bar(cslot);
+              mbar_arrive_expect_tx(cb, kNf4CodeSlotBytes);
+              if (!kBmn) {   // forward: rows nb.. of W, the 32 code bytes and the one scale of k-block kb
+                tma_load_2d(cdst, &tm_w0, cb, kb * 32, nb);
+                tma_load_2d(cdst + 4096, &tm_w1, cb, nb, kb);
+              } else {       // backward: rows kb*64.. of W (the contraction index), 128 columns = 64 code bytes, 2 blocks
+                tma_load_2d(cdst, &tm_w0, cb, nb >> 1, kb * kBlockK);
+                tma_load_2d(cdst + 4096, &tm_w1, cb, kb * kBlockK, nb >> 6);
+              }
+            }
+            __syncwarp();
+          }
+          if (++cslot == kNf4CodeSlots) { cslot = 0; cphase ^= 1; }
+          codd ^= 1;
+        }
+      }
+    }
     // Item order.  Fused: the rank-r item of tile i-1 comes D k-blocks into tile i (its operand is made by the
     // epilogue meanwhile).  K-extended: the rank-r item is simply the last k-block of its own tile.
     int prev_n0 = 0;
-    for (int i = 0; i < n_my && ok; ++i) {
+    for (int i = 0; i < n_my && ok && !(kNf4 && op == 1); ++i) {
       const int item = pair + i * G, sp = item % SK;
       const PairTile tc = pair_tile(item / SK, p);
       const int m0 = tc.m_idx * kPairBlockM + static_cast<int>(rank) * 128, n0 = tc.n_idx * BN;
@@ -223,7 +291,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       if (kExt && ok && sp == SK - 1 && p.r_pad > 0) load_tail(m0, n0);
       prev_n0 = n0;
     }
-    if (!kExt && ok && n_my > 0) load_tail(0, prev_n0);
+    if (!kExt && ok && n_my > 0 && !(kNf4 && op == 1)) load_tail(0, prev_n0);
   } else if (warp == 4) {
     // ================================ MMA issuer (leader CTA only) ================================
     // Whole warp of the leader CTA runs the loop; one lane polls, one elected lane issues every MMA and commit.
@@ -291,6 +359,57 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
         if (kExt && ok && has_tail) mma_tail(buf, use);
       }
       if (!kExt && ok && n_my > 0) mma_tail((n_my - 1) & 1, (n_my - 1) >> 1);
+    }
+  } else if (kNf4 && warp >= 9) {
+    // ================================ NF4 dequantisation (warps 9..12, 128 threads per CTA) ================================
+    // Thread d owns one 64-element block of every main k-block: 32 code bytes and one scale in, 128 bytes of bf16 out.
+    //   forward  (weight rows K-major):  row d of this CTA's weight rows, the k-block's 64 input features
+    //   backward (weight MN-major):      contraction row d % 64 of the k-block, column group d / 64 (64 input features)
+    // Every element is bf16(level * absmax): one float32 product, one round-to-nearest-even.
+    const int d = threadIdx.x - kPairThreads;
+    const int row = kBmn ? (d & 63) : d;
+    const int grp = kBmn ? (d >> 6) : 0;
+    const bool has_row = kBmn || d < (BN >> 1);
+    const uint32_t code_off = kBmn ? static_cast<uint32_t>(row * 64 + grp * 32) : static_cast<uint32_t>(row * 32);
+    const uint32_t scale_off = 4096u + 4u * static_cast<uint32_t>(kBmn ? grp * 64 + row : row);
+    int slot = 0, phase = 0, cslot = 0, cphase = 0;
+    bool ok = true;
+    for (int i = 0; i < n_my && ok; ++i) {
+      const int sp = (pair + i * G) % SK;
+      const int kb0 = sp * p.kb_per_split, kb1 = min(KB, kb0 + p.kb_per_split);
+      const bool has_tail = sp == SK - 1 && p.r_pad > 0;
+      for (int kb = kb0; kb < kb1 + (has_tail ? 1 : 0) && ok; ++kb) {
+        const bool main_item = kb < kb1;
+        if (main_item) ok = warp_wait(cfull_bar(cslot), cphase, abort_flag, p.status, DEV_TIMEOUT_FULL, false, 0);
+        if (ok) ok = warp_wait(empty_bar(slot), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY, false, 0);
+        if (!ok) break;
+        if (main_item) {
+          (void)mbar_try_wait(cfull_bar(cslot), cphase);     // every reading thread observes the completed copy itself
+          const uint8_t* src = code_ring + cslot * kNf4CodeSlotBytes;
+          if (has_row) {
+            const uint4 c0 = *reinterpret_cast<const uint4*>(src + code_off);
+            const uint4 c1 = *reinterpret_cast<const uint4*>(src + code_off + 16);
+            const float scale = *reinterpret_cast<const float*>(src + scale_off);
+            uint8_t* dst = smem + slot * kStage + 16384 + grp * 8192;
+            const uint32_t cw[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {     // 4 code bytes -> 8 elements -> one 16-byte chunk of the swizzled row
+              uint32_t w[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float2 lv = nf4_lut[(cw[q] >> (8 * j)) & 0xFFu];
+                w[j] = pack_bf16x2(lv.x * scale, lv.y * scale);
+              }
+              *reinterpret_cast<uint4*>(dst + sw128_offset(row, q)) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+          fence_proxy_async_smem();           // the tensor core reads the tile through the async proxy
+          mbar_arrive(cempty_bar(cslot));
+          if (++cslot == kNf4CodeSlots) { cslot = 0; cphase ^= 1; }
+        }
+        mbar_arrive_cluster(map_to_cta(full_bar(slot), 0));
+        if (++slot == S) { slot = 0; phase ^= 1; }
+      }
     }
   } else {
     // ================================ epilogue (128 threads per CTA) ================================
@@ -479,8 +598,9 @@ cudaError_t launch_splitk_reduce(const float* part, __nv_bfloat16* out, long lon
                     out, n_elems, splits);
 }
 
-size_t gemm_pair_smem_bytes(int stages) {
-  return static_cast<size_t>(stages) * kPairStageBytesFwd + 2 * kStagingBytes + kGemmBarriers * 8 + 16 + 1024;
+size_t gemm_pair_smem_bytes(int stages, bool nf4) {
+  return static_cast<size_t>(stages) * kPairStageBytesFwd + 2 * kStagingBytes + kPairBarrierBytes + 1024 +
+         (nf4 ? kNf4CodeSlots * kNf4CodeSlotBytes + 256 * sizeof(float2) : 0);
 }
 
 cudaError_t gemm_pair_configure() {
@@ -491,33 +611,51 @@ cudaError_t gemm_pair_configure() {
     e = cudaFuncSetAttribute(lora_gemm_pair_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(lora_gemm_pair_kernel<true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(lora_gemm_pair_kernel<false, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(lora_gemm_pair_kernel<true, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
   return e;
 }
 
 cudaError_t launch_gemm_pair_fwd(const CUtensorMap& tmX, const CUtensorMap& tmW0, const CUtensorMap& tmW1,
                                  const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
                                  const GemmParams& p, int ctas, cudaStream_t stream) {
-  return launch_pdl(lora_gemm_pair_kernel<false, false>, dim3(ctas), dim3(kPairThreads), gemm_pair_smem_bytes(p.stages), stream,
+  return launch_pdl(lora_gemm_pair_kernel<false, false>, dim3(ctas), dim3(kPairThreads), gemm_pair_smem_bytes(p.stages, false), stream,
                     tmX, tmW0, tmW1, tmA, tmB, tmY, p);
 }
 
 cudaError_t launch_gemm_pair_fwd_ext(const CUtensorMap& tmX, const CUtensorMap& tmW, const CUtensorMap& tmPt,
                                      const CUtensorMap& tmB, const CUtensorMap& tmY, const GemmParams& p, int ctas,
                                      cudaStream_t stream) {
-  return launch_pdl(lora_gemm_pair_kernel<false, true>, dim3(ctas), dim3(kPairThreads), gemm_pair_smem_bytes(p.stages), stream,
+  return launch_pdl(lora_gemm_pair_kernel<false, true>, dim3(ctas), dim3(kPairThreads), gemm_pair_smem_bytes(p.stages, false), stream,
                     tmX, tmW, tmW, tmPt, tmB, tmY, p);
 }
 
 cudaError_t launch_gemm_pair_dx(const CUtensorMap& tmdY, const CUtensorMap& tmW, const CUtensorMap& tmQt,
                                 const CUtensorMap& tmA, const CUtensorMap& tmdX, const GemmParams& p, int ctas,
                                 cudaStream_t stream) {
-  return launch_pdl(lora_gemm_pair_kernel<true, true>, dim3(ctas), dim3(kPairThreads), gemm_pair_smem_bytes(p.stages), stream,
+  return launch_pdl(lora_gemm_pair_kernel<true, true>, dim3(ctas), dim3(kPairThreads), gemm_pair_smem_bytes(p.stages, false), stream,
                     tmdY, tmW, tmW, tmQt, tmA, tmdX, p);
+}
+
+cudaError_t launch_gemm_pair_fwd_nf4(const CUtensorMap& tmX, const CUtensorMap& tmCodes, const CUtensorMap& tmAbsmax,
+                                     const CUtensorMap& tmPt, const CUtensorMap& tmB, const CUtensorMap& tmY,
+                                     const GemmParams& p, int ctas, cudaStream_t stream) {
+  return launch_pdl(lora_gemm_pair_kernel<false, true, false, true>, dim3(ctas), dim3(kPairThreadsNf4),
+                    gemm_pair_smem_bytes(p.stages, true), stream, tmX, tmCodes, tmAbsmax, tmPt, tmB, tmY, p);
+}
+
+cudaError_t launch_gemm_pair_dx_nf4(const CUtensorMap& tmdY, const CUtensorMap& tmCodes, const CUtensorMap& tmAbsmax,
+                                    const CUtensorMap& tmQt, const CUtensorMap& tmA, const CUtensorMap& tmdX,
+                                    const GemmParams& p, int ctas, cudaStream_t stream) {
+  return launch_pdl(lora_gemm_pair_kernel<true, true, false, true>, dim3(ctas), dim3(kPairThreadsNf4),
+                    gemm_pair_smem_bytes(p.stages, true), stream, tmdY, tmCodes, tmAbsmax, tmQt, tmA, tmdX, p);
 }
 
 cudaError_t launch_gemm_pair_dw(const CUtensorMap& tmdYt, const CUtensorMap& tmX, const CUtensorMap& tmdW, const GemmParams& p,
                                 int ctas, cudaStream_t stream) {
-  return launch_pdl(lora_gemm_pair_kernel<true, true, true>, dim3(ctas), dim3(kPairThreads), gemm_pair_smem_bytes(p.stages),
+  return launch_pdl(lora_gemm_pair_kernel<true, true, true>, dim3(ctas), dim3(kPairThreads), gemm_pair_smem_bytes(p.stages, false),
                     stream, tmdYt, tmX, tmX, tmX, tmX, tmdW, p);
 }
 

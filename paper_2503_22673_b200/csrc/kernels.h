@@ -64,7 +64,14 @@ size_t gemm_smem_bytes(int stages);
 constexpr int kPairBlockM = 256;
 constexpr int kPairThreads = 288;           // warps 0..3 TMA producers, warp 4 MMA + TMEM, warps 5..8 epilogue
 constexpr int kPairStageBytesFwd = 32768;   // 128 x 64 activations + 128 x 64 weight/adapter rows per CTA
-size_t gemm_pair_smem_bytes(int stages);
+// NF4 weight (K-extended forms only): four more warps dequantise; packed codes + block scales travel through a ring of
+// kNf4CodeSlots slots of 4096 code bytes + 128 float scales
+constexpr int kNf4DequantThreads = 128;
+constexpr int kPairThreadsNf4 = kPairThreads + kNf4DequantThreads;
+constexpr int kNf4CodeSlots = 4;
+constexpr int kNf4CodeSlotBytes = 4096 + 512;
+constexpr int kNf4Block = 64;               // elements per quantisation block (= kBlockK)
+size_t gemm_pair_smem_bytes(int stages, bool nf4 = false);
 cudaError_t gemm_pair_configure();
 // out = bf16(sum of the split_k fp32 partial matrices), fixed order (M x N must be a multiple of 8 elements)
 cudaError_t launch_splitk_reduce(const float* part, __nv_bfloat16* out, long long n_elems, int splits, cudaStream_t stream);
@@ -81,6 +88,19 @@ cudaError_t launch_gemm_pair_fwd_ext(const CUtensorMap& tmX, const CUtensorMap& 
 // backward: tmW box 64(n) x 64(k); tmQt = s (dY B)^T [r_pad, T] box 64(t) x r_pad; tmA box 64(n) x r_pad
 cudaError_t launch_gemm_pair_dx(const CUtensorMap& tmdY, const CUtensorMap& tmW, const CUtensorMap& tmQt,
                                 const CUtensorMap& tmA, const CUtensorMap& tmdX, const GemmParams& p, int ctas,
+                                cudaStream_t stream);
+
+// NF4 frozen weight: tmCodes = packed codes [d_out, d_in/2] uint8, no swizzle, box 32 B x 128 rows (forward) or
+// 64 B x 64 rows (backward); tmAbsmax = block scales [d_in/64, d_out] float, box 128 x 1 (forward) or 64 x 2 (backward);
+// the other maps as in the K-extended bf16 launchers.  Forward block_n any multiple of 16, backward block_n = 256.
+cudaError_t launch_gemm_pair_fwd_nf4(const CUtensorMap& tmX, const CUtensorMap& tmCodes, const CUtensorMap& tmAbsmax,
+                                     const CUtensorMap& tmPt, const CUtensorMap& tmB, const CUtensorMap& tmY,
+                                     const GemmParams& p, int ctas, cudaStream_t stream);
+cudaError_t launch_gemm_pair_dx_nf4(const CUtensorMap& tmdY, const CUtensorMap& tmCodes, const CUtensorMap& tmAbsmax,
+                                    const CUtensorMap& tmQt, const CUtensorMap& tmA, const CUtensorMap& tmdX,
+                                    const GemmParams& p, int ctas, cudaStream_t stream);
+// W [d_out, d_in] bf16 -> NF4 codes [d_out, d_in/2] + block scales [d_in/64, d_out] (nf4_quant.cu)
+cudaError_t launch_nf4_quantize(const __nv_bfloat16* W, long long d_out, long long d_in, uint8_t* codes, float* absmax,
                                 cudaStream_t stream);
 
 // dense weight gradient dW[d_out, d_in] = dY^T X (p.r_pad = 0: no rank-r k-block): tmdYt = dY [T, d_out] box 64(o) x 64(t),

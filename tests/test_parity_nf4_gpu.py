@@ -1,0 +1,132 @@
+"""GPU parity of the quantised-LoRA path (Section 4.5, Q+LoRA): NF4 quantiser bit-exact against the oracle's, and the
+layer with the NF4 weight against the oracle on the same codes and scales, through the C ABI.
+
+Tolerances as for the bf16 layer: max|gpu - ref| / max|ref| <= 2e-2 (Y, dX), <= 5e-3 (dA, dB).  Codes and scales are
+integer / exact float32 decisions and must match bit for bit."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import nf4_oracle as nf4
+from oracle import lora_oracle as oracle
+from paper_2503_22673_b200 import binding, inputs
+from tests.test_parity_gpu import dev, guarded, guards_intact, host64
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 2e-2
+TOL_F32 = 5e-3
+
+
+def _bf16_weight(d_out, d_in, seed):
+    p, t = inputs.draw_custom(8, d_in, d_out, 8, 1.0, seed=seed)
+    return t["W"]                                              # bf16 bit patterns, W ~ N(0, 1/d_in)
+
+
+@pytest.mark.parametrize("d_out,d_in", [(4, 64), (72, 192), (1000, 1024), (4096, 4096)])
+def test_quantiser_is_bit_exact(d_out, d_in):
+    bits = _bf16_weight(d_out, d_in, seed=d_out)
+    W = inputs.bf16_to_f64(bits).astype(np.float32)
+    W[0, :64] = 0.0                                            # an all-zero block
+    if d_in >= 128:
+        mids = nf4.midpoints()
+        W[1 % d_out, 64] = 1.0                                 # absmax 1 in that block (bf16-exact), then values on / next to midpoints
+        W[1 % d_out, 65:80] = 0.0
+    Wt = torch.tensor(W).to(torch.bfloat16)                    # exact: every value is already bf16 (or 0 / 1)
+    W = Wt.float().numpy()
+    codes, absmax = binding.nf4_quantize(Wt.cuda().contiguous())
+    torch.cuda.synchronize()
+    ref_codes, ref_absmax = nf4.quantize(W)
+    assert np.array_equal(absmax.cpu().numpy(), ref_absmax)
+    assert np.array_equal(codes.cpu().numpy(), ref_codes)
+
+
+def test_quantiser_hand_worked_block():
+    from tests.test_oracle import _read_golden
+    g = _read_golden(os.path.join(os.path.dirname(__file__), "golden", "nf4_block_example.txt"))
+    W = torch.zeros((4, 64), dtype=torch.bfloat16)
+    W[0, :8] = torch.tensor(g["w8"][0], dtype=torch.bfloat16)
+    codes, absmax = binding.nf4_quantize(W.cuda())
+    torch.cuda.synchronize()
+    assert absmax[0, 0].item() == 4.0 and torch.all(absmax[0, 1:] == 0)
+    assert codes[0, :5].cpu().tolist() == [int(v) for v in g["bytes5"][0]]
+    assert torch.all(codes[1:] == 119)
+
+
+def run_nf4_layer(p, t, codes, absmax):
+    d = {k: dev(t[k]) for k in ("X", "A", "B", "dY")}
+    cd, ad = torch.from_numpy(codes).cuda(), torch.from_numpy(absmax).cuda()
+    plan = binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r)
+    bufs, out = {}, {}
+    for name, shape, dt in (("Y", (p.T, p.d_out), torch.bfloat16), ("dX", (p.T, p.d_in), torch.bfloat16),
+                            ("dA", (p.r, p.d_in), torch.float32), ("dB", (p.d_out, p.r), torch.float32)):
+        bufs[name], out[name] = guarded(shape, dt)
+    plan.fwd_nf4(d["X"], cd, ad, d["A"], d["B"], p.scale, out["Y"])
+    plan.bwd_nf4(d["dY"], d["X"], cd, ad, d["A"], d["B"], p.scale, out["dX"], out["dA"], out["dB"])
+    code, msg = plan.device_status()
+    assert code == 0, msg
+    for name in out:
+        assert guards_intact(bufs[name], out[name].numel()), f"{name}: write outside the tensor"
+        assert not torch.isnan(out[name].float()).any(), f"{name}: element left unwritten"
+    plan.close()
+    return out
+
+
+NF4_SHAPES = [
+    # T, d_in, d_out, r, scale           (d_in a multiple of 64; T > 128: CTA-pair kernels)
+    (129, 64, 8, 8, 2.0),
+    (300, 192, 200, 16, 1.7),
+    (640, 768, 1160, 16, 2.0),
+    (1000, 2048, 520, 64, 0.5),
+    (2100, 512, 3080, 32, 2.0),           # more tiles than CTA pairs
+    (4500, 1024, 4096, 16, 2.0),
+]
+
+
+@pytest.mark.parametrize("T,d_in,d_out,r,scale", NF4_SHAPES)
+def test_nf4_layer_elementwise(T, d_in, d_out, r, scale):
+    p, t = inputs.draw_custom(T, d_in, d_out, r, scale, seed=4)
+    W32 = inputs.bf16_to_f64(t["W"]).astype(np.float32)
+    codes, absmax = nf4.quantize(W32)                          # the ORACLE's codes go to both sides
+    out = run_nf4_layer(p, t, codes, absmax)
+    f = {k: inputs.bf16_to_f64(t[k]) for k in ("X", "A", "B", "dY")}
+    Y = nf4.forward(f["X"], codes, absmax, f["A"], f["B"], p.scale)
+    dX, dA, dB = nf4.backward(f["dY"], f["X"], codes, absmax, f["A"], f["B"], p.scale)
+    errs = {"Y": oracle.rel_err(host64(out["Y"]), Y), "dX": oracle.rel_err(host64(out["dX"]), dX),
+            "dA": oracle.rel_err(host64(out["dA"]), dA), "dB": oracle.rel_err(host64(out["dB"]), dB)}
+    assert errs["Y"] <= TOL_BF16 and errs["dX"] <= TOL_BF16, errs
+    assert errs["dA"] <= TOL_F32 and errs["dB"] <= TOL_F32, errs
+
+
+def test_nf4_weight_only_is_tight():
+    """A = 0, B = 0 and one-hot X / dY rows read single rows and columns of the dequantised weight: Y and dX must then be
+    the oracle's bf16(level * absmax) values exactly (one product, one rounding, no accumulation)."""
+    T, d_in, d_out, r = 256, 256, 256, 8
+    p, t = inputs.draw_custom(T, d_in, d_out, r, 1.0, seed=6)
+    W32 = inputs.bf16_to_f64(t["W"]).astype(np.float32)
+    codes, absmax = nf4.quantize(W32)
+    what = nf4.dequantize(codes, absmax)
+    eye = torch.eye(256, dtype=torch.bfloat16)
+    t2 = dict(t)
+    bits = lambda x: x.contiguous().view(torch.int16).numpy().view(np.uint16)
+    t2["X"], t2["dY"] = bits(eye), bits(eye)
+    t2["A"] = np.zeros_like(t["A"])
+    t2["B"] = np.zeros_like(t["B"])
+    out = run_nf4_layer(p, t2, codes, absmax)
+    assert np.array_equal(host64(out["Y"]), what.T)            # Y = I w_hat^T
+    assert np.array_equal(host64(out["dX"]), what)             # dX = I w_hat
+
+
+def test_nf4_rejects_unsupported():
+    plan = binding.LoraLinearPlan(64, 128, 128, 8)             # T <= 128: single-CTA plan
+    x = torch.zeros((64, 128), dtype=torch.bfloat16, device="cuda")
+    c = torch.zeros((128, 64), dtype=torch.uint8, device="cuda")
+    a = torch.zeros((2, 128), dtype=torch.float32, device="cuda")
+    A = torch.zeros((8, 128), dtype=torch.bfloat16, device="cuda")
+    B = torch.zeros((128, 8), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.LoraError) as e:
+        plan.fwd_nf4(x, c, a, A, B, 1.0)
+    assert e.value.code == binding.LORA_ERR_UNSUPPORTED_SHAPE
+    plan.close()
