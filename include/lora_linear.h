@@ -168,17 +168,28 @@ int lora_dense_dw(lora_plan_t* plan, const void* dY, const void* X, void* dW, vo
  *     (float32 division; the lower level on an exact tie; an all-zero block gets code 7 = level 0); byte k of a row holds
  *     element 2k in its low nibble and element 2k + 1 in its high nibble;
  *   - the value the GEMMs use is  bf16( float32(level[code]) * absmax )  (one float32 product, one rounding).
- * lora_nf4_quantize builds codes and scales from a bf16 weight on the device (one warp per block).
+ * lora_nf4_quantize builds codes and scales from a bf16 weight on the device (one warp per block);
+ * lora_nf4_dequantize expands them to a bf16 matrix W [d_out, d_in] (a streaming kernel, 0.5 + 2 bytes per element).
  * lora_linear_fwd_nf4 / lora_linear_bwd_nf4 compute exactly what lora_linear_fwd / lora_linear_bwd compute with that
- * dequantised weight in place of W; dA and dB do not involve W.  The weight is never materialised in bf16: packed codes
- * and scales are staged by TMA and expanded inside the GEMM kernels, straight into the tensor-core operand tiles.
- * Both need the workspace and a plan with T > 128 (CTA-pair kernels); otherwise LORA_ERR_UNSUPPORTED_SHAPE /
- * LORA_ERR_WORKSPACE.  All pointers are device pointers, 16-byte aligned. */
+ * dequantised weight in place of W; dA and dB do not involve W.  `w_scratch` selects how:
+ *   - w_scratch != NULL (caller-owned device memory, d_out * d_in * 2 bytes, 16-byte aligned, contents undefined
+ *     afterwards; one buffer can serve every layer of that size): the weight is expanded into it once per call and the
+ *     bf16 kernels run on it.  This is the fast form for training batches: each weight element is converted once, not
+ *     once per 256-token tile, and the GEMMs keep their shared-memory bandwidth for the tensor cores.
+ *   - w_scratch == NULL: nothing is materialised; packed codes and scales are staged by TMA and expanded inside the GEMM
+ *     kernels, straight into the tensor-core operand tiles.  No extra memory, but the conversion is repeated for every
+ *     256-token tile and competes with the tensor cores for shared-memory bandwidth (measured 2-2.5x slower at
+ *     T = 4096..8192).  Needs a plan with T > 128, else LORA_ERR_UNSUPPORTED_SHAPE.
+ * Both forms give bit-identical weights to the GEMMs.  The workspace must be registered (LORA_ERR_WORKSPACE
+ * otherwise; forward needs it in the NULL form and whenever the plan's forward uses it).  All pointers are device
+ * pointers, 16-byte aligned. */
 int lora_nf4_quantize(const void* W, int64_t d_out, int64_t d_in, void* W_codes, void* W_absmax, void* stream);
+int lora_nf4_dequantize(const void* W_codes, const void* W_absmax, int64_t d_out, int64_t d_in, void* W, void* stream);
 int lora_linear_fwd_nf4(lora_plan_t* plan, const void* X, const void* W_codes, const void* W_absmax, const void* A,
-                        const void* B, float scale, void* Y, void* stream);
+                        const void* B, float scale, void* Y, void* w_scratch, void* stream);
 int lora_linear_bwd_nf4(lora_plan_t* plan, const void* dY, const void* X, const void* W_codes, const void* W_absmax,
-                        const void* A, const void* B, float scale, void* dX, void* dA, void* dB, void* stream);
+                        const void* A, const void* B, float scale, void* dX, void* dA, void* dB, void* w_scratch,
+                        void* stream);
 
 /* One training step of the layer with HOST input/output buffers: copies h_X, h_A, h_B, h_dY to the
  * device staging area, runs forward and backward, copies Y, dX, dA, dB back, all on `stream`

@@ -27,7 +27,7 @@ EXPORTS = [
     "lora_select_config", "lora_workspace_bytes", "lora_plan_create", "lora_plan_destroy",
     "lora_plan_workspace_bytes", "lora_plan_set_workspace", "lora_plan_get_config", "lora_plan_describe",
     "lora_linear_fwd", "lora_linear_bwd", "lora_linear_bwd_saved_p", "lora_linear_bwd_dx", "lora_linear_bwd_da", "lora_linear_bwd_db",
-    "lora_dense_dw", "lora_nf4_quantize", "lora_linear_fwd_nf4", "lora_linear_bwd_nf4", "lora_step_host_staging_bytes", "lora_linear_step_host",
+    "lora_dense_dw", "lora_nf4_quantize", "lora_nf4_dequantize", "lora_linear_fwd_nf4", "lora_linear_bwd_nf4", "lora_step_host_staging_bytes", "lora_linear_step_host",
     "lora_last_device_status", "lora_strerror", "lora_launch_count",
     "lora_grad_contract_noalloc", "lora_grad_contract_noalloc_max_scratch",
 ]
@@ -81,8 +81,9 @@ def load(rebuild: bool = False) -> ctypes.CDLL:
     lib.lora_linear_bwd_db.argtypes = [vp, vp, ctypes.c_float, vp, vp]
     lib.lora_dense_dw.argtypes = [vp, vp, vp, vp, vp]
     lib.lora_nf4_quantize.argtypes = [vp, i64, i64, vp, vp, vp]
-    lib.lora_linear_fwd_nf4.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp]
-    lib.lora_linear_bwd_nf4.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
+    lib.lora_nf4_dequantize.argtypes = [vp, vp, i64, i64, vp, vp]
+    lib.lora_linear_fwd_nf4.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp]
+    lib.lora_linear_bwd_nf4.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp]
     lib.lora_step_host_staging_bytes.argtypes = [ctypes.POINTER(LoraShape), sz_p]
     lib.lora_linear_step_host.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, vp,
                                           ctypes.c_size_t, vp]
@@ -250,8 +251,17 @@ class LoraLinearPlan:
         return dX, dA, dB
 
     # -- NF4 frozen weight (Q+LoRA) ---------------------------------------------------------------
-    def fwd_nf4(self, X, W_codes, W_absmax, A, B, scale: float, Y: Optional[torch.Tensor] = None, stream=None):
-        """Y = X w_hat^T + scale (X A^T) B^T with w_hat = the NF4 weight (codes [d_out, d_in/2] uint8, absmax [d_in/64, d_out] fp32)."""
+    def _scratch_ptr(self, w_scratch):
+        if w_scratch is None:
+            return ctypes.c_void_p(0)
+        _want(w_scratch, "w_scratch", (self.d_out, self.d_in), torch.bfloat16, self.device)
+        return _ptr(w_scratch)
+
+    def fwd_nf4(self, X, W_codes, W_absmax, A, B, scale: float, Y: Optional[torch.Tensor] = None, w_scratch=None, stream=None):
+        """Y = X w_hat^T + scale (X A^T) B^T with w_hat = the NF4 weight (codes [d_out, d_in/2] uint8, absmax [d_in/64, d_out] fp32).
+
+        ``w_scratch`` ([d_out, d_in] bf16, reusable across layers): expand the weight once and run the bf16 kernels (fast
+        form); None: expand inside the GEMM kernels (no extra memory, slower for large batches)."""
         bf = torch.bfloat16
         _want(X, "X", (self.T, self.d_in), bf, self.device)
         _want(W_codes, "W_codes", (self.d_out, self.d_in // 2), torch.uint8, self.device)
@@ -263,10 +273,10 @@ class LoraLinearPlan:
         _want(Y, "Y", (self.T, self.d_out), bf, self.device)
         self.ensure_workspace()
         _check(self._lib.lora_linear_fwd_nf4(self._h, _ptr(X), _ptr(W_codes), _ptr(W_absmax), _ptr(A), _ptr(B), float(scale),
-                                             _ptr(Y), _stream_ptr(stream)), "lora_linear_fwd_nf4")
+                                             _ptr(Y), self._scratch_ptr(w_scratch), _stream_ptr(stream)), "lora_linear_fwd_nf4")
         return Y
 
-    def bwd_nf4(self, dY, X, W_codes, W_absmax, A, B, scale: float, dX=None, dA=None, dB=None, stream=None):
+    def bwd_nf4(self, dY, X, W_codes, W_absmax, A, B, scale: float, dX=None, dA=None, dB=None, w_scratch=None, stream=None):
         """(dX, dA, dB) of the layer with the NF4 weight."""
         bf = torch.bfloat16
         _want(dY, "dY", (self.T, self.d_out), bf, self.device)
@@ -286,7 +296,8 @@ class LoraLinearPlan:
         _want(dB, "dB", (self.d_out, self.r), torch.float32, self.device)
         self.ensure_workspace()
         _check(self._lib.lora_linear_bwd_nf4(self._h, _ptr(dY), _ptr(X), _ptr(W_codes), _ptr(W_absmax), _ptr(A), _ptr(B),
-                                             float(scale), _ptr(dX), _ptr(dA), _ptr(dB), _stream_ptr(stream)),
+                                             float(scale), _ptr(dX), _ptr(dA), _ptr(dB), self._scratch_ptr(w_scratch),
+                                             _stream_ptr(stream)),
                "lora_linear_bwd_nf4")
         return dX, dA, dB
 
@@ -378,3 +389,15 @@ def nf4_quantize(W: torch.Tensor, stream=None):
     absmax = torch.empty((d_in // 64, d_out), dtype=torch.float32, device=W.device)
     _check(load().lora_nf4_quantize(_ptr(W), d_out, d_in, _ptr(codes), _ptr(absmax), _stream_ptr(stream)), "lora_nf4_quantize")
     return codes, absmax
+
+
+def nf4_dequantize(codes: torch.Tensor, absmax: torch.Tensor, W: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """bf16 weight [d_out, d_in] from NF4 codes and block scales: every element bf16(level * absmax)."""
+    d_out, half = codes.shape
+    d_in = half * 2
+    if codes.dtype != torch.uint8 or absmax.dtype != torch.float32 or tuple(absmax.shape) != (d_in // 64, d_out):
+        raise ValueError("nf4_dequantize: codes [d_out, d_in/2] uint8 and absmax [d_in/64, d_out] fp32 expected")
+    if W is None:
+        W = torch.empty((d_out, d_in), dtype=torch.bfloat16, device=codes.device)
+    _check(load().lora_nf4_dequantize(_ptr(codes), _ptr(absmax), d_out, d_in, _ptr(W), _stream_ptr(stream)), "lora_nf4_dequantize")
+    return W

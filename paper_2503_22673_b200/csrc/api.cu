@@ -981,21 +981,48 @@ int lora_nf4_quantize(const void* W, int64_t d_out, int64_t d_in, void* codes, v
   return LORA_OK;
 }
 
+int lora_nf4_dequantize(const void* W_codes, const void* W_absmax, int64_t d_out, int64_t d_in, void* W, void* stream) {
+  if (!W || !W_codes || !W_absmax) return LORA_ERR_INVALID_ARG;
+  if (d_out <= 0 || d_in <= 0) return LORA_ERR_INVALID_ARG;
+  if (d_in % kNf4Block != 0 || d_out % 4 != 0 || d_out > (1ll << 24) || d_in > (1ll << 24)) return LORA_ERR_UNSUPPORTED_SHAPE;
+  if (!aligned16(W) || !aligned16(W_codes) || !aligned16(W_absmax)) return LORA_ERR_MISALIGNED;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return LORA_ERR_CUDA;
+  if (launch_nf4_dequantize(static_cast<const uint8_t*>(W_codes), static_cast<const float*>(W_absmax), d_out, d_in,
+                            static_cast<__nv_bfloat16*>(W), sms, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return LORA_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return LORA_OK;
+}
+
 int lora_linear_fwd_nf4(lora_plan_t* plan, const void* X, const void* W_codes, const void* W_absmax, const void* A,
-                        const void* B, float scale, void* Y, void* stream) {
+                        const void* B, float scale, void* Y, void* w_scratch, void* stream) {
   if (plan == nullptr) return LORA_ERR_INVALID_ARG;
   if (plan->shape.T == 0) return LORA_OK;
   if (!X || !W_codes || !W_absmax || !A || !B || !Y) return LORA_ERR_INVALID_ARG;
-  if (!aligned16(X) || !aligned16(W_codes) || !aligned16(W_absmax) || !aligned16(A) || !aligned16(B) || !aligned16(Y))
+  if (!aligned16(X) || !aligned16(W_codes) || !aligned16(W_absmax) || !aligned16(A) || !aligned16(B) || !aligned16(Y) ||
+      !aligned16(w_scratch))
     return LORA_ERR_MISALIGNED;
+  if (plan->shape.d_in % kNf4Block != 0 || plan->shape.d_out % 4 != 0) return LORA_ERR_UNSUPPORTED_SHAPE;
+  DeviceGuard guard(plan->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (w_scratch != nullptr) {
+    // expand once, then the bf16 path: every weight element is converted once per call instead of once per 256-token tile
+    if (launch_nf4_dequantize(static_cast<const uint8_t*>(W_codes), static_cast<const float*>(W_absmax), plan->shape.d_out,
+                              plan->shape.d_in, static_cast<__nv_bfloat16*>(w_scratch), plan->num_sms, st) != cudaSuccess)
+      return LORA_ERR_CUDA;
+    g_launches.fetch_add(1);
+    return launch_fwd(plan, X, w_scratch, A, B, scale, Y, st);
+  }
   const int rc = check_nf4(plan);
   if (rc != LORA_OK) return rc;
-  DeviceGuard guard(plan->device);
-  return launch_fwd_nf4(plan, X, W_codes, W_absmax, A, B, scale, Y, static_cast<cudaStream_t>(stream));
+  return launch_fwd_nf4(plan, X, W_codes, W_absmax, A, B, scale, Y, st);
 }
 
 int lora_linear_bwd_nf4(lora_plan_t* plan, const void* dY, const void* X, const void* W_codes, const void* W_absmax,
-                        const void* A, const void* B, float scale, void* dX, void* dA, void* dB, void* stream) {
+                        const void* A, const void* B, float scale, void* dX, void* dA, void* dB, void* w_scratch,
+                        void* stream) {
   if (plan == nullptr) return LORA_ERR_INVALID_ARG;
   if (!dA || !dB) return LORA_ERR_INVALID_ARG;
   if (!aligned16(dA) || !aligned16(dB)) return LORA_ERR_MISALIGNED;
@@ -1009,8 +1036,20 @@ int lora_linear_bwd_nf4(lora_plan_t* plan, const void* dY, const void* X, const 
   }
   if (!dY || !X || !W_codes || !W_absmax || !A || !B || !dX) return LORA_ERR_INVALID_ARG;
   if (!aligned16(dY) || !aligned16(X) || !aligned16(W_codes) || !aligned16(W_absmax) || !aligned16(A) || !aligned16(B) ||
-      !aligned16(dX))
+      !aligned16(dX) || !aligned16(w_scratch))
     return LORA_ERR_MISALIGNED;
+  if (plan->shape.d_in % kNf4Block != 0 || plan->shape.d_out % 4 != 0) return LORA_ERR_UNSUPPORTED_SHAPE;
+  if (w_scratch != nullptr) {
+    if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
+    if (launch_nf4_dequantize(static_cast<const uint8_t*>(W_codes), static_cast<const float*>(W_absmax), plan->shape.d_out,
+                              plan->shape.d_in, static_cast<__nv_bfloat16*>(w_scratch), plan->num_sms, st) != cudaSuccess)
+      return LORA_ERR_CUDA;
+    g_launches.fetch_add(1);
+    int rc2 = launch_dx(plan, dY, w_scratch, A, B, scale, dX, st);
+    if (rc2 == LORA_OK) rc2 = launch_da(plan, X, A, scale, dA, st);
+    if (rc2 == LORA_OK) rc2 = launch_db(plan, dY, scale, dB, st);
+    return rc2;
+  }
   int rc = check_nf4(plan);
   if (rc != LORA_OK) return rc;
   rc = launch_dx_nf4(plan, dY, W_codes, W_absmax, A, B, scale, dX, st);

@@ -99,7 +99,10 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   // NF4 only: ring of packed codes + block scales, and the byte -> (level of low nibble, level of high nibble) table
   uint8_t* code_ring = staging_ptr + 2 * kStagingBytes + kPairBarrierBytes;
-  float2* nf4_lut = reinterpret_cast<float2*>(code_ring + kNf4CodeSlots * kNf4CodeSlotBytes);
+  // level table replicated once per lane: entry (code, lane) at word code * 32 + lane, so a warp's 32 lookups with
+  // arbitrary codes hit 32 different banks (a shared 16- or 256-entry table serialises on bank conflicts and made the
+  // shared-memory pipe the bottleneck)
+  float* nf4_lut = reinterpret_cast<float*>(code_ring + kNf4CodeSlots * kNf4CodeSlotBytes);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -107,13 +110,13 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
-      mbar_init(full_bar(s), kNf4 ? 1 + 2 * kNf4DequantThreads : 2);   // NF4: every dequantising thread of the pair arrives
+      mbar_init(full_bar(s), kNf4 ? 1 + 2 * kNf4WarpsPerGroup : 2);   // NF4: the dequantising warps of one group, both CTAs
       mbar_init(empty_bar(s), 1);
     }
     if (kNf4) {
       for (int c = 0; c < kNf4CodeSlots; ++c) {
         mbar_init(cfull_bar(c), 1);
-        mbar_init(cempty_bar(c), kNf4DequantThreads);
+        mbar_init(cempty_bar(c), kNf4WarpsPerGroup);
       }
     }
     for (int b = 0; b < 2; ++b) {
@@ -136,8 +139,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
     tmem_relinquish_pair();
   }
   if (kNf4 && threadIdx.x >= kPairThreads) {
-    for (int b = threadIdx.x - kPairThreads; b < 256; b += kNf4DequantThreads)
-      nf4_lut[b] = make_float2(c_nf4_levels[b & 15], c_nf4_levels[b >> 4]);
+    for (int b = threadIdx.x - kPairThreads; b < 16 * 32; b += kNf4DequantThreads) nf4_lut[b] = c_nf4_levels[b >> 5];
   }
   tc_fence_before();
   __syncthreads();
@@ -360,19 +362,23 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       }
       if (!kExt && ok && n_my > 0) mma_tail((n_my - 1) & 1, (n_my - 1) >> 1);
     }
-  } else if (kNf4 && warp >= 9) {
-    // ================================ NF4 dequantisation (warps 9..12, 128 threads per CTA) ================================
-    // Thread d owns one 64-element block of every main k-block: 32 code bytes and one scale in, 128 bytes of bf16 out.
-    //   forward  (weight rows K-major):  row d of this CTA's weight rows, the k-block's 64 input features
-    //   backward (weight MN-major):      contraction row d % 64 of the k-block, column group d / 64 (64 input features)
+  } else if (kNf4 && warp >= kPairThreads / 32) {
+    // ================================ NF4 dequantisation (warps 9..16, 256 threads per CTA) ================================
+    // The eight warps form kNf4Groups groups of kNf4WarpsPerGroup warps; ring items go to the groups round-robin, so
+    // several items are converted at once.  One item's conversion is a long dependent chain (wait, code fetch, table
+    // look-ups, stores, proxy fence: measured ~3000 cycles when all warps shared each item) while the tensor core
+    // consumes an item in ~512 cycles; only concurrency across items hides that chain.
+    // A group's 64 threads own the 128 quantisation blocks of an item, two each (32 code bytes + one scale in, 128 bytes
+    // of bf16 out per block):
+    //   forward  (weight rows K-major):  block u = row u of this CTA's weight rows, the k-block's 64 input features
+    //   backward (weight MN-major):      block u = contraction row u % 64 of the k-block, column group u / 64
     // Every element is bf16(level * absmax): one float32 product, one round-to-nearest-even.
-    const int d = threadIdx.x - kPairThreads;
-    const int row = kBmn ? (d & 63) : d;
-    const int grp = kBmn ? (d >> 6) : 0;
-    const bool has_row = kBmn || d < (BN >> 1);
-    const uint32_t code_off = kBmn ? static_cast<uint32_t>(row * 64 + grp * 32) : static_cast<uint32_t>(row * 32);
-    const uint32_t scale_off = 4096u + 4u * static_cast<uint32_t>(kBmn ? grp * 64 + row : row);
-    int slot = 0, phase = 0, cslot = 0, cphase = 0;
+    const int dwarp = warp - kPairThreads / 32;
+    const int gid = dwarp / kNf4WarpsPerGroup;
+    const int t = (dwarp % kNf4WarpsPerGroup) * 32 + lane;
+    const uint32_t lut_lane = smem_u32(nf4_lut) + 4u * lane;
+    const uint32_t code_ring_u32 = smem_u32(code_ring);
+    int slot = 0, phase = 0, cslot = 0, cphase = 0, turn = 0;
     bool ok = true;
     for (int i = 0; i < n_my && ok; ++i) {
       const int sp = (pair + i * G) % SK;
@@ -380,34 +386,49 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       const bool has_tail = sp == SK - 1 && p.r_pad > 0;
       for (int kb = kb0; kb < kb1 + (has_tail ? 1 : 0) && ok; ++kb) {
         const bool main_item = kb < kb1;
-        if (main_item) ok = warp_wait(cfull_bar(cslot), cphase, abort_flag, p.status, DEV_TIMEOUT_FULL, false, 0);
-        if (ok) ok = warp_wait(empty_bar(slot), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY, false, 0);
-        if (!ok) break;
-        if (main_item) {
-          (void)mbar_try_wait(cfull_bar(cslot), cphase);     // every reading thread observes the completed copy itself
-          const uint8_t* src = code_ring + cslot * kNf4CodeSlotBytes;
-          if (has_row) {
-            const uint4 c0 = *reinterpret_cast<const uint4*>(src + code_off);
-            const uint4 c1 = *reinterpret_cast<const uint4*>(src + code_off + 16);
-            const float scale = *reinterpret_cast<const float*>(src + scale_off);
-            uint8_t* dst = smem + slot * kStage + 16384 + grp * 8192;
-            const uint32_t cw[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+        if (turn == gid) {
+          if (main_item) ok = warp_wait(cfull_bar(cslot), cphase, abort_flag, p.status, DEV_TIMEOUT_FULL, false, 0);
+          if (ok) ok = warp_wait(empty_bar(slot), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY, false, 0);
+          if (!ok) break;
+          if (main_item) {
+            (void)mbar_try_wait(cfull_bar(cslot), cphase);     // every reading thread observes the completed copy itself
+            const uint32_t src = code_ring_u32 + cslot * kNf4CodeSlotBytes;
+            const uint32_t stage_b = ring + slot * kStage + 16384;
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {     // 4 code bytes -> 8 elements -> one 16-byte chunk of the swizzled row
-              uint32_t w[4];
+            for (int h = 0; h < 128 / (32 * kNf4WarpsPerGroup); ++h) {
+              const int u = t + h * 32 * kNf4WarpsPerGroup;
+              const int row = kBmn ? (u & 63) : u;
+              const int grp = kBmn ? (u >> 6) : 0;
+              if (!kBmn && u >= (BN >> 1)) continue;           // forward: this CTA holds block_n / 2 weight rows
+              const uint32_t code_addr = src + (kBmn ? static_cast<uint32_t>(row * 64 + grp * 32) : static_cast<uint32_t>(row * 32));
+              const uint4 c0 = lds_v4(code_addr), c1 = lds_v4(code_addr + 16);
+              const float scale = lds_f32(src + 4096u + 4u * static_cast<uint32_t>(u));
+              const uint32_t dst = stage_b + grp * 8192;
+              const uint32_t cw[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                const float2 lv = nf4_lut[(cw[q] >> (8 * j)) & 0xFFu];
-                w[j] = pack_bf16x2(lv.x * scale, lv.y * scale);
+              for (int q = 0; q < 8; ++q) {     // 4 code bytes -> 8 elements -> one 16-byte chunk of the swizzled row
+                uint32_t w[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const float lo = lds_const_f32(lut_lane + (((cw[q] >> (8 * j)) & 0xFu) << 7));
+                  const float hi = lds_const_f32(lut_lane + (((cw[q] >> (8 * j + 4)) & 0xFu) << 7));
+                  w[j] = pack_bf16x2(lo * scale, hi * scale);
+                }
+                sts_v4(dst + sw128_offset(row, q), w[0], w[1], w[2], w[3]);
               }
-              *reinterpret_cast<uint4*>(dst + sw128_offset(row, q)) = make_uint4(w[0], w[1], w[2], w[3]);
             }
+            fence_proxy_async_smem();           // the tensor core reads the tile through the async proxy
           }
-          fence_proxy_async_smem();           // the tensor core reads the tile through the async proxy
-          mbar_arrive(cempty_bar(cslot));
-          if (++cslot == kNf4CodeSlots) { cslot = 0; cphase ^= 1; }
+          // one arrival per warp: every lane's writes and fence come before the warp barrier, the elected lane's
+          // release-arrive after it
+          __syncwarp();
+          if (lane == 0) {
+            if (main_item) mbar_arrive(cempty_bar(cslot));
+            mbar_arrive_cluster(map_to_cta(full_bar(slot), 0));
+          }
         }
-        mbar_arrive_cluster(map_to_cta(full_bar(slot), 0));
+        if (++turn == kNf4Groups) turn = 0;
+        if (main_item && ++cslot == kNf4CodeSlots) { cslot = 0; cphase ^= 1; }
         if (++slot == S) { slot = 0; phase ^= 1; }
       }
     }
@@ -600,7 +621,7 @@ cudaError_t launch_splitk_reduce(const float* part, __nv_bfloat16* out, long lon
 
 size_t gemm_pair_smem_bytes(int stages, bool nf4) {
   return static_cast<size_t>(stages) * kPairStageBytesFwd + 2 * kStagingBytes + kPairBarrierBytes + 1024 +
-         (nf4 ? kNf4CodeSlots * kNf4CodeSlotBytes + 256 * sizeof(float2) : 0);
+         (nf4 ? kNf4CodeSlots * kNf4CodeSlotBytes + 16 * 32 * sizeof(float) : 0);
 }
 
 cudaError_t gemm_pair_configure() {

@@ -64,11 +64,13 @@ size_t gemm_smem_bytes(int stages);
 constexpr int kPairBlockM = 256;
 constexpr int kPairThreads = 288;           // warps 0..3 TMA producers, warp 4 MMA + TMEM, warps 5..8 epilogue
 constexpr int kPairStageBytesFwd = 32768;   // 128 x 64 activations + 128 x 64 weight/adapter rows per CTA
-// NF4 weight (K-extended forms only): four more warps dequantise; packed codes + block scales travel through a ring of
+// NF4 weight (K-extended forms only): eight more warps dequantise; packed codes + block scales travel through a ring of
 // kNf4CodeSlots slots of 4096 code bytes + 128 float scales
-constexpr int kNf4DequantThreads = 128;
+constexpr int kNf4DequantThreads = 256;
+constexpr int kNf4Groups = 4;               // ring items are dealt round-robin to groups of dequantising warps
+constexpr int kNf4WarpsPerGroup = kNf4DequantThreads / 32 / kNf4Groups;
 constexpr int kPairThreadsNf4 = kPairThreads + kNf4DequantThreads;
-constexpr int kNf4CodeSlots = 4;
+constexpr int kNf4CodeSlots = 6;
 constexpr int kNf4CodeSlotBytes = 4096 + 512;
 constexpr int kNf4Block = 64;               // elements per quantisation block (= kBlockK)
 size_t gemm_pair_smem_bytes(int stages, bool nf4 = false);
@@ -102,6 +104,10 @@ cudaError_t launch_gemm_pair_dx_nf4(const CUtensorMap& tmdY, const CUtensorMap& 
 // W [d_out, d_in] bf16 -> NF4 codes [d_out, d_in/2] + block scales [d_in/64, d_out] (nf4_quant.cu)
 cudaError_t launch_nf4_quantize(const __nv_bfloat16* W, long long d_out, long long d_in, uint8_t* codes, float* absmax,
                                 cudaStream_t stream);
+
+// NF4 codes + block scales -> bf16 weight [d_out, d_in], every element bf16(level * absmax) (nf4_quant.cu)
+cudaError_t launch_nf4_dequantize(const uint8_t* codes, const float* absmax, long long d_out, long long d_in, __nv_bfloat16* W,
+                                  int num_sms, cudaStream_t stream);
 
 // dense weight gradient dW[d_out, d_in] = dY^T X (p.r_pad = 0: no rank-r k-block): tmdYt = dY [T, d_out] box 64(o) x 64(t),
 // tmX = X [T, d_in] box 64(i) x 64(t), tmdW box 64 x 128; p.M = d_out, p.N = d_in, p.K = T

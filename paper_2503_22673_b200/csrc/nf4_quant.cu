@@ -5,8 +5,12 @@
 //   * code = number of midpoints between neighbouring NF4 levels that lie strictly below x = w / absmax (float32),
 //     i.e. the nearest level, the lower one on a tie; an all-zero block has absmax 0 and code 7 (level 0)
 //   * byte k of a row of `codes` [d_out, d_in / 2] holds element 2k in its low nibble, element 2k + 1 in its high nibble
-// One warp per block: a lane owns two neighbouring elements, i.e. one output byte.
+// Quantiser: one warp per block, a lane owns two neighbouring elements, i.e. one output byte.
+// Expander (codes + scales -> bf16 weight, every element bf16(level * absmax): one float32 product, one rounding): a
+// thread turns 4 code bytes into 8 bf16 (16 bytes), so a warp reads 128 contiguous code bytes and writes 512 contiguous
+// bytes; the level table sits in shared memory once per lane (no bank conflicts for arbitrary codes).
 #include "kernels.h"
+#include "sm100_ptx.cuh"
 
 namespace lora {
 
@@ -49,7 +53,56 @@ __global__ void __launch_bounds__(256) lora_nf4_quantize_kernel(const __nv_bfloa
   if (lane == 0) absmax[b * d_out + o] = m;
 }
 
+__global__ void __launch_bounds__(256) lora_nf4_dequantize_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ absmax,
+                                                                  long long d_out, long long d_in, uint4* __restrict__ W) {
+  __shared__ float lut[16 * 32];
+  pdl_launch_dependents();
+  for (int b = threadIdx.x; b < 16 * 32; b += blockDim.x) lut[b] = c_nf4_quant_levels[b >> 5];
+  __syncthreads();
+  pdl_wait();
+  const float* lut_lane = lut + (threadIdx.x & 31);
+  const int words_row = static_cast<int>(d_in / 8);            // 4 code bytes = 8 elements per thread and step
+  // a block walks whole rows (no index division); a thread fetches up to four code words (t, t + 256, ...) and their
+  // scales before it converts any of them, so that four loads per thread are in flight
+  for (long long o = blockIdx.x; o < d_out; o += gridDim.x) {
+    const uint32_t* crow = codes + o * words_row;
+    uint4* wrow = W + o * words_row;
+    for (int base = 0; base < words_row; base += 4 * blockDim.x) {
+      uint32_t cw[4];
+      float scale[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int wcol = base + k * blockDim.x + threadIdx.x;
+        cw[k] = wcol < words_row ? __ldg(crow + wcol) : 0u;
+        scale[k] = wcol < words_row ? __ldg(absmax + static_cast<long long>(wcol >> 3) * d_out + o) : 0.f;   // 8 words = one block
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int wcol = base + k * blockDim.x + threadIdx.x;
+        if (wcol >= words_row) continue;
+        uint32_t w[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float lo = lut_lane[((cw[k] >> (8 * j)) & 0xFu) << 5];
+          const float hi = lut_lane[((cw[k] >> (8 * j + 4)) & 0xFu) << 5];
+          w[j] = pack_bf16x2(lo * scale[k], hi * scale[k]);
+        }
+        wrow[wcol] = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    }
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_nf4_dequantize(const uint8_t* codes, const float* absmax, long long d_out, long long d_in, __nv_bfloat16* W,
+                                  int num_sms, cudaStream_t stream) {
+  long long blocks = d_out;
+  const long long cap = static_cast<long long>(num_sms > 0 ? num_sms : 148) * 16;
+  if (blocks > cap) blocks = cap;
+  return launch_pdl(lora_nf4_dequantize_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, stream,
+                    reinterpret_cast<const uint32_t*>(codes), absmax, d_out, d_in, reinterpret_cast<uint4*>(W));
+}
 
 cudaError_t launch_nf4_quantize(const __nv_bfloat16* W, long long d_out, long long d_in, uint8_t* codes, float* absmax,
                                 cudaStream_t stream) {

@@ -287,6 +287,30 @@ __device__ __forceinline__ uint32_t sw128_offset(uint32_t row, uint32_t chunk) {
 }
 
 // ----------------------------------------------------------------------------------------
+// explicit shared-space accesses by 32-bit shared address (pointers derived from the aligned dynamic shared-memory
+// base are generic to the compiler, and generic accesses are slower and cannot be reordered around each other)
+// ----------------------------------------------------------------------------------------
+// read of a table that is constant after start-up: the compiler may schedule, hoist or merge it freely
+__device__ __forceinline__ float lds_const_f32(uint32_t addr) {
+  float v;
+  asm("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float lds_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts_v4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
+  asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+
+// ----------------------------------------------------------------------------------------
 // CTA pairs (cta_group::2): cluster helpers, peer barriers, 2-CTA TMA / MMA / TMEM forms
 // ----------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t cluster_cta_rank() {

@@ -55,7 +55,17 @@ def test_quantiser_hand_worked_block():
     assert torch.all(codes[1:] == 119)
 
 
-def run_nf4_layer(p, t, codes, absmax):
+def test_dequantiser_is_bit_exact():
+    bits = _bf16_weight(520, 1024, seed=3)
+    W = inputs.bf16_to_f64(bits).astype(np.float32)
+    W[5, 128:192] = 0.0
+    codes, absmax = nf4.quantize(W)
+    got = binding.nf4_dequantize(torch.from_numpy(codes).cuda(), torch.from_numpy(absmax).cuda())
+    torch.cuda.synchronize()
+    assert np.array_equal(host64(got), nf4.dequantize(codes, absmax))
+
+
+def run_nf4_layer(p, t, codes, absmax, use_scratch=False):
     d = {k: dev(t[k]) for k in ("X", "A", "B", "dY")}
     cd, ad = torch.from_numpy(codes).cuda(), torch.from_numpy(absmax).cuda()
     plan = binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r)
@@ -63,8 +73,13 @@ def run_nf4_layer(p, t, codes, absmax):
     for name, shape, dt in (("Y", (p.T, p.d_out), torch.bfloat16), ("dX", (p.T, p.d_in), torch.bfloat16),
                             ("dA", (p.r, p.d_in), torch.float32), ("dB", (p.d_out, p.r), torch.float32)):
         bufs[name], out[name] = guarded(shape, dt)
-    plan.fwd_nf4(d["X"], cd, ad, d["A"], d["B"], p.scale, out["Y"])
-    plan.bwd_nf4(d["dY"], d["X"], cd, ad, d["A"], d["B"], p.scale, out["dX"], out["dA"], out["dB"])
+    sbuf, scratch = guarded((p.d_out, p.d_in), torch.bfloat16) if use_scratch else (None, None)
+    plan.fwd_nf4(d["X"], cd, ad, d["A"], d["B"], p.scale, out["Y"], w_scratch=scratch)
+    if use_scratch:
+        scratch.fill_(float("nan"))                     # backward must rebuild the weight itself
+    plan.bwd_nf4(d["dY"], d["X"], cd, ad, d["A"], d["B"], p.scale, out["dX"], out["dA"], out["dB"], w_scratch=scratch)
+    if use_scratch:
+        assert guards_intact(sbuf, scratch.numel()), "w_scratch: write outside the buffer"
     code, msg = plan.device_status()
     assert code == 0, msg
     for name in out:
@@ -85,12 +100,13 @@ NF4_SHAPES = [
 ]
 
 
+@pytest.mark.parametrize("use_scratch", [False, True], ids=["in_kernel", "scratch"])
 @pytest.mark.parametrize("T,d_in,d_out,r,scale", NF4_SHAPES)
-def test_nf4_layer_elementwise(T, d_in, d_out, r, scale):
+def test_nf4_layer_elementwise(T, d_in, d_out, r, scale, use_scratch):
     p, t = inputs.draw_custom(T, d_in, d_out, r, scale, seed=4)
     W32 = inputs.bf16_to_f64(t["W"]).astype(np.float32)
     codes, absmax = nf4.quantize(W32)                          # the ORACLE's codes go to both sides
-    out = run_nf4_layer(p, t, codes, absmax)
+    out = run_nf4_layer(p, t, codes, absmax, use_scratch)
     f = {k: inputs.bf16_to_f64(t[k]) for k in ("X", "A", "B", "dY")}
     Y = nf4.forward(f["X"], codes, absmax, f["A"], f["B"], p.scale)
     dX, dA, dB = nf4.backward(f["dY"], f["X"], codes, absmax, f["A"], f["B"], p.scale)
@@ -100,7 +116,21 @@ def test_nf4_layer_elementwise(T, d_in, d_out, r, scale):
     assert errs["dA"] <= TOL_F32 and errs["dB"] <= TOL_F32, errs
 
 
-def test_nf4_weight_only_is_tight():
+def test_nf4_scratch_form_covers_small_batches():
+    """With a scratch weight the bf16 kernels run, so batches of at most 128 tokens work too."""
+    p, t = inputs.draw_custom(100, 128, 72, 8, 2.0, seed=8)
+    W32 = inputs.bf16_to_f64(t["W"]).astype(np.float32)
+    codes, absmax = nf4.quantize(W32)
+    out = run_nf4_layer(p, t, codes, absmax, use_scratch=True)
+    f = {k: inputs.bf16_to_f64(t[k]) for k in ("X", "A", "B", "dY")}
+    Y = nf4.forward(f["X"], codes, absmax, f["A"], f["B"], p.scale)
+    dX, dA, dB = nf4.backward(f["dY"], f["X"], codes, absmax, f["A"], f["B"], p.scale)
+    assert oracle.rel_err(host64(out["Y"]), Y) <= TOL_BF16 and oracle.rel_err(host64(out["dX"]), dX) <= TOL_BF16
+    assert oracle.rel_err(host64(out["dA"]), dA) <= TOL_F32 and oracle.rel_err(host64(out["dB"]), dB) <= TOL_F32
+
+
+@pytest.mark.parametrize("use_scratch", [False, True], ids=["in_kernel", "scratch"])
+def test_nf4_weight_only_is_tight(use_scratch):
     """A = 0, B = 0 and one-hot X / dY rows read single rows and columns of the dequantised weight: Y and dX must then be
     the oracle's bf16(level * absmax) values exactly (one product, one rounding, no accumulation)."""
     T, d_in, d_out, r = 256, 256, 256, 8
@@ -114,7 +144,7 @@ def test_nf4_weight_only_is_tight():
     t2["X"], t2["dY"] = bits(eye), bits(eye)
     t2["A"] = np.zeros_like(t["A"])
     t2["B"] = np.zeros_like(t["B"])
-    out = run_nf4_layer(p, t2, codes, absmax)
+    out = run_nf4_layer(p, t2, codes, absmax, use_scratch)
     assert np.array_equal(host64(out["Y"]), what.T)            # Y = I w_hat^T
     assert np.array_equal(host64(out["dX"]), what)             # dX = I w_hat
 
