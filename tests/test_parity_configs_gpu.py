@@ -99,3 +99,66 @@ def test_seven_projection_layer_full_size():
             x_dev.clear()
             x_dev[p.x_group] = dev(t["X"])
         check_projection(p, t, x_dev[p.x_group])
+
+
+# ---------------------------------------------------------------------------------------------
+# the two further rows at full size: dense weight gradient (full fine-tuning) and the NF4 weight (Q+LoRA)
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("idx", [1, 3])
+def test_dense_dw_full_size_sampled(idx):
+    """dW = dY^T X at the benchmark sizes: sampled rows of dW (each row o is dY[:, o]^T X, one fp64 matrix-vector
+    product) against the oracle's definition, rows on both sides of the 128/256-row tile borders included; plus the
+    identity  <dW, M> = <dY, X M^T>  for a random bf16 M on the complete output (fp64 on the device)."""
+    (p, t), = list(inputs.draw_workload(idx, seed=0))
+    X, dY = dev(t["X"]), dev(t["dY"])
+    plan = binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r)
+    dW = plan.dense_dw(dY, X)
+    code, msg = plan.device_status()
+    assert code == 0, msg
+    rows = sample_rows(p.d_out, n_random=24, seed=1)
+    Xf = inputs.bf16_to_f64(t["X"])
+    ref = oracle.dense_weight_grad(inputs.bf16_to_f64(t["dY"][:, rows]), Xf)
+    del Xf
+    err = oracle.rel_err(host64(dW[torch.from_numpy(rows).cuda()]), ref)
+    assert err <= TOL_BF16, (p.name, err)
+    M = torch.randn((p.d_out, p.d_in), device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    lhs = dot64(dW, M)
+    rhs = dot64(dY, (X.float() @ M.float().T))        # library matmul only inside the CHECK, fp32 accumulate
+    scale = (dW.double().norm() * M.double().norm()).item()
+    assert abs(lhs - rhs) / scale <= 1e-3, (p.name, lhs, rhs, scale)
+    plan.close()
+    del X, dY, dW, M
+    gc.collect()
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("use_scratch", [True, False], ids=["scratch", "in_kernel"])
+def test_nf4_full_size_config1(use_scratch):
+    """Q+LoRA at the q_proj size (T = 8192, 4096 -> 4096, r = 16): the GPU quantiser's codes and scales must equal the
+    oracle's bit for bit; Y and dX on sampled rows and dA, dB in full against the oracle on the dequantised weight."""
+    from oracle import nf4_oracle as nf4
+    (p, t), = list(inputs.draw_workload(1, seed=0))
+    d = {k: dev(v) for k, v in t.items()}
+    codes, absmax = binding.nf4_quantize(d["W"])
+    ref_codes, ref_absmax = nf4.quantize(inputs.bf16_to_f64(t["W"]).astype(np.float32))
+    assert np.array_equal(codes.cpu().numpy(), ref_codes) and np.array_equal(absmax.cpu().numpy(), ref_absmax)
+    plan = binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r)
+    scratch = torch.empty((p.d_out, p.d_in), dtype=torch.bfloat16, device="cuda") if use_scratch else None
+    Y = plan.fwd_nf4(d["X"], codes, absmax, d["A"], d["B"], p.scale, w_scratch=scratch)
+    dX, dA, dB = plan.bwd_nf4(d["dY"], d["X"], codes, absmax, d["A"], d["B"], p.scale, w_scratch=scratch)
+    code, msg = plan.device_status()
+    assert code == 0, msg
+    rows = sample_rows(p.T)
+    rows_t = torch.from_numpy(rows).cuda()
+    What, A, B = nf4.dequantize(ref_codes, ref_absmax), inputs.bf16_to_f64(t["A"]), inputs.bf16_to_f64(t["B"])
+    Yr = oracle.forward_rows(np.arange(len(rows)), inputs.bf16_to_f64(t["X"][rows]), What, A, B, p.scale)
+    dXr = oracle.backward_dx_rows(np.arange(len(rows)), inputs.bf16_to_f64(t["dY"][rows]), What, A, B, p.scale)
+    dAr, dBr = oracle.backward_adapter_grads(inputs.bf16_to_f64(t["dY"]), inputs.bf16_to_f64(t["X"]), A, B, p.scale)
+    errs = {"Y": oracle.rel_err(host64(Y[rows_t]), Yr), "dX": oracle.rel_err(host64(dX[rows_t]), dXr),
+            "dA": oracle.rel_err(host64(dA), dAr), "dB": oracle.rel_err(host64(dB), dBr)}
+    plan.close()
+    assert errs["Y"] <= TOL_BF16 and errs["dX"] <= TOL_BF16, errs
+    assert errs["dA"] <= TOL_F32 and errs["dB"] <= TOL_F32, errs
+    del d, Y, dX, dA, dB
+    gc.collect()
+    torch.cuda.empty_cache()
