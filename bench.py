@@ -64,11 +64,13 @@ class ClockSampler:
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
+        import tempfile
         self.proc = None
+        self.out = tempfile.TemporaryFile(mode="w+")      # a file, not a pipe: a full pipe would stall nvidia-smi
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20"],
-                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                stdout=self.out, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
 
@@ -86,10 +88,13 @@ class ClockSampler:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
         try:
-            out, _ = self.proc.communicate(timeout=5)
+            self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-            out, _ = self.proc.communicate()
+            self.proc.wait()
+        self.out.seek(0)
+        out = self.out.read()
+        self.out.close()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
         rows = []
         for line in out.splitlines():
@@ -343,7 +348,7 @@ def run_ours(args):
     # ---- the same steps once more with events between the kernels: per-kernel durations.  An event record between two
     #      launches suppresses their programmatic overlap, so this pass is a little slower than the timed region; its
     #      own per-step time is reported as ms_per_step_instrumented ----
-    events = [[[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in protos] for _ in range(args.steps)]
+    events = [[[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in protos] for _ in range(args.steps)]
     i_a, i_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
     i_a.record()
@@ -355,36 +360,43 @@ def run_ours(args):
     ms_step_instr = i_a.elapsed_time(i_b) / args.steps
     clocks = sampler.stop(t_host0, t_host2) if sampler is not None else None
 
-    # per-kernel mean durations (ms) and rooflines
+    # per-stage mean durations (ms) from the instrumented pass.  Events: 0 before the forward call, 1 after it, 2 after the
+    # dY B pre-pass, 3 after the dX GEMM launch, 4 after the dA stage, 5 after the dB stage
     kern = {}
     for j, p in enumerate(protos):
-        dur = [statistics.mean(events[k][j][i].elapsed_time(events[k][j][i + 1]) for k in range(args.steps)) for i in range(4)]
-        gemm_flops = 2.0 * p.T * p.d_in * p.d_out + 2.0 * p.T * p.r * (p.d_in + p.d_out)
+        dur = [statistics.mean(events[k][j][i].elapsed_time(events[k][j][i + 1]) for k in range(args.steps)) for i in range(5)]
+        fwd_flops = 2.0 * p.T * p.d_in * p.d_out + 2.0 * p.T * p.r * (p.d_in + p.d_out)
+        dxg_flops = 2.0 * p.T * p.d_in * p.d_out + 2.0 * p.T * p.r * p.d_in            # dense + the rank-r k-block (Q A)
+        q_bytes = 2.0 * p.T * p.d_out + 2.0 * p.T * p.r + 2.0 * p.r * p.d_out           # dY once, B in, Qt out
         da_bytes = 2.0 * p.T * p.d_in + 2.0 * p.T * p.r * 2 + 4.0 * p.r * p.d_in      # X once, Qt in, Pt out, dA out
         db_bytes = 2.0 * p.T * p.d_out + 2.0 * p.T * p.r + 4.0 * p.r * p.d_out        # dY once, Pt in, dB out
         kern[p.name] = {
-            "fwd_gemm": {"ms": dur[0], "tflops": gemm_flops / dur[0] / 1e9,
-                         "frac_of_bf16_peak": gemm_flops / dur[0] / 1e9 / pk["bf16_tflops"]},
-            "dx_gemm": {"ms": dur[1], "tflops": gemm_flops / dur[1] / 1e9,
-                        "frac_of_bf16_peak": gemm_flops / dur[1] / 1e9 / pk["bf16_tflops"]},
-            "dA": {"ms": dur[2], "gbs": da_bytes / dur[2] / 1e6, "frac_of_hbm_peak": da_bytes / dur[2] / 1e6 / pk["hbm_gbs"]},
-            "dB": {"ms": dur[3], "gbs": db_bytes / dur[3] / 1e6, "frac_of_hbm_peak": db_bytes / dur[3] / 1e6 / pk["hbm_gbs"]},
+            "fwd_stage": {"ms": dur[0], "tflops": fwd_flops / dur[0] / 1e9,
+                          "frac_of_bf16_peak": fwd_flops / dur[0] / 1e9 / pk["bf16_tflops"]},
+            "q_prepass": {"ms": dur[1], "gbs": q_bytes / dur[1] / 1e6, "frac_of_hbm_peak": q_bytes / dur[1] / 1e6 / pk["hbm_gbs"]},
+            "dx_gemm": {"ms": dur[2], "tflops": dxg_flops / dur[2] / 1e9,
+                        "frac_of_bf16_peak": dxg_flops / dur[2] / 1e9 / pk["bf16_tflops"]},
+            "dA": {"ms": dur[3], "gbs": da_bytes / dur[3] / 1e6, "frac_of_hbm_peak": da_bytes / dur[3] / 1e6 / pk["hbm_gbs"]},
+            "dB": {"ms": dur[4], "gbs": db_bytes / dur[4] / 1e6, "frac_of_hbm_peak": db_bytes / dur[4] / 1e6 / pk["hbm_gbs"]},
         }
-    # dominant kernel for the roofline: the forward GEMM where the forward call is ONE launch (fused adapter), so the
-    # event pair brackets exactly that kernel; otherwise the dX stage (Q pre-pass + K-extended GEMM, 3 launches)
-    dom_p = max(protos, key=lambda p: kern[p.name]["fwd_gemm"]["ms"] + kern[p.name]["dx_gemm"]["ms"])
+    # dominant kernel for the roofline: the dX GEMM launch of the projection with the longest GEMMs.  Its event pair
+    # brackets exactly ONE kernel (the K-extended CTA-pair GEMM; the dY B pre-pass sits before the first of the two events)
+    # unless the plan splits it along K or the batch is too small for CTA pairs (then the bracket holds what dx_launches says)
+    dom_p = max(protos, key=lambda p: kern[p.name]["fwd_stage"]["ms"] + kern[p.name]["dx_gemm"]["ms"])
     dom_plan = plans[protos.index(dom_p)].config()
-    single = dom_plan["cta_group"] == 1 or dom_plan["fwd_ext"] == 0
-    dom_k = "fwd_gemm" if single else "dx_gemm"
-    dom = kern[dom_p.name][dom_k]
+    dom = kern[dom_p.name]["dx_gemm"]
+    dx_launches = 1 + (1 if dom_plan["dx_split_k"] > 1 and dom_plan["cta_group"] == 2 else 0)
     roofline = {"bound": "tensor",
-                "kernel": (f"lora_gemm_pair_kernel, forward with fused adapter ({dom_p.name}), one launch" if single else
-                           f"dX stage ({dom_p.name}): Q pre-pass + K-extended lora_gemm_pair_kernel"),
+                "kernel": f"lora_gemm_pair_kernel<1,1>: dX = dY W + (s dY B) A as one K-extended GEMM ({dom_p.name})"
+                          if dom_plan["cta_group"] == 2 else f"lora_gemm_kernel<1> (single-CTA dX GEMM, {dom_p.name})",
+                "launches_in_bracket": dx_launches,
                 "achieved": dom["tflops"], "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
                 "frac": dom["tflops"] / pk["bf16_tflops"], "peak_kind": f"bf16 burst, of {pk['source']}",
+                "frac_of_sustained": dom["tflops"] / pk["bf16_tflops_sustained"],
                 "ms_per_launch": dom["ms"],
-                "traffic": (NCU_TRAFFIC["bytes_per_launch"][dom_k] if NCU_TRAFFIC["gemm_sha"] == gemm_source_sha()
-                            and args.workload == 1 and single else None)}
+                "flops_per_launch": 2.0 * dom_p.T * dom_p.d_in * dom_p.d_out + 2.0 * dom_p.T * dom_p.r * dom_p.d_in,
+                "traffic": (NCU_TRAFFIC["bytes_per_launch"]["dx_gemm"] if NCU_TRAFFIC["gemm_sha"] == gemm_source_sha()
+                            and args.workload == 1 else None)}
 
     # ---- variant: backward that reuses the forward's X A^T (lora_linear_bwd_saved_p), same inputs and rotation ----
     def step_saved(k):
@@ -475,38 +487,58 @@ def run_ours(args):
                                             "of the LoRA step"}
     del dw_out
 
-    # ---- end to end: host buffers through the C ABI, copies inside the timed region ----
-    h_sets, staging = [], []
+    # ---- end to end: host buffers through the C ABI (lora_linear_step_host), copies inside the timed region.  Every step
+    #      copies its inputs from pinned host memory, runs forward + backward and copies Y, dX, dA, dB back.  Two lanes
+    #      (plan + staging + host output buffers + stream each) alternate, so that the copy-in of one step overlaps the
+    #      copy-out of the previous one on the two DMA directions; each step's own chain stays in order on its stream ----
+    n_lanes = 1 if args.workload == 4 else 2
+    h_in = []
     for j, (p, d0) in enumerate(sets[0]):
-        h = {k: d0[k].cpu().pin_memory() for k in ("X", "A", "B", "dY")}
-        ho = {k: torch.empty_like(d0[k], device="cpu").pin_memory() for k in ("Y", "dX", "dA", "dB")}
-        h_sets.append((h, ho))
-        staging.append(torch.empty(plans[j].step_host_staging_bytes(), dtype=torch.uint8, device=device))
+        h_in.append({k: d0[k].cpu().pin_memory() for k in ("X", "A", "B", "dY")})
+    lanes = []
+    for ln in range(n_lanes):
+        lp = plans if ln == 0 else [binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r, device=local_rank) for p in protos]
+        for pl in lp:
+            pl.ensure_workspace()
+        outs = [{k: torch.empty_like(d0[k], device="cpu").pin_memory() for k in ("Y", "dX", "dA", "dB")} for _, d0 in sets[0]]
+        stg = [torch.empty(lp[j].step_host_staging_bytes(), dtype=torch.uint8, device=device) for j in range(len(protos))]
+        lanes.append({"plans": lp, "out": outs, "staging": stg, "stream": torch.cuda.Stream(device=device)})
 
-    def step_host():
+    def step_host(k):
+        ln = lanes[k % n_lanes]
         for j, (p, d0) in enumerate(sets[0]):
-            h, ho = h_sets[j]
-            plans[j].step_host(h["X"], d0["W"], h["A"], h["B"], h["dY"], p.scale, ho["Y"], ho["dX"], ho["dA"], ho["dB"],
-                               staging[j])
+            h, ho = h_in[j], ln["out"][j]
+            ln["plans"][j].step_host(h["X"], d0["W"], h["A"], h["B"], h["dY"], p.scale, ho["Y"], ho["dX"], ho["dA"], ho["dB"],
+                                     ln["staging"][j], stream=ln["stream"])
 
-    n_e2e = max(3, min(args.steps, 10 if args.workload != 4 else 3))
-    for _ in range(2):
-        step_host()
-    torch.cuda.synchronize()
-    e_a, e_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    def run_host(n):
+        cur = torch.cuda.current_stream()
+        start, done = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record(cur)
+        for ln in lanes:
+            ln["stream"].wait_event(start)
+        for k in range(n):
+            step_host(k)
+        for ln in lanes:
+            ev = torch.cuda.Event()
+            ev.record(ln["stream"])
+            cur.wait_event(ev)
+        done.record(cur)
+        torch.cuda.synchronize()
+        return start.elapsed_time(done)
+
+    n_e2e = max(4, min(args.steps, 20 if args.workload != 4 else 3))
+    run_host(2 * n_lanes)
     barrier()
-    e_a.record()
-    for _ in range(n_e2e):
-        step_host()
-    e_b.record()
-    torch.cuda.synchronize()
+    ms_e2e = max_over_ranks(run_host(n_e2e) / n_e2e, device, world)
     barrier()
-    ms_e2e = max_over_ranks(e_a.elapsed_time(e_b) / n_e2e, device, world)
-    h2d = sum(t.numel() * t.element_size() for h, _ in h_sets for t in h.values())
-    d2h = sum(t.numel() * t.element_size() for _, ho in h_sets for t in ho.values())
+    h2d = sum(t.numel() * t.element_size() for h in h_in for t in h.values())
+    d2h = sum(t.numel() * t.element_size() for ho in lanes[0]["out"] for t in ho.values())
     e2e = {"value": job_value(world, flops_step, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-           "ms_per_step": ms_e2e, "steps": n_e2e,
-           "note": "host X, A, B, dY in; Y, dX, dA, dB out (pinned); frozen W resident on the device"}
+           "ms_per_step": ms_e2e, "steps": n_e2e, "lanes": n_lanes,
+           "pcie_gbs": {"h2d": h2d / ms_e2e / 1e6, "d2h": d2h / ms_e2e / 1e6},
+           "note": "host X, A, B, dY in; Y, dX, dA, dB out (pinned); frozen W resident on the device; "
+                   f"{n_lanes} lane(s) of lora_linear_step_host alternate so that copies of neighbouring steps overlap"}
 
     if rank != 0:
         return

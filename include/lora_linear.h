@@ -142,10 +142,14 @@ int lora_linear_bwd_saved_p(lora_plan_t* plan, const void* dY, const void* X, co
 /* The three stages of lora_linear_bwd as separate calls, for callers that schedule them themselves.
  * They communicate through the plan's workspace and must run in this order on one stream (or with
  * equivalent event dependencies):
+ *   lora_linear_bwd_q    optional: only the skinny pre-pass scale (dY B)^T -> workspace (streams dY once).  The next
+ *                        lora_linear_bwd_dx on the plan (same dY, B, scale) then launches the GEMM alone.  A no-op for
+ *                        plans with T <= 128, whose dX kernel computes dY B itself.
  *   lora_linear_bwd_dx   dX = dY W + scale (dY B) A ; leaves scale (dY B)^T in the workspace
  *   lora_linear_bwd_da   dA = scale (dY B)^T X, streams X once ; leaves scale (X A^T)^T in the workspace
  *   lora_linear_bwd_db   dB = scale dY^T (X A^T), streams dY once
  * `scale` must be the same in all three. */
+int lora_linear_bwd_q(lora_plan_t* plan, const void* dY, const void* B, float scale, void* stream);
 int lora_linear_bwd_dx(lora_plan_t* plan, const void* dY, const void* W, const void* A, const void* B,
                        float scale, void* dX, void* stream);
 int lora_linear_bwd_da(lora_plan_t* plan, const void* X, const void* A, float scale, void* dA, void* stream);

@@ -26,7 +26,7 @@ LORA_ERR_NO_DEVICE = -7
 EXPORTS = [
     "lora_select_config", "lora_workspace_bytes", "lora_plan_create", "lora_plan_destroy",
     "lora_plan_workspace_bytes", "lora_plan_set_workspace", "lora_plan_get_config", "lora_plan_describe",
-    "lora_linear_fwd", "lora_linear_bwd", "lora_linear_bwd_saved_p", "lora_linear_bwd_dx", "lora_linear_bwd_da", "lora_linear_bwd_db",
+    "lora_linear_fwd", "lora_linear_bwd", "lora_linear_bwd_saved_p", "lora_linear_bwd_q", "lora_linear_bwd_dx", "lora_linear_bwd_da", "lora_linear_bwd_db",
     "lora_dense_dw", "lora_nf4_quantize", "lora_nf4_dequantize", "lora_linear_fwd_nf4", "lora_linear_bwd_nf4", "lora_step_host_staging_bytes", "lora_linear_step_host",
     "lora_last_device_status", "lora_strerror", "lora_launch_count",
     "lora_grad_contract_noalloc", "lora_grad_contract_noalloc_max_scratch",
@@ -76,6 +76,7 @@ def load(rebuild: bool = False) -> ctypes.CDLL:
     lib.lora_linear_fwd.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp]
     lib.lora_linear_bwd.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
     lib.lora_linear_bwd_saved_p.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
+    lib.lora_linear_bwd_q.argtypes = [vp, vp, vp, ctypes.c_float, vp]
     lib.lora_linear_bwd_dx.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp]
     lib.lora_linear_bwd_da.argtypes = [vp, vp, vp, ctypes.c_float, vp, vp]
     lib.lora_linear_bwd_db.argtypes = [vp, vp, ctypes.c_float, vp, vp]
@@ -315,12 +316,16 @@ class LoraLinearPlan:
         return dW
 
     def bwd_stages(self, dY, X, W, A, B, scale: float, dX, dA, dB, stream=None, events=None):
-        """The same three kernels as ``bwd``, issued through the stage entry points; ``events`` (four
-        torch.cuda.Event, optional) are recorded before, between and after them on the stream."""
+        """The same kernels as ``bwd``, issued through the stage entry points; ``events`` (five torch.cuda.Event,
+        optional) are recorded on the stream: before the dY B pre-pass, then after the pre-pass (so that events 1 and 2
+        bracket exactly the dX GEMM launch), after the dX GEMM, after the dA stage and after the dB stage."""
         self.ensure_workspace()
         sp = _stream_ptr(stream)
         st = stream if stream is not None else torch.cuda.current_stream()
         if events is not None:
+            events[0].record(st)
+            _check(self._lib.lora_linear_bwd_q(self._h, _ptr(dY), _ptr(B), float(scale), sp), "lora_linear_bwd_q")
+            events = events[1:]
             events[0].record(st)
         _check(self._lib.lora_linear_bwd_dx(self._h, _ptr(dY), _ptr(W), _ptr(A), _ptr(B), float(scale), _ptr(dX), sp),
                "lora_linear_bwd_dx")

@@ -135,8 +135,12 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
     // Forward, fused vs K-extended.  Fused adapter columns cost r_pad / 256 of every MMA (time ~ T d_in d_out r_pad);
     // the alternative is a skinny X A^T pre-pass (time ~ T d_in, one more read of X) and 256-wide tiles.  Their ratio
     // is ~1e-5 d_out r_pad at the measured rates (1.2 PFLOP/s GEMM, 3 TB/s pre-pass), so the pre-pass wins for wide
-    // outputs or large ranks: 14336 x 16 and 4096 x 64 take it, 4096 x 16 and 1024 x 16 stay fused.
-    c->fwd_ext = (static_cast<long long>(s->d_out) * c->r_pad >= 100000) ? 1 : 0;
+    // outputs or large ranks.  Measured break-even: 4096 x 16 (fused 0.984 ms vs 0.926 ms K-extended at T = 32768 under
+    // the power cap, where the wasted adapter columns also cost clock; 0.473 vs 0.456 ms per step at T = 8192), while
+    // 1024 x 16 is faster fused (0.280 vs 0.291 ms): 14336 x 16, 4096 x 64 and 4096 x 16 take the pre-pass.
+    // (between 65536 and 1e5 only from 4096 tokens on: below that the two extra launches weigh more than the columns)
+    const long long dr = static_cast<long long>(s->d_out) * c->r_pad;
+    c->fwd_ext = (dr >= 100000 || (dr >= 65536 && T >= 4096)) ? 1 : 0;
     if (const char* f = std::getenv("LORA_FORCE_FWD_EXT")) c->fwd_ext = std::atoi(f) != 0 ? 1 : 0;
     // Split along K: when the tiling leaves at least three quarters of the CTA pairs idle and the contraction is long
     // (>= 64 k-blocks), each tile is cut into k-ranges handled by different pairs (fp32 partial tiles, fixed-order
@@ -337,6 +341,7 @@ struct lora_plan {
   void* workspace;
   size_t workspace_bytes;
   bool q_ready;          // set while lora_linear_bwd_saved_p runs: Qt was already produced by its dB kernel
+  bool q_staged;         // lora_linear_bwd_q ran: the next lora_linear_bwd_dx skips its own pre-pass
   bool p_saved;          // the workspace holds Pt = s (X A^T)^T of the last forward call
   float p_saved_scale;
 };
@@ -810,6 +815,7 @@ int lora_plan_create(const lora_shape_t* shape, int device, lora_plan_t** out) {
   pl->workspace = nullptr;
   pl->workspace_bytes = 0;
   pl->q_ready = false;
+  pl->q_staged = false;
   pl->p_saved = false;
   pl->p_saved_scale = 0.f;
   pl->d_status = nullptr;
@@ -932,6 +938,18 @@ int lora_linear_bwd_saved_p(lora_plan_t* plan, const void* dY, const void* X, co
   return rc;
 }
 
+int lora_linear_bwd_q(lora_plan_t* plan, const void* dY, const void* B, float scale, void* stream) {
+  if (plan == nullptr) return LORA_ERR_INVALID_ARG;
+  if (plan->shape.T == 0 || plan->cfg.cta_group != 2) return LORA_OK;   // small batches: the dX kernel computes dY B itself
+  if (!dY || !B) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(dY) || !aligned16(B)) return LORA_ERR_MISALIGNED;
+  if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
+  DeviceGuard guard(plan->device);
+  const int rc = launch_side_prepass(plan, dY, plan->shape.d_out, B, true, scale, ws_ptrs(plan).qt, static_cast<cudaStream_t>(stream));
+  if (rc == LORA_OK) plan->q_staged = true;
+  return rc;
+}
+
 int lora_linear_bwd_dx(lora_plan_t* plan, const void* dY, const void* W, const void* A, const void* B, float scale,
                        void* dX, void* stream) {
   if (plan == nullptr) return LORA_ERR_INVALID_ARG;
@@ -940,7 +958,11 @@ int lora_linear_bwd_dx(lora_plan_t* plan, const void* dY, const void* W, const v
   if (!aligned16(dY) || !aligned16(W) || !aligned16(A) || !aligned16(B) || !aligned16(dX)) return LORA_ERR_MISALIGNED;
   if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
   DeviceGuard guard(plan->device);
-  return launch_dx(plan, dY, W, A, B, scale, dX, static_cast<cudaStream_t>(stream));
+  plan->q_ready = plan->q_staged;          // lora_linear_bwd_q already left s (dY B)^T in the workspace
+  plan->q_staged = false;
+  const int rc = launch_dx(plan, dY, W, A, B, scale, dX, static_cast<cudaStream_t>(stream));
+  plan->q_ready = false;
+  return rc;
 }
 
 int lora_linear_bwd_da(lora_plan_t* plan, const void* X, const void* A, float scale, void* dA, void* stream) {

@@ -43,7 +43,8 @@ def test_selector_invariants(shape):
     assert c["cta_group"] == (2 if T > 128 else 1)
     if c["cta_group"] == 2:
         assert c["block_m"] == 256
-        assert c["fwd_ext"] == (1 if d_out * c["r_pad"] >= 100000 else 0)
+        dr = d_out * c["r_pad"]
+        assert c["fwd_ext"] == (1 if dr >= 100000 or (dr >= 65536 and T >= 4096) else 0)
         # fused forward: tile + adapter columns share one MMA; K-extended forward: no adapter columns
         assert c["fwd_block_n"] % 16 == 0 and c["fwd_block_n"] + (0 if c["fwd_ext"] else c["r_pad"]) <= 256
         assert c["dx_block_n"] % 16 == 0 and c["dx_block_n"] <= 256                  # K-extended GEMM: no adapter columns
@@ -85,7 +86,9 @@ def test_selector_picks_by_grid_size():
     assert small["cta_group"] == 1 and small["fwd_block_n"] == 64 and small["fwd_ctas"] == 8
     assert big["cta_group"] == 2 and big["fwd_ext"] == 1 and big["fwd_block_n"] == 256 and big["fwd_ctas"] == 148
     q = binding.select_config(8192, 4096, 4096, 16, 148)
-    assert q["fwd_ext"] == 0 and q["fwd_block_n"] == 240 and q["dx_block_n"] == 256
+    assert q["fwd_ext"] == 1 and q["fwd_block_n"] == 256 and q["dx_block_n"] == 256      # pre-pass beats adapter columns
+    q_small = binding.select_config(1024, 4096, 4096, 16, 148)                            # few tokens: stay fused
+    assert q_small["fwd_ext"] == 0 and q_small["fwd_block_n"] == 240
     kv = binding.select_config(32768, 4096, 1024, 16, 148)        # 1024 columns: 5 x 208 wastes less than 5 x 240
     assert kv["fwd_block_n"] == 208
 
