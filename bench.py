@@ -309,8 +309,10 @@ def run_ours(args):
             if ev is not None:
                 ev[0].record()
             plans[j].fwd(d["X"], d["W"], d["A"], d["B"], proj.scale, d["Y"])
-            plans[j].bwd_stages(d["dY"], d["X"], d["W"], d["A"], d["B"], proj.scale, d["dX"], d["dA"], d["dB"],
-                                events=ev[1:] if ev is not None else None)
+            if ev is None:       # the product path: lora_linear_bwd (dX GEMM beside the dA / dB passes where the plan says so)
+                plans[j].bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], proj.scale, d["dX"], d["dA"], d["dB"])
+            else:                # the same kernels one after the other through the stage calls, with events between them
+                plans[j].bwd_stages(d["dY"], d["X"], d["W"], d["A"], d["B"], proj.scale, d["dX"], d["dA"], d["dB"], events=ev[1:])
 
     def barrier():
         if world > 1:

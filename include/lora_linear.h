@@ -89,6 +89,10 @@ typedef struct lora_kernel_config {
   int32_t q_stages;
   int32_t dx_split_k;      /* k-splits per tile of the dX GEMM                                           */
   int32_t fwd_ext;         /* 1: forward runs as X A^T pre-pass + K-extended GEMM (needs the workspace)  */
+  int32_t overlap_sms;     /* lora_linear_bwd: SMs left to the dA / dB passes, which run beside the dX GEMM on a    */
+  int32_t ov_dx_ctas;      /*   second stream (0: serial order); persistent CTAs of the dX GEMM and token chunks of */
+  int32_t ov_da_token_chunks; /* the two passes in that mode                                                        */
+  int32_t ov_db_token_chunks;
   int32_t dw_block_n;      /* dense weight gradient GEMM (lora_dense_dw): d_in columns per tile,         */
   int32_t dw_split_k;      /*   splits along the tokens, persistent CTAs                                 */
   int32_t dw_ctas;
@@ -126,7 +130,14 @@ int lora_linear_fwd(lora_plan_t* plan, const void* X, const void* W, const void*
 
 /* Backward:  dX = dY W + scale (dY B) A,  dA = scale (dY B)^T X,  dB = scale dY^T (X A^T).
  * Does not depend on a preceding forward call (X A^T is recomputed).  Needs the workspace.
- * dA and dB are fp32 and are overwritten. */
+ * dA and dB are fp32 and are overwritten.
+ * Where cfg.overlap_sms > 0 (opt-in: environment variable LORA_OVERLAP_SMS = number of SMs to leave free, read when the
+ * plan is created; off by default because it measured no reliable gain), the tensor-bound dX GEMM and the two HBM-bound
+ * adapter-gradient passes run at the same time: the GEMM on `stream` with a few SMs fewer, the passes on a second,
+ * plan-owned stream that is forked from and joined back into `stream` by events inside this call.  For the caller the
+ * call still behaves as one piece of work on `stream`; results are bit-identical to the serial order of the stage calls
+ * below except for the grid-dependent order of the fp32 partial sums of dA and dB, which stays fixed for a given plan.
+ * (Such a plan owns one extra stream and two events besides its status block.) */
 int lora_linear_bwd(lora_plan_t* plan, const void* dY, const void* X, const void* W, const void* A,
                     const void* B, float scale, void* dX, void* dA, void* dB, void* stream);
 

@@ -41,7 +41,8 @@ class LoraKernelConfig(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "block_m", "fwd_block_n", "dx_block_n", "block_k", "stages", "group_m", "split_k", "r_pad", "fwd_ctas",
         "dx_ctas", "tail_delay", "grad_feat_chunk", "grad_stages", "da_feat_chunks", "da_token_chunks",
-        "db_feat_chunks", "db_token_chunks", "db_feat_chunk", "cta_group", "dx_stages", "prefetch_dist", "db_stages", "q_feat_chunk", "q_feat_chunks", "q_token_chunks", "q_stages", "dx_split_k", "fwd_ext", "dw_block_n", "dw_split_k", "dw_ctas")]
+        "db_feat_chunks", "db_token_chunks", "db_feat_chunk", "cta_group", "dx_stages", "prefetch_dist", "db_stages", "q_feat_chunk", "q_feat_chunks", "q_token_chunks", "q_stages", "dx_split_k", "fwd_ext", "overlap_sms", "ov_dx_ctas", "ov_da_token_chunks", "ov_db_token_chunks",
+        "dw_block_n", "dw_split_k", "dw_ctas")]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}

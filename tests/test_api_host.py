@@ -80,6 +80,24 @@ def test_selector_invariants(shape):
     assert c["db_feat_chunks"] == -(-d_out // c["db_feat_chunk"])
 
 
+@pytest.mark.parametrize("shape,can", [((8192, 4096, 4096, 16), True), ((16384, 14336, 4096, 64), True),
+                                       ((256, 512, 512, 8), False), ((128, 4096, 4096, 16), False)])
+def test_selector_overlapped_backward_is_opt_in(shape, can, monkeypatch):
+    """The dA / dB passes run beside the dX GEMM only when LORA_OVERLAP_SMS asks for it (measured: no reliable gain),
+    and only on grids with at least one tile per CTA pair."""
+    T, d_in, d_out, r = shape
+    monkeypatch.delenv("LORA_OVERLAP_SMS", raising=False)
+    c = binding.select_config(T, d_in, d_out, r, 148)
+    assert c["overlap_sms"] == 0 and c["ov_dx_ctas"] == c["dx_ctas"] and c["ov_da_token_chunks"] == c["da_token_chunks"]
+    monkeypatch.setenv("LORA_OVERLAP_SMS", "16")
+    c = binding.select_config(T, d_in, d_out, r, 148)
+    assert (c["overlap_sms"] == 16) == can
+    if can:
+        assert c["ov_dx_ctas"] == 2 * (74 - 8)
+        assert 1 <= c["ov_da_token_chunks"] <= c["da_token_chunks"] and 1 <= c["ov_db_token_chunks"] <= c["db_token_chunks"]
+        assert c["da_feat_chunks"] * c["ov_da_token_chunks"] <= max(16, c["da_feat_chunks"])
+
+
 def test_selector_picks_by_grid_size():
     small = binding.select_config(128, 512, 512, 8, 148)          # one 128-row tile: single-CTA kernel, narrow tiles
     big = binding.select_config(16384, 4096, 14336, 16, 148)
