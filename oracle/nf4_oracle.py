@@ -5,7 +5,7 @@ code, table or constant generator with the CUDA library.
 
 Section 4.5 ("Quantised LoRA", Q+LoRA) trains the same LoRA layer with the frozen W held in
 NF4 (Dettmers et al. 2023, QLoRA: 4-bit NormalFloat with block-wise absmax scaling).  The
-paper fixes no storage format, so this build defines one (the kernels follow the same
+paper fixes no storage format, so this library defines one (the kernels follow the same
 written rules, in code of their own):
 
   * W [d_out, d_in] is cut into blocks of 64 consecutive elements along d_in (d_in % 64 == 0).

@@ -233,7 +233,7 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
   // and the two HBM-bound adapter-gradient passes run on them at the same time on a second stream.  Measured (ms per
   // step, serial vs overlapped, same run): 8192 x 4096 x 4096 0.442 / 0.426 (R = 16), 0.437 (R = 24), 0.530 (R = 8: the
   // passes reach only ~40 GB/s per SM and outlast the GEMM); 16384 x 4096 x 14336 2.909 / 2.907; 16384 x 14336 x 4096
-  // r = 64 3.055 / 3.159.  A gain within the box-to-box noise on the short step and none or a loss under the power cap
+  // r = 64 3.055 / 3.159.  A gain within the run-to-run spread on the short step and none or a loss under the power cap
   // of the long ones, so the default stays the serial order.
   c->overlap_sms = 0;
   c->ov_dx_ctas = c->dx_ctas;
