@@ -87,7 +87,7 @@ class Projection:
 
 
 def workload(idx: int, T: Optional[int] = None) -> List[Projection]:
-    """The five benchmark workloads; ``T`` overrides the token count (for reduced cases)."""
+    """The five benchmark workloads, plus (5) the paper's own q/k/v/o, r = 32 setting; ``T`` overrides the token count."""
     if idx == 0:
         return [Projection("tiny", T or 256, 512, 512, 8, 2.0)]
     if idx == 1:
@@ -106,6 +106,16 @@ def workload(idx: int, T: Optional[int] = None) -> List[Projection]:
             Projection("gate_proj", t, 4096, 14336, 16, 2.0, x_group=2),
             Projection("up_proj", t, 4096, 14336, 16, 2.0, x_group=2),
             Projection("down_proj", t, 14336, 4096, 16, 2.0, x_group=3),
+        ]
+    if idx == 5:
+        # the paper's own adapter setting (Section 4.5: q, k, v, o adapted, lora_r = 32, alpha = 64, i.e. scale 2) on its
+        # Llama-3.1-8B batch shape (throughput table: 6 sequences of 8k tokens per GPU = 49152 packed tokens)
+        t = T or 49152
+        return [
+            Projection("q_proj", t, 4096, 4096, 32, 2.0, x_group=0),
+            Projection("k_proj", t, 4096, 1024, 32, 2.0, x_group=0),
+            Projection("v_proj", t, 4096, 1024, 32, 2.0, x_group=0),
+            Projection("o_proj", t, 4096, 4096, 32, 2.0, x_group=1),
         ]
     raise ValueError(f"unknown workload {idx}")
 
@@ -130,6 +140,9 @@ def cu_seqlens(idx: int, T: int, seed: int = 0) -> np.ndarray:
         lens = packed_lengths(T, seed)
     elif idx == 1:
         lens = np.full(4, T // 4, dtype=np.int64)
+        lens[-1] += T - int(lens.sum())
+    elif idx == 5:
+        lens = np.full(6, T // 6, dtype=np.int64)
         lens[-1] += T - int(lens.sum())
     else:
         lens = np.asarray([T], dtype=np.int64)

@@ -63,3 +63,15 @@ def test_packed_lengths_cover_the_batch():
 def test_flop_count_formula():
     p = inputs.workload(1)[0]
     assert p.flops == 4 * 8192 * 4096 * 4096 + 6 * 8192 * 16 * 8192
+
+
+def test_paper_setting_workload():
+    ps = inputs.workload(5)
+    assert [p.name for p in ps] == ["q_proj", "k_proj", "v_proj", "o_proj"]
+    assert all(p.T == 49152 and p.r == 32 and p.scale == 2.0 and p.d_in == 4096 for p in ps)
+    assert [p.d_out for p in ps] == [4096, 1024, 1024, 4096]
+    assert ps[0].x_group == ps[1].x_group == ps[2].x_group != ps[3].x_group
+    cs = inputs.cu_seqlens(5, 49152)
+    assert cs[0] == 0 and cs[-1] == 49152 and len(cs) == 7 and np.all(np.diff(cs) == 8192)
+    small = list(inputs.draw_workload(5, seed=0, T=64))
+    assert len(small) == 4 and small[1][1]["X"] is small[0][1]["X"] or np.array_equal(small[1][1]["X"], small[0][1]["X"])

@@ -162,3 +162,15 @@ def test_nf4_full_size_config1(use_scratch):
     del d, Y, dX, dA, dB
     gc.collect()
     torch.cuda.empty_cache()
+
+
+def test_paper_adapter_setting_full_size():
+    """The paper's own setting (Section 4.5: q/k/v/o adapters, lora_r = 32, alpha = 64) at its batch shape, 6 x 8k = 49152
+    packed tokens: the 4096-wide q projection and the 1024-wide k projection (v and o repeat their shapes)."""
+    x_dev = None
+    for p, t in inputs.draw_workload(5, seed=0):
+        if p.name not in ("q_proj", "k_proj"):
+            break
+        if x_dev is None:
+            x_dev = dev(t["X"])
+        check_projection(p, t, x_dev)
