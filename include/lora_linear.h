@@ -154,8 +154,9 @@ int lora_linear_bwd_saved_p(lora_plan_t* plan, const void* dY, const void* X, co
  * They communicate through the plan's workspace and must run in this order on one stream (or with
  * equivalent event dependencies):
  *   lora_linear_bwd_q    optional: only the skinny pre-pass scale (dY B)^T -> workspace (streams dY once).  The next
- *                        lora_linear_bwd_dx on the plan (same dY, B, scale) then launches the GEMM alone.  A no-op for
- *                        plans with T <= 128, whose dX kernel computes dY B itself.
+ *                        lora_linear_bwd_dx on the plan (same dY, B, scale) then launches the GEMM alone; any other
+ *                        backward call on the plan in between discards the staged product.  A no-op for plans with
+ *                        T <= 128, whose dX kernel computes dY B itself.
  *   lora_linear_bwd_dx   dX = dY W + scale (dY B) A ; leaves scale (dY B)^T in the workspace
  *   lora_linear_bwd_da   dA = scale (dY B)^T X, streams X once ; leaves scale (X A^T)^T in the workspace
  *   lora_linear_bwd_db   dB = scale dY^T (X A^T), streams dY once

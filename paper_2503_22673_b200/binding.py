@@ -316,6 +316,18 @@ class LoraLinearPlan:
         _check(self._lib.lora_dense_dw(self._h, _ptr(dY), _ptr(X), _ptr(dW), _stream_ptr(stream)), "lora_dense_dw")
         return dW
 
+    def bwd_q(self, dY, B, scale: float, stream=None) -> None:
+        """Stage scale (dY B)^T in the workspace; the next ``bwd_dx`` then launches the dX GEMM alone."""
+        self.ensure_workspace()
+        _check(self._lib.lora_linear_bwd_q(self._h, _ptr(dY), _ptr(B), float(scale), _stream_ptr(stream)), "lora_linear_bwd_q")
+
+    def bwd_dx(self, dY, W, A, B, scale: float, dX, stream=None):
+        """dX = dY W + scale (dY B) A alone (first stage of the backward pass)."""
+        self.ensure_workspace()
+        _check(self._lib.lora_linear_bwd_dx(self._h, _ptr(dY), _ptr(W), _ptr(A), _ptr(B), float(scale), _ptr(dX),
+                                            _stream_ptr(stream)), "lora_linear_bwd_dx")
+        return dX
+
     def bwd_stages(self, dY, X, W, A, B, scale: float, dX, dA, dB, stream=None, events=None):
         """The same kernels as ``bwd``, issued through the stage entry points; ``events`` (five torch.cuda.Event,
         optional) are recorded on the stream: before the dY B pre-pass, then after the pre-pass (so that events 1 and 2

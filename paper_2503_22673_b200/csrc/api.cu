@@ -907,6 +907,7 @@ int lora_plan_set_workspace(lora_plan_t* plan, void* dev_ptr, size_t bytes) {
   plan->workspace = dev_ptr;
   plan->workspace_bytes = bytes;
   plan->p_saved = false;
+  plan->q_staged = false;
   return LORA_OK;
 }
 
@@ -959,6 +960,7 @@ int lora_linear_bwd(lora_plan_t* plan, const void* dY, const void* X, const void
   if (!aligned16(dY) || !aligned16(X) || !aligned16(W) || !aligned16(A) || !aligned16(B) || !aligned16(dX))
     return LORA_ERR_MISALIGNED;
   if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
+  plan->q_staged = false;      // this call overwrites the staged s (dY B)^T
   if (plan->cfg.overlap_sms > 0) {
     // dY B pre-pass, then the dX GEMM on `stream` beside dA -> dB on the plan's second stream (fork / join by events)
     const lora_kernel_config_t& c = plan->cfg;
@@ -993,6 +995,7 @@ int lora_linear_bwd_saved_p(lora_plan_t* plan, const void* dY, const void* X, co
     return LORA_ERR_MISALIGNED;
   if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
   if (!plan->p_saved || plan->p_saved_scale != scale) return LORA_ERR_INVALID_ARG;   // no forward result to reuse
+  plan->q_staged = false;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   DeviceGuard guard(plan->device);
   int rc = launch_db(plan, dY, scale, dB, st, B);          // dB from the saved Pt; leaves Qt
@@ -1127,6 +1130,7 @@ int lora_linear_bwd_nf4(lora_plan_t* plan, const void* dY, const void* X, const 
   if (!aligned16(dY) || !aligned16(X) || !aligned16(W_codes) || !aligned16(W_absmax) || !aligned16(A) || !aligned16(B) ||
       !aligned16(dX) || !aligned16(w_scratch))
     return LORA_ERR_MISALIGNED;
+  plan->q_staged = false;
   if (plan->shape.d_in % kNf4Block != 0 || plan->shape.d_out % 4 != 0) return LORA_ERR_UNSUPPORTED_SHAPE;
   if (w_scratch != nullptr) {
     if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;

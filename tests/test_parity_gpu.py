@@ -357,3 +357,24 @@ def test_overlapped_backward_matches_the_stage_calls(monkeypatch):
     assert oracle.rel_err(host64(outs[0][1]), dA) <= TOL_F32 and oracle.rel_err(host64(outs[0][2]), dB) <= TOL_F32
     assert oracle.rel_err(host64(outs[0][1]), host64(dA_s)) <= 1e-5 and oracle.rel_err(host64(outs[0][2]), host64(dB_s)) <= 1e-5
     plan.close()
+
+
+def test_staged_pre_pass_is_used_once_and_discarded_by_other_calls():
+    """lora_linear_bwd_q stages s (dY B)^T for the NEXT lora_linear_bwd_dx only: with the matching dY the staged GEMM gives
+    the same bits as the unstaged call, and a full backward in between (other dY) makes a later bwd_dx run its own pre-pass."""
+    p, t = inputs.draw_custom(520, 264, 776, 16, 2.0, seed=21)
+    _, t2 = inputs.draw_custom(520, 264, 776, 16, 2.0, seed=22)
+    d = {k: dev(v) for k, v in t.items()}
+    dY2 = dev(t2["dY"])
+    plan = binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r)
+    ref = plan.bwd_dx(d["dY"], d["W"], d["A"], d["B"], p.scale, torch.empty_like(d["X"])).clone()
+    plan.bwd_q(d["dY"], d["B"], p.scale)
+    staged = plan.bwd_dx(d["dY"], d["W"], d["A"], d["B"], p.scale, torch.empty_like(d["X"]))
+    assert torch.equal(staged, ref)
+    plan.bwd_q(dY2, d["B"], p.scale)                                   # staged for dY2 ...
+    plan.bwd(dY2, d["X"], d["W"], d["A"], d["B"], p.scale)             # ... but a full backward comes first
+    again = plan.bwd_dx(d["dY"], d["W"], d["A"], d["B"], p.scale, torch.empty_like(d["X"]))
+    assert torch.equal(again, ref)
+    code, msg = plan.device_status()
+    assert code == 0, msg
+    plan.close()
