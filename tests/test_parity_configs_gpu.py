@@ -174,3 +174,54 @@ def test_paper_adapter_setting_full_size():
         if x_dev is None:
             x_dev = dev(t["X"])
         check_projection(p, t, x_dev)
+
+
+def test_more_than_2_31_elements_per_tensor():
+    """Index arithmetic beyond 32 bits: X and dX hold 540000 x 4096 = 2.2e9 elements (4.4 GB each).  The oracle cannot hold
+    such a matrix in float64, so: sampled rows of Y and dX (first, last, around the 2^31-element boundary, random) against
+    the oracle row by row; dA and dB against the sum of the layer's own results on the two halves of the token range
+    (additivity over token rows, each half below 2^31 elements) and the adjoint identity <dA, A> = <dB, B>."""
+    T, d_in, d_out, r, scale = 540000, 4096, 520, 16, 2.0
+    g = torch.Generator(device="cuda").manual_seed(7)
+    X = torch.randn((T, d_in), device="cuda", generator=g, dtype=torch.float32).to(torch.bfloat16)
+    dY = torch.randn((T, d_out), device="cuda", generator=g, dtype=torch.float32).to(torch.bfloat16)
+    W = (torch.randn((d_out, d_in), device="cuda", generator=g) / 64).to(torch.bfloat16)
+    A = (torch.randn((r, d_in), device="cuda", generator=g) / 64).to(torch.bfloat16)
+    B = (torch.randn((d_out, r), device="cuda", generator=g) * 0.14).to(torch.bfloat16)
+    plan = binding.LoraLinearPlan(T, d_in, d_out, r)
+    Y = plan.fwd(X, W, A, B, scale)
+    dX, dA, dB = plan.bwd(dY, X, W, A, B, scale)
+    code, msg = plan.device_status()
+    assert code == 0, msg
+    plan.close()
+    edge = (1 << 31) // d_in                                            # first row past 2^31 elements of X
+    rows = np.unique(np.concatenate([sample_rows(T, 24, seed=3), [edge - 129, edge - 1, edge, edge + 1, edge + 127, edge + 128]]))
+    rt = torch.from_numpy(rows).cuda()
+    Wf, Af, Bf = host64(W), host64(A), host64(B)
+    Yr = oracle.forward(host64(X[rt]), Wf, Af, Bf, scale)
+    dXr = oracle.backward_dx_rows(np.arange(len(rows)), host64(dY[rt]), Wf, Af, Bf, scale)
+    assert oracle.rel_err(host64(Y[rt]), Yr) <= TOL_BF16
+    assert oracle.rel_err(host64(dX[rt]), dXr) <= TOL_BF16
+    half = 270080                                                       # a multiple of 128: both halves below 2^31 elements
+    dA_sum = torch.zeros_like(dA, dtype=torch.float64)
+    dB_sum = torch.zeros_like(dB, dtype=torch.float64)
+    for lo, hi in ((0, half), (half, T)):
+        ph = binding.LoraLinearPlan(hi - lo, d_in, d_out, r)
+        _, dA_h, dB_h = ph.bwd(dY[lo:hi], X[lo:hi], W, A, B, scale)
+        dA_sum += dA_h.double()
+        dB_sum += dB_h.double()
+        ph.close()
+    assert oracle.rel_err(host64(dA), dA_sum.cpu().numpy()) <= 1e-4
+    assert oracle.rel_err(host64(dB), dB_sum.cpu().numpy()) <= 1e-4
+    # the halves themselves against the oracle on a slab it can hold: the first 8192 tokens
+    ps = binding.LoraLinearPlan(8192, d_in, d_out, r)
+    _, dA_s, dB_s = ps.bwd(dY[:8192], X[:8192], W, A, B, scale)
+    dAr, dBr = oracle.backward_adapter_grads(host64(dY[:8192]), host64(X[:8192]), Af, Bf, scale)
+    assert oracle.rel_err(host64(dA_s), dAr) <= TOL_F32 and oracle.rel_err(host64(dB_s), dBr) <= TOL_F32
+    ps.close()
+    a, b = dot64(dA, A), dot64(dB, B)
+    scale_ab = (dA.double().norm() * A.double().norm() + dB.double().norm() * B.double().norm()).item()
+    assert abs(a - b) / scale_ab <= 5e-3
+    del X, dY, Y, dX
+    gc.collect()
+    torch.cuda.empty_cache()
