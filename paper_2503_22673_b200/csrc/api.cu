@@ -335,8 +335,37 @@ EncodeTiledFn encode_fn() {
 }
 
 // 2-D row-major tensor of `elem_bytes`-wide elements, 128-byte swizzle, zero fill outside the tensor.
+// A tensor map is a pure function of (address, shape, pitch, box, type, swizzle), so encoded maps are kept in a small
+// per-thread table: a step of the layer re-encodes the same ~40 maps every time, and on launch-bound shapes (a few
+// hundred tokens) the driver's encode calls were the larger part of the host time per launch.
+struct TmapKey {
+  const void* ptr;
+  uint64_t inner, outer, pitch;
+  uint32_t box_inner, box_outer, dt, swz;
+  bool operator==(const TmapKey& o) const {
+    return ptr == o.ptr && inner == o.inner && outer == o.outer && pitch == o.pitch && box_inner == o.box_inner &&
+           box_outer == o.box_outer && dt == o.dt && swz == o.swz;
+  }
+};
+struct TmapSlot {
+  bool used = false;
+  TmapKey key;
+  CUtensorMap map;
+};
+constexpr int kTmapCacheSlots = 512;        // direct-mapped; a colliding entry is simply re-encoded
+
 bool make_tmap(CUtensorMap* m, const void* ptr, CUtensorMapDataType dt, int elem_bytes, uint64_t inner, uint64_t outer,
                uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_outer, bool swizzle128 = true) {
+  static thread_local TmapSlot cache[kTmapCacheSlots];
+  const TmapKey key{ptr, inner, outer, pitch_bytes, box_inner, box_outer, static_cast<uint32_t>(dt), swizzle128 ? 1u : 0u};
+  uint64_t h = reinterpret_cast<uintptr_t>(ptr) * 0x9E3779B97F4A7C15ull;
+  h ^= (inner * 0xC2B2AE3D27D4EB4Full) ^ (outer * 0x165667B19E3779F9ull) ^ (static_cast<uint64_t>(box_inner) << 40) ^
+       (static_cast<uint64_t>(box_outer) << 20) ^ (pitch_bytes << 7) ^ key.dt ^ (key.swz << 5);
+  TmapSlot& slot = cache[(h >> 32) % kTmapCacheSlots];
+  if (slot.used && slot.key == key) {
+    *m = slot.map;
+    return true;
+  }
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
   const cuuint64_t dims[2] = {inner, outer};
@@ -348,7 +377,11 @@ bool make_tmap(CUtensorMap* m, const void* ptr, CUtensorMapDataType dt, int elem
                         swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
+  if (r != CUDA_SUCCESS) return false;
+  slot.used = true;
+  slot.key = key;
+  slot.map = *m;
+  return true;
 }
 
 bool make_bf16_tmap(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t outer, uint64_t pitch_elems,
