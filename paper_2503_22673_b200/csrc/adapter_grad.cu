@@ -207,10 +207,17 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
           uint32_t v[16];
           tmem_ld16(tmem_p + lane_addr + pb * p.r_pad + c16 * 16, v);
           tmem_ld_wait();
-          if (t < p.T) {
+          if (t < p.T && !p.direct) {
 #pragma unroll
             for (int q = 0; q < 16; ++q)
               p.p_part[(static_cast<size_t>(fc) * p.r_pad + c16 * 16 + q) * p.ld_t + t] = __uint_as_float(v[q]);
+          } else if (t < p.T) {
+            // this CTA holds every feature: the side product is complete, write bf16(scale * .) straight to its place
+            unsigned short* pt = reinterpret_cast<unsigned short*>(p.pt_out);
+#pragma unroll
+            for (int q = 0; q < 16; ++q)
+              pt[static_cast<size_t>(c16 * 16 + q) * p.ld_t + t] =
+                  static_cast<unsigned short>(pack_bf16x2(__uint_as_float(v[q]) * p.scale, 0.f) & 0xFFFFu);
           }
         }
         tc_fence_before();
@@ -229,10 +236,20 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
             uint32_t v[16];
             tmem_ld16(tmem_base + lane_addr + nb * p.r_pad + c16 * 16, v);
             tmem_ld_wait();
-            if (c < p.C) {
+            if (c < p.C && !p.direct) {
 #pragma unroll
               for (int q = 0; q < 16; ++q)
                 p.out_part[(static_cast<size_t>(tc) * p.r_pad + c16 * 16 + q) * p.c_pad + c] = __uint_as_float(v[q]);
+            } else if (c < p.C) {
+              // the only token chunk: the sums are final, write them where the finalize kernel would have
+#pragma unroll
+              for (int q = 0; q < 16; ++q) {
+                const int j = c16 * 16 + q;
+                if (j < p.r) {
+                  if (p.out_is_da) p.out[static_cast<size_t>(j) * p.C + c] = __uint_as_float(v[q]);
+                  else p.out[static_cast<size_t>(c) * p.r + j] = __uint_as_float(v[q]);
+                }
+              }
             }
           }
         }
@@ -308,11 +325,19 @@ cudaError_t grad_configure() {
   return cudaFuncSetAttribute(lora_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
 }
 
-cudaError_t launch_grad(const CUtensorMap& tmS, const CUtensorMap& tmR, const CUtensorMap& tmA, const GradParams& p,
+bool grad_is_direct(const GradParams& p) {
+  return (!p.do_out || p.n_token_chunks == 1) && (!p.with_p || p.n_feat_chunks == 1);
+}
+
+cudaError_t launch_grad(const CUtensorMap& tmS, const CUtensorMap& tmR, const CUtensorMap& tmA, const GradParams& p_in,
                         cudaStream_t stream) {
+  GradParams p = p_in;
+  // No cross-CTA sum left (one token chunk for the gradient, one feature chunk for the side product): the streaming
+  // kernel writes the results itself and the finalize launch is dropped.  Only tiny problems have such grids.
+  p.direct = grad_is_direct(p) ? 1 : 0;
   dim3 grid(p.n_feat_chunks, p.n_token_chunks);
   cudaError_t e = launch_pdl(lora_grad_kernel, grid, dim3(kGradThreads), grad_smem_bytes(p), stream, tmS, tmR, tmA, p);
-  if (e != cudaSuccess) return e;
+  if (e != cudaSuccess || p.direct) return e;
   const long long n = (p.do_out ? static_cast<long long>(p.r) * p.C : 0) + (p.with_p ? static_cast<long long>(p.r_pad) * p.T : 0);
   return launch_pdl(lora_grad_finalize_kernel, dim3(static_cast<unsigned>((n + 255) / 256)), dim3(256), 0, stream, p);
 }

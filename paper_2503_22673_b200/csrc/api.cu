@@ -69,6 +69,10 @@ int pick_pair_block_n(long long T, long long N, int r_pad, int num_pairs) {
   return best;
 }
 
+// Streams of at most this many bytes run on a grid without cross-CTA sums (one launch instead of two): the whole
+// problem is a few microseconds of work and the second launch would cost more than the parallelism gains.
+constexpr long long kTinyStreamBytes = 1 << 20;
+
 struct GradGrid {
   int feat_chunk, n_feat, n_tok, stages;
 };
@@ -85,6 +89,9 @@ GradGrid pick_grad_grid(long long T, long long C, int r_pad, bool with_p, int nu
   int n_tok = num_sms / g.n_feat;             // at most one CTA per SM: a second wave would double the time
   if (n_tok > n_slabs) n_tok = n_slabs;
   if (n_tok < 1) n_tok = 1;
+  // tiny stream: one token chunk, so that no finalize launch is needed (pays only if the side product, where there is
+  // one, needs no cross-CTA sum either)
+  if (kTinyStreamBytes >= 2 * T * C && (!with_p || g.n_feat == 1)) n_tok = 1;
   g.n_tok = n_tok;
   const size_t stage = kGradStageBytes + (with_p ? 2 * static_cast<size_t>(r_pad) * 128 : 0);
   const size_t fixed = 4 * static_cast<size_t>(r_pad) * 128 + 2048;
@@ -456,6 +463,8 @@ int launch_side_prepass(lora_plan* pl, const void* S, long long C, const void* s
   const int n_slabs = w.n_slabs;
   int nf = ceil_div(pl->num_sms, n_slabs);
   if (nf > 4) nf = 4;
+  if (kTinyStreamBytes >= 2 * static_cast<long long>(s.T) * C) nf = 1;   // tiny stream: every CTA sees all features, so the
+                                                                          // side product needs no cross-CTA sum, no finalize launch
   const int fc = ceil_div(ceil_div(C, nf), 128) * 128;
   nf = ceil_div(C, fc);
   int nt = pl->num_sms / nf;
@@ -481,7 +490,7 @@ int launch_side_prepass(lora_plan* pl, const void* S, long long C, const void* s
   g.ld_t = w.ld_t;
   g.status = pl->d_status;
   if (launch_grad(tmS, tmS, tmSide, g, st) != cudaSuccess) return LORA_ERR_CUDA;
-  g_launches.fetch_add(2);
+  g_launches.fetch_add(grad_is_direct(g) ? 1 : 2);
   return LORA_OK;
 }
 
@@ -649,7 +658,7 @@ int launch_da(lora_plan* pl, const void* X, const void* A, float scale, void* dA
     g.ld_t = w.ld_t;
     g.status = pl->d_status;
     if (launch_grad(tmS, tmR, tmA, g, st) != cudaSuccess) return LORA_ERR_CUDA;
-    g_launches.fetch_add(2);
+    g_launches.fetch_add(grad_is_direct(g) ? 1 : 2);
   }
   return LORA_OK;
 }
@@ -693,7 +702,7 @@ int launch_db(lora_plan* pl, const void* dY, float scale, void* dB, cudaStream_t
     g.ld_t = w.ld_t;
     g.status = pl->d_status;
     if (launch_grad(tmS, tmR, with_q ? tmSide : tmR, g, st) != cudaSuccess) return LORA_ERR_CUDA;
-    g_launches.fetch_add(2);
+    g_launches.fetch_add(grad_is_direct(g) ? 1 : 2);
   }
   return LORA_OK;
 }

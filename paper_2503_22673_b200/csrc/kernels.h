@@ -139,6 +139,7 @@ struct GradParams {
   int side_mn;            // side operand: 0 = A [r, C] (K-major rows), 1 = B [C, r] (MN-major, natural layout)
   int do_out;             // 0: side product only (no second factor, no gradient)
   int out_is_da;          // 1: out[j * C + c] (dA), 0: out[c * r + j] (dB)
+  int direct;             // set by launch_grad: no cross-CTA sums are needed, the kernel writes out / pt_out itself
   float scale;
   float* out;             // final fp32 gradient
   float* out_part;        // [n_token_chunks][r_pad][C_pad]  partial sums (fixed-order reduction)
@@ -156,5 +157,7 @@ cudaError_t grad_configure();
 // fixed-order finalize kernel (2 launches).
 cudaError_t launch_grad(const CUtensorMap& tmS, const CUtensorMap& tmR, const CUtensorMap& tmA,
                         const GradParams& p, cudaStream_t stream);
+// true when launch_grad will run the streaming kernel alone (1 launch instead of 2)
+bool grad_is_direct(const GradParams& p);
 
 }  // namespace lora
