@@ -465,6 +465,10 @@ int launch_side_prepass(lora_plan* pl, const void* S, long long C, const void* s
   if (nf > 4) nf = 4;
   if (kTinyStreamBytes >= 2 * static_cast<long long>(s.T) * C) nf = 1;   // tiny stream: every CTA sees all features, so the
                                                                           // side product needs no cross-CTA sum, no finalize launch
+  if (const char* f = std::getenv("LORA_PREPASS_NF")) {                   // tuning knob
+    const int v = std::atoi(f);
+    if (v >= 1 && v <= 4) nf = v;
+  }
   const int fc = ceil_div(ceil_div(C, nf), 128) * 128;
   nf = ceil_div(C, fc);
   int nt = pl->num_sms / nf;
