@@ -102,6 +102,33 @@ GradGrid pick_grad_grid(long long T, long long C, int r_pad, bool with_p, int nu
   return g;
 }
 
+// Grid of a side-product-only pass (X A^T or dY B): feature chunks x token chunks.  No TMEM bound on the feature chunk.
+//  * as few feature chunks (at most 4) as fill the SMs together with the 128-token slabs;
+//  * ONE feature chunk for tiny streams and from 64 token slabs (8192 tokens) on: every CTA then sees all features, the
+//    kernel writes the bf16 result itself and the finalize launch goes away (pre-pass stage 31.1 -> 30.7 us at
+//    8192 x 4096, 107.9 -> 100.0 us at 16384 x 14336, one launch fewer each).
+struct SideGrid {
+  int feat_chunk, n_feat, n_tok;
+};
+
+SideGrid pick_side_grid(long long T, long long C, int num_sms) {
+  const int n_slabs = ceil_div(T, kGradSlab);
+  int nf = ceil_div(num_sms, n_slabs);
+  if (nf > 4) nf = 4;
+  if (kTinyStreamBytes >= 2 * T * C || n_slabs >= 64) nf = 1;
+  if (const char* f = std::getenv("LORA_PREPASS_NF")) {      // tuning knob
+    const int v = std::atoi(f);
+    if (v >= 1 && v <= 4) nf = v;
+  }
+  SideGrid g;
+  g.feat_chunk = ceil_div(ceil_div(C, nf), 128) * 128;
+  g.n_feat = ceil_div(C, g.feat_chunk);
+  g.n_tok = num_sms / g.n_feat;
+  if (g.n_tok > n_slabs) g.n_tok = n_slabs;
+  if (g.n_tok < 1) g.n_tok = 1;
+  return g;
+}
+
 int check_shape(const lora_shape_t* s) {
   if (s == nullptr) return LORA_ERR_INVALID_ARG;
   if (s->T < 0 || s->d_in <= 0 || s->d_out <= 0 || s->r <= 0) return LORA_ERR_INVALID_ARG;
@@ -269,19 +296,13 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
       }
     }
   }
-  {  // Q = dY B pre-pass of the CTA-pair backward: side product only, so the feature chunk is not bound by TMEM
-    const int n_slabs = ceil_div(T, kGradSlab);
-    int nf = ceil_div(num_sms, n_slabs);
-    int fc = ceil_div(ceil_div(s->d_out, nf), 128) * 128;
-    nf = ceil_div(s->d_out, fc);
-    int nt = num_sms / nf;
-    if (nt > n_slabs) nt = n_slabs;
-    if (nt < 1) nt = 1;
-    c->q_feat_chunk = fc;
-    c->q_feat_chunks = nf;
-    c->q_token_chunks = nt;
+  {  // Q = dY B pre-pass of the CTA-pair backward
+    const SideGrid q = pick_side_grid(T, s->d_out, num_sms);
+    c->q_feat_chunk = q.feat_chunk;
+    c->q_feat_chunks = q.n_feat;
+    c->q_token_chunks = q.n_tok;
     c->q_stages = 4;
-  }   // feature chunk of the dB kernel (differs from dA's only for small d_out)
+  }
   return LORA_OK;
 }
 
@@ -459,21 +480,9 @@ int launch_side_prepass(lora_plan* pl, const void* S, long long C, const void* s
   if (side_mn) ok = ok && make_bf16_tmap(&tmSide, side, s.r, C, s.r, 64, 64);
   else ok = ok && make_bf16_tmap(&tmSide, side, C, s.r, C, 64, c.r_pad);
   if (!ok) return LORA_ERR_CUDA;
-  // grid: as few feature chunks as fill the SMs together with the 128-token slabs (no TMEM bound: side product only)
+  const SideGrid sg = pick_side_grid(s.T, C, pl->num_sms);
   const int n_slabs = w.n_slabs;
-  int nf = ceil_div(pl->num_sms, n_slabs);
-  if (nf > 4) nf = 4;
-  if (kTinyStreamBytes >= 2 * static_cast<long long>(s.T) * C) nf = 1;   // tiny stream: every CTA sees all features, so the
-                                                                          // side product needs no cross-CTA sum, no finalize launch
-  if (const char* f = std::getenv("LORA_PREPASS_NF")) {                   // tuning knob
-    const int v = std::atoi(f);
-    if (v >= 1 && v <= 4) nf = v;
-  }
-  const int fc = ceil_div(ceil_div(C, nf), 128) * 128;
-  nf = ceil_div(C, fc);
-  int nt = pl->num_sms / nf;
-  if (nt > n_slabs) nt = n_slabs;
-  if (nt < 1) nt = 1;
+  const int fc = sg.feat_chunk, nf = sg.n_feat, nt = sg.n_tok;
   GradParams g{};
   g.T = static_cast<int>(s.T);
   g.C = static_cast<int>(C);
