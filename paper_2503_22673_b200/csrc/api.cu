@@ -54,6 +54,15 @@ int pick_pair_block_n(long long T, long long N, int r_pad, int num_pairs) {
     const int v = std::atoi(f);
     if (v >= 64 && v % 16 == 0 && v + r_pad <= 256) return v;
   }
+  if (r_pad == 0) {
+    // K-extended GEMMs (no adapter columns; weight-side operand mostly MN-major).  Measured on dW 8192 x 4096 x 4096, us per
+    // launch by width: 128: 262, 160: 236, 192: 201, 208: 240, 224: 209, 240: 219, 256: 184 - a wave costs 38-40 us up to
+    // 192 columns (the 256-row activation tile is fetched per k-block whatever the width) and 46 us at 256, and widths
+    // that are not multiples of 64 pay plain stores for their ragged last chunk.  So: 256 whenever that still gives
+    // three quarters of the CTA pairs a tile; starved grids go through the width search below (narrower tiles buy parallelism there).
+    const long long tiles256 = static_cast<long long>(ceil_div(T, kPairBlockM)) * ceil_div(N, 256);
+    if (tiles256 * 4 >= static_cast<long long>(num_pairs) * 3) return 256;   // one 256-wide wave (46 us) beats one 240-wide (55 us)
+  }
   int best = 256 - r_pad;
   double best_cost = 1e300;
   const int lo = r_pad + 32 > 144 ? r_pad + 32 : 144;
