@@ -161,6 +161,10 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
   c->stages = 4;
   c->dx_stages = 4;
   c->group_m = 8;
+  if (const char* f = std::getenv("LORA_FORCE_GROUP_M")) {   // tuning knob: m-tiles per rasterisation band
+    const int v = std::atoi(f);
+    if (v >= 1 && v <= 64) c->group_m = v;
+  }
   c->split_k = 1;
   c->dx_split_k = 1;
   c->tail_delay = 8;
