@@ -35,7 +35,7 @@ UNIT = "TFLOP/s"
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel from an
 # ncu capture summarised under profiles/; only valid for the kernel source it was taken on.
-NCU_TRAFFIC = {"gemm_sha": "cf932fe86503db69", "bytes_per_launch": {"fwd_gemm": 221.3e6, "dx_gemm": 219.7e6}}
+NCU_TRAFFIC = {"gemm_sha": "7c3994e03b7d900f", "bytes_per_launch": {"fwd_gemm": 221.3e6, "dx_gemm": 219.7e6}}
 
 
 def peaks():

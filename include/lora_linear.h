@@ -118,6 +118,13 @@ int lora_plan_workspace_bytes(const lora_plan_t* plan, size_t* fwd_bytes, size_t
  * owned by the caller and must outlive every backward call that uses the plan. */
 int lora_plan_set_workspace(lora_plan_t* plan, void* dev_ptr, size_t bytes);
 
+/* Gradient accumulation over micro-batches (the paper trains with global batches of 32-96 sequences, i.e. several
+ * backward passes per optimiser step): with `enable` != 0 every backward call on the plan ADDS its dA and dB to the
+ * caller's buffers instead of overwriting them (dA += ..., dB += ...; the caller zeroes them before the first
+ * micro-batch).  The sum stays deterministic: old value + the call's partial sums in their fixed order.  dX is always
+ * overwritten.  Off by default. */
+int lora_plan_set_grad_accumulation(lora_plan_t* plan, int enable);
+
 /* Copy the selector's choice / a one-line description into caller memory. */
 int lora_plan_get_config(const lora_plan_t* plan, lora_kernel_config_t* out);
 int lora_plan_describe(const lora_plan_t* plan, char* buf, size_t n);

@@ -25,7 +25,7 @@ LORA_ERR_NO_DEVICE = -7
 
 EXPORTS = [
     "lora_select_config", "lora_workspace_bytes", "lora_plan_create", "lora_plan_destroy",
-    "lora_plan_workspace_bytes", "lora_plan_set_workspace", "lora_plan_get_config", "lora_plan_describe",
+    "lora_plan_workspace_bytes", "lora_plan_set_workspace", "lora_plan_set_grad_accumulation", "lora_plan_get_config", "lora_plan_describe",
     "lora_linear_fwd", "lora_linear_bwd", "lora_linear_bwd_saved_p", "lora_linear_bwd_q", "lora_linear_bwd_dx", "lora_linear_bwd_da", "lora_linear_bwd_db",
     "lora_dense_dw", "lora_nf4_quantize", "lora_nf4_dequantize", "lora_linear_fwd_nf4", "lora_linear_bwd_nf4", "lora_step_host_staging_bytes", "lora_linear_step_host",
     "lora_last_device_status", "lora_strerror", "lora_launch_count",
@@ -72,6 +72,7 @@ def load(rebuild: bool = False) -> ctypes.CDLL:
     lib.lora_plan_destroy.argtypes = [vp]
     lib.lora_plan_workspace_bytes.argtypes = [vp, sz_p, sz_p]
     lib.lora_plan_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
+    lib.lora_plan_set_grad_accumulation.argtypes = [vp, ctypes.c_int]
     lib.lora_plan_get_config.argtypes = [vp, ctypes.POINTER(LoraKernelConfig)]
     lib.lora_plan_describe.argtypes = [vp, ctypes.c_char_p, ctypes.c_size_t]
     lib.lora_linear_fwd.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp]
@@ -208,6 +209,10 @@ class LoraLinearPlan:
         self._ws = ws
         n = 0 if ws is None else ws.numel() * ws.element_size()
         _check(self._lib.lora_plan_set_workspace(self._h, _ptr(ws), n), "lora_plan_set_workspace")
+
+    def set_grad_accumulation(self, enable: bool) -> None:
+        """Backward calls add dA / dB to the given buffers instead of overwriting them (micro-batch accumulation)."""
+        _check(self._lib.lora_plan_set_grad_accumulation(self._h, 1 if enable else 0), "lora_plan_set_grad_accumulation")
 
     # -- the two calls -------------------------------------------------------------------------
     def fwd(self, X, W, A, B, scale: float, Y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:

@@ -246,8 +246,8 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
               for (int q = 0; q < 16; ++q) {
                 const int j = c16 * 16 + q;
                 if (j < p.r) {
-                  if (p.out_is_da) p.out[static_cast<size_t>(j) * p.C + c] = __uint_as_float(v[q]);
-                  else p.out[static_cast<size_t>(c) * p.r + j] = __uint_as_float(v[q]);
+                  float* dst = p.out_is_da ? p.out + static_cast<size_t>(j) * p.C + c : p.out + static_cast<size_t>(c) * p.r + j;
+                  *dst = p.accumulate ? *dst + __uint_as_float(v[q]) : __uint_as_float(v[q]);
                 }
               }
             }
@@ -302,8 +302,8 @@ __global__ void __launch_bounds__(256) lora_grad_finalize_kernel(const GradParam
     const int j = static_cast<int>(idx / p.C), c = static_cast<int>(idx - static_cast<long long>(j) * p.C);
     const float acc = ordered_sum(p.out_part + static_cast<size_t>(j) * p.c_pad + c, p.n_token_chunks,
                                   static_cast<size_t>(p.r_pad) * p.c_pad);
-    if (p.out_is_da) p.out[static_cast<size_t>(j) * p.C + c] = acc;
-    else p.out[static_cast<size_t>(c) * p.r + j] = acc;
+    float* dst = p.out_is_da ? p.out + static_cast<size_t>(j) * p.C + c : p.out + static_cast<size_t>(c) * p.r + j;
+    *dst = p.accumulate ? *dst + acc : acc;      // gradient accumulation: old value + (partials in fixed order)
   } else if (idx < n_out + n_pt) {
     const long long i2 = idx - n_out;
     const int j = static_cast<int>(i2 / p.T), t = static_cast<int>(i2 - static_cast<long long>(j) * p.T);

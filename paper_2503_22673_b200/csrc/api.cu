@@ -448,6 +448,7 @@ struct lora_plan {
   void* workspace;
   size_t workspace_bytes;
   bool q_ready;          // set while lora_linear_bwd_saved_p runs: Qt was already produced by its dB kernel
+  bool accumulate;       // dA / dB are added to instead of overwritten (lora_plan_set_grad_accumulation)
   bool q_staged;         // lora_linear_bwd_q ran: the next lora_linear_bwd_dx skips its own pre-pass
   cudaStream_t side_stream;   // overlapped backward: the adapter-gradient passes run here beside the dX GEMM
   cudaEvent_t ev_fork, ev_join;
@@ -675,6 +676,7 @@ int launch_da(lora_plan* pl, const void* X, const void* A, float scale, void* dA
     g.side_mn = 0;
     g.do_out = 1;
     g.out_is_da = 1;
+    g.accumulate = pl->accumulate ? 1 : 0;
     g.scale = scale;
     g.out = static_cast<float*>(dA);
     g.out_part = reinterpret_cast<float*>(ws + w.da_part);
@@ -719,6 +721,7 @@ int launch_db(lora_plan* pl, const void* dY, float scale, void* dB, cudaStream_t
     g.side_mn = with_q ? 1 : 0;
     g.do_out = 1;
     g.out_is_da = 0;
+    g.accumulate = pl->accumulate ? 1 : 0;
     g.scale = scale;
     g.out = static_cast<float*>(dB);
     g.out_part = reinterpret_cast<float*>(ws + w.db_part);
@@ -922,6 +925,7 @@ int lora_plan_create(const lora_shape_t* shape, int device, lora_plan_t** out) {
   pl->workspace_bytes = 0;
   pl->q_ready = false;
   pl->q_staged = false;
+  pl->accumulate = false;
   pl->p_saved = false;
   pl->p_saved_scale = 0.f;
   pl->d_status = nullptr;
@@ -979,6 +983,12 @@ int lora_plan_set_workspace(lora_plan_t* plan, void* dev_ptr, size_t bytes) {
   return LORA_OK;
 }
 
+int lora_plan_set_grad_accumulation(lora_plan_t* plan, int enable) {
+  if (plan == nullptr) return LORA_ERR_INVALID_ARG;
+  plan->accumulate = enable != 0;
+  return LORA_OK;
+}
+
 int lora_plan_get_config(const lora_plan_t* plan, lora_kernel_config_t* out) {
   if (plan == nullptr || out == nullptr) return LORA_ERR_INVALID_ARG;
   *out = plan->cfg;
@@ -1019,6 +1029,7 @@ int lora_linear_bwd(lora_plan_t* plan, const void* dY, const void* X, const void
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   DeviceGuard guard(plan->device);
   if (plan->shape.T == 0) {   // empty batch: the sums over tokens are empty
+    if (plan->accumulate) return LORA_OK;
     if (cudaMemsetAsync(dA, 0, sizeof(float) * plan->shape.r * plan->shape.d_in, st) != cudaSuccess ||
         cudaMemsetAsync(dB, 0, sizeof(float) * plan->shape.d_out * plan->shape.r, st) != cudaSuccess)
       return LORA_ERR_CUDA;
@@ -1107,6 +1118,7 @@ int lora_linear_bwd_da(lora_plan_t* plan, const void* X, const void* A, float sc
   if (plan == nullptr || !dA) return LORA_ERR_INVALID_ARG;
   if (!aligned16(dA)) return LORA_ERR_MISALIGNED;
   DeviceGuard guard(plan->device);
+  if (plan->shape.T == 0 && plan->accumulate) return LORA_OK;
   if (plan->shape.T == 0)
     return cudaMemsetAsync(dA, 0, sizeof(float) * plan->shape.r * plan->shape.d_in, static_cast<cudaStream_t>(stream)) ==
                    cudaSuccess ? LORA_OK : LORA_ERR_CUDA;
@@ -1120,6 +1132,7 @@ int lora_linear_bwd_db(lora_plan_t* plan, const void* dY, float scale, void* dB,
   if (plan == nullptr || !dB) return LORA_ERR_INVALID_ARG;
   if (!aligned16(dB)) return LORA_ERR_MISALIGNED;
   DeviceGuard guard(plan->device);
+  if (plan->shape.T == 0 && plan->accumulate) return LORA_OK;
   if (plan->shape.T == 0)
     return cudaMemsetAsync(dB, 0, sizeof(float) * plan->shape.d_out * plan->shape.r, static_cast<cudaStream_t>(stream)) ==
                    cudaSuccess ? LORA_OK : LORA_ERR_CUDA;
@@ -1189,6 +1202,7 @@ int lora_linear_bwd_nf4(lora_plan_t* plan, const void* dY, const void* X, const 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   DeviceGuard guard(plan->device);
   if (plan->shape.T == 0) {
+    if (plan->accumulate) return LORA_OK;
     if (cudaMemsetAsync(dA, 0, sizeof(float) * plan->shape.r * plan->shape.d_in, st) != cudaSuccess ||
         cudaMemsetAsync(dB, 0, sizeof(float) * plan->shape.d_out * plan->shape.r, st) != cudaSuccess)
       return LORA_ERR_CUDA;

@@ -139,6 +139,7 @@ struct GradParams {
   int side_mn;            // side operand: 0 = A [r, C] (K-major rows), 1 = B [C, r] (MN-major, natural layout)
   int do_out;             // 0: side product only (no second factor, no gradient)
   int out_is_da;          // 1: out[j * C + c] (dA), 0: out[c * r + j] (dB)
+  int accumulate;         // 1: out += result (gradient accumulation over micro-batches), 0: out = result
   int direct;             // set by launch_grad: no cross-CTA sums are needed, the kernel writes out / pt_out itself
   float scale;
   float* out;             // final fp32 gradient

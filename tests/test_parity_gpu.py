@@ -378,3 +378,33 @@ def test_staged_pre_pass_is_used_once_and_discarded_by_other_calls():
     code, msg = plan.device_status()
     assert code == 0, msg
     plan.close()
+
+
+@pytest.mark.parametrize("T1,T2,d_in,d_out,r", [(300, 212, 264, 520, 16),        # tiny: the streaming kernels write dA / dB themselves
+                                                 (4096, 2100, 1024, 1160, 32)])   # partial sums + finalize kernel
+def test_gradient_accumulation_over_micro_batches(T1, T2, d_in, d_out, r):
+    """With lora_plan_set_grad_accumulation the backward calls add into dA / dB: two micro-batches give the gradients of the
+    concatenated batch (the sums over token rows are additive), dX stays per micro-batch."""
+    scale = 2.0
+    p, t = inputs.draw_custom(T1 + T2, d_in, d_out, r, scale, seed=31)
+    d = {k: dev(v) for k, v in t.items()}
+    dA = torch.zeros((r, d_in), dtype=torch.float32, device="cuda")
+    dB = torch.zeros((d_out, r), dtype=torch.float32, device="cuda")
+    dX = torch.empty((T1 + T2, d_in), dtype=torch.bfloat16, device="cuda")
+    for lo, hi in ((0, T1), (T1, T1 + T2)):
+        plan = binding.LoraLinearPlan(hi - lo, d_in, d_out, r)
+        plan.set_grad_accumulation(True)
+        plan.bwd(d["dY"][lo:hi], d["X"][lo:hi], d["W"], d["A"], d["B"], scale, dX[lo:hi], dA, dB)
+        code, msg = plan.device_status()
+        assert code == 0, msg
+        plan.close()
+    f = {k: inputs.bf16_to_f64(v) for k, v in t.items()}
+    dXr, dAr, dBr = oracle.backward(f["dY"], f["X"], f["W"], f["A"], f["B"], scale)
+    assert oracle.rel_err(host64(dX), dXr) <= TOL_BF16
+    assert oracle.rel_err(host64(dA), dAr) <= TOL_F32 and oracle.rel_err(host64(dB), dBr) <= TOL_F32
+    # switched off again, the same call overwrites
+    plan = binding.LoraLinearPlan(T2, d_in, d_out, r)
+    plan.bwd(d["dY"][T1:], d["X"][T1:], d["W"], d["A"], d["B"], scale, dX[T1:], dA, dB)
+    _, dA2, dB2 = oracle.backward(f["dY"][T1:], f["X"][T1:], f["W"], f["A"], f["B"], scale)
+    assert oracle.rel_err(host64(dA), dA2) <= TOL_F32 and oracle.rel_err(host64(dB), dB2) <= TOL_F32
+    plan.close()
