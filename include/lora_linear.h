@@ -111,7 +111,7 @@ int lora_plan_create(const lora_shape_t* shape, int device, lora_plan_t** out);
 int lora_plan_destroy(lora_plan_t* plan);
 
 /* Scratch sizes of a plan; either pointer may be NULL.  fwd_bytes is 0 unless the selector chose the K-extended
- * forward (cfg.fwd_ext, large ranks), which uses the same workspace as backward. */
+ * forward (cfg.fwd_ext), which uses the same workspace as backward. */
 int lora_plan_workspace_bytes(const lora_plan_t* plan, size_t* fwd_bytes, size_t* bwd_bytes);
 
 /* Register caller-owned device scratch (256-byte aligned, at least bwd_bytes).  The memory stays
@@ -130,8 +130,12 @@ int lora_plan_get_config(const lora_plan_t* plan, lora_kernel_config_t* out);
 int lora_plan_describe(const lora_plan_t* plan, char* buf, size_t n);
 
 /* Forward:  Y = X W^T + scale (X A^T) B^T.
- * One fused kernel: TMA-staged bf16 tiles, tcgen05 MMA into TMEM; X A^T rides the main loop as
- * extra accumulator columns and the rank-r product is one more MMA group before the epilogue. */
+ * TMA-staged bf16 tiles, tcgen05 MMA into TMEM.  Two forms, chosen per shape (cfg.fwd_ext):
+ *   fused       one kernel; X A^T rides the main loop as extra accumulator columns and the rank-r product is one more
+ *               MMA group before the epilogue (narrow outputs, small batches; needs no workspace);
+ *   K-extended  a skinny pass over X produces scale (X A^T)^T, which then enters the GEMM as one more k-block, so that
+ *               every MMA column is an output column (wide outputs, large ranks, >= 4096 tokens; needs the workspace:
+ *               LORA_ERR_WORKSPACE otherwise, see lora_plan_workspace_bytes). */
 int lora_linear_fwd(lora_plan_t* plan, const void* X, const void* W, const void* A, const void* B,
                     float scale, void* Y, void* stream);
 
