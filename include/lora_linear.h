@@ -19,13 +19,15 @@
  *   - Every function returns an int: LORA_OK (0) or a negative lora_status_t.  Nothing throws,
  *     nothing calls exit().
  *   - Tensor pointers are DEVICE pointers owned by the caller (unless a parameter is named h_*),
- *     16-byte aligned.  Inputs are read-only; outputs are overwritten, never accumulated into.
+ *     16-byte aligned.  Inputs are read-only; outputs are overwritten.  The one exception is opt-in per plan:
+ *     after lora_plan_set_grad_accumulation(plan, 1) the backward calls ADD to dA and dB (dX is still overwritten).
  *     No output may alias an input or another output.
  *   - d_in and d_out must be multiples of 8; r a multiple of 8 with 8 <= r <= 64; T >= 0.
  *   - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work and return; they do not
  *     synchronise.  A plan must not be used from two host threads, or on two streams, at once.
  *   - The library never allocates device memory except one 256-byte status word block per plan;
- *     backward scratch is caller-provided (lora_plan_set_workspace).
+ *     scratch is caller-provided (lora_plan_set_workspace): backward always needs it, forward needs it whenever the
+ *     selector chose the K-extended form (cfg.fwd_ext; lora_plan_workspace_bytes reports fwd_bytes > 0 then).
  *   - There is no CPU fallback: without a CUDA device of compute capability 10.x the calls fail
  *     with LORA_ERR_NO_DEVICE.
  */
@@ -102,7 +104,9 @@ typedef struct lora_kernel_config {
  * Needs no GPU.  Returns LORA_ERR_UNSUPPORTED_SHAPE for shapes the kernels do not cover. */
 int lora_select_config(const lora_shape_t* shape, int num_sms, lora_kernel_config_t* out);
 
-/* Host-only: bytes of backward scratch lora_linear_bwd needs for a shape (forward needs none). */
+/* Host-only: bytes of scratch lora_linear_bwd needs for a shape.  The forward uses the same scratch when the selector
+ * picks its K-extended form for the shape (lora_kernel_config_t.fwd_ext = 1, e.g. every 4096-wide or wider output
+ * from 4096 tokens on); the fused form needs none.  lora_plan_workspace_bytes reports both figures for a plan. */
 int lora_workspace_bytes(const lora_shape_t* shape, int num_sms, size_t* bwd_bytes);
 
 /* Create / destroy a plan for one shape on CUDA device `device` (runs the selector, allocates the
@@ -227,6 +231,22 @@ int lora_linear_step_host(lora_plan_t* plan, const void* h_X, const void* W, con
                           const void* h_B, const void* h_dY, float scale, void* h_Y, void* h_dX,
                           void* h_dA, void* h_dB, void* staging, size_t staging_bytes, void* stream);
 
+/* Failure detection.  Every device-side wait (on an mbarrier fed by TMA, by the tensor core or by other warps) gives
+ * up after a limit of SM clock ticks; the kernel then records which wait ran out and in which CTA in the plan's status
+ * block, lets its copies in flight land, frees its tensor memory and returns, so the context stays usable.
+ * lora_last_device_status reports and clears the record.
+ *   lora_plan_set_wait_limit   limit for the plan's later launches, in SM clock ticks (default 4e9, about 2 s; 0 restores
+ *                              the default; values below 1000 are raised to 1000).  Also settable for new plans through
+ *                              the environment variable LORA_DEBUG_WAIT_CAP.
+ *   lora_debug_starved_wait    test hook: launches ONE CTA of the adapter-gradient kernel over S [T, C] bf16 (T <= 1024,
+ *                              C <= 512, C % 8 == 0) whose second-factor loader issues nothing, so that the MMA warp's
+ *                              bounded wait runs out while no copy is outstanding except the few stages of S that
+ *                              complete on their own.  `out` ([C, r] fp32) is never written.  Nothing faults or traps; with
+ *                              a short limit the launch ends within a millisecond and the next
+ *                              lora_last_device_status returns LORA_ERR_DEVICE_TIMEOUT.  */
+int lora_plan_set_wait_limit(lora_plan_t* plan, int64_t cycles);
+int lora_debug_starved_wait(lora_plan_t* plan, const void* S, int64_t T, int64_t C, void* out, void* stream);
+
 /* Token contraction without any allocation (the paper has no counterpart; this is a library convenience).
  *
  *     out[c, j] = sum_t S[t, c] * Rt[j, t]          S [T, C] bf16, Rt [r, ld_rt] bf16 (ld_rt >= T), out [C, r] fp32
@@ -239,16 +259,22 @@ int lora_linear_step_host(lora_plan_t* plan, const void* h_X, const void* W, con
  * allocates or frees: the partial sums and status word live in one static device array
  * of lora_grad_contract_noalloc_max_scratch() bytes (8 MiB) that every GPU loading the library holds until
  * the process exits.
- *   - Shapes whose partial sums do not fit (roughly SMs/ceil(C/512) x r_pad x C x 4 bytes > 8 MiB) are
- *     rejected with LORA_ERR_WORKSPACE; C % 8 == 0, r in {8,...,64}, ld_rt % 8 == 0, T >= 1.
+ *   - C % 8 == 0, r in {8,...,64}, ld_rt % 8 == 0, T >= 1.  The grid takes as many token chunks as the array has room
+ *     for their partial sums (r_pad x C_pad floats each, r_pad = r rounded up to 16, C_pad = C rounded up to 32), down to
+ *     a single chunk, which needs none: wide matrices run with fewer CTAs, they are not refused.  Only a shape whose
+ *     single layer of partial sums exceeds the array (r_pad x C_pad x 4 bytes > 8 MiB - 4 KiB, i.e. C beyond 32736 at
+ *     r = 64 or 131040 at r = 16) is rejected with LORA_ERR_WORKSPACE.
  *   - The first call on a device looks up the array's device address and raises the kernel's shared-memory
  *     limit; make that first call before any stream capture.  The current device is used.
  *   - All calls share the one array and it keeps the last call's contents; the call clears the status
  *     words on `stream` first and rewrites every partial sum before reading it.  Two calls whose kernels overlap on the GPU (different streams, or
  *     different host threads) race on it: serialise them.
- *   - A bounded device wait that ran out is not reported by this call (there is no plan to ask). */
+ *   - A bounded device wait that ran out leaves `out` incomplete while the call itself has long returned LORA_OK:
+ *     lora_grad_contract_noalloc_status synchronises `stream`, reads the status word of the current device's array
+ *     (a 4-byte copy, no allocation) and sets *code to LORA_OK or LORA_ERR_DEVICE_TIMEOUT. */
 int lora_grad_contract_noalloc(const void* S, const void* Rt, int64_t T, int64_t C, int64_t r, int64_t ld_rt,
                                void* out, void* stream);
+int lora_grad_contract_noalloc_status(void* stream, int* code);
 int64_t lora_grad_contract_noalloc_max_scratch(void);
 
 /* Synchronise `stream`, then report whether any kernel of this plan gave up on a bounded wait.

@@ -29,7 +29,8 @@ EXPORTS = [
     "lora_linear_fwd", "lora_linear_bwd", "lora_linear_bwd_saved_p", "lora_linear_bwd_q", "lora_linear_bwd_dx", "lora_linear_bwd_da", "lora_linear_bwd_db",
     "lora_dense_dw", "lora_nf4_quantize", "lora_nf4_dequantize", "lora_linear_fwd_nf4", "lora_linear_bwd_nf4", "lora_step_host_staging_bytes", "lora_linear_step_host",
     "lora_last_device_status", "lora_strerror", "lora_launch_count",
-    "lora_grad_contract_noalloc", "lora_grad_contract_noalloc_max_scratch",
+    "lora_grad_contract_noalloc", "lora_grad_contract_noalloc_max_scratch", "lora_grad_contract_noalloc_status",
+    "lora_plan_set_wait_limit", "lora_debug_starved_wait",
 ]
 
 
@@ -96,6 +97,9 @@ def load(rebuild: bool = False) -> ctypes.CDLL:
     lib.lora_launch_count.argtypes = []
     lib.lora_launch_count.restype = i64
     lib.lora_grad_contract_noalloc.argtypes = [vp, vp, i64, i64, i64, i64, vp, vp]
+    lib.lora_grad_contract_noalloc_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
+    lib.lora_plan_set_wait_limit.argtypes = [vp, i64]
+    lib.lora_debug_starved_wait.argtypes = [vp, vp, i64, i64, vp, vp]
     lib.lora_grad_contract_noalloc_max_scratch.argtypes = []
     lib.lora_grad_contract_noalloc_max_scratch.restype = i64
     for name in EXPORTS:
@@ -209,6 +213,16 @@ class LoraLinearPlan:
         self._ws = ws
         n = 0 if ws is None else ws.numel() * ws.element_size()
         _check(self._lib.lora_plan_set_workspace(self._h, _ptr(ws), n), "lora_plan_set_workspace")
+
+    def set_wait_limit(self, cycles: int) -> None:
+        """Limit of every device-side wait of this plan's later launches, in SM clock ticks (0: the default, ~2 s)."""
+        _check(self._lib.lora_plan_set_wait_limit(self._h, int(cycles)), "lora_plan_set_wait_limit")
+
+    def debug_starved_wait(self, S: torch.Tensor, out: torch.Tensor, stream=None) -> None:
+        """Test hook: one CTA of the adapter-gradient kernel whose second factor never arrives (its wait runs out)."""
+        T, C = S.shape
+        _check(self._lib.lora_debug_starved_wait(self._h, _ptr(S), T, C, _ptr(out), _stream_ptr(stream)),
+               "lora_debug_starved_wait")
 
     def set_grad_accumulation(self, enable: bool) -> None:
         """Backward calls add dA / dB to the given buffers instead of overwriting them (micro-batch accumulation)."""
@@ -401,6 +415,13 @@ def grad_contract_noalloc(S: torch.Tensor, Rt: torch.Tensor, out: torch.Tensor, 
     _check(load().lora_grad_contract_noalloc(_ptr(S), _ptr(Rt), T, C, r, ld, _ptr(out), _stream_ptr(stream)),
            "lora_grad_contract_noalloc")
     return out
+
+
+def grad_contract_noalloc_status(stream=None) -> int:
+    """LORA_OK, or LORA_ERR_DEVICE_TIMEOUT when a bounded wait of an allocation-free call ran out (synchronises the stream)."""
+    code = ctypes.c_int(0)
+    _check(load().lora_grad_contract_noalloc_status(_stream_ptr(stream), ctypes.byref(code)), "lora_grad_contract_noalloc_status")
+    return int(code.value)
 
 
 def nf4_quantize(W: torch.Tensor, stream=None):

@@ -105,7 +105,7 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
       const int t0 = s * kGradSlab;
       for (int nb = 0; nb < NB && ok; ++nb) {
         if (odd == warp) {
-          ok = warp_wait(empty_bar(slot), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY, false, 20);
+          ok = warp_wait(empty_bar(slot), phase ^ 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_EMPTY, false, 20);
           if (ok && elect_one()) {
             const uint32_t dst = ring + slot * stage_bytes, fb = full_bar(slot);
             const int cc = c0 + nb * 128;
@@ -130,8 +130,8 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
     // ================================ loader of the second factor (one 128-token slab at a time) ================================
     bool ok = true;
     int rb = 0, rphase = 0;
-    for (int s = s_begin; s < s_end && ok && p.do_out; ++s) {
-      ok = warp_wait(rt_empty(rb), rphase ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY, false, 20);
+    for (int s = s_begin; s < s_end && ok && p.do_out && !p.debug_no_second_factor; ++s) {
+      ok = warp_wait(rt_empty(rb), rphase ^ 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_EMPTY, false, 20);
       if (ok && elect_one()) {
         const int t0 = s * kGradSlab;
         mbar_arrive_expect_tx(rt_full(rb), 2 * rt_box);
@@ -154,10 +154,10 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
     bool ok = true;
     int slot = 0, phase = 0, rb = 0, rphase = 0;
     for (int s = s_begin; s < s_end && ok; ++s) {
-      if (p.do_out) ok = warp_wait(rt_full(rb), rphase, abort_flag, p.status, DEV_TIMEOUT_FULL, false, 0);
-      if (ok && p.with_p) ok = warp_wait(p_empty(rb), rphase ^ 1, abort_flag, p.status, DEV_TIMEOUT_ACC_EMPTY, false, 0);
+      if (p.do_out) ok = warp_wait(rt_full(rb), rphase, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_FULL, false, 0);
+      if (ok && p.with_p) ok = warp_wait(p_empty(rb), rphase ^ 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_ACC_EMPTY, false, 0);
       for (int nb = 0; nb < NB && ok; ++nb) {
-        ok = warp_wait(full_bar(slot), phase, abort_flag, p.status, DEV_TIMEOUT_FULL, false, 0);
+        ok = warp_wait(full_bar(slot), phase, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_FULL, false, 0);
         if (!ok) break;
         tc_fence_after();
         if (elect_one()) {
@@ -200,7 +200,7 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
       int pb = 0, pphase = 0;
       for (int s = s_begin; s < s_end; ++s) {
         const int t = s * kGradSlab + row;
-        bool ok = warp_wait(p_full(pb), pphase, abort_flag, p.status, DEV_TIMEOUT_SIDE, false, 32);
+        bool ok = warp_wait(p_full(pb), pphase, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_SIDE, false, 32);
         if (named_bar_or(1, 128, !ok)) { alive = false; break; }
         tc_fence_after();
         for (int c16 = 0; c16 < p.r_pad / 16; ++c16) {
@@ -226,7 +226,7 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
       }
     }
     if (alive && p.do_out) {
-      bool ok = warp_wait(out_full, 0, abort_flag, p.status, DEV_TIMEOUT_ACC, false, 32);
+      bool ok = warp_wait(out_full, 0, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_ACC, false, 32);
       if (!named_bar_or(1, 128, !ok)) {
         tc_fence_after();
         // ---- this CTA's sums over its token chunk -> out_part[tc][j][c] ----
@@ -445,9 +445,15 @@ extern "C" int lora_grad_contract_noalloc(const void* S, const void* Rt, int64_t
   int stages = static_cast<int>((232448 - fixed) / kGradStageBytes);
   g.stages = stages > kGradMaxStages ? kGradMaxStages : stages;
   g.c_pad = static_cast<int>((C + 31) / 32 * 32);
-  const size_t part_bytes = static_cast<size_t>(n_tok) * g.r_pad * g.c_pad * sizeof(float);
-  if (kNoAllocHeaderBytes + part_bytes > kNoAllocScratchBytes)
-    return LORA_ERR_WORKSPACE;      // the problem needs more scratch than the static array holds
+  // The partial sums of all token chunks must fit the static array.  One layer (r_pad x c_pad floats) that does not fit
+  // is beyond what this entry point serves; otherwise the grid takes as many token chunks as fit, and with a single
+  // chunk the kernel needs no partial sums at all (it writes `out` itself), so a fitting shape is never refused, only
+  // given fewer CTAs.
+  const size_t layer_bytes = static_cast<size_t>(g.r_pad) * g.c_pad * sizeof(float);
+  if (kNoAllocHeaderBytes + layer_bytes > kNoAllocScratchBytes) return LORA_ERR_WORKSPACE;
+  const int fit = static_cast<int>((kNoAllocScratchBytes - kNoAllocHeaderBytes) / layer_bytes);
+  if (n_tok > fit) n_tok = fit >= 2 ? fit : 1;
+  g.n_token_chunks = n_tok;
   g.with_p = 0;
   g.side_mn = 0;
   g.do_out = 1;
@@ -459,6 +465,7 @@ extern "C" int lora_grad_contract_noalloc(const void* S, const void* Rt, int64_t
   g.pt_out = nullptr;
   g.ld_t = static_cast<int>(ld_rt);
   g.status = reinterpret_cast<unsigned*>(nd.scratch);
+  g.wait_limit = kWaitLimitCycles;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // the array keeps the previous call's contents: the status words must start at zero (the partial sums are
   // fully rewritten before they are read)
@@ -468,6 +475,25 @@ extern "C" int lora_grad_contract_noalloc(const void* S, const void* Rt, int64_t
       !noalloc_tmap(&tmR, Rt, static_cast<uint64_t>(T), static_cast<uint64_t>(r), static_cast<uint64_t>(ld_rt), 64, g.r_pad))
     return LORA_ERR_CUDA;
   if (launch_grad(tmS, tmR, tmR, g, st) != cudaSuccess) return LORA_ERR_CUDA;
+  return LORA_OK;
+}
+
+extern "C" int lora_grad_contract_noalloc_status(void* stream, int* code) {
+  using namespace lora;
+  if (code == nullptr) return LORA_ERR_INVALID_ARG;
+  *code = LORA_OK;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNoAllocMaxDevices) return LORA_ERR_NO_DEVICE;
+  unsigned char* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (g_noalloc_dev[dev].ready) scratch = g_noalloc_dev[dev].scratch;
+  }
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return LORA_ERR_CUDA;
+  if (scratch == nullptr) return LORA_OK;       // no call was made on this device yet
+  unsigned word = 0;                             // a copy into pageable host memory: no allocation on the device
+  if (cudaMemcpy(&word, scratch, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return LORA_ERR_CUDA;
+  if (word != 0) *code = LORA_ERR_DEVICE_TIMEOUT;
   return LORA_OK;
 }
 

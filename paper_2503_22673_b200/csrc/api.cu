@@ -454,6 +454,7 @@ struct lora_plan {
   cudaEvent_t ev_fork, ev_join;
   bool p_saved;          // the workspace holds Pt = s (X A^T)^T of the last forward call
   float p_saved_scale;
+  long long wait_limit;  // SM clock ticks after which a device-side spin gives up (lora_plan_set_wait_limit)
 };
 
 namespace {
@@ -516,6 +517,7 @@ int launch_side_prepass(lora_plan* pl, const void* S, long long C, const void* s
   g.pt_out = out_t;
   g.ld_t = w.ld_t;
   g.status = pl->d_status;
+    g.wait_limit = pl->wait_limit;
   if (launch_grad(tmS, tmS, tmSide, g, st) != cudaSuccess) return LORA_ERR_CUDA;
   g_launches.fetch_add(grad_is_direct(g) ? 1 : 2);
   return LORA_OK;
@@ -569,6 +571,7 @@ int launch_fwd(lora_plan* pl, const void* X, const void* W, const void* A, const
   p.rt_out = (pair && !ext) ? pt : nullptr;
   p.ld_rt = pl->ws.ld_t;
   p.status = pl->d_status;
+    p.wait_limit = pl->wait_limit;
   const cudaError_t le = ext    ? launch_gemm_pair_fwd_ext(tmX, tmW, tmA, tmB, tmY, p, c.fwd_ctas, st)
                          : pair ? launch_gemm_pair_fwd(tmX, tmW, tmW1, tmA, tmB, tmY, p, c.fwd_ctas, st)
                                 : launch_gemm_fwd(tmX, tmW, tmA, tmB, tmY, p, c.fwd_ctas, st);
@@ -632,6 +635,7 @@ int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const
     p.rt_out = pair ? nullptr : qt;     // the single-CTA kernel computes Q itself and hands it on
     p.ld_rt = w.ld_t;
     p.status = pl->d_status;
+    p.wait_limit = pl->wait_limit;
     const int ctas = ctas_override > 0 ? ctas_override : c.dx_ctas;
     const cudaError_t le = pair ? launch_gemm_pair_dx(tmdY, tmW, tmB, tmA, tmdX, p, ctas, st)
                                 : launch_gemm_dx(tmdY, tmW, tmB, tmA, tmdX, p, ctas, st);
@@ -685,6 +689,7 @@ int launch_da(lora_plan* pl, const void* X, const void* A, float scale, void* dA
     g.pt_out = pt;
     g.ld_t = w.ld_t;
     g.status = pl->d_status;
+    g.wait_limit = pl->wait_limit;
     if (launch_grad(tmS, tmR, tmA, g, st) != cudaSuccess) return LORA_ERR_CUDA;
     g_launches.fetch_add(grad_is_direct(g) ? 1 : 2);
   }
@@ -730,6 +735,7 @@ int launch_db(lora_plan* pl, const void* dY, float scale, void* dB, cudaStream_t
     g.pt_out = with_q ? q.qt : nullptr;
     g.ld_t = w.ld_t;
     g.status = pl->d_status;
+    g.wait_limit = pl->wait_limit;
     if (launch_grad(tmS, tmR, with_q ? tmSide : tmR, g, st) != cudaSuccess) return LORA_ERR_CUDA;
     g_launches.fetch_add(grad_is_direct(g) ? 1 : 2);
   }
@@ -783,6 +789,7 @@ int launch_fwd_nf4(lora_plan* pl, const void* X, const void* codes, const void* 
   p.kb_per_split = p.kblocks;
   p.split_k = 1;
   p.status = pl->d_status;
+    p.wait_limit = pl->wait_limit;
   const int ctas = 2 * (p.num_tiles < pairs ? p.num_tiles : pairs);
   if (launch_gemm_pair_fwd_nf4(tmX, tmCodes, tmAbsmax, tmPt, tmB, tmY, p, ctas, st) != cudaSuccess) return LORA_ERR_CUDA;
   g_launches.fetch_add(1);
@@ -825,6 +832,7 @@ int launch_dx_nf4(lora_plan* pl, const void* dY, const void* codes, const void* 
   p.kb_per_split = p.kblocks;
   p.split_k = 1;
   p.status = pl->d_status;
+    p.wait_limit = pl->wait_limit;
   const int ctas = 2 * (p.num_tiles < pairs ? p.num_tiles : pairs);
   if (launch_gemm_pair_dx_nf4(tmdY, tmCodes, tmAbsmax, tmQt, tmA, tmdX, p, ctas, st) != cudaSuccess) return LORA_ERR_CUDA;
   g_launches.fetch_add(1);
@@ -867,6 +875,7 @@ int launch_dw(lora_plan* pl, const void* dY, const void* X, void* dW, cudaStream
   p.split_k = ceil_div(p.kblocks, p.kb_per_split);
   p.part = (p.split_k > 1) ? reinterpret_cast<float*>(static_cast<uint8_t*>(pl->workspace) + pl->ws.split_part) : nullptr;
   p.status = pl->d_status;
+    p.wait_limit = pl->wait_limit;
   if (launch_gemm_pair_dw(tmdY, tmX, tmdW, p, c.dw_ctas, st) != cudaSuccess) return LORA_ERR_CUDA;
   g_launches.fetch_add(1);
   if (p.split_k > 1) {
@@ -928,6 +937,11 @@ int lora_plan_create(const lora_shape_t* shape, int device, lora_plan_t** out) {
   pl->accumulate = false;
   pl->p_saved = false;
   pl->p_saved_scale = 0.f;
+  pl->wait_limit = kWaitLimitCycles;
+  if (const char* f = std::getenv("LORA_DEBUG_WAIT_CAP")) {     // debugging: shorter limit, in SM clock ticks
+    const long long v = std::atoll(f);
+    if (v >= 1000) pl->wait_limit = v;
+  }
   pl->d_status = nullptr;
   pl->side_stream = nullptr;
   pl->ev_fork = pl->ev_join = nullptr;
@@ -986,6 +1000,43 @@ int lora_plan_set_workspace(lora_plan_t* plan, void* dev_ptr, size_t bytes) {
 int lora_plan_set_grad_accumulation(lora_plan_t* plan, int enable) {
   if (plan == nullptr) return LORA_ERR_INVALID_ARG;
   plan->accumulate = enable != 0;
+  return LORA_OK;
+}
+
+int lora_plan_set_wait_limit(lora_plan_t* plan, int64_t cycles) {
+  if (plan == nullptr || cycles < 0) return LORA_ERR_INVALID_ARG;
+  plan->wait_limit = cycles == 0 ? kWaitLimitCycles : (cycles < 1000 ? 1000 : cycles);
+  return LORA_OK;
+}
+
+int lora_debug_starved_wait(lora_plan_t* plan, const void* S, int64_t T, int64_t C, void* out, void* stream) {
+  if (plan == nullptr || S == nullptr || out == nullptr) return LORA_ERR_INVALID_ARG;
+  if (T < 1 || T > 1024 || C < 8 || C > 512 || C % 8 != 0) return LORA_ERR_UNSUPPORTED_SHAPE;
+  if (!aligned16(S) || !aligned16(out)) return LORA_ERR_MISALIGNED;
+  DeviceGuard guard(plan->device);
+  const int r_pad = plan->cfg.r_pad;
+  CUtensorMap tmS;
+  if (!make_bf16_tmap(&tmS, S, C, T, C, 64, kGradSlab)) return LORA_ERR_CUDA;
+  GradParams g{};
+  g.T = static_cast<int>(T);
+  g.C = static_cast<int>(C);
+  g.r = static_cast<int>(plan->shape.r);
+  g.r_pad = r_pad;
+  g.feat_chunk = ceil_div(C, 128) * 128;
+  g.n_feat_chunks = 1;
+  g.n_token_chunks = 1;              // one CTA, direct mode: nothing but `status` can be written
+  g.n_slabs = ceil_div(T, kGradSlab);
+  g.stages = 2;
+  g.do_out = 1;
+  g.scale = 1.f;
+  g.out = static_cast<float*>(out);
+  g.c_pad = static_cast<int>(C);
+  g.ld_t = static_cast<int>(T);
+  g.status = plan->d_status;
+  g.wait_limit = plan->wait_limit;
+  g.debug_no_second_factor = 1;      // the MMA warp never receives its second factor: its bounded wait runs out
+  if (launch_grad(tmS, tmS, tmS, g, static_cast<cudaStream_t>(stream)) != cudaSuccess) return LORA_ERR_CUDA;
+  g_launches.fetch_add(1);
   return LORA_OK;
 }
 

@@ -111,7 +111,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY   [M, K
       bool ok = true;
       auto acquire = [&]() -> int {
         const int slot = it % S;
-        ok = mbar_wait(empty_bar(slot), ((it / S) & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY);
+        ok = mbar_wait(empty_bar(slot), ((it / S) & 1) ^ 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_EMPTY);
         ++it;
         return slot;
       };
@@ -166,11 +166,11 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY   [M, K
       auto mma_main = [&](int i, int kb) {
         const int buf = i & 1, use = i >> 1;
         if (kb == 0) {
-          ok = mbar_wait(acc_empty(buf), (use & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_ACC_EMPTY);
+          ok = mbar_wait(acc_empty(buf), (use & 1) ^ 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_ACC_EMPTY);
           if (!ok) return;
         }
         const int slot = it % S;
-        ok = mbar_wait(full_bar(slot), (it / S) & 1, abort_flag, p.status, DEV_TIMEOUT_FULL);
+        ok = mbar_wait(full_bar(slot), (it / S) & 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_FULL);
         ++it;
         if (!ok) return;
         tc_fence_after();
@@ -187,10 +187,10 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY   [M, K
       };
       auto mma_tail = [&](int i) {
         const int buf = i & 1, use = i >> 1;
-        ok = mbar_wait(ps_ready(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_PS);
+        ok = mbar_wait(ps_ready(buf), use & 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_PS);
         if (!ok) return;
         const int slot = it % S;
-        ok = mbar_wait(full_bar(slot), (it / S) & 1, abort_flag, p.status, DEV_TIMEOUT_FULL);
+        ok = mbar_wait(full_bar(slot), (it / S) & 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_FULL);
         ++it;
         if (!ok) return;
         tc_fence_after();
@@ -225,7 +225,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY   [M, K
       const int m0 = tc.m_idx * kBlockM, n0 = tc.n_idx * p.block_n;
       const int buf = i & 1, use = i >> 1;
       if (e == 0) tma_store_wait_read<0>();       // staging[0] is about to hold the rank-r operand
-      bool ok = mbar_wait(side_full(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_SIDE);
+      bool ok = mbar_wait(side_full(buf), use & 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_SIDE);
       if (named_bar_or(1, 128, !ok)) break;
       tc_fence_after();
       // ---- P (or Q) : TMEM -> scale -> bf16 -> shared memory (K-major, 128-byte swizzle) ----
@@ -253,7 +253,7 @@ lora_gemm_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY   [M, K
       tc_fence_before();
       mbar_arrive(ps_ready(buf));
       // ---- accumulator: TMEM -> bf16 -> swizzled staging -> TMA store, 64 columns at a time ----
-      ok = mbar_wait(acc_full(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_ACC);
+      ok = mbar_wait(acc_full(buf), use & 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_ACC);
       if (named_bar_or(1, 128, !ok)) break;
       tc_fence_after();
       for (int c = 0; c < n_chunks; ++c) {

@@ -172,7 +172,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
     // claims the next ring item; returns its slot or -1 when the item belongs to the other warp pair
     auto acquire = [&]() -> int {
       const int mine = (odd == par), cur = slot;
-      if (mine) ok = warp_wait(empty_bar(cur), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY, false, 20);
+      if (mine) ok = warp_wait(empty_bar(cur), phase ^ 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_EMPTY, false, 20);
       if (++slot == S) { slot = 0; phase ^= 1; }
       odd ^= 1;
       return mine ? cur : -1;
@@ -258,7 +258,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
         const int kb0 = sp * p.kb_per_split, kb1 = min(KB, kb0 + p.kb_per_split);
         for (int kb = kb0; kb < kb1 && ok; ++kb) {
           if (codd == par) {
-            ok = warp_wait(cempty_bar(cslot), cphase ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY, false, 20);
+            ok = warp_wait(cempty_bar(cslot), cphase ^ 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_EMPTY, false, 20);
             if (ok && elect_one()) {
               const uint32_t cdst = smem_u32(code_ring) + cslot * kNf4CodeSlotBytes, cb = cfull_bar(cslot);
               mbar_arrive_expect_tx(cb, kNf4CodeSlotBytes);
@@ -313,7 +313,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       bool ok = true;
       auto next = [&]() { if (++slot == S) { slot = 0; phase ^= 1; } };
       auto mma_main = [&](int buf, bool first_kb, bool last_kb, bool has_tail) {
-        ok = warp_wait(full_bar(slot), phase, abort_flag, p.status, DEV_TIMEOUT_FULL, true, 0);
+        ok = warp_wait(full_bar(slot), phase, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_FULL, true, 0);
         if (!ok) return;
         tc_fence_after();
         if (elect_one()) {
@@ -333,8 +333,8 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
         next();
       };
       auto mma_tail = [&](int buf, int use) {
-        if (!kExt) ok = warp_wait(ps_ready(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_PS, true, 0);
-        if (ok) ok = warp_wait(full_bar(slot), phase, abort_flag, p.status, DEV_TIMEOUT_FULL, true, 0);
+        if (!kExt) ok = warp_wait(ps_ready(buf), use & 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_PS, true, 0);
+        if (ok) ok = warp_wait(full_bar(slot), phase, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_FULL, true, 0);
         if (!ok) return;
         tc_fence_after();
         if (elect_one()) {
@@ -352,7 +352,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
         const int sp = (pair + i * G) % SK;
         const int kb0 = sp * p.kb_per_split, kb1 = min(KB, kb0 + p.kb_per_split);
         const bool has_tail = !kExt || (sp == SK - 1 && p.r_pad > 0);
-        ok = warp_wait(acc_empty(buf), (use & 1) ^ 1, abort_flag, p.status, DEV_TIMEOUT_ACC_EMPTY, true, 0);
+        ok = warp_wait(acc_empty(buf), (use & 1) ^ 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_ACC_EMPTY, true, 0);
         for (int kb = kb0; kb < kb1 && ok; ++kb) {
           if (!kExt && i > 0 && kb == D) mma_tail(buf ^ 1, (i - 1) >> 1);
           if (ok) mma_main(buf, kb == kb0, kb == kb1 - 1, has_tail);
@@ -387,8 +387,8 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       for (int kb = kb0; kb < kb1 + (has_tail ? 1 : 0) && ok; ++kb) {
         const bool main_item = kb < kb1;
         if (turn == gid) {
-          if (main_item) ok = warp_wait(cfull_bar(cslot), cphase, abort_flag, p.status, DEV_TIMEOUT_FULL, false, 0);
-          if (ok) ok = warp_wait(empty_bar(slot), phase ^ 1, abort_flag, p.status, DEV_TIMEOUT_EMPTY, false, 0);
+          if (main_item) ok = warp_wait(cfull_bar(cslot), cphase, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_FULL, false, 0);
+          if (ok) ok = warp_wait(empty_bar(slot), phase ^ 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_EMPTY, false, 0);
           if (!ok) break;
           if (main_item) {
             (void)mbar_try_wait(cfull_bar(cslot), cphase);     // every reading thread observes the completed copy itself
@@ -449,7 +449,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       if (e == 0) tma_store_wait_read<0>();       // the previous tile's stores have left both staging buffers
       if (!kExt) {
         // ---- fused forward: P = X A^T from TMEM -> scale -> bf16 -> shared memory as the rank-r MMA operand ----
-        ok = warp_wait(side_full(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_SIDE, false, 64);
+        ok = warp_wait(side_full(buf), use & 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_SIDE, false, 64);
         if (named_bar_or(1, 128, !ok)) break;
         tc_fence_after();
         for (int c16 = 0; c16 < p.r_pad / 16; ++c16) {
@@ -476,7 +476,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
         tc_fence_before();
         mbar_arrive_cluster(map_to_cta(ps_ready(buf), 0));
       }
-      ok = warp_wait(acc_full(buf), use & 1, abort_flag, p.status, DEV_TIMEOUT_ACC, false, 32);
+      ok = warp_wait(acc_full(buf), use & 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_ACC, false, 32);
       if (named_bar_or(1, 128, !ok)) break;
       tc_fence_after();
       if (kExt && SK > 1) {

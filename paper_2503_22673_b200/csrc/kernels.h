@@ -27,6 +27,9 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
+// Default limit of every device-side spin, in SM clock ticks (~2 s at 2 GHz)
+constexpr long long kWaitLimitCycles = 4000000000LL;
+
 // ---- dense GEMM + fused rank-r adapter (forward Y, backward dX) -------------------------------
 constexpr int kBlockM = 128;          // token rows per tile (one TMEM lane per row)
 constexpr int kBlockK = 64;           // contraction elements per stage (one 128-byte swizzle row)
@@ -51,6 +54,7 @@ struct GemmParams {
   __nv_bfloat16* rt_out;  // backward only: scale * (dY B)^T as bf16 [r_pad][ld_rt]; nullptr otherwise
   int ld_rt;
   unsigned* status;       // device status word
+  long long wait_limit;   // SM clock ticks after which a spin gives up and reports through `status`
   int split_k;            // K-extended pair kernel: k-splits per tile (1 = none) and main k-blocks per split
   int kb_per_split;
   float* part;            // fp32 partial tiles [split_k][M][N] when split_k > 1
@@ -149,6 +153,8 @@ struct GradParams {
   __nv_bfloat16* pt_out;  // [r_pad][ld_t]: scale * (X A^T)^T as bf16 (with_p)
   int ld_t;
   unsigned* status;
+  long long wait_limit;   // SM clock ticks after which a spin gives up and reports through `status`
+  int debug_no_second_factor;   // test hook: the second-factor loader issues nothing, so the MMA warp's wait runs out
 };
 
 size_t grad_smem_bytes(const GradParams& p);

@@ -22,8 +22,8 @@ enum DevStatus : unsigned {
   DEV_TIMEOUT_OTHER = 7u,
 };
 
-// ~2 s at 2 GHz; every spin gives up after this many clock ticks
-__device__ constexpr long long kWaitLimitCycles = 4000000000LL;
+// Every spin gives up after `limit` SM clock ticks, a launch parameter (`wait_limit` of the kernel's parameter block;
+// default kWaitLimitCycles of kernels.h), so that a test can make a wait run out within a millisecond.
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -69,13 +69,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait.  Returns false when the limit ran out or another thread of the CTA already
 // gave up (abort_flag); the first thread to give up records `code` in *status.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          unsigned* status, unsigned code) {
+                                          unsigned* status, long long limit, unsigned code) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitCycles) {
+    if (clock64() - t0 > limit) {
       *abort_flag = 1;
       atomicCAS(status, 0u, code | (static_cast<unsigned>(blockIdx.x) << 8));
       return false;
@@ -86,7 +86,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // One lane polls, the rest of the warp sleeps in the shuffle: waiting warps must not eat the issue slots of
 // the warp that feeds the tensor pipe.  `backoff_ns` > 0 adds a nanosleep between polls (long waits).
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status,
-                                          unsigned code, bool cluster_scope, unsigned backoff_ns) {
+                                          long long limit, unsigned code, bool cluster_scope, unsigned backoff_ns) {
   int ok = 1;
   if ((threadIdx.x & 31) == 0) {
     auto probe = [&]() {
@@ -106,7 +106,7 @@ __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatil
         if (probe()) break;
         if (backoff_ns) __nanosleep(backoff_ns);
         if (*abort_flag) { ok = 0; break; }
-        if (clock64() - t0 > kWaitLimitCycles) {
+        if (clock64() - t0 > limit) {
           *abort_flag = 1;
           atomicCAS(status, 0u, code | (static_cast<unsigned>(blockIdx.x) << 8));
           ok = 0;
@@ -344,13 +344,13 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
 }
 // bounded wait on a barrier that CTAs of the whole cluster arrive on
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                                  unsigned* status, unsigned code) {
+                                                  unsigned* status, long long limit, unsigned code) {
   if (mbar_try_wait_cluster(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
     if (mbar_try_wait_cluster(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitCycles) {
+    if (clock64() - t0 > limit) {
       *abort_flag = 1;
       atomicCAS(status, 0u, code | (static_cast<unsigned>(blockIdx.x) << 8));
       return false;

@@ -1,10 +1,14 @@
 """GPU parity at the full benchmark sizes, in the launch configuration bench.py times (default plan).
 
-The oracle cannot produce a full 16384 x 14336 output in seconds, so Y and dX are compared on sampled token rows
-(rows are independent: oracle.forward_rows / backward_dx_rows compute them one by one; every column tile is
-covered because whole rows are compared, and the sample holds the first and last row of the matrix, rows on both
-sides of tile borders and random ones).  dA and dB are compared in full.  Two adjoint identities that hold at
-any size are checked on the GPU outputs as a whole:  <dY, Y> = <dX, X>  and  <dA, A> = <dB, B>.
+Single-projection workloads (q_proj, gate/up_proj, down_proj): the WHOLE of Y and dX is compared element by element
+with the oracle, which is evaluated in blocks of 2048 token rows so that the float64 arrays stay small (token rows are
+independent); the error measure max|gpu - ref| / max|ref| is taken over the complete matrix.  The same holds for all
+seven projections of the whole-layer workload (T = 32768).  The paper's own r = 32 setting (T = 49152), the dense
+weight gradient and the NF4 weight are compared on a dense row sample:
+two rows of every 128-row slab (so every tile row, every persistent-loop position and both TMEM accumulator buffers are
+hit), the rows on both sides of the tile borders, the first and the last row; all columns of each sampled row.
+dA and dB are always compared in full.  Two adjoint identities that hold at any size are checked on the GPU outputs as
+a whole:  <dY, Y> = <dX, X>  and  <dA, A> = <dB, B>.
 
 Tolerances: max|gpu - ref| / max|ref| <= 2e-2 (Y, dX, bf16), <= 5e-3 (dA, dB, fp32).
 """
@@ -38,11 +42,36 @@ def sample_rows(T, n_random=40, seed=0):
     return np.asarray(rows, dtype=np.int64)
 
 
+def slab_rows(T, seed=0, slab=128):
+    """Two rows of every `slab`-row slab (one at a position that walks through the slab, one random) plus the border rows."""
+    rng = np.random.default_rng(seed)
+    n = -(-T // slab)
+    walk = np.arange(n) * slab + (np.arange(n) * 37) % slab
+    rnd = np.arange(n) * slab + rng.integers(0, slab, n)
+    rows = np.concatenate([walk, rnd, sample_rows(T, 0)])
+    return np.unique(rows[rows < T]).astype(np.int64)
+
+
+BLOCK_ROWS = 2048
+
+
+def full_rel_err(gpu, act_bits, ref_rows_fn):
+    """max|gpu - ref| / max|ref| over the complete [T, n] matrix, the oracle evaluated BLOCK_ROWS token rows at a time."""
+    num = den = 0.0
+    for lo in range(0, act_bits.shape[0], BLOCK_ROWS):
+        hi = min(lo + BLOCK_ROWS, act_bits.shape[0])
+        ref = ref_rows_fn(inputs.bf16_to_f64(act_bits[lo:hi]))
+        got = host64(gpu[lo:hi])
+        num = max(num, float(np.max(np.abs(got - ref))))
+        den = max(den, float(np.max(np.abs(ref))))
+    return num / den if den > 0 else (0.0 if num == 0 else float("inf"))
+
+
 def dot64(a, b):
     return float((a.double() * b.double()).sum().item())
 
 
-def check_projection(p, t, x_dev=None):
+def check_projection(p, t, x_dev=None, whole=False):
     d = {k: dev(v) for k, v in t.items() if k != "X"}
     d["X"] = x_dev if x_dev is not None else dev(t["X"])
     plan = binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r)
@@ -50,14 +79,19 @@ def check_projection(p, t, x_dev=None):
     dX, dA, dB = plan.bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], p.scale)
     code, msg = plan.device_status()
     assert code == 0, msg
-    rows = sample_rows(p.T)
     W, A, B = (inputs.bf16_to_f64(t[k]) for k in ("W", "A", "B"))
-    rows_t = torch.from_numpy(rows).cuda()
-    # ---- sampled rows of Y and dX ----
-    Yr = oracle.forward_rows(np.arange(len(rows)), inputs.bf16_to_f64(t["X"][rows]), W, A, B, p.scale)
-    dXr = oracle.backward_dx_rows(np.arange(len(rows)), inputs.bf16_to_f64(t["dY"][rows]), W, A, B, p.scale)
-    eY = oracle.rel_err(host64(Y[rows_t]), Yr)
-    eX = oracle.rel_err(host64(dX[rows_t]), dXr)
+    if whole:
+        # ---- every element of Y and dX ----
+        eY = full_rel_err(Y, t["X"], lambda xb: oracle.forward(xb, W, A, B, p.scale))
+        eX = full_rel_err(dX, t["dY"], lambda gb: oracle.backward_dx_rows(np.arange(gb.shape[0]), gb, W, A, B, p.scale))
+    else:
+        # ---- two rows of every 128-row slab + border rows of Y and dX ----
+        rows = slab_rows(p.T)
+        rows_t = torch.from_numpy(rows).cuda()
+        Yr = oracle.forward_rows(np.arange(len(rows)), inputs.bf16_to_f64(t["X"][rows]), W, A, B, p.scale)
+        dXr = oracle.backward_dx_rows(np.arange(len(rows)), inputs.bf16_to_f64(t["dY"][rows]), W, A, B, p.scale)
+        eY = oracle.rel_err(host64(Y[rows_t]), Yr)
+        eX = oracle.rel_err(host64(dX[rows_t]), dXr)
     del W
     # ---- adapter gradients in full ----
     Xf = inputs.bf16_to_f64(t["X"])
@@ -89,7 +123,7 @@ def check_projection(p, t, x_dev=None):
 @pytest.mark.parametrize("idx", [1, 2, 3])
 def test_single_projection_workloads_full_size(idx):
     (p, t), = list(inputs.draw_workload(idx, seed=0))
-    check_projection(p, t)
+    check_projection(p, t, whole=True)
 
 
 def test_seven_projection_layer_full_size():
@@ -98,7 +132,7 @@ def test_seven_projection_layer_full_size():
         if p.x_group not in x_dev:
             x_dev.clear()
             x_dev[p.x_group] = dev(t["X"])
-        check_projection(p, t, x_dev[p.x_group])
+        check_projection(p, t, x_dev[p.x_group], whole=True)
 
 
 # ---------------------------------------------------------------------------------------------
@@ -106,8 +140,8 @@ def test_seven_projection_layer_full_size():
 # ---------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("idx", [1, 3])
 def test_dense_dw_full_size_sampled(idx):
-    """dW = dY^T X at the benchmark sizes: sampled rows of dW (each row o is dY[:, o]^T X, one fp64 matrix-vector
-    product) against the oracle's definition, rows on both sides of the 128/256-row tile borders included; plus the
+    """dW = dY^T X at the benchmark sizes: two rows of every 128-row slab of dW (each row o is dY[:, o]^T X, one fp64
+    matrix-vector product) against the oracle's definition, rows on both sides of the tile borders included; plus the
     identity  <dW, M> = <dY, X M^T>  for a random bf16 M on the complete output (fp64 on the device)."""
     (p, t), = list(inputs.draw_workload(idx, seed=0))
     X, dY = dev(t["X"]), dev(t["dY"])
@@ -115,7 +149,7 @@ def test_dense_dw_full_size_sampled(idx):
     dW = plan.dense_dw(dY, X)
     code, msg = plan.device_status()
     assert code == 0, msg
-    rows = sample_rows(p.d_out, n_random=24, seed=1)
+    rows = slab_rows(p.d_out, seed=1)
     Xf = inputs.bf16_to_f64(t["X"])
     ref = oracle.dense_weight_grad(inputs.bf16_to_f64(t["dY"][:, rows]), Xf)
     del Xf
@@ -135,7 +169,7 @@ def test_dense_dw_full_size_sampled(idx):
 @pytest.mark.parametrize("use_scratch", [True, False], ids=["scratch", "in_kernel"])
 def test_nf4_full_size_config1(use_scratch):
     """Q+LoRA at the q_proj size (T = 8192, 4096 -> 4096, r = 16): the GPU quantiser's codes and scales must equal the
-    oracle's bit for bit; Y and dX on sampled rows and dA, dB in full against the oracle on the dequantised weight."""
+    oracle's bit for bit; Y and dX on two rows of every 128-row slab and dA, dB in full against the oracle on the dequantised weight."""
     from oracle import nf4_oracle as nf4
     (p, t), = list(inputs.draw_workload(1, seed=0))
     d = {k: dev(v) for k, v in t.items()}
@@ -148,7 +182,7 @@ def test_nf4_full_size_config1(use_scratch):
     dX, dA, dB = plan.bwd_nf4(d["dY"], d["X"], codes, absmax, d["A"], d["B"], p.scale, w_scratch=scratch)
     code, msg = plan.device_status()
     assert code == 0, msg
-    rows = sample_rows(p.T)
+    rows = slab_rows(p.T)
     rows_t = torch.from_numpy(rows).cuda()
     What, A, B = nf4.dequantize(ref_codes, ref_absmax), inputs.bf16_to_f64(t["A"]), inputs.bf16_to_f64(t["B"])
     Yr = oracle.forward_rows(np.arange(len(rows)), inputs.bf16_to_f64(t["X"][rows]), What, A, B, p.scale)

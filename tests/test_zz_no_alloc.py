@@ -1,10 +1,12 @@
-"""The allocation-free contraction entry point against the planned backward pass.
+"""The allocation-free contraction entry point, against the plain definition and the planned backward pass.
 
-Some users of the library cannot allocate device memory at call time (a fixed pool, a latency-critical
-loop).  For them `lora_grad_contract_noalloc` keeps its scratch in a static device array.  This test calls
-it through the C ABI twice in a row - the array is shared and keeps old contents, so the second call would
-expose anything left uncleared - and compares with dB from `lora_linear_bwd`, within the fp32 adapter
-gradient tolerance used everywhere else (5e-3 of the largest entry).
+Some users of the library cannot allocate device memory at call time (a fixed pool that forbids cudaMalloc after
+start-up, a latency-critical loop).  For them `lora_grad_contract_noalloc` keeps its scratch in a static device
+array.  This test calls it through the C ABI twice in a row - the array is shared and keeps old contents, so the
+second call would expose anything left uncleared - and compares the result
+  * with the definition  out[c, j] = sum_t S[t, c] Rt[j, t]  evaluated in float64 on the very bf16 values passed in, and
+  * with dB from `lora_linear_bwd` (the existing entry point that runs the same contraction with planned scratch),
+both within the fp32 adapter-gradient tolerance used everywhere else (5e-3 of the largest entry).
 """
 import gc
 
@@ -26,43 +28,80 @@ def _rel(a, b):
     return float((a - b).abs().max() / b.abs().max())
 
 
-def test_noalloc_contraction_matches_planned_backward_twice():
+def _second_factor(t, s, ld):
+    """bf16 bit patterns of scale * (X A^T)^T, [r, ld] with zero padding past T, and the same values in float64."""
+    Xf, Af = inputs.bf16_to_f64(t["X"]), inputs.bf16_to_f64(t["A"])
+    P = (s * (Xf @ Af.T)).T.astype(np.float32)                       # [r, T]
+    bits = np.zeros((P.shape[0], ld), dtype=np.uint16)
+    bits[:, :P.shape[1]] = inputs.f32_to_bf16_bits(P)
+    return bits, inputs.bf16_to_f64(bits[:, :P.shape[1]])
+
+
+CASES = [
+    # T, d_in, d_out, r, scale, seed, ld - T
+    (1500, 520, 1032, 16, 2.0, 21, 4),      # several feature chunks and token chunks, partial sums in the static array
+    (900, 264, 392, 32, 0.5, 22, 4),
+    (700, 136, 200, 8, 2.0, 23, 36),        # r = 8: rows 8..15 of the second-factor box lie outside Rt (zero fill); ld > T
+    (100, 72, 136, 24, 1.0, 24, 4),         # one slab: a single token chunk, the kernel writes `out` itself
+]
+
+
+def test_noalloc_contraction_matches_definition_and_planned_backward_twice():
     lib = binding.load()
     assert lib.lora_grad_contract_noalloc_max_scratch() == 8 << 20
-    cases = [(1500, 520, 1032, 16, 2.0, 21), (900, 264, 392, 32, 0.5, 22)]
-    for T, d_in, d_out, r, s, seed in cases:
+    for T, d_in, d_out, r, s, seed, extra in CASES:
         p, t = inputs.draw_custom(T, d_in, d_out, r, s, seed=seed)
         d = {k: _dev(v) for k, v in t.items()}
         plan = binding.LoraLinearPlan(T, d_in, d_out, r)
-        _, _, dB_ref = plan.bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], s)
+        _, _, dB_planned = plan.bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], s)
         torch.cuda.synchronize()
-        # the second factor the planned path builds internally: scale * (X A^T)^T rounded to bf16, [r, ld]
-        ld = (T + 7) // 8 * 8
-        Pt = torch.zeros((r, ld), dtype=torch.bfloat16, device="cuda")
-        Pt[:, :T] = ((d["X"].float() @ d["A"].float().t()) * s).t().to(torch.bfloat16)
+        ld = (T + extra + 7) // 8 * 8
+        pt_bits, pt64 = _second_factor(t, s, ld)
+        Pt = _dev(pt_bits)
+        expected = torch.from_numpy(inputs.bf16_to_f64(t["dY"]).T @ pt64.T).cuda()      # [d_out, r], float64
         for call in range(2):
             out = torch.full((d_out, r), float("nan"), dtype=torch.float32, device="cuda")
             gc.collect()                                           # tensors of earlier tests go now, not during the call
             torch.cuda.synchronize()
-            before = torch.cuda.memory_allocated()
+            before, free_before = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
             binding.grad_contract_noalloc(d["dY"], Pt, out)
             torch.cuda.synchronize()
-            assert torch.cuda.memory_allocated() <= before        # nothing was taken from torch's allocator
+            assert torch.cuda.memory_allocated() <= before        # nothing was taken from torch's allocator ...
+            if call == 1:                                          # ... nor from the driver (the first call on a device may
+                assert torch.cuda.mem_get_info()[0] >= free_before  # load the kernel; the second one must not move it)
+            assert binding.grad_contract_noalloc_status() == binding.LORA_OK
             assert not torch.isnan(out).any(), (T, call)
-            assert _rel(out, dB_ref) <= TOL_F32, (T, d_out, r, call, _rel(out, dB_ref))
+            assert _rel(out.double(), expected) <= TOL_F32, (T, d_out, r, call, _rel(out.double(), expected))
+            assert _rel(out, dB_planned) <= TOL_F32, (T, d_out, r, call, _rel(out, dB_planned))
             del out
         plan.close()
+
+
+def test_noalloc_contraction_wide_rank64_runs_with_fewer_token_chunks():
+    """16384 x 4096 with r = 64: the full grid's partial sums (24 token chunks x 1 MiB) exceed the 8 MiB array, so the
+    call runs with the 7 token chunks that fit instead of refusing.  Checked against the float64 definition."""
+    T, C, r = 16384, 4096, 64
+    g = np.random.Generator(np.random.Philox(key=77))
+    s_bits = inputs.f32_to_bf16_bits(g.standard_normal((T, C), dtype=np.float32))
+    r_bits = inputs.f32_to_bf16_bits(g.standard_normal((r, T), dtype=np.float32))
+    S, Rt = _dev(s_bits), _dev(r_bits)
+    expected = torch.from_numpy(inputs.bf16_to_f64(s_bits).T @ inputs.bf16_to_f64(r_bits).T).cuda()
+    for call in range(2):
+        out = torch.full((C, r), float("nan"), dtype=torch.float32, device="cuda")
+        binding.grad_contract_noalloc(S, Rt, out)
+        assert binding.grad_contract_noalloc_status() == binding.LORA_OK
+        assert _rel(out.double(), expected) <= TOL_F32, (call, _rel(out.double(), expected))
 
 
 def test_noalloc_contraction_rejects_what_does_not_fit():
     lib = binding.load()
     stream = torch.cuda.current_stream().cuda_stream
     # real, fully sized tensors: nothing can be touched out of bounds whatever the call decides
-    T, C, r = 16384, 4096, 64
+    T, C, r = 128, 40000, 64
     S = torch.zeros((T, C), dtype=torch.bfloat16, device="cuda")
     Rt = torch.zeros((r, T), dtype=torch.bfloat16, device="cuda")
     o = torch.zeros((C, r), dtype=torch.float32, device="cuda")
-    # 16 feature chunks x 9 token chunks x 64 x 4096 fp32 partial sums = 9.4 MiB > the 8 MiB static array
+    # one layer of partial sums, 64 x 40000 floats = 9.8 MiB, is more than the 8 MiB static array holds
     rc = lib.lora_grad_contract_noalloc(S.data_ptr(), Rt.data_ptr(), T, C, r, T, o.data_ptr(), stream)
     assert rc == binding.LORA_ERR_WORKSPACE
     rc = lib.lora_grad_contract_noalloc(S.data_ptr(), Rt.data_ptr(), 128, 60, 16, 128, o.data_ptr(), stream)
