@@ -1,15 +1,18 @@
 #!/usr/bin/env python
 """Throughput of the LoRA projection layer (forward + backward) on B200.
 
-A step is one pass of the whole hot path - forward GEMM with the fused adapter, dX GEMM with the fused
-adapter, dA kernel, dB kernel - over one batch of seeded synthetic input.  The default workload is the
-Llama-3-8B q_proj shape (T = 8192 packed tokens, 4096 -> 4096, r = 16, s = 2).
+A step is one pass of the whole hot path - forward (X A^T pass + GEMM with the rank-r product as an extra k-block, or the
+fused kernel), then backward (dY B and X A^T in one skinny launch, the dX GEMM, dA and dB in one skinny launch) - for every
+projection of the workload, over one batch of seeded synthetic input.  The default workload is the whole Llama-3-8B decoder
+layer: seven projections (q, k, v, o, gate, up, down), T = 32768 packed tokens, r = 16, s = 2.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload {0..4}] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload {0..5}] [--impl reference] [--quick]
 
-Prints ONE JSON line.  With N > 1 (torchrun, one rank per GPU) every rank runs an independent replica
-on its own batch: the layer has no collective, so the job's value is the sum over ranks divided by the
-slowest rank's time.
+Prints ONE JSON line: the headline workload's timed region (`value`), the same step looped for >= 2 s (`sustained`), per-stage
+durations with their roofline fractions (`kernels`, `roofline`, `roofline_hbm`), the other workloads from short runs in the
+same process (`per_config`), variants, the end-to-end figure with host buffers, and the CPU oracle timed beside it.
+With N > 1 (torchrun, one rank per GPU) every rank runs an independent replica on its own batch: the layer has no collective,
+so the job's value is the sum over ranks divided by the slowest rank's time.
 """
 from __future__ import annotations
 
@@ -33,9 +36,11 @@ L2_BYTES = 126 * 1024 * 1024
 METRIC = "lora_linear_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel from an
-# ncu capture summarised under profiles/; only valid for the kernel source it was taken on.
-NCU_TRAFFIC = {"gemm_sha": "7c3994e03b7d900f", "bytes_per_launch": {"fwd_gemm": 221.3e6, "dx_gemm": 219.7e6}}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the ncu captures summarised under profiles/;
+# each entry is valid only for the kernel source it was taken on (sha of the files named in *_source_sha) and for the
+# projection shape it names.  GEMM: dX GEMM of a 32768 x 4096 x 14336 projection; stream: the dA + dB launch of q_proj at
+# T = 32768 (captured at T = 8192 and scaled by the tokens: the traffic is the two streamed matrices, proportional to T).
+NCU_TRAFFIC = {"gemm_sha": "", "gemm_bytes_per_launch": {}, "stream_sha": "", "stream_bytes_per_launch": {}}
 
 
 def peaks():
@@ -48,11 +53,12 @@ def peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
-def gemm_source_sha() -> str:
+def source_sha(prefix: str) -> str:
+    """sha of the kernel sources whose names start with `prefix` plus the shared headers (keys the stored ncu traffic)."""
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2503_22673_b200", "csrc")
     for name in sorted(os.listdir(csrc)):
-        if name.startswith("gemm") or name in ("sm100_ptx.cuh", "kernels.h"):
+        if name.startswith(prefix) or name in ("sm100_ptx.cuh", "kernels.h"):
             with open(os.path.join(csrc, name), "rb") as f:
                 h.update(f.read())
     return h.hexdigest()[:16]
@@ -106,11 +112,17 @@ class ClockSampler:
                              [n for n, v in zip(names, parts[3:7]) if v.lower().startswith("active")]))
             except ValueError:
                 continue
+        self.rows = rows
+        return self.window(t0, t1)
+
+    def window(self, t0: float = None, t1: float = None, label: str = "timed region"):
+        rows = getattr(self, "rows", [])
         inside = [r for r in rows if t0 is not None and r[0] is not None and t0 <= r[0] <= t1]
-        window = "timed region" if inside else "whole run (no sample fell inside the timed region)"
+        window = label if inside else f"whole run (no sample fell inside the {label})"
         use = inside if inside else rows
         sm = [r[1] for r in use]
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(r[2] for r in use) if use else None,
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_min_mhz": min(sm) if sm else None,
+                "sm_max_mhz": max(r[2] for r in use) if use else None,
                 "samples": len(use), "window": window, "reasons": sorted({n for r in use for n in r[3]})}
 
 
@@ -154,68 +166,79 @@ def blas_threads() -> int:
     return len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
 
 
-def oracle_step_time(proj, f64, rows: int) -> float:
-    """One oracle forward + backward on the first `rows` token rows (all of W, A, B)."""
-    from oracle import lora_oracle as oracle
-    X, dY = f64["X"][:rows], f64["dY"][:rows]
-    t0 = time.perf_counter()
-    oracle.forward(X, f64["W"], f64["A"], f64["B"], proj.scale)
-    oracle.backward(dY, X, f64["W"], f64["A"], f64["B"], proj.scale)
-    return time.perf_counter() - t0
-
-
 def sample_flops(proj, rows: int) -> float:
     return 4.0 * rows * proj.d_in * proj.d_out + 6.0 * rows * proj.r * (proj.d_in + proj.d_out)
 
 
 def oracle_inputs(workload_idx: int, max_rows: int):
+    """The first `max_rows` token rows of every projection of the workload, widened to float64 (full W, A, B)."""
     from paper_2503_22673_b200 import inputs
-    proto = inputs.workload(workload_idx)[0]
-    rows = min(proto.T, max_rows)
-    proj, t = next(iter(inputs.draw_workload(workload_idx, seed=0, T=rows)))
-    f64 = {k: inputs.bf16_to_f64(v) for k, v in t.items()}
-    return proto, proj, f64, rows
+    protos = inputs.workload(workload_idx)
+    rows = min(protos[0].T, max_rows)
+    drawn = []
+    for proj, t in inputs.draw_workload(workload_idx, seed=0, T=rows):
+        drawn.append((proj, {k: inputs.bf16_to_f64(v) for k, v in t.items()}))
+    return protos, drawn, rows
 
 
-def pick_rows(proj, f64, avail: int, budget_s: float) -> int:
+def oracle_step_time(drawn, rows: int) -> float:
+    """One oracle forward + backward of every projection on its first `rows` token rows."""
+    from oracle import lora_oracle as oracle
+    t0 = time.perf_counter()
+    for proj, f64 in drawn:
+        X, dY = f64["X"][:rows], f64["dY"][:rows]
+        oracle.forward(X, f64["W"], f64["A"], f64["B"], proj.scale)
+        oracle.backward(dY, X, f64["W"], f64["A"], f64["B"], proj.scale)
+    return time.perf_counter() - t0
+
+
+def pick_rows(drawn, avail: int, budget_s: float) -> int:
     cal = min(avail, 128)
-    t_cal = oracle_step_time(proj, f64, cal)              # calibration (also warms the BLAS pool)
-    t_cal = min(t_cal, oracle_step_time(proj, f64, cal))
+    t_cal = oracle_step_time(drawn, cal)                  # calibration (also warms the BLAS pool)
+    t_cal = min(t_cal, oracle_step_time(drawn, cal))
     rows = int(budget_s / max(t_cal / cal, 1e-9))
-    rows = min(avail, max(cal, rows - rows % 128))
-    return rows
+    return min(avail, max(cal, rows - rows % 128))
 
 
 def cpu_baseline(workload_idx: int, budget_s: float = 12.0):
-    proto, proj, f64, avail = oracle_inputs(workload_idx, 4096)
-    rows = pick_rows(proj, f64, avail, budget_s)
-    t = oracle_step_time(proj, f64, rows)
-    return {"value": sample_flops(proto, rows) / t / 1e12, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-            "sample": f"{proto.name}: {rows} of {proto.T} token rows, full W/A/B, fp64 numpy, one fwd+bwd in {t:.2f} s",
+    protos, drawn, avail = oracle_inputs(workload_idx, 2048 if len(inputs_workload(workload_idx)) > 1 else 4096)
+    rows = pick_rows(drawn, avail, budget_s)
+    t = oracle_step_time(drawn, rows)
+    flops = sum(sample_flops(p, rows) for p in protos)
+    names = "+".join(p.name for p in protos)
+    return {"value": flops / t / 1e12, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+            "sample": f"{names}: {rows} of {protos[0].T} token rows of every projection, full W/A/B, fp64 numpy, one fwd+bwd in {t:.2f} s",
             "tokens_per_s": rows / t}
+
+
+def inputs_workload(idx):
+    from paper_2503_22673_b200 import inputs
+    return inputs.workload(idx)
 
 
 def run_reference(args):
     rank, _, _ = dist_env()
     if rank != 0:
         return
-    proto, proj, f64, avail = oracle_inputs(args.workload, 4096)
+    protos, drawn, avail = oracle_inputs(args.workload, 2048 if len(inputs_workload(args.workload)) > 1 else 4096)
     total_steps = max(args.steps + args.warmup, 1)
-    rows = pick_rows(proj, f64, avail, min(3.0, 100.0 / total_steps))
+    rows = pick_rows(drawn, avail, min(3.0, 100.0 / total_steps))
     for _ in range(args.warmup):
-        oracle_step_time(proj, f64, rows)
+        oracle_step_time(drawn, rows)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle_step_time(proj, f64, rows)
+        oracle_step_time(drawn, rows)
     dt = time.perf_counter() - t0
-    value = sample_flops(proto, rows) * args.steps / dt / 1e12
-    sample = f"{proto.name}: {rows} of {proto.T} token rows per step, full W/A/B, fp64 numpy"
+    flops = sum(sample_flops(p, rows) for p in protos)
+    value = flops * args.steps / dt / 1e12
+    sample = (f"{'+'.join(p.name for p in protos)}: {rows} of {protos[0].T} token rows of every projection per step, "
+              "full W/A/B, fp64 numpy")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / max(args.steps, 1) * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": workload_name(args.workload), "T": proto.T, "d_in": proto.d_in, "d_out": proto.d_out,
-                   "r": proto.r, "scale": proto.scale, "sampled_rows_per_step": rows},
+        "config": {"workload": workload_name(args.workload), "projections": [p.name for p in protos], "T": protos[0].T,
+                   "r": protos[0].r, "scale": protos[0].scale, "sampled_rows_per_step": rows},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "tokens_per_s": rows * args.steps / dt, "gpu_launches": 0,
@@ -230,8 +253,205 @@ def to_dev(bits: np.ndarray, device) -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).to(device)
 
 
+class Workload:
+    """Device tensors, plans and the step function of one workload (n_sets independent input/output sets, rotated per step)."""
+
+    def __init__(self, idx: int, rank: int, local_rank: int, device, n_sets: int = None):
+        from paper_2503_22673_b200 import binding, inputs
+        self.idx, self.device, self.binding = idx, device, binding
+        self.protos = inputs.workload(idx)
+        self.bytes_per_set = sum(2 * (p.T * p.d_in * 2 + p.T * p.d_out * 2) + 2 * p.d_out * p.d_in for p in self.protos)
+        if n_sets is None:
+            n_sets = 2 if idx >= 2 else max(2, min(6, -(-4 * L2_BYTES // self.bytes_per_set)))
+        self.n_sets = n_sets
+        self.sets = []
+        for s_i in range(n_sets):
+            cur, x_dev = [], {}
+            for proj, t in inputs.draw_workload(idx, seed=1000 * rank + s_i):
+                d = {k: to_dev(v, device) for k, v in t.items() if k != "X"}
+                if proj.x_group not in x_dev:                 # projections that share X (q/k/v, gate/up) share the tensor
+                    x_dev[proj.x_group] = to_dev(t["X"], device)
+                d["X"] = x_dev[proj.x_group]
+                d["Y"] = torch.empty((proj.T, proj.d_out), dtype=torch.bfloat16, device=device)
+                d["dX"] = torch.empty((proj.T, proj.d_in), dtype=torch.bfloat16, device=device)
+                d["dA"] = torch.empty((proj.r, proj.d_in), dtype=torch.float32, device=device)
+                d["dB"] = torch.empty((proj.d_out, proj.r), dtype=torch.float32, device=device)
+                cur.append((proj, d))
+            self.sets.append(cur)
+        self.plans = [binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r, device=local_rank) for p in self.protos]
+        for pl in self.plans:
+            pl.ensure_workspace()
+        self.flops_step = float(sum(p.flops for p in self.protos))
+        self.tokens_step = self.protos[0].T
+        self.stage_names = [("fwd_stage",) + pl.bwd_stage_names() for pl in self.plans]
+
+    def step(self, k, events=None, saved_p=False):
+        cur = self.sets[k % self.n_sets]
+        for j, (proj, d) in enumerate(cur):
+            pl = self.plans[j]
+            if events is None:       # the product path: lora_linear_fwd + lora_linear_bwd
+                pl.fwd(d["X"], d["W"], d["A"], d["B"], proj.scale, d["Y"])
+                pl.bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], proj.scale, d["dX"], d["dA"], d["dB"], saved_p=saved_p)
+            else:                    # the same launches through the stage calls, with an event before and after each stage
+                ev = events[j]
+                ev[0].record()
+                pl.fwd(d["X"], d["W"], d["A"], d["B"], proj.scale, d["Y"])
+                pl.bwd_stages(d["dY"], d["X"], d["W"], d["A"], d["B"], proj.scale, d["dX"], d["dA"], d["dB"], events=ev[1:])
+
+    def check_status(self, where):
+        for pl in self.plans:
+            code, msg = pl.device_status()
+            if code != 0:
+                raise SystemExit(f"bench.py: device status {where}: {msg}")
+
+    def close(self):
+        for pl in self.plans:
+            pl.close()
+        self.sets = []
+        import gc
+        gc.collect()
+        torch.cuda.empty_cache()
+
+
+def stage_bytes(p, stage: str) -> float:
+    """Algorithmic bytes of one launch (group) of the skinny stages: the streamed matrices once, the small factors, the result."""
+    x, dy = 2.0 * p.T * p.d_in, 2.0 * p.T * p.d_out
+    small_t = 2.0 * p.T * p.r                      # one [r, T] bf16 factor
+    return {"sides": x + dy + 2 * small_t + 2.0 * p.r * (p.d_in + p.d_out),
+            "grads": x + dy + 2 * small_t + 4.0 * p.r * (p.d_in + p.d_out),
+            "q_prepass": dy + small_t + 2.0 * p.r * p.d_out,
+            "dA": x + 2 * small_t + 4.0 * p.r * p.d_in,
+            "dB": dy + small_t + 4.0 * p.r * p.d_out}[stage]
+
+
+def measure(wl: Workload, steps: int, warmup: int, pk, world: int, device, barrier, sampler=None):
+    """Timed region (K steps back to back between two events) and the instrumented pass (events between the stages)."""
+    binding = wl.binding
+    n_warm = max(warmup, 3)
+    for k in range(n_warm):
+        wl.step(k)
+    torch.cuda.synchronize()
+    wl.check_status("after warm-up")
+    ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for k in range(n_warm):              # once more, so that the timed region starts from a loaded, warm GPU
+        wl.step(k)
+    launches0 = binding.launch_count()
+    barrier()
+    torch.cuda.synchronize()
+    t_host0 = time.time()
+    ev_a.record()
+    for k in range(steps):
+        wl.step(n_warm + k)
+    ev_b.record()
+    torch.cuda.synchronize()
+    t_host1 = time.time()
+    barrier()
+    launches = binding.launch_count() - launches0
+    ms_step = max_over_ranks(ev_a.elapsed_time(ev_b), device, world) / steps
+    # SM clock of the last GEMM launch of every projection, measured inside the kernel
+    gemm_clock = {p.name: round(pl.last_gemm_clock()[0], 1) for p, pl in zip(wl.protos, wl.plans)}
+
+    # ---- the same steps once more with events between the stages: per-stage durations.  An event record between two
+    #      launches suppresses their programmatic overlap, so this pass is a little slower than the timed region ----
+    n_instr = min(steps, 20)
+    events = [[[torch.cuda.Event(enable_timing=True) for _ in range(len(names) + 1)] for names in wl.stage_names]
+              for _ in range(n_instr)]
+    i_a, i_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    i_a.record()
+    for k in range(n_instr):
+        wl.step(n_warm + k, events[k])
+    i_b.record()
+    torch.cuda.synchronize()
+    t_host2 = time.time()
+    ms_step_instr = i_a.elapsed_time(i_b) / n_instr
+    wl.check_status("after the timed region")
+
+    kern = {}
+    for j, p in enumerate(wl.protos):
+        names = wl.stage_names[j]
+        dur = [statistics.mean(events[k][j][i].elapsed_time(events[k][j][i + 1]) for k in range(n_instr)) for i in range(len(names))]
+        cfg = wl.plans[j].config()
+        entry = {}
+        for name, ms in zip(names, dur):
+            if name == "fwd_stage":
+                fl = 2.0 * p.T * p.d_in * p.d_out + 2.0 * p.T * p.r * (p.d_in + p.d_out)
+                entry[name] = {"ms": ms, "tflops": fl / ms / 1e9, "frac_of_bf16_peak": fl / ms / 1e9 / pk["bf16_tflops"],
+                               "launches": "X A^T pass + K-extended GEMM" if cfg["fwd_ext"] and cfg["cta_group"] == 2 else "fused GEMM"}
+            elif name == "dx_gemm":
+                fl = 2.0 * p.T * p.d_in * p.d_out + 2.0 * p.T * p.r * p.d_in          # dense + the rank-r k-block (Q A)
+                entry[name] = {"ms": ms, "tflops": fl / ms / 1e9, "frac_of_bf16_peak": fl / ms / 1e9 / pk["bf16_tflops"],
+                               "frac_of_bf16_sustained": fl / ms / 1e9 / pk["bf16_tflops_sustained"]}
+            else:
+                by = stage_bytes(p, name)
+                entry[name] = {"ms": ms, "gbs": by / ms / 1e6, "frac_of_hbm_peak": by / ms / 1e6 / pk["hbm_gbs"],
+                               "bytes": by}
+        kern[p.name] = entry
+    return {"ms_per_step": ms_step, "ms_per_step_instrumented": ms_step_instr, "launches": launches, "kernels": kern,
+            "gemm_sm_mhz_in_kernel": gemm_clock, "t_host": (t_host0, t_host1, t_host2), "n_warm": n_warm}
+
+
+def kernel_b2b(wl: Workload, pk, n: int = 16):
+    """Every skinny stage of every projection launched n times back to back (inputs rotate between the sets, so the
+    stream never sits in L2): the launch's own steady-state duration, with the programmatic overlap of consecutive
+    launches that the step itself enjoys and the instrumented pass suppresses."""
+    out = {}
+    for j, p in enumerate(wl.protos):
+        pl = wl.plans[j]
+        lib, h = pl._lib, pl._h
+        from paper_2503_22673_b200.binding import _ptr, _stream_ptr
+        sp = _stream_ptr(None)
+        res = {}
+        for name in pl.bwd_stage_names():
+            if name == "dx_gemm":
+                continue
+
+            def call(k, name=name):
+                d = wl.sets[k % wl.n_sets][j][1]
+                s = float(p.scale)
+                if name == "sides":
+                    return lib.lora_linear_bwd_sides(h, _ptr(d["dY"]), _ptr(d["X"]), _ptr(d["A"]), _ptr(d["B"]), s, sp)
+                if name == "grads":
+                    return lib.lora_linear_bwd_grads(h, _ptr(d["dY"]), _ptr(d["X"]), _ptr(d["A"]), s, _ptr(d["dA"]), _ptr(d["dB"]), sp)
+                if name == "q_prepass":
+                    return lib.lora_linear_bwd_q(h, _ptr(d["dY"]), _ptr(d["B"]), s, sp)
+                if name == "dA":
+                    return lib.lora_linear_bwd_da(h, _ptr(d["X"]), _ptr(d["A"]), s, _ptr(d["dA"]), sp)
+                return lib.lora_linear_bwd_db(h, _ptr(d["dY"]), s, _ptr(d["dB"]), sp)
+
+            for k in range(3):
+                call(k)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record()
+            for k in range(n):
+                call(3 + k)
+            b.record()
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / n
+            by = stage_bytes(p, name)
+            res[name] = {"ms": ms, "gbs": by / ms / 1e6, "frac_of_hbm_peak": by / ms / 1e6 / pk["hbm_gbs"]}
+        out[p.name] = res
+    return out
+
+
+def timed_loop(fn, n, barrier, device, world):
+    for k in range(3):
+        fn(k)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    a.record()
+    for k in range(n):
+        fn(3 + k)
+    b.record()
+    torch.cuda.synchronize()
+    barrier()
+    return max_over_ranks(a.elapsed_time(b) / n, device, world)
+
+
 def run_ours(args):
-    from paper_2503_22673_b200 import binding, inputs
+    from paper_2503_22673_b200 import binding
     rank, local_rank, world = dist_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py: no CUDA device - the layer has no CPU fallback")
@@ -241,275 +461,145 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
     pk = peaks()
-    # nvidia-smi takes a while to start: launch it now, keep the samples whose timestamps fall into the timed region
+    # nvidia-smi takes a while to start: launch it now, keep the samples whose timestamps fall into the timed regions
     sampler = ClockSampler(local_rank) if rank == 0 else None
-
-    # ---- inputs: n_sets independent seeded batches, rotated so that no step finds its operands in L2 ----
-    protos = inputs.workload(args.workload)
-    bytes_per_set = sum(2 * (p.T * p.d_in * 2 + p.T * p.d_out * 2) + 2 * p.d_out * p.d_in for p in protos)
-    n_sets = max(2, min(6, -(-4 * L2_BYTES // bytes_per_set)))
-    if args.workload >= 4:
-        n_sets = 2
-    sets = []
-    for s_i in range(n_sets):
-        cur = []
-        for proj, t in inputs.draw_workload(args.workload, seed=1000 * rank + s_i):
-            d = {k: to_dev(v, device) for k, v in t.items()}
-            d["Y"] = torch.empty((proj.T, proj.d_out), dtype=torch.bfloat16, device=device)
-            d["dX"] = torch.empty((proj.T, proj.d_in), dtype=torch.bfloat16, device=device)
-            d["dA"] = torch.empty((proj.r, proj.d_in), dtype=torch.float32, device=device)
-            d["dB"] = torch.empty((proj.d_out, proj.r), dtype=torch.float32, device=device)
-            cur.append((proj, d))
-        sets.append(cur)
-    if args.grouped and args.workload == 4:
-        # q/k/v and gate/up consume the same X: each group becomes ONE projection (stacked A, block-diagonal B)
-        from paper_2503_22673_b200.grouped import GroupedLoraPlan
-        groups = [[0, 1, 2], [3], [4, 5], [6]]
-        new_protos, new_sets = [], [[] for _ in sets]
-        for idxs in groups:
-            p0 = protos[idxs[0]]
-            if len(idxs) == 1:
-                new_protos.append(p0)
-                for si, cur in enumerate(sets):
-                    new_sets[si].append(cur[idxs[0]])
-                continue
-            d_outs = [protos[i].d_out for i in idxs]
-            gp = inputs.Projection("+".join(protos[i].name for i in idxs), p0.T, p0.d_in, sum(d_outs), p0.r * len(idxs),
-                                   p0.scale)
-            new_protos.append(gp)
-            helper = GroupedLoraPlan(p0.T, p0.d_in, d_outs, p0.r, device=local_rank)
-            for si, cur in enumerate(sets):
-                W, A, B = helper.pack([cur[i][1]["W"] for i in idxs], [cur[i][1]["A"] for i in idxs],
-                                      [cur[i][1]["B"] for i in idxs])
-                d = {"X": cur[idxs[0]][1]["X"], "W": W, "A": A, "B": B,
-                     "dY": torch.cat([cur[i][1]["dY"] for i in idxs], dim=1).contiguous()}
-                d["Y"] = torch.empty((gp.T, gp.d_out), dtype=torch.bfloat16, device=device)
-                d["dX"] = torch.empty((gp.T, gp.d_in), dtype=torch.bfloat16, device=device)
-                d["dA"] = torch.empty((gp.r, gp.d_in), dtype=torch.float32, device=device)
-                d["dB"] = torch.empty((gp.d_out, gp.r), dtype=torch.float32, device=device)
-                new_sets[si].append((gp, d))
-            helper.close()
-        flops_algorithmic = float(sum(p.flops for p in protos))      # the seven projections' own FLOPs
-        protos, sets = new_protos, new_sets
-        del new_sets
-        import gc
-        gc.collect()
-        torch.cuda.empty_cache()
-    else:
-        flops_algorithmic = float(sum(p.flops for p in protos))
-    plans = [binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r, device=local_rank) for p in protos]
-    for pl in plans:
-        pl.ensure_workspace()
-    flops_step = flops_algorithmic
-    tokens_step = protos[0].T
-
-    def step(k, events=None):
-        cur = sets[k % n_sets]
-        for j, (proj, d) in enumerate(cur):
-            ev = events[j] if events is not None else None
-            if ev is not None:
-                ev[0].record()
-            plans[j].fwd(d["X"], d["W"], d["A"], d["B"], proj.scale, d["Y"])
-            if ev is None:       # the product path: lora_linear_bwd (dX GEMM beside the dA / dB passes where the plan says so)
-                plans[j].bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], proj.scale, d["dX"], d["dA"], d["dB"])
-            else:                # the same kernels one after the other through the stage calls, with events between them
-                plans[j].bwd_stages(d["dY"], d["X"], d["W"], d["A"], d["B"], proj.scale, d["dX"], d["dA"], d["dB"], events=ev[1:])
 
     def barrier():
         if world > 1:
             import torch.distributed as dist
             dist.barrier()
 
-    n_warm = max(args.warmup, 3)
-    for k in range(n_warm):
-        step(k)
-    torch.cuda.synchronize()
-    for pl in plans:
-        code, msg = pl.device_status()
-        if code != 0:
-            raise SystemExit(f"bench.py: device status after warm-up: {msg}")
+    wl = Workload(args.workload, rank, local_rank, device)
+    protos, plans = wl.protos, wl.plans
+    m = measure(wl, args.steps, args.warmup, pk, world, device, barrier)
+    ms_step, kern = m["ms_per_step"], m["kernels"]
+    flops_step, tokens_step = wl.flops_step, wl.tokens_step
 
-    # ---- timed region: K steps back to back, device-timed (events only around the region) ----
-    ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    for k in range(n_warm):              # once more, so that the timed region starts from a loaded, warm GPU
-        step(k)
-    launches0 = binding.launch_count()
+    # ---- sustained leg: the same step looped back to back for at least two seconds (clock samples inside it) ----
+    n_sus = max(args.steps, int(2200.0 / ms_step) + 1) if not args.quick else args.steps
+    s_a, s_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     torch.cuda.synchronize()
-    t_host0 = time.time()
-    ev_a.record()
-    for k in range(args.steps):
-        step(n_warm + k)
-    ev_b.record()
+    t_sus0 = time.time()
+    s_a.record()
+    for k in range(n_sus):
+        wl.step(k)
+    s_b.record()
     torch.cuda.synchronize()
-    t_host1 = time.time()
+    t_sus1 = time.time()
     barrier()
-    launches = binding.launch_count() - launches0
-    ms_total = max_over_ranks(ev_a.elapsed_time(ev_b), device, world)
-    ms_step = ms_total / args.steps
+    ms_sus = max_over_ranks(s_a.elapsed_time(s_b), device, world) / n_sus
+    sus_clock = {p.name: round(pl.last_gemm_clock()[0], 1) for p, pl in zip(protos, plans)}
+    b2b = kernel_b2b(wl, pk)
+    clocks_raw = sampler.stop(*m["t_host"][:2]) if sampler is not None else None
+    clocks = clocks_raw
+    sus_clocks = sampler.window(t_sus0, t_sus1, "sustained leg") if sampler is not None else None
 
-    # ---- the same steps once more with events between the kernels: per-kernel durations.  An event record between two
-    #      launches suppresses their programmatic overlap, so this pass is a little slower than the timed region; its
-    #      own per-step time is reported as ms_per_step_instrumented ----
-    events = [[[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in protos] for _ in range(args.steps)]
-    i_a, i_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    i_a.record()
-    for k in range(args.steps):
-        step(n_warm + k, events[k])
-    i_b.record()
-    torch.cuda.synchronize()
-    t_host2 = time.time()
-    ms_step_instr = i_a.elapsed_time(i_b) / args.steps
-    clocks = sampler.stop(t_host0, t_host2) if sampler is not None else None
-
-    # per-stage mean durations (ms) from the instrumented pass.  Events: 0 before the forward call, 1 after it, 2 after the
-    # dY B pre-pass, 3 after the dX GEMM launch, 4 after the dA stage, 5 after the dB stage
-    kern = {}
-    for j, p in enumerate(protos):
-        dur = [statistics.mean(events[k][j][i].elapsed_time(events[k][j][i + 1]) for k in range(args.steps)) for i in range(5)]
-        fwd_flops = 2.0 * p.T * p.d_in * p.d_out + 2.0 * p.T * p.r * (p.d_in + p.d_out)
-        dxg_flops = 2.0 * p.T * p.d_in * p.d_out + 2.0 * p.T * p.r * p.d_in            # dense + the rank-r k-block (Q A)
-        q_bytes = 2.0 * p.T * p.d_out + 2.0 * p.T * p.r + 2.0 * p.r * p.d_out           # dY once, B in, Qt out
-        da_bytes = 2.0 * p.T * p.d_in + 2.0 * p.T * p.r * 2 + 4.0 * p.r * p.d_in      # X once, Qt in, Pt out, dA out
-        db_bytes = 2.0 * p.T * p.d_out + 2.0 * p.T * p.r + 4.0 * p.r * p.d_out        # dY once, Pt in, dB out
-        kern[p.name] = {
-            "fwd_stage": {"ms": dur[0], "tflops": fwd_flops / dur[0] / 1e9,
-                          "frac_of_bf16_peak": fwd_flops / dur[0] / 1e9 / pk["bf16_tflops"]},
-            "q_prepass": {"ms": dur[1], "gbs": q_bytes / dur[1] / 1e6, "frac_of_hbm_peak": q_bytes / dur[1] / 1e6 / pk["hbm_gbs"]},
-            "dx_gemm": {"ms": dur[2], "tflops": dxg_flops / dur[2] / 1e9,
-                        "frac_of_bf16_peak": dxg_flops / dur[2] / 1e9 / pk["bf16_tflops"]},
-            "dA": {"ms": dur[3], "gbs": da_bytes / dur[3] / 1e6, "frac_of_hbm_peak": da_bytes / dur[3] / 1e6 / pk["hbm_gbs"]},
-            "dB": {"ms": dur[4], "gbs": db_bytes / dur[4] / 1e6, "frac_of_hbm_peak": db_bytes / dur[4] / 1e6 / pk["hbm_gbs"]},
-        }
-    # dominant kernel for the roofline: the dX GEMM launch of the projection with the longest GEMMs.  Its event pair
-    # brackets exactly ONE kernel (the K-extended CTA-pair GEMM; the dY B pre-pass sits before the first of the two events)
-    # unless the plan splits it along K or the batch is too small for CTA pairs (then the bracket holds what dx_launches says)
+    # dominant kernel for the roofline: the dX GEMM launch of the projection with the longest GEMMs (its event pair
+    # brackets exactly ONE kernel: the K-extended CTA-pair GEMM; the skinny launch that feeds it sits before the first event)
     dom_p = max(protos, key=lambda p: kern[p.name]["fwd_stage"]["ms"] + kern[p.name]["dx_gemm"]["ms"])
     dom_plan = plans[protos.index(dom_p)].config()
     dom = kern[dom_p.name]["dx_gemm"]
     dx_launches = 1 + (1 if dom_plan["dx_split_k"] > 1 and dom_plan["cta_group"] == 2 else 0)
+    gemm_key = f"{dom_p.T}x{dom_p.d_in}x{dom_p.d_out}"
     roofline = {"bound": "tensor",
-                "kernel": f"lora_gemm_pair_kernel<1,1>: dX = dY W + (s dY B) A as one K-extended GEMM ({dom_p.name})"
+                "kernel": f"lora_gemm_pair_kernel<1,1>: dX = dY W + (s dY B) A as one K-extended GEMM ({dom_p.name}, {gemm_key})"
                           if dom_plan["cta_group"] == 2 else f"lora_gemm_kernel<1> (single-CTA dX GEMM, {dom_p.name})",
                 "launches_in_bracket": dx_launches,
-                "achieved": dom["tflops"], "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": dom["tflops"] / pk["bf16_tflops"], "peak_kind": f"bf16 burst, of {pk['source']}",
-                "frac_of_sustained": dom["tflops"] / pk["bf16_tflops_sustained"],
+                "achieved": dom["tflops"], "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                "frac": dom["tflops"] / pk["bf16_tflops_sustained"],
+                "peak_kind": f"bf16 sustained (the kernel is timed inside a long step), of {pk['source']}",
+                "frac_of_burst": dom["tflops"] / pk["bf16_tflops"], "burst_peak": pk["bf16_tflops"],
+                "sm_mhz_in_kernel": m["gemm_sm_mhz_in_kernel"].get(dom_p.name),
                 "ms_per_launch": dom["ms"],
                 "flops_per_launch": 2.0 * dom_p.T * dom_p.d_in * dom_p.d_out + 2.0 * dom_p.T * dom_p.r * dom_p.d_in,
-                "traffic": (NCU_TRAFFIC["bytes_per_launch"]["dx_gemm"] if NCU_TRAFFIC["gemm_sha"] == gemm_source_sha()
-                            and args.workload == 1 else None)}
+                "traffic": (NCU_TRAFFIC["gemm_bytes_per_launch"].get(gemm_key)
+                            if NCU_TRAFFIC["gemm_sha"] == source_sha("gemm") else None)}
+    # the skinny stage furthest below the HBM roofline (stage = one launch; duration between the events around it)
+    worst = None
+    for p in protos:
+        for name, e in kern[p.name].items():
+            if "frac_of_hbm_peak" in e and (worst is None or e["frac_of_hbm_peak"] < worst[2]["frac_of_hbm_peak"]):
+                worst = (p, name, e)
+    roofline_hbm = None
+    if worst is not None:
+        wp, wname, we = worst
+        skey = f"{wname}:{wp.T}x{wp.d_in}x{wp.d_out}"
+        roofline_hbm = {"bound": "hbm", "kernel": f"lora_grad_kernel, stage '{wname}' of {wp.name} ({wp.T} x {wp.d_in} -> {wp.d_out})",
+                        "achieved": we["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": we["frac_of_hbm_peak"],
+                        "peak_kind": f"STREAM-style copy, of {pk['source']}", "ms_per_launch": we["ms"], "bytes_per_launch": we["bytes"],
+                        "back_to_back": b2b.get(wp.name, {}).get(wname),
+                        "traffic": (NCU_TRAFFIC["stream_bytes_per_launch"].get(skey)
+                                    if NCU_TRAFFIC["stream_sha"] == source_sha("adapter_grad") else None)}
 
-    # ---- variant: backward that reuses the forward's X A^T (lora_linear_bwd_saved_p), same inputs and rotation ----
-    def step_saved(k):
-        cur = sets[k % n_sets]
-        for j, (proj, d) in enumerate(cur):
-            plans[j].fwd(d["X"], d["W"], d["A"], d["B"], proj.scale, d["Y"])
-            plans[j].bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], proj.scale, d["dX"], d["dA"], d["dB"], saved_p=True)
+    variants = {}
+    n_var = max(3, min(args.steps, 20))
+    if not args.quick:
+        # ---- variant: backward that reuses the forward's X A^T (lora_linear_bwd_saved_p), same inputs and rotation ----
+        ms_var = timed_loop(lambda k: wl.step(k, saved_p=True), n_var, barrier, device, world)
+        variants["bwd_saved_p"] = {"ms_per_step": ms_var, "value": job_value(world, flops_step, ms_var), "unit": UNIT,
+                                   "steps": n_var, "note": "forward + lora_linear_bwd_saved_p (X A^T kept from the forward)"}
+        # ---- variant: quantised LoRA (NF4 frozen weight): lora_linear_fwd_nf4 + lora_linear_bwd_nf4, same inputs.  Two forms:
+        #      weight expanded once per call into a scratch buffer (fast), or expanded inside the GEMM kernels (no extra memory)
+        if all(p.d_in % 64 == 0 for p in protos):
+            q_sets = [[binding.nf4_quantize(d["W"]) for _, d in cur] for cur in wl.sets]
+            w_scratch = {}
+            for p in protos:
+                if (p.d_out, p.d_in) not in w_scratch:
+                    w_scratch[(p.d_out, p.d_in)] = torch.empty((p.d_out, p.d_in), dtype=torch.bfloat16, device=device)
 
-    n_var = max(3, min(args.steps, 50))
-    for k in range(3):
-        step_saved(k)
-    torch.cuda.synchronize()
-    v_a, v_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    v_a.record()
-    for k in range(n_var):
-        step_saved(3 + k)
-    v_b.record()
-    torch.cuda.synchronize()
-    barrier()
-    ms_var = max_over_ranks(v_a.elapsed_time(v_b) / n_var, device, world)
-    variants = {"bwd_saved_p": {"ms_per_step": ms_var, "value": job_value(world, flops_step, ms_var), "unit": UNIT,
-                                "steps": n_var, "note": "forward + lora_linear_bwd_saved_p (X A^T kept from the forward)"}}
+            def step_nf4(k, scratch):
+                cur, qs = wl.sets[k % wl.n_sets], q_sets[k % wl.n_sets]
+                for j, (proj, d) in enumerate(cur):
+                    ws = w_scratch[(proj.d_out, proj.d_in)] if scratch else None
+                    plans[j].fwd_nf4(d["X"], qs[j][0], qs[j][1], d["A"], d["B"], proj.scale, d["Y"], w_scratch=ws)
+                    plans[j].bwd_nf4(d["dY"], d["X"], qs[j][0], qs[j][1], d["A"], d["B"], proj.scale, d["dX"], d["dA"], d["dB"],
+                                     w_scratch=ws)
 
-    # ---- variant: quantised LoRA (NF4 frozen weight): lora_linear_fwd_nf4 + lora_linear_bwd_nf4, same inputs.  Two forms:
-    #      weight expanded once per call into a scratch buffer (fast), or expanded inside the GEMM kernels (no extra memory)
-    if all(p.d_in % 64 == 0 for p in protos):
-        q_sets = [[binding.nf4_quantize(d["W"]) for _, d in cur] for cur in sets]
-        w_scratch = {}
-        for p in protos:
-            if (p.d_out, p.d_in) not in w_scratch:
-                w_scratch[(p.d_out, p.d_in)] = torch.empty((p.d_out, p.d_in), dtype=torch.bfloat16, device=device)
+            forms = [("q_lora_nf4", True, "weight expanded once per call into a bf16 scratch buffer, then the bf16 kernels")]
+            if all(p.T > 128 for p in protos):
+                forms.append(("q_lora_nf4_in_kernel", False, "no scratch: weight expanded inside the GEMM kernels, per 256-token tile"))
+            for key, scratch, how in forms:
+                ms_q = timed_loop(lambda k: step_nf4(k, scratch), n_var, barrier, device, world)
+                variants[key] = {"ms_per_step": ms_q, "value": job_value(world, flops_step, ms_q), "unit": UNIT, "steps": n_var,
+                                 "tokens_per_s": world * tokens_step / ms_q * 1e3,
+                                 "note": "forward + backward with the frozen W in NF4 (4.5 bits per weight); " + how +
+                                         "; same algorithmic FLOPs as the bf16 step"}
+            del q_sets, w_scratch
+        # ---- extra kernel: the dense weight gradient of full fine-tuning, dW = dY^T X (lora_dense_dw), per projection ----
+        dw_out = [torch.empty((p.d_out, p.d_in), dtype=torch.bfloat16, device=device) for p in protos]
 
-        def step_nf4(k, scratch):
-            cur, qs = sets[k % n_sets], q_sets[k % n_sets]
-            for j, (proj, d) in enumerate(cur):
-                ws = w_scratch[(proj.d_out, proj.d_in)] if scratch else None
-                plans[j].fwd_nf4(d["X"], qs[j][0], qs[j][1], d["A"], d["B"], proj.scale, d["Y"], w_scratch=ws)
-                plans[j].bwd_nf4(d["dY"], d["X"], qs[j][0], qs[j][1], d["A"], d["B"], proj.scale, d["dX"], d["dA"], d["dB"],
-                                 w_scratch=ws)
+        def step_dw(k):
+            for j, (proj, d) in enumerate(wl.sets[k % wl.n_sets]):
+                plans[j].dense_dw(d["dY"], d["X"], dw_out[j])
 
-        forms = [("q_lora_nf4", True, "weight expanded once per call into a bf16 scratch buffer, then the bf16 kernels")]
-        if all(p.T > 128 for p in protos):
-            forms.append(("q_lora_nf4_in_kernel", False, "no scratch: weight expanded inside the GEMM kernels, per 256-token tile"))
-        for key, scratch, how in forms:
-            for k in range(3):
-                step_nf4(k, scratch)
-            torch.cuda.synchronize()
-            q_a, q_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            barrier()
-            q_a.record()
-            for k in range(n_var):
-                step_nf4(3 + k, scratch)
-            q_b.record()
-            torch.cuda.synchronize()
-            barrier()
-            ms_q = max_over_ranks(q_a.elapsed_time(q_b) / n_var, device, world)
-            variants[key] = {"ms_per_step": ms_q, "value": job_value(world, flops_step, ms_q), "unit": UNIT, "steps": n_var,
-                             "tokens_per_s": world * tokens_step / ms_q * 1e3,
-                             "note": "forward + backward with the frozen W in NF4 (4.5 bits per weight); " + how +
-                                     "; same algorithmic FLOPs as the bf16 step"}
-        del q_sets, w_scratch
-
-    # ---- extra kernel: the dense weight gradient of full fine-tuning, dW = dY^T X (lora_dense_dw), per projection ----
-    dw_out = [torch.empty((p.d_out, p.d_in), dtype=torch.bfloat16, device=device) for p in protos]
-
-    def step_dw(k):
-        cur = sets[k % n_sets]
-        for j, (proj, d) in enumerate(cur):
-            plans[j].dense_dw(d["dY"], d["X"], dw_out[j])
-
-    for k in range(3):
-        step_dw(k)
-    torch.cuda.synchronize()
-    w_a, w_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    w_a.record()
-    for k in range(n_var):
-        step_dw(3 + k)
-    w_b.record()
-    torch.cuda.synchronize()
-    barrier()
-    ms_dw = max_over_ranks(w_a.elapsed_time(w_b) / n_var, device, world)
-    dw_flops = float(sum(2.0 * p.T * p.d_in * p.d_out for p in protos))
-    variants["full_ft_dense_dw"] = {"ms_per_step": ms_dw, "value": job_value(world, dw_flops, ms_dw), "unit": UNIT,
-                                    "frac_of_bf16_peak": dw_flops / ms_dw / 1e9 / pk["bf16_tflops"], "steps": n_var,
-                                    "note": "lora_dense_dw alone (dW = dY^T X, 2 T d_in d_out FLOPs per projection); not part "
-                                            "of the LoRA step"}
-    del dw_out
+        ms_dw = timed_loop(step_dw, n_var, barrier, device, world)
+        dw_flops = float(sum(2.0 * p.T * p.d_in * p.d_out for p in protos))
+        variants["full_ft_dense_dw"] = {"ms_per_step": ms_dw, "value": job_value(world, dw_flops, ms_dw), "unit": UNIT,
+                                        "frac_of_bf16_peak": dw_flops / ms_dw / 1e9 / pk["bf16_tflops"], "steps": n_var,
+                                        "note": "lora_dense_dw alone (dW = dY^T X, 2 T d_in d_out FLOPs per projection); not part "
+                                                "of the LoRA step"}
+        del dw_out
 
     # ---- end to end: host buffers through the C ABI (lora_linear_step_host), copies inside the timed region.  Every step
     #      copies its inputs from pinned host memory, runs forward + backward and copies Y, dX, dA, dB back.  Two lanes
     #      (plan + staging + host output buffers + stream each) alternate, so that the copy-in of one step overlaps the
     #      copy-out of the previous one on the two DMA directions; each step's own chain stays in order on its stream ----
     n_lanes = 1 if args.workload >= 4 else 2
-    h_in = []
-    for j, (p, d0) in enumerate(sets[0]):
-        h_in.append({k: d0[k].cpu().pin_memory() for k in ("X", "A", "B", "dY")})
+    sets0 = wl.sets[0]
+    h_in = [{k: d0[k].cpu().pin_memory() for k in ("X", "A", "B", "dY")} for _, d0 in sets0]
     lanes = []
     for ln in range(n_lanes):
         lp = plans if ln == 0 else [binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r, device=local_rank) for p in protos]
         for pl in lp:
             pl.ensure_workspace()
-        outs = [{k: torch.empty_like(d0[k], device="cpu").pin_memory() for k in ("Y", "dX", "dA", "dB")} for _, d0 in sets[0]]
+        outs = [{k: torch.empty_like(d0[k], device="cpu").pin_memory() for k in ("Y", "dX", "dA", "dB")} for _, d0 in sets0]
         stg = [torch.empty(lp[j].step_host_staging_bytes(), dtype=torch.uint8, device=device) for j in range(len(protos))]
         lanes.append({"plans": lp, "out": outs, "staging": stg, "stream": torch.cuda.Stream(device=device)})
 
     def step_host(k):
         ln = lanes[k % n_lanes]
-        for j, (p, d0) in enumerate(sets[0]):
+        for j, (p, d0) in enumerate(sets0):
             h, ho = h_in[j], ln["out"][j]
             ln["plans"][j].step_host(h["X"], d0["W"], h["A"], h["B"], h["dY"], p.scale, ho["Y"], ho["dX"], ho["dA"], ho["dB"],
                                      ln["staging"][j], stream=ln["stream"])
@@ -530,8 +620,8 @@ def run_ours(args):
         torch.cuda.synchronize()
         return start.elapsed_time(done)
 
-    n_e2e = max(4, min(args.steps, 20 if args.workload < 4 else 3))
-    run_host(2 * n_lanes)
+    n_e2e = max(3, min(args.steps, 20 if args.workload < 4 else 3))
+    run_host(2 * n_lanes if args.workload < 4 else 1)
     barrier()
     ms_e2e = max_over_ranks(run_host(n_e2e) / n_e2e, device, world)
     barrier()
@@ -542,24 +632,59 @@ def run_ours(args):
            "pcie_gbs": {"h2d": h2d / ms_e2e / 1e6, "d2h": d2h / ms_e2e / 1e6},
            "note": "host X, A, B, dY in; Y, dX, dA, dB out (pinned); frozen W resident on the device; "
                    f"{n_lanes} lane(s) of lora_linear_step_host alternate so that copies of neighbouring steps overlap"}
+    plan_desc = plans[0].describe()
+    del lanes, h_in
+    wl.close()
+
+    # ---- the other workloads, from short runs in the same process (rank 0's figures; every rank runs them) ----
+    per_config = {}
+    if not args.quick and world == 1:
+        for idx in [i for i in (0, 1, 2, 3, 4, 5) if i != args.workload]:
+            w2 = Workload(idx, rank, local_rank, device)
+            k2 = {0: 200, 1: 100, 2: 20, 3: 20, 4: 5, 5: 10}[idx]
+            m2 = measure(w2, k2, 3, pk, world, device, barrier)
+            v2 = job_value(1, w2.flops_step, m2["ms_per_step"])
+            stages = {}
+            for pn, e in m2["kernels"].items():
+                stages[pn] = {sn: ({"us": round(se["ms"] * 1e3, 1), "frac_of_hbm_peak": round(se["frac_of_hbm_peak"], 3)}
+                                   if "frac_of_hbm_peak" in se else
+                                   {"us": round(se["ms"] * 1e3, 1), "tflops": round(se["tflops"], 1)}) for sn, se in e.items()}
+            b2 = kernel_b2b(w2, pk)
+            per_config[f"workload{idx}"] = {
+                "workload": workload_name(idx), "steps": k2, "ms_per_step": m2["ms_per_step"], "tflops": v2,
+                "tokens_per_s": w2.tokens_step / m2["ms_per_step"] * 1e3,
+                "frac_of_bf16_burst": v2 / pk["bf16_tflops"], "frac_of_bf16_sustained": v2 / pk["bf16_tflops_sustained"],
+                "gemm_sm_mhz_in_kernel": m2["gemm_sm_mhz_in_kernel"], "stages": stages,
+                "skinny_back_to_back": {pn: {sn: {"us": round(se["ms"] * 1e3, 1), "frac_of_hbm_peak": round(se["frac_of_hbm_peak"], 3)}
+                                             for sn, se in e.items()} for pn, e in b2.items()},
+                "input_sets_rotated": w2.n_sets}
+            w2.close()
 
     if rank != 0:
         return
     cpu = cpu_baseline(args.workload) if world == 1 and not args.no_cpu_baseline else None
     value = job_value(world, flops_step, ms_step)
+    v_sus = job_value(world, flops_step, ms_sus)
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": n_warm,
-        "ms_per_step": ms_step, "ms_per_step_instrumented": ms_step_instr, "higher_is_better": True, "scaling": "weak",
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": m["n_warm"],
+        "ms_per_step": ms_step, "ms_per_step_instrumented": m["ms_per_step_instrumented"], "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": workload_name(args.workload), "projections": [p.name for p in protos], "T": protos[0].T,
-                   "r": protos[0].r, "scale": protos[0].scale, "input_sets_rotated": n_sets, "grouped": bool(args.grouped and args.workload == 4),
-                   "l2": f"{n_sets} independent input/output sets ({bytes_per_set * n_sets / 2**20:.0f} MiB) rotated per step; "
+                   "r": protos[0].r, "scale": protos[0].scale, "input_sets_rotated": wl.n_sets,
+                   "l2": f"{wl.n_sets} independent input/output sets ({wl.bytes_per_set * wl.n_sets / 2**20:.0f} MiB) rotated per step; "
                          "each step's operands exceed the 126 MB L2",
                    "replicas": "independent replica per GPU, no collective"},
         "tokens_per_s": world * tokens_step / ms_step * 1e3,
-        "frac_of_bf16_peak": value / world / pk["bf16_tflops"], "peak_source": pk["source"],
-        "kernels": kern, "variants": variants, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
-        "plan": plans[0].describe(),
+        "frac_of_bf16_peak": value / world / pk["bf16_tflops"], "frac_of_bf16_sustained_peak": value / world / pk["bf16_tflops_sustained"],
+        "peak_source": pk["source"], "peaks": {k: pk[k] for k in ("bf16_tflops", "bf16_tflops_sustained", "hbm_gbs")},
+        "sustained": {"value": v_sus, "unit": UNIT, "ms_per_step": ms_sus, "steps": n_sus, "seconds": ms_sus * n_sus / 1e3,
+                      "tokens_per_s": world * tokens_step / ms_sus * 1e3,
+                      "frac_of_bf16_burst": v_sus / world / pk["bf16_tflops"], "frac_of_bf16_sustained": v_sus / world / pk["bf16_tflops_sustained"],
+                      "gemm_sm_mhz_in_kernel": sus_clock, "clocks": sus_clocks},
+        "gemm_sm_mhz_in_kernel": m["gemm_sm_mhz_in_kernel"],
+        "kernels": kern, "skinny_back_to_back": b2b, "variants": variants, "roofline": roofline, "roofline_hbm": roofline_hbm,
+        "per_config": per_config, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": m["launches"], "clocks": clocks,
+        "plan": plan_desc,
     }
     print(json.dumps(line), flush=True)
 
@@ -567,13 +692,14 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", type=int, default=4)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--grouped", action="store_true",
-                    help="workload 4 only: run q/k/v and gate/up as one grouped projection each (shared X)")
+    ap.add_argument("--quick", action="store_true",
+                    help="only the timed region, the instrumented pass and the end-to-end leg of the chosen workload "
+                         "(no sustained leg, variants or other workloads); for profiler captures")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -76,7 +76,7 @@ typedef struct lora_kernel_config {
   int32_t tail_delay;      /* k-blocks of the next tile issued before a tile's rank-r MMA      */
   int32_t grad_feat_chunk; /* features per CTA of the adapter-gradient kernels                 */
   int32_t grad_stages;     /* ring depth of the adapter-gradient kernels                       */
-  int32_t da_feat_chunks;  /* dA kernel grid: feature chunks x token chunks                    */
+  int32_t da_feat_chunks;  /* dA kernel grid: feature chunks x token chunks (one cluster each) */
   int32_t da_token_chunks;
   int32_t db_feat_chunks;  /* dB kernel grid                                                   */
   int32_t db_token_chunks;
@@ -91,10 +91,18 @@ typedef struct lora_kernel_config {
   int32_t q_stages;
   int32_t dx_split_k;      /* k-splits per tile of the dX GEMM                                           */
   int32_t fwd_ext;         /* 1: forward runs as X A^T pre-pass + K-extended GEMM (needs the workspace)  */
-  int32_t overlap_sms;     /* lora_linear_bwd: SMs left to the dA / dB passes, which run beside the dX GEMM on a    */
-  int32_t ov_dx_ctas;      /*   second stream (0: serial order); persistent CTAs of the dX GEMM and token chunks of */
-  int32_t ov_da_token_chunks; /* the two passes in that mode                                                        */
-  int32_t ov_db_token_chunks;
+  int32_t bwd_merged;      /* 1: lora_linear_bwd = [dY B + X A^T in one launch] dX GEMM [dA + dB in one launch];      */
+                           /* 0: dY B | dX GEMM | dA (+ X A^T) | dB, one launch each                                  */
+  int32_t pair_feat_chunk; /* the dA + dB launch of the merged form: features per CTA, feature chunks of both, cluster */
+  int32_t pair_feat_chunks;
+  int32_t pair_token_chunks;
+  int32_t da_with_p;       /* split form: 1: X A^T is recomputed inside the dA launch; 0: in its own skinny pass over X */
+  int32_t dan_feat_chunk;  /* dA launch without X A^T (saved-P backward, or da_with_p = 0): features per CTA, grid    */
+  int32_t dan_feat_chunks;
+  int32_t dan_token_chunks;
+  int32_t dbq_feat_chunk;  /* dB launch that also computes dY B (saved-P backward): features per CTA, grid            */
+  int32_t dbq_feat_chunks;
+  int32_t dbq_token_chunks;
   int32_t dw_block_n;      /* dense weight gradient GEMM (lora_dense_dw): d_in columns per tile,         */
   int32_t dw_split_k;      /*   splits along the tokens, persistent CTAs                                 */
   int32_t dw_ctas;
@@ -146,13 +154,10 @@ int lora_linear_fwd(lora_plan_t* plan, const void* X, const void* W, const void*
 /* Backward:  dX = dY W + scale (dY B) A,  dA = scale (dY B)^T X,  dB = scale dY^T (X A^T).
  * Does not depend on a preceding forward call (X A^T is recomputed).  Needs the workspace.
  * dA and dB are fp32 and are overwritten.
- * Where cfg.overlap_sms > 0 (opt-in: environment variable LORA_OVERLAP_SMS = number of SMs to leave free, read when the
- * plan is created; off by default because it measured no reliable gain), the tensor-bound dX GEMM and the two HBM-bound
- * adapter-gradient passes run at the same time: the GEMM on `stream` with a few SMs fewer, the passes on a second,
- * plan-owned stream that is forked from and joined back into `stream` by events inside this call.  For the caller the
- * call still behaves as one piece of work on `stream`; results are bit-identical to the serial order of the stage calls
- * below except for the grid-dependent order of the fp32 partial sums of dA and dB, which stays fixed for a given plan.
- * (Such a plan owns one extra stream and two events besides its status block.) */
+ * Launches (cfg.bwd_merged = 1, the default): dY B and X A^T side by side in one skinny launch, the dX GEMM, dA and dB side
+ * by side in one skinny launch.  (cfg.bwd_merged = 0: dY B pre-pass, dX GEMM, dA with X A^T riding along or preceded by
+ * its own pass over X, dB.)  No launch only finishes another's sums: dA and dB are added up over the token chunks inside thread-block clusters, the
+ * skinny products over feature chunks by the last CTA to arrive, both in a fixed order (bitwise reproducible). */
 int lora_linear_bwd(lora_plan_t* plan, const void* dY, const void* X, const void* W, const void* A,
                     const void* B, float scale, void* dX, void* dA, void* dB, void* stream);
 
@@ -177,6 +182,15 @@ int lora_linear_bwd_saved_p(lora_plan_t* plan, const void* dY, const void* X, co
  *   lora_linear_bwd_db   dB = scale dY^T (X A^T), streams dY once
  * `scale` must be the same in all three. */
 int lora_linear_bwd_q(lora_plan_t* plan, const void* dY, const void* B, float scale, void* stream);
+/* The two skinny launches of the merged form as separate calls (the order is lora_linear_bwd_sides, lora_linear_bwd_dx,
+ * lora_linear_bwd_grads, same scale):
+ *   lora_linear_bwd_sides   scale (dY B)^T and scale (X A^T)^T -> workspace in ONE launch (streams dY and X once); the next
+ *                           lora_linear_bwd_dx on the plan launches the GEMM alone
+ *   lora_linear_bwd_grads   dA and dB in ONE launch from the two products in the workspace (streams X and dY once) */
+int lora_linear_bwd_sides(lora_plan_t* plan, const void* dY, const void* X, const void* A, const void* B, float scale,
+                          void* stream);
+int lora_linear_bwd_grads(lora_plan_t* plan, const void* dY, const void* X, const void* A, float scale, void* dA, void* dB,
+                          void* stream);
 int lora_linear_bwd_dx(lora_plan_t* plan, const void* dY, const void* W, const void* A, const void* B,
                        float scale, void* dX, void* stream);
 int lora_linear_bwd_da(lora_plan_t* plan, const void* X, const void* A, float scale, void* dA, void* stream);
@@ -281,6 +295,12 @@ int64_t lora_grad_contract_noalloc_max_scratch(void);
  * *code is LORA_OK or LORA_ERR_DEVICE_TIMEOUT; msg (may be NULL) receives a short description.
  * The status word is cleared. */
 int lora_last_device_status(lora_plan_t* plan, void* stream, int* code, char* msg, size_t n);
+
+/* SM clock of the last CTA-pair GEMM launch of this plan (forward or dX, whichever ran last), measured inside the kernel:
+ * one thread reads the nanosecond wall timer and the SM cycle counter when its CTA starts working and when it leaves; their
+ * ratio is the frequency the launch really ran at (external polling of the driver's clock readout is too slow to see
+ * millisecond launches under a power cap).  Synchronises `stream`.  *sm_mhz = 0 when no such launch ran yet. */
+int lora_plan_last_gemm_clock(lora_plan_t* plan, void* stream, double* sm_mhz, double* busy_us);
 
 /* Static string for a status code. */
 const char* lora_strerror(int code);

@@ -30,7 +30,8 @@ EXPORTS = [
     "lora_dense_dw", "lora_nf4_quantize", "lora_nf4_dequantize", "lora_linear_fwd_nf4", "lora_linear_bwd_nf4", "lora_step_host_staging_bytes", "lora_linear_step_host",
     "lora_last_device_status", "lora_strerror", "lora_launch_count",
     "lora_grad_contract_noalloc", "lora_grad_contract_noalloc_max_scratch", "lora_grad_contract_noalloc_status",
-    "lora_plan_set_wait_limit", "lora_debug_starved_wait",
+    "lora_plan_set_wait_limit", "lora_debug_starved_wait", "lora_linear_bwd_sides", "lora_linear_bwd_grads",
+    "lora_plan_last_gemm_clock",
 ]
 
 
@@ -42,7 +43,7 @@ class LoraKernelConfig(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "block_m", "fwd_block_n", "dx_block_n", "block_k", "stages", "group_m", "split_k", "r_pad", "fwd_ctas",
         "dx_ctas", "tail_delay", "grad_feat_chunk", "grad_stages", "da_feat_chunks", "da_token_chunks",
-        "db_feat_chunks", "db_token_chunks", "db_feat_chunk", "cta_group", "dx_stages", "prefetch_dist", "db_stages", "q_feat_chunk", "q_feat_chunks", "q_token_chunks", "q_stages", "dx_split_k", "fwd_ext", "overlap_sms", "ov_dx_ctas", "ov_da_token_chunks", "ov_db_token_chunks",
+        "db_feat_chunks", "db_token_chunks", "db_feat_chunk", "cta_group", "dx_stages", "prefetch_dist", "db_stages", "q_feat_chunk", "q_feat_chunks", "q_token_chunks", "q_stages", "dx_split_k", "fwd_ext", "bwd_merged", "pair_feat_chunk", "pair_feat_chunks", "pair_token_chunks", "da_with_p", "dan_feat_chunk", "dan_feat_chunks", "dan_token_chunks", "dbq_feat_chunk", "dbq_feat_chunks", "dbq_token_chunks",
         "dw_block_n", "dw_split_k", "dw_ctas")]
 
     def as_dict(self):
@@ -81,6 +82,8 @@ def load(rebuild: bool = False) -> ctypes.CDLL:
     lib.lora_linear_bwd_saved_p.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
     lib.lora_linear_bwd_q.argtypes = [vp, vp, vp, ctypes.c_float, vp]
     lib.lora_linear_bwd_dx.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp]
+    lib.lora_linear_bwd_sides.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp]
+    lib.lora_linear_bwd_grads.argtypes = [vp, vp, vp, vp, ctypes.c_float, vp, vp, vp]
     lib.lora_linear_bwd_da.argtypes = [vp, vp, vp, ctypes.c_float, vp, vp]
     lib.lora_linear_bwd_db.argtypes = [vp, vp, ctypes.c_float, vp, vp]
     lib.lora_dense_dw.argtypes = [vp, vp, vp, vp, vp]
@@ -99,6 +102,7 @@ def load(rebuild: bool = False) -> ctypes.CDLL:
     lib.lora_grad_contract_noalloc.argtypes = [vp, vp, i64, i64, i64, i64, vp, vp]
     lib.lora_grad_contract_noalloc_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
     lib.lora_plan_set_wait_limit.argtypes = [vp, i64]
+    lib.lora_plan_last_gemm_clock.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
     lib.lora_debug_starved_wait.argtypes = [vp, vp, i64, i64, vp, vp]
     lib.lora_grad_contract_noalloc_max_scratch.argtypes = []
     lib.lora_grad_contract_noalloc_max_scratch.restype = i64
@@ -213,6 +217,13 @@ class LoraLinearPlan:
         self._ws = ws
         n = 0 if ws is None else ws.numel() * ws.element_size()
         _check(self._lib.lora_plan_set_workspace(self._h, _ptr(ws), n), "lora_plan_set_workspace")
+
+    def last_gemm_clock(self, stream=None) -> Tuple[float, float]:
+        """(SM MHz, microseconds) of this plan's last CTA-pair GEMM launch, measured inside the kernel."""
+        mhz, us = ctypes.c_double(0.0), ctypes.c_double(0.0)
+        _check(self._lib.lora_plan_last_gemm_clock(self._h, _stream_ptr(stream), ctypes.byref(mhz), ctypes.byref(us)),
+               "lora_plan_last_gemm_clock")
+        return float(mhz.value), float(us.value)
 
     def set_wait_limit(self, cycles: int) -> None:
         """Limit of every device-side wait of this plan's later launches, in SM clock ticks (0: the default, ~2 s)."""
@@ -347,28 +358,41 @@ class LoraLinearPlan:
                                             _stream_ptr(stream)), "lora_linear_bwd_dx")
         return dX
 
+    def bwd_stage_names(self) -> Tuple[str, ...]:
+        """The launches ``bwd`` issues on this plan, in order (see ``bwd_stages``)."""
+        return ("sides", "dx_gemm", "grads") if self.config()["bwd_merged"] else ("q_prepass", "dx_gemm", "dA", "dB")
+
     def bwd_stages(self, dY, X, W, A, B, scale: float, dX, dA, dB, stream=None, events=None):
-        """The same kernels as ``bwd``, issued through the stage entry points; ``events`` (five torch.cuda.Event,
-        optional) are recorded on the stream: before the dY B pre-pass, then after the pre-pass (so that events 1 and 2
-        bracket exactly the dX GEMM launch), after the dX GEMM, after the dA stage and after the dB stage."""
+        """The same kernels as ``bwd``, issued through the stage entry points.  Merged form: dY B and X A^T in one launch,
+        the dX GEMM, dA and dB in one launch; split form: dY B pre-pass, dX GEMM, dA stage, dB.  ``events`` (one
+        torch.cuda.Event more than there are stages, optional) are recorded on the stream before the first stage and
+        after every stage, so that events k and k + 1 bracket exactly stage k of ``bwd_stage_names()``."""
         self.ensure_workspace()
         sp = _stream_ptr(stream)
         st = stream if stream is not None else torch.cuda.current_stream()
-        if events is not None:
-            events[0].record(st)
-            _check(self._lib.lora_linear_bwd_q(self._h, _ptr(dY), _ptr(B), float(scale), sp), "lora_linear_bwd_q")
-            events = events[1:]
-            events[0].record(st)
-        _check(self._lib.lora_linear_bwd_dx(self._h, _ptr(dY), _ptr(W), _ptr(A), _ptr(B), float(scale), _ptr(dX), sp),
-               "lora_linear_bwd_dx")
-        if events is not None:
-            events[1].record(st)
-        _check(self._lib.lora_linear_bwd_da(self._h, _ptr(X), _ptr(A), float(scale), _ptr(dA), sp), "lora_linear_bwd_da")
-        if events is not None:
-            events[2].record(st)
-        _check(self._lib.lora_linear_bwd_db(self._h, _ptr(dY), float(scale), _ptr(dB), sp), "lora_linear_bwd_db")
-        if events is not None:
-            events[3].record(st)
+        lib, h, s = self._lib, self._h, float(scale)
+
+        def mark(k):
+            if events is not None:
+                events[k].record(st)
+
+        mark(0)
+        if self.config()["bwd_merged"]:
+            _check(lib.lora_linear_bwd_sides(h, _ptr(dY), _ptr(X), _ptr(A), _ptr(B), s, sp), "lora_linear_bwd_sides")
+            mark(1)
+            _check(lib.lora_linear_bwd_dx(h, _ptr(dY), _ptr(W), _ptr(A), _ptr(B), s, _ptr(dX), sp), "lora_linear_bwd_dx")
+            mark(2)
+            _check(lib.lora_linear_bwd_grads(h, _ptr(dY), _ptr(X), _ptr(A), s, _ptr(dA), _ptr(dB), sp), "lora_linear_bwd_grads")
+            mark(3)
+        else:
+            _check(lib.lora_linear_bwd_q(h, _ptr(dY), _ptr(B), s, sp), "lora_linear_bwd_q")
+            mark(1)
+            _check(lib.lora_linear_bwd_dx(h, _ptr(dY), _ptr(W), _ptr(A), _ptr(B), s, _ptr(dX), sp), "lora_linear_bwd_dx")
+            mark(2)
+            _check(lib.lora_linear_bwd_da(h, _ptr(X), _ptr(A), s, _ptr(dA), sp), "lora_linear_bwd_da")
+            mark(3)
+            _check(lib.lora_linear_bwd_db(h, _ptr(dY), s, _ptr(dB), sp), "lora_linear_bwd_db")
+            mark(4)
         return dX, dA, dB
 
     # -- host-buffer step (end-to-end measurement and host callers) ------------------------------

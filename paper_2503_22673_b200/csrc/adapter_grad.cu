@@ -6,19 +6,24 @@
 // Both are out[c, j] = sum_t S[t, c] * Rt[j, t]: the streamed matrix S is the MN-major A operand of a
 // tcgen05 MMA (M = 128 features, N = r_pad, K = tokens) read from the very 128-byte-swizzled tiles TMA
 // delivers, so the token reduction runs on the tensor cores while the kernel stays bound by the HBM
-// stream.  The dA kernel additionally recomputes X A^T for the slab it holds (same tiles, this time as the
-// K-major operand with M = 128 tokens), because the backward pass is not given the forward's X A^T.
+// stream.  The same tiles, read as the K-major operand with M = 128 tokens, give the SIDE product
+// S side^T of the slab: X A^T inside the dA launch (the backward pass is not given the forward's X A^T), or dY B.
+// The side operand has two forms: A [r, C] (K-major rows) or B [C, r] (MN-major, its natural layout); with
+// do_out = 0 the kernel computes only the side product (the X A^T and dY B pre-passes of the K-extended GEMMs).
 //
-// Grid: (feature chunks, token chunks), at most one CTA per SM.  A CTA keeps feat_chunk x r_pad fp32 sums in
-// TMEM over all of its token slabs.  Cross-CTA sums (over token chunks for the gradient, over feature chunks
-// for X A^T) are written as fp32 partials and added in a fixed order by lora_grad_finalize_kernel, so the
-// result is bitwise reproducible and no CTA ever waits for another.
+// Grid: (feature chunks, token chunks), one CTA per SM, ONE launch, no CTA outside a cluster ever waits for another.
+//  * Gradient: a CTA keeps feat_chunk x r_pad fp32 sums in TMEM over all slabs of its token chunk.  The token chunks
+//    of one feature chunk form a thread-block cluster (up to 16 CTAs along y).  At the end every CTA copies its sums
+//    to its own shared memory, the cluster synchronises, and CTA k of the cluster adds slice k of all copies over
+//    distributed shared memory IN RANK ORDER and writes that slice of dA / dB: bitwise reproducible, no partial sums
+//    in global memory, no second launch.
+//  * Side product: a CTA holds only its feature chunk's share of a slab's X A^T.  With one feature chunk it writes
+//    the bf16 result itself; otherwise it writes an fp32 partial, bumps the slab's arrival counter, and the CTA that
+//    arrives last adds the partials IN CHUNK ORDER, scales, rounds and writes the slab (and resets the counter).
 //
-// The side product has two operand forms: A [r, C] (K-major rows, for X A^T) or B [C, r] (MN-major, its natural
-// layout, for dY B); with do_out = 0 the kernel computes only the side product (the Q = dY B pre-pass of backward).
-//
-// Warps: 0, 1 TMA producers of the streamed tiles (even / odd ring items: one warp's copies sustain only
-// ~30 B/clk), 2 MMA issuer + TMEM, 3 loader of the second factor, 4..7 epilogue.
+// Warps: 0..3 TMA producers of the streamed tiles (ring items round-robin: one warp's copies sustain only ~37 B/clk),
+// 4 MMA issuer + TMEM, 5 loader of the second factor, 6..9 and 10..13 two epilogue groups (slabs alternate between them,
+// so that the fence + atomic round trip of one slab's side product overlaps the next slab's drain).
 #include "kernels.h"
 #include "sm100_ptx.cuh"
 
@@ -30,52 +35,84 @@ namespace lora {
 
 namespace {
 
-constexpr int kGradBarriers = 2 * kGradMaxStages + 10;
+constexpr int kGradBarriers = 2 * kGradMaxStages + 2 * kGradMaxRtBufs + 2 * kGradPBufs + 1;
+constexpr int kGradTailBytes = kGradBarriers * 8 + 32;      // barriers, TMEM slot, abort flag, two broadcast words
+constexpr int kGradMmaWarp = kGradProducerWarps;
+constexpr int kGradLoaderWarp = kGradProducerWarps + 1;
+constexpr int kGradEpiWarp0 = kGradProducerWarps + 2;
+constexpr int kGradEpiThreads = 128 * kGradEpiGroups;
 
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t cluster_addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(cluster_addr) : "memory");
+  return v;
+}
+
+// One launch runs one or two JOBS side by side (e.g. dA over X next to dB over dY, or X A^T next to dY B): CTAs with
+// blockIdx.x < split_x belong to job 0, the others to job 1.  A job's CTAs are numbered (feature chunk, token chunk):
+// with a gradient the token chunk is blockIdx.y (= rank in the cluster), otherwise both indices are folded into x.
 __global__ void __launch_bounds__(kGradThreads, 1)
-lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix [T, C], box 64(c) x 128(t)
-                 const __grid_constant__ CUtensorMap tm_r,   // second factor [r_pad, T], box 64(t) x r_pad
-                 const __grid_constant__ CUtensorMap tm_a,   // side operand (with_p): A [r, C] box 64(c) x r_pad, or
-                                                             // B [C, r] box 64(r, zero-filled) x 64(c) when side_mn
-                 const GradParams p) {
+lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s0,  // job 0: streamed matrix [T, C], box 64(c) x 128(t)
+                 const __grid_constant__ CUtensorMap tm_r0,  //        second factor [r_pad, T], box 64(t) x r_pad
+                 const __grid_constant__ CUtensorMap tm_a0,  //        side operand (with_p): A [r, C] box 64(c) x r_pad, or
+                                                             //        B [C, r] box 64(r, zero-filled) x 64(c) when side_mn
+                 const __grid_constant__ CUtensorMap tm_s1,  // job 1, same roles
+                 const __grid_constant__ CUtensorMap tm_r1,
+                 const __grid_constant__ CUtensorMap tm_a1,
+                 const GradLaunch L) {
   pdl_launch_dependents();
+  const bool job1 = static_cast<int>(blockIdx.x) >= L.split_x;
+  const GradParams p = job1 ? L.job[1] : L.job[0];
+  const CUtensorMap& tm_s = job1 ? tm_s1 : tm_s0;
+  const CUtensorMap& tm_r = job1 ? tm_r1 : tm_r0;
+  const CUtensorMap& tm_a = job1 ? tm_a1 : tm_a0;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const int NB = p.feat_chunk >> 7;                 // 128-feature accumulator blocks
+  const int NB = p.feat_chunk >> 7;                 // 128-feature accumulator blocks of a full chunk
   const int rt_box = p.r_pad * 128;                 // bytes of one 64-wide box with r_pad rows
   const int side_box = p.side_mn ? 8192 : rt_box;   // bytes of the side operand for 64 features
   const int stage_bytes = kGradStageBytes + (p.with_p ? 2 * side_box : 0);   // S tile (+ the matching side operand)
+  const int ring_bytes = p.stages * stage_bytes;
   const uint32_t ring = smem_u32(smem);
-  const uint32_t rt_base = ring + p.stages * stage_bytes;               // 2 buffers x 2 boxes of the second factor
-  uint8_t* tail = smem + p.stages * stage_bytes + 4 * rt_box;
+  const uint32_t rt_base = ring + ring_bytes;                           // rt_bufs buffers x 2 boxes of the second factor
+  const int RB = p.rt_bufs;
+  uint8_t* tail = smem + ring_bytes + 2 * RB * rt_box;
   uint64_t* bars = reinterpret_cast<uint64_t*>(tail);
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (kGradMaxStages + s); };
   auto rt_full = [&](int b) { return bar0 + 8u * (2 * kGradMaxStages + b); };
-  auto rt_empty = [&](int b) { return bar0 + 8u * (2 * kGradMaxStages + 2 + b); };
-  auto p_full = [&](int b) { return bar0 + 8u * (2 * kGradMaxStages + 4 + b); };
-  auto p_empty = [&](int b) { return bar0 + 8u * (2 * kGradMaxStages + 6 + b); };
-  const uint32_t out_full = bar0 + 8u * (2 * kGradMaxStages + 8);
+  auto rt_empty = [&](int b) { return bar0 + 8u * (2 * kGradMaxStages + kGradMaxRtBufs + b); };
+  auto p_full = [&](int b) { return bar0 + 8u * (2 * kGradMaxStages + 2 * kGradMaxRtBufs + b); };
+  auto p_empty = [&](int b) { return bar0 + 8u * (2 * kGradMaxStages + 2 * kGradMaxRtBufs + kGradPBufs + b); };
+  const uint32_t out_full = bar0 + 8u * (2 * kGradMaxStages + 2 * kGradMaxRtBufs + 2 * kGradPBufs);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kGradBarriers);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* epi_word = reinterpret_cast<volatile int*>(tmem_slot + 2);      // one broadcast word per epilogue group
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int fc = blockIdx.x, tc = blockIdx.y;
+  const int local_x = static_cast<int>(blockIdx.x) - (job1 ? L.split_x : 0);
+  const int fc = p.do_out ? local_x : local_x % p.n_feat_chunks;
+  const int tc = p.do_out ? static_cast<int>(blockIdx.y) : local_x / p.n_feat_chunks;
   const int c0 = fc * p.feat_chunk;
+  const int nb_count = min(NB, (p.C - c0 + 127) >> 7);          // blocks of THIS chunk (the last chunk may be short)
   const int s_begin = static_cast<int>(static_cast<long long>(tc) * p.n_slabs / p.n_token_chunks);
   const int s_end = static_cast<int>(static_cast<long long>(tc + 1) * p.n_slabs / p.n_token_chunks);
   const int S = p.stages;
+  bool alive = true;            // false once a bounded wait of this thread's role gave up
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) {
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
     }
-    for (int b = 0; b < 2; ++b) {
+    for (int b = 0; b < RB; ++b) {
       mbar_init(rt_full(b), 1);
       mbar_init(rt_empty(b), 1);
+    }
+    for (int b = 0; b < kGradPBufs; ++b) {
       mbar_init(p_full(b), 1);
       mbar_init(p_empty(b), 128);
     }
@@ -86,8 +123,8 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
     tma_prefetch_desc(&tm_r);
     if (p.with_p) tma_prefetch_desc(&tm_a);
   }
-  if (warp == 2) {
-    tmem_alloc(smem_u32(tmem_slot), 512);
+  if (warp == kGradMmaWarp) {
+    tmem_alloc(smem_u32(tmem_slot), p.tmem_cols);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -95,16 +132,20 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
   tc_fence_after();
   pdl_wait();                   // global memory of earlier kernels is visible from here on
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_p = tmem_base + (p.do_out ? NB * p.r_pad : 0);     // two r_pad-column buffers for the side product
+  const uint32_t tmem_p = tmem_base + (p.do_out ? NB * p.r_pad : 0);     // kGradPBufs r_pad-column buffers for the side product
 
-  if (warp < 2) {
-    // ================================ TMA producers: streamed tiles, even / odd ring items ================================
-    int slot = 0, phase = 0, odd = 0;
-    bool ok = true;
+  if (warp < kGradProducerWarps) {
+    // ================================ TMA producers: streamed tiles, ring items round-robin ================================
+    // At most S warps take part.  A producer that waits for the k-th release of a slot relies on the (k-1)-th having
+    // happened (the wait only sees the parity of the phase): its previous item, PW items back, guarantees that only
+    // when PW <= S.
+    const int PW = min(kGradProducerWarps, S);
+    int slot = 0, phase = 0, turn = 0;
+    bool ok = warp < PW;
     for (int s = s_begin; s < s_end && ok; ++s) {
       const int t0 = s * kGradSlab;
-      for (int nb = 0; nb < NB && ok; ++nb) {
-        if (odd == warp) {
+      for (int nb = 0; nb < nb_count && ok; ++nb) {
+        if (turn == warp) {
           ok = warp_wait(empty_bar(slot), phase ^ 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_EMPTY, false, 20);
           if (ok && elect_one()) {
             const uint32_t dst = ring + slot * stage_bytes, fb = full_bar(slot);
@@ -123,10 +164,10 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
           __syncwarp();
         }
         if (++slot == S) { slot = 0; phase ^= 1; }
-        odd ^= 1;
+        if (++turn == PW) turn = 0;
       }
     }
-  } else if (warp == 3) {
+  } else if (warp == kGradLoaderWarp) {
     // ================================ loader of the second factor (one 128-token slab at a time) ================================
     bool ok = true;
     int rb = 0, rphase = 0;
@@ -139,9 +180,9 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
         tma_load_2d(rt_base + (2 * rb + 1) * rt_box, &tm_r, rt_full(rb), t0 + 64, 0);
       }
       __syncwarp();
-      if (++rb == 2) { rb = 0; rphase ^= 1; }
+      if (++rb == RB) { rb = 0; rphase ^= 1; }
     }
-  } else if (warp == 2) {
+  } else if (warp == kGradMmaWarp) {
     // ================================ MMA issuer ================================
     const uint32_t idesc_out = mma_idesc_bf16(128, p.r_pad, true, false);   // A operand = S tile, MN-major
     const uint32_t idesc_p = mma_idesc_bf16(128, p.r_pad, false, p.side_mn != 0);   // A operand = S tile, K-major
@@ -152,11 +193,12 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
     const uint32_t sstep = p.side_mn ? 128u : 2u;                           // descriptor step per 16 features
     const uint64_t r_k0 = smem_desc_sw128(rt_base, 16, 1024);               // second factor
     bool ok = true;
-    int slot = 0, phase = 0, rb = 0, rphase = 0;
+    int slot = 0, phase = 0, rb = 0, rphase = 0, pb = 0, pphase = 0;
     for (int s = s_begin; s < s_end && ok; ++s) {
       if (p.do_out) ok = warp_wait(rt_full(rb), rphase, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_FULL, false, 0);
-      if (ok && p.with_p) ok = warp_wait(p_empty(rb), rphase ^ 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_ACC_EMPTY, false, 0);
-      for (int nb = 0; nb < NB && ok; ++nb) {
+      if (ok && p.with_p)
+        ok = warp_wait(p_empty(pb), pphase ^ 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_ACC_EMPTY, false, 0);
+      for (int nb = 0; nb < nb_count && ok; ++nb) {
         ok = warp_wait(full_bar(slot), phase, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_FULL, false, 0);
         if (!ok) break;
         tc_fence_after();
@@ -173,41 +215,46 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
           if (p.with_p) {
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk)   // 128 features = 2 boxes x 4 x K16
-              mma_bf16_ss(tmem_p + rb * p.r_pad, a_k0 + so + (kk >> 2) * 1024 + (kk & 3) * 2,
+              mma_bf16_ss(tmem_p + pb * p.r_pad, a_k0 + so + (kk >> 2) * 1024 + (kk & 3) * 2,
                           w_k0 + so + (kk >> 2) * sbox + (kk & 3) * sstep, idesc_p, (nb != 0 || kk != 0) ? 1u : 0u);
           }
           mma_commit(empty_bar(slot));
-          if (nb == NB - 1) {
+          if (nb == nb_count - 1) {
             if (p.do_out) mma_commit(rt_empty(rb));
-            if (p.with_p) mma_commit(p_full(rb));
+            if (p.with_p) mma_commit(p_full(pb));
           }
         }
         __syncwarp();
         if (++slot == S) { slot = 0; phase ^= 1; }
       }
-      if (++rb == 2) { rb = 0; rphase ^= 1; }
+      if (++rb == RB) { rb = 0; rphase ^= 1; }
+      if (++pb == kGradPBufs) { pb = 0; pphase ^= 1; }
     }
     if (ok && p.do_out && elect_one()) mma_commit(out_full);
     __syncwarp();
   } else {
-    // ================================ epilogue (warps 4..7, 128 threads) ================================
-    const int quarter = warp & 3;
+    // ================================ epilogue (two groups of four warps) ================================
+    const int grp = (warp - kGradEpiWarp0) >> 2;
+    const int quarter = warp & 3;                  // the TMEM lane quarter a warp may read is fixed by its index
     const int row = quarter * 32 + lane;
+    const int gtid = (warp - kGradEpiWarp0 - 4 * grp) * 32 + lane;
     const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
-    bool alive = true;
+    const int bar_id = 1 + grp;
     if (p.with_p) {
-      // ---- X A^T of each slab, partial over this CTA's features -> p_part[fc][j][t] ----
-      int pb = 0, pphase = 0;
-      for (int s = s_begin; s < s_end; ++s) {
+      // ---- the side product of each slab: this CTA's share over its features ----
+      int ls = 0;
+      for (int s = s_begin; s < s_end; ++s, ++ls) {
+        if ((ls & (kGradEpiGroups - 1)) != grp) continue;
+        const int pb = ls & (kGradPBufs - 1), pphase = (ls / kGradPBufs) & 1;
         const int t = s * kGradSlab + row;
         bool ok = warp_wait(p_full(pb), pphase, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_SIDE, false, 32);
-        if (named_bar_or(1, 128, !ok)) { alive = false; break; }
+        if (named_bar_or(bar_id, 128, !ok)) { alive = false; break; }
         tc_fence_after();
         for (int c16 = 0; c16 < p.r_pad / 16; ++c16) {
           uint32_t v[16];
           tmem_ld16(tmem_p + lane_addr + pb * p.r_pad + c16 * 16, v);
           tmem_ld_wait();
-          if (t < p.T && !p.direct) {
+          if (t < p.T && p.n_feat_chunks > 1) {
 #pragma unroll
             for (int q = 0; q < 16; ++q)
               p.p_part[(static_cast<size_t>(fc) * p.r_pad + c16 * 16 + q) * p.ld_t + t] = __uint_as_float(v[q]);
@@ -222,38 +269,118 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
         }
         tc_fence_before();
         mbar_arrive(p_empty(pb));
-        if (++pb == 2) { pb = 0; pphase ^= 1; }
+        if (p.n_feat_chunks > 1) {
+          // The group's partials must be visible device-wide before its arrival is counted: the barrier orders every
+          // thread's stores before thread 0's fence, and a fence is cumulative over what its thread has synchronised with.
+          named_bar_sync(bar_id, 128);
+          if (gtid == 0) {
+            __threadfence();
+            epi_word[grp] = atomicAdd(p.side_count + s, 1);
+          }
+          named_bar_sync(bar_id, 128);
+          if (epi_word[grp] == p.n_feat_chunks - 1) {
+            // last feature chunk to arrive for this slab: add all partials in chunk order
+            __threadfence();
+            if (t < p.T) {
+              unsigned short* pt = reinterpret_cast<unsigned short*>(p.pt_out);
+              for (int j0 = 0; j0 < p.r_pad; j0 += 16) {
+                float acc[16];
+#pragma unroll
+                for (int q = 0; q < 16; ++q) acc[q] = 0.f;
+                for (int f = 0; f < p.n_feat_chunks; ++f) {
+                  const float* src = p.p_part + (static_cast<size_t>(f) * p.r_pad + j0) * p.ld_t + t;
+                  float v[16];
+#pragma unroll
+                  for (int q = 0; q < 16; ++q) v[q] = __ldcg(src + static_cast<size_t>(q) * p.ld_t);
+#pragma unroll
+                  for (int q = 0; q < 16; ++q) acc[q] += v[q];
+                }
+#pragma unroll
+                for (int q = 0; q < 16; ++q)
+                  pt[static_cast<size_t>(j0 + q) * p.ld_t + t] =
+                      static_cast<unsigned short>(pack_bf16x2(acc[q] * p.scale, 0.f) & 0xFFFFu);
+              }
+            }
+            if (gtid == 0) p.side_count[s] = 0;          // ready for the next launch
+          }
+        }
       }
     }
     if (alive && p.do_out) {
-      bool ok = warp_wait(out_full, 0, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_ACC, false, 32);
-      if (!named_bar_or(1, 128, !ok)) {
-        tc_fence_after();
-        // ---- this CTA's sums over its token chunk -> out_part[tc][j][c] ----
-        for (int nb = 0; nb < NB; ++nb) {
-          const int c = c0 + nb * 128 + row;
+      const bool ok = warp_wait(out_full, 0, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_ACC, false, 32);
+      if (named_bar_or(bar_id, 128, !ok)) alive = false;
+      tc_fence_after();
+    }
+  }
+
+  // ================================ gradient: sum over the token chunks inside the cluster ================================
+  // Every thread of every CTA of the cluster passes the same cluster barriers (all loop bounds are launch constants).
+  if (p.do_out) {
+    const int CS = p.n_token_chunks;                       // = cluster size along y, so cluster rank = tc
+    int bpp = ring_bytes / (p.r_pad * 512);                // blocks whose sums fit into the (now idle) ring at once
+    if (bpp < 1) bpp = 1;
+    float* stage_f = reinterpret_cast<float*>(smem);
+    for (int b0 = 0; b0 < nb_count; b0 += bpp) {
+      const int b1 = min(nb_count, b0 + bpp);
+      if (warp >= kGradEpiWarp0 && alive && !*abort_flag) {
+        // ---- TMEM -> this CTA's shared memory (blocks alternate between the two epilogue groups) ----
+        const int grp = (warp - kGradEpiWarp0) >> 2;
+        const int row = (warp & 3) * 32 + lane;
+        const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        for (int nb = b0 + grp; nb < b1; nb += kGradEpiGroups) {
+          const int nbl = nb - b0;
           for (int c16 = 0; c16 < p.r_pad / 16; ++c16) {
             uint32_t v[16];
             tmem_ld16(tmem_base + lane_addr + nb * p.r_pad + c16 * 16, v);
             tmem_ld_wait();
-            if (c < p.C && !p.direct) {
+            if (p.out_is_da) {        // [block][j][feature]
 #pragma unroll
-              for (int q = 0; q < 16; ++q)
-                p.out_part[(static_cast<size_t>(tc) * p.r_pad + c16 * 16 + q) * p.c_pad + c] = __uint_as_float(v[q]);
-            } else if (c < p.C) {
-              // the only token chunk: the sums are final, write them where the finalize kernel would have
+              for (int q = 0; q < 16; ++q) stage_f[(nbl * p.r_pad + c16 * 16 + q) * 128 + row] = __uint_as_float(v[q]);
+            } else {                  // [block][feature][j]
+              float4* dst = reinterpret_cast<float4*>(stage_f + (nbl * 128 + row) * p.r_pad + c16 * 16);
 #pragma unroll
-              for (int q = 0; q < 16; ++q) {
-                const int j = c16 * 16 + q;
-                if (j < p.r) {
-                  float* dst = p.out_is_da ? p.out + static_cast<size_t>(j) * p.C + c : p.out + static_cast<size_t>(c) * p.r + j;
-                  *dst = p.accumulate ? *dst + __uint_as_float(v[q]) : __uint_as_float(v[q]);
-                }
-              }
+              for (int q = 0; q < 4; ++q)
+                dst[q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]), __uint_as_float(v[4 * q + 2]),
+                                     __uint_as_float(v[4 * q + 3]));
             }
           }
         }
       }
+      cluster_sync_all();            // every CTA's copy is complete and visible to the cluster
+      if (warp >= kGradEpiWarp0 && !*abort_flag) {
+        // ---- CTA k adds slice k of all copies, in rank order, and writes that slice of the gradient ----
+        const int tot4 = (b1 - b0) * p.r_pad * 32;         // float4 groups of this pass
+        const int n4 = (tot4 + CS - 1) / CS;               // ... per CTA of the cluster (the last slice may be short)
+        const int etid = threadIdx.x - kGradEpiWarp0 * 32;
+        for (int i = etid; i < n4 && tc * n4 + i < tot4; i += kGradEpiThreads) {
+          const int q4 = tc * n4 + i;
+          const uint32_t off = static_cast<uint32_t>(q4) * 16u;
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int rr = 0; rr < CS; ++rr) {
+            const float4 v = ld_cluster_f4(map_to_cta(ring + off, static_cast<uint32_t>(rr)));
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+          }
+          const int e = q4 * 4;
+          if (p.out_is_da) {
+            const int rowc = e & 127, jj = (e >> 7) % p.r_pad, nbl = (e >> 7) / p.r_pad;
+            const int c = c0 + (b0 + nbl) * 128 + rowc;
+            if (jj < p.r && c < p.C) {
+              float4* dst = reinterpret_cast<float4*>(p.out + static_cast<size_t>(jj) * p.C + c);
+              if (p.accumulate) { const float4 o = *dst; acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w; }
+              *dst = acc;
+            }
+          } else {
+            const int jj = e % p.r_pad, rowc = (e / p.r_pad) & 127, nbl = e / (p.r_pad * 128);
+            const int c = c0 + (b0 + nbl) * 128 + rowc;
+            if (jj < p.r && c < p.C) {
+              float4* dst = reinterpret_cast<float4*>(p.out + static_cast<size_t>(c) * p.r + jj);
+              if (p.accumulate) { const float4 o = *dst; acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w; }
+              *dst = acc;
+            }
+          }
+        }
+      }
+      cluster_sync_all();            // no CTA overwrites its copy, or leaves, while a peer may still read it
     }
   }
 
@@ -266,51 +393,10 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s,   // streamed matrix 
     }
   }
   __syncthreads();
-  if (warp == 2) {
+  if (warp == kGradMmaWarp) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, 512);
-  }
-}
-
-// Sum of `n` floats spaced `stride` apart, added in index order; loads are issued eight at a time so that their
-// latencies overlap (the additions stay sequential, so the result does not depend on the batching).  Larger batches
-// were measured slower (32 at a time: 80 registers, +4 us on the dA finalize).
-__device__ __forceinline__ float ordered_sum(const float* p, int n, size_t stride) {
-  float acc = 0.f;
-  int k = 0;
-  for (; k + 8 <= n; k += 8) {
-    float v[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = __ldcg(p + static_cast<size_t>(k + i) * stride);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) acc += v[i];
-  }
-  for (; k < n; ++k) acc += __ldcg(p + static_cast<size_t>(k) * stride);
-  return acc;
-}
-
-// Fixed-order sums of the partials:  out = sum over token chunks of out_part ;  Pt = bf16(scale * sum over feature
-// chunks of p_part).  One thread per output element, consecutive threads on consecutive addresses.
-__global__ void __launch_bounds__(256) lora_grad_finalize_kernel(const GradParams p) {
-  pdl_launch_dependents();
-  pdl_wait();
-  const long long n_out = p.do_out ? static_cast<long long>(p.r) * p.C : 0;
-  const long long n_pt = p.with_p ? static_cast<long long>(p.r_pad) * p.T : 0;
-  const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (idx < n_out) {
-    const int j = static_cast<int>(idx / p.C), c = static_cast<int>(idx - static_cast<long long>(j) * p.C);
-    const float acc = ordered_sum(p.out_part + static_cast<size_t>(j) * p.c_pad + c, p.n_token_chunks,
-                                  static_cast<size_t>(p.r_pad) * p.c_pad);
-    float* dst = p.out_is_da ? p.out + static_cast<size_t>(j) * p.C + c : p.out + static_cast<size_t>(c) * p.r + j;
-    *dst = p.accumulate ? *dst + acc : acc;      // gradient accumulation: old value + (partials in fixed order)
-  } else if (idx < n_out + n_pt) {
-    const long long i2 = idx - n_out;
-    const int j = static_cast<int>(i2 / p.T), t = static_cast<int>(i2 - static_cast<long long>(j) * p.T);
-    const float acc = ordered_sum(p.p_part + static_cast<size_t>(j) * p.ld_t + t, p.n_feat_chunks,
-                                  static_cast<size_t>(p.r_pad) * p.ld_t);
-    reinterpret_cast<unsigned short*>(p.pt_out)[static_cast<size_t>(j) * p.ld_t + t] =
-        static_cast<unsigned short>(pack_bf16x2(acc * p.scale, 0.f) & 0xFFFFu);
+    tmem_dealloc(tmem_base, p.tmem_cols);
   }
 }
 
@@ -318,28 +404,155 @@ __global__ void __launch_bounds__(256) lora_grad_finalize_kernel(const GradParam
 
 size_t grad_smem_bytes(const GradParams& p) {
   const size_t stage = kGradStageBytes + (p.with_p ? 2 * (p.side_mn ? size_t(8192) : static_cast<size_t>(p.r_pad) * 128) : 0);
-  return static_cast<size_t>(p.stages) * stage + 4 * static_cast<size_t>(p.r_pad) * 128 + kGradBarriers * 8 + 16 + 1024;
+  return static_cast<size_t>(p.stages) * stage + 2 * static_cast<size_t>(p.rt_bufs) * p.r_pad * 128 + kGradTailBytes + 1024;
 }
 
 cudaError_t grad_configure() {
-  return cudaFuncSetAttribute(lora_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+  cudaError_t e = cudaFuncSetAttribute(lora_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(lora_grad_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+  return e;
 }
 
-bool grad_is_direct(const GradParams& p) {
-  return (!p.do_out || p.n_token_chunks == 1) && (!p.with_p || p.n_feat_chunks == 1);
+int grad_max_resident_ctas(int cluster, size_t smem_bytes) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(1, static_cast<unsigned>(cluster), 1);
+  cfg.blockDim = dim3(kGradThreads);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 1;
+  attr[0].val.clusterDim.y = static_cast<unsigned>(cluster);
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, lora_grad_kernel, &cfg) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  return n * cluster;
 }
 
-cudaError_t launch_grad(const CUtensorMap& tmS, const CUtensorMap& tmR, const CUtensorMap& tmA, const GradParams& p_in,
+GradGrid grad_pick_grid(long long T, long long C, long long C2, int r_pad, bool with_p, bool side_mn, const int* caps) {
+  const int nblk1 = static_cast<int>((C + 127) / 128), nblk2 = static_cast<int>((C2 + 127) / 128);
+  const int n_slabs = static_cast<int>((T + kGradSlab - 1) / kGradSlab);
+  int nb_max = (512 - (with_p ? kGradPBufs * r_pad : 0)) / r_pad;          // TMEM: NB x r_pad + side buffers <= 512 columns
+  if (nb_max < 1) nb_max = 1;
+  const int nblk_max = nblk1 > nblk2 ? nblk1 : nblk2;
+  if (nb_max > nblk_max) nb_max = nblk_max;
+  GradGrid best{};
+  double best_t = 1e300;
+  for (int cs = 1; cs <= kGradMaxCluster; ++cs) {
+    if (cs > n_slabs || caps[cs] < cs) continue;
+    const int slabs_per = (n_slabs + cs - 1) / cs;
+    for (int nb = 1; nb <= nb_max; ++nb) {
+      const int n_feat = (nblk1 + nb - 1) / nb + (nblk2 + nb - 1) / nb;
+      if (n_feat * cs > caps[cs]) continue;
+      // time in tile units (one 128 x 128 tile of the stream): the busiest CTA's tiles, but never less than the stream
+      // needs when every SM pulls its share of the HBM bandwidth (about 120 busy SMs saturate it); side-product partial
+      // sums add r_pad / (32 nb) of a tile's bytes per tile (written and read back); a cluster reduction ~1.5 tiles
+      double t = static_cast<double>(nb) * slabs_per;
+      const double sat = static_cast<double>(nblk1 + nblk2) * n_slabs / 120.0;
+      if (t < sat) t = sat;
+      if (with_p && n_feat > 1) t *= 1.0 + r_pad / (32.0 * nb);
+      if (cs > 1) t += 1.5;
+      if (t < best_t - 1e-9) {
+        best_t = t;
+        best.feat_chunk = nb * 128;
+        best.n_feat = n_feat;
+        best.n_tok = cs;
+      }
+    }
+  }
+  if (best.feat_chunk == 0) {
+    // more feature chunks than CTAs are resident at once even at the widest chunk: widest chunk, no cluster, several waves
+    best.feat_chunk = nb_max * 128;
+    best.n_feat = (nblk1 + nb_max - 1) / nb_max + (nblk2 + nb_max - 1) / nb_max;
+    best.n_tok = 1;
+  }
+  const size_t side_box = side_mn ? size_t(8192) : static_cast<size_t>(r_pad) * 128;
+  const size_t stage = kGradStageBytes + (with_p ? 2 * side_box : 0);
+  best.stages = grad_stages(r_pad, with_p, side_mn, true);
+  best.tmem_cols = grad_tmem_cols(best.feat_chunk, r_pad, true, with_p);
+  return best;
+}
+
+int grad_rt_bufs(int r_pad, bool do_out) { return !do_out ? 1 : (r_pad <= 32 ? 4 : 3); }
+
+int grad_stages(int r_pad, bool with_p, bool side_mn, bool do_out) {
+  const size_t side_box = side_mn ? size_t(8192) : static_cast<size_t>(r_pad) * 128;
+  const size_t stage = kGradStageBytes + (with_p ? 2 * side_box : 0);
+  const size_t fixed = 2 * static_cast<size_t>(grad_rt_bufs(r_pad, do_out)) * r_pad * 128 + kGradTailBytes + 1024;
+  int stages = static_cast<int>((232448 - fixed) / stage);
+  if (stages > kGradMaxStages) stages = kGradMaxStages;
+  return stages < 2 ? 2 : stages;
+}
+
+int grad_tmem_cols(int feat_chunk, int r_pad, bool do_out, bool with_p) {
+  const int need = (do_out ? (feat_chunk / 128) * r_pad : 0) + (with_p ? kGradPBufs * r_pad : 0);
+  int cols = 32;
+  while (cols < need) cols <<= 1;
+  return cols;
+}
+
+void grad_default_caps(int num_sms, int* caps) {
+  // Without a device to ask: SMs come in groups of about 18 (a GPC), a cluster must fit inside one group, and the largest
+  // clusters find room in all but one group
+  const int groups = num_sms / 18 > 0 ? num_sms / 18 : 1;
+  caps[0] = 0;
+  for (int cs = 1; cs <= kGradMaxCluster; ++cs) {
+    int cap = (cs > 8 && groups > 1 ? groups - 1 : groups) * ((18 / cs) * cs);
+    if (cap > num_sms / cs * cs) cap = num_sms / cs * cs;
+    caps[cs] = cs == 1 ? num_sms : cap;
+  }
+}
+
+void grad_device_caps(int num_sms, int* caps) {
+  caps[0] = 0;
+  caps[1] = num_sms;
+  for (int cs = 2; cs <= kGradMaxCluster; ++cs) caps[cs] = grad_max_resident_ctas(cs, 232448);
+}
+
+cudaError_t launch_grad2(const CUtensorMap* const tm0[3], const GradParams& p0, const CUtensorMap* const tm1[3],
+                         const GradParams* p1, cudaStream_t stream) {
+  GradLaunch L{};
+  L.job[0] = p0;
+  L.job[1] = p1 != nullptr ? *p1 : p0;
+  // x extent of a job: feature chunks (gradient: the token chunks are the cluster along y) or feature x token chunks
+  const int x0 = p0.do_out ? p0.n_feat_chunks : p0.n_feat_chunks * p0.n_token_chunks;
+  const int x1 = p1 == nullptr ? 0 : (p1->do_out ? p1->n_feat_chunks : p1->n_feat_chunks * p1->n_token_chunks);
+  L.split_x = x0;
+  const int cluster = p0.do_out ? p0.n_token_chunks : 1;
+  if (p1 != nullptr && (p1->do_out != p0.do_out || (p0.do_out && p1->n_token_chunks != p0.n_token_chunks)))
+    return cudaErrorInvalidValue;          // both jobs of a launch share the cluster shape
+  size_t smem = grad_smem_bytes(p0);
+  if (p1 != nullptr && grad_smem_bytes(*p1) > smem) smem = grad_smem_bytes(*p1);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(x0 + x1), static_cast<unsigned>(cluster), 1);
+  cfg.blockDim = dim3(kGradThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.numAttrs = 1;
+  if (cluster > 1) {
+    // the token chunks of a feature chunk are one cluster: their gradient sums meet in distributed shared memory
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 1;
+    attr[1].val.clusterDim.y = static_cast<unsigned>(cluster);
+    attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+  }
+  cfg.attrs = attr;
+  const CUtensorMap* const* t1 = p1 != nullptr ? tm1 : tm0;
+  return cudaLaunchKernelEx(&cfg, lora_grad_kernel, *tm0[0], *tm0[1], *tm0[2], *t1[0], *t1[1], *t1[2], L);
+}
+
+cudaError_t launch_grad(const CUtensorMap& tmS, const CUtensorMap& tmR, const CUtensorMap& tmA, const GradParams& p,
                         cudaStream_t stream) {
-  GradParams p = p_in;
-  // No cross-CTA sum left (one token chunk for the gradient, one feature chunk for the side product): the streaming
-  // kernel writes the results itself and the finalize launch is dropped.  Only tiny problems have such grids.
-  p.direct = grad_is_direct(p) ? 1 : 0;
-  dim3 grid(p.n_feat_chunks, p.n_token_chunks);
-  cudaError_t e = launch_pdl(lora_grad_kernel, grid, dim3(kGradThreads), grad_smem_bytes(p), stream, tmS, tmR, tmA, p);
-  if (e != cudaSuccess || p.direct) return e;
-  const long long n = (p.do_out ? static_cast<long long>(p.r) * p.C : 0) + (p.with_p ? static_cast<long long>(p.r_pad) * p.T : 0);
-  return launch_pdl(lora_grad_finalize_kernel, dim3(static_cast<unsigned>((n + 255) / 256)), dim3(256), 0, stream, p);
+  const CUtensorMap* const tm[3] = {&tmS, &tmR, &tmA};
+  return launch_grad2(tm, p, nullptr, nullptr, stream);
 }
 
 // ================================================================================================
@@ -347,16 +560,16 @@ cudaError_t launch_grad(const CUtensorMap& tmS, const CUtensorMap& tmR, const CU
 // ================================================================================================
 namespace {
 
-// Scratch held by every GPU that loads this library, until the process exits: one status block and the
-// per-token-chunk partial sums of the contraction kernel.
-constexpr size_t kNoAllocScratchBytes = 8u << 20;
+// Scratch held by every GPU that loads this library, until the process exits.  The contraction kernel sums its
+// token chunks on chip (thread-block cluster), so the only global scratch it needs is its status block.
+constexpr size_t kNoAllocScratchBytes = 4096;
 constexpr size_t kNoAllocHeaderBytes = 4096;     // [0,256) status words, rest reserved
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
 
 struct NoAllocDevice {
   bool ready = false;
   unsigned char* scratch = nullptr;   // device address of g_noalloc_scratch on this device
-  int num_sms = 0;
+  int caps[kGradMaxCluster + 1] = {};  // CTAs resident at once for clusters of 1 .. 16 CTAs
 };
 constexpr int kNoAllocMaxDevices = 64;
 NoAllocDevice g_noalloc_dev[kNoAllocMaxDevices];
@@ -420,55 +633,39 @@ extern "C" int lora_grad_contract_noalloc(const void* S, const void* Rt, int64_t
         return LORA_ERR_CUDA;
       }
       slot.scratch = static_cast<unsigned char*>(ptr);
-      slot.num_sms = sms;
+      grad_device_caps(sms, slot.caps);
       slot.ready = true;
     }
     nd = slot;
   }
-  // grid: the same rule the planned path uses (feature chunks x token chunks, at most one CTA per SM)
+  // grid: the same rule the planned path uses (feature chunks x one cluster of token chunks)
   GradParams g{};
   g.T = static_cast<int>(T);
   g.C = static_cast<int>(C);
   g.r = static_cast<int>(r);
   g.r_pad = static_cast<int>((r + 15) / 16 * 16);
-  int fc = g.r_pad <= 32 ? 512 : 768;
-  const int c128 = static_cast<int>((C + 127) / 128 * 128);
-  if (fc > c128) fc = c128;
-  g.feat_chunk = fc;
-  g.n_feat_chunks = static_cast<int>((C + fc - 1) / fc);
+  const GradGrid gg = grad_pick_grid(T, C, 0, g.r_pad, false, false, nd.caps);
+  g.feat_chunk = gg.feat_chunk;
+  g.n_feat_chunks = gg.n_feat;
+  g.n_token_chunks = gg.n_tok;
   g.n_slabs = static_cast<int>((T + kGradSlab - 1) / kGradSlab);
-  int n_tok = nd.num_sms / g.n_feat_chunks;
-  if (n_tok < 1) n_tok = 1;
-  if (n_tok > g.n_slabs) n_tok = g.n_slabs;
-  g.n_token_chunks = n_tok;
-  const size_t fixed = 4 * static_cast<size_t>(g.r_pad) * 128 + 4096;
-  int stages = static_cast<int>((232448 - fixed) / kGradStageBytes);
-  g.stages = stages > kGradMaxStages ? kGradMaxStages : stages;
-  g.c_pad = static_cast<int>((C + 31) / 32 * 32);
-  // The partial sums of all token chunks must fit the static array.  One layer (r_pad x c_pad floats) that does not fit
-  // is beyond what this entry point serves; otherwise the grid takes as many token chunks as fit, and with a single
-  // chunk the kernel needs no partial sums at all (it writes `out` itself), so a fitting shape is never refused, only
-  // given fewer CTAs.
-  const size_t layer_bytes = static_cast<size_t>(g.r_pad) * g.c_pad * sizeof(float);
-  if (kNoAllocHeaderBytes + layer_bytes > kNoAllocScratchBytes) return LORA_ERR_WORKSPACE;
-  const int fit = static_cast<int>((kNoAllocScratchBytes - kNoAllocHeaderBytes) / layer_bytes);
-  if (n_tok > fit) n_tok = fit >= 2 ? fit : 1;
-  g.n_token_chunks = n_tok;
+  g.stages = gg.stages;
+  g.rt_bufs = grad_rt_bufs(g.r_pad, true);
+  g.tmem_cols = gg.tmem_cols;
   g.with_p = 0;
   g.side_mn = 0;
   g.do_out = 1;
   g.out_is_da = 0;
   g.scale = 1.0f;
   g.out = static_cast<float*>(out);
-  g.out_part = reinterpret_cast<float*>(nd.scratch + kNoAllocHeaderBytes);
   g.p_part = nullptr;
+  g.side_count = nullptr;
   g.pt_out = nullptr;
   g.ld_t = static_cast<int>(ld_rt);
   g.status = reinterpret_cast<unsigned*>(nd.scratch);
   g.wait_limit = kWaitLimitCycles;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // the array keeps the previous call's contents: the status words must start at zero (the partial sums are
-  // fully rewritten before they are read)
+  // the array keeps the previous call's contents: the status words must start at zero
   if (cudaMemsetAsync(nd.scratch, 0, kNoAllocHeaderBytes, st) != cudaSuccess) return LORA_ERR_CUDA;
   CUtensorMap tmS, tmR;
   if (!noalloc_tmap(&tmS, S, static_cast<uint64_t>(C), static_cast<uint64_t>(T), static_cast<uint64_t>(C), 64, kGradSlab) ||

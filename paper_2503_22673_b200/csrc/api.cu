@@ -6,6 +6,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "kernels.h"
@@ -78,64 +79,60 @@ int pick_pair_block_n(long long T, long long N, int r_pad, int num_pairs) {
   return best;
 }
 
-// Streams of at most this many bytes run on a grid without cross-CTA sums (one launch instead of two): the whole
-// problem is a few microseconds of work and the second launch would cost more than the parallelism gains.
+// Streams of at most this many bytes are a few microseconds of work: they run on the smallest grid (one CTA per feature
+// chunk of a gradient, one feature chunk for a side product), where nothing is summed across CTAs.
 constexpr long long kTinyStreamBytes = 1 << 20;
 
-struct GradGrid {
-  int feat_chunk, n_feat, n_tok, stages;
-};
-
-GradGrid pick_grad_grid(long long T, long long C, int r_pad, bool with_p, int num_sms) {
-  GradGrid g;
-  // TMEM: (feat_chunk / 128) accumulator blocks of r_pad columns + two r_pad-column buffers for X A^T <= 512
-  int fc = (r_pad <= 32) ? 512 : 768;
-  const int c128 = ceil_div(C, 128) * 128;
-  if (fc > c128) fc = c128;
-  g.feat_chunk = fc;
-  g.n_feat = ceil_div(C, fc);
-  const int n_slabs = ceil_div(T, kGradSlab);
-  int n_tok = num_sms / g.n_feat;             // at most one CTA per SM: a second wave would double the time
-  if (n_tok > n_slabs) n_tok = n_slabs;
-  if (n_tok < 1) n_tok = 1;
-  // tiny stream: one token chunk, so that no finalize launch is needed (pays only if the side product, where there is
-  // one, needs no cross-CTA sum either)
-  if (kTinyStreamBytes >= 2 * T * C && (!with_p || g.n_feat == 1)) n_tok = 1;
-  g.n_tok = n_tok;
-  const size_t stage = kGradStageBytes + (with_p ? 2 * static_cast<size_t>(r_pad) * 128 : 0);
-  const size_t fixed = 4 * static_cast<size_t>(r_pad) * 128 + 2048;
-  int stages = static_cast<int>((232448 - fixed) / stage);
-  if (stages > kGradMaxStages) stages = kGradMaxStages;
-  if (stages < 2) stages = 2;
-  g.stages = stages;
-  return g;
-}
-
-// Grid of a side-product-only pass (X A^T or dY B): feature chunks x token chunks.  No TMEM bound on the feature chunk.
-//  * as few feature chunks (at most 4) as fill the SMs together with the 128-token slabs;
-//  * ONE feature chunk for tiny streams and from 64 token slabs (8192 tokens) on: every CTA then sees all features, the
-//    kernel writes the bf16 result itself and the finalize launch goes away (pre-pass stage 31.1 -> 30.7 us at
-//    8192 x 4096, 107.9 -> 100.0 us at 16384 x 14336, one launch fewer each).
+// Grid of a side-product-only job (X A^T or dY B) that may use `ctas` CTAs: feature chunks x token chunks, no TMEM bound on
+// the feature chunk.  Token slabs are independent, so ONE feature chunk is best whenever whole slabs spread evenly over the
+// CTAs: every CTA sees all features of its slabs and writes the bf16 result itself.  When a CTA would get one or two very
+// long slabs (few slabs, or wide matrices beside a narrow one in the same launch) the features are cut into 2, 4 or 8
+// chunks, whose fp32 partials the last CTA to arrive for a slab adds up.  Cost of a candidate = bytes of its busiest CTA
+// (+ 64 features' worth per slab for the arrival round trip when there are partials); ties go to fewer chunks.
 struct SideGrid {
   int feat_chunk, n_feat, n_tok;
 };
 
-SideGrid pick_side_grid(long long T, long long C, int num_sms) {
+constexpr int kSideMaxChunks = 8;
+
+SideGrid pick_side_grid(long long T, long long C, int ctas) {
   const int n_slabs = ceil_div(T, kGradSlab);
-  int nf = ceil_div(num_sms, n_slabs);
-  if (nf > 4) nf = 4;
-  if (kTinyStreamBytes >= 2 * T * C || n_slabs >= 64) nf = 1;
+  const int nblk = ceil_div(C, 128);
+  if (ctas < 1) ctas = 1;
+  int best_nf = 1;
+  double best_cost = 1e300;
+  for (int nf = 1; nf <= kSideMaxChunks && nf <= nblk && nf <= ctas; nf *= 2) {
+    const int fc = ceil_div(nblk, nf) * 128;
+    const int n_feat = ceil_div(C, fc);
+    int n_tok = ctas / n_feat;
+    if (n_tok > n_slabs) n_tok = n_slabs;
+    if (n_tok < 1) n_tok = 1;
+    const double cost = static_cast<double>(ceil_div(n_slabs, n_tok)) * (fc + (n_feat > 1 ? 64 : 0));
+    if (cost < best_cost * 0.97) {        // a split must pay for itself by a clear margin
+      best_cost = cost;
+      best_nf = nf;
+    }
+  }
+  if (kTinyStreamBytes >= 2 * T * C) best_nf = 1;
   if (const char* f = std::getenv("LORA_PREPASS_NF")) {      // tuning knob
     const int v = std::atoi(f);
-    if (v >= 1 && v <= 4) nf = v;
+    if (v >= 1 && v <= kSideMaxChunks && v <= nblk) best_nf = v;
   }
   SideGrid g;
-  g.feat_chunk = ceil_div(ceil_div(C, nf), 128) * 128;
+  g.feat_chunk = ceil_div(nblk, best_nf) * 128;
   g.n_feat = ceil_div(C, g.feat_chunk);
-  g.n_tok = num_sms / g.n_feat;
+  g.n_tok = ctas / g.n_feat;
   if (g.n_tok > n_slabs) g.n_tok = n_slabs;
   if (g.n_tok < 1) g.n_tok = 1;
   return g;
+}
+
+// CTAs of a two-job side-product launch are shared out in proportion to the jobs' bytes
+int side_pair_split(long long C0, long long C1, int num_sms) {
+  int g0 = static_cast<int>((static_cast<double>(num_sms) * C0) / static_cast<double>(C0 + C1) + 0.5);
+  if (g0 < 1) g0 = 1;
+  if (g0 > num_sms - 1) g0 = num_sms - 1;
+  return g0;
 }
 
 int check_shape(const lora_shape_t* s) {
@@ -147,11 +144,19 @@ int check_shape(const lora_shape_t* s) {
   return LORA_OK;
 }
 
-int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
+// `caps_in`: caps_in[cs] = CTAs of the streaming kernel resident at once in clusters of cs CTAs, cs = 1 .. 16 (asked from the
+// device when a plan is created); nullptr: estimated from the SM count.
+int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c, const int* caps_in = nullptr) {
   const int rc = check_shape(s);
   if (rc != LORA_OK) return rc;
   if (num_sms <= 0 || c == nullptr) return LORA_ERR_INVALID_ARG;
   std::memset(c, 0, sizeof(*c));
+  int caps[kGradMaxCluster + 1];
+  if (caps_in != nullptr) {
+    for (int i = 0; i <= kGradMaxCluster; ++i) caps[i] = caps_in[i];
+  } else {
+    grad_default_caps(num_sms, caps);
+  }
   const long long T = s->T > 0 ? s->T : 1;
   c->block_m = kBlockM;
   c->block_k = kBlockK;
@@ -266,8 +271,21 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
       if (v < c->dx_ctas) c->dx_ctas = v;
     }
   }
-  const GradGrid ga = pick_grad_grid(T, s->d_in, c->r_pad, true, num_sms);
-  const GradGrid gb = pick_grad_grid(T, s->d_out, c->r_pad, false, num_sms);
+  // Backward owes three skinny products besides the dX GEMM: s (dY B)^T before it, and dA, dB, which need s (X A^T)^T.
+  //  merged form (bwd_merged = 1): ONE launch computes dY B and X A^T side by side before the GEMM, ONE launch dA and dB
+  //    after it.  Four passes over the activations (X and dY twice each), two launches, every CTA of a side product sees
+  //    whole token slabs and every CTA of a gradient whole 128-feature blocks, so almost nothing is summed across CTAs.
+  //  split form (bwd_merged = 0): dY B | GEMM | dA with X A^T riding along (da_with_p; for ranks above 32 its partial sums
+  //    over feature chunks approach the size of the stream and X A^T gets its own pass) | dB: three passes, three launches.
+  c->bwd_merged = 1;
+  if (const char* f = std::getenv("LORA_FORCE_BWD_MERGED")) c->bwd_merged = std::atoi(f) != 0 ? 1 : 0;
+  c->da_with_p = c->r_pad <= 32 ? 1 : 0;
+  if (const char* f = std::getenv("LORA_FORCE_DA_WITH_P")) c->da_with_p = std::atoi(f) != 0 ? 1 : 0;
+  const bool tiny_a = kTinyStreamBytes >= 2 * T * s->d_in, tiny_b = kTinyStreamBytes >= 2 * T * s->d_out;
+  int caps1[kGradMaxCluster + 1] = {};                 // tiny streams: no clusters
+  caps1[1] = caps[1];
+  const GradGrid ga = grad_pick_grid(T, s->d_in, 0, c->r_pad, c->da_with_p != 0, false, tiny_a ? caps1 : caps);
+  const GradGrid gb = grad_pick_grid(T, s->d_out, 0, c->r_pad, false, false, tiny_b ? caps1 : caps);
   c->grad_feat_chunk = ga.feat_chunk;
   c->grad_stages = ga.stages;
   c->db_stages = gb.stages;
@@ -276,38 +294,21 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
   c->db_feat_chunks = gb.n_feat;
   c->db_token_chunks = gb.n_tok;
   c->db_feat_chunk = gb.feat_chunk;
-  // Overlapped backward (lora_linear_bwd), opt-in through LORA_OVERLAP_SMS = R: the tensor-bound dX GEMM leaves R SMs free
-  // and the two HBM-bound adapter-gradient passes run on them at the same time on a second stream.  Measured (ms per
-  // step, serial vs overlapped, same run): 8192 x 4096 x 4096 0.442 / 0.426 (R = 16), 0.437 (R = 24), 0.530 (R = 8: the
-  // passes reach only ~40 GB/s per SM and outlast the GEMM); 16384 x 4096 x 14336 2.909 / 2.907; 16384 x 14336 x 4096
-  // r = 64 3.055 / 3.159.  A gain within the run-to-run spread on the short step and none or a loss under the power cap
-  // of the long ones, so the default stays the serial order.
-  c->overlap_sms = 0;
-  c->ov_dx_ctas = c->dx_ctas;
-  c->ov_da_token_chunks = c->da_token_chunks;
-  c->ov_db_token_chunks = c->db_token_chunks;
-  if (c->cta_group == 2 && c->dx_split_k == 1) {
-    const int pairs = num_sms / 2;
-    int R = 0;
-    if (const char* f = std::getenv("LORA_OVERLAP_SMS")) R = std::atoi(f) / 2 * 2;
-    if (R >= 2 && R / 2 < pairs) {
-      const long long dx_t = static_cast<long long>(ceil_div(T, kPairBlockM)) * ceil_div(s->d_in, c->dx_block_n);
-      if (dx_t >= pairs) {
-        c->overlap_sms = R;
-        c->ov_dx_ctas = 2 * (pairs - R / 2);
-        const int n_slabs = ceil_div(T, kGradSlab);
-        auto tok = [&](int n_feat) {
-          int n = R / n_feat;
-          if (n < 1) n = 1;
-          if (n > n_slabs) n = n_slabs;
-          return n;
-        };
-        c->ov_da_token_chunks = tok(c->da_feat_chunks);
-        c->ov_db_token_chunks = tok(c->db_feat_chunks);
-        if (c->ov_da_token_chunks > c->da_token_chunks) c->ov_da_token_chunks = c->da_token_chunks;   // partials fit the workspace
-        if (c->ov_db_token_chunks > c->db_token_chunks) c->ov_db_token_chunks = c->db_token_chunks;
-      }
-    }
+  {
+    // dA without the side product (split form with da_with_p = 0, saved-P backward); dB with dY B riding along (saved-P
+    // backward, split form); dA and dB side by side in one launch (merged form): common chunk width and cluster size
+    const GradGrid gan = grad_pick_grid(T, s->d_in, 0, c->r_pad, false, false, tiny_a ? caps1 : caps);
+    const GradGrid gbq = grad_pick_grid(T, s->d_out, 0, c->r_pad, true, true, tiny_b ? caps1 : caps);
+    const GradGrid gp = grad_pick_grid(T, s->d_in, s->d_out, c->r_pad, false, false, (tiny_a && tiny_b) ? caps1 : caps);
+    c->dan_feat_chunk = gan.feat_chunk;
+    c->dan_feat_chunks = gan.n_feat;
+    c->dan_token_chunks = gan.n_tok;
+    c->dbq_feat_chunk = gbq.feat_chunk;
+    c->dbq_feat_chunks = gbq.n_feat;
+    c->dbq_token_chunks = gbq.n_tok;
+    c->pair_feat_chunk = gp.feat_chunk;
+    c->pair_feat_chunks = gp.n_feat;
+    c->pair_token_chunks = gp.n_tok;
   }
   {  // Q = dY B pre-pass of the CTA-pair backward
     const SideGrid q = pick_side_grid(T, s->d_out, num_sms);
@@ -323,29 +324,27 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c) {
 // backward workspace layout
 // ------------------------------------------------------------------------------------------------
 struct WsLayout {
-  size_t qt, pt, q_part, p_part, da_part, db_part, split_part, total;
-  int ld_t, c_pad_a, c_pad_b, n_slabs;
+  size_t qt, pt, q_part, p_part, count, split_part, total;
+  int ld_t, n_slabs;
 };
 
 WsLayout ws_layout(const lora_shape_t& s, const lora_kernel_config_t& c) {
   WsLayout w;
   const long long T = s.T > 0 ? s.T : 1;
   w.ld_t = static_cast<int>(align_up(static_cast<size_t>(T), 64));
-  w.c_pad_a = static_cast<int>(align_up(static_cast<size_t>(s.d_in), 32));
-  w.c_pad_b = static_cast<int>(align_up(static_cast<size_t>(s.d_out), 32));
   w.n_slabs = ceil_div(T, kGradSlab);
   size_t off = 0;
   w.qt = off;       off += align_up(static_cast<size_t>(c.r_pad) * w.ld_t * 2, kAlign);
   w.pt = off;       off += align_up(static_cast<size_t>(c.r_pad) * w.ld_t * 2, kAlign);
   {
-    int side_chunks = c.q_feat_chunks > c.db_feat_chunks ? c.q_feat_chunks : c.db_feat_chunks;
-    if (side_chunks < 4) side_chunks = 4;   // the X A^T pre-pass of a K-extended forward uses at most 4 feature chunks
-    w.q_part = off;
-    off += align_up(static_cast<size_t>(side_chunks) * c.r_pad * w.ld_t * 4, kAlign);
+    // fp32 partials of a side product computed with more than one feature chunk: the side-only jobs use at most
+    // kSideMaxChunks; the launches where it rides a gradient have one per feature chunk of that grid
+    int q_chunks = c.dbq_feat_chunks > kSideMaxChunks ? c.dbq_feat_chunks : kSideMaxChunks;
+    int p_chunks = c.da_feat_chunks > kSideMaxChunks ? c.da_feat_chunks : kSideMaxChunks;
+    w.q_part = off;   off += align_up(static_cast<size_t>(q_chunks) * c.r_pad * w.ld_t * 4, kAlign);
+    w.p_part = off;   off += align_up(static_cast<size_t>(p_chunks) * c.r_pad * w.ld_t * 4, kAlign);
   }
-  w.p_part = off;   off += align_up(static_cast<size_t>(c.da_feat_chunks) * c.r_pad * w.ld_t * 4, kAlign);
-  w.da_part = off;  off += align_up(static_cast<size_t>(c.da_token_chunks) * c.r_pad * w.c_pad_a * 4, kAlign);
-  w.db_part = off;  off += align_up(static_cast<size_t>(c.db_token_chunks) * c.r_pad * w.c_pad_b * 4, kAlign);
+  w.count = off;    off += align_up(2 * static_cast<size_t>(w.n_slabs) * sizeof(int), kAlign);   // per-slab arrival counters, two jobs
   {
     const size_t f = c.split_k > 1 ? static_cast<size_t>(c.split_k) * T * s.d_out * 4 : 0;
     const size_t b = c.dx_split_k > 1 ? static_cast<size_t>(c.dx_split_k) * T * s.d_in * 4 : 0;
@@ -450,14 +449,32 @@ struct lora_plan {
   bool q_ready;          // set while lora_linear_bwd_saved_p runs: Qt was already produced by its dB kernel
   bool accumulate;       // dA / dB are added to instead of overwritten (lora_plan_set_grad_accumulation)
   bool q_staged;         // lora_linear_bwd_q ran: the next lora_linear_bwd_dx skips its own pre-pass
-  cudaStream_t side_stream;   // overlapped backward: the adapter-gradient passes run here beside the dX GEMM
-  cudaEvent_t ev_fork, ev_join;
+  int caps[kGradMaxCluster + 1];   // caps[cs]: CTAs of the streaming kernel resident at once in clusters of cs CTAs
+  bool counters_clean;   // the workspace's arrival counters are known to be zero
   bool p_saved;          // the workspace holds Pt = s (X A^T)^T of the last forward call
   float p_saved_scale;
   long long wait_limit;  // SM clock ticks after which a device-side spin gives up (lora_plan_set_wait_limit)
 };
 
 namespace {
+
+// caps[cs] = CTAs of the streaming kernel resident at once in clusters of cs CTAs on `device` (current): asked once per
+// device; a size the device refuses gets 0 and is never chosen.
+void device_caps(int device, int num_sms, int* caps) {
+  static std::mutex mu;
+  static int table[64][kGradMaxCluster + 1];
+  static bool ready[64] = {};
+  std::lock_guard<std::mutex> lock(mu);
+  if (device < 0 || device >= 64) {
+    grad_device_caps(num_sms, caps);
+    return;
+  }
+  if (!ready[device]) {
+    grad_device_caps(num_sms, table[device]);
+    ready[device] = true;
+  }
+  for (int i = 0; i <= kGradMaxCluster; ++i) caps[i] = table[device][i];
+}
 
 struct DeviceGuard {
   int prev = -1;
@@ -483,43 +500,87 @@ WsPtrs ws_ptrs(lora_plan* pl) {
   return q;
 }
 
-// Skinny side-product pass: out_t = s (S side^T)^T as bf16 [r_pad, ld_t], S = X with side = A [r, C] (K-major) or
-// S = dY with side = B [C, r] (MN-major).  Streams S once; partials over feature chunks are summed in fixed order.
-int launch_side_prepass(lora_plan* pl, const void* S, long long C, const void* side, bool side_mn, float scale,
-                        __nv_bfloat16* out_t, cudaStream_t st) {
+// The arrival counters of the side-product partials live in the caller's workspace.  Every launch leaves them at zero;
+// they are cleared on `st` before the first launch after the workspace was registered (or after a wait ran out).
+bool ensure_counters(lora_plan* pl, cudaStream_t st) {
+  if (pl->counters_clean) return true;
+  if (cudaMemsetAsync(static_cast<uint8_t*>(pl->workspace) + pl->ws.count, 0, 2 * static_cast<size_t>(pl->ws.n_slabs) * sizeof(int), st) !=
+      cudaSuccess)
+    return false;
+  pl->counters_clean = true;
+  return true;
+}
+
+// One side-product job: out_t = s (S side^T)^T as bf16 [r_pad, ld_t], S = X with side = A [r, C] (K-major) or S = dY with
+// side = B [C, r] (MN-major).  Streams S once on at most `ctas` CTAs; `which` (0 / 1) picks the job's own partial-sum region
+// and counter range, so that two jobs can run side by side.
+struct SideJob {
+  CUtensorMap tmS, tmSide;
+  GradParams g;
+};
+
+bool fill_side_job(lora_plan* pl, const void* S, long long C, const void* side, bool side_mn, float scale, __nv_bfloat16* out_t,
+                   int ctas, int which, SideJob* job) {
   const lora_shape_t& s = pl->shape;
   const lora_kernel_config_t& c = pl->cfg;
   const WsLayout& w = pl->ws;
-  CUtensorMap tmS, tmSide;
-  bool ok = make_bf16_tmap(&tmS, S, C, s.T, C, 64, kGradSlab);
-  if (side_mn) ok = ok && make_bf16_tmap(&tmSide, side, s.r, C, s.r, 64, 64);
-  else ok = ok && make_bf16_tmap(&tmSide, side, C, s.r, C, 64, c.r_pad);
-  if (!ok) return LORA_ERR_CUDA;
-  const SideGrid sg = pick_side_grid(s.T, C, pl->num_sms);
-  const int n_slabs = w.n_slabs;
-  const int fc = sg.feat_chunk, nf = sg.n_feat, nt = sg.n_tok;
+  bool ok = make_bf16_tmap(&job->tmS, S, C, s.T, C, 64, kGradSlab);
+  if (side_mn) ok = ok && make_bf16_tmap(&job->tmSide, side, s.r, C, s.r, 64, 64);
+  else ok = ok && make_bf16_tmap(&job->tmSide, side, C, s.r, C, 64, c.r_pad);
+  if (!ok) return false;
+  const SideGrid sg = pick_side_grid(s.T, C, ctas);
   GradParams g{};
   g.T = static_cast<int>(s.T);
   g.C = static_cast<int>(C);
   g.r = static_cast<int>(s.r);
   g.r_pad = c.r_pad;
-  g.feat_chunk = fc;
-  g.n_feat_chunks = nf;
-  g.n_token_chunks = nt;
-  g.n_slabs = n_slabs;
-  g.stages = side_mn ? 4 : ((232448 - 4 * c.r_pad * 128 - 2048) / (kGradStageBytes + 2 * c.r_pad * 128) > 6
-                                ? 6 : (232448 - 4 * c.r_pad * 128 - 2048) / (kGradStageBytes + 2 * c.r_pad * 128));
+  g.feat_chunk = sg.feat_chunk;
+  g.n_feat_chunks = sg.n_feat;
+  g.n_token_chunks = sg.n_tok;
+  g.n_slabs = w.n_slabs;
+  g.stages = grad_stages(c.r_pad, true, side_mn, false);
+  g.rt_bufs = grad_rt_bufs(c.r_pad, false);
+  g.tmem_cols = grad_tmem_cols(sg.feat_chunk, c.r_pad, false, true);
   g.with_p = 1;
   g.side_mn = side_mn ? 1 : 0;
   g.do_out = 0;
   g.scale = scale;
-  g.p_part = reinterpret_cast<float*>(static_cast<uint8_t*>(pl->workspace) + w.q_part);
+  uint8_t* ws = static_cast<uint8_t*>(pl->workspace);
+  g.p_part = reinterpret_cast<float*>(ws + (which == 0 ? w.q_part : w.p_part));
+  g.side_count = reinterpret_cast<int*>(ws + w.count) + (which == 0 ? 0 : w.n_slabs);
   g.pt_out = out_t;
   g.ld_t = w.ld_t;
   g.status = pl->d_status;
-    g.wait_limit = pl->wait_limit;
-  if (launch_grad(tmS, tmS, tmSide, g, st) != cudaSuccess) return LORA_ERR_CUDA;
-  g_launches.fetch_add(grad_is_direct(g) ? 1 : 2);
+  g.wait_limit = pl->wait_limit;
+  job->g = g;
+  return true;
+}
+
+// one side product alone (X A^T before a K-extended forward GEMM, dY B before the dX GEMM)
+int launch_side_prepass(lora_plan* pl, const void* S, long long C, const void* side, bool side_mn, float scale,
+                        __nv_bfloat16* out_t, cudaStream_t st) {
+  SideJob j;
+  if (!fill_side_job(pl, S, C, side, side_mn, scale, out_t, pl->num_sms, side_mn ? 0 : 1, &j)) return LORA_ERR_CUDA;
+  if (j.g.n_feat_chunks > 1 && !ensure_counters(pl, st)) return LORA_ERR_CUDA;
+  if (launch_grad(j.tmS, j.tmS, j.tmSide, j.g, st) != cudaSuccess) return LORA_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return LORA_OK;
+}
+
+// Qt = s (dY B)^T and Pt = s (X A^T)^T in ONE launch: the two jobs share the SMs in proportion to their bytes
+int launch_side_pair(lora_plan* pl, const void* dY, const void* B, const void* X, const void* A, float scale, cudaStream_t st) {
+  const lora_shape_t& s = pl->shape;
+  const WsPtrs q = ws_ptrs(pl);
+  const int g0 = side_pair_split(s.d_out, s.d_in, pl->num_sms);
+  SideJob jq, jp;
+  if (!fill_side_job(pl, dY, s.d_out, B, true, scale, q.qt, g0, 0, &jq) ||
+      !fill_side_job(pl, X, s.d_in, A, false, scale, q.pt, pl->num_sms - g0, 1, &jp))
+    return LORA_ERR_CUDA;
+  if ((jq.g.n_feat_chunks > 1 || jp.g.n_feat_chunks > 1) && !ensure_counters(pl, st)) return LORA_ERR_CUDA;
+  const CUtensorMap* const t0[3] = {&jq.tmS, &jq.tmS, &jq.tmSide};
+  const CUtensorMap* const t1[3] = {&jp.tmS, &jp.tmS, &jp.tmSide};
+  if (launch_grad2(t0, jq.g, t1, &jp.g, st) != cudaSuccess) return LORA_ERR_CUDA;
+  g_launches.fetch_add(1);
   return LORA_OK;
 }
 
@@ -651,95 +712,160 @@ int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const
   return LORA_OK;
 }
 
-// ---- dA = Qt-contraction over X; recomputes X A^T and leaves Pt = s (X A^T)^T ----
-int launch_da(lora_plan* pl, const void* X, const void* A, float scale, void* dA, cudaStream_t st, bool with_p = true,
-              int tok_override = 0) {
+// ---- gradient jobs: dA = Qt-contraction over X, dB = Pt-contraction over dY ----
+struct GradJob {
+  CUtensorMap tmS, tmR, tmSide;
+  GradParams g;
+};
+
+// dA over X with second factor Qt; with_p: X A^T rides along and Pt = s (X A^T)^T is left in the workspace.
+// (feat_chunk, n_feat, n_tok) = grid of the launch this job belongs to (its own feature chunks are derived from feat_chunk).
+bool fill_da_job(lora_plan* pl, const void* X, const void* A, float scale, void* dA, bool with_p, int feat_chunk, int n_tok,
+                 GradJob* job) {
   const lora_shape_t& s = pl->shape;
   const lora_kernel_config_t& c = pl->cfg;
   const WsLayout& w = pl->ws;
   const WsPtrs q = ws_ptrs(pl);
-  uint8_t* ws = q.base;
-  __nv_bfloat16 *qt = q.qt, *pt = q.pt;
-  {
-    CUtensorMap tmS, tmR, tmA;
-    bool ok = make_bf16_tmap(&tmS, X, s.d_in, s.T, s.d_in, 64, kGradSlab);
-    ok = ok && make_bf16_tmap(&tmR, qt, s.T, c.r_pad, w.ld_t, 64, c.r_pad);
-    ok = ok && make_bf16_tmap(&tmA, A, s.d_in, s.r, s.d_in, 64, c.r_pad);
-    if (!ok) return LORA_ERR_CUDA;
-    GradParams g{};
-    g.T = static_cast<int>(s.T);
-    g.C = static_cast<int>(s.d_in);
-    g.r = static_cast<int>(s.r);
-    g.r_pad = c.r_pad;
-    g.feat_chunk = c.grad_feat_chunk;
-    g.n_feat_chunks = c.da_feat_chunks;
-    g.n_token_chunks = tok_override > 0 ? tok_override : c.da_token_chunks;
-    g.n_slabs = w.n_slabs;
-    g.stages = with_p ? c.grad_stages : c.db_stages;
-    g.with_p = with_p ? 1 : 0;
-    g.side_mn = 0;
-    g.do_out = 1;
-    g.out_is_da = 1;
-    g.accumulate = pl->accumulate ? 1 : 0;
-    g.scale = scale;
-    g.out = static_cast<float*>(dA);
-    g.out_part = reinterpret_cast<float*>(ws + w.da_part);
-    g.c_pad = w.c_pad_a;
-    g.p_part = reinterpret_cast<float*>(ws + w.p_part);
-    g.pt_out = pt;
-    g.ld_t = w.ld_t;
-    g.status = pl->d_status;
-    g.wait_limit = pl->wait_limit;
-    if (launch_grad(tmS, tmR, tmA, g, st) != cudaSuccess) return LORA_ERR_CUDA;
-    g_launches.fetch_add(grad_is_direct(g) ? 1 : 2);
-  }
+  bool ok = make_bf16_tmap(&job->tmS, X, s.d_in, s.T, s.d_in, 64, kGradSlab);
+  ok = ok && make_bf16_tmap(&job->tmR, q.qt, s.T, c.r_pad, w.ld_t, 64, c.r_pad);
+  ok = ok && make_bf16_tmap(&job->tmSide, A, s.d_in, s.r, s.d_in, 64, c.r_pad);
+  if (!ok) return false;
+  GradParams g{};
+  g.T = static_cast<int>(s.T);
+  g.C = static_cast<int>(s.d_in);
+  g.r = static_cast<int>(s.r);
+  g.r_pad = c.r_pad;
+  g.feat_chunk = feat_chunk;
+  g.n_feat_chunks = ceil_div(s.d_in, feat_chunk);
+  g.n_token_chunks = n_tok;
+  g.n_slabs = w.n_slabs;
+  g.stages = grad_stages(c.r_pad, with_p, false, true);
+  g.rt_bufs = grad_rt_bufs(c.r_pad, true);
+  g.tmem_cols = grad_tmem_cols(feat_chunk, c.r_pad, true, with_p);
+  g.with_p = with_p ? 1 : 0;
+  g.side_mn = 0;
+  g.do_out = 1;
+  g.out_is_da = 1;
+  g.accumulate = pl->accumulate ? 1 : 0;
+  g.scale = scale;
+  g.out = static_cast<float*>(dA);
+  g.p_part = reinterpret_cast<float*>(q.base + w.p_part);
+  g.side_count = reinterpret_cast<int*>(q.base + w.count) + w.n_slabs;
+  g.pt_out = q.pt;
+  g.ld_t = w.ld_t;
+  g.status = pl->d_status;
+  g.wait_limit = pl->wait_limit;
+  job->g = g;
+  return true;
+}
+
+// dB over dY with second factor Pt; B_for_q: dY B rides along and Qt = s (dY B)^T is left in the workspace (saved-P backward)
+bool fill_db_job(lora_plan* pl, const void* dY, float scale, void* dB, const void* B_for_q, int feat_chunk, int n_tok,
+                 GradJob* job) {
+  const lora_shape_t& s = pl->shape;
+  const lora_kernel_config_t& c = pl->cfg;
+  const WsLayout& w = pl->ws;
+  const WsPtrs q = ws_ptrs(pl);
+  const bool with_q = B_for_q != nullptr;
+  bool ok = make_bf16_tmap(&job->tmS, dY, s.d_out, s.T, s.d_out, 64, kGradSlab);
+  ok = ok && make_bf16_tmap(&job->tmR, q.pt, s.T, c.r_pad, w.ld_t, 64, c.r_pad);
+  if (with_q) ok = ok && make_bf16_tmap(&job->tmSide, B_for_q, s.r, s.d_out, s.r, 64, 64);
+  else job->tmSide = job->tmR;
+  if (!ok) return false;
+  GradParams g{};
+  g.T = static_cast<int>(s.T);
+  g.C = static_cast<int>(s.d_out);
+  g.r = static_cast<int>(s.r);
+  g.r_pad = c.r_pad;
+  g.feat_chunk = feat_chunk;
+  g.n_feat_chunks = ceil_div(s.d_out, feat_chunk);
+  g.n_token_chunks = n_tok;
+  g.n_slabs = w.n_slabs;
+  g.stages = grad_stages(c.r_pad, with_q, true, true);
+  g.rt_bufs = grad_rt_bufs(c.r_pad, true);
+  g.tmem_cols = grad_tmem_cols(feat_chunk, c.r_pad, true, with_q);
+  g.with_p = with_q ? 1 : 0;
+  g.side_mn = with_q ? 1 : 0;
+  g.do_out = 1;
+  g.out_is_da = 0;
+  g.accumulate = pl->accumulate ? 1 : 0;
+  g.scale = scale;
+  g.out = static_cast<float*>(dB);
+  g.p_part = with_q ? reinterpret_cast<float*>(q.base + w.q_part) : nullptr;
+  g.side_count = reinterpret_cast<int*>(q.base + w.count);
+  g.pt_out = with_q ? q.qt : nullptr;
+  g.ld_t = w.ld_t;
+  g.status = pl->d_status;
+  g.wait_limit = pl->wait_limit;
+  job->g = g;
+  return true;
+}
+
+int launch_da(lora_plan* pl, const void* X, const void* A, float scale, void* dA, cudaStream_t st, bool with_p) {
+  const lora_kernel_config_t& c = pl->cfg;
+  const bool cfg_grid = with_p == (c.da_with_p != 0);       // the plan's default dA launch, else the form without X A^T
+  if (with_p && !cfg_grid) return LORA_ERR_INVALID_ARG;     // only the plan's own with-side grid is sized for TMEM and scratch
+  GradJob j;
+  if (!fill_da_job(pl, X, A, scale, dA, with_p, cfg_grid ? c.grad_feat_chunk : c.dan_feat_chunk,
+                   cfg_grid ? c.da_token_chunks : c.dan_token_chunks, &j))
+    return LORA_ERR_CUDA;
+  if (with_p && j.g.n_feat_chunks > 1 && !ensure_counters(pl, st)) return LORA_ERR_CUDA;
+  if (launch_grad(j.tmS, j.tmR, j.tmSide, j.g, st) != cudaSuccess) return LORA_ERR_CUDA;
+  g_launches.fetch_add(1);
   return LORA_OK;
 }
 
-// ---- dB = Pt-contraction over dY ----
-int launch_db(lora_plan* pl, const void* dY, float scale, void* dB, cudaStream_t st, const void* B_for_q = nullptr,
-              int tok_override = 0) {
-  const lora_shape_t& s = pl->shape;
+int launch_db(lora_plan* pl, const void* dY, float scale, void* dB, cudaStream_t st, const void* B_for_q = nullptr) {
   const lora_kernel_config_t& c = pl->cfg;
-  const WsLayout& w = pl->ws;
-  const WsPtrs q = ws_ptrs(pl);
-  uint8_t* ws = q.base;
-  __nv_bfloat16* pt = q.pt;
-  {
-    const bool with_q = B_for_q != nullptr;     // also leave Qt = s (dY B)^T (saved-P backward)
-    CUtensorMap tmS, tmR, tmSide;
-    bool ok = make_bf16_tmap(&tmS, dY, s.d_out, s.T, s.d_out, 64, kGradSlab);
-    ok = ok && make_bf16_tmap(&tmR, pt, s.T, c.r_pad, w.ld_t, 64, c.r_pad);
-    if (with_q) ok = ok && make_bf16_tmap(&tmSide, B_for_q, s.r, s.d_out, s.r, 64, 64);
-    if (!ok) return LORA_ERR_CUDA;
-    GradParams g{};
-    g.T = static_cast<int>(s.T);
-    g.C = static_cast<int>(s.d_out);
-    g.r = static_cast<int>(s.r);
-    g.r_pad = c.r_pad;
-    g.feat_chunk = c.db_feat_chunk;
-    g.n_feat_chunks = c.db_feat_chunks;
-    g.n_token_chunks = tok_override > 0 ? tok_override : c.db_token_chunks;
-    g.n_slabs = w.n_slabs;
-    g.stages = with_q ? 4 : c.db_stages;
-    g.with_p = with_q ? 1 : 0;
-    g.side_mn = with_q ? 1 : 0;
-    g.do_out = 1;
-    g.out_is_da = 0;
-    g.accumulate = pl->accumulate ? 1 : 0;
-    g.scale = scale;
-    g.out = static_cast<float*>(dB);
-    g.out_part = reinterpret_cast<float*>(ws + w.db_part);
-    g.c_pad = w.c_pad_b;
-    g.p_part = with_q ? reinterpret_cast<float*>(ws + w.q_part) : nullptr;
-    g.pt_out = with_q ? q.qt : nullptr;
-    g.ld_t = w.ld_t;
-    g.status = pl->d_status;
-    g.wait_limit = pl->wait_limit;
-    if (launch_grad(tmS, tmR, with_q ? tmSide : tmR, g, st) != cudaSuccess) return LORA_ERR_CUDA;
-    g_launches.fetch_add(grad_is_direct(g) ? 1 : 2);
-  }
+  const bool with_q = B_for_q != nullptr;
+  GradJob j;
+  if (!fill_db_job(pl, dY, scale, dB, B_for_q, with_q ? c.dbq_feat_chunk : c.db_feat_chunk,
+                   with_q ? c.dbq_token_chunks : c.db_token_chunks, &j))
+    return LORA_ERR_CUDA;
+  if (with_q && j.g.n_feat_chunks > 1 && !ensure_counters(pl, st)) return LORA_ERR_CUDA;
+  if (launch_grad(j.tmS, j.tmR, j.tmSide, j.g, st) != cudaSuccess) return LORA_ERR_CUDA;
+  g_launches.fetch_add(1);
   return LORA_OK;
+}
+
+// dA and dB in ONE launch (both second factors are ready): the feature chunks of X and of dY side by side
+int launch_grad_pair(lora_plan* pl, const void* X, const void* dY, const void* A, float scale, void* dA, void* dB,
+                     cudaStream_t st) {
+  const lora_kernel_config_t& c = pl->cfg;
+  GradJob ja, jb;
+  if (!fill_da_job(pl, X, A, scale, dA, false, c.pair_feat_chunk, c.pair_token_chunks, &ja) ||
+      !fill_db_job(pl, dY, scale, dB, nullptr, c.pair_feat_chunk, c.pair_token_chunks, &jb))
+    return LORA_ERR_CUDA;
+  const CUtensorMap* const t0[3] = {&ja.tmS, &ja.tmR, &ja.tmSide};
+  const CUtensorMap* const t1[3] = {&jb.tmS, &jb.tmR, &jb.tmSide};
+  if (launch_grad2(t0, ja.g, t1, &jb.g, st) != cudaSuccess) return LORA_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return LORA_OK;
+}
+
+// ---- dA stage of the plain backward: dA, and Pt = s (X A^T)^T left for the dB launch.  X A^T rides the dA launch or,
+//      for large ranks, comes from its own skinny pass over X first (cfg.da_with_p) ----
+int launch_da_stage(lora_plan* pl, const void* X, const void* A, float scale, void* dA, cudaStream_t st) {
+  const bool with_p = pl->cfg.da_with_p != 0;
+  int rc = LORA_OK;
+  if (!with_p) rc = launch_side_prepass(pl, X, pl->shape.d_in, A, false, scale, ws_ptrs(pl).pt, st);
+  if (rc == LORA_OK) rc = launch_da(pl, X, A, scale, dA, st, with_p);
+  return rc;
+}
+
+// ---- everything of the backward pass that follows the dX GEMM: dA and dB (Qt is in the workspace; Pt only if p_ready) ----
+int launch_adapter_grads(lora_plan* pl, const void* dY, const void* X, const void* A, float scale, void* dA, void* dB,
+                         bool p_ready, cudaStream_t st) {
+  int rc = LORA_OK;
+  if (pl->cfg.bwd_merged) {
+    if (!p_ready) rc = launch_side_prepass(pl, X, pl->shape.d_in, A, false, scale, ws_ptrs(pl).pt, st);
+    if (rc == LORA_OK) rc = launch_grad_pair(pl, X, dY, A, scale, dA, dB, st);
+    return rc;
+  }
+  if (p_ready) rc = launch_da(pl, X, A, scale, dA, st, false);
+  else rc = launch_da_stage(pl, X, A, scale, dA, st);
+  if (rc == LORA_OK) rc = launch_db(pl, dY, scale, dB, st);
+  return rc;
 }
 
 // ---- NF4 frozen weight (Q+LoRA): both GEMMs run K-extended on CTA pairs with the dequantising kernel variant ----
@@ -802,8 +928,10 @@ int launch_dx_nf4(lora_plan* pl, const void* dY, const void* codes, const void* 
   const lora_shape_t& s = pl->shape;
   const lora_kernel_config_t& c = pl->cfg;
   __nv_bfloat16* qt = ws_ptrs(pl).qt;
-  int rc = launch_side_prepass(pl, dY, s.d_out, B, true, scale, qt, st);   // Qt = s (dY B)^T
-  if (rc != LORA_OK) return rc;
+  if (!pl->q_ready) {
+    const int rc = launch_side_prepass(pl, dY, s.d_out, B, true, scale, qt, st);   // Qt = s (dY B)^T
+    if (rc != LORA_OK) return rc;
+  }
   const int pairs = pl->num_sms / 2;
   const int bn = 256;                 // each CTA's 128 weight columns are two whole quantisation blocks
   CUtensorMap tmdY, tmCodes, tmAbsmax, tmQt, tmA, tmdX;
@@ -924,7 +1052,14 @@ int lora_plan_create(const lora_shape_t* shape, int device, lora_plan_t** out) {
   pl->shape = *shape;
   pl->device = device;
   pl->num_sms = prop.multiProcessorCount;
-  rc = select_config(shape, pl->num_sms, &pl->cfg);
+  pl->d_status = nullptr;
+  if (gemm_configure() != cudaSuccess || gemm_pair_configure() != cudaSuccess || grad_configure() != cudaSuccess || encode_fn() == nullptr) {
+    cudaGetLastError();
+    delete pl;
+    return LORA_ERR_CUDA;
+  }
+  device_caps(device, pl->num_sms, pl->caps);
+  rc = select_config(shape, pl->num_sms, &pl->cfg, pl->caps);
   if (rc != LORA_OK) {
     delete pl;
     return rc;
@@ -942,18 +1077,8 @@ int lora_plan_create(const lora_shape_t* shape, int device, lora_plan_t** out) {
     const long long v = std::atoll(f);
     if (v >= 1000) pl->wait_limit = v;
   }
-  pl->d_status = nullptr;
-  pl->side_stream = nullptr;
-  pl->ev_fork = pl->ev_join = nullptr;
-  if (pl->cfg.overlap_sms > 0 &&
-      (cudaStreamCreateWithFlags(&pl->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
-       cudaEventCreateWithFlags(&pl->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-       cudaEventCreateWithFlags(&pl->ev_join, cudaEventDisableTiming) != cudaSuccess)) {
-    cudaGetLastError();
-    pl->cfg.overlap_sms = 0;         // no second stream: fall back to the serial order
-  }
-  if (gemm_configure() != cudaSuccess || gemm_pair_configure() != cudaSuccess || grad_configure() != cudaSuccess || encode_fn() == nullptr ||
-      cudaMalloc(&pl->d_status, 256) != cudaSuccess || cudaMemset(pl->d_status, 0, 256) != cudaSuccess) {
+  pl->counters_clean = false;
+  if (cudaMalloc(&pl->d_status, 256) != cudaSuccess || cudaMemset(pl->d_status, 0, 256) != cudaSuccess) {
     cudaGetLastError();
     if (pl->d_status) cudaFree(pl->d_status);
     delete pl;
@@ -967,9 +1092,6 @@ int lora_plan_destroy(lora_plan_t* plan) {
   if (plan == nullptr) return LORA_ERR_INVALID_ARG;
   DeviceGuard guard(plan->device);
   if (plan->d_status) cudaFree(plan->d_status);
-  if (plan->ev_fork) cudaEventDestroy(plan->ev_fork);
-  if (plan->ev_join) cudaEventDestroy(plan->ev_join);
-  if (plan->side_stream) cudaStreamDestroy(plan->side_stream);
   delete plan;
   return LORA_OK;
 }
@@ -994,6 +1116,7 @@ int lora_plan_set_workspace(lora_plan_t* plan, void* dev_ptr, size_t bytes) {
   plan->workspace_bytes = bytes;
   plan->p_saved = false;
   plan->q_staged = false;
+  plan->counters_clean = false;
   return LORA_OK;
 }
 
@@ -1027,10 +1150,11 @@ int lora_debug_starved_wait(lora_plan_t* plan, const void* S, int64_t T, int64_t
   g.n_token_chunks = 1;              // one CTA, direct mode: nothing but `status` can be written
   g.n_slabs = ceil_div(T, kGradSlab);
   g.stages = 2;
+  g.rt_bufs = 2;
+  g.tmem_cols = grad_tmem_cols(g.feat_chunk, r_pad, true, false);
   g.do_out = 1;
   g.scale = 1.f;
   g.out = static_cast<float*>(out);
-  g.c_pad = static_cast<int>(C);
   g.ld_t = static_cast<int>(T);
   g.status = plan->d_status;
   g.wait_limit = plan->wait_limit;
@@ -1051,14 +1175,14 @@ int lora_plan_describe(const lora_plan_t* plan, char* buf, size_t n) {
   const lora_kernel_config_t& c = plan->cfg;
   std::snprintf(buf, n,
                 "T=%lld d_in=%lld d_out=%lld r=%lld | sms=%d cta_group=%d tile fwd %dx%dx64 dx %dx%dx64 stages=%d/%d group_m=%d "
-                "split_k=%d/%d r_pad=%d ctas fwd=%d dx=%d tail_delay=%d | grad chunk=%d/%d stages=%d/%d dA grid=%dx%d dB grid=%dx%d "
-                "| bwd workspace=%zu B",
+                "split_k=%d/%d r_pad=%d ctas fwd=%d dx=%d tail_delay=%d | grad chunk=%d/%d stages=%d/%d dA grid=%dx%d%s dB grid=%dx%d "
+                "(feature chunks x cluster of token chunks) | bwd workspace=%zu B",
                 (long long)plan->shape.T, (long long)plan->shape.d_in, (long long)plan->shape.d_out,
                 (long long)plan->shape.r, plan->num_sms, c.cta_group, c.block_m, c.fwd_block_n, c.block_m, c.dx_block_n,
                 c.stages, c.dx_stages, c.group_m, c.split_k, c.dx_split_k,
                 c.r_pad, c.fwd_ctas, c.dx_ctas, c.tail_delay, c.grad_feat_chunk, c.db_feat_chunk, c.grad_stages, c.db_stages,
                 c.da_feat_chunks,
-                c.da_token_chunks, c.db_feat_chunks, c.db_token_chunks, plan->ws.total);
+                c.da_token_chunks, c.da_with_p ? " +XA^T" : " (XA^T in its own pass)", c.db_feat_chunks, c.db_token_chunks, plan->ws.total);
   return LORA_OK;
 }
 
@@ -1091,27 +1215,48 @@ int lora_linear_bwd(lora_plan_t* plan, const void* dY, const void* X, const void
     return LORA_ERR_MISALIGNED;
   if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
   plan->q_staged = false;      // this call overwrites the staged s (dY B)^T
-  if (plan->cfg.overlap_sms > 0) {
-    // dY B pre-pass, then the dX GEMM on `stream` beside dA -> dB on the plan's second stream (fork / join by events)
-    const lora_kernel_config_t& c = plan->cfg;
-    int rc = launch_side_prepass(plan, dY, plan->shape.d_out, B, true, scale, ws_ptrs(plan).qt, st);
-    if (rc != LORA_OK) return rc;
-    if (cudaEventRecord(plan->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(plan->side_stream, plan->ev_fork, 0) != cudaSuccess)
-      return LORA_ERR_CUDA;
-    plan->q_ready = true;
-    rc = launch_dx(plan, dY, W, A, B, scale, dX, st, c.ov_dx_ctas);
-    plan->q_ready = false;
-    if (rc == LORA_OK) rc = launch_da(plan, X, A, scale, dA, plan->side_stream, true, c.ov_da_token_chunks);
-    if (rc == LORA_OK) rc = launch_db(plan, dY, scale, dB, plan->side_stream, nullptr, c.ov_db_token_chunks);
-    // join even after a failed launch, so that `stream` never runs ahead of work already queued on the second stream
-    if (cudaEventRecord(plan->ev_join, plan->side_stream) != cudaSuccess || cudaStreamWaitEvent(st, plan->ev_join, 0) != cudaSuccess)
-      return LORA_ERR_CUDA;
-    return rc;
+  int rc = LORA_OK;
+  bool p_ready = false;
+  if (plan->cfg.bwd_merged && plan->cfg.cta_group == 2) {
+    rc = launch_side_pair(plan, dY, B, X, A, scale, st);        // s (dY B)^T and s (X A^T)^T in one launch
+    plan->q_ready = p_ready = true;
   }
-  int rc = launch_dx(plan, dY, W, A, B, scale, dX, st);
-  if (rc == LORA_OK) rc = launch_da(plan, X, A, scale, dA, st);
-  if (rc == LORA_OK) rc = launch_db(plan, dY, scale, dB, st);
+  if (rc == LORA_OK) rc = launch_dx(plan, dY, W, A, B, scale, dX, st);
+  plan->q_ready = false;
+  if (rc == LORA_OK) rc = launch_adapter_grads(plan, dY, X, A, scale, dA, dB, p_ready, st);
   return rc;
+}
+
+int lora_linear_bwd_sides(lora_plan_t* plan, const void* dY, const void* X, const void* A, const void* B, float scale,
+                          void* stream) {
+  if (plan == nullptr) return LORA_ERR_INVALID_ARG;
+  if (plan->shape.T == 0) return LORA_OK;
+  if (!dY || !X || !A || !B) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(dY) || !aligned16(X) || !aligned16(A) || !aligned16(B)) return LORA_ERR_MISALIGNED;
+  if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
+  DeviceGuard guard(plan->device);
+  const int rc = launch_side_pair(plan, dY, B, X, A, scale, static_cast<cudaStream_t>(stream));
+  if (rc == LORA_OK) plan->q_staged = plan->cfg.cta_group == 2;    // the single-CTA dX kernel computes dY B itself
+  return rc;
+}
+
+int lora_linear_bwd_grads(lora_plan_t* plan, const void* dY, const void* X, const void* A, float scale, void* dA, void* dB,
+                          void* stream) {
+  if (plan == nullptr || !dA || !dB) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(dA) || !aligned16(dB)) return LORA_ERR_MISALIGNED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  DeviceGuard guard(plan->device);
+  if (plan->shape.T == 0) {
+    if (plan->accumulate) return LORA_OK;
+    if (cudaMemsetAsync(dA, 0, sizeof(float) * plan->shape.r * plan->shape.d_in, st) != cudaSuccess ||
+        cudaMemsetAsync(dB, 0, sizeof(float) * plan->shape.d_out * plan->shape.r, st) != cudaSuccess)
+      return LORA_ERR_CUDA;
+    return LORA_OK;
+  }
+  if (!dY || !X || !A) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(dY) || !aligned16(X) || !aligned16(A)) return LORA_ERR_MISALIGNED;
+  if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
+  return launch_grad_pair(plan, X, dY, A, scale, dA, dB, st);
 }
 
 int lora_linear_bwd_saved_p(lora_plan_t* plan, const void* dY, const void* X, const void* W, const void* A, const void* B,
@@ -1176,7 +1321,7 @@ int lora_linear_bwd_da(lora_plan_t* plan, const void* X, const void* A, float sc
   if (!X || !A) return LORA_ERR_INVALID_ARG;
   if (!aligned16(X) || !aligned16(A)) return LORA_ERR_MISALIGNED;
   if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
-  return launch_da(plan, X, A, scale, dA, static_cast<cudaStream_t>(stream));
+  return launch_da_stage(plan, X, A, scale, dA, static_cast<cudaStream_t>(stream));
 }
 
 int lora_linear_bwd_db(lora_plan_t* plan, const void* dY, float scale, void* dB, void* stream) {
@@ -1271,16 +1416,27 @@ int lora_linear_bwd_nf4(lora_plan_t* plan, const void* dY, const void* X, const 
                               plan->shape.d_in, static_cast<__nv_bfloat16*>(w_scratch), plan->num_sms, st) != cudaSuccess)
       return LORA_ERR_CUDA;
     g_launches.fetch_add(1);
-    int rc2 = launch_dx(plan, dY, w_scratch, A, B, scale, dX, st);
-    if (rc2 == LORA_OK) rc2 = launch_da(plan, X, A, scale, dA, st);
-    if (rc2 == LORA_OK) rc2 = launch_db(plan, dY, scale, dB, st);
+    int rc2 = LORA_OK;
+    bool p_ready = false;
+    if (plan->cfg.bwd_merged && plan->cfg.cta_group == 2) {
+      rc2 = launch_side_pair(plan, dY, B, X, A, scale, st);
+      plan->q_ready = p_ready = true;
+    }
+    if (rc2 == LORA_OK) rc2 = launch_dx(plan, dY, w_scratch, A, B, scale, dX, st);
+    plan->q_ready = false;
+    if (rc2 == LORA_OK) rc2 = launch_adapter_grads(plan, dY, X, A, scale, dA, dB, p_ready, st);
     return rc2;
   }
   int rc = check_nf4(plan);
   if (rc != LORA_OK) return rc;
-  rc = launch_dx_nf4(plan, dY, W_codes, W_absmax, A, B, scale, dX, st);
-  if (rc == LORA_OK) rc = launch_da(plan, X, A, scale, dA, st);
-  if (rc == LORA_OK) rc = launch_db(plan, dY, scale, dB, st);
+  bool p_ready = false;
+  if (plan->cfg.bwd_merged) {
+    rc = launch_side_pair(plan, dY, B, X, A, scale, st);
+    plan->q_ready = p_ready = true;
+  }
+  if (rc == LORA_OK) rc = launch_dx_nf4(plan, dY, W_codes, W_absmax, A, B, scale, dX, st);
+  plan->q_ready = false;
+  if (rc == LORA_OK) rc = launch_adapter_grads(plan, dY, X, A, scale, dA, dB, p_ready, st);
   return rc;
 }
 
@@ -1383,6 +1539,24 @@ int lora_last_device_status(lora_plan_t* plan, void* stream, int* code, char* ms
                                "other wait"};
   if (msg && n) std::snprintf(msg, n, "device wait ran out: %s (CTA %u)", what[word & 7u], word >> 8);
   if (cudaMemset(plan->d_status, 0, 256) != cudaSuccess) return LORA_ERR_CUDA;
+  plan->counters_clean = false;      // an abandoned launch may have left arrival counters behind
+  return LORA_OK;
+}
+
+int lora_plan_last_gemm_clock(lora_plan_t* plan, void* stream, double* sm_mhz, double* busy_us) {
+  if (plan == nullptr || sm_mhz == nullptr || busy_us == nullptr) return LORA_ERR_INVALID_ARG;
+  DeviceGuard guard(plan->device);
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return LORA_ERR_CUDA;
+  unsigned long long rec[4] = {0, 0, 0, 0};
+  if (cudaMemcpy(rec, reinterpret_cast<unsigned char*>(plan->d_status) + 64, sizeof(rec), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return LORA_ERR_CUDA;
+  *sm_mhz = 0.0;
+  *busy_us = 0.0;
+  if (rec[1] > rec[0] && rec[3] > rec[2]) {
+    const double ns = static_cast<double>(rec[1] - rec[0]);
+    *busy_us = ns * 1e-3;
+    *sm_mhz = static_cast<double>(rec[3] - rec[2]) / ns * 1e3;     // ticks per nanosecond -> MHz
+  }
   return LORA_OK;
 }
 

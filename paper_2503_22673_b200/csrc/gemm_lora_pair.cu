@@ -147,6 +147,14 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
   tc_fence_after();
   pdl_wait();                   // everything above overlapped the previous kernel's tail; global memory from here on
   const uint32_t tmem_base = *tmem_slot;
+  // one thread of the grid notes wall time and SM clock when its CTA starts working and when it leaves: the host derives
+  // the SM frequency this launch really ran at (bytes 64..95 of the status block, see lora_plan_last_gemm_clock)
+  unsigned long long t_begin = 0;
+  long long c_begin = 0;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_begin));
+    c_begin = clock64();
+  }
 
   const int G = gridDim.x >> 1;                 // CTA pairs
   const int pair = blockIdx.x >> 1;
@@ -584,6 +592,15 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
     __syncwarp();
     tc_fence_after();
     tmem_dealloc_pair(tmem_base, 512);
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    unsigned long long t_end;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_end));
+    unsigned long long* rec = reinterpret_cast<unsigned long long*>(p.status) + 8;
+    rec[0] = t_begin;
+    rec[1] = t_end;
+    rec[2] = static_cast<unsigned long long>(c_begin);
+    rec[3] = static_cast<unsigned long long>(clock64());
   }
 }
 

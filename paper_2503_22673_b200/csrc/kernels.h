@@ -127,29 +127,36 @@ cudaError_t launch_gemm_dx(const CUtensorMap& tmdY, const CUtensorMap& tmW, cons
                            cudaStream_t stream);
 cudaError_t gemm_configure();   // opt in to the large dynamic shared memory (once per device)
 
-// ---- adapter gradients: tall-skinny contraction over tokens -----------------------------------
-constexpr int kGradThreads = 256;          // warps 0,1 TMA producers, 2 MMA + TMEM, 3 second-factor loader, 4..7 epilogue
+// ---- adapter gradients and skinny side products: tall-skinny contractions over one stream of tokens --------
+constexpr int kGradProducerWarps = 4;      // warps 0..3: TMA producers of the streamed tiles (ring items round-robin)
+constexpr int kGradEpiGroups = 2;          // two groups of four epilogue warps; the per-slab work alternates between them
+constexpr int kGradThreads = 32 * (kGradProducerWarps + 2 + 4 * kGradEpiGroups);   // + MMA warp + second-factor loader
 constexpr int kGradSlab = 128;             // tokens per slab
 constexpr int kGradStageBytes = 2 * kBlockM * 128;   // 128 tokens x 128 features, bf16
 constexpr int kGradMaxStages = 6;
+constexpr int kGradMaxRtBufs = 4;          // ring of second-factor slabs (a gradient CTA with one block needs one per tile)
+constexpr int kGradPBufs = 4;              // TMEM buffers of the per-slab side product (r_pad columns each)
+constexpr int kGradMaxCluster = 16;        // token chunks of one feature chunk form a thread-block cluster of this size at most
 
 struct GradParams {
   int T, C;               // tokens, features of the streamed matrix (d_in for dA, d_out for dB)
   int r, r_pad;
   int feat_chunk;         // features per CTA (multiple of 128)
-  int n_feat_chunks, n_token_chunks, n_slabs;
+  int n_feat_chunks;      // grid x
+  int n_token_chunks;     // grid y = cluster size along y when do_out (the cluster sums the gradient over its token chunks)
+  int n_slabs;
   int stages;
+  int rt_bufs;            // depth of the second-factor ring (1 .. kGradMaxRtBufs)
+  int tmem_cols;          // TMEM columns to allocate (power of two >= 32)
   int with_p;             // 1: also accumulate the side product S * side^T for each slab (X A^T, or dY B)
   int side_mn;            // side operand: 0 = A [r, C] (K-major rows), 1 = B [C, r] (MN-major, natural layout)
   int do_out;             // 0: side product only (no second factor, no gradient)
   int out_is_da;          // 1: out[j * C + c] (dA), 0: out[c * r + j] (dB)
   int accumulate;         // 1: out += result (gradient accumulation over micro-batches), 0: out = result
-  int direct;             // set by launch_grad: no cross-CTA sums are needed, the kernel writes out / pt_out itself
   float scale;
   float* out;             // final fp32 gradient
-  float* out_part;        // [n_token_chunks][r_pad][C_pad]  partial sums (fixed-order reduction)
-  int c_pad;              // row pitch of out_part
-  float* p_part;          // [n_feat_chunks][r_pad][ld_t] partial X A^T (with_p)
+  float* p_part;          // [n_feat_chunks][r_pad][ld_t] partial X A^T (with_p and more than one feature chunk)
+  int* side_count;        // [n_slabs] arrival counters of the side-product partials; zero before and after every launch
   __nv_bfloat16* pt_out;  // [r_pad][ld_t]: scale * (X A^T)^T as bf16 (with_p)
   int ld_t;
   unsigned* status;
@@ -157,14 +164,46 @@ struct GradParams {
   int debug_no_second_factor;   // test hook: the second-factor loader issues nothing, so the MMA warp's wait runs out
 };
 
+// What the grid rule chose for one streaming launch
+struct GradGrid {
+  int feat_chunk, n_feat, n_tok, stages, tmem_cols;
+};
+// Grid of a launch that computes the gradient of one streamed matrix with C features (with or without the side product),
+// or of two matrices with C and C2 features side by side (C2 = 0: one job): feature chunk width and cluster size
+// (= token chunks) with the lowest modelled time among those that fit TMEM (feat_chunk / 128 x r_pad + side buffers <= 512
+// columns) and are resident at once (caps[cs] = CTAs resident at once in clusters of cs CTAs, cs = 1 .. kGradMaxCluster).
+// n_feat counts the feature chunks of both jobs.
+GradGrid grad_pick_grid(long long T, long long C, long long C2, int r_pad, bool with_p, bool side_mn, const int* caps);
+// caps[0 .. kGradMaxCluster] estimated from the SM count alone (host-only selector calls) / asked from the current device
+void grad_default_caps(int num_sms, int* caps);
+void grad_device_caps(int num_sms, int* caps);
+// TMEM columns a launch allocates: gradient sums + side-product buffers, rounded up to a power of two >= 32
+int grad_tmem_cols(int feat_chunk, int r_pad, bool do_out, bool with_p);
+
+// depth of the second-factor ring and of the stream ring that fit 227 KiB of shared memory together
+int grad_rt_bufs(int r_pad, bool do_out);
+int grad_stages(int r_pad, bool with_p, bool side_mn, bool do_out);
+
+// One launch of the streaming kernel: one or two jobs side by side (CTAs with blockIdx.x < split_x run job 0)
+struct GradLaunch {
+  GradParams job[2];
+  int split_x;
+};
+
 size_t grad_smem_bytes(const GradParams& p);
+// opt in to the large dynamic shared memory and to clusters of more than 8 CTAs (once per device)
 cudaError_t grad_configure();
+// Largest grid (in CTAs) of `cluster`-CTA clusters along y that is resident at once on the current device, for the given
+// launch shape; 0 when the query fails.
+int grad_max_resident_ctas(int cluster, size_t smem_bytes);
 // tmS: streamed matrix [T, C] box [64 features, 128 tokens]; tmR: [r_pad, T] box [64 tokens, r_pad];
-// tmA: A [r, C] box [64 features, r_pad] (only read when with_p).  Launches the streaming kernel and the
-// fixed-order finalize kernel (2 launches).
+// tmA: side operand (only read when with_p).  ONE launch: the gradient is summed over the token chunks inside the cluster
+// (distributed shared memory, rank order), the side product over the feature chunks by the last CTA to arrive (chunk order).
 cudaError_t launch_grad(const CUtensorMap& tmS, const CUtensorMap& tmR, const CUtensorMap& tmA,
                         const GradParams& p, cudaStream_t stream);
-// true when launch_grad will run the streaming kernel alone (1 launch instead of 2)
-bool grad_is_direct(const GradParams& p);
+// Two jobs in one launch (p1 == nullptr: one job).  tm0 / tm1 = {streamed matrix, second factor, side operand} of each
+// job.  Both jobs compute a gradient with the same cluster size, or both compute only a side product.
+cudaError_t launch_grad2(const CUtensorMap* const tm0[3], const GradParams& p0, const CUtensorMap* const tm1[3],
+                         const GradParams* p1, cudaStream_t stream);
 
 }  // namespace lora

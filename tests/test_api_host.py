@@ -69,33 +69,38 @@ def test_selector_invariants(shape):
     if T >= 1024:
         assert c["split_k"] == 1 and c["dx_split_k"] == 1          # the benchmark shapes fill the GPU without it
     n_slabs = -(-T // 128)
-    assert 1 <= c["da_token_chunks"] <= n_slabs and 1 <= c["db_token_chunks"] <= n_slabs
-    for fc, nf, nt, st, with_p in ((c["grad_feat_chunk"], c["da_feat_chunks"], c["da_token_chunks"], c["grad_stages"], 1),
-                                   (c["db_feat_chunk"], c["db_feat_chunks"], c["db_token_chunks"], c["db_stages"], 0)):
-        assert fc % 128 == 0 and (fc // 128) * c["r_pad"] + 2 * c["r_pad"] <= 512        # TMEM columns
-        assert nf * nt <= max(148, nf)                                                   # one wave of CTAs
+    assert c["da_with_p"] == (1 if c["r_pad"] <= 32 else 0)       # large ranks recompute X A^T in their own pass over X
+    grids = ((c["grad_feat_chunk"], c["da_feat_chunks"], c["da_token_chunks"], c["grad_stages"], c["da_with_p"], 0, d_in),
+             (c["db_feat_chunk"], c["db_feat_chunks"], c["db_token_chunks"], c["db_stages"], 0, 0, d_out),
+             (c["dan_feat_chunk"], c["dan_feat_chunks"], c["dan_token_chunks"], c["db_stages"], 0, 0, d_in),
+             (c["dbq_feat_chunk"], c["dbq_feat_chunks"], c["dbq_token_chunks"], 4, 1, 1, d_out))
+    for fc, nf, nt, st, with_p, side_mn, C in grids:
+        assert fc % 128 == 0 and (fc // 128) * c["r_pad"] + with_p * 4 * c["r_pad"] <= 512   # TMEM: sums + side buffers
+        assert nf == -(-C // fc)
+        assert 1 <= nt <= 16 and nt <= n_slabs                     # the token chunks of a feature chunk are ONE cluster
+        assert nf * nt <= 148                                      # resident at once
         assert 2 <= st <= 6
-        assert st * (32768 + with_p * 2 * c["r_pad"] * 128) + 4 * c["r_pad"] * 128 + 2048 <= 232448
-    assert c["da_feat_chunks"] == -(-d_in // c["grad_feat_chunk"])
-    assert c["db_feat_chunks"] == -(-d_out // c["db_feat_chunk"])
+        side = (8192 if side_mn else c["r_pad"] * 128) * 2 * with_p
+        assert st * (32768 + side) + 4 * c["r_pad"] * 128 + 2048 <= 232448
 
 
-@pytest.mark.parametrize("shape,can", [((8192, 4096, 4096, 16), True), ((16384, 14336, 4096, 64), True),
-                                       ((256, 512, 512, 8), False), ((128, 4096, 4096, 16), False)])
-def test_selector_overlapped_backward_is_opt_in(shape, can, monkeypatch):
-    """The dA / dB passes run beside the dX GEMM only when LORA_OVERLAP_SMS asks for it (measured: no reliable gain),
-    and only on grids with at least one tile per CTA pair."""
-    T, d_in, d_out, r = shape
-    monkeypatch.delenv("LORA_OVERLAP_SMS", raising=False)
-    c = binding.select_config(T, d_in, d_out, r, 148)
-    assert c["overlap_sms"] == 0 and c["ov_dx_ctas"] == c["dx_ctas"] and c["ov_da_token_chunks"] == c["da_token_chunks"]
-    monkeypatch.setenv("LORA_OVERLAP_SMS", "16")
-    c = binding.select_config(T, d_in, d_out, r, 148)
-    assert (c["overlap_sms"] == 16) == can
-    if can:
-        assert c["ov_dx_ctas"] == 2 * (74 - 8)
-        assert 1 <= c["ov_da_token_chunks"] <= c["da_token_chunks"] and 1 <= c["ov_db_token_chunks"] <= c["db_token_chunks"]
-        assert c["da_feat_chunks"] * c["ov_da_token_chunks"] <= max(16, c["da_feat_chunks"])
+def test_selector_grad_grids_of_the_benchmark_shapes():
+    """The dA + dB launch of the merged backward: 128-feature blocks of X and dY side by side, each block's token chunks
+    one small cluster, so that the grid is as close to the SM count as whole clusters allow."""
+    q = binding.select_config(8192, 4096, 4096, 16, 148)
+    assert q["bwd_merged"] == 1
+    assert (q["pair_feat_chunk"], q["pair_feat_chunks"], q["pair_token_chunks"]) == (128, 64, 2)
+    gate = binding.select_config(16384, 4096, 14336, 16, 148)       # 32 + 112 blocks: one CTA each, no sum across CTAs
+    assert (gate["pair_feat_chunk"], gate["pair_feat_chunks"], gate["pair_token_chunks"]) == (128, 144, 1)
+    down = binding.select_config(16384, 14336, 4096, 64, 148)
+    assert (down["pair_feat_chunks"], down["pair_token_chunks"]) == (144, 1) and down["da_with_p"] == 0
+    kv = binding.select_config(32768, 4096, 1024, 16, 148)
+    assert (kv["pair_feat_chunks"], kv["pair_token_chunks"]) == (40, 3)
+    tiny = binding.select_config(256, 512, 512, 8, 148)            # 256 KiB streams: no cluster, nothing summed across CTAs
+    assert tiny["da_token_chunks"] == 1 and tiny["db_token_chunks"] == 1 and tiny["pair_token_chunks"] == 1
+    for c in (q, gate, down, kv, tiny):
+        assert c["pair_feat_chunk"] % 128 == 0 and (c["pair_feat_chunk"] // 128) * c["r_pad"] <= 512
+        assert c["pair_feat_chunks"] * c["pair_token_chunks"] <= 148 and 1 <= c["pair_token_chunks"] <= 16
 
 
 def test_selector_picks_by_grid_size():

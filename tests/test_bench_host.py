@@ -46,7 +46,9 @@ def test_single_rank_helpers():
     assert bench.workload_name(1).startswith("config1 q_proj")
     pk = bench.peaks()
     assert pk["hbm_gbs"] > 1000 and pk["bf16_tflops"] > 500 and pk["source"] in ("measured", "fallback")
-    assert len(bench.gemm_source_sha()) == 16
+    assert len(bench.source_sha("gemm")) == 16 and bench.source_sha("gemm") != bench.source_sha("adapter_grad")
+    p = bench.inputs_workload(1)[0]
+    assert bench.stage_bytes(p, "grads") > bench.stage_bytes(p, "dA") + bench.stage_bytes(p, "dB") - 4.0 * p.T * p.r - 1
 
 
 def test_reference_arm_prints_one_line_on_rank0_and_nothing_elsewhere():

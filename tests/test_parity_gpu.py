@@ -179,17 +179,28 @@ def test_bitwise_reproducible():
         assert torch.equal(a[k].view(it), b[k].view(it)), k
 
 
-def test_stage_entry_points_match_the_single_call():
-    p, t = inputs.draw_custom(700, 520, 392, 16, 2.0, seed=13)
-    d = {k: dev(v) for k, v in t.items()}
-    plan = binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r)
-    dX1, dA1, dB1 = plan.bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], p.scale)
-    dX2, dA2, dB2 = torch.empty_like(dX1), torch.empty_like(dA1), torch.empty_like(dB1)
-    plan.bwd_stages(d["dY"], d["X"], d["W"], d["A"], d["B"], p.scale, dX2, dA2, dB2)
-    torch.cuda.synchronize()
-    assert torch.equal(dX1.view(torch.int16), dX2.view(torch.int16))
-    assert torch.equal(dA1, dA2) and torch.equal(dB1, dB2)
-    plan.close()
+@pytest.mark.parametrize("merged", ["1", "0"])
+def test_stage_entry_points_match_the_single_call(merged, monkeypatch):
+    """lora_linear_bwd against the same launches issued one by one through the stage calls (both forms of the backward
+    pass: dY B + X A^T | GEMM | dA + dB, and dY B | GEMM | dA | dB): bit-identical."""
+    monkeypatch.setenv("LORA_FORCE_BWD_MERGED", merged)
+    for T in (700, 100):                                            # CTA pairs; single-CTA GEMM that computes dY B itself
+        p, t = inputs.draw_custom(T, 520, 392, 16, 2.0, seed=13)
+        d = {k: dev(v) for k, v in t.items()}
+        plan = binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r)
+        assert plan.config()["bwd_merged"] == int(merged)
+        assert len(plan.bwd_stage_names()) == (3 if merged == "1" else 4)
+        dX1, dA1, dB1 = plan.bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], p.scale)
+        dX2, dA2, dB2 = torch.empty_like(dX1), torch.empty_like(dA1), torch.empty_like(dB1)
+        plan.bwd_stages(d["dY"], d["X"], d["W"], d["A"], d["B"], p.scale, dX2, dA2, dB2)
+        torch.cuda.synchronize()
+        assert torch.equal(dX1.view(torch.int16), dX2.view(torch.int16))
+        assert torch.equal(dA1, dA2) and torch.equal(dB1, dB2)
+        f = {k: inputs.bf16_to_f64(v) for k, v in t.items()}
+        dXr, dAr, dBr = oracle.backward(f["dY"], f["X"], f["W"], f["A"], f["B"], p.scale)
+        assert oracle.rel_err(host64(dX2), dXr) <= TOL_BF16
+        assert oracle.rel_err(host64(dA2), dAr) <= TOL_F32 and oracle.rel_err(host64(dB2), dBr) <= TOL_F32
+        plan.close()
 
 
 # ---------------------------------------------------------------------------------------------
@@ -327,36 +338,17 @@ def test_split_k_paths_match_oracle(monkeypatch):
             assert torch.equal(a[k].view(it), b[k].view(it)), k
 
 
-def test_overlapped_backward_matches_the_stage_calls(monkeypatch):
-    """lora_linear_bwd with the dA / dB passes on the plan's second stream beside the dX GEMM (forced here on a mid-size
-    shape) against the oracle and against the serial stage calls: dX is bit-identical (same GEMM, fewer CTAs walk the
-    same tiles), dA / dB differ only by the grid-dependent order of fp32 partial sums; the overlapped call is itself
-    bitwise reproducible."""
-    monkeypatch.setenv("LORA_OVERLAP_SMS", "16")
-    p, t = inputs.draw_custom(4096, 2048, 2304, 16, 2.0, seed=12)
-    d = {k: dev(v) for k, v in t.items()}
-    plan = binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r)
-    cfg = plan.config()
-    assert cfg["overlap_sms"] == 16 and cfg["ov_dx_ctas"] == 132
-    outs = []
-    for _ in range(2):
-        outs.append(plan.bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], p.scale))
-    code, msg = plan.device_status()
-    assert code == 0, msg
-    for a, b in zip(outs[0], outs[1]):
-        assert torch.equal(a, b)
-    dX_s = torch.empty_like(outs[0][0])
-    dA_s = torch.empty_like(outs[0][1])
-    dB_s = torch.empty_like(outs[0][2])
-    plan.bwd_stages(d["dY"], d["X"], d["W"], d["A"], d["B"], p.scale, dX_s, dA_s, dB_s)
-    torch.cuda.synchronize()
-    assert torch.equal(outs[0][0], dX_s)
-    f = {k: inputs.bf16_to_f64(v) for k, v in t.items()}
-    dX, dA, dB = oracle.backward(f["dY"], f["X"], f["W"], f["A"], f["B"], p.scale)
-    assert oracle.rel_err(host64(outs[0][0]), dX) <= TOL_BF16
-    assert oracle.rel_err(host64(outs[0][1]), dA) <= TOL_F32 and oracle.rel_err(host64(outs[0][2]), dB) <= TOL_F32
-    assert oracle.rel_err(host64(outs[0][1]), host64(dA_s)) <= 1e-5 and oracle.rel_err(host64(outs[0][2]), host64(dB_s)) <= 1e-5
-    plan.close()
+@pytest.mark.parametrize("force", ["0", "1"])
+def test_both_forms_of_the_x_a_product_in_backward(force, monkeypatch):
+    """Backward recomputes X A^T either inside the dA launch (default up to rank 32) or in its own skinny pass over X
+    (default for larger ranks); both forms, forced here at r = 16 and r = 64, against the oracle."""
+    monkeypatch.setenv("LORA_FORCE_DA_WITH_P", force)
+    monkeypatch.setenv("LORA_FORCE_BWD_MERGED", "0")              # the split form: dY B | GEMM | dA | dB
+    for T, d_in, d_out, r, s in ((4096, 2048, 2304, 16, 2.0), (1500, 1032, 520, 64, 0.5)):
+        p, t = inputs.draw_custom(T, d_in, d_out, r, s, seed=12)
+        plan_cfg = binding.select_config(T, d_in, d_out, r, 148)
+        assert plan_cfg["da_with_p"] == int(force)
+        check_full(p, t)
 
 
 def test_staged_pre_pass_is_used_once_and_discarded_by_other_calls():

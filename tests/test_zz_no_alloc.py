@@ -39,16 +39,16 @@ def _second_factor(t, s, ld):
 
 CASES = [
     # T, d_in, d_out, r, scale, seed, ld - T
-    (1500, 520, 1032, 16, 2.0, 21, 4),      # several feature chunks and token chunks, partial sums in the static array
+    (1500, 520, 1032, 16, 2.0, 21, 4),      # several feature chunks, a cluster of token chunks each
     (900, 264, 392, 32, 0.5, 22, 4),
     (700, 136, 200, 8, 2.0, 23, 36),        # r = 8: rows 8..15 of the second-factor box lie outside Rt (zero fill); ld > T
-    (100, 72, 136, 24, 1.0, 24, 4),         # one slab: a single token chunk, the kernel writes `out` itself
+    (100, 72, 136, 24, 1.0, 24, 4),         # one slab: a single token chunk, no cluster
 ]
 
 
 def test_noalloc_contraction_matches_definition_and_planned_backward_twice():
     lib = binding.load()
-    assert lib.lora_grad_contract_noalloc_max_scratch() == 8 << 20
+    assert lib.lora_grad_contract_noalloc_max_scratch() == 4096
     for T, d_in, d_out, r, s, seed, extra in CASES:
         p, t = inputs.draw_custom(T, d_in, d_out, r, s, seed=seed)
         d = {k: _dev(v) for k, v in t.items()}
@@ -77,9 +77,9 @@ def test_noalloc_contraction_matches_definition_and_planned_backward_twice():
         plan.close()
 
 
-def test_noalloc_contraction_wide_rank64_runs_with_fewer_token_chunks():
-    """16384 x 4096 with r = 64: the full grid's partial sums (24 token chunks x 1 MiB) exceed the 8 MiB array, so the
-    call runs with the 7 token chunks that fit instead of refusing.  Checked against the float64 definition."""
+def test_noalloc_contraction_at_a_benchmark_size():
+    """16384 x 4096 with r = 64 (the down-projection's dB shape): clusters of 16 token chunks, four accumulator blocks per
+    CTA.  Checked against the float64 definition, twice."""
     T, C, r = 16384, 4096, 64
     g = np.random.Generator(np.random.Philox(key=77))
     s_bits = inputs.f32_to_bf16_bits(g.standard_normal((T, C), dtype=np.float32))
@@ -93,17 +93,17 @@ def test_noalloc_contraction_wide_rank64_runs_with_fewer_token_chunks():
         assert _rel(out.double(), expected) <= TOL_F32, (call, _rel(out.double(), expected))
 
 
-def test_noalloc_contraction_rejects_what_does_not_fit():
+def test_noalloc_contraction_rejects_sizes_beyond_its_limits():
     lib = binding.load()
     stream = torch.cuda.current_stream().cuda_stream
     # real, fully sized tensors: nothing can be touched out of bounds whatever the call decides
-    T, C, r = 128, 40000, 64
+    T, C, r = 8, (1 << 24) + 8, 8
     S = torch.zeros((T, C), dtype=torch.bfloat16, device="cuda")
     Rt = torch.zeros((r, T), dtype=torch.bfloat16, device="cuda")
     o = torch.zeros((C, r), dtype=torch.float32, device="cuda")
-    # one layer of partial sums, 64 x 40000 floats = 9.8 MiB, is more than the 8 MiB static array holds
+    # more than 2^24 features: beyond what the entry point serves
     rc = lib.lora_grad_contract_noalloc(S.data_ptr(), Rt.data_ptr(), T, C, r, T, o.data_ptr(), stream)
-    assert rc == binding.LORA_ERR_WORKSPACE
+    assert rc == binding.LORA_ERR_UNSUPPORTED_SHAPE
     rc = lib.lora_grad_contract_noalloc(S.data_ptr(), Rt.data_ptr(), 128, 60, 16, 128, o.data_ptr(), stream)
     assert rc == binding.LORA_ERR_UNSUPPORTED_SHAPE
     rc = lib.lora_grad_contract_noalloc(None, Rt.data_ptr(), 128, 64, 16, 128, o.data_ptr(), stream)
