@@ -585,55 +585,56 @@ def run_ours(args):
     #      copies its inputs from pinned host memory, runs forward + backward and copies Y, dX, dA, dB back.  Two lanes
     #      (plan + staging + host output buffers + stream each) alternate, so that the copy-in of one step overlaps the
     #      copy-out of the previous one on the two DMA directions; each step's own chain stays in order on its stream ----
-    n_lanes = 1 if args.workload >= 4 else 2
-    sets0 = wl.sets[0]
-    h_in = [{k: d0[k].cpu().pin_memory() for k in ("X", "A", "B", "dY")} for _, d0 in sets0]
-    lanes = []
-    for ln in range(n_lanes):
-        lp = plans if ln == 0 else [binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r, device=local_rank) for p in protos]
-        for pl in lp:
-            pl.ensure_workspace()
-        outs = [{k: torch.empty_like(d0[k], device="cpu").pin_memory() for k in ("Y", "dX", "dA", "dB")} for _, d0 in sets0]
-        stg = [torch.empty(lp[j].step_host_staging_bytes(), dtype=torch.uint8, device=device) for j in range(len(protos))]
-        lanes.append({"plans": lp, "out": outs, "staging": stg, "stream": torch.cuda.Stream(device=device)})
+    e2e = None
+    if not args.quick:
+        n_lanes = 1 if args.workload >= 4 else 2
+        sets0 = wl.sets[0]
+        h_in = [{k: d0[k].cpu().pin_memory() for k in ("X", "A", "B", "dY")} for _, d0 in sets0]
+        lanes = []
+        for ln in range(n_lanes):
+            lp = plans if ln == 0 else [binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r, device=local_rank) for p in protos]
+            for pl in lp:
+                pl.ensure_workspace()
+            outs = [{k: torch.empty_like(d0[k], device="cpu").pin_memory() for k in ("Y", "dX", "dA", "dB")} for _, d0 in sets0]
+            stg = [torch.empty(lp[j].step_host_staging_bytes(), dtype=torch.uint8, device=device) for j in range(len(protos))]
+            lanes.append({"plans": lp, "out": outs, "staging": stg, "stream": torch.cuda.Stream(device=device)})
 
-    def step_host(k):
-        ln = lanes[k % n_lanes]
-        for j, (p, d0) in enumerate(sets0):
-            h, ho = h_in[j], ln["out"][j]
-            ln["plans"][j].step_host(h["X"], d0["W"], h["A"], h["B"], h["dY"], p.scale, ho["Y"], ho["dX"], ho["dA"], ho["dB"],
-                                     ln["staging"][j], stream=ln["stream"])
+        def step_host(k):
+            ln = lanes[k % n_lanes]
+            for j, (p, d0) in enumerate(sets0):
+                h, ho = h_in[j], ln["out"][j]
+                ln["plans"][j].step_host(h["X"], d0["W"], h["A"], h["B"], h["dY"], p.scale, ho["Y"], ho["dX"], ho["dA"], ho["dB"],
+                                         ln["staging"][j], stream=ln["stream"])
 
-    def run_host(n):
-        cur = torch.cuda.current_stream()
-        start, done = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        start.record(cur)
-        for ln in lanes:
-            ln["stream"].wait_event(start)
-        for k in range(n):
-            step_host(k)
-        for ln in lanes:
-            ev = torch.cuda.Event()
-            ev.record(ln["stream"])
-            cur.wait_event(ev)
-        done.record(cur)
-        torch.cuda.synchronize()
-        return start.elapsed_time(done)
+        def run_host(n):
+            cur = torch.cuda.current_stream()
+            start, done = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            start.record(cur)
+            for ln in lanes:
+                ln["stream"].wait_event(start)
+            for k in range(n):
+                step_host(k)
+            for ln in lanes:
+                ev = torch.cuda.Event()
+                ev.record(ln["stream"])
+                cur.wait_event(ev)
+            done.record(cur)
+            torch.cuda.synchronize()
+            return start.elapsed_time(done)
 
-    n_e2e = max(3, min(args.steps, 20 if args.workload < 4 else 3))
-    run_host(2 * n_lanes if args.workload < 4 else 1)
-    barrier()
-    ms_e2e = max_over_ranks(run_host(n_e2e) / n_e2e, device, world)
-    barrier()
-    h2d = sum(t.numel() * t.element_size() for h in h_in for t in h.values())
-    d2h = sum(t.numel() * t.element_size() for ho in lanes[0]["out"] for t in ho.values())
-    e2e = {"value": job_value(world, flops_step, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-           "ms_per_step": ms_e2e, "steps": n_e2e, "lanes": n_lanes,
-           "pcie_gbs": {"h2d": h2d / ms_e2e / 1e6, "d2h": d2h / ms_e2e / 1e6},
-           "note": "host X, A, B, dY in; Y, dX, dA, dB out (pinned); frozen W resident on the device; "
-                   f"{n_lanes} lane(s) of lora_linear_step_host alternate so that copies of neighbouring steps overlap"}
+        n_e2e = max(3, min(args.steps, 20 if args.workload < 4 else 3))
+        run_host(2 * n_lanes if args.workload < 4 else 1)
+        barrier()
+        ms_e2e = max_over_ranks(run_host(n_e2e) / n_e2e, device, world)
+        barrier()
+        h2d = sum(t.numel() * t.element_size() for h in h_in for t in h.values())
+        d2h = sum(t.numel() * t.element_size() for ho in lanes[0]["out"] for t in ho.values())
+        e2e = {"value": job_value(world, flops_step, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "ms_per_step": ms_e2e, "steps": n_e2e, "lanes": n_lanes,
+               "pcie_gbs": {"h2d": h2d / ms_e2e / 1e6, "d2h": d2h / ms_e2e / 1e6},
+               "note": "host X, A, B, dY in; Y, dX, dA, dB out (pinned); frozen W resident on the device; "
+                       f"{n_lanes} lane(s) of lora_linear_step_host alternate so that copies of neighbouring steps overlap"}
     plan_desc = plans[0].describe()
-    del lanes, h_in
     wl.close()
 
     # ---- the other workloads, from short runs in the same process (rank 0's figures; every rank runs them) ----
@@ -698,8 +699,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--quick", action="store_true",
-                    help="only the timed region, the instrumented pass and the end-to-end leg of the chosen workload "
-                         "(no sustained leg, variants or other workloads); for profiler captures")
+                    help="only the timed region and the instrumented pass of the chosen workload (no sustained leg, variants, "
+                         "end-to-end leg or other workloads); for profiler captures")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -118,7 +118,9 @@ int lora_select_config(const lora_shape_t* shape, int num_sms, lora_kernel_confi
 int lora_workspace_bytes(const lora_shape_t* shape, int num_sms, size_t* bwd_bytes);
 
 /* Create / destroy a plan for one shape on CUDA device `device` (runs the selector, allocates the
- * 256-byte device status block).  The plan is host memory owned by the library. */
+ * 256-byte device status block).  The plan is host memory owned by the library.
+ * With the environment variable LORA_LOG=1 every new plan prints one line to stderr with what the selector chose
+ * (the text lora_plan_describe returns). */
 int lora_plan_create(const lora_shape_t* shape, int device, lora_plan_t** out);
 int lora_plan_destroy(lora_plan_t* plan);
 
@@ -196,6 +198,41 @@ int lora_linear_bwd_dx(lora_plan_t* plan, const void* dY, const void* W, const v
 int lora_linear_bwd_da(lora_plan_t* plan, const void* X, const void* A, float scale, void* dA, void* stream);
 int lora_linear_bwd_db(lora_plan_t* plan, const void* dY, float scale, void* dB, void* stream);
 
+/* Grouped projections: G = 2..4 projections that consume the SAME activations X (the attention q/k/v projections, the MLP
+ * gate/up projections; Section 4.5 adapts q, k, v, o with lora_r = 32) as one layer call.  Group g has its own frozen
+ * W_g [d_g, d_in] and its own adapter A_g [r, d_in], B_g [d_g, r]; all groups share T, d_in, r and scale:
+ *
+ *     Y_g = X W_g^T + scale (X A_g^T) B_g^T        dX = sum_g ( dY_g W_g + scale (dY_g B_g) A_g )
+ *     dA_g = scale (dY_g B_g)^T X                  dB_g = scale dY_g^T (X A_g^T)
+ *
+ * i.e. exactly what G separate lora_linear_fwd / lora_linear_bwd calls compute, with the G partial dX added up.
+ * Operands are the groups' tensors stacked along their row (W, A, B) or column (Y, dY) index, in group order:
+ *     W_cat [sum d_g, d_in]   A_cat [G r, d_in]   B_cat [sum d_g, r]   Y_cat, dY_cat [T, sum d_g]     bf16
+ *     dX [T, d_in] bf16       dA_cat [G r, d_in]  dB_cat [sum d_g, r]                                  fp32
+ * (group g's Y is the column range [off_g, off_g + d_g) of Y_cat, a strided view).  What grouping buys: X is streamed once
+ * per stage for all groups; the forward is ONE GEMM over sum d_g output columns (narrow projections such as the 1024-wide
+ * k/v no longer leave CTA pairs idle) whose rank-r k-block picks, per output tile, the rows of scale (X A^T)^T and of B
+ * that belong to the tile's group; dX is ONE GEMM over the contraction sum d_g plus one rank-r k-block per group; all dY_g B_g
+ * and X A_cat^T run in one skinny launch, all dA_g and dB_g in another.  No block of zeros is multiplied and nothing is
+ * computed only to be dropped.
+ * Limits (LORA_ERR_UNSUPPORTED_SHAPE otherwise; run the projections through their own plans then): T > 128;
+ * r in {16, 32, 48, 64}; every d_g a multiple of 256; G + ceil(G r / 64) <= 6.
+ * A grouped plan is created by lora_plan_create_grouped and used with the two *_grouped calls only (the plain calls return
+ * LORA_ERR_INVALID_ARG on it and vice versa); workspace, wait limit, gradient accumulation, status and destruction go through
+ * the same lora_plan_* calls.  Both calls need the workspace (lora_plan_workspace_bytes). */
+typedef struct lora_group_shape {
+  int64_t T;        /* tokens                                 */
+  int64_t d_in;     /* input features, shared                 */
+  int64_t r;        /* adapter rank of every group            */
+  int32_t n_groups; /* 2 .. 4                                 */
+  int64_t d_out[4]; /* output features of each group          */
+} lora_group_shape_t;
+int lora_plan_create_grouped(const lora_group_shape_t* shape, int device, lora_plan_t** out);
+int lora_linear_fwd_grouped(lora_plan_t* plan, const void* X, const void* W_cat, const void* A_cat, const void* B_cat,
+                            float scale, void* Y_cat, void* stream);
+int lora_linear_bwd_grouped(lora_plan_t* plan, const void* dY_cat, const void* X, const void* W_cat, const void* A_cat,
+                            const void* B_cat, float scale, void* dX, void* dA_cat, void* dB_cat, void* stream);
+
 /* Dense weight gradient of full fine-tuning (Section 4.5, "Full-model tuning": every weight is updated, so the frozen-W
  * shortcut of LoRA no longer applies and the layer also owes  dW = dY^T X):
  *     dW[o, i] = sum_t dY[t, o] X[t, i]        dY [T, d_out] bf16, X [T, d_in] bf16  ->  dW [d_out, d_in] bf16
@@ -270,19 +307,17 @@ int lora_debug_starved_wait(lora_plan_t* plan, const void* S, int64_t T, int64_t
  * they call in: code running under a memory pool that forbids cudaMalloc after start-up, real-time or
  * inference loops where an allocation would stall the device, and hosts that hand this library a fixed
  * memory budget.  No plan is needed (creating one allocates a status block).  Nothing in this call
- * allocates or frees: the partial sums and status word live in one static device array
- * of lora_grad_contract_noalloc_max_scratch() bytes (8 MiB) that every GPU loading the library holds until
- * the process exits.
- *   - C % 8 == 0, r in {8,...,64}, ld_rt % 8 == 0, T >= 1.  The grid takes as many token chunks as the array has room
- *     for their partial sums (r_pad x C_pad floats each, r_pad = r rounded up to 16, C_pad = C rounded up to 32), down to
- *     a single chunk, which needs none: wide matrices run with fewer CTAs, they are not refused.  Only a shape whose
- *     single layer of partial sums exceeds the array (r_pad x C_pad x 4 bytes > 8 MiB - 4 KiB, i.e. C beyond 32736 at
- *     r = 64 or 131040 at r = 16) is rejected with LORA_ERR_WORKSPACE.
- *   - The first call on a device looks up the array's device address and raises the kernel's shared-memory
- *     limit; make that first call before any stream capture.  The current device is used.
- *   - All calls share the one array and it keeps the last call's contents; the call clears the status
- *     words on `stream` first and rewrites every partial sum before reading it.  Two calls whose kernels overlap on the GPU (different streams, or
- *     different host threads) race on it: serialise them.
+ * allocates or frees: the only global scratch the kernel needs - its status block, where a device-side wait that ran out
+ * is recorded - lives in one static device array of lora_grad_contract_noalloc_max_scratch() bytes (4 KiB) that every
+ * GPU loading the library holds until the process exits.  (The sums over token chunks meet on chip, in the distributed
+ * shared memory of a thread-block cluster, so there are no partial sums in global memory to make room for.)
+ *   - Limits: C % 8 == 0, r in {8,...,64}, ld_rt % 8 == 0, 1 <= T <= 2^30, C <= 2^24; anything beyond is rejected with
+ *     LORA_ERR_UNSUPPORTED_SHAPE (LORA_ERR_INVALID_ARG for null pointers or ld_rt < T) before anything is launched.
+ *   - The first call on a device looks up the array's device address, raises the kernel's shared-memory
+ *     limit and asks how many clusters fit the device; make that first call before any stream capture.  The current
+ *     device is used.
+ *   - All calls share the one array and it keeps the last call's contents; the call clears it on `stream` first.
+ *     Two calls whose kernels overlap on the GPU (different streams, or different host threads) race on it: serialise them.
  *   - A bounded device wait that ran out leaves `out` incomplete while the call itself has long returned LORA_OK:
  *     lora_grad_contract_noalloc_status synchronises `stream`, reads the status word of the current device's array
  *     (a 4-byte copy, no allocation) and sets *code to LORA_OK or LORA_ERR_DEVICE_TIMEOUT. */

@@ -31,7 +31,7 @@ EXPORTS = [
     "lora_last_device_status", "lora_strerror", "lora_launch_count",
     "lora_grad_contract_noalloc", "lora_grad_contract_noalloc_max_scratch", "lora_grad_contract_noalloc_status",
     "lora_plan_set_wait_limit", "lora_debug_starved_wait", "lora_linear_bwd_sides", "lora_linear_bwd_grads",
-    "lora_plan_last_gemm_clock",
+    "lora_plan_last_gemm_clock", "lora_plan_create_grouped", "lora_linear_fwd_grouped", "lora_linear_bwd_grouped",
 ]
 
 
@@ -101,6 +101,9 @@ def load(rebuild: bool = False) -> ctypes.CDLL:
     lib.lora_launch_count.restype = i64
     lib.lora_grad_contract_noalloc.argtypes = [vp, vp, i64, i64, i64, i64, vp, vp]
     lib.lora_grad_contract_noalloc_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
+    lib.lora_plan_create_grouped.argtypes = [vp, ctypes.c_int, ctypes.POINTER(vp)]
+    lib.lora_linear_fwd_grouped.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp]
+    lib.lora_linear_bwd_grouped.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp]
     lib.lora_plan_set_wait_limit.argtypes = [vp, i64]
     lib.lora_plan_last_gemm_clock.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
     lib.lora_debug_starved_wait.argtypes = [vp, vp, i64, i64, vp, vp]

@@ -49,24 +49,21 @@ __device__ __forceinline__ float4 ld_cluster_f4(uint32_t cluster_addr) {
   return v;
 }
 
-// One launch runs one or two JOBS side by side (e.g. dA over X next to dB over dY, or X A^T next to dY B): CTAs with
-// blockIdx.x < split_x belong to job 0, the others to job 1.  A job's CTAs are numbered (feature chunk, token chunk):
-// with a gradient the token chunk is blockIdx.y (= rank in the cluster), otherwise both indices are folded into x.
+// One launch runs up to kGradMaxJobs JOBS side by side (e.g. dA over X next to dB over dY, or X A^T next to dY B; the
+// grouped projections add one job per group): CTAs with blockIdx.x in [x_end[j-1], x_end[j]) belong to job j.  A job's
+// CTAs are numbered (feature chunk, token chunk): with a gradient the token chunk is blockIdx.y (= rank in the cluster),
+// otherwise both indices are folded into x.  maps.m[3 j + 0 .. 2] = job j's streamed matrix [T, C] box 64(c) x 128(t),
+// second factor [r_pad, T] box 64(t) x r_pad, side operand (with_p): A [r, C] box 64(c) x r_pad, or B [C, r] box
+// 64(r, zero-filled) x 64(c) when side_mn.
 __global__ void __launch_bounds__(kGradThreads, 1)
-lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s0,  // job 0: streamed matrix [T, C], box 64(c) x 128(t)
-                 const __grid_constant__ CUtensorMap tm_r0,  //        second factor [r_pad, T], box 64(t) x r_pad
-                 const __grid_constant__ CUtensorMap tm_a0,  //        side operand (with_p): A [r, C] box 64(c) x r_pad, or
-                                                             //        B [C, r] box 64(r, zero-filled) x 64(c) when side_mn
-                 const __grid_constant__ CUtensorMap tm_s1,  // job 1, same roles
-                 const __grid_constant__ CUtensorMap tm_r1,
-                 const __grid_constant__ CUtensorMap tm_a1,
-                 const GradLaunch L) {
+lora_grad_kernel(const __grid_constant__ GradMaps maps, const __grid_constant__ GradLaunch L) {
   pdl_launch_dependents();
-  const bool job1 = static_cast<int>(blockIdx.x) >= L.split_x;
-  const GradParams p = job1 ? L.job[1] : L.job[0];
-  const CUtensorMap& tm_s = job1 ? tm_s1 : tm_s0;
-  const CUtensorMap& tm_r = job1 ? tm_r1 : tm_r0;
-  const CUtensorMap& tm_a = job1 ? tm_a1 : tm_a0;
+  int job = 0;
+  while (job + 1 < L.n_jobs && static_cast<int>(blockIdx.x) >= L.x_end[job]) ++job;
+  const GradParams p = L.job[job];
+  const CUtensorMap& tm_s = maps.m[3 * job];
+  const CUtensorMap& tm_r = maps.m[3 * job + 1];
+  const CUtensorMap& tm_a = maps.m[3 * job + 2];
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int NB = p.feat_chunk >> 7;                 // 128-feature accumulator blocks of a full chunk
@@ -93,7 +90,7 @@ lora_grad_kernel(const __grid_constant__ CUtensorMap tm_s0,  // job 0: streamed 
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int local_x = static_cast<int>(blockIdx.x) - (job1 ? L.split_x : 0);
+  const int local_x = static_cast<int>(blockIdx.x) - (job > 0 ? L.x_end[job - 1] : 0);
   const int fc = p.do_out ? local_x : local_x % p.n_feat_chunks;
   const int tc = p.do_out ? static_cast<int>(blockIdx.y) : local_x / p.n_feat_chunks;
   const int c0 = fc * p.feat_chunk;
@@ -434,11 +431,25 @@ int grad_max_resident_ctas(int cluster, size_t smem_bytes) {
 }
 
 GradGrid grad_pick_grid(long long T, long long C, long long C2, int r_pad, bool with_p, bool side_mn, const int* caps) {
-  const int nblk1 = static_cast<int>((C + 127) / 128), nblk2 = static_cast<int>((C2 + 127) / 128);
+  const long long cs[2] = {C, C2};
+  return grad_pick_grid_jobs(T, cs, C2 > 0 ? 2 : 1, r_pad, with_p, side_mn, caps);
+}
+
+GradGrid grad_pick_grid_jobs(long long T, const long long* C, int n_jobs, int r_pad, bool with_p, bool side_mn, const int* caps) {
+  int nblk_sum = 0, nblk_max = 0;
+  for (int j = 0; j < n_jobs; ++j) {
+    const int b = static_cast<int>((C[j] + 127) / 128);
+    nblk_sum += b;
+    if (b > nblk_max) nblk_max = b;
+  }
+  auto chunks = [&](int nb) {
+    int n = 0;
+    for (int j = 0; j < n_jobs; ++j) n += (static_cast<int>((C[j] + 127) / 128) + nb - 1) / nb;
+    return n;
+  };
   const int n_slabs = static_cast<int>((T + kGradSlab - 1) / kGradSlab);
   int nb_max = (512 - (with_p ? kGradPBufs * r_pad : 0)) / r_pad;          // TMEM: NB x r_pad + side buffers <= 512 columns
   if (nb_max < 1) nb_max = 1;
-  const int nblk_max = nblk1 > nblk2 ? nblk1 : nblk2;
   if (nb_max > nblk_max) nb_max = nblk_max;
   GradGrid best{};
   double best_t = 1e300;
@@ -446,13 +457,13 @@ GradGrid grad_pick_grid(long long T, long long C, long long C2, int r_pad, bool 
     if (cs > n_slabs || caps[cs] < cs) continue;
     const int slabs_per = (n_slabs + cs - 1) / cs;
     for (int nb = 1; nb <= nb_max; ++nb) {
-      const int n_feat = (nblk1 + nb - 1) / nb + (nblk2 + nb - 1) / nb;
+      const int n_feat = chunks(nb);
       if (n_feat * cs > caps[cs]) continue;
       // time in tile units (one 128 x 128 tile of the stream): the busiest CTA's tiles, but never less than the stream
       // needs when every SM pulls its share of the HBM bandwidth (about 120 busy SMs saturate it); side-product partial
       // sums add r_pad / (32 nb) of a tile's bytes per tile (written and read back); a cluster reduction ~1.5 tiles
       double t = static_cast<double>(nb) * slabs_per;
-      const double sat = static_cast<double>(nblk1 + nblk2) * n_slabs / 120.0;
+      const double sat = static_cast<double>(nblk_sum) * n_slabs / 120.0;
       if (t < sat) t = sat;
       if (with_p && n_feat > 1) t *= 1.0 + r_pad / (32.0 * nb);
       if (cs > 1) t += 1.5;
@@ -467,7 +478,7 @@ GradGrid grad_pick_grid(long long T, long long C, long long C2, int r_pad, bool 
   if (best.feat_chunk == 0) {
     // more feature chunks than CTAs are resident at once even at the widest chunk: widest chunk, no cluster, several waves
     best.feat_chunk = nb_max * 128;
-    best.n_feat = (nblk1 + nb_max - 1) / nb_max + (nblk2 + nb_max - 1) / nb_max;
+    best.n_feat = chunks(nb_max);
     best.n_tok = 1;
   }
   const size_t side_box = side_mn ? size_t(8192) : static_cast<size_t>(r_pad) * 128;
@@ -513,22 +524,34 @@ void grad_device_caps(int num_sms, int* caps) {
   for (int cs = 2; cs <= kGradMaxCluster; ++cs) caps[cs] = grad_max_resident_ctas(cs, 232448);
 }
 
-cudaError_t launch_grad2(const CUtensorMap* const tm0[3], const GradParams& p0, const CUtensorMap* const tm1[3],
-                         const GradParams* p1, cudaStream_t stream) {
+cudaError_t launch_grad_jobs(const GradJobDesc* jobs, int n_jobs, cudaStream_t stream) {
+  if (n_jobs < 1 || n_jobs > kGradMaxJobs) return cudaErrorInvalidValue;
+  GradMaps maps;
   GradLaunch L{};
-  L.job[0] = p0;
-  L.job[1] = p1 != nullptr ? *p1 : p0;
-  // x extent of a job: feature chunks (gradient: the token chunks are the cluster along y) or feature x token chunks
-  const int x0 = p0.do_out ? p0.n_feat_chunks : p0.n_feat_chunks * p0.n_token_chunks;
-  const int x1 = p1 == nullptr ? 0 : (p1->do_out ? p1->n_feat_chunks : p1->n_feat_chunks * p1->n_token_chunks);
-  L.split_x = x0;
-  const int cluster = p0.do_out ? p0.n_token_chunks : 1;
-  if (p1 != nullptr && (p1->do_out != p0.do_out || (p0.do_out && p1->n_token_chunks != p0.n_token_chunks)))
-    return cudaErrorInvalidValue;          // both jobs of a launch share the cluster shape
-  size_t smem = grad_smem_bytes(p0);
-  if (p1 != nullptr && grad_smem_bytes(*p1) > smem) smem = grad_smem_bytes(*p1);
+  L.n_jobs = n_jobs;
+  const int do_out = jobs[0].p.do_out;
+  const int cluster = do_out ? jobs[0].p.n_token_chunks : 1;
+  size_t smem = 0;
+  int x = 0;
+  for (int j = 0; j < n_jobs; ++j) {
+    const GradParams& p = jobs[j].p;
+    // all jobs of a launch share the cluster shape: all compute a gradient with the same number of token chunks, or none does
+    if (p.do_out != do_out || (do_out && p.n_token_chunks != cluster)) return cudaErrorInvalidValue;
+    L.job[j] = p;
+    maps.m[3 * j] = jobs[j].tmS;
+    maps.m[3 * j + 1] = jobs[j].tmR;
+    maps.m[3 * j + 2] = jobs[j].tmSide;
+    // x extent of a job: feature chunks (gradient: the token chunks are the cluster along y) or feature x token chunks
+    x += do_out ? p.n_feat_chunks : p.n_feat_chunks * p.n_token_chunks;
+    L.x_end[j] = x;
+    if (grad_smem_bytes(p) > smem) smem = grad_smem_bytes(p);
+  }
+  for (int j = n_jobs; j < kGradMaxJobs; ++j) {
+    L.x_end[j] = x;
+    maps.m[3 * j] = maps.m[3 * j + 1] = maps.m[3 * j + 2] = jobs[0].tmS;
+  }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(static_cast<unsigned>(x0 + x1), static_cast<unsigned>(cluster), 1);
+  cfg.gridDim = dim3(static_cast<unsigned>(x), static_cast<unsigned>(cluster), 1);
   cfg.blockDim = dim3(kGradThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
@@ -545,14 +568,17 @@ cudaError_t launch_grad2(const CUtensorMap* const tm0[3], const GradParams& p0, 
     cfg.numAttrs = 2;
   }
   cfg.attrs = attr;
-  const CUtensorMap* const* t1 = p1 != nullptr ? tm1 : tm0;
-  return cudaLaunchKernelEx(&cfg, lora_grad_kernel, *tm0[0], *tm0[1], *tm0[2], *t1[0], *t1[1], *t1[2], L);
+  return cudaLaunchKernelEx(&cfg, lora_grad_kernel, maps, L);
 }
 
 cudaError_t launch_grad(const CUtensorMap& tmS, const CUtensorMap& tmR, const CUtensorMap& tmA, const GradParams& p,
                         cudaStream_t stream) {
-  const CUtensorMap* const tm[3] = {&tmS, &tmR, &tmA};
-  return launch_grad2(tm, p, nullptr, nullptr, stream);
+  GradJobDesc j;
+  j.tmS = tmS;
+  j.tmR = tmR;
+  j.tmSide = tmA;
+  j.p = p;
+  return launch_grad_jobs(&j, 1, stream);
 }
 
 // ================================================================================================

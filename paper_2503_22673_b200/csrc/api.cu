@@ -454,6 +454,13 @@ struct lora_plan {
   bool p_saved;          // the workspace holds Pt = s (X A^T)^T of the last forward call
   float p_saved_scale;
   long long wait_limit;  // SM clock ticks after which a device-side spin gives up (lora_plan_set_wait_limit)
+  // grouped projections (lora_plan_create_grouped): G projections that share X; shape.d_out is the sum of their widths
+  int n_groups;          // 0: an ordinary plan
+  long long group_off[5];   // first output column of every group, and the total
+  struct GroupedWs {
+    size_t qt, pt, part, count, total;    // Qt_all / Pt_all [G r, ld_t] bf16, partial-sum regions, counters
+    size_t part_stride;                   // bytes of one job's partial-sum region
+  } gws;
 };
 
 namespace {
@@ -577,9 +584,14 @@ int launch_side_pair(lora_plan* pl, const void* dY, const void* B, const void* X
       !fill_side_job(pl, X, s.d_in, A, false, scale, q.pt, pl->num_sms - g0, 1, &jp))
     return LORA_ERR_CUDA;
   if ((jq.g.n_feat_chunks > 1 || jp.g.n_feat_chunks > 1) && !ensure_counters(pl, st)) return LORA_ERR_CUDA;
-  const CUtensorMap* const t0[3] = {&jq.tmS, &jq.tmS, &jq.tmSide};
-  const CUtensorMap* const t1[3] = {&jp.tmS, &jp.tmS, &jp.tmSide};
-  if (launch_grad2(t0, jq.g, t1, &jp.g, st) != cudaSuccess) return LORA_ERR_CUDA;
+  GradJobDesc jobs[2];
+  jobs[0].tmS = jobs[0].tmR = jq.tmS;
+  jobs[0].tmSide = jq.tmSide;
+  jobs[0].p = jq.g;
+  jobs[1].tmS = jobs[1].tmR = jp.tmS;
+  jobs[1].tmSide = jp.tmSide;
+  jobs[1].p = jp.g;
+  if (launch_grad_jobs(jobs, 2, st) != cudaSuccess) return LORA_ERR_CUDA;
   g_launches.fetch_add(1);
   return LORA_OK;
 }
@@ -633,6 +645,7 @@ int launch_fwd(lora_plan* pl, const void* X, const void* W, const void* A, const
   p.ld_rt = pl->ws.ld_t;
   p.status = pl->d_status;
     p.wait_limit = pl->wait_limit;
+    p.tail_parts = 1;
   const cudaError_t le = ext    ? launch_gemm_pair_fwd_ext(tmX, tmW, tmA, tmB, tmY, p, c.fwd_ctas, st)
                          : pair ? launch_gemm_pair_fwd(tmX, tmW, tmW1, tmA, tmB, tmY, p, c.fwd_ctas, st)
                                 : launch_gemm_fwd(tmX, tmW, tmA, tmB, tmY, p, c.fwd_ctas, st);
@@ -697,6 +710,7 @@ int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const
     p.ld_rt = w.ld_t;
     p.status = pl->d_status;
     p.wait_limit = pl->wait_limit;
+    p.tail_parts = 1;
     const int ctas = ctas_override > 0 ? ctas_override : c.dx_ctas;
     const cudaError_t le = pair ? launch_gemm_pair_dx(tmdY, tmW, tmB, tmA, tmdX, p, ctas, st)
                                 : launch_gemm_dx(tmdY, tmW, tmB, tmA, tmdX, p, ctas, st);
@@ -836,9 +850,16 @@ int launch_grad_pair(lora_plan* pl, const void* X, const void* dY, const void* A
   if (!fill_da_job(pl, X, A, scale, dA, false, c.pair_feat_chunk, c.pair_token_chunks, &ja) ||
       !fill_db_job(pl, dY, scale, dB, nullptr, c.pair_feat_chunk, c.pair_token_chunks, &jb))
     return LORA_ERR_CUDA;
-  const CUtensorMap* const t0[3] = {&ja.tmS, &ja.tmR, &ja.tmSide};
-  const CUtensorMap* const t1[3] = {&jb.tmS, &jb.tmR, &jb.tmSide};
-  if (launch_grad2(t0, ja.g, t1, &jb.g, st) != cudaSuccess) return LORA_ERR_CUDA;
+  GradJobDesc jobs[2];
+  jobs[0].tmS = ja.tmS;
+  jobs[0].tmR = ja.tmR;
+  jobs[0].tmSide = ja.tmSide;
+  jobs[0].p = ja.g;
+  jobs[1].tmS = jb.tmS;
+  jobs[1].tmR = jb.tmR;
+  jobs[1].tmSide = jb.tmSide;
+  jobs[1].p = jb.g;
+  if (launch_grad_jobs(jobs, 2, st) != cudaSuccess) return LORA_ERR_CUDA;
   g_launches.fetch_add(1);
   return LORA_OK;
 }
@@ -916,6 +937,7 @@ int launch_fwd_nf4(lora_plan* pl, const void* X, const void* codes, const void* 
   p.split_k = 1;
   p.status = pl->d_status;
     p.wait_limit = pl->wait_limit;
+    p.tail_parts = 1;
   const int ctas = 2 * (p.num_tiles < pairs ? p.num_tiles : pairs);
   if (launch_gemm_pair_fwd_nf4(tmX, tmCodes, tmAbsmax, tmPt, tmB, tmY, p, ctas, st) != cudaSuccess) return LORA_ERR_CUDA;
   g_launches.fetch_add(1);
@@ -961,6 +983,7 @@ int launch_dx_nf4(lora_plan* pl, const void* dY, const void* codes, const void* 
   p.split_k = 1;
   p.status = pl->d_status;
     p.wait_limit = pl->wait_limit;
+    p.tail_parts = 1;
   const int ctas = 2 * (p.num_tiles < pairs ? p.num_tiles : pairs);
   if (launch_gemm_pair_dx_nf4(tmdY, tmCodes, tmAbsmax, tmQt, tmA, tmdX, p, ctas, st) != cudaSuccess) return LORA_ERR_CUDA;
   g_launches.fetch_add(1);
@@ -1004,6 +1027,7 @@ int launch_dw(lora_plan* pl, const void* dY, const void* X, void* dW, cudaStream
   p.part = (p.split_k > 1) ? reinterpret_cast<float*>(static_cast<uint8_t*>(pl->workspace) + pl->ws.split_part) : nullptr;
   p.status = pl->d_status;
     p.wait_limit = pl->wait_limit;
+    p.tail_parts = 1;
   if (launch_gemm_pair_dw(tmdY, tmX, tmdW, p, c.dw_ctas, st) != cudaSuccess) return LORA_ERR_CUDA;
   g_launches.fetch_add(1);
   if (p.split_k > 1) {
@@ -1015,9 +1039,334 @@ int launch_dw(lora_plan* pl, const void* dY, const void* X, void* dW, cudaStream
   return LORA_OK;
 }
 
+// ------------------------------------------------------------------------------------------------
+// grouped projections: several projections that consume the same X (q/k/v, gate/up) as ONE forward GEMM over the
+// concatenated output columns, ONE dX GEMM over the concatenated contraction, and two skinny launches
+// ------------------------------------------------------------------------------------------------
+constexpr int kGroupRowsPerJob = 64;       // rank rows one streaming job handles (its r_pad)
+
+// generic side-product job: out_t[rows, T] = scale (S side^T)^T for `rows` adapter rows
+bool build_side_job(lora_plan* pl, const void* S, long long C, long long pitch, const void* side, bool side_mn, long long side_pitch,
+                    int rows, float scale, __nv_bfloat16* out_t, float* part, int* count, int ctas, GradJobDesc* job) {
+  const long long T = pl->shape.T;
+  bool ok = make_bf16_tmap(&job->tmS, S, C, T, pitch, 64, kGradSlab);
+  if (side_mn) ok = ok && make_bf16_tmap(&job->tmSide, side, rows, C, side_pitch, 64, 64);
+  else ok = ok && make_bf16_tmap(&job->tmSide, side, C, rows, side_pitch, 64, rows);
+  if (!ok) return false;
+  job->tmR = job->tmS;
+  const SideGrid sg = pick_side_grid(T, C, ctas);
+  GradParams g{};
+  g.T = static_cast<int>(T);
+  g.C = static_cast<int>(C);
+  g.r = rows;
+  g.r_pad = rows;
+  g.feat_chunk = sg.feat_chunk;
+  g.n_feat_chunks = sg.n_feat;
+  g.n_token_chunks = sg.n_tok;
+  g.n_slabs = pl->ws.n_slabs;
+  g.stages = grad_stages(rows, true, side_mn, false);
+  g.rt_bufs = grad_rt_bufs(rows, false);
+  g.tmem_cols = grad_tmem_cols(sg.feat_chunk, rows, false, true);
+  g.with_p = 1;
+  g.side_mn = side_mn ? 1 : 0;
+  g.do_out = 0;
+  g.scale = scale;
+  g.p_part = part;
+  g.side_count = count;
+  g.pt_out = out_t;
+  g.ld_t = pl->ws.ld_t;
+  g.status = pl->d_status;
+  g.wait_limit = pl->wait_limit;
+  job->p = g;
+  return true;
+}
+
+// generic gradient job: out = S^T Rt^T over the tokens, Rt [rows, T]
+bool build_grad_job(lora_plan* pl, const void* S, long long C, long long pitch, const __nv_bfloat16* Rt, int rows, void* out,
+                    bool out_is_da, int feat_chunk, int n_tok, GradJobDesc* job) {
+  const long long T = pl->shape.T;
+  bool ok = make_bf16_tmap(&job->tmS, S, C, T, pitch, 64, kGradSlab);
+  ok = ok && make_bf16_tmap(&job->tmR, Rt, T, rows, pl->ws.ld_t, 64, rows);
+  if (!ok) return false;
+  job->tmSide = job->tmR;
+  GradParams g{};
+  g.T = static_cast<int>(T);
+  g.C = static_cast<int>(C);
+  g.r = rows;
+  g.r_pad = rows;
+  g.feat_chunk = feat_chunk;
+  g.n_feat_chunks = ceil_div(C, feat_chunk);
+  g.n_token_chunks = n_tok;
+  g.n_slabs = pl->ws.n_slabs;
+  g.stages = grad_stages(kGroupRowsPerJob, false, false, true);     // every job of the launch sizes its ring for the widest
+  g.rt_bufs = grad_rt_bufs(kGroupRowsPerJob, true);
+  g.tmem_cols = grad_tmem_cols(feat_chunk, rows, true, false);
+  g.do_out = 1;
+  g.out_is_da = out_is_da ? 1 : 0;
+  g.accumulate = pl->accumulate ? 1 : 0;
+  g.scale = 1.f;
+  g.out = static_cast<float*>(out);
+  g.ld_t = pl->ws.ld_t;
+  g.status = pl->d_status;
+  g.wait_limit = pl->wait_limit;
+  job->p = g;
+  return true;
+}
+
+// the side-product jobs of a grouped launch: [G jobs dY_g B_g ->] Qt rows of group g, and X A_cat^T in chunks of at most 64
+// adapter rows -> Pt rows; CTAs are shared out in proportion to the bytes each job streams
+int launch_grouped_sides(lora_plan* pl, const void* dY, const void* B, const void* X, const void* A, float scale, bool with_q,
+                         cudaStream_t st) {
+  const int G = pl->n_groups;
+  const long long r = pl->shape.r, D = pl->shape.d_out, d_in = pl->shape.d_in, R = G * r;
+  uint8_t* ws = static_cast<uint8_t*>(pl->workspace);
+  __nv_bfloat16* qt = reinterpret_cast<__nv_bfloat16*>(ws + pl->gws.qt);
+  __nv_bfloat16* pt = reinterpret_cast<__nv_bfloat16*>(ws + pl->gws.pt);
+  const int ld_t = pl->ws.ld_t;
+  const int n_p = ceil_div(R, kGroupRowsPerJob);
+  const int n_jobs = (with_q ? G : 0) + n_p;
+  double bytes = 0;
+  for (int g = 0; g < G && with_q; ++g) bytes += static_cast<double>(pl->group_off[g + 1] - pl->group_off[g]);
+  bytes += static_cast<double>(n_p) * d_in;
+  GradJobDesc jobs[kGradMaxJobs];
+  int j = 0, left = pl->num_sms;
+  auto share = [&](long long C, int jobs_left) {
+    int c = static_cast<int>(pl->num_sms * (static_cast<double>(C) / bytes) + 0.5);
+    if (c < 1) c = 1;
+    if (c > left - (jobs_left - 1)) c = left - (jobs_left - 1);
+    left -= c;
+    return c;
+  };
+  bool partials = false;
+  for (int g = 0; g < G && with_q; ++g, ++j) {
+    const long long off = pl->group_off[g], dg = pl->group_off[g + 1] - off;
+    if (!build_side_job(pl, static_cast<const __nv_bfloat16*>(dY) + off, dg, D, static_cast<const __nv_bfloat16*>(B) + off * r, true, r,
+                        static_cast<int>(r), scale, qt + static_cast<size_t>(g) * r * ld_t,
+                        reinterpret_cast<float*>(ws + pl->gws.part + j * pl->gws.part_stride),
+                        reinterpret_cast<int*>(ws + pl->gws.count) + j * pl->ws.n_slabs, share(dg, n_jobs - j), &jobs[j]))
+      return LORA_ERR_CUDA;
+    partials = partials || jobs[j].p.n_feat_chunks > 1;
+  }
+  for (int c = 0; c < n_p; ++c, ++j) {
+    const long long row0 = static_cast<long long>(c) * kGroupRowsPerJob;
+    const int rows = static_cast<int>(R - row0 < kGroupRowsPerJob ? R - row0 : kGroupRowsPerJob);
+    if (!build_side_job(pl, X, d_in, d_in, static_cast<const __nv_bfloat16*>(A) + row0 * d_in, false, d_in, rows, scale,
+                        pt + static_cast<size_t>(row0) * ld_t, reinterpret_cast<float*>(ws + pl->gws.part + j * pl->gws.part_stride),
+                        reinterpret_cast<int*>(ws + pl->gws.count) + j * pl->ws.n_slabs, share(d_in, n_jobs - j), &jobs[j]))
+      return LORA_ERR_CUDA;
+    partials = partials || jobs[j].p.n_feat_chunks > 1;
+  }
+  if (partials && !pl->counters_clean) {
+    if (cudaMemsetAsync(ws + pl->gws.count, 0, static_cast<size_t>(kGradMaxJobs) * pl->ws.n_slabs * sizeof(int), st) != cudaSuccess)
+      return LORA_ERR_CUDA;
+    pl->counters_clean = true;
+  }
+  if (launch_grad_jobs(jobs, n_jobs, st) != cudaSuccess) return LORA_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return LORA_OK;
+}
+
+// dA_cat (chunks of at most 64 adapter rows over X) and dB_g (every group over its columns of dY) in ONE launch
+int launch_grouped_grads(lora_plan* pl, const void* dY, const void* X, void* dA, void* dB, cudaStream_t st) {
+  const int G = pl->n_groups;
+  const long long r = pl->shape.r, D = pl->shape.d_out, d_in = pl->shape.d_in, R = G * r;
+  uint8_t* ws = static_cast<uint8_t*>(pl->workspace);
+  const __nv_bfloat16* qt = reinterpret_cast<const __nv_bfloat16*>(ws + pl->gws.qt);
+  const __nv_bfloat16* pt = reinterpret_cast<const __nv_bfloat16*>(ws + pl->gws.pt);
+  const int ld_t = pl->ws.ld_t;
+  const int n_a = ceil_div(R, kGroupRowsPerJob);
+  long long C[kGradMaxJobs];
+  int n_jobs = 0;
+  for (int c = 0; c < n_a; ++c) C[n_jobs++] = d_in;
+  for (int g = 0; g < G; ++g) C[n_jobs++] = pl->group_off[g + 1] - pl->group_off[g];
+  const GradGrid gg = grad_pick_grid_jobs(pl->shape.T, C, n_jobs, kGroupRowsPerJob, false, false, pl->caps);
+  GradJobDesc jobs[kGradMaxJobs];
+  int j = 0;
+  for (int c = 0; c < n_a; ++c, ++j) {
+    const long long row0 = static_cast<long long>(c) * kGroupRowsPerJob;
+    const int rows = static_cast<int>(R - row0 < kGroupRowsPerJob ? R - row0 : kGroupRowsPerJob);
+    if (!build_grad_job(pl, X, d_in, d_in, qt + static_cast<size_t>(row0) * ld_t, rows, static_cast<float*>(dA) + row0 * d_in, true,
+                        gg.feat_chunk, gg.n_tok, &jobs[j]))
+      return LORA_ERR_CUDA;
+  }
+  for (int g = 0; g < G; ++g, ++j) {
+    const long long off = pl->group_off[g], dg = pl->group_off[g + 1] - off;
+    if (!build_grad_job(pl, static_cast<const __nv_bfloat16*>(dY) + off, dg, D, pt + static_cast<size_t>(g) * r * ld_t, static_cast<int>(r),
+                        static_cast<float*>(dB) + off * r, false, gg.feat_chunk, gg.n_tok, &jobs[j]))
+      return LORA_ERR_CUDA;
+  }
+  if (launch_grad_jobs(jobs, n_jobs, st) != cudaSuccess) return LORA_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return LORA_OK;
+}
+
+// forward GEMM over the concatenated output columns; the rank-r k-block of a tile takes its group's rows of s (X A^T)^T
+int launch_grouped_fwd_gemm(lora_plan* pl, const void* X, const void* W, const void* B, float scale, void* Y, cudaStream_t st) {
+  const lora_shape_t& s = pl->shape;
+  const int pairs = pl->num_sms / 2, bn = 256, r = static_cast<int>(s.r);
+  uint8_t* ws = static_cast<uint8_t*>(pl->workspace);
+  CUtensorMap tmX, tmW, tmPt, tmB, tmY;
+  bool ok = make_bf16_tmap(&tmX, X, s.d_in, s.T, s.d_in, 64, kBlockM);
+  ok = ok && make_bf16_tmap(&tmW, W, s.d_in, s.d_out, s.d_in, 64, bn / 2);
+  ok = ok && make_bf16_tmap(&tmPt, ws + pl->gws.pt, s.T, pl->n_groups * r, pl->ws.ld_t, 64, r);
+  ok = ok && make_bf16_tmap(&tmB, B, s.r, s.d_out, s.r, 64, bn / 2);
+  ok = ok && make_bf16_tmap(&tmY, Y, s.d_out, s.T, s.d_out, 64, kBlockM);
+  if (!ok) return LORA_ERR_CUDA;
+  GemmParams p{};
+  p.out = static_cast<__nv_bfloat16*>(Y);
+  p.ld_out = static_cast<int>(s.d_out);
+  p.M = static_cast<int>(s.T);
+  p.N = static_cast<int>(s.d_out);
+  p.K = static_cast<int>(s.d_in);
+  p.r_pad = r;
+  p.block_n = bn;
+  p.tiles_m = ceil_div(s.T, kPairBlockM);
+  p.tiles_n = ceil_div(s.d_out, bn);
+  p.num_tiles = p.tiles_m * p.tiles_n;
+  p.kblocks = ceil_div(s.d_in, kBlockK);
+  p.group_m = pl->cfg.group_m;
+  p.stages = 6;
+  p.tail_delay = pl->cfg.tail_delay;
+  p.scale = scale;
+  p.kb_per_split = p.kblocks;
+  p.split_k = 1;
+  p.ld_rt = pl->ws.ld_t;
+  p.status = pl->d_status;
+  p.wait_limit = pl->wait_limit;
+  p.tail_parts = 1;
+  p.n_groups = pl->n_groups;
+  for (int g = 0; g < pl->n_groups; ++g) p.group_end[g] = static_cast<int>(pl->group_off[g + 1]);
+  const int ctas = 2 * (p.num_tiles < pairs ? p.num_tiles : pairs);
+  if (launch_gemm_pair_fwd_ext(tmX, tmW, tmPt, tmB, tmY, p, ctas, st) != cudaSuccess) return LORA_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return LORA_OK;
+}
+
+// dX GEMM over the concatenated contraction (all groups' dY columns), plus one rank-r k-block per group
+int launch_grouped_dx_gemm(lora_plan* pl, const void* dY, const void* W, const void* A, float scale, void* dX, cudaStream_t st) {
+  const lora_shape_t& s = pl->shape;
+  const int pairs = pl->num_sms / 2, r = static_cast<int>(s.r), R = pl->n_groups * r;
+  uint8_t* ws = static_cast<uint8_t*>(pl->workspace);
+  const int bn = pick_pair_block_n(s.T, s.d_in, 0, pairs);
+  CUtensorMap tmdY, tmW, tmQt, tmA, tmdX;
+  bool ok = make_bf16_tmap(&tmdY, dY, s.d_out, s.T, s.d_out, 64, kBlockM);
+  ok = ok && make_bf16_tmap(&tmW, W, s.d_in, s.d_out, s.d_in, 64, 64);
+  ok = ok && make_bf16_tmap(&tmQt, ws + pl->gws.qt, s.T, R, pl->ws.ld_t, 64, r);
+  ok = ok && make_bf16_tmap(&tmA, A, s.d_in, R, s.d_in, 64, r);
+  ok = ok && make_bf16_tmap(&tmdX, dX, s.d_in, s.T, s.d_in, 64, kBlockM);
+  if (!ok) return LORA_ERR_CUDA;
+  GemmParams p{};
+  p.out = static_cast<__nv_bfloat16*>(dX);
+  p.ld_out = static_cast<int>(s.d_in);
+  p.M = static_cast<int>(s.T);
+  p.N = static_cast<int>(s.d_in);
+  p.K = static_cast<int>(s.d_out);
+  p.r_pad = r;
+  p.block_n = bn;
+  p.tiles_m = ceil_div(s.T, kPairBlockM);
+  p.tiles_n = ceil_div(s.d_in, bn);
+  p.num_tiles = p.tiles_m * p.tiles_n;
+  p.kblocks = ceil_div(s.d_out, kBlockK);
+  p.group_m = pl->cfg.group_m;
+  p.stages = 6;
+  p.tail_delay = pl->cfg.tail_delay;
+  p.scale = scale;
+  p.kb_per_split = p.kblocks;
+  p.split_k = 1;
+  p.ld_rt = pl->ws.ld_t;
+  p.status = pl->d_status;
+  p.wait_limit = pl->wait_limit;
+  p.tail_parts = pl->n_groups;
+  const int ctas = 2 * (p.num_tiles < pairs ? p.num_tiles : pairs);
+  if (launch_gemm_pair_dx(tmdY, tmW, tmQt, tmA, tmdX, p, ctas, st) != cudaSuccess) return LORA_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return LORA_OK;
+}
+
+int check_group_shape(const lora_group_shape_t* g) {
+  if (g == nullptr) return LORA_ERR_INVALID_ARG;
+  if (g->T <= 0 || g->d_in <= 0 || g->r <= 0 || g->n_groups < 2 || g->n_groups > 4) return LORA_ERR_INVALID_ARG;
+  if (g->T <= kBlockM || g->T > (1ll << 30) || g->d_in > (1ll << 24) || g->d_in % 8 != 0) return LORA_ERR_UNSUPPORTED_SHAPE;
+  if (g->r % 16 != 0 || g->r > 64) return LORA_ERR_UNSUPPORTED_SHAPE;        // a group's rows are whole 16-row MMA k-steps
+  const int n_jobs_sides = g->n_groups + ceil_div(g->n_groups * g->r, kGroupRowsPerJob);
+  if (n_jobs_sides > kGradMaxJobs) return LORA_ERR_UNSUPPORTED_SHAPE;
+  long long total = 0;
+  for (int i = 0; i < g->n_groups; ++i) {
+    if (g->d_out[i] <= 0) return LORA_ERR_INVALID_ARG;
+    if (g->d_out[i] % 256 != 0) return LORA_ERR_UNSUPPORTED_SHAPE;            // output tiles must not straddle two groups
+    total += g->d_out[i];
+  }
+  if (total > (1ll << 24)) return LORA_ERR_UNSUPPORTED_SHAPE;
+  return LORA_OK;
+}
+
 }  // namespace
 
 extern "C" {
+
+int lora_plan_create_grouped(const lora_group_shape_t* gshape, int device, lora_plan_t** out) {
+  if (out == nullptr) return LORA_ERR_INVALID_ARG;
+  *out = nullptr;
+  int rc = check_group_shape(gshape);
+  if (rc != LORA_OK) return rc;
+  lora_shape_t flat;
+  flat.T = gshape->T;
+  flat.d_in = gshape->d_in;
+  flat.r = gshape->r;
+  flat.d_out = 0;
+  for (int i = 0; i < gshape->n_groups; ++i) flat.d_out += gshape->d_out[i];
+  lora_plan_t* pl = nullptr;
+  rc = lora_plan_create(&flat, device, &pl);
+  if (rc != LORA_OK) return rc;
+  if (pl->num_sms < 2 * kGradMaxJobs) {
+    lora_plan_destroy(pl);
+    return LORA_ERR_NO_DEVICE;
+  }
+  pl->n_groups = gshape->n_groups;
+  pl->group_off[0] = 0;
+  for (int i = 0; i < gshape->n_groups; ++i) pl->group_off[i + 1] = pl->group_off[i] + gshape->d_out[i];
+  // workspace: the stacked products of all groups, one partial-sum region and one counter range per streaming job
+  const size_t R = static_cast<size_t>(gshape->n_groups) * gshape->r;
+  size_t off = 0;
+  pl->gws.qt = off;     off += align_up(R * pl->ws.ld_t * 2, kAlign);
+  pl->gws.pt = off;     off += align_up(R * pl->ws.ld_t * 2, kAlign);
+  pl->gws.part_stride = align_up(static_cast<size_t>(kSideMaxChunks) * kGroupRowsPerJob * pl->ws.ld_t * 4, kAlign);
+  pl->gws.part = off;   off += kGradMaxJobs * pl->gws.part_stride;
+  pl->gws.count = off;  off += align_up(static_cast<size_t>(kGradMaxJobs) * pl->ws.n_slabs * sizeof(int), kAlign);
+  pl->gws.total = off;
+  pl->ws.total = off;                                     // what lora_plan_workspace_bytes / lora_plan_set_workspace go by
+  *out = pl;
+  return LORA_OK;
+}
+
+int lora_linear_fwd_grouped(lora_plan_t* plan, const void* X, const void* W_cat, const void* A_cat, const void* B_cat, float scale,
+                            void* Y_cat, void* stream) {
+  if (plan == nullptr || plan->n_groups < 2) return LORA_ERR_INVALID_ARG;
+  if (!X || !W_cat || !A_cat || !B_cat || !Y_cat) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(W_cat) || !aligned16(A_cat) || !aligned16(B_cat) || !aligned16(Y_cat)) return LORA_ERR_MISALIGNED;
+  if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
+  DeviceGuard guard(plan->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int rc = launch_grouped_sides(plan, nullptr, nullptr, X, A_cat, scale, false, st);      // Pt_all = s (X A_cat^T)^T
+  if (rc == LORA_OK) rc = launch_grouped_fwd_gemm(plan, X, W_cat, B_cat, scale, Y_cat, st);
+  return rc;
+}
+
+int lora_linear_bwd_grouped(lora_plan_t* plan, const void* dY_cat, const void* X, const void* W_cat, const void* A_cat,
+                            const void* B_cat, float scale, void* dX, void* dA_cat, void* dB_cat, void* stream) {
+  if (plan == nullptr || plan->n_groups < 2) return LORA_ERR_INVALID_ARG;
+  if (!dY_cat || !X || !W_cat || !A_cat || !B_cat || !dX || !dA_cat || !dB_cat) return LORA_ERR_INVALID_ARG;
+  if (!aligned16(dY_cat) || !aligned16(X) || !aligned16(W_cat) || !aligned16(A_cat) || !aligned16(B_cat) || !aligned16(dX) ||
+      !aligned16(dA_cat) || !aligned16(dB_cat))
+    return LORA_ERR_MISALIGNED;
+  if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
+  DeviceGuard guard(plan->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int rc = launch_grouped_sides(plan, dY_cat, B_cat, X, A_cat, scale, true, st);          // Qt_all and Pt_all, one launch
+  if (rc == LORA_OK) rc = launch_grouped_dx_gemm(plan, dY_cat, W_cat, A_cat, scale, dX, st);
+  if (rc == LORA_OK) rc = launch_grouped_grads(plan, dY_cat, X, dA_cat, dB_cat, st);
+  return rc;
+}
 
 int lora_select_config(const lora_shape_t* shape, int num_sms, lora_kernel_config_t* out) {
   return select_config(shape, num_sms, out);
@@ -1078,6 +1427,14 @@ int lora_plan_create(const lora_shape_t* shape, int device, lora_plan_t** out) {
     if (v >= 1000) pl->wait_limit = v;
   }
   pl->counters_clean = false;
+  pl->n_groups = 0;
+  if (const char* f = std::getenv("LORA_LOG")) {          // LORA_LOG=1: one line per plan with what the selector chose
+    if (std::atoi(f) != 0) {
+      char line[1024];
+      lora_plan_describe(pl, line, sizeof(line));
+      std::fprintf(stderr, "[lora_linear] plan %p: %s\n", static_cast<void*>(pl), line);
+    }
+  }
   if (cudaMalloc(&pl->d_status, 256) != cudaSuccess || cudaMemset(pl->d_status, 0, 256) != cudaSuccess) {
     cudaGetLastError();
     if (pl->d_status) cudaFree(pl->d_status);
@@ -1098,7 +1455,7 @@ int lora_plan_destroy(lora_plan_t* plan) {
 
 int lora_plan_workspace_bytes(const lora_plan_t* plan, size_t* fwd_bytes, size_t* bwd_bytes) {
   if (plan == nullptr) return LORA_ERR_INVALID_ARG;
-  if (fwd_bytes) *fwd_bytes = (plan->cfg.cta_group == 2 && plan->cfg.fwd_ext) ? plan->ws.total : 0;
+  if (fwd_bytes) *fwd_bytes = (plan->n_groups != 0 || (plan->cfg.cta_group == 2 && plan->cfg.fwd_ext)) ? plan->ws.total : 0;
   if (bwd_bytes) *bwd_bytes = plan->ws.total;
   return LORA_OK;
 }
@@ -1188,7 +1545,7 @@ int lora_plan_describe(const lora_plan_t* plan, char* buf, size_t n) {
 
 int lora_linear_fwd(lora_plan_t* plan, const void* X, const void* W, const void* A, const void* B, float scale,
                     void* Y, void* stream) {
-  if (plan == nullptr) return LORA_ERR_INVALID_ARG;
+  if (plan == nullptr || plan->n_groups != 0) return LORA_ERR_INVALID_ARG;
   if (plan->shape.T == 0) return LORA_OK;
   if (!X || !W || !A || !B || !Y) return LORA_ERR_INVALID_ARG;
   if (!aligned16(X) || !aligned16(W) || !aligned16(A) || !aligned16(B) || !aligned16(Y)) return LORA_ERR_MISALIGNED;
@@ -1198,7 +1555,7 @@ int lora_linear_fwd(lora_plan_t* plan, const void* X, const void* W, const void*
 
 int lora_linear_bwd(lora_plan_t* plan, const void* dY, const void* X, const void* W, const void* A, const void* B,
                     float scale, void* dX, void* dA, void* dB, void* stream) {
-  if (plan == nullptr) return LORA_ERR_INVALID_ARG;
+  if (plan == nullptr || plan->n_groups != 0) return LORA_ERR_INVALID_ARG;
   if (!dA || !dB) return LORA_ERR_INVALID_ARG;
   if (!aligned16(dA) || !aligned16(dB)) return LORA_ERR_MISALIGNED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);

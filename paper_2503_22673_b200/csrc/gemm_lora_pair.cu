@@ -219,10 +219,19 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       }
       __syncwarp();
     };
-    auto load_tail = [&](int m0, int n0) {
+    // K-extended forms, grouped projections: the rank-r k-block of a FORWARD tile takes the rows of s (X A^T)^T that belong
+    // to the tile's group (srow = group x r_pad, one part); the dX GEMM adds one part per group (rows part x r_pad of
+    // s (dY B)^T and of the stacked A).  Ungrouped: one part, row 0.
+    auto load_tail = [&](int m0, int n0, int part) {
       const int cur = acquire();
       if (cur < 0 || !ok) return;
       const int nb = n0 + static_cast<int>(rank) * (BN >> 1);
+      int srow = part * p.r_pad;
+      if (kExt && !kBmn && p.n_groups > 1) {
+        int g = 0;
+        while (g + 1 < p.n_groups && n0 >= p.group_end[g]) ++g;
+        srow = g * p.r_pad;
+      }
       const uint32_t a_dst = ring + cur * kStage, b_dst = a_dst + 16384;
       const uint32_t fb = map_to_cta(full_bar(cur), 0);
       if (elect_one()) {
@@ -236,8 +245,8 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
             const uint32_t side_bytes = 2 * 2 * p.r_pad * 128;
             const uint32_t tail_bytes = kNf4 ? (kBmn ? 2 * 2 * p.r_pad * 128 : BN * 128) : 0;
             if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), side_bytes + tail_bytes);
-            tma_load_2d_pair(a_dst, &tm_side, fb, m0, 0);
-            tma_load_2d_pair(a_dst + p.r_pad * 128, &tm_side, fb, m0 + 64, 0);
+            tma_load_2d_pair(a_dst, &tm_side, fb, m0, srow);
+            tma_load_2d_pair(a_dst + p.r_pad * 128, &tm_side, fb, m0 + 64, srow);
             if (kNf4 && !kBmn) {
               tma_load_2d_pair(b_dst, &tm_tail, fb, 0, nb);
             } else if (kNf4) {
@@ -250,8 +259,8 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
           tma_load_2d_pair(b_dst, &tm_tail, fb, 0, nb);
         } else {
           if (rank == 0) mbar_arrive_expect_tx(full_bar(cur), 2 * 2 * p.r_pad * 128);
-          tma_load_2d_pair(b_dst, &tm_tail, fb, nb, 0);
-          tma_load_2d_pair(b_dst + 8192, &tm_tail, fb, nb + 64, 0);
+          tma_load_2d_pair(b_dst, &tm_tail, fb, nb, srow);
+          tma_load_2d_pair(b_dst + 8192, &tm_tail, fb, nb + 64, srow);
         }
       }
       __syncwarp();
@@ -294,14 +303,15 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       const int m0 = tc.m_idx * kPairBlockM + static_cast<int>(rank) * 128, n0 = tc.n_idx * BN;
       const int kb0 = sp * p.kb_per_split, kb1 = min(KB, kb0 + p.kb_per_split);
       for (int kb = kb0; kb < kb1 && ok; ++kb) {
-        if (!kExt && i > 0 && kb == D) load_tail(0, prev_n0);
+        if (!kExt && i > 0 && kb == D) load_tail(0, prev_n0, 0);
         if (ok) load_main(m0, n0, kb * kBlockK);
       }
-      if (!kExt && ok && i > 0 && D == KB) load_tail(0, prev_n0);
-      if (kExt && ok && sp == SK - 1 && p.r_pad > 0) load_tail(m0, n0);
+      if (!kExt && ok && i > 0 && D == KB) load_tail(0, prev_n0, 0);
+      if (kExt && sp == SK - 1 && p.r_pad > 0)
+        for (int part = 0; part < p.tail_parts && ok; ++part) load_tail(m0, n0, part);
       prev_n0 = n0;
     }
-    if (!kExt && ok && n_my > 0 && !(kNf4 && op == 1)) load_tail(0, prev_n0);
+    if (!kExt && ok && n_my > 0 && !(kNf4 && op == 1)) load_tail(0, prev_n0, 0);
   } else if (warp == 4) {
     // ================================ MMA issuer (leader CTA only) ================================
     // Whole warp of the leader CTA runs the loop; one lane polls, one elected lane issues every MMA and commit.
@@ -340,7 +350,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
         __syncwarp();
         next();
       };
-      auto mma_tail = [&](int buf, int use) {
+      auto mma_tail = [&](int buf, int use, bool last_part) {
         if (!kExt) ok = warp_wait(ps_ready(buf), use & 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_PS, true, 0);
         if (ok) ok = warp_wait(full_bar(slot), phase, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_FULL, true, 0);
         if (!ok) return;
@@ -350,7 +360,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
           for (int ks = 0; ks < p.r_pad / 16; ++ks)
             mma_bf16_ss_pair(tmem_base + buf * 256, pd0 + (kExt ? so : 0u) + ks * kPStep, bd0 + so + ks * kBStep, idesc_tail, 1u);
           mma_commit_pair(empty_bar(slot));
-          mma_commit_pair(acc_full(buf));
+          if (last_part) mma_commit_pair(acc_full(buf));
         }
         __syncwarp();
         next();
@@ -362,13 +372,14 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
         const bool has_tail = !kExt || (sp == SK - 1 && p.r_pad > 0);
         ok = warp_wait(acc_empty(buf), (use & 1) ^ 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_ACC_EMPTY, true, 0);
         for (int kb = kb0; kb < kb1 && ok; ++kb) {
-          if (!kExt && i > 0 && kb == D) mma_tail(buf ^ 1, (i - 1) >> 1);
+          if (!kExt && i > 0 && kb == D) mma_tail(buf ^ 1, (i - 1) >> 1, true);
           if (ok) mma_main(buf, kb == kb0, kb == kb1 - 1, has_tail);
         }
-        if (!kExt && ok && i > 0 && D == KB) mma_tail(buf ^ 1, (i - 1) >> 1);
-        if (kExt && ok && has_tail) mma_tail(buf, use);
+        if (!kExt && ok && i > 0 && D == KB) mma_tail(buf ^ 1, (i - 1) >> 1, true);
+        if (kExt && has_tail)
+          for (int part = 0; part < p.tail_parts && ok; ++part) mma_tail(buf, use, part == p.tail_parts - 1);
       }
-      if (!kExt && ok && n_my > 0) mma_tail((n_my - 1) & 1, (n_my - 1) >> 1);
+      if (!kExt && ok && n_my > 0) mma_tail((n_my - 1) & 1, (n_my - 1) >> 1, true);
     }
   } else if (kNf4 && warp >= kPairThreads / 32) {
     // ================================ NF4 dequantisation (warps 9..16, 256 threads per CTA) ================================
@@ -392,7 +403,7 @@ lora_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_act,   // X / dY [M
       const int sp = (pair + i * G) % SK;
       const int kb0 = sp * p.kb_per_split, kb1 = min(KB, kb0 + p.kb_per_split);
       const bool has_tail = sp == SK - 1 && p.r_pad > 0;
-      for (int kb = kb0; kb < kb1 + (has_tail ? 1 : 0) && ok; ++kb) {
+      for (int kb = kb0; kb < kb1 + (has_tail ? p.tail_parts : 0) && ok; ++kb) {
         const bool main_item = kb < kb1;
         if (turn == gid) {
           if (main_item) ok = warp_wait(cfull_bar(cslot), cphase, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_FULL, false, 0);

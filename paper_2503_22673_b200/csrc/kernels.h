@@ -60,6 +60,10 @@ struct GemmParams {
   float* part;            // fp32 partial tiles [split_k][M][N] when split_k > 1
   __nv_bfloat16* out;     // CTA-pair kernel only: output base and row pitch (elements) for the ragged last chunk
   int ld_out;
+  // K-extended CTA-pair kernel, grouped projections (several projections share the activations; see lora_linear_fwd_grouped):
+  int tail_parts;         // rank-r k-blocks per tile (>= 1; the dX GEMM of G groups adds G of them, rows part x r_pad)
+  int n_groups;           // forward: output-column groups (<= 1: ungrouped); a tile's rank-r k-block uses the rows
+  int group_end[4];       //   group x r_pad of s (X A^T)^T, group = first g with n0 < group_end[g]
 };
 
 size_t gemm_smem_bytes(int stages);
@@ -174,6 +178,8 @@ struct GradGrid {
 // columns) and are resident at once (caps[cs] = CTAs resident at once in clusters of cs CTAs, cs = 1 .. kGradMaxCluster).
 // n_feat counts the feature chunks of both jobs.
 GradGrid grad_pick_grid(long long T, long long C, long long C2, int r_pad, bool with_p, bool side_mn, const int* caps);
+// the same for n_jobs streamed matrices with C[j] features side by side (r_pad: the largest of the jobs)
+GradGrid grad_pick_grid_jobs(long long T, const long long* C, int n_jobs, int r_pad, bool with_p, bool side_mn, const int* caps);
 // caps[0 .. kGradMaxCluster] estimated from the SM count alone (host-only selector calls) / asked from the current device
 void grad_default_caps(int num_sms, int* caps);
 void grad_device_caps(int num_sms, int* caps);
@@ -184,10 +190,21 @@ int grad_tmem_cols(int feat_chunk, int r_pad, bool do_out, bool with_p);
 int grad_rt_bufs(int r_pad, bool do_out);
 int grad_stages(int r_pad, bool with_p, bool side_mn, bool do_out);
 
-// One launch of the streaming kernel: one or two jobs side by side (CTAs with blockIdx.x < split_x run job 0)
+// One launch of the streaming kernel: up to kGradMaxJobs jobs side by side (CTAs with blockIdx.x in [x_end[j-1], x_end[j])
+// run job j)
+constexpr int kGradMaxJobs = 6;
 struct GradLaunch {
-  GradParams job[2];
-  int split_x;
+  GradParams job[kGradMaxJobs];
+  int x_end[kGradMaxJobs];
+  int n_jobs;
+};
+struct GradMaps {
+  CUtensorMap m[3 * kGradMaxJobs];       // per job: streamed matrix, second factor, side operand
+};
+// what the host passes per job
+struct GradJobDesc {
+  CUtensorMap tmS, tmR, tmSide;
+  GradParams p;
 };
 
 size_t grad_smem_bytes(const GradParams& p);
@@ -201,9 +218,7 @@ int grad_max_resident_ctas(int cluster, size_t smem_bytes);
 // (distributed shared memory, rank order), the side product over the feature chunks by the last CTA to arrive (chunk order).
 cudaError_t launch_grad(const CUtensorMap& tmS, const CUtensorMap& tmR, const CUtensorMap& tmA,
                         const GradParams& p, cudaStream_t stream);
-// Two jobs in one launch (p1 == nullptr: one job).  tm0 / tm1 = {streamed matrix, second factor, side operand} of each
-// job.  Both jobs compute a gradient with the same cluster size, or both compute only a side product.
-cudaError_t launch_grad2(const CUtensorMap* const tm0[3], const GradParams& p0, const CUtensorMap* const tm1[3],
-                         const GradParams* p1, cudaStream_t stream);
+// Several jobs in one launch.  All jobs compute a gradient with the same cluster size, or all compute only a side product.
+cudaError_t launch_grad_jobs(const GradJobDesc* jobs, int n_jobs, cudaStream_t stream);
 
 }  // namespace lora

@@ -292,12 +292,16 @@ def test_backward_with_saved_forward_product_matches_oracle():
         plan.close()
 
 
-def test_grouped_projections_sharing_x_match_separate_oracles():
-    """q/k/v-style group as one layer (stacked A, block-diagonal B): every projection must match ITS OWN oracle,
-    and dX the sum of the three."""
+@pytest.mark.parametrize("T,d_in,d_outs,r,scale", [
+    (900, 520, [768, 256, 256], 16, 2.0),          # q/k/v style, r = 16: one 48-row side job, one dA job
+    (1300, 1032, [512, 256, 256], 32, 2.0),        # the paper's adapter rank (Section 4.5): 96 adapter rows -> two X jobs
+    (700, 264, [768, 768], 64, 0.5),               # gate/up style at the largest rank
+    (2100, 512, [256, 512, 256, 256], 16, 1.7),    # four groups, more tiles than CTA pairs per group
+])
+def test_grouped_projections_sharing_x_match_separate_oracles(T, d_in, d_outs, r, scale):
+    """lora_linear_fwd_grouped / lora_linear_bwd_grouped: every projection of the group must match ITS OWN oracle, and dX
+    the sum of the groups' oracles' dX."""
     from paper_2503_22673_b200.grouped import GroupedLoraPlan
-    T, d_in, r, scale = 900, 520, 16, 2.0
-    d_outs = [392, 136, 136]
     projs = [inputs.draw_custom(T, d_in, d, r, scale, seed=30 + g, tag=70 + g) for g, d in enumerate(d_outs)]
     X_bits = projs[0][1]["X"]
     f64 = lambda b: inputs.bf16_to_f64(b)
@@ -305,20 +309,52 @@ def test_grouped_projections_sharing_x_match_separate_oracles():
     W, A, B = gp.pack([dev(t["W"]) for _, t in projs], [dev(t["A"]) for _, t in projs], [dev(t["B"]) for _, t in projs])
     X = dev(X_bits)
     dY = torch.cat([dev(t["dY"]) for _, t in projs], dim=1).contiguous()
-    Y = gp.fwd(X, W, A, B, scale)
-    dX, dAs, dBs = gp.bwd(dY, X, W, A, B, scale)
-    assert gp.plan.device_status()[0] == 0
-    dX_ref = 0.0
-    for g, (p, t) in enumerate(projs):
-        Wg, Ag, Bg, dYg = f64(t["W"]), f64(t["A"]), f64(t["B"]), f64(t["dY"])
-        Yr = oracle.forward(f64(X_bits), Wg, Ag, Bg, scale)
-        dXr, dAr, dBr = oracle.backward(dYg, f64(X_bits), Wg, Ag, Bg, scale)
-        dX_ref = dX_ref + dXr
-        assert oracle.rel_err(host64(gp.split_outputs(Y)[g]), Yr) <= TOL_BF16
-        assert oracle.rel_err(host64(dAs[g]), dAr) <= TOL_F32
-        assert oracle.rel_err(host64(dBs[g]), dBr) <= TOL_F32
-    assert oracle.rel_err(host64(dX), dX_ref) <= TOL_BF16
+    bufs = {}
+    out = {}
+    D = sum(d_outs)
+    for name, shape, dt in (("Y", (T, D), torch.bfloat16), ("dX", (T, d_in), torch.bfloat16),
+                            ("dA", (len(d_outs) * r, d_in), torch.float32), ("dB", (D, r), torch.float32)):
+        bufs[name], out[name] = guarded(shape, dt)
+    for rep in range(2):                                   # twice: the arrival counters must be back at zero
+        Y = gp.fwd(X, W, A, B, scale, out["Y"])
+        dX, dAs, dBs = gp.bwd(dY, X, W, A, B, scale, out["dX"], out["dA"], out["dB"])
+        code, msg = gp.device_status()
+        assert code == 0, msg
+        for name in out:
+            assert guards_intact(bufs[name], out[name].numel()), f"{name}: write outside the tensor"
+            assert not torch.isnan(out[name].float()).any(), f"{name}: element left unwritten"
+        dX_ref = 0.0
+        for g, (p, t) in enumerate(projs):
+            Wg, Ag, Bg, dYg = f64(t["W"]), f64(t["A"]), f64(t["B"]), f64(t["dY"])
+            Yr = oracle.forward(f64(X_bits), Wg, Ag, Bg, scale)
+            dXr, dAr, dBr = oracle.backward(dYg, f64(X_bits), Wg, Ag, Bg, scale)
+            dX_ref = dX_ref + dXr
+            assert oracle.rel_err(host64(gp.split_outputs(Y)[g]), Yr) <= TOL_BF16, (g, rep)
+            assert oracle.rel_err(host64(dAs[g]), dAr) <= TOL_F32, (g, rep)
+            assert oracle.rel_err(host64(dBs[g]), dBr) <= TOL_F32, (g, rep)
+        assert oracle.rel_err(host64(dX), dX_ref) <= TOL_BF16
     gp.close()
+
+
+def test_grouped_plan_rejects_what_it_does_not_cover():
+    from paper_2503_22673_b200.grouped import GroupedLoraPlan
+    for args in ((900, 520, [768, 200], 16), (900, 520, [768, 256], 24), (100, 520, [768, 256], 16), (900, 520, [256] * 4, 64)):
+        with pytest.raises(binding.LoraError) as e:
+            GroupedLoraPlan(*args)
+        assert e.value.code == binding.LORA_ERR_UNSUPPORTED_SHAPE, args
+    gp = GroupedLoraPlan(900, 520, [768, 256], 16)
+    plain = binding.LoraLinearPlan(900, 520, 1024, 16)
+    X = torch.zeros((900, 520), dtype=torch.bfloat16, device="cuda")
+    W = torch.zeros((1024, 520), dtype=torch.bfloat16, device="cuda")
+    A = torch.zeros((16, 520), dtype=torch.bfloat16, device="cuda")
+    B = torch.zeros((1024, 16), dtype=torch.bfloat16, device="cuda")
+    Y = torch.zeros((900, 1024), dtype=torch.bfloat16, device="cuda")
+    lib = binding.load()
+    sp = torch.cuda.current_stream().cuda_stream
+    assert lib.lora_linear_fwd(gp._h, X.data_ptr(), W.data_ptr(), A.data_ptr(), B.data_ptr(), 1.0, Y.data_ptr(), sp) == binding.LORA_ERR_INVALID_ARG
+    assert lib.lora_linear_fwd_grouped(plain._h, X.data_ptr(), W.data_ptr(), A.data_ptr(), B.data_ptr(), 1.0, Y.data_ptr(), sp) == binding.LORA_ERR_INVALID_ARG
+    gp.close()
+    plain.close()
 
 
 def test_split_k_paths_match_oracle(monkeypatch):
