@@ -256,10 +256,10 @@ def to_dev(bits: np.ndarray, device) -> torch.Tensor:
 class Workload:
     """Device tensors, plans and the step function of one workload (n_sets independent input/output sets, rotated per step)."""
 
-    def __init__(self, idx: int, rank: int, local_rank: int, device, n_sets: int = None):
+    def __init__(self, idx: int, rank: int, local_rank: int, device, n_sets: int = None, tokens: int = None):
         from paper_2503_22673_b200 import binding, inputs
         self.idx, self.device, self.binding = idx, device, binding
-        self.protos = inputs.workload(idx)
+        self.protos = inputs.workload(idx, tokens)
         self.bytes_per_set = sum(2 * (p.T * p.d_in * 2 + p.T * p.d_out * 2) + 2 * p.d_out * p.d_in for p in self.protos)
         if n_sets is None:
             n_sets = 2 if idx >= 2 else max(2, min(6, -(-4 * L2_BYTES // self.bytes_per_set)))
@@ -267,7 +267,7 @@ class Workload:
         self.sets = []
         for s_i in range(n_sets):
             cur, x_dev = [], {}
-            for proj, t in inputs.draw_workload(idx, seed=1000 * rank + s_i):
+            for proj, t in inputs.draw_workload(idx, seed=1000 * rank + s_i, T=tokens):
                 d = {k: to_dev(v, device) for k, v in t.items() if k != "X"}
                 if proj.x_group not in x_dev:                 # projections that share X (q/k/v, gate/up) share the tensor
                     x_dev[proj.x_group] = to_dev(t["X"], device)
@@ -469,7 +469,7 @@ def run_ours(args):
             import torch.distributed as dist
             dist.barrier()
 
-    wl = Workload(args.workload, rank, local_rank, device)
+    wl = Workload(args.workload, rank, local_rank, device, tokens=args.tokens)
     protos, plans = wl.protos, wl.plans
     m = measure(wl, args.steps, args.warmup, pk, world, device, barrier)
     ms_step, kern = m["ms_per_step"], m["kernels"]
@@ -566,6 +566,51 @@ def run_ours(args):
                                  "note": "forward + backward with the frozen W in NF4 (4.5 bits per weight); " + how +
                                          "; same algorithmic FLOPs as the bf16 step"}
             del q_sets, w_scratch
+        # ---- variant: projections that share X (q/k/v, gate/up) through the grouped calls, the others through their own plans ----
+        group_ids = {4: [[0, 1, 2], [4, 5]], 5: [[0, 1, 2]]}.get(args.workload, [])
+        if group_ids and all(p.r % 16 == 0 for p in protos):
+            from paper_2503_22673_b200.grouped import GroupedLoraPlan
+            grouped, in_group = [], set()
+            for ids in group_ids:
+                in_group.update(ids)
+                p0 = protos[ids[0]]
+                gp = GroupedLoraPlan(p0.T, p0.d_in, [protos[i].d_out for i in ids], p0.r, device=local_rank)
+                per_set = []
+                for cur in wl.sets:
+                    W, A, B = gp.pack([cur[i][1]["W"] for i in ids], [cur[i][1]["A"] for i in ids], [cur[i][1]["B"] for i in ids])
+                    dYc = torch.cat([cur[i][1]["dY"] for i in ids], dim=1).contiguous()
+                    per_set.append({"X": cur[ids[0]][1]["X"], "W": W, "A": A, "B": B, "dY": dYc,
+                                    "Y": torch.empty_like(dYc), "dX": torch.empty_like(cur[ids[0]][1]["X"]),
+                                    "dA": torch.empty((gp.G * gp.r, gp.d_in), dtype=torch.float32, device=device),
+                                    "dB": torch.empty((gp.D, gp.r), dtype=torch.float32, device=device)})
+                grouped.append((gp, p0.scale, per_set))
+            singles = [j for j in range(len(protos)) if j not in in_group]
+
+            def step_grouped(k):
+                for gp, sc, per_set in grouped:
+                    d = per_set[k % wl.n_sets]
+                    gp.fwd(d["X"], d["W"], d["A"], d["B"], sc, d["Y"])
+                    gp.bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], sc, d["dX"], d["dA"], d["dB"])
+                cur = wl.sets[k % wl.n_sets]
+                for j in singles:
+                    proj, d = cur[j]
+                    plans[j].fwd(d["X"], d["W"], d["A"], d["B"], proj.scale, d["Y"])
+                    plans[j].bwd(d["dY"], d["X"], d["W"], d["A"], d["B"], proj.scale, d["dX"], d["dA"], d["dB"])
+
+            ms_g = timed_loop(step_grouped, n_var, barrier, device, world)
+            for gp, _, _ in grouped:
+                code, msg = gp.device_status()
+                if code != 0:
+                    raise SystemExit(f"bench.py: device status after the grouped variant: {msg}")
+            variants["grouped_shared_x"] = {
+                "ms_per_step": ms_g, "value": job_value(world, flops_step, ms_g), "unit": UNIT, "steps": n_var,
+                "tokens_per_s": world * tokens_step / ms_g * 1e3,
+                "note": "projections sharing X through lora_linear_fwd_grouped / lora_linear_bwd_grouped ("
+                        + ", ".join("+".join(protos[i].name for i in ids) for ids in group_ids)
+                        + "), the others through their own plans; same algorithmic FLOPs (dX of a group is one sum)"}
+            for gp, _, _ in grouped:
+                gp.close()
+            del grouped
         # ---- extra kernel: the dense weight gradient of full fine-tuning, dW = dY^T X (lora_dense_dw), per projection ----
         dw_out = [torch.empty((p.d_out, p.d_in), dtype=torch.bfloat16, device=device) for p in protos]
 
@@ -698,6 +743,9 @@ def main():
     ap.add_argument("--workload", type=int, default=4)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tokens", type=int, default=None,
+                    help="override the workload's token count (profiler captures of a kernel at a size small enough to capture; "
+                         "the line's config then names the reduced T)")
     ap.add_argument("--quick", action="store_true",
                     help="only the timed region and the instrumented pass of the chosen workload (no sustained leg, variants, "
                          "end-to-end leg or other workloads); for profiler captures")

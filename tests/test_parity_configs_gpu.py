@@ -210,6 +210,46 @@ def test_paper_adapter_setting_full_size():
         check_projection(p, t, x_dev)
 
 
+@pytest.mark.parametrize("wl,ids", [(4, (0, 1, 2)), (4, (4, 5)), (5, (0, 1, 2))], ids=["qkv_r16", "gate_up_r16", "qkv_r32"])
+def test_grouped_projections_full_size(wl, ids):
+    """The grouped calls at the benchmark sizes (q/k/v and gate/up of the whole-layer workload, q/k/v of the paper's own
+    r = 32 setting at 49152 tokens): every projection against ITS OWN oracle - two rows of every 128-row slab of Y_g, dA_g
+    and dB_g in full - and dX against the sum of the groups' oracles on the same row sample."""
+    from paper_2503_22673_b200.grouped import GroupedLoraPlan
+    projs = [(p, t) for j, (p, t) in enumerate(inputs.draw_workload(wl, seed=0)) if j in ids]
+    p0 = projs[0][0]
+    gp = GroupedLoraPlan(p0.T, p0.d_in, [p.d_out for p, _ in projs], p0.r)
+    W, A, B = gp.pack([dev(t["W"]) for _, t in projs], [dev(t["A"]) for _, t in projs], [dev(t["B"]) for _, t in projs])
+    X = dev(projs[0][1]["X"])
+    dY = torch.cat([dev(t["dY"]) for _, t in projs], dim=1).contiguous()
+    Y = gp.fwd(X, W, A, B, p0.scale)
+    dX, dAs, dBs = gp.bwd(dY, X, W, A, B, p0.scale)
+    code, msg = gp.device_status()
+    assert code == 0, msg
+    rows = slab_rows(p0.T)
+    rows_t = torch.from_numpy(rows).cuda()
+    Xr = inputs.bf16_to_f64(projs[0][1]["X"][rows])
+    Xf = inputs.bf16_to_f64(projs[0][1]["X"])
+    dX_ref = 0.0
+    errs = {}
+    for g, (p, t) in enumerate(projs):
+        Wg, Ag, Bg = (inputs.bf16_to_f64(t[k]) for k in ("W", "A", "B"))
+        Yr = oracle.forward(Xr, Wg, Ag, Bg, p.scale)
+        dX_ref = dX_ref + oracle.backward_dx_rows(np.arange(len(rows)), inputs.bf16_to_f64(t["dY"][rows]), Wg, Ag, Bg, p.scale)
+        dAr, dBr = oracle.backward_adapter_grads(inputs.bf16_to_f64(t["dY"]), Xf, Ag, Bg, p.scale)
+        errs[p.name] = (oracle.rel_err(host64(gp.split_outputs(Y)[g][rows_t]), Yr), oracle.rel_err(host64(dAs[g]), dAr),
+                        oracle.rel_err(host64(dBs[g]), dBr))
+        del Wg
+    eX = oracle.rel_err(host64(dX[rows_t]), dX_ref)
+    gp.close()
+    for name, (eY, eA, eB) in errs.items():
+        assert eY <= TOL_BF16 and eA <= TOL_F32 and eB <= TOL_F32, (name, errs)
+    assert eX <= TOL_BF16, eX
+    del X, dY, Y, dX, W
+    gc.collect()
+    torch.cuda.empty_cache()
+
+
 def test_more_than_2_31_elements_per_tensor():
     """Index arithmetic beyond 32 bits: X and dX hold 540000 x 4096 = 2.2e9 elements (4.4 GB each).  The oracle cannot hold
     such a matrix in float64, so: sampled rows of Y and dX (first, last, around the 2^31-element boundary, random) against
