@@ -69,7 +69,10 @@ lora_grad_kernel(const __grid_constant__ GradMaps maps, const __grid_constant__ 
   const int NB = p.feat_chunk >> 7;                 // 128-feature accumulator blocks of a full chunk
   const int rt_box = p.r_pad * 128;                 // bytes of one 64-wide box with r_pad rows
   const int side_box = p.side_mn ? 8192 : rt_box;   // bytes of the side operand for 64 features
-  const int stage_bytes = kGradStageBytes + (p.with_p ? 2 * side_box : 0);   // S tile (+ the matching side operand)
+  // A gradient CTA with ONE block and no side product needs a new slab of the second factor with every tile: the slab then
+  // travels in the tile's own stage (same barrier, same producer), and the loader warp and its ring are idle.
+  const bool rt_in_stage = p.rt_in_stage != 0;
+  const int stage_bytes = kGradStageBytes + (p.with_p ? 2 * side_box : 0) + (rt_in_stage ? 2 * rt_box : 0);
   const int ring_bytes = p.stages * stage_bytes;
   const uint32_t ring = smem_u32(smem);
   const uint32_t rt_base = ring + ring_bytes;                           // rt_bufs buffers x 2 boxes of the second factor
@@ -156,6 +159,9 @@ lora_grad_kernel(const __grid_constant__ GradMaps maps, const __grid_constant__ 
             } else if (p.with_p) {
               tma_load_2d(dst + 32768, &tm_a, fb, 0, cc);
               tma_load_2d(dst + 32768 + side_box, &tm_a, fb, 0, cc + 64);
+            } else if (rt_in_stage) {
+              tma_load_2d(dst + 32768, &tm_r, fb, t0, 0);
+              tma_load_2d(dst + 32768 + rt_box, &tm_r, fb, t0 + 64, 0);
             }
           }
           __syncwarp();
@@ -168,7 +174,7 @@ lora_grad_kernel(const __grid_constant__ GradMaps maps, const __grid_constant__ 
     // ================================ loader of the second factor (one 128-token slab at a time) ================================
     bool ok = true;
     int rb = 0, rphase = 0;
-    for (int s = s_begin; s < s_end && ok && p.do_out && !p.debug_no_second_factor; ++s) {
+    for (int s = s_begin; s < s_end && ok && p.do_out && !rt_in_stage && !p.debug_no_second_factor; ++s) {
       ok = warp_wait(rt_empty(rb), rphase ^ 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_EMPTY, false, 20);
       if (ok && elect_one()) {
         const int t0 = s * kGradSlab;
@@ -188,11 +194,12 @@ lora_grad_kernel(const __grid_constant__ GradMaps maps, const __grid_constant__ 
     const uint64_t w_k0 = smem_desc_sw128(ring + 32768, 16, 1024);          // side operand of the stage
     const uint32_t sbox = static_cast<uint32_t>(side_box) >> 4;
     const uint32_t sstep = p.side_mn ? 128u : 2u;                           // descriptor step per 16 features
-    const uint64_t r_k0 = smem_desc_sw128(rt_base, 16, 1024);               // second factor
+    const uint64_t r_k0 = smem_desc_sw128(rt_in_stage ? ring + 32768 : rt_base, 16, 1024);   // second factor
     bool ok = true;
     int slot = 0, phase = 0, rb = 0, rphase = 0, pb = 0, pphase = 0;
     for (int s = s_begin; s < s_end && ok; ++s) {
-      if (p.do_out) ok = warp_wait(rt_full(rb), rphase, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_FULL, false, 0);
+      if (p.do_out && !rt_in_stage)
+        ok = warp_wait(rt_full(rb), rphase, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_FULL, false, 0);
       if (ok && p.with_p)
         ok = warp_wait(p_empty(pb), pphase ^ 1, abort_flag, p.status, p.wait_limit, DEV_TIMEOUT_ACC_EMPTY, false, 0);
       for (int nb = 0; nb < nb_count && ok; ++nb) {
@@ -201,7 +208,7 @@ lora_grad_kernel(const __grid_constant__ GradMaps maps, const __grid_constant__ 
         tc_fence_after();
         if (elect_one()) {
           const uint32_t so = static_cast<uint32_t>(slot * stage_bytes) >> 4;
-          const uint32_t ro = static_cast<uint32_t>(2 * rb * rt_box) >> 4;
+          const uint32_t ro = rt_in_stage ? so : static_cast<uint32_t>(2 * rb * rt_box) >> 4;
           const uint32_t rbox = static_cast<uint32_t>(rt_box) >> 4;
           if (p.do_out) {
 #pragma unroll
@@ -217,7 +224,7 @@ lora_grad_kernel(const __grid_constant__ GradMaps maps, const __grid_constant__ 
           }
           mma_commit(empty_bar(slot));
           if (nb == nb_count - 1) {
-            if (p.do_out) mma_commit(rt_empty(rb));
+            if (p.do_out && !rt_in_stage) mma_commit(rt_empty(rb));
             if (p.with_p) mma_commit(p_full(pb));
           }
         }
@@ -400,8 +407,21 @@ lora_grad_kernel(const __grid_constant__ GradMaps maps, const __grid_constant__ 
 }  // namespace
 
 size_t grad_smem_bytes(const GradParams& p) {
-  const size_t stage = kGradStageBytes + (p.with_p ? 2 * (p.side_mn ? size_t(8192) : static_cast<size_t>(p.r_pad) * 128) : 0);
+  const size_t stage = kGradStageBytes + (p.with_p ? 2 * (p.side_mn ? size_t(8192) : static_cast<size_t>(p.r_pad) * 128) : 0) +
+                       (p.rt_in_stage ? 2 * static_cast<size_t>(p.r_pad) * 128 : 0);
   return static_cast<size_t>(p.stages) * stage + 2 * static_cast<size_t>(p.rt_bufs) * p.r_pad * 128 + kGradTailBytes + 1024;
+}
+
+void grad_set_ring(GradParams* p) {
+  const bool in_stage = p->do_out && !p->with_p && p->feat_chunk == 128 && !p->debug_no_second_factor;
+  p->rt_in_stage = in_stage ? 1 : 0;
+  p->rt_bufs = !p->do_out ? 1 : (in_stage ? 1 : (p->r_pad <= 32 ? 4 : 3));
+  const size_t side_box = p->side_mn ? size_t(8192) : static_cast<size_t>(p->r_pad) * 128;
+  const size_t stage = kGradStageBytes + (p->with_p ? 2 * side_box : 0) + (in_stage ? 2 * static_cast<size_t>(p->r_pad) * 128 : 0);
+  const size_t fixed = 2 * static_cast<size_t>(p->rt_bufs) * p->r_pad * 128 + kGradTailBytes + 1024;
+  int stages = static_cast<int>((232448 - fixed) / stage);
+  if (stages > kGradMaxStages) stages = kGradMaxStages;
+  p->stages = stages < 2 ? 2 : stages;
 }
 
 cudaError_t grad_configure() {
@@ -483,20 +503,18 @@ GradGrid grad_pick_grid_jobs(long long T, const long long* C, int n_jobs, int r_
   }
   const size_t side_box = side_mn ? size_t(8192) : static_cast<size_t>(r_pad) * 128;
   const size_t stage = kGradStageBytes + (with_p ? 2 * side_box : 0);
-  best.stages = grad_stages(r_pad, with_p, side_mn, true);
+  {
+    GradParams t{};
+    t.do_out = 1;
+    t.with_p = with_p ? 1 : 0;
+    t.side_mn = side_mn ? 1 : 0;
+    t.r_pad = r_pad;
+    t.feat_chunk = best.feat_chunk;
+    grad_set_ring(&t);
+    best.stages = t.stages;
+  }
   best.tmem_cols = grad_tmem_cols(best.feat_chunk, r_pad, true, with_p);
   return best;
-}
-
-int grad_rt_bufs(int r_pad, bool do_out) { return !do_out ? 1 : (r_pad <= 32 ? 4 : 3); }
-
-int grad_stages(int r_pad, bool with_p, bool side_mn, bool do_out) {
-  const size_t side_box = side_mn ? size_t(8192) : static_cast<size_t>(r_pad) * 128;
-  const size_t stage = kGradStageBytes + (with_p ? 2 * side_box : 0);
-  const size_t fixed = 2 * static_cast<size_t>(grad_rt_bufs(r_pad, do_out)) * r_pad * 128 + kGradTailBytes + 1024;
-  int stages = static_cast<int>((232448 - fixed) / stage);
-  if (stages > kGradMaxStages) stages = kGradMaxStages;
-  return stages < 2 ? 2 : stages;
 }
 
 int grad_tmem_cols(int feat_chunk, int r_pad, bool do_out, bool with_p) {
@@ -534,9 +552,10 @@ cudaError_t launch_grad_jobs(const GradJobDesc* jobs, int n_jobs, cudaStream_t s
   size_t smem = 0;
   int x = 0;
   for (int j = 0; j < n_jobs; ++j) {
-    const GradParams& p = jobs[j].p;
+    GradParams p = jobs[j].p;
     // all jobs of a launch share the cluster shape: all compute a gradient with the same number of token chunks, or none does
     if (p.do_out != do_out || (do_out && p.n_token_chunks != cluster)) return cudaErrorInvalidValue;
+    grad_set_ring(&p);                    // ring depth, second-factor ring / in-stage slab: one rule for every caller
     L.job[j] = p;
     maps.m[3 * j] = jobs[j].tmS;
     maps.m[3 * j + 1] = jobs[j].tmR;
@@ -675,8 +694,6 @@ extern "C" int lora_grad_contract_noalloc(const void* S, const void* Rt, int64_t
   g.n_feat_chunks = gg.n_feat;
   g.n_token_chunks = gg.n_tok;
   g.n_slabs = static_cast<int>((T + kGradSlab - 1) / kGradSlab);
-  g.stages = gg.stages;
-  g.rt_bufs = grad_rt_bufs(g.r_pad, true);
   g.tmem_cols = gg.tmem_cols;
   g.with_p = 0;
   g.side_mn = 0;

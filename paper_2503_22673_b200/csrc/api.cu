@@ -315,7 +315,13 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c, c
     c->q_feat_chunk = q.feat_chunk;
     c->q_feat_chunks = q.n_feat;
     c->q_token_chunks = q.n_tok;
-    c->q_stages = 4;
+    GradParams t{};
+    t.with_p = 1;
+    t.side_mn = 1;
+    t.r_pad = c->r_pad;
+    t.feat_chunk = q.feat_chunk;
+    grad_set_ring(&t);
+    c->q_stages = t.stages;
   }
   return LORA_OK;
 }
@@ -545,8 +551,6 @@ bool fill_side_job(lora_plan* pl, const void* S, long long C, const void* side, 
   g.n_feat_chunks = sg.n_feat;
   g.n_token_chunks = sg.n_tok;
   g.n_slabs = w.n_slabs;
-  g.stages = grad_stages(c.r_pad, true, side_mn, false);
-  g.rt_bufs = grad_rt_bufs(c.r_pad, false);
   g.tmem_cols = grad_tmem_cols(sg.feat_chunk, c.r_pad, false, true);
   g.with_p = 1;
   g.side_mn = side_mn ? 1 : 0;
@@ -753,8 +757,6 @@ bool fill_da_job(lora_plan* pl, const void* X, const void* A, float scale, void*
   g.n_feat_chunks = ceil_div(s.d_in, feat_chunk);
   g.n_token_chunks = n_tok;
   g.n_slabs = w.n_slabs;
-  g.stages = grad_stages(c.r_pad, with_p, false, true);
-  g.rt_bufs = grad_rt_bufs(c.r_pad, true);
   g.tmem_cols = grad_tmem_cols(feat_chunk, c.r_pad, true, with_p);
   g.with_p = with_p ? 1 : 0;
   g.side_mn = 0;
@@ -795,8 +797,6 @@ bool fill_db_job(lora_plan* pl, const void* dY, float scale, void* dB, const voi
   g.n_feat_chunks = ceil_div(s.d_out, feat_chunk);
   g.n_token_chunks = n_tok;
   g.n_slabs = w.n_slabs;
-  g.stages = grad_stages(c.r_pad, with_q, true, true);
-  g.rt_bufs = grad_rt_bufs(c.r_pad, true);
   g.tmem_cols = grad_tmem_cols(feat_chunk, c.r_pad, true, with_q);
   g.with_p = with_q ? 1 : 0;
   g.side_mn = with_q ? 1 : 0;
@@ -1064,8 +1064,6 @@ bool build_side_job(lora_plan* pl, const void* S, long long C, long long pitch, 
   g.n_feat_chunks = sg.n_feat;
   g.n_token_chunks = sg.n_tok;
   g.n_slabs = pl->ws.n_slabs;
-  g.stages = grad_stages(rows, true, side_mn, false);
-  g.rt_bufs = grad_rt_bufs(rows, false);
   g.tmem_cols = grad_tmem_cols(sg.feat_chunk, rows, false, true);
   g.with_p = 1;
   g.side_mn = side_mn ? 1 : 0;
@@ -1098,8 +1096,6 @@ bool build_grad_job(lora_plan* pl, const void* S, long long C, long long pitch, 
   g.n_feat_chunks = ceil_div(C, feat_chunk);
   g.n_token_chunks = n_tok;
   g.n_slabs = pl->ws.n_slabs;
-  g.stages = grad_stages(kGroupRowsPerJob, false, false, true);     // every job of the launch sizes its ring for the widest
-  g.rt_bufs = grad_rt_bufs(kGroupRowsPerJob, true);
   g.tmem_cols = grad_tmem_cols(feat_chunk, rows, true, false);
   g.do_out = 1;
   g.out_is_da = out_is_da ? 1 : 0;
@@ -1506,8 +1502,6 @@ int lora_debug_starved_wait(lora_plan_t* plan, const void* S, int64_t T, int64_t
   g.n_feat_chunks = 1;
   g.n_token_chunks = 1;              // one CTA, direct mode: nothing but `status` can be written
   g.n_slabs = ceil_div(T, kGradSlab);
-  g.stages = 2;
-  g.rt_bufs = 2;
   g.tmem_cols = grad_tmem_cols(g.feat_chunk, r_pad, true, false);
   g.do_out = 1;
   g.scale = 1.f;

@@ -151,6 +151,7 @@ struct GradParams {
   int n_slabs;
   int stages;
   int rt_bufs;            // depth of the second-factor ring (1 .. kGradMaxRtBufs)
+  int rt_in_stage;        // 1: the second factor's slab travels in each tile's own stage (one-block gradient CTAs)
   int tmem_cols;          // TMEM columns to allocate (power of two >= 32)
   int with_p;             // 1: also accumulate the side product S * side^T for each slab (X A^T, or dY B)
   int side_mn;            // side operand: 0 = A [r, C] (K-major rows), 1 = B [C, r] (MN-major, natural layout)
@@ -186,9 +187,7 @@ void grad_device_caps(int num_sms, int* caps);
 // TMEM columns a launch allocates: gradient sums + side-product buffers, rounded up to a power of two >= 32
 int grad_tmem_cols(int feat_chunk, int r_pad, bool do_out, bool with_p);
 
-// depth of the second-factor ring and of the stream ring that fit 227 KiB of shared memory together
-int grad_rt_bufs(int r_pad, bool do_out);
-int grad_stages(int r_pad, bool with_p, bool side_mn, bool do_out);
+
 
 // One launch of the streaming kernel: up to kGradMaxJobs jobs side by side (CTAs with blockIdx.x in [x_end[j-1], x_end[j])
 // run job j)
@@ -208,6 +207,8 @@ struct GradJobDesc {
 };
 
 size_t grad_smem_bytes(const GradParams& p);
+// ring geometry of a job from its other fields (do_out, with_p, side_mn, r_pad, feat_chunk): sets stages, rt_bufs, rt_in_stage
+void grad_set_ring(GradParams* p);
 // opt in to the large dynamic shared memory and to clusters of more than 8 CTAs (once per device)
 cudaError_t grad_configure();
 // Largest grid (in CTAs) of `cluster`-CTA clusters along y that is resident at once on the current device, for the given

@@ -83,10 +83,24 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
-// One lane polls, the rest of the warp sleeps in the shuffle: waiting warps must not eat the issue slots of
-// the warp that feeds the tensor pipe.  `backoff_ns` > 0 adds a nanosleep between polls (long waits).
+// Whole-warp wait.  Fast path: every lane probes once (one broadcast read of the barrier word, no divergence, no shuffle):
+// a wait that finds its barrier complete costs ~80 cycles instead of ~190, which is what the MMA-issuing warps of the
+// streaming kernel pay per 32 KiB tile.  Slow path: one lane polls, the rest of the warp sleeps in the shuffle, so that
+// waiting warps do not eat the issue slots of the warp that feeds the tensor pipe.  `backoff_ns` > 0 adds a nanosleep
+// between polls (long waits).
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status,
                                           long long limit, unsigned code, bool cluster_scope, unsigned backoff_ns) {
+  {
+    uint32_t r0;
+    if (cluster_scope) {
+      asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+                   "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(r0) : "r"(bar), "r"(parity) : "memory");
+    } else {
+      asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                   "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(r0) : "r"(bar), "r"(parity) : "memory");
+    }
+    if (__all_sync(0xffffffffu, r0 != 0)) return true;
+  }
   int ok = 1;
   if ((threadIdx.x & 31) == 0) {
     auto probe = [&]() {
