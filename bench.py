@@ -33,14 +33,24 @@ import numpy as np
 import torch
 
 L2_BYTES = 126 * 1024 * 1024
+NF4_BAND_BYTES = 16 * 1024 * 1024      # scratch buffer of the banded Q+LoRA variant (the largest weight of the layer is 112 MiB)
 METRIC = "lora_linear_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the ncu captures summarised under profiles/;
-# each entry is valid only for the kernel source it was taken on (sha of the files named in *_source_sha) and for the
-# projection shape it names.  GEMM: dX GEMM of a 32768 x 4096 x 14336 projection; stream: the dA + dB launch of q_proj at
-# T = 32768 (captured at T = 8192 and scaled by the tokens: the traffic is the two streamed matrices, proportional to T).
-NCU_TRAFFIC = {"gemm_sha": "", "gemm_bytes_per_launch": {}, "stream_sha": "", "stream_bytes_per_launch": {}}
+# an entry is valid only for the kernel source it was taken on (source_sha of the GEMM files, of the streaming kernel's) and
+# for the stage and projection shape its key names.  Both captures ran on a smaller token count (the GEMM's at T = 16384, the
+# streaming launches' at T = 8192) and are scaled by the tokens: GEMM traffic is per band of m-tiles and the number of bands
+# grows with T; a streaming launch's traffic is the two streamed matrices, proportional to T.
+NCU_TRAFFIC = {
+    "gemm_sha": "7ffd987e862cc4b4",
+    "gemm_bytes_per_launch": {"32768x14336x4096": 4345182208},       # 2 x (1717.8 + 454.8 MB) captured at T = 16384
+    "stream_sha": "f6480168ab5dc96b",
+    "stream_bytes_per_launch": {                                      # 4 x the launches captured at T = 8192
+        "sides:32768x4096x4096": 552952832, "grads:32768x4096x4096": 554292224,
+        "sides:32768x4096x1024": 349594624, "grads:32768x4096x1024": 347867136,
+        "sides:32768x4096x14336": 1236064256, "grads:32768x4096x14336": 1223135232,
+        "sides:32768x14336x4096": 1240367104, "grads:32768x14336x4096": 1222888448}}
 
 
 def peaks():
@@ -548,16 +558,23 @@ def run_ours(args):
                 if (p.d_out, p.d_in) not in w_scratch:
                     w_scratch[(p.d_out, p.d_in)] = torch.empty((p.d_out, p.d_in), dtype=torch.bfloat16, device=device)
 
+            band = None
+            if all(p.T > 128 for p in protos):
+                band_bytes = max(NF4_BAND_BYTES, max(pl.nf4_scratch_bytes()[0] for pl in plans))
+                band = torch.empty((band_bytes // 2,), dtype=torch.bfloat16, device=device)   # ONE buffer for every projection
+
             def step_nf4(k, scratch):
                 cur, qs = wl.sets[k % wl.n_sets], q_sets[k % wl.n_sets]
                 for j, (proj, d) in enumerate(cur):
-                    ws = w_scratch[(proj.d_out, proj.d_in)] if scratch else None
+                    ws = band if scratch == "band" else w_scratch[(proj.d_out, proj.d_in)] if scratch else None
                     plans[j].fwd_nf4(d["X"], qs[j][0], qs[j][1], d["A"], d["B"], proj.scale, d["Y"], w_scratch=ws)
                     plans[j].bwd_nf4(d["dY"], d["X"], qs[j][0], qs[j][1], d["A"], d["B"], proj.scale, d["dX"], d["dA"], d["dB"],
                                      w_scratch=ws)
 
             forms = [("q_lora_nf4", True, "weight expanded once per call into a bf16 scratch buffer, then the bf16 kernels")]
-            if all(p.T > 128 for p in protos):
+            if band is not None:
+                forms.append(("q_lora_nf4_banded", "band", f"one {band.numel() * 2 >> 20} MiB scratch buffer for all projections: the "
+                              "weight is expanded and multiplied band by band (bands of output features forward, of input features backward)"))
                 forms.append(("q_lora_nf4_in_kernel", False, "no scratch: weight expanded inside the GEMM kernels, per 256-token tile"))
             for key, scratch, how in forms:
                 ms_q = timed_loop(lambda k: step_nf4(k, scratch), n_var, barrier, device, world)
@@ -565,7 +582,7 @@ def run_ours(args):
                                  "tokens_per_s": world * tokens_step / ms_q * 1e3,
                                  "note": "forward + backward with the frozen W in NF4 (4.5 bits per weight); " + how +
                                          "; same algorithmic FLOPs as the bf16 step"}
-            del q_sets, w_scratch
+            del q_sets, w_scratch, band
         # ---- variant: projections that share X (q/k/v, gate/up) through the grouped calls, the others through their own plans ----
         group_ids = {4: [[0, 1, 2], [4, 5]], 5: [[0, 1, 2]]}.get(args.workload, [])
         if group_ids and all(p.r % 16 == 0 for p in protos):

@@ -258,6 +258,12 @@ int lora_dense_dw(lora_plan_t* plan, const void* dY, const void* X, void* dW, vo
  *     afterwards; one buffer can serve every layer of that size): the weight is expanded into it once per call and the
  *     bf16 kernels run on it.  This is the fast form for training batches: each weight element is converted once, not
  *     once per 256-token tile, and the GEMMs keep their shared-memory bandwidth for the tensor cores.
+ *   - w_scratch != NULL but SMALLER than the weight, its size announced with lora_plan_set_nf4_scratch_bytes (below):
+ *     the weight is expanded band by band (forward: bands of output features, i.e. weight rows; backward: bands of
+ *     input features, i.e. weight columns; a band is a whole number of GEMM n-tiles) and the bf16 GEMM runs once per band
+ *     on that band's output columns.  Every element is still converted once per call and the results are bit-identical
+ *     to the whole-weight form (same tiles, same order of summation); a band of a few MB stays in L2 between its
+ *     expansion and the GEMM that reads it.  Costs one expansion launch and one partly filled last wave per band.
  *   - w_scratch == NULL: nothing is materialised; packed codes and scales are staged by TMA and expanded inside the GEMM
  *     kernels, straight into the tensor-core operand tiles.  No extra memory, but the conversion is repeated for every
  *     256-token tile and competes with the tensor cores for shared-memory bandwidth (measured 2-2.5x slower at
@@ -265,6 +271,17 @@ int lora_dense_dw(lora_plan_t* plan, const void* dY, const void* X, void* dW, vo
  * Both forms give bit-identical weights to the GEMMs.  The workspace must be registered (LORA_ERR_WORKSPACE
  * otherwise; forward needs it in the NULL form and whenever the plan's forward uses it).  All pointers are device
  * pointers, 16-byte aligned. */
+/* Size of the buffer behind `w_scratch` in the two Q+LoRA calls of this plan.  lora_plan_nf4_scratch_bytes: `full_bytes` =
+ * d_out * d_in * 2 (the whole weight, the default assumption), `min_bytes` = the smallest buffer the banded form accepts
+ * (one n-tile of weight rows or columns: max(fwd_block_n * d_in, dx_block_n * d_out) * 2 bytes).
+ * lora_plan_set_nf4_scratch_bytes: 0 or anything >= full_bytes selects the whole-weight form; a smaller value the banded
+ * form, which needs a plan with T > 128 whose selector did not split the contraction (LORA_ERR_UNSUPPORTED_SHAPE otherwise)
+ * and bytes >= min_bytes (LORA_ERR_WORKSPACE otherwise).  The library picks the band height from the size (as many n-tiles
+ * as fit, fewer when that leaves fewer idle CTA pairs in the bands' last waves).  Host-side setting, not thread-safe
+ * against concurrent calls on the same plan. */
+int lora_plan_nf4_scratch_bytes(const lora_plan_t* plan, size_t* min_bytes, size_t* full_bytes);
+int lora_plan_set_nf4_scratch_bytes(lora_plan_t* plan, size_t bytes);
+
 int lora_nf4_quantize(const void* W, int64_t d_out, int64_t d_in, void* W_codes, void* W_absmax, void* stream);
 int lora_nf4_dequantize(const void* W_codes, const void* W_absmax, int64_t d_out, int64_t d_in, void* W, void* stream);
 int lora_linear_fwd_nf4(lora_plan_t* plan, const void* X, const void* W_codes, const void* W_absmax, const void* A,

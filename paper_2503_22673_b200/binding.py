@@ -32,6 +32,7 @@ EXPORTS = [
     "lora_grad_contract_noalloc", "lora_grad_contract_noalloc_max_scratch", "lora_grad_contract_noalloc_status",
     "lora_plan_set_wait_limit", "lora_debug_starved_wait", "lora_linear_bwd_sides", "lora_linear_bwd_grads",
     "lora_plan_last_gemm_clock", "lora_plan_create_grouped", "lora_linear_fwd_grouped", "lora_linear_bwd_grouped",
+    "lora_plan_nf4_scratch_bytes", "lora_plan_set_nf4_scratch_bytes",
 ]
 
 
@@ -107,6 +108,8 @@ def load(rebuild: bool = False) -> ctypes.CDLL:
     lib.lora_plan_set_wait_limit.argtypes = [vp, i64]
     lib.lora_plan_last_gemm_clock.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
     lib.lora_debug_starved_wait.argtypes = [vp, vp, i64, i64, vp, vp]
+    lib.lora_plan_nf4_scratch_bytes.argtypes = [vp, sz_p, sz_p]
+    lib.lora_plan_set_nf4_scratch_bytes.argtypes = [vp, ctypes.c_size_t]
     lib.lora_grad_contract_noalloc_max_scratch.argtypes = []
     lib.lora_grad_contract_noalloc_max_scratch.restype = i64
     for name in EXPORTS:
@@ -286,17 +289,28 @@ class LoraLinearPlan:
         return dX, dA, dB
 
     # -- NF4 frozen weight (Q+LoRA) ---------------------------------------------------------------
+    def nf4_scratch_bytes(self) -> Tuple[int, int]:
+        """(smallest scratch buffer the banded Q+LoRA form accepts, size of the whole bf16 weight), in bytes."""
+        lo, full = ctypes.c_size_t(0), ctypes.c_size_t(0)
+        _check(self._lib.lora_plan_nf4_scratch_bytes(self._h, ctypes.byref(lo), ctypes.byref(full)), "lora_plan_nf4_scratch_bytes")
+        return int(lo.value), int(full.value)
+
     def _scratch_ptr(self, w_scratch):
+        """Pointer of the scratch buffer; its size is announced to the plan (a buffer smaller than the weight selects the
+        banded form: any contiguous bf16 tensor of at least nf4_scratch_bytes()[0] bytes)."""
         if w_scratch is None:
             return ctypes.c_void_p(0)
-        _want(w_scratch, "w_scratch", (self.d_out, self.d_in), torch.bfloat16, self.device)
+        if w_scratch.dtype != torch.bfloat16 or w_scratch.device != self.device or not w_scratch.is_contiguous():
+            raise ValueError("w_scratch: want a contiguous bf16 tensor on the plan's device")
+        _check(self._lib.lora_plan_set_nf4_scratch_bytes(self._h, w_scratch.numel() * 2), "lora_plan_set_nf4_scratch_bytes")
         return _ptr(w_scratch)
 
     def fwd_nf4(self, X, W_codes, W_absmax, A, B, scale: float, Y: Optional[torch.Tensor] = None, w_scratch=None, stream=None):
         """Y = X w_hat^T + scale (X A^T) B^T with w_hat = the NF4 weight (codes [d_out, d_in/2] uint8, absmax [d_in/64, d_out] fp32).
 
         ``w_scratch`` ([d_out, d_in] bf16, reusable across layers): expand the weight once and run the bf16 kernels (fast
-        form); None: expand inside the GEMM kernels (no extra memory, slower for large batches)."""
+        form); a smaller bf16 buffer (see ``nf4_scratch_bytes``): the same band by band; None: expand inside the GEMM
+        kernels (no extra memory, slower for large batches)."""
         bf = torch.bfloat16
         _want(X, "X", (self.T, self.d_in), bf, self.device)
         _want(W_codes, "W_codes", (self.d_out, self.d_in // 2), torch.uint8, self.device)

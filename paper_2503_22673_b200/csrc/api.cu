@@ -107,7 +107,9 @@ SideGrid pick_side_grid(long long T, long long C, int ctas) {
     int n_tok = ctas / n_feat;
     if (n_tok > n_slabs) n_tok = n_slabs;
     if (n_tok < 1) n_tok = 1;
-    const double cost = static_cast<double>(ceil_div(n_slabs, n_tok)) * (fc + (n_feat > 1 ? 64 : 0));
+    // a split pays per slab for the partial sums (fp32 write, fence, arrival counter, last-arriver sum): measured on the
+    // 32768 x 4096 stream beside a 1024-wide one, 1 chunk x 3 slabs per CTA 58.0 us against 4 chunks x 9 slabs 64.0 us
+    const double cost = static_cast<double>(ceil_div(n_slabs, n_tok)) * (fc + (n_feat > 1 ? 512 : 0));
     if (cost < best_cost * 0.97) {        // a split must pay for itself by a clear margin
       best_cost = cost;
       best_nf = nf;
@@ -460,6 +462,7 @@ struct lora_plan {
   bool p_saved;          // the workspace holds Pt = s (X A^T)^T of the last forward call
   float p_saved_scale;
   long long wait_limit;  // SM clock ticks after which a device-side spin gives up (lora_plan_set_wait_limit)
+  size_t nf4_scratch_bytes;   // bytes behind the w_scratch of the Q+LoRA calls; 0 = the whole weight (lora_plan_set_nf4_scratch_bytes)
   // grouped projections (lora_plan_create_grouped): G projections that share X; shape.d_out is the sum of their widths
   int n_groups;          // 0: an ordinary plan
   long long group_off[5];   // first output column of every group, and the total
@@ -600,8 +603,16 @@ int launch_side_pair(lora_plan* pl, const void* dY, const void* B, const void* X
   return LORA_OK;
 }
 
+// A window of the GEMM's output columns: columns [off, off + n) of Y (forward: output features, W = the n weight rows of the
+// window, row pitch d_in) or of dX (backward: input features, W = the window's n columns of every weight row, row pitch n).
+// The banded Q+LoRA calls run one GEMM launch per window; `first` = the launch that also runs the skinny pre-pass.
+struct ColWindow {
+  long long off, n;
+  bool first;
+};
+
 int launch_fwd(lora_plan* pl, const void* X, const void* W, const void* A, const void* B, float scale, void* Y,
-               cudaStream_t st) {
+               cudaStream_t st, const ColWindow* win = nullptr) {
   const lora_shape_t& s = pl->shape;
   const lora_kernel_config_t& c = pl->cfg;
   const bool pair = c.cta_group == 2;
@@ -609,30 +620,35 @@ int launch_fwd(lora_plan* pl, const void* X, const void* W, const void* A, const
   const bool have_ws = pl->workspace != nullptr && pl->workspace_bytes >= pl->ws.total;
   if (ext && !have_ws) return LORA_ERR_WORKSPACE;
   __nv_bfloat16* pt = have_ws ? ws_ptrs(pl).pt : nullptr;
-  if (ext) {
+  if (ext && (win == nullptr || win->first)) {
     const int rc = launch_side_prepass(pl, X, s.d_in, A, false, scale, pt, st);   // Pt = s (X A^T)^T
     if (rc != LORA_OK) return rc;
+  }
+  const long long n_out = win ? win->n : s.d_out;            // output columns of this launch
+  if (win) {                                                   // W already points at the window's rows
+    B = static_cast<const __nv_bfloat16*>(B) + win->off * s.r;
+    Y = static_cast<__nv_bfloat16*>(Y) + win->off;
   }
   const int half = (c.fwd_block_n + c.r_pad) / 2;
   CUtensorMap tmX, tmW, tmW1, tmA, tmB, tmY;
   bool ok = make_bf16_tmap(&tmX, X, s.d_in, s.T, s.d_in, 64, kBlockM);
-  ok = ok && make_bf16_tmap(&tmW, W, s.d_in, s.d_out, s.d_in, 64, ext ? c.fwd_block_n / 2 : pair ? half : c.fwd_block_n);
-  if (pair && !ext) ok = ok && make_bf16_tmap(&tmW1, W, s.d_in, s.d_out, s.d_in, 64, c.fwd_block_n - half);
+  ok = ok && make_bf16_tmap(&tmW, W, s.d_in, n_out, s.d_in, 64, ext ? c.fwd_block_n / 2 : pair ? half : c.fwd_block_n);
+  if (pair && !ext) ok = ok && make_bf16_tmap(&tmW1, W, s.d_in, n_out, s.d_in, 64, c.fwd_block_n - half);
   if (ext) ok = ok && make_bf16_tmap(&tmA, pt, s.T, c.r_pad, pl->ws.ld_t, 64, c.r_pad);
   else ok = ok && make_bf16_tmap(&tmA, A, s.d_in, s.r, s.d_in, 64, c.r_pad);
-  ok = ok && make_bf16_tmap(&tmB, B, s.r, s.d_out, s.r, 64, pair ? c.fwd_block_n / 2 : c.fwd_block_n);
-  ok = ok && make_bf16_tmap(&tmY, Y, s.d_out, s.T, s.d_out, 64, kBlockM);
+  ok = ok && make_bf16_tmap(&tmB, B, s.r, n_out, s.r, 64, pair ? c.fwd_block_n / 2 : c.fwd_block_n);
+  ok = ok && make_bf16_tmap(&tmY, Y, n_out, s.T, s.d_out, 64, kBlockM);
   if (!ok) return LORA_ERR_CUDA;
   GemmParams p{};
   p.out = static_cast<__nv_bfloat16*>(Y);
   p.ld_out = static_cast<int>(s.d_out);
   p.M = static_cast<int>(s.T);
-  p.N = static_cast<int>(s.d_out);
+  p.N = static_cast<int>(n_out);
   p.K = static_cast<int>(s.d_in);
   p.r_pad = c.r_pad;
   p.block_n = c.fwd_block_n;
   p.tiles_m = ceil_div(s.T, c.block_m);
-  p.tiles_n = ceil_div(s.d_out, c.fwd_block_n);
+  p.tiles_n = ceil_div(n_out, c.fwd_block_n);
   p.num_tiles = p.tiles_m * p.tiles_n;
   p.kblocks = ceil_div(s.d_in, kBlockK);
   p.group_m = c.group_m;
@@ -650,9 +666,12 @@ int launch_fwd(lora_plan* pl, const void* X, const void* W, const void* A, const
   p.status = pl->d_status;
     p.wait_limit = pl->wait_limit;
     p.tail_parts = 1;
-  const cudaError_t le = ext    ? launch_gemm_pair_fwd_ext(tmX, tmW, tmA, tmB, tmY, p, c.fwd_ctas, st)
-                         : pair ? launch_gemm_pair_fwd(tmX, tmW, tmW1, tmA, tmB, tmY, p, c.fwd_ctas, st)
-                                : launch_gemm_fwd(tmX, tmW, tmA, tmB, tmY, p, c.fwd_ctas, st);
+  if (win && p.split_k > 1) return LORA_ERR_UNSUPPORTED_SHAPE;   // the split-K reduction writes whole contiguous outputs
+  int fwd_ctas = c.fwd_ctas;
+  if (win && pair && fwd_ctas > 2 * p.num_tiles) fwd_ctas = 2 * p.num_tiles;
+  const cudaError_t le = ext    ? launch_gemm_pair_fwd_ext(tmX, tmW, tmA, tmB, tmY, p, fwd_ctas, st)
+                         : pair ? launch_gemm_pair_fwd(tmX, tmW, tmW1, tmA, tmB, tmY, p, fwd_ctas, st)
+                                : launch_gemm_fwd(tmX, tmW, tmA, tmB, tmY, p, fwd_ctas, st);
   if (le != cudaSuccess) return LORA_ERR_CUDA;
   g_launches.fetch_add(1);
   if (p.split_k > 1) {
@@ -668,13 +687,19 @@ int launch_fwd(lora_plan* pl, const void* X, const void* W, const void* A, const
 
 // ---- dX = dY W + s (dY B) A ; also leaves Qt = s (dY B)^T in the workspace ----
 int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const void* B, float scale, void* dX,
-              cudaStream_t st, int ctas_override = 0) {
+              cudaStream_t st, int ctas_override = 0, const ColWindow* win = nullptr) {
   const lora_shape_t& s = pl->shape;
   const lora_kernel_config_t& c = pl->cfg;
   const WsLayout& w = pl->ws;
   const WsPtrs q = ws_ptrs(pl);
   __nv_bfloat16* qt = q.qt;
-  if (c.cta_group == 2 && !pl->q_ready) {
+  const long long n_in = win ? win->n : s.d_in;              // input features (columns of dX) of this launch
+  const long long ld_w = win ? win->n : s.d_in;              // a window's weight columns are stored densely
+  if (win) {
+    A = static_cast<const __nv_bfloat16*>(A) + win->off;
+    dX = static_cast<__nv_bfloat16*>(dX) + win->off;
+  }
+  if (c.cta_group == 2 && !pl->q_ready && (win == nullptr || win->first)) {
     // ---- pre-pass: Qt = s (dY B)^T, dY streamed once by the skinny kernel (side product only) ----
     const int rc = launch_side_prepass(pl, dY, s.d_out, B, true, scale, qt, st);
     if (rc != LORA_OK) return rc;
@@ -682,23 +707,23 @@ int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const
   {
     CUtensorMap tmdY, tmW, tmB, tmA, tmdX;
     bool ok = make_bf16_tmap(&tmdY, dY, s.d_out, s.T, s.d_out, 64, kBlockM);
-    ok = ok && make_bf16_tmap(&tmW, W, s.d_in, s.d_out, s.d_in, 64, 64);
+    ok = ok && make_bf16_tmap(&tmW, W, n_in, s.d_out, ld_w, 64, 64);
     const bool pair = c.cta_group == 2;
-    if (pair) ok = ok && make_bf16_tmap(&tmB, qt, s.T, c.r_pad, w.ld_t, 64, c.r_pad);   // Qt from the pre-pass below
+    if (pair) ok = ok && make_bf16_tmap(&tmB, qt, s.T, c.r_pad, w.ld_t, 64, c.r_pad);   // Qt from the pre-pass above
     else ok = ok && make_bf16_tmap(&tmB, B, s.r, s.d_out, s.r, 64, 64);
-    ok = ok && make_bf16_tmap(&tmA, A, s.d_in, s.r, s.d_in, 64, c.r_pad);
-    ok = ok && make_bf16_tmap(&tmdX, dX, s.d_in, s.T, s.d_in, 64, kBlockM);
+    ok = ok && make_bf16_tmap(&tmA, A, n_in, s.r, s.d_in, 64, c.r_pad);
+    ok = ok && make_bf16_tmap(&tmdX, dX, n_in, s.T, s.d_in, 64, kBlockM);
     if (!ok) return LORA_ERR_CUDA;
     GemmParams p{};
     p.out = static_cast<__nv_bfloat16*>(dX);
     p.ld_out = static_cast<int>(s.d_in);
     p.M = static_cast<int>(s.T);
-    p.N = static_cast<int>(s.d_in);
+    p.N = static_cast<int>(n_in);
     p.K = static_cast<int>(s.d_out);
     p.r_pad = c.r_pad;
     p.block_n = c.dx_block_n;
     p.tiles_m = ceil_div(s.T, c.block_m);
-    p.tiles_n = ceil_div(s.d_in, c.dx_block_n);
+    p.tiles_n = ceil_div(n_in, c.dx_block_n);
     p.num_tiles = p.tiles_m * p.tiles_n;
     p.kblocks = ceil_div(s.d_out, kBlockK);
     p.group_m = c.group_m;
@@ -715,7 +740,9 @@ int launch_dx(lora_plan* pl, const void* dY, const void* W, const void* A, const
     p.status = pl->d_status;
     p.wait_limit = pl->wait_limit;
     p.tail_parts = 1;
-    const int ctas = ctas_override > 0 ? ctas_override : c.dx_ctas;
+    if (win && (p.split_k > 1 || !pair)) return LORA_ERR_UNSUPPORTED_SHAPE;
+    int ctas = ctas_override > 0 ? ctas_override : c.dx_ctas;
+    if (win && ctas > 2 * p.num_tiles) ctas = 2 * p.num_tiles;
     const cudaError_t le = pair ? launch_gemm_pair_dx(tmdY, tmW, tmB, tmA, tmdX, p, ctas, st)
                                 : launch_gemm_dx(tmdY, tmW, tmB, tmA, tmdX, p, ctas, st);
     if (le != cudaSuccess) return LORA_ERR_CUDA;
@@ -994,6 +1021,87 @@ int check_nf4(const lora_plan* pl) {
   if (pl->cfg.cta_group != 2) return LORA_ERR_UNSUPPORTED_SHAPE;          // batches of at most 128 tokens: not covered
   if (pl->shape.d_in % kNf4Block != 0) return LORA_ERR_UNSUPPORTED_SHAPE;
   if (pl->workspace == nullptr || pl->workspace_bytes < pl->ws.total) return LORA_ERR_WORKSPACE;
+  return LORA_OK;
+}
+
+// ---- Q+LoRA with a scratch buffer smaller than the weight: the weight is expanded band by band ----
+// Forward: bands of output features (weight rows), each a whole number of n-tiles; backward: bands of input features (weight
+// columns).  Every band is expanded into the scratch buffer and fed to the bf16 GEMM restricted to that band's output
+// columns, so each weight element is still converted once per call and the tiles, their k-order and hence the results are
+// those of the whole-weight scratch form.  A band of a few MB stays in L2 between its expansion and the GEMM that reads it.
+size_t nf4_full_bytes(const lora_plan* pl) { return static_cast<size_t>(pl->shape.d_out) * pl->shape.d_in * 2; }
+
+size_t nf4_min_bytes(const lora_plan* pl) {
+  const size_t f = static_cast<size_t>(pl->cfg.fwd_block_n) * pl->shape.d_in * 2;
+  const size_t b = static_cast<size_t>(pl->cfg.dx_block_n) * pl->shape.d_out * 2;
+  return f > b ? f : b;
+}
+
+bool nf4_banded(const lora_plan* pl) { return pl->nf4_scratch_bytes != 0 && pl->nf4_scratch_bytes < nf4_full_bytes(pl); }
+
+// n-tiles per band: as many as fit `max_tiles`, among those the count with the fewest modelled waves over the whole GEMM (every
+// band ends in a partly filled wave of CTA pairs and pays one expansion launch)
+long long nf4_band_tiles(long long tiles_m, long long tiles_n, long long max_tiles, int pairs) {
+  if (max_tiles >= tiles_n) return tiles_n;
+  long long best = 1;
+  double best_cost = 0;
+  for (long long k = 1; k <= max_tiles; ++k) {
+    const long long full = tiles_n / k, rest = tiles_n - full * k;
+    double cost = static_cast<double>(full) * (static_cast<double>(ceil_div(tiles_m * k, pairs)) + 0.3);
+    if (rest) cost += static_cast<double>(ceil_div(tiles_m * rest, pairs)) + 0.3;
+    if (k == 1 || cost <= best_cost) {
+      best = k;
+      best_cost = cost;
+    }
+  }
+  return best;
+}
+
+int check_nf4_banded(const lora_plan* pl) {
+  const lora_kernel_config_t& c = pl->cfg;
+  if (c.cta_group != 2 || c.split_k != 1 || c.dx_split_k != 1) return LORA_ERR_UNSUPPORTED_SHAPE;   // needs the whole-weight scratch
+  if (pl->nf4_scratch_bytes < nf4_min_bytes(pl)) return LORA_ERR_WORKSPACE;
+  if (pl->workspace == nullptr || pl->workspace_bytes < pl->ws.total) return LORA_ERR_WORKSPACE;
+  return LORA_OK;
+}
+
+int launch_fwd_nf4_banded(lora_plan* pl, const void* X, const void* codes, const void* absmax, const void* A, const void* B,
+                          float scale, void* Y, void* scratch, cudaStream_t st) {
+  const lora_shape_t& s = pl->shape;
+  const lora_kernel_config_t& c = pl->cfg;
+  const long long bn = c.fwd_block_n;
+  const long long max_tiles = static_cast<long long>(pl->nf4_scratch_bytes / (2 * static_cast<size_t>(s.d_in))) / bn;
+  const long long rows = bn * nf4_band_tiles(ceil_div(s.T, c.block_m), ceil_div(s.d_out, bn), max_tiles, pl->num_sms / 2);
+  for (long long off = 0; off < s.d_out; off += rows) {
+    const long long n = s.d_out - off < rows ? s.d_out - off : rows;
+    if (launch_nf4_dequantize_window(static_cast<const uint8_t*>(codes), static_cast<const float*>(absmax), s.d_out, s.d_in, off,
+                                     n, 0, s.d_in, static_cast<__nv_bfloat16*>(scratch), s.d_in, pl->num_sms, st) != cudaSuccess)
+      return LORA_ERR_CUDA;
+    g_launches.fetch_add(1);
+    const ColWindow win{off, n, off == 0};
+    const int rc = launch_fwd(pl, X, scratch, A, B, scale, Y, st, &win);
+    if (rc != LORA_OK) return rc;
+  }
+  return LORA_OK;
+}
+
+int launch_dx_nf4_banded(lora_plan* pl, const void* dY, const void* codes, const void* absmax, const void* A, const void* B,
+                         float scale, void* dX, void* scratch, cudaStream_t st) {
+  const lora_shape_t& s = pl->shape;
+  const lora_kernel_config_t& c = pl->cfg;
+  const long long bn = c.dx_block_n;
+  const long long max_tiles = static_cast<long long>(pl->nf4_scratch_bytes / (2 * static_cast<size_t>(s.d_out))) / bn;
+  const long long cols = bn * nf4_band_tiles(ceil_div(s.T, c.block_m), ceil_div(s.d_in, bn), max_tiles, pl->num_sms / 2);
+  for (long long off = 0; off < s.d_in; off += cols) {
+    const long long n = s.d_in - off < cols ? s.d_in - off : cols;
+    if (launch_nf4_dequantize_window(static_cast<const uint8_t*>(codes), static_cast<const float*>(absmax), s.d_out, s.d_in, 0,
+                                     s.d_out, off, n, static_cast<__nv_bfloat16*>(scratch), n, pl->num_sms, st) != cudaSuccess)
+      return LORA_ERR_CUDA;
+    g_launches.fetch_add(1);
+    const ColWindow win{off, n, off == 0};
+    const int rc = launch_dx(pl, dY, scratch, A, B, scale, dX, st, 0, &win);
+    if (rc != LORA_OK) return rc;
+  }
   return LORA_OK;
 }
 
@@ -1727,6 +1835,11 @@ int lora_linear_fwd_nf4(lora_plan_t* plan, const void* X, const void* W_codes, c
   if (plan->shape.d_in % kNf4Block != 0 || plan->shape.d_out % 4 != 0) return LORA_ERR_UNSUPPORTED_SHAPE;
   DeviceGuard guard(plan->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (w_scratch != nullptr && nf4_banded(plan)) {
+    const int rcb = check_nf4_banded(plan);
+    if (rcb != LORA_OK) return rcb;
+    return launch_fwd_nf4_banded(plan, X, W_codes, W_absmax, A, B, scale, Y, w_scratch, st);
+  }
   if (w_scratch != nullptr) {
     // expand once, then the bf16 path: every weight element is converted once per call instead of once per 256-token tile
     if (launch_nf4_dequantize(static_cast<const uint8_t*>(W_codes), static_cast<const float*>(W_absmax), plan->shape.d_out,
@@ -1761,6 +1874,19 @@ int lora_linear_bwd_nf4(lora_plan_t* plan, const void* dY, const void* X, const 
     return LORA_ERR_MISALIGNED;
   plan->q_staged = false;
   if (plan->shape.d_in % kNf4Block != 0 || plan->shape.d_out % 4 != 0) return LORA_ERR_UNSUPPORTED_SHAPE;
+  if (w_scratch != nullptr && nf4_banded(plan)) {
+    int rcb = check_nf4_banded(plan);
+    if (rcb != LORA_OK) return rcb;
+    bool p_ready = false;
+    if (plan->cfg.bwd_merged) {
+      rcb = launch_side_pair(plan, dY, B, X, A, scale, st);
+      plan->q_ready = p_ready = true;
+    }
+    if (rcb == LORA_OK) rcb = launch_dx_nf4_banded(plan, dY, W_codes, W_absmax, A, B, scale, dX, w_scratch, st);
+    plan->q_ready = false;
+    if (rcb == LORA_OK) rcb = launch_adapter_grads(plan, dY, X, A, scale, dA, dB, p_ready, st);
+    return rcb;
+  }
   if (w_scratch != nullptr) {
     if (plan->workspace == nullptr || plan->workspace_bytes < plan->ws.total) return LORA_ERR_WORKSPACE;
     if (launch_nf4_dequantize(static_cast<const uint8_t*>(W_codes), static_cast<const float*>(W_absmax), plan->shape.d_out,
@@ -1789,6 +1915,24 @@ int lora_linear_bwd_nf4(lora_plan_t* plan, const void* dY, const void* X, const 
   plan->q_ready = false;
   if (rc == LORA_OK) rc = launch_adapter_grads(plan, dY, X, A, scale, dA, dB, p_ready, st);
   return rc;
+}
+
+int lora_plan_nf4_scratch_bytes(const lora_plan_t* plan, size_t* min_bytes, size_t* full_bytes) {
+  if (plan == nullptr || plan->n_groups != 0) return LORA_ERR_INVALID_ARG;
+  if (min_bytes) *min_bytes = nf4_min_bytes(plan);
+  if (full_bytes) *full_bytes = nf4_full_bytes(plan);
+  return LORA_OK;
+}
+
+int lora_plan_set_nf4_scratch_bytes(lora_plan_t* plan, size_t bytes) {
+  if (plan == nullptr || plan->n_groups != 0) return LORA_ERR_INVALID_ARG;
+  if (bytes != 0 && bytes < nf4_full_bytes(plan)) {
+    const lora_kernel_config_t& c = plan->cfg;
+    if (c.cta_group != 2 || c.split_k != 1 || c.dx_split_k != 1) return LORA_ERR_UNSUPPORTED_SHAPE;
+    if (bytes < nf4_min_bytes(plan)) return LORA_ERR_WORKSPACE;
+  }
+  plan->nf4_scratch_bytes = bytes;
+  return LORA_OK;
 }
 
 int lora_dense_dw(lora_plan_t* plan, const void* dY, const void* X, void* dW, void* stream) {

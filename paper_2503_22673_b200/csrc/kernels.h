@@ -116,6 +116,11 @@ cudaError_t launch_nf4_quantize(const __nv_bfloat16* W, long long d_out, long lo
 // NF4 codes + block scales -> bf16 weight [d_out, d_in], every element bf16(level * absmax) (nf4_quant.cu)
 cudaError_t launch_nf4_dequantize(const uint8_t* codes, const float* absmax, long long d_out, long long d_in, __nv_bfloat16* W,
                                   int num_sms, cudaStream_t stream);
+// the same for the window rows [o0, o0 + n_rows) x columns [c0, c0 + n_cols) of the weight (c0, n_cols, ld_w multiples of 8:
+// a thread expands one 32-bit code word into 16 bytes), written to W with a row pitch of ld_w elements
+cudaError_t launch_nf4_dequantize_window(const uint8_t* codes, const float* absmax, long long d_out, long long d_in, long long o0,
+                                         long long n_rows, long long c0, long long n_cols, __nv_bfloat16* W, long long ld_w,
+                                         int num_sms, cudaStream_t stream);
 
 // dense weight gradient dW[d_out, d_in] = dY^T X (p.r_pad = 0: no rank-r k-block): tmdYt = dY [T, d_out] box 64(o) x 64(t),
 // tmX = X [T, d_in] box 64(i) x 64(t), tmdW box 64 x 128; p.M = d_out, p.N = d_in, p.K = T

@@ -53,20 +53,26 @@ __global__ void __launch_bounds__(256) lora_nf4_quantize_kernel(const __nv_bfloa
   if (lane == 0) absmax[b * d_out + o] = m;
 }
 
+// Expands the window rows [o0, o0 + n_rows) x columns [c0, c0 + n_cols) of the quantised weight into W (row pitch ld_w
+// elements, row 0 / column 0 of W = weight element (o0, c0)); the whole weight is the window (0, d_out, 0, d_in).
 __global__ void __launch_bounds__(256) lora_nf4_dequantize_kernel(const uint32_t* __restrict__ codes, const float* __restrict__ absmax,
-                                                                  long long d_out, long long d_in, uint4* __restrict__ W) {
+                                                                  long long d_out, long long d_in, long long o0, long long n_rows,
+                                                                  long long c0, long long n_cols, long long ld_w,
+                                                                  __nv_bfloat16* __restrict__ W) {
   __shared__ float lut[16 * 32];
   pdl_launch_dependents();
   for (int b = threadIdx.x; b < 16 * 32; b += blockDim.x) lut[b] = c_nf4_quant_levels[b >> 5];
   __syncthreads();
   pdl_wait();
   const float* lut_lane = lut + (threadIdx.x & 31);
-  const int words_row = static_cast<int>(d_in / 8);            // 4 code bytes = 8 elements per thread and step
+  const long long words_full = d_in / 8;                        // code words of a whole weight row
+  const int words_row = static_cast<int>(n_cols / 8);           // 4 code bytes = 8 elements per thread and step
+  const long long word0 = c0 / 8;
   // a block walks whole rows (no index division); a thread fetches up to four code words (t, t + 256, ...) and their
   // scales before it converts any of them, so that four loads per thread are in flight
-  for (long long o = blockIdx.x; o < d_out; o += gridDim.x) {
-    const uint32_t* crow = codes + o * words_row;
-    uint4* wrow = W + o * words_row;
+  for (long long o = blockIdx.x; o < n_rows; o += gridDim.x) {
+    const uint32_t* crow = codes + (o0 + o) * words_full + word0;
+    uint4* wrow = reinterpret_cast<uint4*>(W + o * ld_w);
     for (int base = 0; base < words_row; base += 4 * blockDim.x) {
       uint32_t cw[4];
       float scale[4];
@@ -74,7 +80,7 @@ __global__ void __launch_bounds__(256) lora_nf4_dequantize_kernel(const uint32_t
       for (int k = 0; k < 4; ++k) {
         const int wcol = base + k * blockDim.x + threadIdx.x;
         cw[k] = wcol < words_row ? __ldg(crow + wcol) : 0u;
-        scale[k] = wcol < words_row ? __ldg(absmax + static_cast<long long>(wcol >> 3) * d_out + o) : 0.f;   // 8 words = one block
+        scale[k] = wcol < words_row ? __ldg(absmax + ((word0 + wcol) >> 3) * d_out + o0 + o) : 0.f;   // 8 words = one block
       }
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
@@ -95,13 +101,19 @@ __global__ void __launch_bounds__(256) lora_nf4_dequantize_kernel(const uint32_t
 
 }  // namespace
 
-cudaError_t launch_nf4_dequantize(const uint8_t* codes, const float* absmax, long long d_out, long long d_in, __nv_bfloat16* W,
-                                  int num_sms, cudaStream_t stream) {
-  long long blocks = d_out;
+cudaError_t launch_nf4_dequantize_window(const uint8_t* codes, const float* absmax, long long d_out, long long d_in, long long o0,
+                                         long long n_rows, long long c0, long long n_cols, __nv_bfloat16* W, long long ld_w,
+                                         int num_sms, cudaStream_t stream) {
+  long long blocks = n_rows;
   const long long cap = static_cast<long long>(num_sms > 0 ? num_sms : 148) * 16;
   if (blocks > cap) blocks = cap;
   return launch_pdl(lora_nf4_dequantize_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, stream,
-                    reinterpret_cast<const uint32_t*>(codes), absmax, d_out, d_in, reinterpret_cast<uint4*>(W));
+                    reinterpret_cast<const uint32_t*>(codes), absmax, d_out, d_in, o0, n_rows, c0, n_cols, ld_w, W);
+}
+
+cudaError_t launch_nf4_dequantize(const uint8_t* codes, const float* absmax, long long d_out, long long d_in, __nv_bfloat16* W,
+                                  int num_sms, cudaStream_t stream) {
+  return launch_nf4_dequantize_window(codes, absmax, d_out, d_in, 0, d_out, 0, d_in, W, d_in, num_sms, stream);
 }
 
 cudaError_t launch_nf4_quantize(const __nv_bfloat16* W, long long d_out, long long d_in, uint8_t* codes, float* absmax,

@@ -166,7 +166,7 @@ def test_dense_dw_full_size_sampled(idx):
     torch.cuda.empty_cache()
 
 
-@pytest.mark.parametrize("use_scratch", [True, False], ids=["scratch", "in_kernel"])
+@pytest.mark.parametrize("use_scratch", [True, "band", False], ids=["scratch", "banded_8MiB", "in_kernel"])
 def test_nf4_full_size_config1(use_scratch):
     """Q+LoRA at the q_proj size (T = 8192, 4096 -> 4096, r = 16): the GPU quantiser's codes and scales must equal the
     oracle's bit for bit; Y and dX on two rows of every 128-row slab and dA, dB in full against the oracle on the dequantised weight."""
@@ -178,6 +178,8 @@ def test_nf4_full_size_config1(use_scratch):
     assert np.array_equal(codes.cpu().numpy(), ref_codes) and np.array_equal(absmax.cpu().numpy(), ref_absmax)
     plan = binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r)
     scratch = torch.empty((p.d_out, p.d_in), dtype=torch.bfloat16, device="cuda") if use_scratch else None
+    if use_scratch == "band":                          # a quarter of the 32 MiB weight: four bands each way
+        scratch = torch.empty((4 << 20,), dtype=torch.bfloat16, device="cuda")
     Y = plan.fwd_nf4(d["X"], codes, absmax, d["A"], d["B"], p.scale, w_scratch=scratch)
     dX, dA, dB = plan.bwd_nf4(d["dY"], d["X"], codes, absmax, d["A"], d["B"], p.scale, w_scratch=scratch)
     code, msg = plan.device_status()

@@ -65,7 +65,8 @@ def test_dequantiser_is_bit_exact():
     assert np.array_equal(host64(got), nf4.dequantize(codes, absmax))
 
 
-def run_nf4_layer(p, t, codes, absmax, use_scratch=False):
+def run_nf4_layer(p, t, codes, absmax, use_scratch=False, band_tiles=0):
+    """band_tiles > 0: the scratch buffer holds that many n-tiles of the smallest band the plan accepts (banded form)."""
     d = {k: dev(t[k]) for k in ("X", "A", "B", "dY")}
     cd, ad = torch.from_numpy(codes).cuda(), torch.from_numpy(absmax).cuda()
     plan = binding.LoraLinearPlan(p.T, p.d_in, p.d_out, p.r)
@@ -73,12 +74,17 @@ def run_nf4_layer(p, t, codes, absmax, use_scratch=False):
     for name, shape, dt in (("Y", (p.T, p.d_out), torch.bfloat16), ("dX", (p.T, p.d_in), torch.bfloat16),
                             ("dA", (p.r, p.d_in), torch.float32), ("dB", (p.d_out, p.r), torch.float32)):
         bufs[name], out[name] = guarded(shape, dt)
-    sbuf, scratch = guarded((p.d_out, p.d_in), torch.bfloat16) if use_scratch else (None, None)
+    if band_tiles:
+        lo, full = plan.nf4_scratch_bytes()
+        assert full == 2 * p.d_out * p.d_in and 0 < lo <= max(full, lo)
+        sbuf, scratch = guarded((band_tiles * lo // 2,), torch.bfloat16)
+    else:
+        sbuf, scratch = guarded((p.d_out, p.d_in), torch.bfloat16) if use_scratch else (None, None)
     plan.fwd_nf4(d["X"], cd, ad, d["A"], d["B"], p.scale, out["Y"], w_scratch=scratch)
-    if use_scratch:
+    if scratch is not None:
         scratch.fill_(float("nan"))                     # backward must rebuild the weight itself
     plan.bwd_nf4(d["dY"], d["X"], cd, ad, d["A"], d["B"], p.scale, out["dX"], out["dA"], out["dB"], w_scratch=scratch)
-    if use_scratch:
+    if scratch is not None:
         assert guards_intact(sbuf, scratch.numel()), "w_scratch: write outside the buffer"
     code, msg = plan.device_status()
     assert code == 0, msg
@@ -114,6 +120,67 @@ def test_nf4_layer_elementwise(T, d_in, d_out, r, scale, use_scratch):
             "dA": oracle.rel_err(host64(out["dA"]), dA), "dB": oracle.rel_err(host64(out["dB"]), dB)}
     assert errs["Y"] <= TOL_BF16 and errs["dX"] <= TOL_BF16, errs
     assert errs["dA"] <= TOL_F32 and errs["dB"] <= TOL_F32, errs
+
+
+BANDED_SHAPES = [
+    # T, d_in, d_out, r, scale, n-tiles of scratch      (bands of output rows forward, of input columns backward)
+    (640, 768, 1160, 16, 2.0, 1),          # one n-tile per band: five forward bands with a ragged last one, three backward
+    (1000, 2048, 520, 64, 0.5, 1),
+    (2100, 512, 3080, 32, 2.0, 3),         # forward bands of several tiles, a short last band
+    (4500, 1024, 4096, 16, 2.0, 2),
+    (300, 1344, 1344, 16, 1.0, 2),         # 1344 is no multiple of the tile width: narrow last bands in both directions
+]
+
+
+@pytest.mark.parametrize("T,d_in,d_out,r,scale,tiles", BANDED_SHAPES)
+def test_nf4_banded_scratch_matches_whole_weight_form_bitwise(T, d_in, d_out, r, scale, tiles):
+    """A scratch buffer smaller than the weight: the weight is expanded and multiplied band by band.  Same tiles and order of
+    summation as with the whole weight in scratch, so the outputs must agree bit for bit; and both with the oracle."""
+    p, t = inputs.draw_custom(T, d_in, d_out, r, scale, seed=14)
+    codes, absmax = nf4.quantize(inputs.bf16_to_f64(t["W"]).astype(np.float32))
+    whole = run_nf4_layer(p, t, codes, absmax, use_scratch=True)
+    banded = run_nf4_layer(p, t, codes, absmax, band_tiles=tiles)
+    for name in ("Y", "dX", "dA", "dB"):
+        assert torch.equal(whole[name], banded[name]), name
+    f = {k: inputs.bf16_to_f64(t[k]) for k in ("X", "A", "B", "dY")}
+    Y = nf4.forward(f["X"], codes, absmax, f["A"], f["B"], p.scale)
+    dX, dA, dB = nf4.backward(f["dY"], f["X"], codes, absmax, f["A"], f["B"], p.scale)
+    assert oracle.rel_err(host64(banded["Y"]), Y) <= TOL_BF16 and oracle.rel_err(host64(banded["dX"]), dX) <= TOL_BF16
+    assert oracle.rel_err(host64(banded["dA"]), dA) <= TOL_F32 and oracle.rel_err(host64(banded["dB"]), dB) <= TOL_F32
+
+
+def test_nf4_banded_weight_only_is_tight():
+    """One-hot X / dY rows through the banded form: every band lands in its own columns of Y and dX."""
+    T, d_in, d_out, r = 512, 768, 1024, 8
+    p, t = inputs.draw_custom(T, d_in, d_out, r, 1.0, seed=16)
+    codes, absmax = nf4.quantize(inputs.bf16_to_f64(t["W"]).astype(np.float32))
+    what = nf4.dequantize(codes, absmax)
+    bits = lambda x: x.contiguous().view(torch.int16).numpy().view(np.uint16)
+    t2 = dict(t)
+    # forward reads weight columns through one-hot X rows (T = 512 < d_in: the first 512 input features); backward weight
+    # rows through one-hot dY rows (the first 512 output features)
+    t2["X"] = bits(torch.eye(T, d_in, dtype=torch.bfloat16))
+    t2["dY"] = bits(torch.eye(T, d_out, dtype=torch.bfloat16))
+    t2["A"], t2["B"] = np.zeros_like(t["A"]), np.zeros_like(t["B"])
+    out = run_nf4_layer(p, t2, codes, absmax, band_tiles=1)
+    assert np.array_equal(host64(out["Y"]), what[:, :T].T)     # Y[t, :] = w_hat[:, t]
+    assert np.array_equal(host64(out["dX"]), what[:T, :])      # dX[t, :] = w_hat[t, :]
+
+
+def test_nf4_banded_rejects_what_it_cannot_serve():
+    plan = binding.LoraLinearPlan(1000, 512, 1024, 16)
+    lib = binding.load()
+    lo, full = plan.nf4_scratch_bytes()
+    cfg = plan.config()                                          # one n-tile of weight rows (forward) or columns (backward)
+    assert lo == 2 * max(cfg["fwd_block_n"] * 512, cfg["dx_block_n"] * 1024) and full == 2 * 1024 * 512
+    assert lib.lora_plan_set_nf4_scratch_bytes(plan._h, lo - 16) == binding.LORA_ERR_WORKSPACE
+    assert lib.lora_plan_set_nf4_scratch_bytes(plan._h, lo) == binding.LORA_OK
+    assert lib.lora_plan_set_nf4_scratch_bytes(plan._h, 0) == binding.LORA_OK
+    plan.close()
+    small = binding.LoraLinearPlan(64, 128, 512, 8)              # T <= 128: single-CTA plan, whole-weight scratch only
+    assert lib.lora_plan_set_nf4_scratch_bytes(small._h, 2 * 256 * 128) == binding.LORA_ERR_UNSUPPORTED_SHAPE
+    assert lib.lora_plan_set_nf4_scratch_bytes(small._h, 2 * 512 * 128) == binding.LORA_OK
+    small.close()
 
 
 def test_nf4_scratch_form_covers_small_batches():
