@@ -33,6 +33,7 @@ import numpy as np
 import torch
 
 L2_BYTES = 126 * 1024 * 1024
+E2E_STREAMS = int(os.environ.get("LORA_BENCH_E2E_STREAMS", "8"))      # streams the projections of one end-to-end step rotate over (3: 136 ms, 4: 122 ms, 7: 116 ms per layer step)
 NF4_BAND_BYTES = 16 * 1024 * 1024      # scratch buffer of the banded Q+LoRA variant (the largest weight of the layer is 112 MiB)
 METRIC = "lora_linear_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
@@ -659,27 +660,33 @@ def run_ours(args):
                 pl.ensure_workspace()
             outs = [{k: torch.empty_like(d0[k], device="cpu").pin_memory() for k in ("Y", "dX", "dA", "dB")} for _, d0 in sets0]
             stg = [torch.empty(lp[j].step_host_staging_bytes(), dtype=torch.uint8, device=device) for j in range(len(protos))]
-            lanes.append({"plans": lp, "out": outs, "staging": stg, "stream": torch.cuda.Stream(device=device)})
+            # a lane with several projections (each with its own plan, staging and host buffers) runs them on E2E_STREAMS
+            # streams in turn, so that one projection's copy-out overlaps the next ones' copy-in within the step as well
+            n_streams = min(E2E_STREAMS, len(protos))
+            lanes.append({"plans": lp, "out": outs, "staging": stg,
+                          "streams": [torch.cuda.Stream(device=device) for _ in range(n_streams)]})
 
         def step_host(k):
             ln = lanes[k % n_lanes]
             for j, (p, d0) in enumerate(sets0):
                 h, ho = h_in[j], ln["out"][j]
                 ln["plans"][j].step_host(h["X"], d0["W"], h["A"], h["B"], h["dY"], p.scale, ho["Y"], ho["dX"], ho["dA"], ho["dB"],
-                                         ln["staging"][j], stream=ln["stream"])
+                                         ln["staging"][j], stream=ln["streams"][j % len(ln["streams"])])
 
         def run_host(n):
             cur = torch.cuda.current_stream()
             start, done = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             start.record(cur)
             for ln in lanes:
-                ln["stream"].wait_event(start)
+                for st in ln["streams"]:
+                    st.wait_event(start)
             for k in range(n):
                 step_host(k)
             for ln in lanes:
-                ev = torch.cuda.Event()
-                ev.record(ln["stream"])
-                cur.wait_event(ev)
+                for st in ln["streams"]:
+                    ev = torch.cuda.Event()
+                    ev.record(st)
+                    cur.wait_event(ev)
             done.record(cur)
             torch.cuda.synchronize()
             return start.elapsed_time(done)
@@ -695,7 +702,8 @@ def run_ours(args):
                "ms_per_step": ms_e2e, "steps": n_e2e, "lanes": n_lanes,
                "pcie_gbs": {"h2d": h2d / ms_e2e / 1e6, "d2h": d2h / ms_e2e / 1e6},
                "note": "host X, A, B, dY in; Y, dX, dA, dB out (pinned); frozen W resident on the device; "
-                       f"{n_lanes} lane(s) of lora_linear_step_host alternate so that copies of neighbouring steps overlap"}
+                       f"{n_lanes} lane(s) of lora_linear_step_host alternate so that copies of neighbouring steps overlap"
+                       + (f"; the projections of a step rotate over {min(E2E_STREAMS, len(protos))} streams" if len(protos) > 1 else "")}
     plan_desc = plans[0].describe()
     wl.close()
 
