@@ -44,14 +44,14 @@ UNIT = "TFLOP/s"
 # streaming launches' at T = 8192) and are scaled by the tokens: GEMM traffic is per band of m-tiles and the number of bands
 # grows with T; a streaming launch's traffic is the two streamed matrices, proportional to T.
 NCU_TRAFFIC = {
-    "gemm_sha": "7ffd987e862cc4b4",
-    "gemm_bytes_per_launch": {"32768x14336x4096": 4345182208},       # 2 x (1717.8 + 454.8 MB) captured at T = 16384
-    "stream_sha": "f6480168ab5dc96b",
+    "gemm_sha": "528a6efb94fd7e1e",
+    "gemm_bytes_per_launch": {"32768x14336x4096": 3798919680},       # 2 x (1444.2 + 455.3 MB) captured at T = 16384
+    "stream_sha": "310b01e3e28131ab",
     "stream_bytes_per_launch": {                                      # 4 x the launches captured at T = 8192
-        "sides:32768x4096x4096": 552952832, "grads:32768x4096x4096": 554292224,
-        "sides:32768x4096x1024": 349594624, "grads:32768x4096x1024": 347867136,
-        "sides:32768x4096x14336": 1236064256, "grads:32768x4096x14336": 1223135232,
-        "sides:32768x14336x4096": 1240367104, "grads:32768x14336x4096": 1222888448}}
+        "sides:32768x4096x4096": 552556544, "grads:32768x4096x4096": 551930880,
+        "sides:32768x4096x1024": 346225664, "grads:32768x4096x1024": 347225088,
+        "sides:32768x4096x14336": 1235765248, "grads:32768x4096x14336": 1223817216,
+        "sides:32768x14336x4096": 1241160704, "grads:32768x14336x4096": 1224769536}}
 
 
 def peaks():
