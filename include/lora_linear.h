@@ -25,6 +25,10 @@
  *   - d_in and d_out must be multiples of 8; r a multiple of 8 with 8 <= r <= 64; T >= 0.
  *   - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work and return; they do not
  *     synchronise.  A plan must not be used from two host threads, or on two streams, at once.
+ *     The forward and backward calls (plain, saved-P, grouped, NF4, dense dW) therefore work under stream capture: a step
+ *     captured into a CUDA graph replays bit-identically (what a launch-bound batch of a few hundred tokens wants).
+ *     Not capturable: lora_last_device_status, lora_plan_last_gemm_clock and lora_grad_contract_noalloc_status, which
+ *     synchronise the stream and copy to the host.
  *   - The library never allocates device memory except one 256-byte status word block per plan;
  *     scratch is caller-provided (lora_plan_set_workspace): backward always needs it, forward needs it whenever the
  *     selector chose the K-extended form (cfg.fwd_ext; lora_plan_workspace_bytes reports fwd_bytes > 0 then).
