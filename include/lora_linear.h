@@ -270,9 +270,9 @@ int lora_dense_dw(lora_plan_t* plan, const void* dY, const void* X, void* dW, vo
  *     expansion and the GEMM that reads it.  Costs one expansion launch and one partly filled last wave per band.
  *   - w_scratch == NULL: nothing is materialised; packed codes and scales are staged by TMA and expanded inside the GEMM
  *     kernels, straight into the tensor-core operand tiles.  No extra memory, but the conversion is repeated for every
- *     256-token tile and competes with the tensor cores for shared-memory bandwidth (measured 2-2.5x slower at
- *     T = 4096..8192).  Needs a plan with T > 128, else LORA_ERR_UNSUPPORTED_SHAPE.
- * Both forms give bit-identical weights to the GEMMs.  The workspace must be registered (LORA_ERR_WORKSPACE
+ *     256-token tile and competes with the tensor cores for shared-memory bandwidth (measured 1.5-2x slower than the
+ *     scratch forms from T = 8192 on).  Needs a plan with T > 128, else LORA_ERR_UNSUPPORTED_SHAPE.
+ * All three forms give bit-identical weights to the GEMMs.  The workspace must be registered (LORA_ERR_WORKSPACE
  * otherwise; forward needs it in the NULL form and whenever the plan's forward uses it).  All pointers are device
  * pointers, 16-byte aligned. */
 /* Size of the buffer behind `w_scratch` in the two Q+LoRA calls of this plan.  lora_plan_nf4_scratch_bytes: `full_bytes` =
