@@ -410,6 +410,26 @@ def measure(wl: Workload, steps: int, warmup: int, pk, world: int, device, barri
             "gemm_sm_mhz_in_kernel": gemm_clock, "t_host": (t_host0, t_host1, t_host2), "n_warm": n_warm_total}
 
 
+def copy_behind_gemms(wl: Workload, nbytes: float, device, n: int = 6) -> float:
+    """GB/s of a plain device-to-device copy that moves `nbytes` (half read, half written), timed between two events right
+    after a whole step of the workload, n times.  Context for the HBM fractions only: the copy is torch's own kernel, and it
+    shows what a streaming launch can reach at the clocks the power-capped GEMMs leave behind (the measured copy peak in
+    MEASURED_PEAKS.json was taken on an otherwise idle part)."""
+    elems = int(nbytes // 4)                           # bf16: nbytes / 2 bytes each way
+    src = [torch.empty(elems, dtype=torch.bfloat16, device=device).normal_() for _ in range(2)]
+    dst = torch.empty(elems, dtype=torch.bfloat16, device=device)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+    for k in range(n):
+        wl.step(k)
+        ev[k][0].record()
+        dst.copy_(src[k % 2])
+        ev[k][1].record()
+    torch.cuda.synchronize()
+    ms = statistics.mean(a.elapsed_time(b) for a, b in ev)
+    del src, dst
+    return 4.0 * elems / ms / 1e6
+
+
 def kernel_b2b(wl: Workload, pk, n: int = 16):
     """Every skinny stage of every projection launched n times back to back (inputs rotate between the sets, so the
     stream never sits in L2): the launch's own steady-state duration, with the programmatic overlap of consecutive
@@ -575,6 +595,12 @@ def run_ours(args):
                         "back_to_back": b2b.get(wp.name, {}).get(wname),
                         "traffic": (NCU_TRAFFIC["stream_bytes_per_launch"].get(skey)
                                     if NCU_TRAFFIC["stream_sha"] == source_sha("adapter_grad") else None)}
+        if not args.quick:
+            cg = copy_behind_gemms(wl, we["bytes"], device)
+            roofline_hbm["plain_copy_same_bytes_behind_gemms"] = {
+                "gbs": cg, "frac_of_hbm_peak": cg / pk["hbm_gbs"],
+                "note": "a device-to-device copy (torch's kernel, measurement only) moving the stage's byte count, between two "
+                        "events right after a whole step: the copy rate at the clocks the power-capped GEMMs leave behind"}
 
     variants = {}
     n_var = max(3, min(args.steps, 20))
