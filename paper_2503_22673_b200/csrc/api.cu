@@ -167,7 +167,10 @@ int select_config(const lora_shape_t* s, int num_sms, lora_kernel_config_t* c, c
   c->dx_block_n = pick_block_n(T, s->d_in, c->r_pad, num_sms);
   c->stages = 4;
   c->dx_stages = 4;
-  c->group_m = 8;
+  // m-tiles per rasterisation band.  A weight that fits L2 several times over stays there whatever the order, so short bands
+  // (activations fetched once, nothing else re-read) bring DRAM traffic down to the operands themselves: 8192 x 4096 x 4096,
+  // forward GEMM 221 -> 172 MB per launch at the same 172 us.  A weight of L2's size needs tall bands to be reused at all.
+  c->group_m = (2 * s->d_out * s->d_in <= (48ll << 20)) ? 2 : 8;
   if (const char* f = std::getenv("LORA_FORCE_GROUP_M")) {   // tuning knob: m-tiles per rasterisation band
     const int v = std::atoi(f);
     if (v >= 1 && v <= 64) c->group_m = v;
