@@ -84,6 +84,15 @@ def test_selector_invariants(shape):
         assert st * (32768 + side) + 4 * c["r_pad"] * 128 + 2048 <= 232448
 
 
+def test_selector_band_height_follows_the_weight_size():
+    """Rasterisation bands: 2 m-tiles while the weight (at most 48 MiB) stays in L2 whatever the order, 8 for weights of
+    L2's own size, which are only reused inside a tall band."""
+    assert binding.select_config(8192, 4096, 4096, 16, 148)["group_m"] == 2          # 32 MiB
+    assert binding.select_config(32768, 4096, 1024, 16, 148)["group_m"] == 2         # 8 MiB
+    assert binding.select_config(16384, 4096, 14336, 16, 148)["group_m"] == 8        # 112 MiB
+    assert binding.select_config(16384, 14336, 4096, 64, 148)["group_m"] == 8
+
+
 def test_selector_grad_grids_of_the_benchmark_shapes():
     """The dA + dB launch of the merged backward: 128-feature blocks of X and dY side by side, each block's token chunks
     one small cluster, so that the grid is as close to the SM count as whole clusters allow."""
